@@ -1,0 +1,179 @@
+/*
+ * libmdbf — Multi-Envelope Double Binary Factorization (MDBF) linear forward
+ * for NVIDIA B200 (sm_100a).  C ABI.
+ *
+ * The layer is the paper's format (Eq. me-dbf-basis), in the column convention
+ *
+ *     y = W_hat x,   W_hat = (S_A (.) U_A V_A^T) (S_B (.) U_B V_B^T)
+ *
+ *     S_A  d_out x k   +-1      (paper: S_a,  N x R)
+ *     S_B  k x d_in    +-1      (paper: S_b^T, R x M)
+ *     U_A  d_out x l,  V_A  k x l      (paper: A, Q)
+ *     U_B  k x l,      V_B  d_in x l   (paper: G, B)
+ *
+ * evaluated in the interleaved order of Eq. DBF-inference-form generalised by
+ * Eq. me-dbf-expand: scale, sign contraction with S_B, scale, sign contraction
+ * with S_A, scale — each stage being  sum_r diag(u_r) S diag(v_r)  with the
+ * sign matrix shared by the l envelope modes.
+ *
+ * Conventions
+ *   - All matrices are dense row-major.
+ *   - Activations are token-contiguous: x[tau * d_in + i], y[tau * d_out + n]
+ *     (a row-major [T, d] array).
+ *   - Canonical sign packing: 32 signs per uint32 along the reduction
+ *     dimension (k for S_A, d_in for S_B); column c of a row lives in word
+ *     c / 32 at bit c % 32 (bit 0 = least significant); bit set <=> sign -1;
+ *     padding bits of the last word are 0.  The paper only says the sign
+ *     matrices are stored bit-packed (paragraph "Inference"); this layout is
+ *     the library's.
+ *   - Every function returns mdbf_status_t (0 = OK, negative = error), never
+ *     throws, aborts or exits.  mdbf_last_error() returns a thread-local,
+ *     NUL-terminated description of the last failure on the calling thread.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).
+ *   - There is no CPU fallback: every entry point that computes needs a CUDA
+ *     device of compute capability 10.x and fails with MDBF_ERR_ARCH otherwise
+ *     (the host-side sign packer, on_device = 0, is the one exception).
+ */
+#ifndef MDBF_H
+#define MDBF_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t mdbf_status_t;
+enum {
+    MDBF_OK = 0,
+    MDBF_ERR_INVALID_ARG = -1, /* NULL pointer, bad handle, bad selector          */
+    MDBF_ERR_SHAPE = -2,       /* non-positive size, T < 1, T > max_T, l > 64     */
+    MDBF_ERR_DTYPE = -3,       /* unsupported element type                        */
+    MDBF_ERR_ALLOC = -4,       /* device or host allocation failed                */
+    MDBF_ERR_CUDA = -5,        /* a CUDA runtime call failed (see last_error)     */
+    MDBF_ERR_ARCH = -6,        /* no CUDA device, or not compute capability 10.x  */
+    MDBF_ERR_TIMEOUT = -7,     /* a bounded device-side wait expired              */
+    MDBF_ERR_VALUE = -8        /* a sign that is neither +1 nor -1                */
+};
+
+typedef enum { MDBF_F32 = 0, MDBF_F16 = 1, MDBF_BF16 = 2 } mdbf_dtype_t;
+
+/* Kernel selector for mdbf_set_kernel. */
+typedef enum {
+    MDBF_KERNEL_AUTO = 0,   /* choose by (l, T, dtypes)                                         */
+    MDBF_KERNEL_ALU = 1,    /* fp32 CUDA-core path, sign applied by XOR of the IEEE sign bit      */
+    MDBF_KERNEL_DECODE = 2, /* small-T path: register bit->bf16 expansion + warp-level MMA        */
+    MDBF_KERNEL_PREFILL = 3 /* large-T path: tcgen05 MMA with TMEM accumulators                   */
+} mdbf_kernel_t;
+
+typedef struct {
+    int32_t d_out;     /* rows of W_hat (paper: N)                         */
+    int32_t d_in;      /* columns of W_hat (paper: M)                      */
+    int32_t k;         /* inner rank (paper: R)                            */
+    int32_t l;         /* envelope rank, 1 <= l <= 64                      */
+    int32_t env_dtype; /* mdbf_dtype_t the envelope factors are stored in  */
+    int32_t max_T;     /* largest token count a forward call may pass      */
+} mdbf_desc_t;
+
+typedef struct mdbf_handle_s *mdbf_handle_t;
+
+/* ---------------------------------------------------------------- packing
+ * Canonical sign packing (layout above; storage statement: paragraph
+ * "Inference", effective bits-per-weight).
+ *   s     rows x cols int8, every entry +1 or -1
+ *   out   rows x ceil(cols/32) uint32
+ * on_device = 0: both pointers are host memory, the work is done on the host
+ * (no GPU needed); a value other than +-1 returns MDBF_ERR_VALUE.
+ * on_device = 1: both are device memory, the kernel runs asynchronously on
+ * `stream`; values other than -1 are treated as +1.
+ * Caller owns both buffers. */
+mdbf_status_t mdbf_pack_signs(const int8_t *s, int64_t rows, int64_t cols, uint32_t *out,
+                              int on_device, void *stream);
+
+/* Inverse of mdbf_pack_signs: p rows x ceil(cols/32) uint32 -> out rows x cols int8. */
+mdbf_status_t mdbf_unpack_signs(const uint32_t *p, int64_t rows, int64_t cols, int8_t *out,
+                                int on_device, void *stream);
+
+/* ------------------------------------------------------------------ layer
+ * Build a layer (Eq. me-dbf-basis).  Copies everything: the caller keeps
+ * ownership of all inputs and may free them on return.
+ *   S_A d_out x k, S_B k x d_in   int8 +-1
+ *   U_A d_out x l, V_A k x l, U_B k x l, V_B d_in x l   float32; rounded
+ *   (round-to-nearest-even) to desc->env_dtype — the rounded values are the
+ *   layer and can be read back with mdbf_get_envelope.
+ * inputs_on_device: 0 = all seven pointers are host memory, 1 = all device.
+ * The handle owns device copies of the canonical words, of a kernel-private
+ * tiled copy of them, of the envelopes, and scratch for the k x T
+ * intermediate sized for max_T: one forward per handle may be in flight at a
+ * time.  Synchronises `stream` before returning.
+ * Errors: INVALID_ARG (NULL), SHAPE, DTYPE, VALUE (host inputs only), ALLOC,
+ * CUDA, ARCH. */
+mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t *S_B,
+                        const float *U_A, const float *V_A, const float *U_B, const float *V_B,
+                        int inputs_on_device, void *stream, mdbf_handle_t *out);
+
+/* Copy the canonical packed words of S_A (which = 0, d_out x ceil(k/32)) or
+ * S_B (which = 1, k x ceil(d_in/32)) to `out` (host if out_on_device = 0). */
+mdbf_status_t mdbf_get_packed(mdbf_handle_t h, int which, uint32_t *out, int out_on_device,
+                              void *stream);
+
+/* Stored (rounded) envelope factor as float32: which = 0 U_A, 1 V_A, 2 U_B, 3 V_B. */
+mdbf_status_t mdbf_get_envelope(mdbf_handle_t h, int which, float *out, int out_on_device,
+                                void *stream);
+
+/* Read the layer's descriptor back. */
+mdbf_status_t mdbf_get_desc(mdbf_handle_t h, mdbf_desc_t *out);
+
+/* Force a kernel for later forwards on this handle (tests, benchmarks). */
+mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel /* mdbf_kernel_t */);
+
+/* ---------------------------------------------------------------- forward
+ * y = W_hat x (Eq. DBF-inference-form with Eq. me-dbf-expand; steps: scale by
+ * V_B, sign contraction with S_B, contract modes with U_B, scale by V_A, sign
+ * contraction with S_A, contract modes with U_A).
+ *   x  device, T x d_in  of act_dtype (token-contiguous), read only
+ *   y  device, T x d_out of act_dtype, written (round-to-nearest-even)
+ *   act_dtype  MDBF_BF16 or MDBF_F32 (MDBF_F16 is accepted by the ALU path)
+ * Accumulation is fp32.  Asynchronous on `stream`; allocates nothing, does not
+ * synchronise.  x and y must not alias.
+ * Errors: INVALID_ARG, SHAPE (T < 1 or T > max_T), DTYPE, CUDA. */
+mdbf_status_t mdbf_linear_forward(mdbf_handle_t h, const void *x, void *y, int32_t T,
+                                  int32_t act_dtype, void *stream);
+
+/* Same computation with HOST buffers: copies x to a handle-owned device
+ * staging buffer, runs the forward, copies y back, all on `stream`, and
+ * synchronises the stream before returning.  x_host / y_host should be pinned
+ * for full copy bandwidth. */
+mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T,
+                                       int32_t act_dtype, void *stream);
+
+/* The k x T intermediate z of the last forward on this handle (after the
+ * stage with S_B), as float32 token-contiguous T x k, for tests that localise
+ * a disagreement to one stage.  Synchronises `stream`. */
+mdbf_status_t mdbf_get_intermediate(mdbf_handle_t h, float *z, int32_t T, int out_on_device,
+                                    void *stream);
+
+/* Dense W_hat (Eq. me-dbf-basis), fp32, d_out x d_in row-major, device memory,
+ * asynchronous on `stream`.  Check path, not a hot path. */
+mdbf_status_t mdbf_reconstruct(mdbf_handle_t h, float *W, void *stream);
+
+/* Device-side status word of the handle (0, or MDBF_ERR_TIMEOUT when a bounded
+ * wait inside a kernel expired; the kernel then returns without completing y).
+ * Synchronises the device.  Reading clears the word. */
+mdbf_status_t mdbf_poll_status(mdbf_handle_t h, int32_t *device_status);
+
+/* Number of kernels the last forward on this handle launched. */
+mdbf_status_t mdbf_last_launch_count(mdbf_handle_t h, int32_t *count);
+
+/* Free everything the handle owns.  Synchronises the device. */
+mdbf_status_t mdbf_destroy(mdbf_handle_t h);
+
+const char *mdbf_last_error(void);
+
+/* Library version string. */
+const char *mdbf_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MDBF_H */

@@ -1,8 +1,8 @@
 """B200-native MDBF quantized linear forward (libmdbf) — Python binding.
 
-`paper_2512_24545_b200.libmdbf` wraps the C-ABI shared library one-to-one;
+`paper_2512_24545_b200.mdbf` wraps the C-ABI shared library one-to-one;
 `paper_2512_24545_b200.inputs` holds the seeded synthetic input generators.
 Importing the package does not load the CUDA library; the first call into
-`libmdbf` does, and fails loudly when the library has not been built.
+`mdbf` does, and fails loudly when the library has not been built.
 """
-__all__ = ["inputs", "libmdbf"]
+__all__ = ["inputs", "mdbf"]

@@ -1,0 +1,111 @@
+// Internal declarations shared by the libmdbf translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "mdbf.h"
+
+namespace mdbf {
+
+constexpr uint32_t kHandleMagic = 0x4D444246u;  // "MDBF"
+constexpr int kMaxL = 64;
+constexpr int kMaxKSplit = 8;          // stage-B partial sums kept per handle
+constexpr int kDecodeMaxT = 4;         // tokens per call the small-T kernel takes
+
+// Kernel-private tiled copy of a packed sign matrix (see pack.cu):
+// tiles of 32 rows x 128 columns, 512 bytes each, tile (rt, kt) at
+// ((rt * ktiles) + kt) * 128 words; inside a tile lane L = 4*g + q of a warp
+// owns the uint4 { w(g, q), w(g+8, q), w(g+16, q), w(g+24, q) } where
+// w(r, q) is canonical word q of row r of the tile.
+struct TiledSigns {
+    const uint32_t *words;  // device
+    int rtiles;             // ceil(rows / 32)
+    int ktiles;             // ceil(cols / 128)
+};
+
+struct Layer {
+    mdbf_desc_t d;
+    int device;
+    // canonical words
+    uint32_t *wA, *wB;
+    int wordsA, wordsB;           // words per row
+    // tiled words
+    uint32_t *tA, *tB;
+    int rtA, ktA, rtB, ktB;
+    // envelopes in env_dtype, row-major [rows][l]
+    void *UA, *VA, *UB, *VB;
+    // kernel-private bf16 copies of V_A / V_B in MMA B-fragment order (see forward_decode.cu)
+    uint2 *vfA, *vfB;
+    int NT;                       // 8-column mode tiles in the fragment copies: 1, 2, 4 or 8
+    // scratch
+    float *z;                     // [kMaxKSplit][zT][k] stage-B partial sums of the small-T kernel
+    size_t zstride;               // zT * k
+    float *zsum;                  // [max_T][k] summed intermediate (ALU path, inspection)
+    void *xstage, *ystage;        // device staging for the host-buffer entry point
+    int32_t *status;              // device status word
+    int last_ksplit;              // how many partials the last forward wrote (0 = zsum valid)
+};
+
+// thread-local error string
+void set_error(const char *fmt, ...);
+mdbf_status_t cuda_fail(cudaError_t e, const char *what);
+
+#define MDBF_CUDA(call)                                                        \
+    do {                                                                       \
+        cudaError_t e__ = (call);                                              \
+        if (e__ != cudaSuccess) return ::mdbf::cuda_fail(e__, #call);          \
+    } while (0)
+
+// --- element helpers --------------------------------------------------------
+__device__ __forceinline__ float env_load(const void *p, size_t idx, int dtype) {
+    if (dtype == MDBF_F16) return __half2float(reinterpret_cast<const __half *>(p)[idx]);
+    if (dtype == MDBF_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(p)[idx]);
+    return reinterpret_cast<const float *>(p)[idx];
+}
+
+template <typename T> __device__ __forceinline__ float act_load(const T *p, size_t i);
+template <> __device__ __forceinline__ float act_load<float>(const float *p, size_t i) { return p[i]; }
+template <> __device__ __forceinline__ float act_load<__half>(const __half *p, size_t i) { return __half2float(p[i]); }
+template <> __device__ __forceinline__ float act_load<__nv_bfloat16>(const __nv_bfloat16 *p, size_t i) { return __bfloat162float(p[i]); }
+
+template <typename T> __device__ __forceinline__ void act_store(T *p, size_t i, float v);
+template <> __device__ __forceinline__ void act_store<float>(float *p, size_t i, float v) { p[i] = v; }
+template <> __device__ __forceinline__ void act_store<__half>(__half *p, size_t i, float v) { p[i] = __float2half_rn(v); }
+template <> __device__ __forceinline__ void act_store<__nv_bfloat16>(__nv_bfloat16 *p, size_t i, float v) { p[i] = __float2bfloat16_rn(v); }
+
+__host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline size_t dtype_size(int dt) { return dt == MDBF_F32 ? 4 : 2; }
+
+// --- launchers (each returns after enqueueing on `st`) ------------------------
+mdbf_status_t launch_pack(const int8_t *s, int64_t rows, int64_t cols, uint32_t *out, cudaStream_t st);
+mdbf_status_t launch_unpack(const uint32_t *p, int64_t rows, int64_t cols, int8_t *out, cudaStream_t st);
+mdbf_status_t launch_tile(const uint32_t *canon, int rows, int words, uint32_t *tiled, int rtiles,
+                          int ktiles, cudaStream_t st);
+mdbf_status_t launch_env_round(const float *src, void *dst, size_t n, int dtype, cudaStream_t st);
+mdbf_status_t launch_env_read(const void *src, float *dst, size_t n, int dtype, cudaStream_t st);
+mdbf_status_t launch_vfrag(const void *V, int cols, int l, int env_dtype, uint2 *out, int ktiles, int NT,
+                           cudaStream_t st);
+mdbf_status_t launch_reconstruct(const Layer &L, float *W, cudaStream_t st);
+mdbf_status_t launch_forward_alu(Layer &L, const void *x, void *y, int T, int act_dtype,
+                                 cudaStream_t st, int *launches);
+mdbf_status_t launch_forward_decode(Layer &L, const void *x, void *y, int T, cudaStream_t st,
+                                    int *launches);
+mdbf_status_t launch_forward_prefill(Layer &L, const void *x, void *y, int T, cudaStream_t st,
+                                     int *launches);
+mdbf_status_t launch_zsum(Layer &L, int T, cudaStream_t st);
+
+// host-side canonical packer (pack.cu)
+mdbf_status_t host_pack(const int8_t *s, int64_t rows, int64_t cols, uint32_t *out);
+mdbf_status_t host_unpack(const uint32_t *p, int64_t rows, int64_t cols, int8_t *out);
+
+}  // namespace mdbf
+
+struct mdbf_handle_s {
+    uint32_t magic;
+    int32_t kernel;
+    int32_t last_launches;
+    mdbf::Layer L;
+};

@@ -1,0 +1,387 @@
+// C-ABI entry points of libmdbf: argument checking, handle lifetime, dispatch.
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+namespace mdbf {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+mdbf_status_t cuda_fail(cudaError_t e, const char *what) {
+    set_error("CUDA error %d (%s) in %s", (int)e, cudaGetErrorString(e), what);
+    if (e == cudaErrorMemoryAllocation) return MDBF_ERR_ALLOC;
+    return MDBF_ERR_CUDA;
+}
+
+// The product has no CPU fallback: anything that computes needs an sm_100 device.
+static mdbf_status_t require_device(int *dev_out) {
+    int n = 0;
+    cudaError_t e = cudaGetDeviceCount(&n);
+    if (e != cudaSuccess || n == 0) {
+        cudaGetLastError();
+        set_error("libmdbf needs a CUDA device of compute capability 10.x; none is visible (%s)",
+                  e == cudaSuccess ? "device count 0" : cudaGetErrorString(e));
+        return MDBF_ERR_ARCH;
+    }
+    int dev = 0;
+    MDBF_CUDA(cudaGetDevice(&dev));
+    int major = 0;
+    MDBF_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    if (major != 10) {
+        set_error("libmdbf is built for sm_100a only; device %d has compute capability major %d", dev, major);
+        return MDBF_ERR_ARCH;
+    }
+    if (dev_out) *dev_out = dev;
+    return MDBF_OK;
+}
+
+static bool valid_dtype(int dt) { return dt == MDBF_F32 || dt == MDBF_F16 || dt == MDBF_BF16; }
+
+static mdbf_status_t check_handle(mdbf_handle_t h, const char *fn) {
+    if (h == nullptr || h->magic != kHandleMagic) {
+        set_error("%s: invalid handle", fn);
+        return MDBF_ERR_INVALID_ARG;
+    }
+    return MDBF_OK;
+}
+
+static void free_layer(Layer &L) {
+    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.z, L.zsum, L.xstage, L.ystage, L.status};
+    for (void *p : ptrs)
+        if (p) cudaFree(p);
+}
+
+// number of tokens the small-T kernel's partial-sum scratch is sized for
+static int decode_scratch_T(const mdbf_desc_t &d) { return d.max_T < kDecodeMaxT ? d.max_T : kDecodeMaxT; }
+
+}  // namespace mdbf
+
+using namespace mdbf;
+
+extern "C" {
+
+const char *mdbf_last_error(void) { return g_err; }
+const char *mdbf_version(void) { return "libmdbf 0.1 (sm_100a)"; }
+
+mdbf_status_t mdbf_pack_signs(const int8_t *s, int64_t rows, int64_t cols, uint32_t *out, int on_device,
+                              void *stream) {
+    if (!s || !out) { set_error("mdbf_pack_signs: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    if (rows < 0 || cols < 0) { set_error("mdbf_pack_signs: negative size"); return MDBF_ERR_SHAPE; }
+    if (rows == 0 || cols == 0) return MDBF_OK;
+    if (!on_device) return host_pack(s, rows, cols, out);
+    mdbf_status_t rc = require_device(nullptr);
+    if (rc) return rc;
+    return launch_pack(s, rows, cols, out, (cudaStream_t)stream);
+}
+
+mdbf_status_t mdbf_unpack_signs(const uint32_t *p, int64_t rows, int64_t cols, int8_t *out, int on_device,
+                                void *stream) {
+    if (!p || !out) { set_error("mdbf_unpack_signs: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    if (rows < 0 || cols < 0) { set_error("mdbf_unpack_signs: negative size"); return MDBF_ERR_SHAPE; }
+    if (rows == 0 || cols == 0) return MDBF_OK;
+    if (!on_device) return host_unpack(p, rows, cols, out);
+    mdbf_status_t rc = require_device(nullptr);
+    if (rc) return rc;
+    return launch_unpack(p, rows, cols, out, (cudaStream_t)stream);
+}
+
+mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t *S_B, const float *U_A,
+                        const float *V_A, const float *U_B, const float *V_B, int inputs_on_device,
+                        void *stream, mdbf_handle_t *out) {
+    if (!desc || !S_A || !S_B || !U_A || !V_A || !U_B || !V_B || !out) {
+        set_error("mdbf_pack: NULL pointer");
+        return MDBF_ERR_INVALID_ARG;
+    }
+    *out = nullptr;
+    const mdbf_desc_t d = *desc;
+    if (d.d_out < 1 || d.d_in < 1 || d.k < 1 || d.l < 1 || d.l > kMaxL || d.max_T < 1) {
+        set_error("mdbf_pack: bad shape d_out=%d d_in=%d k=%d l=%d max_T=%d (need all >= 1, l <= %d)",
+                  d.d_out, d.d_in, d.k, d.l, d.max_T, kMaxL);
+        return MDBF_ERR_SHAPE;
+    }
+    if (!valid_dtype(d.env_dtype)) { set_error("mdbf_pack: bad env_dtype %d", d.env_dtype); return MDBF_ERR_DTYPE; }
+    int dev = 0;
+    mdbf_status_t rc = require_device(&dev);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    if (!inputs_on_device) {   // validate host signs before touching the device
+        const int8_t *mats[2] = {S_A, S_B};
+        const size_t cnt[2] = {(size_t)d.d_out * d.k, (size_t)d.k * d.d_in};
+        for (int m = 0; m < 2; ++m)
+            for (size_t e = 0; e < cnt[m]; ++e)
+                if (mats[m][e] != 1 && mats[m][e] != -1) {
+                    set_error("mdbf_pack: S_%c entry %zu is %d, expected +1 or -1", m ? 'B' : 'A', e, (int)mats[m][e]);
+                    return MDBF_ERR_VALUE;
+                }
+    }
+
+    mdbf_handle_s *h = new (std::nothrow) mdbf_handle_s();
+    if (!h) { set_error("mdbf_pack: host allocation failed"); return MDBF_ERR_ALLOC; }
+    memset(h, 0, sizeof(*h));
+    Layer &L = h->L;
+    L.d = d;
+    L.device = dev;
+    L.wordsA = ceil_div(d.k, 32);
+    L.wordsB = ceil_div(d.d_in, 32);
+    L.rtA = ceil_div(d.d_out, 32); L.ktA = ceil_div(d.k, 128);
+    L.rtB = ceil_div(d.k, 32);     L.ktB = ceil_div(d.d_in, 128);
+    const size_t es = dtype_size(d.env_dtype);
+    const size_t nUA = (size_t)d.d_out * d.l, nVA = (size_t)d.k * d.l, nUB = nVA, nVB = (size_t)d.d_in * d.l;
+    const size_t nSA = (size_t)d.d_out * d.k, nSB = (size_t)d.k * d.d_in;
+
+    std::vector<void *> temps;
+    auto fail = [&](mdbf_status_t code) {
+        for (void *p : temps) cudaFree(p);
+        free_layer(L);
+        delete h;
+        return code;
+    };
+#define PACK_CUDA(call)                                                  \
+    do {                                                                 \
+        cudaError_t e__ = (call);                                        \
+        if (e__ != cudaSuccess) return fail(cuda_fail(e__, #call));      \
+    } while (0)
+#define PACK_RC(call)                                \
+    do {                                             \
+        mdbf_status_t r__ = (call);                  \
+        if (r__ != MDBF_OK) return fail(r__);        \
+    } while (0)
+
+    PACK_CUDA(cudaMalloc(&L.wA, (size_t)d.d_out * L.wordsA * 4));
+    PACK_CUDA(cudaMalloc(&L.wB, (size_t)d.k * L.wordsB * 4));
+    PACK_CUDA(cudaMalloc(&L.tA, (size_t)L.rtA * L.ktA * 512));
+    PACK_CUDA(cudaMalloc(&L.tB, (size_t)L.rtB * L.ktB * 512));
+    PACK_CUDA(cudaMalloc(&L.UA, nUA * es));
+    PACK_CUDA(cudaMalloc(&L.VA, nVA * es));
+    PACK_CUDA(cudaMalloc(&L.UB, nUB * es));
+    PACK_CUDA(cudaMalloc(&L.VB, nVB * es));
+    L.NT = d.l <= 8 ? 1 : d.l <= 16 ? 2 : d.l <= 32 ? 4 : 8;
+    PACK_CUDA(cudaMalloc(&L.vfA, (size_t)L.ktA * 8 * L.NT * 256));
+    PACK_CUDA(cudaMalloc(&L.vfB, (size_t)L.ktB * 8 * L.NT * 256));
+    L.zstride = (size_t)decode_scratch_T(d) * d.k;
+    PACK_CUDA(cudaMalloc(&L.z, (size_t)kMaxKSplit * L.zstride * sizeof(float)));
+    PACK_CUDA(cudaMalloc(&L.zsum, (size_t)d.max_T * d.k * sizeof(float)));
+    PACK_CUDA(cudaMalloc(&L.xstage, (size_t)d.max_T * d.d_in * 4));
+    PACK_CUDA(cudaMalloc(&L.ystage, (size_t)d.max_T * d.d_out * 4));
+    PACK_CUDA(cudaMalloc(&L.status, sizeof(int32_t)));
+    PACK_CUDA(cudaMemsetAsync(L.status, 0, sizeof(int32_t), st));
+    PACK_CUDA(cudaMemsetAsync(L.zsum, 0, (size_t)d.max_T * d.k * sizeof(float), st));
+
+    // bring inputs to the device if needed
+    const void *src[6] = {S_A, S_B, U_A, V_A, U_B, V_B};
+    const size_t bytes[6] = {nSA, nSB, nUA * 4, nVA * 4, nUB * 4, nVB * 4};
+    const void *dsrc[6];
+    for (int i = 0; i < 6; ++i) {
+        if (inputs_on_device) { dsrc[i] = src[i]; continue; }
+        void *tmp = nullptr;
+        PACK_CUDA(cudaMalloc(&tmp, bytes[i]));
+        temps.push_back(tmp);
+        PACK_CUDA(cudaMemcpyAsync(tmp, src[i], bytes[i], cudaMemcpyHostToDevice, st));
+        dsrc[i] = tmp;
+    }
+    PACK_RC(launch_pack((const int8_t *)dsrc[0], d.d_out, d.k, L.wA, st));
+    PACK_RC(launch_pack((const int8_t *)dsrc[1], d.k, d.d_in, L.wB, st));
+    PACK_RC(launch_tile(L.wA, d.d_out, L.wordsA, L.tA, L.rtA, L.ktA, st));
+    PACK_RC(launch_tile(L.wB, d.k, L.wordsB, L.tB, L.rtB, L.ktB, st));
+    PACK_RC(launch_env_round((const float *)dsrc[2], L.UA, nUA, d.env_dtype, st));
+    PACK_RC(launch_env_round((const float *)dsrc[3], L.VA, nVA, d.env_dtype, st));
+    PACK_RC(launch_env_round((const float *)dsrc[4], L.UB, nUB, d.env_dtype, st));
+    PACK_RC(launch_env_round((const float *)dsrc[5], L.VB, nVB, d.env_dtype, st));
+    PACK_RC(launch_vfrag(L.VA, d.k, d.l, d.env_dtype, L.vfA, L.ktA, L.NT, st));
+    PACK_RC(launch_vfrag(L.VB, d.d_in, d.l, d.env_dtype, L.vfB, L.ktB, L.NT, st));
+    PACK_CUDA(cudaStreamSynchronize(st));
+    for (void *p : temps) cudaFree(p);
+    temps.clear();
+#undef PACK_CUDA
+#undef PACK_RC
+    h->magic = kHandleMagic;
+    h->kernel = MDBF_KERNEL_AUTO;
+    *out = h;
+    return MDBF_OK;
+}
+
+mdbf_status_t mdbf_get_packed(mdbf_handle_t h, int which, uint32_t *out, int out_on_device, void *stream) {
+    mdbf_status_t rc = check_handle(h, "mdbf_get_packed");
+    if (rc) return rc;
+    if (!out || (which != 0 && which != 1)) { set_error("mdbf_get_packed: bad argument"); return MDBF_ERR_INVALID_ARG; }
+    const Layer &L = h->L;
+    const size_t bytes = which == 0 ? (size_t)L.d.d_out * L.wordsA * 4 : (size_t)L.d.k * L.wordsB * 4;
+    cudaStream_t st = (cudaStream_t)stream;
+    MDBF_CUDA(cudaMemcpyAsync(out, which == 0 ? L.wA : L.wB, bytes,
+                              out_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
+    MDBF_CUDA(cudaStreamSynchronize(st));
+    return MDBF_OK;
+}
+
+mdbf_status_t mdbf_get_envelope(mdbf_handle_t h, int which, float *out, int out_on_device, void *stream) {
+    mdbf_status_t rc = check_handle(h, "mdbf_get_envelope");
+    if (rc) return rc;
+    if (!out || which < 0 || which > 3) { set_error("mdbf_get_envelope: bad argument"); return MDBF_ERR_INVALID_ARG; }
+    const Layer &L = h->L;
+    const void *src[4] = {L.UA, L.VA, L.UB, L.VB};
+    const size_t n[4] = {(size_t)L.d.d_out * L.d.l, (size_t)L.d.k * L.d.l, (size_t)L.d.k * L.d.l,
+                         (size_t)L.d.d_in * L.d.l};
+    cudaStream_t st = (cudaStream_t)stream;
+    if (out_on_device) {
+        rc = launch_env_read(src[which], out, n[which], L.d.env_dtype, st);
+        if (rc) return rc;
+        MDBF_CUDA(cudaStreamSynchronize(st));
+        return MDBF_OK;
+    }
+    float *tmp = nullptr;
+    MDBF_CUDA(cudaMalloc(&tmp, n[which] * 4));
+    rc = launch_env_read(src[which], tmp, n[which], L.d.env_dtype, st);
+    cudaError_t e = cudaSuccess;
+    if (rc == MDBF_OK) e = cudaMemcpyAsync(out, tmp, n[which] * 4, cudaMemcpyDeviceToHost, st);
+    if (rc == MDBF_OK && e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(tmp);
+    if (rc) return rc;
+    if (e != cudaSuccess) return cuda_fail(e, "mdbf_get_envelope copy");
+    return MDBF_OK;
+}
+
+mdbf_status_t mdbf_get_desc(mdbf_handle_t h, mdbf_desc_t *out) {
+    mdbf_status_t rc = check_handle(h, "mdbf_get_desc");
+    if (rc) return rc;
+    if (!out) { set_error("mdbf_get_desc: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    *out = h->L.d;
+    return MDBF_OK;
+}
+
+mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel) {
+    mdbf_status_t rc = check_handle(h, "mdbf_set_kernel");
+    if (rc) return rc;
+    if (kernel < MDBF_KERNEL_AUTO || kernel > MDBF_KERNEL_PREFILL) {
+        set_error("mdbf_set_kernel: unknown kernel %d", kernel);
+        return MDBF_ERR_INVALID_ARG;
+    }
+    h->kernel = kernel;
+    return MDBF_OK;
+}
+
+static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32_t T, int32_t act_dtype,
+                                  cudaStream_t st) {
+    Layer &L = h->L;
+    if (T < 1 || T > L.d.max_T) {
+        set_error("mdbf_linear_forward: T=%d outside [1, max_T=%d]", T, L.d.max_T);
+        return MDBF_ERR_SHAPE;
+    }
+    if (!valid_dtype(act_dtype)) { set_error("mdbf_linear_forward: bad act_dtype %d", act_dtype); return MDBF_ERR_DTYPE; }
+    int kernel = h->kernel;
+    const bool tc_ok = (act_dtype == MDBF_BF16) && (L.d.env_dtype != MDBF_F32);
+    if (kernel == MDBF_KERNEL_AUTO) {
+        if (!tc_ok) kernel = MDBF_KERNEL_ALU;
+        else if (T <= kDecodeMaxT && L.d.l <= 32) kernel = MDBF_KERNEL_DECODE;
+        else kernel = MDBF_KERNEL_PREFILL;
+    }
+    if (kernel != MDBF_KERNEL_ALU && !tc_ok) {
+        set_error("mdbf_linear_forward: the tensor-core kernels need bf16 activations and 16-bit envelopes");
+        return MDBF_ERR_DTYPE;
+    }
+    if (kernel == MDBF_KERNEL_DECODE && (T > kDecodeMaxT || L.d.l > 32)) {
+        set_error("mdbf_linear_forward: the small-T kernel handles T <= %d and l <= 32 (got T=%d, l=%d)",
+                  kDecodeMaxT, T, L.d.l);
+        return MDBF_ERR_SHAPE;
+    }
+    int launches = 0;
+    mdbf_status_t rc;
+    if (kernel == MDBF_KERNEL_ALU) rc = launch_forward_alu(L, x, y, T, act_dtype, st, &launches);
+    else if (kernel == MDBF_KERNEL_DECODE) rc = launch_forward_decode(L, x, y, T, st, &launches);
+    else rc = launch_forward_prefill(L, x, y, T, st, &launches);
+    if (rc == MDBF_OK) h->last_launches = launches;
+    return rc;
+}
+
+mdbf_status_t mdbf_linear_forward(mdbf_handle_t h, const void *x, void *y, int32_t T, int32_t act_dtype,
+                                  void *stream) {
+    mdbf_status_t rc = check_handle(h, "mdbf_linear_forward");
+    if (rc) return rc;
+    if (!x || !y) { set_error("mdbf_linear_forward: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    return forward_impl(h, x, y, T, act_dtype, (cudaStream_t)stream);
+}
+
+mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T,
+                                       int32_t act_dtype, void *stream) {
+    mdbf_status_t rc = check_handle(h, "mdbf_linear_forward_host");
+    if (rc) return rc;
+    if (!x_host || !y_host) { set_error("mdbf_linear_forward_host: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    Layer &L = h->L;
+    if (T < 1 || T > L.d.max_T) {
+        set_error("mdbf_linear_forward_host: T=%d outside [1, max_T=%d]", T, L.d.max_T);
+        return MDBF_ERR_SHAPE;
+    }
+    if (!valid_dtype(act_dtype)) { set_error("mdbf_linear_forward_host: bad act_dtype %d", act_dtype); return MDBF_ERR_DTYPE; }
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t es = dtype_size(act_dtype);
+    MDBF_CUDA(cudaMemcpyAsync(L.xstage, x_host, (size_t)T * L.d.d_in * es, cudaMemcpyHostToDevice, st));
+    rc = forward_impl(h, L.xstage, L.ystage, T, act_dtype, st);
+    if (rc) return rc;
+    MDBF_CUDA(cudaMemcpyAsync(y_host, L.ystage, (size_t)T * L.d.d_out * es, cudaMemcpyDeviceToHost, st));
+    MDBF_CUDA(cudaStreamSynchronize(st));
+    return MDBF_OK;
+}
+
+mdbf_status_t mdbf_get_intermediate(mdbf_handle_t h, float *z, int32_t T, int out_on_device, void *stream) {
+    mdbf_status_t rc = check_handle(h, "mdbf_get_intermediate");
+    if (rc) return rc;
+    Layer &L = h->L;
+    if (!z) { set_error("mdbf_get_intermediate: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    if (T < 1 || T > L.d.max_T) { set_error("mdbf_get_intermediate: bad T"); return MDBF_ERR_SHAPE; }
+    cudaStream_t st = (cudaStream_t)stream;
+    rc = launch_zsum(L, T, st);
+    if (rc) return rc;
+    MDBF_CUDA(cudaMemcpyAsync(z, L.zsum, (size_t)T * L.d.k * sizeof(float),
+                              out_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
+    MDBF_CUDA(cudaStreamSynchronize(st));
+    return MDBF_OK;
+}
+
+mdbf_status_t mdbf_reconstruct(mdbf_handle_t h, float *W, void *stream) {
+    mdbf_status_t rc = check_handle(h, "mdbf_reconstruct");
+    if (rc) return rc;
+    if (!W) { set_error("mdbf_reconstruct: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    return launch_reconstruct(h->L, W, (cudaStream_t)stream);
+}
+
+mdbf_status_t mdbf_poll_status(mdbf_handle_t h, int32_t *device_status) {
+    mdbf_status_t rc = check_handle(h, "mdbf_poll_status");
+    if (rc) return rc;
+    if (!device_status) { set_error("mdbf_poll_status: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    MDBF_CUDA(cudaDeviceSynchronize());
+    MDBF_CUDA(cudaMemcpy(device_status, h->L.status, sizeof(int32_t), cudaMemcpyDeviceToHost));
+    MDBF_CUDA(cudaMemset(h->L.status, 0, sizeof(int32_t)));
+    return MDBF_OK;
+}
+
+mdbf_status_t mdbf_last_launch_count(mdbf_handle_t h, int32_t *count) {
+    mdbf_status_t rc = check_handle(h, "mdbf_last_launch_count");
+    if (rc) return rc;
+    if (!count) { set_error("mdbf_last_launch_count: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    *count = h->last_launches;
+    return MDBF_OK;
+}
+
+mdbf_status_t mdbf_destroy(mdbf_handle_t h) {
+    mdbf_status_t rc = check_handle(h, "mdbf_destroy");
+    if (rc) return rc;
+    cudaDeviceSynchronize();
+    free_layer(h->L);
+    h->magic = 0;
+    delete h;
+    return MDBF_OK;
+}
+
+}  // extern "C"

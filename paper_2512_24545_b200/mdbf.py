@@ -1,0 +1,175 @@
+"""ctypes binding of libmdbf.so — same names as include/mdbf.h, argument
+marshalling only.  Every computation runs in the CUDA library; there is no
+fallback: if the library has not been built or no sm_100 device is present the
+calls raise.
+
+Device buffers are passed as raw addresses (e.g. torch.Tensor.data_ptr());
+host buffers as numpy arrays.  Streams are raw cudaStream_t integers
+(torch.cuda.current_stream().cuda_stream) or 0.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmdbf.so")
+
+F32, F16, BF16 = 0, 1, 2
+KERNEL_AUTO, KERNEL_ALU, KERNEL_DECODE, KERNEL_PREFILL = 0, 1, 2, 3
+OK = 0
+ERR_INVALID_ARG, ERR_SHAPE, ERR_DTYPE, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT, ERR_VALUE = (
+    -1, -2, -3, -4, -5, -6, -7, -8)
+DTYPES = {"f32": F32, "f16": F16, "bf16": BF16}
+
+EXPORTS = (
+    "mdbf_pack_signs", "mdbf_unpack_signs", "mdbf_pack", "mdbf_get_packed", "mdbf_get_envelope",
+    "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host",
+    "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_poll_status", "mdbf_last_launch_count",
+    "mdbf_destroy", "mdbf_last_error", "mdbf_version",
+)
+
+
+class MdbfError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"libmdbf status {status}: {message}")
+        self.status = status
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [("d_out", ctypes.c_int32), ("d_in", ctypes.c_int32), ("k", ctypes.c_int32),
+                ("l", ctypes.c_int32), ("env_dtype", ctypes.c_int32), ("max_T", ctypes.c_int32)]
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libmdbf.so (built by paper_2512_24545_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2512_24545_b200.build` "
+            "(there is no CPU fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    L.mdbf_pack_signs.argtypes = [vp, i64, i64, vp, ctypes.c_int, vp]
+    L.mdbf_unpack_signs.argtypes = [vp, i64, i64, vp, ctypes.c_int, vp]
+    L.mdbf_pack.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, vp, vp, ctypes.c_int, vp,
+                            ctypes.POINTER(vp)]
+    L.mdbf_get_packed.argtypes = [vp, ctypes.c_int, vp, ctypes.c_int, vp]
+    L.mdbf_get_envelope.argtypes = [vp, ctypes.c_int, vp, ctypes.c_int, vp]
+    L.mdbf_get_desc.argtypes = [vp, ctypes.POINTER(Desc)]
+    L.mdbf_set_kernel.argtypes = [vp, i32]
+    L.mdbf_linear_forward.argtypes = [vp, vp, vp, i32, i32, vp]
+    L.mdbf_linear_forward_host.argtypes = [vp, vp, vp, i32, i32, vp]
+    L.mdbf_get_intermediate.argtypes = [vp, vp, i32, ctypes.c_int, vp]
+    L.mdbf_reconstruct.argtypes = [vp, vp, vp]
+    L.mdbf_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
+    L.mdbf_last_launch_count.argtypes = [vp, ctypes.POINTER(i32)]
+    L.mdbf_destroy.argtypes = [vp]
+    for name in EXPORTS:
+        getattr(L, name).restype = i32
+    L.mdbf_last_error.restype = ctypes.c_char_p
+    L.mdbf_last_error.argtypes = []
+    L.mdbf_version.restype = ctypes.c_char_p
+    L.mdbf_version.argtypes = []
+    _lib = L
+    return L
+
+
+def last_error() -> str:
+    return lib().mdbf_last_error().decode()
+
+
+def version() -> str:
+    return lib().mdbf_version().decode()
+
+
+def _check(status: int) -> None:
+    if status != OK:
+        raise MdbfError(status, last_error())
+
+
+def _addr(buf) -> int:
+    """Raw address of a numpy array (host) or an int (device pointer)."""
+    if isinstance(buf, np.ndarray):
+        if not buf.flags["C_CONTIGUOUS"]:
+            raise ValueError("host buffers must be C-contiguous")
+        return buf.ctypes.data
+    if buf is None:
+        return 0
+    return int(buf)
+
+
+def mdbf_pack_signs(s, rows: int, cols: int, out, on_device: bool, stream: int = 0) -> None:
+    _check(lib().mdbf_pack_signs(_addr(s), rows, cols, _addr(out), int(on_device), stream))
+
+
+def mdbf_unpack_signs(p, rows: int, cols: int, out, on_device: bool, stream: int = 0) -> None:
+    _check(lib().mdbf_unpack_signs(_addr(p), rows, cols, _addr(out), int(on_device), stream))
+
+
+def mdbf_pack(d_out: int, d_in: int, k: int, l: int, env_dtype: int, max_T: int,
+              S_A, S_B, U_A, V_A, U_B, V_B, inputs_on_device: bool = False, stream: int = 0) -> int:
+    """Returns the handle (an integer address)."""
+    desc = Desc(d_out, d_in, k, l, env_dtype, max_T)
+    h = ctypes.c_void_p()
+    _check(lib().mdbf_pack(ctypes.byref(desc), _addr(S_A), _addr(S_B), _addr(U_A), _addr(V_A),
+                           _addr(U_B), _addr(V_B), int(inputs_on_device), stream, ctypes.byref(h)))
+    return h.value
+
+
+def mdbf_get_packed(h: int, which: int, out, out_on_device: bool = False, stream: int = 0) -> None:
+    _check(lib().mdbf_get_packed(h, which, _addr(out), int(out_on_device), stream))
+
+
+def mdbf_get_envelope(h: int, which: int, out, out_on_device: bool = False, stream: int = 0) -> None:
+    _check(lib().mdbf_get_envelope(h, which, _addr(out), int(out_on_device), stream))
+
+
+def mdbf_get_desc(h: int) -> Desc:
+    d = Desc()
+    _check(lib().mdbf_get_desc(h, ctypes.byref(d)))
+    return d
+
+
+def mdbf_set_kernel(h: int, kernel: int) -> None:
+    _check(lib().mdbf_set_kernel(h, kernel))
+
+
+def mdbf_linear_forward(h: int, x, y, T: int, act_dtype: int, stream: int = 0) -> None:
+    _check(lib().mdbf_linear_forward(h, _addr(x), _addr(y), T, act_dtype, stream))
+
+
+def mdbf_linear_forward_host(h: int, x_host, y_host, T: int, act_dtype: int, stream: int = 0) -> None:
+    _check(lib().mdbf_linear_forward_host(h, _addr(x_host), _addr(y_host), T, act_dtype, stream))
+
+
+def mdbf_get_intermediate(h: int, z, T: int, out_on_device: bool = False, stream: int = 0) -> None:
+    _check(lib().mdbf_get_intermediate(h, _addr(z), T, int(out_on_device), stream))
+
+
+def mdbf_reconstruct(h: int, W, stream: int = 0) -> None:
+    _check(lib().mdbf_reconstruct(h, _addr(W), stream))
+
+
+def mdbf_poll_status(h: int) -> int:
+    v = ctypes.c_int32()
+    _check(lib().mdbf_poll_status(h, ctypes.byref(v)))
+    return v.value
+
+
+def mdbf_last_launch_count(h: int) -> int:
+    v = ctypes.c_int32()
+    _check(lib().mdbf_last_launch_count(h, ctypes.byref(v)))
+    return v.value
+
+
+def mdbf_destroy(h: int) -> None:
+    _check(lib().mdbf_destroy(h))
