@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the MDBF linear forward (libmdbf) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl mdbf|reference]
+
+Prints ONE JSON line.  Default workload `decode_qproj`: the 7B-class q_proj
+shape (d_out = d_in = 4096, l = 16, T = 1, bf16 activations with outlier
+channels, fp16 envelopes) at k = 1664 (~1.0 bpw) and k = 2560 (~1.5 bpw).
+A step is one forward through every layer of a rotation of distinct layers
+whose packed weights exceed L2 several times over, launched back to back on
+one stream, so that every step streams its weights from HBM.
+
+Metric: GB/s of ALGORITHMIC bytes (packed signs + envelopes + x + y, each
+once) for the decode workloads; TFLOP/s of the expanded sign contraction
+2*l*T*k*(d_in + d_out) for the prefill workloads.
+
+Multi-GPU: the path does not shard (one layer = one GPU); `--gpus N` under
+torchrun runs N independent replicas ("replicas only", weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (None until a capture exists for that workload).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------- accounting
+def algorithmic_bytes(spec, T):
+    env_b = 4 if spec.env_dtype == "f32" else 2
+    act_b = 4 if spec.act_dtype == "f32" else 2
+    signs = spec.k * (spec.d_in + spec.d_out) // 8
+    env = env_b * spec.l * (spec.d_in + spec.d_out + 2 * spec.k)
+    act = act_b * T * (spec.d_in + spec.d_out)
+    return signs + env + act
+
+
+def expanded_flops(spec, T):
+    return 2.0 * spec.l * T * spec.k * (spec.d_in + spec.d_out)
+
+
+# ---------------------------------------------------------------- workloads
+def workload_specs(name):
+    """-> (list of (LayerSpec, copies), T, metric kind, description)."""
+    from paper_2512_24545_b200 import inputs
+    if name == "decode_qproj":
+        return [(inputs.qproj(1664), 64), (inputs.qproj(2560), 64)], 1, "hbm", \
+            "q_proj 4096x4096 l=16 T=1, k=1664 and k=2560, 64 distinct layers each"
+    if name.startswith("decode_mlp"):
+        T = int(name.split("_T")[1]) if "_T" in name else 1
+        return [(inputs.mlp("up"), 16), (inputs.mlp("down"), 16)], T, "hbm", \
+            f"MLP up 11008x4096 and down 4096x11008, k=3968 l=16 T={T}, 16 distinct layers each"
+    if name.startswith("block70b"):
+        T = int(name.split("_T")[1]) if "_T" in name else 1
+        return [(s, 4 if T <= 16 else 1) for s in inputs.block70b()], T, "hbm" if T <= 16 else "tensor", \
+            f"70B-class decoder block, 7 linears, l=16 ~1.0 bpw, T={T}"
+    if name.startswith("prefill"):
+        # prefill_<d_out>_l<l>_<bpw10|bpw15>
+        parts = name.split("_")
+        d_out = int(parts[1]) if len(parts) > 1 else 4096
+        l = int(parts[2][1:]) if len(parts) > 2 else 16
+        bpw = 1.5 if (len(parts) > 3 and parts[3] == "bpw15") else 1.0
+        return [(inputs.prefill(d_out, l, bpw), 1)], 2048, "tensor", \
+            f"prefill {d_out}x4096 l={l} ~{bpw} bpw T=2048"
+    raise SystemExit(f"unknown workload {name}")
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled during the timed region."""
+
+    def __init__(self, index):
+        self.index = index
+        self.samples = []
+        self.proc = None
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            f = [x.strip() for x in s.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_setup(n_gpus):
+    import torch
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        return dist, rank, world, local
+    return None, 0, 1, 0
+
+
+# ------------------------------------------------------------------ mdbf arm
+def run_mdbf(args):
+    import torch
+    from paper_2512_24545_b200 import build, inputs, mdbf as M
+    build.build()
+    dist, rank, world, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    peaks, peak_kind = load_peaks()
+    groups, T, bound, desc = workload_specs(args.workload)
+    stream = torch.cuda.Stream()
+    st = stream.cuda_stream
+
+    layers = []          # (handle, spec, x_dev, y_dev, x_host, y_host)
+    total_bytes = 0
+    total_flops = 0.0
+    weight_bytes = 0
+    xs = {}
+    for spec, copies in groups:
+        for c in range(args.copies if args.copies > 0 else copies):
+            sp = inputs.scaled(spec, seed=spec.seed + 1000 * (c + 1)) if c else spec
+            lay = inputs.make_layer(sp)
+            h = M.mdbf_pack(sp.d_out, sp.d_in, sp.k, sp.l, M.DTYPES[sp.env_dtype], T,
+                            *[np.ascontiguousarray(lay[n]) for n in ("S_A", "S_B", "U_A", "V_A", "U_B", "V_B")])
+            if sp.d_in not in xs:
+                xh = torch.from_numpy(inputs.make_activations(sp, T)).to(torch.bfloat16).pin_memory()
+                xs[sp.d_in] = (xh, xh.cuda())
+            xh, xd = xs[sp.d_in]
+            yd = torch.zeros((T, sp.d_out), dtype=torch.bfloat16, device="cuda")
+            yh = torch.zeros((T, sp.d_out), dtype=torch.bfloat16).pin_memory()
+            layers.append((h, sp, xd, yd, xh, yh))
+            total_bytes += algorithmic_bytes(sp, T)
+            total_flops += expanded_flops(sp, T)
+            weight_bytes += algorithmic_bytes(sp, 0)
+    torch.cuda.synchronize()
+
+    flush = None
+    if weight_bytes < 2 * 126e6:       # rotation too small to defeat L2: flush between steps
+        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+
+    def step():
+        for (h, sp, xd, yd, _, _) in layers:
+            M.mdbf_linear_forward(h, xd.data_ptr(), yd.data_ptr(), T, M.BF16, st)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    graph = None
+    with torch.cuda.stream(stream):
+        step()                       # first call sets kernel attributes (not capturable state)
+        torch.cuda.synchronize()
+        if not args.no_graph:
+            # one CUDA graph per step: removes the host launch cost of the back-to-back forwards
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                step()
+            run_step = graph.replay
+        else:
+            run_step = step
+        for _ in range(max(3, args.warmup)):
+            run_step()
+        barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(args.steps)]
+        for (e0, e1) in ev:
+            if flush is not None:
+                flush.fill_(1)
+            e0.record(stream)
+            run_step()
+            e1.record(stream)
+        barrier()
+        clocks = sampler.stop()
+        ms = sum(e0.elapsed_time(e1) for e0, e1 in ev)
+    launches = sum(M.mdbf_last_launch_count(h) for (h, *_rest) in layers) * args.steps
+
+    # end to end: host buffers through the C-ABI, copies inside the timed region
+    e2e_steps = max(1, min(args.steps, 10))
+    for _ in range(2):
+        for (h, sp, _, _, xh, yh) in layers:
+            M.mdbf_linear_forward_host(h, xh.data_ptr(), yh.data_ptr(), T, M.BF16, st)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        for (h, sp, _, _, xh, yh) in layers:
+            M.mdbf_linear_forward_host(h, xh.data_ptr(), yh.data_ptr(), T, M.BF16, st)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    h2d = sum(T * sp.d_in * 2 for (_, sp, *_r) in layers)
+    d2h = sum(T * sp.d_out * 2 for (_, sp, *_r) in layers)
+
+    ms_t = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device="cuda")
+    if dist:
+        dist.all_reduce(ms_t, op=dist.ReduceOp.MAX)
+    ms_max, e2e_ms_max = float(ms_t[0]), float(ms_t[1])
+    sec = ms_max / 1e3
+    if bound == "hbm":
+        metric, unit = "decode_algorithmic_GBps", "GB/s"
+        per_step = total_bytes / 1e9
+        peak = peaks["hbm_gbs"]
+    else:
+        metric, unit = "prefill_expanded_TFLOPs", "TFLOP/s"
+        per_step = total_flops / 1e12
+        peak = peaks["bf16_tflops"] if sec < 1.0 else peaks["bf16_tflops_sustained"]
+    value = world * per_step * args.steps / sec
+    per_gpu = per_step * args.steps / sec
+    e2e_value = world * per_step * e2e_steps / (e2e_ms_max / 1e3)
+
+    out = {
+        "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_max / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "description": desc, "layers": len(layers), "T": T,
+                   "weights_MB": round(weight_bytes / 1e6, 1),
+                   "l2_policy": ("rotation of distinct layers larger than L2" if flush is None
+                                 else "256 MiB L2 flush between steps"),
+                   "launch": "CUDA graph replay per step" if graph is not None else "stream launches",
+                   "replicas": world},
+        "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "roofline": {"bound": bound, "achieved": per_gpu, "peak": peak, "unit": unit,
+                     "frac": per_gpu / peak, "peak_source": f"of {peak_kind}",
+                     "kernel": "decode_stage_kernel" if T <= 4 else "prefill_stage_kernel",
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(groups[0][0], T, bound, budget_s=20.0)
+    for (h, *_r) in layers:
+        M.mdbf_destroy(h)
+    if dist:
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
+# -------------------------------------------------------- oracle (CPU) arm
+def oracle_sample(spec, T, rows_frac):
+    """One bounded sample of the oracle: the dense definition restricted to a
+    leading fraction of the output rows of one layer.  Returns (seconds, fraction)."""
+    from oracle import mdbf_oracle as orc
+    from paper_2512_24545_b200 import inputs
+    lay = inputs.make_layer(spec)
+    x = inputs.make_activations(spec, T)
+    n = max(1, int(round(spec.d_out * rows_frac)))
+    rows = np.arange(n)
+    args = (lay["S_A"], lay["S_B"], lay["U_A"], lay["V_A"], lay["U_B"], lay["V_B"])
+    t0 = time.perf_counter()
+    W = orc.reconstruct_rows(rows, *args)
+    y = W @ x.T.astype(np.float64)
+    dt = time.perf_counter() - t0
+    assert np.all(np.isfinite(y))
+    return dt, n / spec.d_out
+
+
+def cpu_baseline(spec, T, bound, budget_s=15.0):
+    cores = len(os.sched_getaffinity(0))
+    dt, frac = oracle_sample(spec, T, 1.0 / 64)          # probe
+    frac_target = min(1.0, max(1.0 / 64, frac * budget_s / max(dt, 1e-3) * 0.5))
+    dt, frac = oracle_sample(spec, T, frac_target)
+    reps, total = 1, dt
+    while total < budget_s and reps < 200:               # repeat the sample until ~budget_s of CPU work
+        d2, _ = oracle_sample(spec, T, frac_target)
+        total += d2
+        reps += 1
+    dt = total / reps
+    if bound == "hbm":
+        v, unit = algorithmic_bytes(spec, T) * frac / 1e9 / dt, "GB/s"
+    else:
+        v, unit = expanded_flops(spec, T) * frac / 1e12 / dt, "TFLOP/s"
+    return {"value": v, "unit": unit, "cores": cores, "kind": "oracle",
+            "sample": f"fp64 dense definition on the first {frac:.3f} of the output rows of one "
+                      f"{spec.name} layer, T={T}, {reps} repetitions of {dt:.2f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    groups, T, bound, desc = workload_specs(args.workload)
+    spec = groups[0][0]
+    cores = len(os.sched_getaffinity(0))
+    dt, frac = oracle_sample(spec, T, 1.0 / 64)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    frac = min(1.0, max(1.0 / 64, frac * budget / max(dt, 1e-3) * 0.5))
+    for _ in range(args.warmup):
+        oracle_sample(spec, T, frac)
+    total = 0.0
+    for _ in range(args.steps):
+        dt, fr = oracle_sample(spec, T, frac)
+        total += dt
+    if bound == "hbm":
+        metric, unit = "decode_algorithmic_GBps", "GB/s"
+        per = algorithmic_bytes(spec, T) * fr / 1e9
+    else:
+        metric, unit = "prefill_expanded_TFLOPs", "TFLOP/s"
+        per = expanded_flops(spec, T) * fr / 1e12
+    value = per * args.steps / total
+    sample = (f"fp64 dense definition on the first {fr:.3f} of the output rows of one {spec.name} "
+              f"layer per step, T={T}")
+    print(json.dumps({
+        "impl": "reference", "metric": metric, "value": value, "unit": unit,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "description": desc},
+        "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="decode_qproj")
+    ap.add_argument("--impl", default="mdbf", choices=["mdbf", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every forward from the host")
+    ap.add_argument("--copies", type=int, default=0, help="distinct layers per shape (0 = workload default); small values for ncu captures")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_mdbf(args)
+
+
+if __name__ == "__main__":
+    main()
