@@ -40,6 +40,9 @@ struct Layer {
     // kernel-private bf16 copies of V_A / V_B in MMA B-fragment order (see forward_decode.cu)
     uint2 *vfA, *vfB;
     int NT;                       // 8-column mode tiles in the fragment copies: 1, 2, 4 or 8
+    // kernel-private padded copies of V_A / V_B for the large-T kernel: [cols_pad64][LP] raw 16-bit
+    uint16_t *vpA, *vpB;
+    int LP;                       // l rounded up to a power of two
     // scratch
     float *z;                     // [kMaxKSplit][zT][k] stage-B partial sums of the small-T kernel
     size_t zstride;               // zT * k
@@ -88,6 +91,8 @@ mdbf_status_t launch_env_round(const float *src, void *dst, size_t n, int dtype,
 mdbf_status_t launch_env_read(const void *src, float *dst, size_t n, int dtype, cudaStream_t st);
 mdbf_status_t launch_vfrag(const void *V, int cols, int l, int env_dtype, uint2 *out, int ktiles, int NT,
                            cudaStream_t st);
+mdbf_status_t launch_vpad(const void *V, int cols, int l, int env_dtype, uint16_t *out, int cols_pad, int LP,
+                          cudaStream_t st);
 mdbf_status_t launch_reconstruct(const Layer &L, float *W, cudaStream_t st);
 mdbf_status_t launch_forward_alu(Layer &L, const void *x, void *y, int T, int act_dtype,
                                  cudaStream_t st, int *launches);

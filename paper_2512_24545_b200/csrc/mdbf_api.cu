@@ -58,7 +58,7 @@ static mdbf_status_t check_handle(mdbf_handle_t h, const char *fn) {
 }
 
 static void free_layer(Layer &L) {
-    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.z, L.zsum, L.xstage, L.ystage, L.status};
+    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.vpA, L.vpB, L.z, L.zsum, L.xstage, L.ystage, L.status};
     for (void *p : ptrs)
         if (p) cudaFree(p);
 }
@@ -171,6 +171,13 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     L.NT = d.l <= 8 ? 1 : d.l <= 16 ? 2 : d.l <= 32 ? 4 : 8;
     PACK_CUDA(cudaMalloc(&L.vfA, (size_t)L.ktA * 8 * L.NT * 256));
     PACK_CUDA(cudaMalloc(&L.vfB, (size_t)L.ktB * 8 * L.NT * 256));
+    L.LP = 1;
+    while (L.LP < d.l) L.LP *= 2;
+    const int padA = ceil_div(d.k, 64) * 64, padB = ceil_div(d.d_in, 64) * 64;
+    if (d.env_dtype != MDBF_F32) {      // the tensor-core kernels take 16-bit envelopes only
+        PACK_CUDA(cudaMalloc(&L.vpA, (size_t)padA * L.LP * 2));
+        PACK_CUDA(cudaMalloc(&L.vpB, (size_t)padB * L.LP * 2));
+    }
     L.zstride = (size_t)decode_scratch_T(d) * d.k;
     PACK_CUDA(cudaMalloc(&L.z, (size_t)kMaxKSplit * L.zstride * sizeof(float)));
     PACK_CUDA(cudaMalloc(&L.zsum, (size_t)d.max_T * d.k * sizeof(float)));
@@ -202,6 +209,10 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     PACK_RC(launch_env_round((const float *)dsrc[5], L.VB, nVB, d.env_dtype, st));
     PACK_RC(launch_vfrag(L.VA, d.k, d.l, d.env_dtype, L.vfA, L.ktA, L.NT, st));
     PACK_RC(launch_vfrag(L.VB, d.d_in, d.l, d.env_dtype, L.vfB, L.ktB, L.NT, st));
+    if (d.env_dtype != MDBF_F32) {
+        PACK_RC(launch_vpad(L.VA, d.k, d.l, d.env_dtype, L.vpA, padA, L.LP, st));
+        PACK_RC(launch_vpad(L.VB, d.d_in, d.l, d.env_dtype, L.vpB, padB, L.LP, st));
+    }
     PACK_CUDA(cudaStreamSynchronize(st));
     for (void *p : temps) cudaFree(p);
     temps.clear();
