@@ -1,6 +1,7 @@
 // Internal declarations shared by the libmdbf translation units.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_fp16.h>
 #include <cuda_bf16.h>
@@ -40,9 +41,15 @@ struct Layer {
     // kernel-private bf16 copies of V_A / V_B in MMA B-fragment order (see forward_decode.cu)
     uint2 *vfA, *vfB;
     int NT;                       // 8-column mode tiles in the fragment copies: 1, 2, 4 or 8
-    // kernel-private padded copies of V_A / V_B for the large-T kernel: [cols_pad64][LP] raw 16-bit
-    uint16_t *vpA, *vpB;
+    // large-T kernel (present only when max_T exceeds the small-T kernel's range and l <= 32):
     int LP;                       // l rounded up to a power of two
+    uint2 *wkA, *wkB;             // K-blocked sign words [kblocks][rows_pad128]
+    int rpA, rpB;                 // rows padded to 128
+    int padA, padB;               // reduction length (k, d_in) padded to 64
+    float *vtB;                   // V_B transposed, fp32 [LP][padB]
+    __nv_bfloat16 *xsB, *xsA;     // pre-scaled operands [xs_rows][padB], [xs_rows][padA]
+    size_t xs_rows;               // max_T * LP rounded up to 256
+    CUtensorMap tmB, tmA;         // tensor maps of xsB / xsA
     // scratch
     float *z;                     // [kMaxKSplit][zT][k] stage-B partial sums of the small-T kernel
     size_t zstride;               // zT * k
@@ -91,8 +98,10 @@ mdbf_status_t launch_env_round(const float *src, void *dst, size_t n, int dtype,
 mdbf_status_t launch_env_read(const void *src, float *dst, size_t n, int dtype, cudaStream_t st);
 mdbf_status_t launch_vfrag(const void *V, int cols, int l, int env_dtype, uint2 *out, int ktiles, int NT,
                            cudaStream_t st);
-mdbf_status_t launch_vpad(const void *V, int cols, int l, int env_dtype, uint16_t *out, int cols_pad, int LP,
-                          cudaStream_t st);
+mdbf_status_t launch_kblock(const uint32_t *canon, int rows, int nwords, uint2 *out, int rows_pad, int kblocks,
+                            cudaStream_t st);
+mdbf_status_t launch_vtrans(const void *V, int cols, int l, int env_dtype, float *out, int pad, int LP, cudaStream_t st);
+mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad);
 mdbf_status_t launch_reconstruct(const Layer &L, float *W, cudaStream_t st);
 mdbf_status_t launch_forward_alu(Layer &L, const void *x, void *y, int T, int act_dtype,
                                  cudaStream_t st, int *launches);

@@ -1,30 +1,37 @@
 // Large-T ("prefill") path of the MDBF forward on the 5th-generation tensor
-// cores: tcgen05.mma with the accumulator in tensor memory (TMEM).
+// cores: tcgen05.mma with the accumulator in tensor memory (TMEM), the
+// activation operand staged by TMA, the sign operand expanded in shared memory.
 //
 // One stage is the dense contraction behind  sum_t D_{u_t} S D_{v_t}  (Eq.
 // me-dbf-expand) over a block of tokens:
 //
-//     D[r][(tau, t)] = sum_c  S[r][c] * bf16( V[c][t] * in[tau][c] )        (GEMM, width l*T)
-//     out[tau][r]    = sum_t  U[r][t] * D[r][(tau, t)]                      (fused epilogue)
+//     Xs[(tau, t)][c] = bf16( V[c][t] * in[tau][c] )                        (pre-scale, one rounding)
+//     D[r][(tau, t)]  = sum_c  S[r][c] * Xs[(tau, t)][c]                    (GEMM, width l*T, fp32 acc)
+//     out[tau][r]     = sum_t  U[r][t] * D[r][(tau, t)]                     (fused epilogue)
 //
-// with A = S expanded to +-1.0 bf16 (M = 128 rows of S per CTA, K-major) and
-// B = the envelope-scaled activations generated on the fly (N = 256 columns =
-// 256/LP tokens x LP modes, K-major).  Stage B (S_B, V_B, U_B) maps x -> z,
-// stage A (S_A, V_A, U_A) maps z -> y (Eq. DBF-inference-form).
+// Stage B (S_B, V_B, U_B) maps x -> z, stage A (S_A, V_A, U_A) maps z -> y
+// (Eq. DBF-inference-form, column convention).  Three launches per forward:
 //
-// CTA = 9 warps.  Warps 0-7 are producers: per 64-column K block they expand
-// the packed sign words into the 128B-swizzled A tile (a 16-entry nibble table
-// turns 4 bits into four bf16 +-1) and write the B tile
-// (fp32 multiply, one rounding to bf16), then publish the stage through an
-// mbarrier after a generic->async proxy fence.  One lane of warp 8 issues the
-// MMAs (4 x K=16 per stage) and commits each stage back to the producers; a
-// 4-stage ring overlaps generation with the tensor pipe.  After the K loop the
-// producer warps read the 128 x 256 fp32 accumulator from TMEM (tcgen05.ld),
-// contract the LP modes of every token with U in registers and store.
+//   prescale_kernel      Xs_B from x and V_B (element-wise, HBM-bound, ~l*T*d_in*2 bytes written)
+//   gemm_stage_kernel<B> z, and in the same epilogue Xs_A = bf16(V_A * z) for the next stage
+//   gemm_stage_kernel<A> y
 //
-// Every mbarrier wait is bounded: when it expires the kernel records
-// MDBF_ERR_TIMEOUT in the layer's status word, all roles fall through to the
-// common exit, TMEM is released and the kernel returns.
+// GEMM CTA = 128 rows of S x 256 columns (256/LP tokens x LP modes), 6 warps:
+//   warps 0-3  expand 64 packed sign bits per row and K block into the 128B-swizzled bf16 A tile
+//              (+-1.0; three integer ops per pair of elements), later run the epilogue
+//   warp 4     one lane issues the TMA load of the 256 x 64 Xs tile (tensor map, 128B swizzle)
+//   warp 5     one lane issues 4 tcgen05.mma (K = 16 each) per K block and commits the stage
+// in a 4-stage mbarrier ring.  The epilogue reads the 128 x 256 fp32 accumulator from TMEM
+// (tcgen05.ld), contracts the LP modes of every token with U in registers and stores.
+//
+// Generating Xs on the fly inside the GEMM was measured first and rejected: the per-stage
+// global loads and 16-bit conversions saturated the load/store and conversion pipes
+// (tensor pipe 18 % busy); the pre-scaled operand costs < 10 % extra HBM time and removes
+// all of it.
+//
+// Every mbarrier wait is bounded: when it expires the kernel records MDBF_ERR_TIMEOUT in
+// the layer's status word, all roles fall through to the common exit, TMEM is released and
+// the kernel returns.  No TMA multicast is used anywhere.
 #include "common.cuh"
 
 namespace mdbf {
@@ -33,26 +40,29 @@ constexpr int PF_BM = 128;
 constexpr int PF_BN = 256;
 constexpr int PF_BK = 64;
 constexpr int PF_STAGES = 4;
-constexpr int PF_PRODUCERS = 256;
-constexpr int PF_THREADS = PF_PRODUCERS + 32;
+constexpr int PF_EXPANDERS = 128;
+constexpr int PF_THREADS = PF_EXPANDERS + 64;
 constexpr int PF_A_BYTES = PF_BM * PF_BK * 2;      // 16 KB
 constexpr int PF_B_BYTES = PF_BN * PF_BK * 2;      // 32 KB
 constexpr int PF_STAGE_BYTES = PF_A_BYTES + PF_B_BYTES;
 constexpr int PF_SMEM_BYTES = PF_STAGES * PF_STAGE_BYTES + 1024;   // + alignment slack
 constexpr uint32_t PF_MAX_POLLS = 1u << 20;
 
-struct PrefillArgs {
-    const uint32_t *words;   // canonical sign words [rows][nwords]
-    int nwords;
+struct GemmArgs {
+    const uint2 *wk;         // K-blocked sign words [kblocks][rows_pad], 64 bits per row and block
+    int rows_pad;
     int rows, cols;
     const void *U;           // [rows][l] env_dtype
-    const uint16_t *Vp;      // private padded copy [cols_pad][LP], raw 16-bit env values, zero padded
     int env_dtype, l;
-    const void *in;          // stage B: bf16 [T][cols]; stage A: fp32 [T][cols]
-    void *out;               // stage B: fp32 [T][rows]; stage A: bf16 [T][rows]
     int T;
-    int n_eff;               // MMA N: LP * tokens per tile actually used, multiple of 16
-    int vec_ok;              // input rows are 16-byte aligned and cols % 8 == 0
+    int n_eff;               // MMA N: columns of the tile actually used, multiple of 16
+    // stage B only: z out and the next stage's pre-scaled operand
+    float *z;                // [T][rows] fp32
+    const void *Vnext;       // V_A [rows][l] env_dtype
+    __nv_bfloat16 *xs_next;  // [(tau, t)][pad_next]
+    int pad_next;
+    // stage A only
+    __nv_bfloat16 *y;        // [T][rows]
     int32_t *status;
 };
 
@@ -64,6 +74,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -108,6 +121,12 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
 }
+// 2-D tiled TMA load into this CTA's shared memory, completion on an mbarrier (no multicast).
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -141,26 +160,24 @@ __device__ __forceinline__ uint32_t make_idesc(int n) {
     return d;                           // A and B K-major, no negation, dense
 }
 
-__device__ __forceinline__ float raw16_to_float(uint16_t r, int dtype) {
-    if (dtype == MDBF_F16) return __half2float(__ushort_as_half(r));
-    return __uint_as_float((uint32_t)r << 16);
-}
 __device__ __forceinline__ uint32_t pf_pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
+// bits (2i, 2i+1) of an 8-bit value -> two bf16 +-1.0 (bit set = -1.0): the multiply moves bit 0
+// to position 15 and bit 1 to position 31; every other product bit falls outside the mask.
+__device__ __forceinline__ uint32_t sign_pair(uint32_t byte, int i) {
+    return (((byte >> (2 * i)) * 0x40008000u) & 0x80008000u) | 0x3F803F80u;
+}
 
-// --------------------------------------------------------------------- kernel
+// ----------------------------------------------------------------- GEMM stage
 template <int LP, bool STAGE_A>
-__global__ void __launch_bounds__(PF_THREADS, 1) prefill_stage_kernel(const PrefillArgs a) {
-    constexpr int TPT = LP < 4 ? LP : 4;        // modes per producer thread
-    constexpr int TG = LP / TPT;                // mode groups
-    constexpr int TAUPT = 8 / TPT;              // tokens per producer thread
+__global__ void __launch_bounds__(PF_THREADS, 1)
+gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs) {
     constexpr int TT = PF_BN / LP;              // tokens per CTA tile
 
     extern __shared__ unsigned char pf_smem_raw[];
     __shared__ __align__(8) uint64_t bars[2 * PF_STAGES + 1];
-    __shared__ uint2 lut[16];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
     volatile int *abort_flag = &abort_flag_s;
@@ -178,22 +195,14 @@ __global__ void __launch_bounds__(PF_THREADS, 1) prefill_stage_kernel(const Pref
 
     if (tid == 0) {
         for (int s = 0; s < PF_STAGES; ++s) {
-            mbar_init(full_bar + 8 * s, PF_PRODUCERS);
+            mbar_init(full_bar + 8 * s, PF_EXPANDERS + 1);   // expander threads + the TMA issuer's expect_tx
             mbar_init(empty_bar + 8 * s, 1);
         }
         mbar_init(accum_bar, 1);
         abort_flag_s = 0;
         fence_barrier_init();
     }
-    if (tid < 16) {     // nibble -> four bf16 +-1.0 (bit set = -1), element i in half (i & 1) of word (i >> 1)
-        uint32_t w0 = 0x3F803F80u, w1 = 0x3F803F80u;
-        if (tid & 1) w0 |= 0x00008000u;
-        if (tid & 2) w0 |= 0x80000000u;
-        if (tid & 4) w1 |= 0x00008000u;
-        if (tid & 8) w1 |= 0x80000000u;
-        lut[tid] = make_uint2(w0, w1);
-    }
-    if (warp == 8) {
+    if (warp == 5) {
         tmem_alloc(smem_u32(&tmem_base_slot), PF_BN);
         tmem_relinquish();
     }
@@ -202,163 +211,90 @@ __global__ void __launch_bounds__(PF_THREADS, 1) prefill_stage_kernel(const Pref
     tc_fence_after();
     const uint32_t tmem_d = tmem_base_slot;
 
-    if (warp < 8) {
-        // ================================ producers ================================
-        const int arow = tid & 127, ahalf = tid >> 7;                  // A: one 32-bit word per thread per stage
-        const int grow = row0 + arow;
-        const uint32_t *wrow = a.words + (size_t)(grow < a.rows ? grow : 0) * a.nwords;
-        const bool arow_ok = grow < a.rows;
-        const int kc = tid & 7;                                         // B: 16-byte chunk along K
-        const int tg = (tid >> 3) % TG;
-        const int taug = (tid >> 3) / TG;
-        const int t_first = tg * TPT;
-
-        auto load_word = [&](int kb) -> uint32_t {
-            const int wi = kb * 2 + ahalf;
-            return (arow_ok && wi < a.nwords) ? __ldg(wrow + wi) : 0u;
-        };
-        // raw prefetch registers for the next K block
-        uint32_t aw_next = load_word(0);
-        uint32_t vraw[8][(TPT + 1) / 2];       // 8 columns x TPT modes, 16-bit values packed in pairs
-        float xin[TAUPT][8];
-        auto load_v = [&](int kb) {
-            const int c = kb * PF_BK + kc * 8;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint16_t *p = a.Vp + (size_t)(c + i) * LP + t_first;
-                if (TPT == 4) { const uint2 v = __ldg(reinterpret_cast<const uint2 *>(p)); vraw[i][0] = v.x; vraw[i][1] = v.y; }
-                else if (TPT == 2) vraw[i][0] = __ldg(reinterpret_cast<const uint32_t *>(p));
-                else vraw[i][0] = __ldg(p);
-            }
-        };
-        auto load_x = [&](int kb) {
-            const int c = kb * PF_BK + kc * 8;
-#pragma unroll
-            for (int j = 0; j < TAUPT; ++j) {
-                const int tau = tau0 + taug * TAUPT + j;
-                if (tau < a.T && a.vec_ok && c + 8 <= a.cols) {
-                    if (STAGE_A) {
-                        const float4 *p = reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(a.in) + (size_t)tau * a.cols + c);
-                        const float4 lo = __ldg(p), hi = __ldg(p + 1);
-                        xin[j][0] = lo.x; xin[j][1] = lo.y; xin[j][2] = lo.z; xin[j][3] = lo.w;
-                        xin[j][4] = hi.x; xin[j][5] = hi.y; xin[j][6] = hi.z; xin[j][7] = hi.w;
-                    } else {
-                        const uint4 r = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(a.in) + (size_t)tau * a.cols + c));
-                        const uint32_t rr[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            xin[j][2 * e] = __uint_as_float(rr[e] << 16);
-                            xin[j][2 * e + 1] = __uint_as_float(rr[e] & 0xFFFF0000u);
-                        }
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        float v = 0.f;
-                        if (tau < a.T && c + i < a.cols) {
-                            if (STAGE_A) v = reinterpret_cast<const float *>(a.in)[(size_t)tau * a.cols + c + i];
-                            else v = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(a.in)[(size_t)tau * a.cols + c + i]);
-                        }
-                        xin[j][i] = v;
-                    }
-                }
-            }
-        };
-        load_v(0);
-        load_x(0);
-
+    if (warp < 4) {
+        // ============================ sign-tile expanders ============================
+        const int arow = tid;                                     // one row of the tile per thread
+        const uint2 *wp = a.wk + (size_t)row0 + arow;             // + kb * rows_pad
+        uint2 w_next = __ldg(wp);
         bool alive = true;
         for (int kb = 0; kb < nkb && alive; ++kb) {
             const int s = kb % PF_STAGES;
             const uint32_t ph = (uint32_t)(kb / PF_STAGES) & 1u;
-            // consume the prefetched registers
-            const uint32_t aw = aw_next;
-            float vf[8][TPT];
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-#pragma unroll
-                for (int tt = 0; tt < TPT; ++tt) {
-                    const uint32_t pr = vraw[i][tt >> 1];
-                    vf[i][tt] = raw16_to_float((uint16_t)((tt & 1) ? (pr >> 16) : (pr & 0xFFFFu)), a.env_dtype);
-                }
-            float xf[TAUPT][8];
-#pragma unroll
-            for (int j = 0; j < TAUPT; ++j)
-#pragma unroll
-                for (int i = 0; i < 8; ++i) xf[j][i] = xin[j][i];
-            if (kb + 1 < nkb) { aw_next = load_word(kb + 1); load_v(kb + 1); load_x(kb + 1); }
-
+            const uint2 w = w_next;
+            if (kb + 1 < nkb) w_next = __ldg(wp + (size_t)(kb + 1) * a.rows_pad);
             alive = mbar_wait(empty_bar + 8 * s, ph ^ 1u, abort_flag, a.status);
             if (!alive) break;
-            unsigned char *sA = smem_gen + (size_t)s * PF_STAGE_BYTES;
-            unsigned char *sB = sA + PF_A_BYTES;
-            // A: 32 bits -> four 16-byte chunks of row `arow`
+            unsigned char *sA = smem_gen + (size_t)s * PF_STAGE_BYTES + arow * 128;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t byte = (aw >> (8 * j)) & 0xFFu;
-                const uint2 lo = lut[byte & 15u], hi = lut[byte >> 4];
-                const int c8 = ahalf * 4 + j;
-                *reinterpret_cast<uint4 *>(sA + arow * 128 + ((c8 ^ (arow & 7)) << 4)) = make_uint4(lo.x, lo.y, hi.x, hi.y);
-            }
-            // B: rows n = tau_local * LP + t, chunk kc
-#pragma unroll
-            for (int j = 0; j < TAUPT; ++j) {
-                const int taul = taug * TAUPT + j;
-#pragma unroll
-                for (int tt = 0; tt < TPT; ++tt) {
-                    const int n = taul * LP + t_first + tt;
-                    uint4 o;
-                    o.x = pf_pack_bf16x2(vf[0][tt] * xf[j][0], vf[1][tt] * xf[j][1]);
-                    o.y = pf_pack_bf16x2(vf[2][tt] * xf[j][2], vf[3][tt] * xf[j][3]);
-                    o.z = pf_pack_bf16x2(vf[4][tt] * xf[j][4], vf[5][tt] * xf[j][5]);
-                    o.w = pf_pack_bf16x2(vf[6][tt] * xf[j][6], vf[7][tt] * xf[j][7]);
-                    if (n < a.n_eff)
-                        *reinterpret_cast<uint4 *>(sB + n * 128 + ((kc ^ (n & 7)) << 4)) = o;
-                }
+            for (int c8 = 0; c8 < 8; ++c8) {                      // 8 columns -> one 16-byte chunk
+                const uint32_t byte = ((c8 < 4 ? w.x : w.y) >> (8 * (c8 & 3))) & 0xFFu;
+                *reinterpret_cast<uint4 *>(sA + ((c8 ^ (arow & 7)) << 4)) =
+                    make_uint4(sign_pair(byte, 0), sign_pair(byte, 1), sign_pair(byte, 2), sign_pair(byte, 3));
             }
             fence_proxy_async();
             mbar_arrive(full_bar + 8 * s);
         }
 
-        // ================================ epilogue =================================
-        // warp w reads TMEM lanes 32*(w & 3) .. +31 (= rows of the tile), columns 128*(w >> 2) .. +127
-        const int erow = (warp & 3) * 32 + lane;
-        const int egrow = row0 + erow;
-        const int chalf = warp >> 2;
-        float u[LP];
+        // ================================= epilogue ==================================
+        // thread = TMEM lane = row of the tile; columns n = tau_local * LP + t
+        const int egrow = row0 + arow;
+        float u[LP], vn[STAGE_A ? 1 : LP];
 #pragma unroll
-        for (int t = 0; t < LP; ++t)
-            u[t] = (egrow < a.rows && t < a.l) ? env_load(a.U, (size_t)egrow * a.l + t, a.env_dtype) : 0.f;
+        for (int t = 0; t < LP; ++t) {
+            const bool ok = egrow < a.rows && t < a.l;
+            u[t] = ok ? env_load(a.U, (size_t)egrow * a.l + t, a.env_dtype) : 0.f;
+            if (!STAGE_A) vn[t] = ok ? env_load(a.Vnext, (size_t)egrow * a.l + t, a.env_dtype) : 0.f;
+        }
         if (alive) alive = mbar_wait(accum_bar, 0u, abort_flag, a.status);
         tc_fence_after();
         if (alive) {
             float acc = 0.f;
+#pragma unroll 1
+            for (int ld = 0; ld < PF_BN / 32; ++ld) {
+                const int col0 = ld * 32;
+                if (col0 >= a.n_eff) break;                              // warp-uniform
+                uint32_t v[32];
+                tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)col0, v);
+                tmem_ld_wait();
 #pragma unroll
-            for (int ld = 0; ld < 4; ++ld) {
-                const int col0 = chalf * 128 + ld * 32;
-                if (col0 < a.n_eff) {                                   // warp-uniform
-                    uint32_t v[32];
-                    tmem_ld32(tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)col0, v);
-                    tmem_ld_wait();
+                for (int j = 0; j < 32; ++j) {
+                    const int t = j % LP;                // col0 is a multiple of 32 and LP divides 32
+                    acc += u[t] * __uint_as_float(v[j]);
+                    if (t == LP - 1) {
+                        const int tau = tau0 + (col0 + j) / LP;
+                        if (egrow < a.rows && tau < a.T) {
+                            if (STAGE_A) {
+                                a.y[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(acc);
+                            } else {
+                                a.z[(size_t)tau * a.rows + egrow] = acc;
+                                __nv_bfloat16 *xo = a.xs_next + (size_t)tau * LP * a.pad_next + egrow;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int n = col0 + j;
-                        const int t = n % LP;
-                        acc += u[t] * __uint_as_float(v[j]);
-                        if (t == LP - 1) {
-                            const int tau = tau0 + n / LP;
-                            if (egrow < a.rows && tau < a.T) {
-                                if (STAGE_A) reinterpret_cast<__nv_bfloat16 *>(a.out)[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(acc);
-                                else reinterpret_cast<float *>(a.out)[(size_t)tau * a.rows + egrow] = acc;
+                                for (int t2 = 0; t2 < LP; ++t2)
+                                    xo[(size_t)t2 * a.pad_next] = __float2bfloat16_rn(vn[t2] * acc);
                             }
-                            acc = 0.f;
                         }
+                        acc = 0.f;
                     }
                 }
             }
         }
+    } else if (warp == 4) {
+        // ================================ TMA issuer =================================
+        bool alive = true;
+        for (int kb = 0; kb < nkb && alive; ++kb) {
+            const int s = kb % PF_STAGES;
+            const uint32_t ph = (uint32_t)(kb / PF_STAGES) & 1u;
+            alive = mbar_wait(empty_bar + 8 * s, ph ^ 1u, abort_flag, a.status);
+            if (!alive) break;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(full_bar + 8 * s, PF_B_BYTES);
+                tma_load_2d(smem_base + (uint32_t)s * PF_STAGE_BYTES + PF_A_BYTES, &tmap_xs,
+                            kb * PF_BK, tau0 * LP, full_bar + 8 * s);
+            }
+            __syncwarp();
+        }
     } else {
-        // ================================ MMA issuer ===============================
+        // ================================ MMA issuer =================================
         const uint32_t idesc = make_idesc(a.n_eff);
         bool alive = true;
         for (int kb = 0; kb < nkb && alive; ++kb) {
@@ -385,34 +321,126 @@ __global__ void __launch_bounds__(PF_THREADS, 1) prefill_stage_kernel(const Pref
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 8) tmem_dealloc(tmem_d, PF_BN);
+    if (warp == 5) tmem_dealloc(tmem_d, PF_BN);
 }
 
-// private padded copy of V: [cols_pad][LP] raw 16-bit values of the stored envelope type
-__global__ void vpad_kernel(const void *__restrict__ V, int cols, int l, int env_dtype, uint16_t *__restrict__ out,
-                            int cols_pad, int LP) {
-    const size_t total = (size_t)cols_pad * LP;
-    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
-        const int c = (int)(idx / LP), t = (int)(idx % LP);
-        uint16_t r = 0;
-        if (c < cols && t < l) r = reinterpret_cast<const uint16_t *>(V)[(size_t)c * l + t];
-        out[idx] = r;
+// ------------------------------------------------------------------- pre-scale
+// Xs[(tau*LP + t) * pad + c] = bf16( Vt[t][c] * x[tau][c] ), zero for c >= cols.
+// One thread per (tau, 8 columns).
+template <int LP>
+__global__ void __launch_bounds__(256)
+prescale_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ Vt, __nv_bfloat16 *__restrict__ xs,
+                int T, int cols, int pad, int vec_ok) {
+    const int chunks = pad / 8;
+    const size_t total = (size_t)T * chunks;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const int tau = (int)(idx / chunks), c = (int)(idx % chunks) * 8;
+        float xv[8];
+        if (vec_ok && c + 8 <= cols) {
+            const uint4 r = __ldg(reinterpret_cast<const uint4 *>(x + (size_t)tau * cols + c));
+            const uint32_t rr[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                xv[2 * e] = __uint_as_float(rr[e] << 16);
+                xv[2 * e + 1] = __uint_as_float(rr[e] & 0xFFFF0000u);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) xv[i] = (c + i < cols) ? __bfloat162float(x[(size_t)tau * cols + c + i]) : 0.f;
+        }
+#pragma unroll
+        for (int t = 0; t < LP; ++t) {
+            const float4 v0 = __ldg(reinterpret_cast<const float4 *>(Vt + (size_t)t * pad + c));
+            const float4 v1 = __ldg(reinterpret_cast<const float4 *>(Vt + (size_t)t * pad + c + 4));
+            uint4 o;
+            o.x = pf_pack_bf16x2(v0.x * xv[0], v0.y * xv[1]);
+            o.y = pf_pack_bf16x2(v0.z * xv[2], v0.w * xv[3]);
+            o.z = pf_pack_bf16x2(v1.x * xv[4], v1.y * xv[5]);
+            o.w = pf_pack_bf16x2(v1.z * xv[6], v1.w * xv[7]);
+            *reinterpret_cast<uint4 *>(xs + ((size_t)tau * LP + t) * pad + c) = o;
+        }
     }
 }
 
-mdbf_status_t launch_vpad(const void *V, int cols, int l, int env_dtype, uint16_t *out, int cols_pad, int LP,
-                          cudaStream_t st) {
-    const size_t total = (size_t)cols_pad * LP;
-    int grid = (int)((total + 255) / 256);
-    if (grid > 148 * 16) grid = 148 * 16;
-    vpad_kernel<<<grid, 256, 0, st>>>(V, cols, l, env_dtype, out, cols_pad, LP);
+// --------------------------------------------------------- pack-time private copies
+// K-blocked sign words: out[kb * rows_pad + r] = words (2kb, 2kb+1) of row r, zero outside the matrix.
+__global__ void kblock_kernel(const uint32_t *__restrict__ canon, int rows, int nwords, uint2 *__restrict__ out,
+                              int rows_pad, int kblocks) {
+    const size_t total = (size_t)kblocks * rows_pad;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+        const int kb = (int)(idx / rows_pad), r = (int)(idx % rows_pad);
+        uint2 v = make_uint2(0u, 0u);
+        if (r < rows) {
+            if (2 * kb < nwords) v.x = canon[(size_t)r * nwords + 2 * kb];
+            if (2 * kb + 1 < nwords) v.y = canon[(size_t)r * nwords + 2 * kb + 1];
+        }
+        out[idx] = v;
+    }
+}
+// transposed fp32 copy of V: out[t * pad + c] = V[c][t], zero outside
+__global__ void vtrans_kernel(const void *__restrict__ V, int cols, int l, int env_dtype, float *__restrict__ out,
+                              int pad, int LP) {
+    const size_t total = (size_t)LP * pad;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+        const int t = (int)(idx / pad), c = (int)(idx % pad);
+        out[idx] = (c < cols && t < l) ? env_load(V, (size_t)c * l + t, env_dtype) : 0.f;
+    }
+}
+
+static int pf_grid(size_t items) {
+    size_t g = (items + 255) / 256;
+    if (g < 1) g = 1;
+    if (g > 148 * 32) g = 148 * 32;
+    return (int)g;
+}
+
+mdbf_status_t launch_kblock(const uint32_t *canon, int rows, int nwords, uint2 *out, int rows_pad, int kblocks,
+                            cudaStream_t st) {
+    kblock_kernel<<<pf_grid((size_t)kblocks * rows_pad), 256, 0, st>>>(canon, rows, nwords, out, rows_pad, kblocks);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}
+mdbf_status_t launch_vtrans(const void *V, int cols, int l, int env_dtype, float *out, int pad, int LP, cudaStream_t st) {
+    vtrans_kernel<<<pf_grid((size_t)LP * pad), 256, 0, st>>>(V, cols, l, env_dtype, out, pad, LP);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
 
+// Tensor map of a pre-scaled operand: bf16 [rows][pad] row-major, box 64 x 256, 128B swizzle.
+mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad) {
+    typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static encode_fn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        MDBF_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q));
+        if (!p || q != cudaDriverEntryPointSuccess) {
+            set_error("cuTensorMapEncodeTiled is not available from the driver");
+            return MDBF_ERR_CUDA;
+        }
+        fn = reinterpret_cast<encode_fn>(p);
+    }
+    const cuuint64_t gdim[2] = {(cuuint64_t)pad, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)pad * 2};
+    const cuuint32_t box[2] = {PF_BK, PF_BN};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return MDBF_ERR_CUDA;
+    }
+    return MDBF_OK;
+}
+
+// ---------------------------------------------------------------------- launch
 template <int LP, bool STAGE_A>
-static mdbf_status_t launch_pf(const PrefillArgs &a, cudaStream_t st) {
-    auto kern = prefill_stage_kernel<LP, STAGE_A>;
+static mdbf_status_t launch_gemm(const GemmArgs &a, const CUtensorMap &tm, cudaStream_t st) {
+    auto kern = gemm_stage_kernel<LP, STAGE_A>;
     static bool attr_set = false;
     if (!attr_set) {
         MDBF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
@@ -420,50 +448,57 @@ static mdbf_status_t launch_pf(const PrefillArgs &a, cudaStream_t st) {
     }
     const int TT = PF_BN / LP;
     dim3 grid(ceil_div(a.rows, PF_BM), ceil_div(a.T, TT));
-    kern<<<grid, PF_THREADS, PF_SMEM_BYTES, st>>>(a);
+    kern<<<grid, PF_THREADS, PF_SMEM_BYTES, st>>>(a, tm);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
 
-template <bool STAGE_A>
-static mdbf_status_t dispatch_pf(int LP, const PrefillArgs &a, cudaStream_t st) {
-    switch (LP) {
-        case 1: return launch_pf<1, STAGE_A>(a, st);
-        case 2: return launch_pf<2, STAGE_A>(a, st);
-        case 4: return launch_pf<4, STAGE_A>(a, st);
-        case 8: return launch_pf<8, STAGE_A>(a, st);
-        case 16: return launch_pf<16, STAGE_A>(a, st);
-        case 32: return launch_pf<32, STAGE_A>(a, st);
-        case 64: return launch_pf<64, STAGE_A>(a, st);
-    }
-    set_error("prefill stage: unsupported padded envelope rank %d", LP);
-    return MDBF_ERR_SHAPE;
-}
-
-mdbf_status_t launch_forward_prefill(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches) {
+template <int LP>
+static mdbf_status_t run_prefill(Layer &L, const void *x, void *y, int T, cudaStream_t st) {
     const mdbf_desc_t &d = L.d;
-    const int LP = L.LP;
     const int TT = PF_BN / LP;
     const int tok = T < TT ? T : TT;
     const int n_eff = ((tok * LP + 15) / 16) * 16;
-    PrefillArgs b = {};
-    b.words = L.wB; b.nwords = L.wordsB; b.rows = d.k; b.cols = d.d_in;
-    b.U = L.UB; b.Vp = L.vpB; b.env_dtype = d.env_dtype; b.l = d.l;
-    b.in = x; b.out = L.zsum; b.T = T; b.n_eff = n_eff;
-    b.vec_ok = ((reinterpret_cast<uintptr_t>(x) & 15u) == 0 && d.d_in % 8 == 0) ? 1 : 0;
-    b.status = L.status;
-    mdbf_status_t rc = dispatch_pf<false>(LP, b, st);
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(x) & 15u) == 0 && d.d_in % 8 == 0) ? 1 : 0;
+    prescale_kernel<LP><<<pf_grid((size_t)T * (L.padB / 8)), 256, 0, st>>>(
+        reinterpret_cast<const __nv_bfloat16 *>(x), L.vtB, L.xsB, T, d.d_in, L.padB, vec_ok);
+    MDBF_CUDA(cudaGetLastError());
+
+    GemmArgs b = {};
+    b.wk = L.wkB; b.rows_pad = L.rpB; b.rows = d.k; b.cols = d.d_in;
+    b.U = L.UB; b.env_dtype = d.env_dtype; b.l = d.l; b.T = T; b.n_eff = n_eff;
+    b.z = L.zsum; b.Vnext = L.VA; b.xs_next = L.xsA; b.pad_next = L.padA; b.status = L.status;
+    mdbf_status_t rc = launch_gemm<LP, false>(b, L.tmB, st);
     if (rc) return rc;
-    PrefillArgs a = {};
-    a.words = L.wA; a.nwords = L.wordsA; a.rows = d.d_out; a.cols = d.k;
-    a.U = L.UA; a.Vp = L.vpA; a.env_dtype = d.env_dtype; a.l = d.l;
-    a.in = L.zsum; a.out = y; a.T = T; a.n_eff = n_eff;
-    a.vec_ok = (d.k % 8 == 0) ? 1 : 0;
-    a.status = L.status;
-    rc = dispatch_pf<true>(LP, a, st);
+
+    GemmArgs a = {};
+    a.wk = L.wkA; a.rows_pad = L.rpA; a.rows = d.d_out; a.cols = d.k;
+    a.U = L.UA; a.env_dtype = d.env_dtype; a.l = d.l; a.T = T; a.n_eff = n_eff;
+    a.y = reinterpret_cast<__nv_bfloat16 *>(y); a.status = L.status;
+    return launch_gemm<LP, true>(a, L.tmA, st);
+}
+
+mdbf_status_t launch_forward_prefill(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches) {
+    if (!L.xsB) {
+        set_error("mdbf_linear_forward: this layer was packed with max_T <= %d and holds no large-T scratch",
+                  kDecodeMaxT);
+        return MDBF_ERR_SHAPE;
+    }
+    mdbf_status_t rc;
+    switch (L.LP) {
+        case 1: rc = run_prefill<1>(L, x, y, T, st); break;
+        case 2: rc = run_prefill<2>(L, x, y, T, st); break;
+        case 4: rc = run_prefill<4>(L, x, y, T, st); break;
+        case 8: rc = run_prefill<8>(L, x, y, T, st); break;
+        case 16: rc = run_prefill<16>(L, x, y, T, st); break;
+        case 32: rc = run_prefill<32>(L, x, y, T, st); break;
+        default:
+            set_error("mdbf_linear_forward: the large-T kernel handles l <= 32 (got %d)", L.d.l);
+            return MDBF_ERR_SHAPE;
+    }
     if (rc) return rc;
     L.last_ksplit = 0;
-    *launches = 2;
+    *launches = 3;
     return MDBF_OK;
 }
 

@@ -58,7 +58,7 @@ static mdbf_status_t check_handle(mdbf_handle_t h, const char *fn) {
 }
 
 static void free_layer(Layer &L) {
-    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.vpA, L.vpB, L.z, L.zsum, L.xstage, L.ystage, L.status};
+    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.wkA, L.wkB, L.vtB, L.xsB, L.xsA, L.z, L.zsum, L.xstage, L.ystage, L.status};
     for (void *p : ptrs)
         if (p) cudaFree(p);
 }
@@ -173,10 +173,21 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     PACK_CUDA(cudaMalloc(&L.vfB, (size_t)L.ktB * 8 * L.NT * 256));
     L.LP = 1;
     while (L.LP < d.l) L.LP *= 2;
-    const int padA = ceil_div(d.k, 64) * 64, padB = ceil_div(d.d_in, 64) * 64;
-    if (d.env_dtype != MDBF_F32) {      // the tensor-core kernels take 16-bit envelopes only
-        PACK_CUDA(cudaMalloc(&L.vpA, (size_t)padA * L.LP * 2));
-        PACK_CUDA(cudaMalloc(&L.vpB, (size_t)padB * L.LP * 2));
+    L.padA = ceil_div(d.k, 64) * 64; L.padB = ceil_div(d.d_in, 64) * 64;
+    L.rpA = ceil_div(d.d_out, 128) * 128; L.rpB = ceil_div(d.k, 128) * 128;
+    // the large-T kernel takes 16-bit envelopes and l <= 32; its scratch is sized by max_T
+    const bool want_prefill = d.env_dtype != MDBF_F32 && d.l <= 32 && d.max_T > kDecodeMaxT;
+    if (want_prefill) {
+        L.xs_rows = ((size_t)d.max_T * L.LP + 255) / 256 * 256;
+        PACK_CUDA(cudaMalloc(&L.wkA, (size_t)(L.padA / 64) * L.rpA * sizeof(uint2)));
+        PACK_CUDA(cudaMalloc(&L.wkB, (size_t)(L.padB / 64) * L.rpB * sizeof(uint2)));
+        PACK_CUDA(cudaMalloc(&L.vtB, (size_t)L.LP * L.padB * sizeof(float)));
+        PACK_CUDA(cudaMalloc(&L.xsB, L.xs_rows * L.padB * 2));
+        PACK_CUDA(cudaMalloc(&L.xsA, L.xs_rows * L.padA * 2));
+        PACK_CUDA(cudaMemsetAsync(L.xsB, 0, L.xs_rows * L.padB * 2, st));
+        PACK_CUDA(cudaMemsetAsync(L.xsA, 0, L.xs_rows * L.padA * 2, st));
+        PACK_RC(make_xs_tensor_map(&L.tmB, L.xsB, L.xs_rows, L.padB));
+        PACK_RC(make_xs_tensor_map(&L.tmA, L.xsA, L.xs_rows, L.padA));
     }
     L.zstride = (size_t)decode_scratch_T(d) * d.k;
     PACK_CUDA(cudaMalloc(&L.z, (size_t)kMaxKSplit * L.zstride * sizeof(float)));
@@ -209,9 +220,10 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     PACK_RC(launch_env_round((const float *)dsrc[5], L.VB, nVB, d.env_dtype, st));
     PACK_RC(launch_vfrag(L.VA, d.k, d.l, d.env_dtype, L.vfA, L.ktA, L.NT, st));
     PACK_RC(launch_vfrag(L.VB, d.d_in, d.l, d.env_dtype, L.vfB, L.ktB, L.NT, st));
-    if (d.env_dtype != MDBF_F32) {
-        PACK_RC(launch_vpad(L.VA, d.k, d.l, d.env_dtype, L.vpA, padA, L.LP, st));
-        PACK_RC(launch_vpad(L.VB, d.d_in, d.l, d.env_dtype, L.vpB, padB, L.LP, st));
+    if (want_prefill) {
+        PACK_RC(launch_kblock(L.wA, d.d_out, L.wordsA, L.wkA, L.rpA, L.padA / 64, st));
+        PACK_RC(launch_kblock(L.wB, d.k, L.wordsB, L.wkB, L.rpB, L.padB / 64, st));
+        PACK_RC(launch_vtrans(L.VB, d.d_in, d.l, d.env_dtype, L.vtB, L.padB, L.LP, st));
     }
     PACK_CUDA(cudaStreamSynchronize(st));
     for (void *p : temps) cudaFree(p);
@@ -292,14 +304,14 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
     }
     if (!valid_dtype(act_dtype)) { set_error("mdbf_linear_forward: bad act_dtype %d", act_dtype); return MDBF_ERR_DTYPE; }
     int kernel = h->kernel;
-    const bool tc_ok = (act_dtype == MDBF_BF16) && (L.d.env_dtype != MDBF_F32);
+    const bool tc_ok = (act_dtype == MDBF_BF16) && (L.d.env_dtype != MDBF_F32) && L.d.l <= 32;
     if (kernel == MDBF_KERNEL_AUTO) {
         if (!tc_ok) kernel = MDBF_KERNEL_ALU;
-        else if (T <= kDecodeMaxT && L.d.l <= 32) kernel = MDBF_KERNEL_DECODE;
+        else if (T <= kDecodeMaxT) kernel = MDBF_KERNEL_DECODE;
         else kernel = MDBF_KERNEL_PREFILL;
     }
     if (kernel != MDBF_KERNEL_ALU && !tc_ok) {
-        set_error("mdbf_linear_forward: the tensor-core kernels need bf16 activations and 16-bit envelopes");
+        set_error("mdbf_linear_forward: the tensor-core kernels need bf16 activations, 16-bit envelopes and l <= 32");
         return MDBF_ERR_DTYPE;
     }
     if (kernel == MDBF_KERNEL_DECODE && (T > kDecodeMaxT || L.d.l > 32)) {

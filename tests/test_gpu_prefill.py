@@ -23,7 +23,7 @@ def spec_of(d_out, d_in, k, l, **kw):
 
 
 @pytest.mark.parametrize("l,T", [(16, 16), (16, 48), (16, 5), (4, 64), (4, 100), (1, 256), (1, 300),
-                                 (3, 40), (8, 33), (20, 9), (64, 7)])
+                                 (3, 40), (8, 33), (20, 9), (32, 11)])
 def test_prefill_kernel_small_shapes(l, T):
     spec = spec_of(384, 576, 256, l)
     x = inputs.make_activations(spec, T)
@@ -65,3 +65,13 @@ def test_prefill_agrees_with_small_T_kernel_and_auto_dispatch():
         y_auto = g.forward(x64)                       # T = 64 -> large-T kernel
         assert rel_err(y_auto, g.oracle_forward(x64)) <= TOL["bf16"]
         np.testing.assert_array_equal(y_auto, g.forward(x64, kernel=M.KERNEL_PREFILL))
+
+
+def test_envelope_rank_above_32_takes_the_fp32_path():
+    spec = spec_of(96, 160, 64, 40)
+    x = inputs.make_activations(spec, 6)
+    with GpuLayer(spec, 6) as g:
+        assert rel_err(g.forward(x), g.oracle_forward(x)) <= TOL["bf16"]       # AUTO -> ALU kernel
+        with pytest.raises(M.MdbfError) as e:
+            g.forward(x, kernel=M.KERNEL_PREFILL)
+        assert e.value.status == M.ERR_DTYPE
