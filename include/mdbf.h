@@ -147,6 +147,48 @@ mdbf_status_t mdbf_linear_forward(mdbf_handle_t h, const void *x, void *y, int32
 mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T,
                                        int32_t act_dtype, void *stream);
 
+/* ------------------------------------------------- forward without allocation
+ * (The paper has no counterpart: this entry point exists for deployment, not
+ * for the method.)
+ *
+ * Some callers may not allocate device memory: a serving runtime that has
+ * given every byte to its own arena and forbids cudaMalloc from then on, a
+ * plug-in that only ever receives buffers from its host application, a
+ * real-time loop that cannot afford the device-wide synchronisation an
+ * allocation implies.  They cannot use mdbf_pack, which allocates the handle's
+ * buffers.  This call computes the same y = W_hat x from buffers the caller
+ * already owns and needs no handle:
+ *
+ *   desc       shape and env_dtype of the layer (max_T is ignored)
+ *   wA, wB     device; canonical packed words of S_A (d_out x ceil(k/32)) and
+ *              S_B (k x ceil(d_in/32)), as mdbf_pack_signs writes them
+ *   U_A..V_B   device; envelope factors stored in desc->env_dtype, row-major
+ *              d_out x l, k x l, k x l, d_in x l
+ *   x, y       device; T x d_in read, T x d_out written, of act_dtype
+ *              (MDBF_F32, MDBF_F16 or MDBF_BF16); fp32 accumulation
+ *
+ * The k x T intermediate between the two stages is kept in a fixed array
+ * inside the library image (MDBF_STATIC_MAX_KT floats = 1 MiB, resident on
+ * every GPU that loads the library until the process exits); a call with
+ * k * T above that limit returns MDBF_ERR_SHAPE.  The call runs the fp32
+ * CUDA-core kernels (sign applied by XOR of the IEEE sign bit), asynchronously
+ * on `stream`, and calls neither cudaMalloc nor cudaFree nor any allocating
+ * library routine.
+ *
+ * The first call on each device looks the array's device address up (with
+ * that device current); make that first call outside any stream capture.
+ * Every call on a device shares the one array, which keeps whatever the
+ * previous call left in it: each call overwrites all the entries it later
+ * reads, so nothing has to be cleared, but two calls that overlap on the GPU
+ * (different streams, no dependency between them) race on it and both may
+ * return wrong results.  Serialise them.
+ * Errors: INVALID_ARG (NULL), SHAPE, DTYPE, ARCH, CUDA. */
+#define MDBF_STATIC_MAX_KT 262144
+mdbf_status_t mdbf_linear_forward_static(const mdbf_desc_t *desc, const uint32_t *wA, const uint32_t *wB,
+                                         const void *U_A, const void *V_A, const void *U_B,
+                                         const void *V_B, const void *x, void *y, int32_t T,
+                                         int32_t act_dtype, void *stream);
+
 /* The k x T intermediate z of the last forward on this handle (after the
  * stage with S_B), as float32 token-contiguous T x k, for tests that localise
  * a disagreement to one stage.  Synchronises `stream`. */

@@ -28,6 +28,7 @@ DTYPES = {"f32": F32, "f16": F16, "bf16": BF16}
 EXPORTS = (
     "mdbf_pack_signs", "mdbf_unpack_signs", "mdbf_pack", "mdbf_get_packed", "mdbf_get_envelope",
     "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host",
+    "mdbf_linear_forward_static",
     "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_poll_status", "mdbf_last_launch_count",
     "mdbf_destroy", "mdbf_last_error", "mdbf_version",
 )
@@ -68,6 +69,7 @@ def lib() -> ctypes.CDLL:
     L.mdbf_set_kernel.argtypes = [vp, i32]
     L.mdbf_linear_forward.argtypes = [vp, vp, vp, i32, i32, vp]
     L.mdbf_linear_forward_host.argtypes = [vp, vp, vp, i32, i32, vp]
+    L.mdbf_linear_forward_static.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, vp]
     L.mdbf_get_intermediate.argtypes = [vp, vp, i32, ctypes.c_int, vp]
     L.mdbf_reconstruct.argtypes = [vp, vp, vp]
     L.mdbf_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
@@ -149,6 +151,20 @@ def mdbf_linear_forward(h: int, x, y, T: int, act_dtype: int, stream: int = 0) -
 
 def mdbf_linear_forward_host(h: int, x_host, y_host, T: int, act_dtype: int, stream: int = 0) -> None:
     _check(lib().mdbf_linear_forward_host(h, _addr(x_host), _addr(y_host), T, act_dtype, stream))
+
+
+STATIC_MAX_KT = 262144
+
+
+def mdbf_linear_forward_static(d_out: int, d_in: int, k: int, l: int, env_dtype: int, wA, wB, U_A, V_A, U_B, V_B,
+                               x, y, T: int, act_dtype: int, stream: int = 0) -> None:
+    """Forward for callers that may not allocate device memory: no handle, every buffer (packed
+    words, envelopes stored in env_dtype, x, y) is a device address the caller owns; the k x T
+    intermediate sits in a fixed array inside the library (k * T <= STATIC_MAX_KT).  Calls on one
+    device share that array and must not overlap; make the first call outside stream capture."""
+    desc = Desc(d_out, d_in, k, l, env_dtype, T)
+    _check(lib().mdbf_linear_forward_static(ctypes.byref(desc), _addr(wA), _addr(wB), _addr(U_A), _addr(V_A),
+                                            _addr(U_B), _addr(V_B), _addr(x), _addr(y), T, act_dtype, stream))
 
 
 def mdbf_get_intermediate(h: int, z, T: int, out_on_device: bool = False, stream: int = 0) -> None:
