@@ -155,7 +155,7 @@ def dist_setup(n_gpus):
 # ------------------------------------------------------------------ mdbf arm
 def run_mdbf(args):
     import torch
-    from paper_2512_24545_b200 import build, inputs, mdbf as M
+    from paper_2512_24545_b200 import build, inputs, mdbf as M, replicas
     build.build()
     dist, rank, world, local = dist_setup(args.gpus)
     torch.cuda.set_device(local)
@@ -246,10 +246,7 @@ def run_mdbf(args):
     h2d = sum(T * sp.d_in * 2 for (_, sp, *_r) in layers)
     d2h = sum(T * sp.d_out * 2 for (_, sp, *_r) in layers)
 
-    ms_t = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device="cuda")
-    if dist:
-        dist.all_reduce(ms_t, op=dist.ReduceOp.MAX)
-    ms_max, e2e_ms_max = float(ms_t[0]), float(ms_t[1])
+    ms_max, e2e_ms_max = replicas.max_over_ranks([ms, e2e_s * 1e3], dist, device="cuda")
     sec = ms_max / 1e3
     if bound == "hbm":
         metric, unit = "decode_algorithmic_GBps", "GB/s"
@@ -259,9 +256,9 @@ def run_mdbf(args):
         metric, unit = "prefill_expanded_TFLOPs", "TFLOP/s"
         per_step = total_flops / 1e12
         peak = peaks["bf16_tflops"] if sec < 1.0 else peaks["bf16_tflops_sustained"]
-    value = world * per_step * args.steps / sec
+    value = replicas.aggregate_throughput(per_step * args.steps, world, sec)
     per_gpu = per_step * args.steps / sec
-    e2e_value = world * per_step * e2e_steps / (e2e_ms_max / 1e3)
+    e2e_value = replicas.aggregate_throughput(per_step * e2e_steps, world, e2e_ms_max / 1e3)
 
     out = {
         "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
