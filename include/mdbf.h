@@ -63,7 +63,8 @@ typedef enum {
     MDBF_KERNEL_AUTO = 0,   /* choose by (l, T, dtypes)                                         */
     MDBF_KERNEL_ALU = 1,    /* fp32 CUDA-core path, sign applied by XOR of the IEEE sign bit      */
     MDBF_KERNEL_DECODE = 2, /* small-T path: register bit->bf16 expansion + warp-level MMA        */
-    MDBF_KERNEL_PREFILL = 3 /* large-T path: tcgen05 MMA with TMEM accumulators                   */
+    MDBF_KERNEL_PREFILL = 3, /* large-T path: tcgen05 MMA with TMEM accumulators                  */
+    MDBF_KERNEL_TMEM = 4    /* small-T path: tcgen05 MMA, sign operand expanded into TMEM         */
 } mdbf_kernel_t;
 
 typedef struct {

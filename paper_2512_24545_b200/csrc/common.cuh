@@ -41,9 +41,11 @@ struct Layer {
     // kernel-private bf16 copies of V_A / V_B in MMA B-fragment order (see forward_decode.cu)
     uint2 *vfA, *vfB;
     int NT;                       // 8-column mode tiles in the fragment copies: 1, 2, 4 or 8
+    // TMEM-operand small-T kernel (16-bit envelopes, l <= 32): V in MMA k order, 16-bit, [kblocks][LP][64]
+    uint16_t *vpA, *vpB;
     // large-T kernel (present only when max_T exceeds the small-T kernel's range and l <= 32):
     int LP;                       // l rounded up to a power of two
-    uint2 *wkA, *wkB;             // K-blocked sign words [kblocks][rows_pad128]
+    uint2 *wkA, *wkB;             // K-blocked sign words [kblocks][rows_pad128] (tcgen05 kernels)
     int rpA, rpB;                 // rows padded to 128
     int padA, padB;               // reduction length (k, d_in) padded to 64
     float *vtB;                   // V_B transposed, fp32 [LP][padB]
@@ -109,6 +111,10 @@ mdbf_status_t launch_forward_decode(Layer &L, const void *x, void *y, int T, cud
                                     int *launches);
 mdbf_status_t launch_forward_prefill(Layer &L, const void *x, void *y, int T, cudaStream_t st,
                                      int *launches);
+mdbf_status_t launch_forward_tmem(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches);
+bool tmem_path_supports(const Layer &L, int T);
+mdbf_status_t launch_vperm(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int LP,
+                           cudaStream_t st);
 mdbf_status_t launch_zsum(Layer &L, int T, cudaStream_t st);
 
 // host-side canonical packer (pack.cu)

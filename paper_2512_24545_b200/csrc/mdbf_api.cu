@@ -58,7 +58,7 @@ static mdbf_status_t check_handle(mdbf_handle_t h, const char *fn) {
 }
 
 static void free_layer(Layer &L) {
-    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.wkA, L.wkB, L.vtB, L.xsB, L.xsA, L.z, L.zsum, L.xstage, L.ystage, L.status};
+    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.vpA, L.vpB, L.wkA, L.wkB, L.vtB, L.xsB, L.xsA, L.z, L.zsum, L.xstage, L.ystage, L.status};
     for (void *p : ptrs)
         if (p) cudaFree(p);
 }
@@ -177,10 +177,15 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     L.rpA = ceil_div(d.d_out, 128) * 128; L.rpB = ceil_div(d.k, 128) * 128;
     // the large-T kernel takes 16-bit envelopes and l <= 32; its scratch is sized by max_T
     const bool want_prefill = d.env_dtype != MDBF_F32 && d.l <= 32 && d.max_T > kDecodeMaxT;
-    if (want_prefill) {
-        L.xs_rows = ((size_t)d.max_T * L.LP + 255) / 256 * 256;
+    const bool want_tc = d.env_dtype != MDBF_F32 && d.l <= 32;
+    if (want_tc) {
         PACK_CUDA(cudaMalloc(&L.wkA, (size_t)(L.padA / 64) * L.rpA * sizeof(uint2)));
         PACK_CUDA(cudaMalloc(&L.wkB, (size_t)(L.padB / 64) * L.rpB * sizeof(uint2)));
+        PACK_CUDA(cudaMalloc(&L.vpA, (size_t)(L.padA / 64) * L.LP * 64 * sizeof(uint16_t)));
+        PACK_CUDA(cudaMalloc(&L.vpB, (size_t)(L.padB / 64) * L.LP * 64 * sizeof(uint16_t)));
+    }
+    if (want_prefill) {
+        L.xs_rows = ((size_t)d.max_T * L.LP + 255) / 256 * 256;
         PACK_CUDA(cudaMalloc(&L.vtB, (size_t)L.LP * L.padB * sizeof(float)));
         PACK_CUDA(cudaMalloc(&L.xsB, L.xs_rows * L.padB * 2));
         PACK_CUDA(cudaMalloc(&L.xsA, L.xs_rows * L.padA * 2));
@@ -220,9 +225,13 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     PACK_RC(launch_env_round((const float *)dsrc[5], L.VB, nVB, d.env_dtype, st));
     PACK_RC(launch_vfrag(L.VA, d.k, d.l, d.env_dtype, L.vfA, L.ktA, L.NT, st));
     PACK_RC(launch_vfrag(L.VB, d.d_in, d.l, d.env_dtype, L.vfB, L.ktB, L.NT, st));
-    if (want_prefill) {
+    if (want_tc) {
         PACK_RC(launch_kblock(L.wA, d.d_out, L.wordsA, L.wkA, L.rpA, L.padA / 64, st));
         PACK_RC(launch_kblock(L.wB, d.k, L.wordsB, L.wkB, L.rpB, L.padB / 64, st));
+        PACK_RC(launch_vperm(L.VA, d.k, d.l, d.env_dtype, L.vpA, L.padA / 64, L.LP, st));
+        PACK_RC(launch_vperm(L.VB, d.d_in, d.l, d.env_dtype, L.vpB, L.padB / 64, L.LP, st));
+    }
+    if (want_prefill) {
         PACK_RC(launch_vtrans(L.VB, d.d_in, d.l, d.env_dtype, L.vtB, L.padB, L.LP, st));
     }
     PACK_CUDA(cudaStreamSynchronize(st));
@@ -287,7 +296,7 @@ mdbf_status_t mdbf_get_desc(mdbf_handle_t h, mdbf_desc_t *out) {
 mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel) {
     mdbf_status_t rc = check_handle(h, "mdbf_set_kernel");
     if (rc) return rc;
-    if (kernel < MDBF_KERNEL_AUTO || kernel > MDBF_KERNEL_PREFILL) {
+    if (kernel < MDBF_KERNEL_AUTO || kernel > MDBF_KERNEL_TMEM) {
         set_error("mdbf_set_kernel: unknown kernel %d", kernel);
         return MDBF_ERR_INVALID_ARG;
     }
@@ -307,6 +316,7 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
     const bool tc_ok = (act_dtype == MDBF_BF16) && (L.d.env_dtype != MDBF_F32) && L.d.l <= 32;
     if (kernel == MDBF_KERNEL_AUTO) {
         if (!tc_ok) kernel = MDBF_KERNEL_ALU;
+        else if (tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
         else if (T <= kDecodeMaxT) kernel = MDBF_KERNEL_DECODE;
         else kernel = MDBF_KERNEL_PREFILL;
     }
@@ -323,6 +333,7 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
     mdbf_status_t rc;
     if (kernel == MDBF_KERNEL_ALU) rc = launch_forward_alu(L, x, y, T, act_dtype, st, &launches);
     else if (kernel == MDBF_KERNEL_DECODE) rc = launch_forward_decode(L, x, y, T, st, &launches);
+    else if (kernel == MDBF_KERNEL_TMEM) rc = launch_forward_tmem(L, x, y, T, st, &launches);
     else rc = launch_forward_prefill(L, x, y, T, st, &launches);
     if (rc == MDBF_OK) h->last_launches = launches;
     return rc;
