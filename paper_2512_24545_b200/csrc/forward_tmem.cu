@@ -13,10 +13,11 @@
 // must not be re-read from shared memory for every instruction (4 KB per MMA), and one thread
 // cannot issue MMAs faster than one per ~50 clocks.  Hence:
 //
-//   * A lives in TMEM.  Four "expander" warps (thread = sign row = TMEM lane) read 64 packed bits
-//     per row and K block, turn every bit into a +-1.0 bf16 with one shift and one logic op per two
-//     bits, and write 32 TMEM columns with tcgen05.st.  Nothing of the expanded operand touches
-//     shared memory.
+//   * A lives in TMEM.  Eight "expander" warps (thread = sign row = TMEM lane; warps w and w + 4
+//     share a lane quadrant and take the even and the odd K blocks) read 64 packed bits per row and
+//     K block, turn every bit into a +-1.0 bf16 with one shift and one logic op per two bits, and
+//     write 32 TMEM columns with tcgen05.st; the store of one block overlaps the expansion of the
+//     next.  Nothing of the expanded operand touches shared memory.
 //   * Four issuer warps take the K blocks round-robin, each with its own fp32 accumulator in TMEM
 //     (summed in the epilogue), so four MMAs are in flight at any time.  The same warps build
 //     their B tiles (64 K x N, 128B-swizzled, K-major) in shared memory from the staged
@@ -44,12 +45,13 @@ namespace cg = cooperative_groups;
 
 namespace mdbf {
 
-constexpr int TM_EXPANDERS = 128;
+constexpr int TM_EXPANDERS = 256;                      // two groups of 4 warps: even / odd K blocks
 constexpr int TM_ISSUERS = 4;                          // issuer/producer warps, one accumulator each
 constexpr int TM_THREADS = TM_EXPANDERS + TM_ISSUERS * 32 + 64;   // + sign loader warp + V loader warp
+constexpr int TM_W_ISSUER0 = TM_EXPANDERS / 32;        // first issuer warp
 constexpr int TM_VSTAGES = 8;                          // V ring (two per issuer warp)
 constexpr int TM_MAX_SSTAGES = 32;                     // sign ring, 1 KB per stage
-constexpr int TM_MAX_ASTAGES = 8;                      // A stages in TMEM, 32 columns each
+constexpr int TM_MAX_ASTAGES = 8;                      // A stages in TMEM, 32 columns each (6 when TMEM is shared)
 constexpr int TM_MAX_N = 64;
 constexpr int TM_MAX_T = 16;
 constexpr uint32_t TM_MAX_POLLS = 1u << 21;
@@ -238,16 +240,19 @@ __global__ void __launch_bounds__(TM_THREADS, 1) tmem_stage_kernel(const TmArgs 
     const int nkb = max(0, min(a.kb_per_cta, a.nkb_total - kb0));
     const int nas = a.nastages, nss = a.nsstages;
 
-    if (tid == 0) {
-        for (int s = 0; s < TM_MAX_SSTAGES; ++s) { mbar_init(s_full + 8 * s, 1); mbar_init(s_empty + 8 * s, 4); }
-        for (int s = 0; s < TM_VSTAGES; ++s) { mbar_init(v_full + 8 * s, 1); mbar_init(v_empty + 8 * s, 1); }
-        for (int s = 0; s < TM_MAX_ASTAGES; ++s) { mbar_init(a_full + 8 * s, 4); mbar_init(a_empty + 8 * s, 1); }
-        for (int s = 0; s < 2 * TM_ISSUERS; ++s) mbar_init(b_empty + 8 * s, 1);
-        mbar_init(acc_bar, TM_ISSUERS);
-        abort_flag_s = 0;
+    {   // one barrier per thread: s_full, s_empty, v_full, v_empty, a_full, a_empty, b_empty, acc_bar
+        constexpr int NB0 = TM_MAX_SSTAGES, NB1 = 2 * TM_MAX_SSTAGES, NB2 = NB1 + TM_VSTAGES, NB3 = NB2 + TM_VSTAGES,
+                      NB4 = NB3 + TM_MAX_ASTAGES, NB5 = NB4 + TM_MAX_ASTAGES, NB6 = NB5 + 2 * TM_ISSUERS;
+        static_assert(NB6 + 1 <= TM_THREADS, "one thread per barrier");
+        if (tid <= NB6) {
+            const uint32_t count = tid < NB0 ? 1u : tid < NB1 ? 4u : tid < NB3 ? 1u : tid < NB4 ? 4u : tid < NB6 ? 1u
+                                                                                                          : (uint32_t)TM_ISSUERS;
+            mbar_init(smem_u32(&bars[tid]), count);
+        }
+        if (tid == 0) abort_flag_s = 0;
         fence_barrier_init();
     }
-    if (warp == 4) {
+    if (warp == TM_W_ISSUER0) {
         tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)a.tmem_cols);
         tmem_relinquish();
     }
@@ -263,37 +268,51 @@ __global__ void __launch_bounds__(TM_THREADS, 1) tmem_stage_kernel(const TmArgs 
 #pragma unroll
     for (int i = 0; i < MAXTOK; ++i) outv[i] = 0.f;
 
-    if (warp < 4) {
+    const int row_l = (warp & 3) * 32 + lane;               // row of the tile = TMEM lane (expander warps)
+    if (warp < TM_W_ISSUER0) {
         // ============================ expanders, then epilogue ============================
-        const int grow = row0 + tid;
+        const int grp = warp >> 2;                           // 0: even K blocks (and the epilogue), 1: odd
+        const int grow = row0 + row_l;
         float u[LP];
 #pragma unroll
         for (int t = 0; t < LP; ++t)
-            u[t] = (grow < a.rows && t < a.l) ? env_load(a.U, (size_t)grow * a.l + t, a.env_dtype) : 0.f;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+            u[t] = (grp == 0 && grow < a.rows && t < a.l) ? env_load(a.U, (size_t)grow * a.l + t, a.env_dtype) : 0.f;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         bool alive = true;
-        for (int kb = 0; kb < nkb && alive; ++kb) {
-            const int rs = kb % nss, as = kb % nas;
-            alive = mbar_wait(s_full + 8 * rs, (uint32_t)(kb / nss) & 1u, abort_flag, a.status);
+        int rs = grp % nss, as = grp % nas;
+        uint32_t rs_ph = 0, as_ph = 0;
+        int prev_as = -1;
+        for (int kb = grp; kb < nkb && alive; kb += 2) {
+            alive = mbar_wait(s_full + 8 * rs, rs_ph, abort_flag, a.status);
             if (!alive) break;
-            const uint2 w = *reinterpret_cast<const uint2 *>(smem_gen + off_s + rs * 1024 + tid * 8);
+            const uint2 w = *reinterpret_cast<const uint2 *>(smem_gen + off_s + rs * 1024 + row_l * 8);
             __syncwarp();
             if (lane == 0) mbar_arrive(s_empty + 8 * rs);
-            alive = mbar_wait(a_empty + 8 * as, ((uint32_t)(kb / nas) & 1u) ^ 1u, abort_flag, a.status);
-            if (!alive) break;
-            tc_fence_after();
             uint32_t v[32];
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 v[i] = ((w.x << (15 - i)) & 0x80008000u) | 0x3F803F80u;
                 v[16 + i] = ((w.y << (15 - i)) & 0x80008000u) | 0x3F803F80u;
             }
+            if (prev_as >= 0) {                              // the previous block's store had this long to land
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(a_full + 8 * prev_as);
+            }
+            alive = mbar_wait(a_empty + 8 * as, as_ph ^ 1u, abort_flag, a.status);
+            if (!alive) break;
+            tc_fence_after();
             tmem_st32(tmem_a0 + lane_base + (uint32_t)(as * 32), v);
-            tmem_st_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(a_full + 8 * as);
+            prev_as = as;
+            rs += 2; if (rs >= nss) { rs -= nss; rs_ph ^= 1u; }
+            as += 2; if (as >= nas) { as -= nas; as_ph ^= 1u; }
         }
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (alive && prev_as >= 0 && lane == 0) mbar_arrive(a_full + 8 * prev_as);
+        if (grp != 0) alive = false;                         // the odd group has no part in the epilogue
         if (alive) alive = mbar_wait(acc_bar, 0u, abort_flag, a.status);
         tc_fence_after();
         if (alive) {
@@ -302,14 +321,17 @@ __global__ void __launch_bounds__(TM_THREADS, 1) tmem_stage_kernel(const TmArgs 
             for (int cc = 0; cc < TM_MAX_N / 16; ++cc) {
                 if (cc * 16 < a.n_mma) {                                   // warp-uniform
                     float sum[16];
+                    uint32_t d[TM_ISSUERS][16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) sum[j] = 0.f;
-                    for (int acc = 0; acc < nacc; ++acc) {
-                        uint32_t d[16];
-                        tmem_ld16(tmem + lane_base + (uint32_t)(acc * a.n_mma + cc * 16), d);
-                        tmem_ld_wait();
+                    for (int acc = 0; acc < TM_ISSUERS; ++acc)
+                        if (acc < nacc) tmem_ld16(tmem + lane_base + (uint32_t)(acc * a.n_mma + cc * 16), d[acc]);
+                    tmem_ld_wait();
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) sum[j] += __uint_as_float(d[j]);
+                    for (int j = 0; j < 16; ++j) {
+                        sum[j] = 0.f;
+#pragma unroll
+                        for (int acc = 0; acc < TM_ISSUERS; ++acc)
+                            if (acc < nacc) sum[j] += __uint_as_float(d[acc][j]);
                     }
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
@@ -319,30 +341,52 @@ __global__ void __launch_bounds__(TM_THREADS, 1) tmem_stage_kernel(const TmArgs 
                 }
             }
         }
+        if (grp == 0) {
 #pragma unroll
-        for (int tau = 0; tau < MAXTOK; ++tau)
-            if (tau < a.T) part[tau * 128 + tid] = outv[tau];
-    } else if (warp < 4 + TM_ISSUERS) {
+            for (int tau = 0; tau < MAXTOK; ++tau)
+                if (tau < a.T) part[tau * 128 + row_l] = outv[tau];
+        }
+    } else if (warp < TM_W_ISSUER0 + TM_ISSUERS) {
         // ===================== B-tile producers and MMA issuers ==========================
-        const int w = warp - 4;
+        const int w = warp - TM_W_ISSUER0;
         const int ptid = tid - TM_EXPANDERS;                 // 0..127 among the producer warps
         // B tiles start as zeros (rows beyond T*LP are never written again)
         for (int i = ptid; i < TM_ISSUERS * 2 * bbytes / 16; i += TM_ISSUERS * 32)
             reinterpret_cast<uint4 *>(smem_gen)[i] = make_uint4(0u, 0u, 0u, 0u);
         pdl_wait();                                          // the activations come from the previous kernel
-        // stage in[tau][c0 .. c0 + kslice) as fp32, zero beyond the matrix
+        // stage in[tau][c0 .. c0 + kslice) as fp32, zero beyond the matrix; four columns per thread and step
         {
             const int c0 = kb0 * 64;
-            const int total = a.T * kslice;
+            const int quads = kslice >> 2;                   // kslice is a multiple of 64
+            const int total = a.T * quads;
+            const bool vec = (a.cols & 3) == 0 && (reinterpret_cast<uintptr_t>(a.in) & 15u) == 0;   // aligned rows
+#pragma unroll 4
             for (int idx = ptid; idx < total; idx += TM_ISSUERS * 32) {
-                const int tau = idx / kslice, c = idx - tau * kslice;
+                const int tau = idx / quads, c = (idx - tau * quads) << 2;
                 const int gc = c0 + c;
-                float v = 0.f;
-                if (gc < a.cols) {
-                    if (STAGE_A) v = reinterpret_cast<const float *>(a.in)[(size_t)tau * a.cols + gc];
-                    else v = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(a.in)[(size_t)tau * a.cols + gc]);
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (vec && gc + 4 <= a.cols) {
+                    if (STAGE_A) {
+                        v = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(a.in) + (size_t)tau * a.cols + gc);
+                    } else {
+                        const uint2 r = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(a.in) +
+                                                                         (size_t)tau * a.cols + gc);
+                        v = make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xFFFF0000u),
+                                        __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xFFFF0000u));
+                    }
+                } else {
+                    float e[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        e[q] = 0.f;
+                        if (gc + q < a.cols) {
+                            if (STAGE_A) e[q] = reinterpret_cast<const float *>(a.in)[(size_t)tau * a.cols + gc + q];
+                            else e[q] = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(a.in)[(size_t)tau * a.cols + gc + q]);
+                        }
+                    }
+                    v = make_float4(e[0], e[1], e[2], e[3]);
                 }
-                xin[idx] = v;
+                *reinterpret_cast<float4 *>(xin + tau * kslice + c) = v;
             }
         }
         fence_proxy_async();                                 // the zeroed tiles are read by the tensor core
@@ -352,8 +396,10 @@ __global__ void __launch_bounds__(TM_THREADS, 1) tmem_stage_kernel(const TmArgs 
         const int nchunks = a.T * LP * 8;                    // 16-byte chunks of real rows in a B tile
         bool alive = true;
         int it = 0;
+        int as = w % nas;                                    // A stage of K block kb = w, w + 4, ...
+        uint32_t as_ph = (uint32_t)(w / nas) & 1u;
         for (int kb = w; kb < nkb && alive; kb += TM_ISSUERS, ++it) {
-            const int buf = it & 1, vs = kb % TM_VSTAGES, as = kb % nas;
+            const int buf = it & 1, vs = kb % TM_VSTAGES;
             alive = mbar_wait(b_empty + 8 * (w * 2 + buf), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag, a.status);
             if (!alive) break;
             alive = mbar_wait(v_full + 8 * vs, (uint32_t)(kb / TM_VSTAGES) & 1u, abort_flag, a.status);
@@ -361,6 +407,7 @@ __global__ void __launch_bounds__(TM_THREADS, 1) tmem_stage_kernel(const TmArgs 
             unsigned char *bt = smem_gen + (size_t)(w * 2 + buf) * bbytes;
             const unsigned char *vb = smem_gen + off_v + vs * vbytes;
             const float *xk = xin + kb * 64;
+#pragma unroll 4
             for (int i = lane; i < nchunks; i += 32) {
                 const int n = i >> 3, j = i & 7;
                 const int tau = n / LP, t = n % LP;
@@ -378,7 +425,7 @@ __global__ void __launch_bounds__(TM_THREADS, 1) tmem_stage_kernel(const TmArgs 
             fence_proxy_async();
             __syncwarp();
             if (lane == 0) mbar_arrive(v_empty + 8 * vs);
-            alive = mbar_wait(a_full + 8 * as, (uint32_t)(kb / nas) & 1u, abort_flag, a.status);
+            alive = mbar_wait(a_full + 8 * as, as_ph, abort_flag, a.status);
             if (!alive) break;
             tc_fence_after();
             if (lane == 0) {
@@ -391,13 +438,15 @@ __global__ void __launch_bounds__(TM_THREADS, 1) tmem_stage_kernel(const TmArgs 
                 umma_commit(b_empty + 8 * (w * 2 + buf));
             }
             __syncwarp();
+            as += TM_ISSUERS;
+            while (as >= nas) { as -= nas; as_ph ^= 1u; }
         }
         if (lane == 0) {
             if (alive && it > 0) umma_commit(acc_bar);       // arrives when this issuer's MMAs have retired
             else mbar_arrive(acc_bar);
         }
         __syncwarp();
-    } else if (warp == 4 + TM_ISSUERS) {
+    } else if (warp == TM_W_ISSUER0 + TM_ISSUERS) {
         // ============================== sign-word loader ================================
         if (lane == 0) {
             bool alive = true;
@@ -433,15 +482,20 @@ __global__ void __launch_bounds__(TM_THREADS, 1) tmem_stage_kernel(const TmArgs 
     tc_fence_before();
     cluster.sync();
     if (warp < 4 && cluster.block_rank() == 0) {
+        const int tid_r = row_l;
         const unsigned nranks = cluster.num_blocks();
-        for (unsigned rk = 1; rk < nranks; ++rk) {
-            const float *rp = cluster.map_shared_rank(part, rk);
 #pragma unroll
-            for (int tau = 0; tau < MAXTOK; ++tau)
-                if (tau < a.T) outv[tau] += rp[tau * 128 + tid];
-        }
+        for (int tau = 0; tau < MAXTOK; ++tau)
+            if (tau < a.T) {
+                float rv[8];
+#pragma unroll
+                for (unsigned rk = 1; rk < 8; ++rk)          // all remote loads in flight together
+                    rv[rk] = rk < nranks ? cluster.map_shared_rank(part, rk)[tau * 128 + tid_r] : 0.f;
+#pragma unroll
+                for (unsigned rk = 1; rk < 8; ++rk) outv[tau] += rv[rk];
+            }
         pdl_wait();                                          // order the stores after the previous kernel
-        const int grow = row0 + tid;
+        const int grow = row0 + tid_r;
         if (grow < a.rows && !*abort_flag) {
 #pragma unroll
             for (int tau = 0; tau < MAXTOK; ++tau)
@@ -452,7 +506,7 @@ __global__ void __launch_bounds__(TM_THREADS, 1) tmem_stage_kernel(const TmArgs 
         }
     }
     cluster.sync();
-    if (warp == 4) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
+    if (warp == TM_W_ISSUER0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
 }
 
 // ----------------------------------------------------------- pack-time private copy
@@ -483,6 +537,326 @@ mdbf_status_t launch_vperm(const void *V, int cols, int l, int env_dtype, uint16
     return MDBF_OK;
 }
 
+// =====================================================================================
+// One token (T = 1): the activation moves into the A operand.
+//
+//     D[r][t] = sum_c  ( S[r][c] * in[c] ) * V[c][t]
+//
+// A[r][c] is the bf16 activation with the packed bit XOR-ed into its sign (the same shift + one
+// logic op per two bits as the +-1 expansion), B is V itself: immutable, kept as ready-made
+// 128B-swizzled bf16 tile images (vtile_kernel) that a bulk copy drops straight into the B stage.
+// No B tile is built at run time, everything except the activation slice is in flight before the
+// dependency wait, and the issuer warps only issue.  One tcgen05.commit per K block releases the
+// A stage and the V stage together (same ring index).
+struct TxArgs {
+    const uint2 *wk;          // K-blocked sign words [kblocks][rows_pad]
+    int rows_pad;
+    int rows, cols;
+    const uint16_t *vtile;    // bf16 V tile images [kblocks][NB * 64], 128B-swizzled, NB = max(LP, 16)
+    const void *U;            // [rows][l] env_dtype
+    int env_dtype, l;
+    const void *in;           // stage B: bf16 x [cols]; stage A: fp32 z [cols]
+    void *out;                // stage B: fp32 z [rows]; stage A: bf16 y [rows]
+    int nkb_total, kb_per_cta;
+    int nastages, nsstages, tmem_cols;
+    int32_t *status;
+};
+
+// Shared-memory plan (dynamic, 1024-byte aligned):
+//   vring [nastages][NB * 128 B]   V tile images (B operand)
+//   sring [nsstages][1024 B]       packed sign words
+//   xp    [kb_per_cta * 32] u32    activation pairs in MMA k order (bf16x2)
+//   part  [128] float              partial outputs (cluster reduction)
+template <int LP, bool STAGE_A>
+__global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(const TxArgs a) {
+    using namespace tm;
+    constexpr int NB = LP < 16 ? 16 : LP;                    // MMA N
+    constexpr int VBYTES = NB * 128;
+    extern __shared__ unsigned char tm_smem_raw[];
+    __shared__ __align__(8) uint64_t bars[2 * TM_MAX_SSTAGES + 3 * TM_MAX_ASTAGES + 1];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag_s;
+    volatile int *abort_flag = &abort_flag_s;
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t smem_base = (smem_u32(tm_smem_raw) + 1023u) & ~1023u;
+    unsigned char *smem_gen = tm_smem_raw + (smem_base - smem_u32(tm_smem_raw));
+    const int nas = a.nastages, nss = a.nsstages;
+    const uint32_t off_s = (uint32_t)(nas * VBYTES);
+    const uint32_t off_x = off_s + (uint32_t)(nss * 1024);
+    const uint32_t off_p = off_x + (uint32_t)(a.kb_per_cta * 128);
+    uint32_t *xp = reinterpret_cast<uint32_t *>(smem_gen + off_x);
+    float *part = reinterpret_cast<float *>(smem_gen + off_p);
+
+    constexpr int NB0 = TM_MAX_SSTAGES, NB1 = 2 * TM_MAX_SSTAGES, NB2 = NB1 + TM_MAX_ASTAGES,
+                  NB3 = NB2 + TM_MAX_ASTAGES, NB4 = NB3 + TM_MAX_ASTAGES;
+    const uint32_t s_full = smem_u32(&bars[0]), s_empty = smem_u32(&bars[NB0]), v_full = smem_u32(&bars[NB1]),
+                   a_full = smem_u32(&bars[NB2]), a_empty = smem_u32(&bars[NB3]), acc_bar = smem_u32(&bars[NB4]);
+
+    const int row0 = blockIdx.x * 128;
+    const int kb0 = blockIdx.y * a.kb_per_cta;
+    const int nkb = max(0, min(a.kb_per_cta, a.nkb_total - kb0));
+
+    if (tid <= NB4) {       // s_full 1, s_empty 4, v_full 1, a_full 4, a_empty 1, acc_bar TM_ISSUERS
+        const uint32_t count = tid < NB0 ? 1u : tid < NB1 ? 4u : tid < NB2 ? 1u : tid < NB3 ? 4u : tid < NB4 ? 1u
+                                                                                                      : (uint32_t)TM_ISSUERS;
+        mbar_init(smem_u32(&bars[tid]), count);
+    }
+    if (tid == 0) abort_flag_s = 0;
+    fence_barrier_init();
+    if (warp == TM_W_ISSUER0) {
+        tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)a.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_slot;
+    const uint32_t tmem_a0 = tmem + (uint32_t)(TM_ISSUERS * NB);
+
+    pdl_launch_dependents();
+
+    const int row_l = (warp & 3) * 32 + lane;
+    float outv = 0.f;
+
+    if (warp < TM_W_ISSUER0) {
+        // ============================ expanders, then epilogue ============================
+        const int grp = warp >> 2;
+        const int grow = row0 + row_l;
+        float u[LP];
+#pragma unroll
+        for (int t = 0; t < LP; ++t)
+            u[t] = (grp == 0 && grow < a.rows && t < a.l) ? env_load(a.U, (size_t)grow * a.l + t, a.env_dtype) : 0.f;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+
+        // stage the activation slice as bf16 pairs in MMA k order: pair `col` of a K block holds
+        // columns 32*(col/16) + col%16 and that + 16; four pairs per thread and step
+        pdl_wait();
+        {
+            const int c0 = kb0 * 64;
+            const int quads = a.kb_per_cta * 8;
+            const bool vec = (a.cols & 3) == 0 && (reinterpret_cast<uintptr_t>(a.in) & 15u) == 0;
+            for (int q = tid; q < quads; q += TM_EXPANDERS) {
+                const int kbl = q >> 3, col = (q & 7) << 2;
+                const int c_lo = c0 + kbl * 64 + 32 * (col >> 4) + (col & 15);
+                float lo[4], hi[4];
+                if (vec && c_lo + 20 <= a.cols) {
+                    if (STAGE_A) {
+                        const float4 l4 = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(a.in) + c_lo);
+                        const float4 h4 = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(a.in) + c_lo + 16);
+                        lo[0] = l4.x; lo[1] = l4.y; lo[2] = l4.z; lo[3] = l4.w;
+                        hi[0] = h4.x; hi[1] = h4.y; hi[2] = h4.z; hi[3] = h4.w;
+                    } else {
+                        const uint2 l2 = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(a.in) + c_lo);
+                        const uint2 h2 = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(a.in) + c_lo + 16);
+                        lo[0] = __uint_as_float(l2.x << 16); lo[1] = __uint_as_float(l2.x & 0xFFFF0000u);
+                        lo[2] = __uint_as_float(l2.y << 16); lo[3] = __uint_as_float(l2.y & 0xFFFF0000u);
+                        hi[0] = __uint_as_float(h2.x << 16); hi[1] = __uint_as_float(h2.x & 0xFFFF0000u);
+                        hi[2] = __uint_as_float(h2.y << 16); hi[3] = __uint_as_float(h2.y & 0xFFFF0000u);
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int cl = c_lo + e, ch = c_lo + 16 + e;
+                        lo[e] = 0.f; hi[e] = 0.f;
+                        if (STAGE_A) {
+                            if (cl < a.cols) lo[e] = reinterpret_cast<const float *>(a.in)[cl];
+                            if (ch < a.cols) hi[e] = reinterpret_cast<const float *>(a.in)[ch];
+                        } else {
+                            if (cl < a.cols) lo[e] = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(a.in)[cl]);
+                            if (ch < a.cols) hi[e] = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(a.in)[ch]);
+                        }
+                    }
+                }
+                *reinterpret_cast<uint4 *>(xp + kbl * 32 + col) =
+                    make_uint4(pack_bf16x2(lo[0], hi[0]), pack_bf16x2(lo[1], hi[1]), pack_bf16x2(lo[2], hi[2]),
+                               pack_bf16x2(lo[3], hi[3]));
+            }
+        }
+        asm volatile("bar.sync 2, 256;\n" ::: "memory");
+
+        bool alive = true;
+        int rs = grp % nss, as = grp % nas;
+        uint32_t rs_ph = 0, as_ph = 0;
+        int prev_as = -1;
+        for (int kb = grp; kb < nkb && alive; kb += 2) {
+            alive = mbar_wait(s_full + 8 * rs, rs_ph, abort_flag, a.status);
+            if (!alive) break;
+            const uint2 w = *reinterpret_cast<const uint2 *>(smem_gen + off_s + rs * 1024 + row_l * 8);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s_empty + 8 * rs);
+            uint32_t v[32];
+            const uint4 *xq = reinterpret_cast<const uint4 *>(xp + kb * 32);
+#pragma unroll
+            for (int i4 = 0; i4 < 4; ++i4) {
+                const uint4 xa = xq[i4], xb = xq[4 + i4];                 // pairs 4*i4 .. +3 of word 0 and word 1
+                const uint32_t xl[4] = {xa.x, xa.y, xa.z, xa.w}, xh[4] = {xb.x, xb.y, xb.z, xb.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int i = i4 * 4 + e;
+                    v[i] = ((w.x << (15 - i)) & 0x80008000u) ^ xl[e];
+                    v[16 + i] = ((w.y << (15 - i)) & 0x80008000u) ^ xh[e];
+                }
+            }
+            if (prev_as >= 0) {
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(a_full + 8 * prev_as);
+            }
+            alive = mbar_wait(a_empty + 8 * as, as_ph ^ 1u, abort_flag, a.status);
+            if (!alive) break;
+            tc_fence_after();
+            tmem_st32(tmem_a0 + lane_base + (uint32_t)(as * 32), v);
+            prev_as = as;
+            rs += 2; if (rs >= nss) { rs -= nss; rs_ph ^= 1u; }
+            as += 2; if (as >= nas) { as -= nas; as_ph ^= 1u; }
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (alive && prev_as >= 0 && lane == 0) mbar_arrive(a_full + 8 * prev_as);
+        if (grp != 0) alive = false;
+        if (alive) alive = mbar_wait(acc_bar, 0u, abort_flag, a.status);
+        tc_fence_after();
+        if (alive) {
+            const int nacc = nkb < TM_ISSUERS ? nkb : TM_ISSUERS;
+#pragma unroll
+            for (int cc = 0; cc < NB / 16; ++cc) {
+                uint32_t d[TM_ISSUERS][16];
+#pragma unroll
+                for (int acc = 0; acc < TM_ISSUERS; ++acc)
+                    if (acc < nacc) tmem_ld16(tmem + lane_base + (uint32_t)(acc * NB + cc * 16), d[acc]);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    float sum = 0.f;
+#pragma unroll
+                    for (int acc = 0; acc < TM_ISSUERS; ++acc)
+                        if (acc < nacc) sum += __uint_as_float(d[acc][j]);
+                    if (cc * 16 + j < LP) outv += u[(cc * 16 + j) % LP] * sum;
+                }
+            }
+        }
+        if (grp == 0) part[row_l] = outv;
+    } else if (warp < TM_W_ISSUER0 + TM_ISSUERS) {
+        // ================================== MMA issuers ===================================
+        const int w = warp - TM_W_ISSUER0;
+        const uint32_t idesc = make_idesc(NB);
+        const uint32_t d_tmem = tmem + (uint32_t)(w * NB);
+        bool alive = true;
+        int it = 0;
+        int as = w % nas;
+        uint32_t as_ph = (uint32_t)(w / nas) & 1u;
+        for (int kb = w; kb < nkb && alive; kb += TM_ISSUERS, ++it) {
+            alive = mbar_wait(v_full + 8 * as, as_ph, abort_flag, a.status);
+            if (!alive) break;
+            alive = mbar_wait(a_full + 8 * as, as_ph, abort_flag, a.status);
+            if (!alive) break;
+            tc_fence_after();
+            if (lane == 0) {
+                const uint64_t bdesc = make_smem_desc(smem_base + (uint32_t)(as * VBYTES));
+                const uint32_t a_t = tmem_a0 + (uint32_t)(as * 32);
+#pragma unroll
+                for (int k4 = 0; k4 < 4; ++k4)
+                    umma_ts(d_tmem, a_t + (uint32_t)(8 * k4), bdesc + (uint64_t)(2 * k4), idesc, (it > 0 || k4 > 0) ? 1u : 0u);
+                umma_commit(a_empty + 8 * as);               // frees the A stage and the V stage
+            }
+            __syncwarp();
+            as += TM_ISSUERS;
+            while (as >= nas) { as -= nas; as_ph ^= 1u; }
+        }
+        if (lane == 0) {
+            if (alive && it > 0) umma_commit(acc_bar);
+            else mbar_arrive(acc_bar);
+        }
+        __syncwarp();
+    } else if (warp == TM_W_ISSUER0 + TM_ISSUERS) {
+        // ============================== sign-word loader ================================
+        if (lane == 0) {
+            bool alive = true;
+            int rs = 0;
+            uint32_t ph = 0;
+            for (int kb = 0; kb < nkb && alive; ++kb) {
+                alive = mbar_wait(s_empty + 8 * rs, ph ^ 1u, abort_flag, a.status);
+                if (!alive) break;
+                mbar_arrive_expect_tx(s_full + 8 * rs, 1024u);
+                bulk_load(smem_base + off_s + (uint32_t)(rs * 1024), a.wk + (size_t)(kb0 + kb) * a.rows_pad + row0, 1024u,
+                          s_full + 8 * rs);
+                if (++rs == nss) { rs = 0; ph ^= 1u; }
+            }
+            if (!alive) drain_delay();
+        }
+        __syncwarp();
+    } else {
+        // ================================ V-tile loader ==================================
+        if (lane == 0) {
+            bool alive = true;
+            int vs = 0;
+            uint32_t ph = 0;
+            for (int kb = 0; kb < nkb && alive; ++kb) {
+                alive = mbar_wait(a_empty + 8 * vs, ph ^ 1u, abort_flag, a.status);
+                if (!alive) break;
+                mbar_arrive_expect_tx(v_full + 8 * vs, (uint32_t)VBYTES);
+                bulk_load(smem_base + (uint32_t)(vs * VBYTES), a.vtile + (size_t)(kb0 + kb) * NB * 64, (uint32_t)VBYTES,
+                          v_full + 8 * vs);
+                if (++vs == nas) { vs = 0; ph ^= 1u; }
+            }
+            if (!alive) drain_delay();
+        }
+        __syncwarp();
+    }
+
+    // ------------------------------ cluster reduction and store ------------------------------
+    tc_fence_before();
+    cluster.sync();
+    if (warp < 4 && cluster.block_rank() == 0) {
+        const unsigned nranks = cluster.num_blocks();
+        float rv[8];
+#pragma unroll
+        for (unsigned rk = 1; rk < 8; ++rk) rv[rk] = rk < nranks ? cluster.map_shared_rank(part, rk)[row_l] : 0.f;
+#pragma unroll
+        for (unsigned rk = 1; rk < 8; ++rk) outv += rv[rk];
+        const int grow = row0 + row_l;
+        if (grow < a.rows && !*abort_flag) {
+            if (STAGE_A) reinterpret_cast<__nv_bfloat16 *>(a.out)[grow] = __float2bfloat16_rn(outv);
+            else reinterpret_cast<float *>(a.out)[grow] = outv;
+        }
+    }
+    cluster.sync();
+    if (warp == TM_W_ISSUER0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
+}
+
+// bf16 V tile images for the one-token kernel: K block kb is NB rows (modes) x 64 k, K-major with
+// 128-byte rows and the 128B swizzle; element (t, p) holds V[c][t], c = kb*64 + 32*(p/32) + (p%32)/2
+// + 16*(p%2), at 16-bit index kb*NB*64 + t*64 + ((p/8) ^ (t%8))*8 + p%8; zero outside the matrix.
+__global__ void vtile_kernel(const void *__restrict__ V, int cols, int l, int env_dtype, uint16_t *__restrict__ out,
+                             int kblocks, int NB) {
+    const size_t total = (size_t)kblocks * NB * 64;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+        const int p = (int)(idx & 63);
+        const int t = (int)((idx >> 6) % NB);
+        const int kb = (int)((idx >> 6) / NB);
+        const int c = kb * 64 + 32 * (p >> 5) + ((p & 31) >> 1) + 16 * (p & 1);
+        float v = 0.f;
+        if (c < cols && t < l) v = env_load(V, (size_t)c * l + t, env_dtype);
+        const __nv_bfloat16 b = __float2bfloat16_rn(v);
+        out[(size_t)kb * NB * 64 + t * 64 + (((p >> 3) ^ (t & 7)) << 3) + (p & 7)] = *reinterpret_cast<const uint16_t *>(&b);
+    }
+}
+
+mdbf_status_t launch_vtile(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int NB,
+                           cudaStream_t st) {
+    const size_t total = (size_t)kblocks * NB * 64;
+    int grid = (int)((total + 255) / 256);
+    if (grid > 148 * 16) grid = 148 * 16;
+    if (grid < 1) grid = 1;
+    vtile_kernel<<<grid, 256, 0, st>>>(V, cols, l, env_dtype, out, kblocks, NB);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}
+
 // ---------------------------------------------------------------------- launch
 struct TmPlan {
     int ks, kb_per_cta, nastages, nsstages, tmem_cols, n_mma;
@@ -498,10 +872,12 @@ static bool plan_stage(int rows, int cols, int LP, int T, TmPlan *p) {
     const int rb = ceil_div(rows, 128), nkb = ceil_div(cols, 64);
     // TMEM columns: one accumulator per issuer, then the A stages (32 columns each)
     const int acc_cols = TM_ISSUERS * n_mma;
-    const int nas = (acc_cols + 4 * 32 <= 256) ? 4 : 8;
-    const int need = acc_cols + nas * 32;
-    if (need > 512) return false;
-    const int tmem_cols = need <= 256 ? 256 : 512;
+    // Half of TMEM (256 columns) when at least four A stages fit beside the accumulators, so that two
+    // CTAs - this kernel's and the next one's, started early - can share an SM; else all of it.
+    const int tmem_cols = (acc_cols + 4 * 32 <= 256) ? 256 : 512;
+    int nas = (tmem_cols - acc_cols) / 32;
+    if (nas > TM_MAX_ASTAGES) nas = TM_MAX_ASTAGES;
+    if (nas < 2) return false;
     long best_cost = -1;
     int best_ks = 0;
     for (int ks = 1; ks <= 8; ks *= 2) {
@@ -524,6 +900,85 @@ static bool plan_stage(int rows, int cols, int LP, int T, TmPlan *p) {
     p->smem = 1024 + (size_t)TM_ISSUERS * 2 * n_mma * 128 + (size_t)TM_VSTAGES * LP * 128 + (size_t)p->nsstages * 1024 +
               (size_t)T * p->kb_per_cta * 64 * 4 + (size_t)T * 128 * 4;
     return p->smem <= 220 * 1024;
+}
+
+// One-token plan: cluster size along the reduction (see plan_stage), ring depths, TMEM columns.
+static bool plan_t1(int rows, int cols, int LP, TmPlan *p) {
+    const int NB = LP < 16 ? 16 : LP;
+    const int rb = ceil_div(rows, 128), nkb = ceil_div(cols, 64);
+    const int acc_cols = TM_ISSUERS * NB;
+    const int tmem_cols = (acc_cols + 4 * 32 <= 256) ? 256 : 512;
+    int nas = (tmem_cols - acc_cols) / 32;
+    if (nas > TM_MAX_ASTAGES) nas = TM_MAX_ASTAGES;
+    long best_cost = -1;
+    int best_ks = 0;
+    for (int ks = 1; ks <= 8; ks *= 2) {
+        const int per = ceil_div(nkb, ks);
+        if (ks > 1 && per * (ks - 1) >= nkb) continue;
+        const long waves = ceil_div(rb * ks, 148);
+        const long cost = waves * (per + 16);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ks = ks; }
+    }
+    p->ks = best_ks;
+    p->kb_per_cta = ceil_div(nkb, best_ks);
+    p->nastages = nas;
+    p->nsstages = p->kb_per_cta < TM_MAX_SSTAGES ? p->kb_per_cta : TM_MAX_SSTAGES;
+    if (p->nsstages < 2) p->nsstages = 2;
+    p->tmem_cols = tmem_cols;
+    p->n_mma = NB;
+    p->smem = 1024 + (size_t)nas * NB * 128 + (size_t)p->nsstages * 1024 + (size_t)p->kb_per_cta * 128 + 512;
+    return p->smem <= 220 * 1024;
+}
+
+template <int LP, bool STAGE_A>
+static mdbf_status_t launch_t1(const TxArgs &a, const TmPlan &p, cudaStream_t st) {
+    auto kern = tmem_t1_kernel<LP, STAGE_A>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        MDBF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ceil_div(a.rows, 128), p.ks, 1);
+    cfg.blockDim = dim3(TM_THREADS);
+    cfg.dynamicSmemBytes = p.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = p.ks;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    MDBF_CUDA(cudaLaunchKernelEx(&cfg, kern, a));
+    return MDBF_OK;
+}
+
+template <int LP>
+static mdbf_status_t run_t1(Layer &L, const void *x, void *y, cudaStream_t st) {
+    const mdbf_desc_t &d = L.d;
+    TmPlan pb, pa;
+    if (!plan_t1(d.k, d.d_in, LP, &pb) || !plan_t1(d.d_out, d.k, LP, &pa)) {
+        set_error("mdbf_linear_forward: the one-token TMEM kernel does not fit this shape");
+        return MDBF_ERR_SHAPE;
+    }
+    TxArgs b = {};
+    b.wk = L.wkB; b.rows_pad = L.rpB; b.rows = d.k; b.cols = d.d_in;
+    b.vtile = L.vxB; b.U = L.UB; b.env_dtype = d.env_dtype; b.l = d.l;
+    b.in = x; b.out = L.zsum;
+    b.nkb_total = ceil_div(d.d_in, 64); b.kb_per_cta = pb.kb_per_cta;
+    b.nastages = pb.nastages; b.nsstages = pb.nsstages; b.tmem_cols = pb.tmem_cols; b.status = L.status;
+    mdbf_status_t rc = launch_t1<LP, false>(b, pb, st);
+    if (rc) return rc;
+    TxArgs s = {};
+    s.wk = L.wkA; s.rows_pad = L.rpA; s.rows = d.d_out; s.cols = d.k;
+    s.vtile = L.vxA; s.U = L.UA; s.env_dtype = d.env_dtype; s.l = d.l;
+    s.in = L.zsum; s.out = y;
+    s.nkb_total = ceil_div(d.k, 64); s.kb_per_cta = pa.kb_per_cta;
+    s.nastages = pa.nastages; s.nsstages = pa.nsstages; s.tmem_cols = pa.tmem_cols; s.status = L.status;
+    return launch_t1<LP, true>(s, pa, st);
 }
 
 bool tmem_path_supports(const Layer &L, int T) {
@@ -590,6 +1045,20 @@ mdbf_status_t launch_forward_tmem(Layer &L, const void *x, void *y, int T, cudaS
     }
     const bool bf = L.d.env_dtype == MDBF_BF16;
     mdbf_status_t rc;
+    if (T == 1 && L.vxA && L.vxB) {
+        switch (L.LP) {
+            case 1: rc = run_t1<1>(L, x, y, st); break;
+            case 2: rc = run_t1<2>(L, x, y, st); break;
+            case 4: rc = run_t1<4>(L, x, y, st); break;
+            case 8: rc = run_t1<8>(L, x, y, st); break;
+            case 16: rc = run_t1<16>(L, x, y, st); break;
+            default: rc = run_t1<32>(L, x, y, st); break;
+        }
+        if (rc) return rc;
+        L.last_ksplit = 0;
+        *launches = 2;
+        return MDBF_OK;
+    }
 #define MDBF_TM_CASE(lp) case lp: rc = bf ? run_tm<lp, true>(L, x, y, T, st) : run_tm<lp, false>(L, x, y, T, st); break;
     switch (L.LP) {
         MDBF_TM_CASE(1) MDBF_TM_CASE(2) MDBF_TM_CASE(4) MDBF_TM_CASE(8) MDBF_TM_CASE(16) MDBF_TM_CASE(32)

@@ -166,12 +166,13 @@ def test_linearity_column_independence_and_duality():
     x4 = inputs.make_activations(spec, 4)
     with GpuLayer(spec, 4, lay=lay) as g:
         y4 = g.forward(x4)
-        for t in range(4):                     # T-batched equals per-column
-            y1 = g.forward(x4[t:t + 1])
-            assert rel_err(y1, y4[t:t + 1]) <= 1e-6
+        for t in (0, 2):                       # T-batched equals per-column (same kernel variant: exact)
+            assert rel_err(g.forward(x4[t:t + 2]), y4[t:t + 2]) <= 1e-6
+        for t in range(4):                     # one token may take another variant: equal within rounding
+            assert rel_err(g.forward(x4[t:t + 1]), y4[t:t + 1]) <= 2 * TOL["bf16"]
         # linearity: power-of-two scaling is exact in bf16/fp32 arithmetic
-        y_scaled = g.forward(4.0 * x4[:1])
-        np.testing.assert_array_equal(y_scaled, 4.0 * y4[:1])
+        y_scaled = g.forward(4.0 * x4)
+        np.testing.assert_array_equal(y_scaled, 4.0 * y4)
         # additivity within rounding
         xs = inputs.round_to(x4[0:1] + x4[1:2], "bf16")
         assert rel_err(g.forward(xs), (y4[0:1] + y4[1:2])) <= 2 * TOL["bf16"]

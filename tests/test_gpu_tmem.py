@@ -48,6 +48,25 @@ def test_tmem_kernel_small_shapes(l, T):
         np.testing.assert_array_equal(y, g.forward(x))            # AUTO picks this kernel; deterministic
 
 
+@pytest.mark.parametrize("l", [1, 2, 3, 4, 8, 12, 16, 24, 32])
+@pytest.mark.parametrize("env", ["f16", "bf16"])
+def test_one_token_kernel(l, env):
+    """T = 1 takes the variant with the activation folded into the TMEM operand."""
+    spec = spec_of(419, 1000, 700, l, env_dtype=env)
+    x = inputs.make_activations(spec, 1)
+    with GpuLayer(spec, 4) as g:
+        ref = g.oracle_forward(x)
+        y = g.forward(x, kernel=M.KERNEL_TMEM)
+        assert M.mdbf_poll_status(g.h) == 0
+        assert rel_err(y, ref) <= TOL["bf16"]
+        _, z_ref = orc.forward_staged(*g.oracle_args(), x.T.astype(np.float64))
+        assert rel_err(g.intermediate(1), z_ref.T) <= TOL["bf16"]
+        x4 = inputs.make_activations(spec, 4)                     # same layer, wider batch: the B-scaled variant
+        y4 = g.forward(x4, kernel=M.KERNEL_TMEM) if 4 * g.spec.l <= 64 and l in (1, 2, 4, 8, 16) else g.forward(x4)
+        assert rel_err(y4, g.oracle_forward(x4)) <= TOL["bf16"]
+        assert rel_err(g.forward(x4[:1], kernel=M.KERNEL_TMEM), y4[:1]) <= 2 * TOL["bf16"]
+
+
 @pytest.mark.parametrize("shape", [(1, 1, 1, 1), (31, 127, 33, 2), (129, 1025, 257, 9), (1000, 2100, 1300, 16),
                                    (256, 4096, 512, 16), (2048, 192, 3000, 16)])
 def test_tmem_kernel_edge_shapes(shape):
@@ -72,8 +91,10 @@ def test_tmem_kernel_bf16_envelopes_and_cross_check():
         for y in (y_tm, y_dec, y_pf):
             assert rel_err(y, ref) <= TOL["bf16"]
         assert rel_err(y_tm, y_pf) <= 2 * TOL["bf16"]
-        for t in range(4):                                       # column independence
-            assert rel_err(g.forward(x[t:t + 1], kernel=M.KERNEL_TMEM), y_tm[t:t + 1]) <= 1e-6
+        for t in (0, 2):                                         # column independence inside one kernel variant
+            assert rel_err(g.forward(x[t:t + 2], kernel=M.KERNEL_TMEM), y_tm[t:t + 2]) <= 1e-6
+        for t in range(4):                                       # one token takes another variant: same within rounding
+            assert rel_err(g.forward(x[t:t + 1], kernel=M.KERNEL_TMEM), y_tm[t:t + 1]) <= 2 * TOL["bf16"]
 
 
 def test_tmem_kernel_rejects_wide_batches():
