@@ -148,6 +148,10 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
           "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
         : "memory");
 }
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&v)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};\n"
+                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
     asm volatile(
@@ -676,28 +680,35 @@ __global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(c
         }
         asm volatile("bar.sync 2, 256;\n" ::: "memory");
 
+        // Per K block: the packed words of the NEXT block and the activation pairs of this one are
+        // requested first, then the previous block's TMEM stores are retired, then 4 x (8 logic ops +
+        // one 8-column TMEM store); the loads overlap the waits instead of heading a serial chain.
         bool alive = true;
         int rs = grp % nss, as = grp % nas;
-        uint32_t rs_ph = 0, as_ph = 0;
+        uint32_t rs_ph = (uint32_t)(grp / nss) & 1u, as_ph = (uint32_t)(grp / nas) & 1u;
         int prev_as = -1;
-        for (int kb = grp; kb < nkb && alive; kb += 2) {
+        uint2 w = make_uint2(0u, 0u);
+        if (grp < nkb) {
             alive = mbar_wait(s_full + 8 * rs, rs_ph, abort_flag, a.status);
-            if (!alive) break;
-            const uint2 w = *reinterpret_cast<const uint2 *>(smem_gen + off_s + rs * 1024 + row_l * 8);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(s_empty + 8 * rs);
-            uint32_t v[32];
+            if (alive) {
+                w = *reinterpret_cast<const uint2 *>(smem_gen + off_s + rs * 1024 + row_l * 8);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(s_empty + 8 * rs);
+            }
+        }
+        for (int kb = grp; kb < nkb && alive; kb += 2) {
             const uint4 *xq = reinterpret_cast<const uint4 *>(xp + kb * 32);
+            uint4 xr[8];
 #pragma unroll
-            for (int i4 = 0; i4 < 4; ++i4) {
-                const uint4 xa = xq[i4], xb = xq[4 + i4];                 // pairs 4*i4 .. +3 of word 0 and word 1
-                const uint32_t xl[4] = {xa.x, xa.y, xa.z, xa.w}, xh[4] = {xb.x, xb.y, xb.z, xb.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int i = i4 * 4 + e;
-                    v[i] = ((w.x << (15 - i)) & 0x80008000u) ^ xl[e];
-                    v[16 + i] = ((w.y << (15 - i)) & 0x80008000u) ^ xh[e];
-                }
+            for (int q = 0; q < 8; ++q) xr[q] = xq[q];
+            uint2 w_next = make_uint2(0u, 0u);
+            if (kb + 2 < nkb) {
+                rs += 2; while (rs >= nss) { rs -= nss; rs_ph ^= 1u; }
+                alive = mbar_wait(s_full + 8 * rs, rs_ph, abort_flag, a.status);
+                if (!alive) break;
+                w_next = *reinterpret_cast<const uint2 *>(smem_gen + off_s + rs * 1024 + row_l * 8);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(s_empty + 8 * rs);
             }
             if (prev_as >= 0) {
                 tmem_st_wait();
@@ -708,10 +719,23 @@ __global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(c
             alive = mbar_wait(a_empty + 8 * as, as_ph ^ 1u, abort_flag, a.status);
             if (!alive) break;
             tc_fence_after();
-            tmem_st32(tmem_a0 + lane_base + (uint32_t)(as * 32), v);
+            const uint32_t a_col = tmem_a0 + lane_base + (uint32_t)(as * 32);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {                    // TMEM columns 8q .. 8q+7 = pairs 8q .. 8q+7
+                const uint32_t word = q < 2 ? w.x : w.y;
+                const uint32_t xs8[8] = {xr[2 * q].x, xr[2 * q].y, xr[2 * q].z, xr[2 * q].w,
+                                         xr[2 * q + 1].x, xr[2 * q + 1].y, xr[2 * q + 1].z, xr[2 * q + 1].w};
+                uint32_t v[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int i = (q & 1) * 8 + e;           // bits (i, i + 16) of the word
+                    v[e] = ((word << (15 - i)) & 0x80008000u) ^ xs8[e];
+                }
+                tmem_st8(a_col + (uint32_t)(8 * q), v);
+            }
             prev_as = as;
-            rs += 2; if (rs >= nss) { rs -= nss; rs_ph ^= 1u; }
-            as += 2; if (as >= nas) { as -= nas; as_ph ^= 1u; }
+            as += 2; while (as >= nas) { as -= nas; as_ph ^= 1u; }
+            w = w_next;
         }
         tmem_st_wait();
         tc_fence_before();
@@ -915,7 +939,7 @@ static bool plan_t1(int rows, int cols, int LP, TmPlan *p) {
     for (int ks = 1; ks <= 8; ks *= 2) {
         const int per = ceil_div(nkb, ks);
         if (ks > 1 && per * (ks - 1) >= nkb) continue;
-        const long waves = ceil_div(rb * ks, 148);
+        const long waves = ceil_div(rb * ks, tmem_cols <= 256 ? 296 : 148);   // CTAs that fit at once
         const long cost = waves * (per + 16);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ks = ks; }
     }
