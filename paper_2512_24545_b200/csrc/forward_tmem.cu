@@ -51,7 +51,7 @@ constexpr int TM_THREADS = TM_EXPANDERS + TM_ISSUERS * 32 + 64;   // + sign load
 constexpr int TM_W_ISSUER0 = TM_EXPANDERS / 32;        // first issuer warp
 constexpr int TM_VSTAGES = 8;                          // V ring (two per issuer warp)
 constexpr int TM_MAX_SSTAGES = 32;                     // sign ring, 1 KB per stage
-constexpr int TM_MAX_ASTAGES = 8;                      // A stages in TMEM, 32 columns each (6 when TMEM is shared)
+constexpr int TM_MAX_ASTAGES = 12;                     // A stages in TMEM, 32 columns each (6 when TMEM is shared)
 constexpr int TM_MAX_N = 64;
 constexpr int TM_MAX_T = 16;
 constexpr uint32_t TM_MAX_POLLS = 1u << 21;
@@ -552,6 +552,11 @@ mdbf_status_t launch_vperm(const void *V, int cols, int l, int env_dtype, uint16
 // No B tile is built at run time, everything except the activation slice is in flight before the
 // dependency wait, and the issuer warps only issue.  One tcgen05.commit per K block releases the
 // A stage and the V stage together (same ring index).
+constexpr int TX_GROUPS = 2;                           // expander groups of 4 warps; group g takes K blocks g, g + 2, ...
+constexpr int TX_EXPANDERS = TX_GROUPS * 128;
+constexpr int TX_W_ISSUER0 = TX_EXPANDERS / 32;
+constexpr int TX_THREADS = TX_EXPANDERS + TM_ISSUERS * 32 + 64;   // 448: two CTAs fit on an SM
+
 struct TxArgs {
     const uint2 *wk;          // K-blocked sign words [kblocks][rows_pad]
     int rows_pad;
@@ -563,6 +568,7 @@ struct TxArgs {
     void *out;                // stage B: fp32 z [rows]; stage A: bf16 y [rows]
     int nkb_total, kb_per_cta;
     int nastages, nsstages, tmem_cols;
+    int stage_a;              // 0: stage B (bf16 in, fp32 out), 1: stage A (fp32 in, bf16 out); one kernel for both keeps its code hot
     int32_t *status;
 };
 
@@ -571,9 +577,10 @@ struct TxArgs {
 //   sring [nsstages][1024 B]       packed sign words
 //   xp    [kb_per_cta * 32] u32    activation pairs in MMA k order (bf16x2)
 //   part  [128] float              partial outputs (cluster reduction)
-template <int LP, bool STAGE_A>
-__global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(const TxArgs a) {
+template <int LP>
+__global__ void __launch_bounds__(TX_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(const TxArgs a) {
     using namespace tm;
+    const bool STAGE_A = a.stage_a != 0;
     constexpr int NB = LP < 16 ? 16 : LP;                    // MMA N
     constexpr int VBYTES = NB * 128;
     extern __shared__ unsigned char tm_smem_raw[];
@@ -609,7 +616,7 @@ __global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(c
     }
     if (tid == 0) abort_flag_s = 0;
     fence_barrier_init();
-    if (warp == TM_W_ISSUER0) {
+    if (warp == TX_W_ISSUER0) {
         tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)a.tmem_cols);
         tmem_relinquish();
     }
@@ -624,7 +631,7 @@ __global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(c
     const int row_l = (warp & 3) * 32 + lane;
     float outv = 0.f;
 
-    if (warp < TM_W_ISSUER0) {
+    if (warp < TX_W_ISSUER0) {
         // ============================ expanders, then epilogue ============================
         const int grp = warp >> 2;
         const int grow = row0 + row_l;
@@ -641,7 +648,7 @@ __global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(c
             const int c0 = kb0 * 64;
             const int quads = a.kb_per_cta * 8;
             const bool vec = (a.cols & 3) == 0 && (reinterpret_cast<uintptr_t>(a.in) & 15u) == 0;
-            for (int q = tid; q < quads; q += TM_EXPANDERS) {
+            for (int q = tid; q < quads; q += TX_EXPANDERS) {
                 const int kbl = q >> 3, col = (q & 7) << 2;
                 const int c_lo = c0 + kbl * 64 + 32 * (col >> 4) + (col & 15);
                 float lo[4], hi[4];
@@ -678,7 +685,7 @@ __global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(c
                                pack_bf16x2(lo[3], hi[3]));
             }
         }
-        asm volatile("bar.sync 2, 256;\n" ::: "memory");
+        asm volatile("bar.sync 2, %0;\n" ::"n"(TX_EXPANDERS) : "memory");
 
         // Per K block: the packed words of the NEXT block and the activation pairs of this one are
         // requested first, then the previous block's TMEM stores are retired, then 4 x (8 logic ops +
@@ -696,14 +703,14 @@ __global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(c
                 if (lane == 0) mbar_arrive(s_empty + 8 * rs);
             }
         }
-        for (int kb = grp; kb < nkb && alive; kb += 2) {
+        for (int kb = grp; kb < nkb && alive; kb += TX_GROUPS) {
             const uint4 *xq = reinterpret_cast<const uint4 *>(xp + kb * 32);
             uint4 xr[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q) xr[q] = xq[q];
             uint2 w_next = make_uint2(0u, 0u);
-            if (kb + 2 < nkb) {
-                rs += 2; while (rs >= nss) { rs -= nss; rs_ph ^= 1u; }
+            if (kb + TX_GROUPS < nkb) {
+                rs += TX_GROUPS; while (rs >= nss) { rs -= nss; rs_ph ^= 1u; }
                 alive = mbar_wait(s_full + 8 * rs, rs_ph, abort_flag, a.status);
                 if (!alive) break;
                 w_next = *reinterpret_cast<const uint2 *>(smem_gen + off_s + rs * 1024 + row_l * 8);
@@ -734,7 +741,7 @@ __global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(c
                 tmem_st8(a_col + (uint32_t)(8 * q), v);
             }
             prev_as = as;
-            as += 2; while (as >= nas) { as -= nas; as_ph ^= 1u; }
+            as += TX_GROUPS; while (as >= nas) { as -= nas; as_ph ^= 1u; }
             w = w_next;
         }
         tmem_st_wait();
@@ -764,9 +771,9 @@ __global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(c
             }
         }
         if (grp == 0) part[row_l] = outv;
-    } else if (warp < TM_W_ISSUER0 + TM_ISSUERS) {
+    } else if (warp < TX_W_ISSUER0 + TM_ISSUERS) {
         // ================================== MMA issuers ===================================
-        const int w = warp - TM_W_ISSUER0;
+        const int w = warp - TX_W_ISSUER0;
         const uint32_t idesc = make_idesc(NB);
         const uint32_t d_tmem = tmem + (uint32_t)(w * NB);
         bool alive = true;
@@ -796,7 +803,7 @@ __global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(c
             else mbar_arrive(acc_bar);
         }
         __syncwarp();
-    } else if (warp == TM_W_ISSUER0 + TM_ISSUERS) {
+    } else if (warp == TX_W_ISSUER0 + TM_ISSUERS) {
         // ============================== sign-word loader ================================
         if (lane == 0) {
             bool alive = true;
@@ -849,7 +856,7 @@ __global__ void __launch_bounds__(TM_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(c
         }
     }
     cluster.sync();
-    if (warp == TM_W_ISSUER0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
+    if (warp == TX_W_ISSUER0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
 }
 
 // bf16 V tile images for the one-token kernel: K block kb is NB rows (modes) x 64 k, K-major with
@@ -931,7 +938,7 @@ static bool plan_t1(int rows, int cols, int LP, TmPlan *p) {
     const int NB = LP < 16 ? 16 : LP;
     const int rb = ceil_div(rows, 128), nkb = ceil_div(cols, 64);
     const int acc_cols = TM_ISSUERS * NB;
-    const int tmem_cols = (acc_cols + 4 * 32 <= 256) ? 256 : 512;
+    const int tmem_cols = (acc_cols + 4 * 32 <= 256) ? 256 : 512;    // half of TMEM when it fits: two CTAs per SM
     int nas = (tmem_cols - acc_cols) / 32;
     if (nas > TM_MAX_ASTAGES) nas = TM_MAX_ASTAGES;
     long best_cost = -1;
@@ -954,9 +961,9 @@ static bool plan_t1(int rows, int cols, int LP, TmPlan *p) {
     return p->smem <= 220 * 1024;
 }
 
-template <int LP, bool STAGE_A>
+template <int LP>
 static mdbf_status_t launch_t1(const TxArgs &a, const TmPlan &p, cudaStream_t st) {
-    auto kern = tmem_t1_kernel<LP, STAGE_A>;
+    auto kern = tmem_t1_kernel<LP>;
     static bool attr_set = false;
     if (!attr_set) {
         MDBF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
@@ -964,7 +971,7 @@ static mdbf_status_t launch_t1(const TxArgs &a, const TmPlan &p, cudaStream_t st
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ceil_div(a.rows, 128), p.ks, 1);
-    cfg.blockDim = dim3(TM_THREADS);
+    cfg.blockDim = dim3(TX_THREADS);
     cfg.dynamicSmemBytes = p.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
@@ -991,18 +998,18 @@ static mdbf_status_t run_t1(Layer &L, const void *x, void *y, cudaStream_t st) {
     TxArgs b = {};
     b.wk = L.wkB; b.rows_pad = L.rpB; b.rows = d.k; b.cols = d.d_in;
     b.vtile = L.vxB; b.U = L.UB; b.env_dtype = d.env_dtype; b.l = d.l;
-    b.in = x; b.out = L.zsum;
+    b.in = x; b.out = L.zsum; b.stage_a = 0;
     b.nkb_total = ceil_div(d.d_in, 64); b.kb_per_cta = pb.kb_per_cta;
     b.nastages = pb.nastages; b.nsstages = pb.nsstages; b.tmem_cols = pb.tmem_cols; b.status = L.status;
-    mdbf_status_t rc = launch_t1<LP, false>(b, pb, st);
+    mdbf_status_t rc = launch_t1<LP>(b, pb, st);
     if (rc) return rc;
     TxArgs s = {};
     s.wk = L.wkA; s.rows_pad = L.rpA; s.rows = d.d_out; s.cols = d.k;
     s.vtile = L.vxA; s.U = L.UA; s.env_dtype = d.env_dtype; s.l = d.l;
-    s.in = L.zsum; s.out = y;
+    s.in = L.zsum; s.out = y; s.stage_a = 1;
     s.nkb_total = ceil_div(d.k, 64); s.kb_per_cta = pa.kb_per_cta;
     s.nastages = pa.nastages; s.nsstages = pa.nsstages; s.tmem_cols = pa.tmem_cols; s.status = L.status;
-    return launch_t1<LP, true>(s, pa, st);
+    return launch_t1<LP>(s, pa, st);
 }
 
 bool tmem_path_supports(const Layer &L, int T) {
