@@ -43,7 +43,9 @@ struct Layer {
     int NT;                       // 8-column mode tiles in the fragment copies: 1, 2, 4 or 8
     // TMEM-operand small-T kernel (16-bit envelopes, l <= 32): V in MMA k order, 16-bit, [kblocks][LP][64]
     uint16_t *vpA, *vpB;
-    uint16_t *vxA, *vxB;          // bf16 V tile images for the one-token kernel: [kblocks][max(LP,16)][64], swizzled
+    uint16_t *vxA, *vxB;          // bf16 V tile images for the one-token kernel: [kb_pad][max(LP,16)][64], swizzled
+    uint2 *wk2A, *wk2B;           // sign words, row-block major [row block][kb_pad][128] (one-token kernel)
+    int kbpA, kbpB;               // K blocks per row block in wk2 / vx (even, zero padded)
     // large-T kernel (present only when max_T exceeds the small-T kernel's range and l <= 32):
     int LP;                       // l rounded up to a power of two
     uint2 *wkA, *wkB;             // K-blocked sign words [kblocks][rows_pad128] (tcgen05 kernels)
@@ -116,6 +118,9 @@ mdbf_status_t launch_forward_tmem(Layer &L, const void *x, void *y, int T, cudaS
 bool tmem_path_supports(const Layer &L, int T);
 mdbf_status_t launch_vperm(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int LP,
                            cudaStream_t st);
+mdbf_status_t launch_forward_tmem_t1(Layer &L, const void *x, void *y, cudaStream_t st);
+mdbf_status_t launch_wk2(const uint32_t *canon, int rows, int nwords, uint2 *out, int rblocks, int kb_pad,
+                         cudaStream_t st);
 mdbf_status_t launch_vtile(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int NB,
                            cudaStream_t st);
 mdbf_status_t launch_zsum(Layer &L, int T, cudaStream_t st);

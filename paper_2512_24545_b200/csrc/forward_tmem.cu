@@ -39,14 +39,13 @@
 // returns.  No TMA multicast is used.
 #include <cooperative_groups.h>
 
-#include "common.cuh"
+#include "tmem_ptx.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace mdbf {
 
 constexpr int TM_EXPANDERS = 256;                      // two groups of 4 warps: even / odd K blocks
-constexpr int TM_ISSUERS = 4;                          // issuer/producer warps, one accumulator each
 constexpr int TM_THREADS = TM_EXPANDERS + TM_ISSUERS * 32 + 64;   // + sign loader warp + V loader warp
 constexpr int TM_W_ISSUER0 = TM_EXPANDERS / 32;        // first issuer warp
 constexpr int TM_VSTAGES = 8;                          // V ring (two per issuer warp)
@@ -54,7 +53,6 @@ constexpr int TM_MAX_SSTAGES = 32;                     // sign ring, 1 KB per st
 constexpr int TM_MAX_ASTAGES = 12;                     // A stages in TMEM, 32 columns each (6 when TMEM is shared)
 constexpr int TM_MAX_N = 64;
 constexpr int TM_MAX_T = 16;
-constexpr uint32_t TM_MAX_POLLS = 1u << 21;
 
 struct TmArgs {
     const uint2 *wk;          // K-blocked sign words [kblocks][rows_pad]
@@ -74,129 +72,6 @@ struct TmArgs {
     int32_t *status;
 };
 
-// ------------------------------------------------------------------ PTX wrappers
-namespace tm {
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status) {
-    for (uint32_t it = 0; it < TM_MAX_POLLS; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 255u && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    atomicExch(status, (int32_t)MDBF_ERR_TIMEOUT);
-    return false;
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
-__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(dst_smem), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(taddr), "r"(ncols) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
-}
-// contiguous global -> this CTA's shared memory, completion on an mbarrier (no multicast)
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n"
-        ::"r"(taddr),
-          "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
-          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
-          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
-        : "memory");
-}
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&v)[8]) {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};\n"
-                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
-}
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
-
-// K-major shared-memory operand, 128-byte rows, 128B swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
-    d |= (uint64_t)1u << 16;
-    d |= (uint64_t)((1024u >> 4) & 0x3FFFu) << 32;
-    d |= (uint64_t)1u << 46;
-    d |= (uint64_t)2u << 61;
-    return d;
-}
-__device__ __forceinline__ uint32_t make_idesc(int n) {
-    uint32_t d = 0;
-    d |= 1u << 4;                       // D: fp32
-    d |= 1u << 7;                       // A: bf16
-    d |= 1u << 10;                      // B: bf16
-    d |= (uint32_t)(n >> 3) << 17;      // N
-    d |= (uint32_t)(128 >> 4) << 24;    // M
-    return d;
-}
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&v);
-}
-template <bool ENV_BF16> __device__ __forceinline__ float env16(uint32_t h) {
-    if (ENV_BF16) return __uint_as_float(h << 16);
-    return __half2float(__ushort_as_half((unsigned short)h));
-}
-// After an expired wait the loaders stop issuing; this bounded pause (about a millisecond) lets
-// the bulk copies already in flight land before the CTA gives its shared memory back.
-__device__ __forceinline__ void drain_delay() {
-    const long long t0 = clock64();
-    while (clock64() - t0 < 2000000ll) {}
-}
-}  // namespace tm
 
 // Shared-memory plan (dynamic, 1024-byte aligned):
 //   bbuf   [4 issuers][2][n_mma * 128 B]      B tiles
@@ -541,353 +416,6 @@ mdbf_status_t launch_vperm(const void *V, int cols, int l, int env_dtype, uint16
     return MDBF_OK;
 }
 
-// =====================================================================================
-// One token (T = 1): the activation moves into the A operand.
-//
-//     D[r][t] = sum_c  ( S[r][c] * in[c] ) * V[c][t]
-//
-// A[r][c] is the bf16 activation with the packed bit XOR-ed into its sign (the same shift + one
-// logic op per two bits as the +-1 expansion), B is V itself: immutable, kept as ready-made
-// 128B-swizzled bf16 tile images (vtile_kernel) that a bulk copy drops straight into the B stage.
-// No B tile is built at run time, everything except the activation slice is in flight before the
-// dependency wait, and the issuer warps only issue.  One tcgen05.commit per K block releases the
-// A stage and the V stage together (same ring index).
-constexpr int TX_GROUPS = 2;                           // expander groups of 4 warps; group g takes K blocks g, g + 2, ...
-constexpr int TX_EXPANDERS = TX_GROUPS * 128;
-constexpr int TX_W_ISSUER0 = TX_EXPANDERS / 32;
-constexpr int TX_THREADS = TX_EXPANDERS + TM_ISSUERS * 32 + 64;   // 448: two CTAs fit on an SM
-
-struct TxArgs {
-    const uint2 *wk;          // K-blocked sign words [kblocks][rows_pad]
-    int rows_pad;
-    int rows, cols;
-    const uint16_t *vtile;    // bf16 V tile images [kblocks][NB * 64], 128B-swizzled, NB = max(LP, 16)
-    const void *U;            // [rows][l] env_dtype
-    int env_dtype, l;
-    const void *in;           // stage B: bf16 x [cols]; stage A: fp32 z [cols]
-    void *out;                // stage B: fp32 z [rows]; stage A: bf16 y [rows]
-    int nkb_total, kb_per_cta;
-    int nastages, nsstages, tmem_cols;
-    int stage_a;              // 0: stage B (bf16 in, fp32 out), 1: stage A (fp32 in, bf16 out); one kernel for both keeps its code hot
-    int32_t *status;
-};
-
-// Shared-memory plan (dynamic, 1024-byte aligned):
-//   vring [nastages][NB * 128 B]   V tile images (B operand)
-//   sring [nsstages][1024 B]       packed sign words
-//   xp    [kb_per_cta * 32] u32    activation pairs in MMA k order (bf16x2)
-//   part  [128] float              partial outputs (cluster reduction)
-template <int LP>
-__global__ void __launch_bounds__(TX_THREADS, LP <= 16 ? 2 : 1) tmem_t1_kernel(const TxArgs a) {
-    using namespace tm;
-    const bool STAGE_A = a.stage_a != 0;
-    constexpr int NB = LP < 16 ? 16 : LP;                    // MMA N
-    constexpr int VBYTES = NB * 128;
-    extern __shared__ unsigned char tm_smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * TM_MAX_SSTAGES + 3 * TM_MAX_ASTAGES + 1];
-    __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag_s;
-    volatile int *abort_flag = &abort_flag_s;
-
-    cg::cluster_group cluster = cg::this_cluster();
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t smem_base = (smem_u32(tm_smem_raw) + 1023u) & ~1023u;
-    unsigned char *smem_gen = tm_smem_raw + (smem_base - smem_u32(tm_smem_raw));
-    const int nas = a.nastages, nss = a.nsstages;
-    const uint32_t off_s = (uint32_t)(nas * VBYTES);
-    const uint32_t off_x = off_s + (uint32_t)(nss * 1024);
-    const uint32_t off_p = off_x + (uint32_t)(a.kb_per_cta * 128);
-    uint32_t *xp = reinterpret_cast<uint32_t *>(smem_gen + off_x);
-    float *part = reinterpret_cast<float *>(smem_gen + off_p);
-
-    constexpr int NB0 = TM_MAX_SSTAGES, NB1 = 2 * TM_MAX_SSTAGES, NB2 = NB1 + TM_MAX_ASTAGES,
-                  NB3 = NB2 + TM_MAX_ASTAGES, NB4 = NB3 + TM_MAX_ASTAGES;
-    const uint32_t s_full = smem_u32(&bars[0]), s_empty = smem_u32(&bars[NB0]), v_full = smem_u32(&bars[NB1]),
-                   a_full = smem_u32(&bars[NB2]), a_empty = smem_u32(&bars[NB3]), acc_bar = smem_u32(&bars[NB4]);
-
-    const int row0 = blockIdx.x * 128;
-    const int kb0 = blockIdx.y * a.kb_per_cta;
-    const int nkb = max(0, min(a.kb_per_cta, a.nkb_total - kb0));
-
-    if (tid <= NB4) {       // s_full 1, s_empty 4, v_full 1, a_full 4, a_empty 1, acc_bar TM_ISSUERS
-        const uint32_t count = tid < NB0 ? 1u : tid < NB1 ? 4u : tid < NB2 ? 1u : tid < NB3 ? 4u : tid < NB4 ? 1u
-                                                                                                      : (uint32_t)TM_ISSUERS;
-        mbar_init(smem_u32(&bars[tid]), count);
-    }
-    if (tid == 0) abort_flag_s = 0;
-    fence_barrier_init();
-    if (warp == TX_W_ISSUER0) {
-        tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)a.tmem_cols);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = tmem_base_slot;
-    const uint32_t tmem_a0 = tmem + (uint32_t)(TM_ISSUERS * NB);
-
-    pdl_launch_dependents();
-
-    const int row_l = (warp & 3) * 32 + lane;
-    float outv = 0.f;
-
-    if (warp < TX_W_ISSUER0) {
-        // ============================ expanders, then epilogue ============================
-        const int grp = warp >> 2;
-        const int grow = row0 + row_l;
-        float u[LP];
-#pragma unroll
-        for (int t = 0; t < LP; ++t)
-            u[t] = (grp == 0 && grow < a.rows && t < a.l) ? env_load(a.U, (size_t)grow * a.l + t, a.env_dtype) : 0.f;
-        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-
-        // stage the activation slice as bf16 pairs in MMA k order: pair `col` of a K block holds
-        // columns 32*(col/16) + col%16 and that + 16; four pairs per thread and step
-        pdl_wait();
-        {
-            const int c0 = kb0 * 64;
-            const int quads = a.kb_per_cta * 8;
-            const bool vec = (a.cols & 3) == 0 && (reinterpret_cast<uintptr_t>(a.in) & 15u) == 0;
-            for (int q = tid; q < quads; q += TX_EXPANDERS) {
-                const int kbl = q >> 3, col = (q & 7) << 2;
-                const int c_lo = c0 + kbl * 64 + 32 * (col >> 4) + (col & 15);
-                float lo[4], hi[4];
-                if (vec && c_lo + 20 <= a.cols) {
-                    if (STAGE_A) {
-                        const float4 l4 = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(a.in) + c_lo);
-                        const float4 h4 = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(a.in) + c_lo + 16);
-                        lo[0] = l4.x; lo[1] = l4.y; lo[2] = l4.z; lo[3] = l4.w;
-                        hi[0] = h4.x; hi[1] = h4.y; hi[2] = h4.z; hi[3] = h4.w;
-                    } else {
-                        const uint2 l2 = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(a.in) + c_lo);
-                        const uint2 h2 = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(a.in) + c_lo + 16);
-                        lo[0] = __uint_as_float(l2.x << 16); lo[1] = __uint_as_float(l2.x & 0xFFFF0000u);
-                        lo[2] = __uint_as_float(l2.y << 16); lo[3] = __uint_as_float(l2.y & 0xFFFF0000u);
-                        hi[0] = __uint_as_float(h2.x << 16); hi[1] = __uint_as_float(h2.x & 0xFFFF0000u);
-                        hi[2] = __uint_as_float(h2.y << 16); hi[3] = __uint_as_float(h2.y & 0xFFFF0000u);
-                    }
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int cl = c_lo + e, ch = c_lo + 16 + e;
-                        lo[e] = 0.f; hi[e] = 0.f;
-                        if (STAGE_A) {
-                            if (cl < a.cols) lo[e] = reinterpret_cast<const float *>(a.in)[cl];
-                            if (ch < a.cols) hi[e] = reinterpret_cast<const float *>(a.in)[ch];
-                        } else {
-                            if (cl < a.cols) lo[e] = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(a.in)[cl]);
-                            if (ch < a.cols) hi[e] = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(a.in)[ch]);
-                        }
-                    }
-                }
-                *reinterpret_cast<uint4 *>(xp + kbl * 32 + col) =
-                    make_uint4(pack_bf16x2(lo[0], hi[0]), pack_bf16x2(lo[1], hi[1]), pack_bf16x2(lo[2], hi[2]),
-                               pack_bf16x2(lo[3], hi[3]));
-            }
-        }
-        asm volatile("bar.sync 2, %0;\n" ::"n"(TX_EXPANDERS) : "memory");
-
-        // Per K block: the packed words of the NEXT block and the activation pairs of this one are
-        // requested first, then the previous block's TMEM stores are retired, then 4 x (8 logic ops +
-        // one 8-column TMEM store); the loads overlap the waits instead of heading a serial chain.
-        bool alive = true;
-        int rs = grp % nss, as = grp % nas;
-        uint32_t rs_ph = (uint32_t)(grp / nss) & 1u, as_ph = (uint32_t)(grp / nas) & 1u;
-        int prev_as = -1;
-        uint2 w = make_uint2(0u, 0u);
-        if (grp < nkb) {
-            alive = mbar_wait(s_full + 8 * rs, rs_ph, abort_flag, a.status);
-            if (alive) {
-                w = *reinterpret_cast<const uint2 *>(smem_gen + off_s + rs * 1024 + row_l * 8);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(s_empty + 8 * rs);
-            }
-        }
-        for (int kb = grp; kb < nkb && alive; kb += TX_GROUPS) {
-            const uint4 *xq = reinterpret_cast<const uint4 *>(xp + kb * 32);
-            uint4 xr[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) xr[q] = xq[q];
-            uint2 w_next = make_uint2(0u, 0u);
-            if (kb + TX_GROUPS < nkb) {
-                rs += TX_GROUPS; while (rs >= nss) { rs -= nss; rs_ph ^= 1u; }
-                alive = mbar_wait(s_full + 8 * rs, rs_ph, abort_flag, a.status);
-                if (!alive) break;
-                w_next = *reinterpret_cast<const uint2 *>(smem_gen + off_s + rs * 1024 + row_l * 8);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(s_empty + 8 * rs);
-            }
-            if (prev_as >= 0) {
-                tmem_st_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(a_full + 8 * prev_as);
-            }
-            alive = mbar_wait(a_empty + 8 * as, as_ph ^ 1u, abort_flag, a.status);
-            if (!alive) break;
-            tc_fence_after();
-            const uint32_t a_col = tmem_a0 + lane_base + (uint32_t)(as * 32);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {                    // TMEM columns 8q .. 8q+7 = pairs 8q .. 8q+7
-                const uint32_t word = q < 2 ? w.x : w.y;
-                const uint32_t xs8[8] = {xr[2 * q].x, xr[2 * q].y, xr[2 * q].z, xr[2 * q].w,
-                                         xr[2 * q + 1].x, xr[2 * q + 1].y, xr[2 * q + 1].z, xr[2 * q + 1].w};
-                uint32_t v[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int i = (q & 1) * 8 + e;           // bits (i, i + 16) of the word
-                    v[e] = ((word << (15 - i)) & 0x80008000u) ^ xs8[e];
-                }
-                tmem_st8(a_col + (uint32_t)(8 * q), v);
-            }
-            prev_as = as;
-            as += TX_GROUPS; while (as >= nas) { as -= nas; as_ph ^= 1u; }
-            w = w_next;
-        }
-        tmem_st_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (alive && prev_as >= 0 && lane == 0) mbar_arrive(a_full + 8 * prev_as);
-        if (grp != 0) alive = false;
-        if (alive) alive = mbar_wait(acc_bar, 0u, abort_flag, a.status);
-        tc_fence_after();
-        if (alive) {
-            const int nacc = nkb < TM_ISSUERS ? nkb : TM_ISSUERS;
-#pragma unroll
-            for (int cc = 0; cc < NB / 16; ++cc) {
-                uint32_t d[TM_ISSUERS][16];
-#pragma unroll
-                for (int acc = 0; acc < TM_ISSUERS; ++acc)
-                    if (acc < nacc) tmem_ld16(tmem + lane_base + (uint32_t)(acc * NB + cc * 16), d[acc]);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    float sum = 0.f;
-#pragma unroll
-                    for (int acc = 0; acc < TM_ISSUERS; ++acc)
-                        if (acc < nacc) sum += __uint_as_float(d[acc][j]);
-                    if (cc * 16 + j < LP) outv += u[(cc * 16 + j) % LP] * sum;
-                }
-            }
-        }
-        if (grp == 0) part[row_l] = outv;
-    } else if (warp < TX_W_ISSUER0 + TM_ISSUERS) {
-        // ================================== MMA issuers ===================================
-        const int w = warp - TX_W_ISSUER0;
-        const uint32_t idesc = make_idesc(NB);
-        const uint32_t d_tmem = tmem + (uint32_t)(w * NB);
-        bool alive = true;
-        int it = 0;
-        int as = w % nas;
-        uint32_t as_ph = (uint32_t)(w / nas) & 1u;
-        for (int kb = w; kb < nkb && alive; kb += TM_ISSUERS, ++it) {
-            alive = mbar_wait(v_full + 8 * as, as_ph, abort_flag, a.status);
-            if (!alive) break;
-            alive = mbar_wait(a_full + 8 * as, as_ph, abort_flag, a.status);
-            if (!alive) break;
-            tc_fence_after();
-            if (lane == 0) {
-                const uint64_t bdesc = make_smem_desc(smem_base + (uint32_t)(as * VBYTES));
-                const uint32_t a_t = tmem_a0 + (uint32_t)(as * 32);
-#pragma unroll
-                for (int k4 = 0; k4 < 4; ++k4)
-                    umma_ts(d_tmem, a_t + (uint32_t)(8 * k4), bdesc + (uint64_t)(2 * k4), idesc, (it > 0 || k4 > 0) ? 1u : 0u);
-                umma_commit(a_empty + 8 * as);               // frees the A stage and the V stage
-            }
-            __syncwarp();
-            as += TM_ISSUERS;
-            while (as >= nas) { as -= nas; as_ph ^= 1u; }
-        }
-        if (lane == 0) {
-            if (alive && it > 0) umma_commit(acc_bar);
-            else mbar_arrive(acc_bar);
-        }
-        __syncwarp();
-    } else if (warp == TX_W_ISSUER0 + TM_ISSUERS) {
-        // ============================== sign-word loader ================================
-        if (lane == 0) {
-            bool alive = true;
-            int rs = 0;
-            uint32_t ph = 0;
-            for (int kb = 0; kb < nkb && alive; ++kb) {
-                alive = mbar_wait(s_empty + 8 * rs, ph ^ 1u, abort_flag, a.status);
-                if (!alive) break;
-                mbar_arrive_expect_tx(s_full + 8 * rs, 1024u);
-                bulk_load(smem_base + off_s + (uint32_t)(rs * 1024), a.wk + (size_t)(kb0 + kb) * a.rows_pad + row0, 1024u,
-                          s_full + 8 * rs);
-                if (++rs == nss) { rs = 0; ph ^= 1u; }
-            }
-            if (!alive) drain_delay();
-        }
-        __syncwarp();
-    } else {
-        // ================================ V-tile loader ==================================
-        if (lane == 0) {
-            bool alive = true;
-            int vs = 0;
-            uint32_t ph = 0;
-            for (int kb = 0; kb < nkb && alive; ++kb) {
-                alive = mbar_wait(a_empty + 8 * vs, ph ^ 1u, abort_flag, a.status);
-                if (!alive) break;
-                mbar_arrive_expect_tx(v_full + 8 * vs, (uint32_t)VBYTES);
-                bulk_load(smem_base + (uint32_t)(vs * VBYTES), a.vtile + (size_t)(kb0 + kb) * NB * 64, (uint32_t)VBYTES,
-                          v_full + 8 * vs);
-                if (++vs == nas) { vs = 0; ph ^= 1u; }
-            }
-            if (!alive) drain_delay();
-        }
-        __syncwarp();
-    }
-
-    // ------------------------------ cluster reduction and store ------------------------------
-    tc_fence_before();
-    cluster.sync();
-    if (warp < 4 && cluster.block_rank() == 0) {
-        const unsigned nranks = cluster.num_blocks();
-        float rv[8];
-#pragma unroll
-        for (unsigned rk = 1; rk < 8; ++rk) rv[rk] = rk < nranks ? cluster.map_shared_rank(part, rk)[row_l] : 0.f;
-#pragma unroll
-        for (unsigned rk = 1; rk < 8; ++rk) outv += rv[rk];
-        const int grow = row0 + row_l;
-        if (grow < a.rows && !*abort_flag) {
-            if (STAGE_A) reinterpret_cast<__nv_bfloat16 *>(a.out)[grow] = __float2bfloat16_rn(outv);
-            else reinterpret_cast<float *>(a.out)[grow] = outv;
-        }
-    }
-    cluster.sync();
-    if (warp == TX_W_ISSUER0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
-}
-
-// bf16 V tile images for the one-token kernel: K block kb is NB rows (modes) x 64 k, K-major with
-// 128-byte rows and the 128B swizzle; element (t, p) holds V[c][t], c = kb*64 + 32*(p/32) + (p%32)/2
-// + 16*(p%2), at 16-bit index kb*NB*64 + t*64 + ((p/8) ^ (t%8))*8 + p%8; zero outside the matrix.
-__global__ void vtile_kernel(const void *__restrict__ V, int cols, int l, int env_dtype, uint16_t *__restrict__ out,
-                             int kblocks, int NB) {
-    const size_t total = (size_t)kblocks * NB * 64;
-    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
-        const int p = (int)(idx & 63);
-        const int t = (int)((idx >> 6) % NB);
-        const int kb = (int)((idx >> 6) / NB);
-        const int c = kb * 64 + 32 * (p >> 5) + ((p & 31) >> 1) + 16 * (p & 1);
-        float v = 0.f;
-        if (c < cols && t < l) v = env_load(V, (size_t)c * l + t, env_dtype);
-        const __nv_bfloat16 b = __float2bfloat16_rn(v);
-        out[(size_t)kb * NB * 64 + t * 64 + (((p >> 3) ^ (t & 7)) << 3) + (p & 7)] = *reinterpret_cast<const uint16_t *>(&b);
-    }
-}
-
-mdbf_status_t launch_vtile(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int NB,
-                           cudaStream_t st) {
-    const size_t total = (size_t)kblocks * NB * 64;
-    int grid = (int)((total + 255) / 256);
-    if (grid > 148 * 16) grid = 148 * 16;
-    if (grid < 1) grid = 1;
-    vtile_kernel<<<grid, 256, 0, st>>>(V, cols, l, env_dtype, out, kblocks, NB);
-    MDBF_CUDA(cudaGetLastError());
-    return MDBF_OK;
-}
-
 // ---------------------------------------------------------------------- launch
 struct TmPlan {
     int ks, kb_per_cta, nastages, nsstages, tmem_cols, n_mma;
@@ -931,85 +459,6 @@ static bool plan_stage(int rows, int cols, int LP, int T, TmPlan *p) {
     p->smem = 1024 + (size_t)TM_ISSUERS * 2 * n_mma * 128 + (size_t)TM_VSTAGES * LP * 128 + (size_t)p->nsstages * 1024 +
               (size_t)T * p->kb_per_cta * 64 * 4 + (size_t)T * 128 * 4;
     return p->smem <= 220 * 1024;
-}
-
-// One-token plan: cluster size along the reduction (see plan_stage), ring depths, TMEM columns.
-static bool plan_t1(int rows, int cols, int LP, TmPlan *p) {
-    const int NB = LP < 16 ? 16 : LP;
-    const int rb = ceil_div(rows, 128), nkb = ceil_div(cols, 64);
-    const int acc_cols = TM_ISSUERS * NB;
-    const int tmem_cols = (acc_cols + 4 * 32 <= 256) ? 256 : 512;    // half of TMEM when it fits: two CTAs per SM
-    int nas = (tmem_cols - acc_cols) / 32;
-    if (nas > TM_MAX_ASTAGES) nas = TM_MAX_ASTAGES;
-    long best_cost = -1;
-    int best_ks = 0;
-    for (int ks = 1; ks <= 8; ks *= 2) {
-        const int per = ceil_div(nkb, ks);
-        if (ks > 1 && per * (ks - 1) >= nkb) continue;
-        const long waves = ceil_div(rb * ks, tmem_cols <= 256 ? 296 : 148);   // CTAs that fit at once
-        const long cost = waves * (per + 16);
-        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ks = ks; }
-    }
-    p->ks = best_ks;
-    p->kb_per_cta = ceil_div(nkb, best_ks);
-    p->nastages = nas;
-    p->nsstages = p->kb_per_cta < TM_MAX_SSTAGES ? p->kb_per_cta : TM_MAX_SSTAGES;
-    if (p->nsstages < 2) p->nsstages = 2;
-    p->tmem_cols = tmem_cols;
-    p->n_mma = NB;
-    p->smem = 1024 + (size_t)nas * NB * 128 + (size_t)p->nsstages * 1024 + (size_t)p->kb_per_cta * 128 + 512;
-    return p->smem <= 220 * 1024;
-}
-
-template <int LP>
-static mdbf_status_t launch_t1(const TxArgs &a, const TmPlan &p, cudaStream_t st) {
-    auto kern = tmem_t1_kernel<LP>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        MDBF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
-        attr_set = true;
-    }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(ceil_div(a.rows, 128), p.ks, 1);
-    cfg.blockDim = dim3(TX_THREADS);
-    cfg.dynamicSmemBytes = p.smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1;
-    attr[0].val.clusterDim.y = p.ks;
-    attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
-    MDBF_CUDA(cudaLaunchKernelEx(&cfg, kern, a));
-    return MDBF_OK;
-}
-
-template <int LP>
-static mdbf_status_t run_t1(Layer &L, const void *x, void *y, cudaStream_t st) {
-    const mdbf_desc_t &d = L.d;
-    TmPlan pb, pa;
-    if (!plan_t1(d.k, d.d_in, LP, &pb) || !plan_t1(d.d_out, d.k, LP, &pa)) {
-        set_error("mdbf_linear_forward: the one-token TMEM kernel does not fit this shape");
-        return MDBF_ERR_SHAPE;
-    }
-    TxArgs b = {};
-    b.wk = L.wkB; b.rows_pad = L.rpB; b.rows = d.k; b.cols = d.d_in;
-    b.vtile = L.vxB; b.U = L.UB; b.env_dtype = d.env_dtype; b.l = d.l;
-    b.in = x; b.out = L.zsum; b.stage_a = 0;
-    b.nkb_total = ceil_div(d.d_in, 64); b.kb_per_cta = pb.kb_per_cta;
-    b.nastages = pb.nastages; b.nsstages = pb.nsstages; b.tmem_cols = pb.tmem_cols; b.status = L.status;
-    mdbf_status_t rc = launch_t1<LP>(b, pb, st);
-    if (rc) return rc;
-    TxArgs s = {};
-    s.wk = L.wkA; s.rows_pad = L.rpA; s.rows = d.d_out; s.cols = d.k;
-    s.vtile = L.vxA; s.U = L.UA; s.env_dtype = d.env_dtype; s.l = d.l;
-    s.in = L.zsum; s.out = y; s.stage_a = 1;
-    s.nkb_total = ceil_div(d.k, 64); s.kb_per_cta = pa.kb_per_cta;
-    s.nastages = pa.nastages; s.nsstages = pa.nsstages; s.tmem_cols = pa.tmem_cols; s.status = L.status;
-    return launch_t1<LP>(s, pa, st);
 }
 
 bool tmem_path_supports(const Layer &L, int T) {
@@ -1077,14 +526,7 @@ mdbf_status_t launch_forward_tmem(Layer &L, const void *x, void *y, int T, cudaS
     const bool bf = L.d.env_dtype == MDBF_BF16;
     mdbf_status_t rc;
     if (T == 1 && L.vxA && L.vxB) {
-        switch (L.LP) {
-            case 1: rc = run_t1<1>(L, x, y, st); break;
-            case 2: rc = run_t1<2>(L, x, y, st); break;
-            case 4: rc = run_t1<4>(L, x, y, st); break;
-            case 8: rc = run_t1<8>(L, x, y, st); break;
-            case 16: rc = run_t1<16>(L, x, y, st); break;
-            default: rc = run_t1<32>(L, x, y, st); break;
-        }
+        rc = launch_forward_tmem_t1(L, x, y, st);
         if (rc) return rc;
         L.last_ksplit = 0;
         *launches = 2;

@@ -58,7 +58,7 @@ static mdbf_status_t check_handle(mdbf_handle_t h, const char *fn) {
 }
 
 static void free_layer(Layer &L) {
-    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.vpA, L.vpB, L.vxA, L.vxB, L.wkA, L.wkB, L.vtB, L.xsB, L.xsA, L.z, L.zsum, L.xstage, L.ystage, L.status};
+    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.vpA, L.vpB, L.vxA, L.vxB, L.wk2A, L.wk2B, L.wkA, L.wkB, L.vtB, L.xsB, L.xsA, L.z, L.zsum, L.xstage, L.ystage, L.status};
     for (void *p : ptrs)
         if (p) cudaFree(p);
 }
@@ -184,8 +184,11 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
         PACK_CUDA(cudaMalloc(&L.vpA, (size_t)(L.padA / 64) * L.LP * 64 * sizeof(uint16_t)));
         PACK_CUDA(cudaMalloc(&L.vpB, (size_t)(L.padB / 64) * L.LP * 64 * sizeof(uint16_t)));
         const int NB = L.LP < 16 ? 16 : L.LP;
-        PACK_CUDA(cudaMalloc(&L.vxA, (size_t)(L.padA / 64) * NB * 64 * sizeof(uint16_t)));
-        PACK_CUDA(cudaMalloc(&L.vxB, (size_t)(L.padB / 64) * NB * 64 * sizeof(uint16_t)));
+        L.kbpA = ceil_div(L.padA / 64, 2) * 2; L.kbpB = ceil_div(L.padB / 64, 2) * 2;
+        PACK_CUDA(cudaMalloc(&L.vxA, (size_t)L.kbpA * NB * 64 * sizeof(uint16_t)));
+        PACK_CUDA(cudaMalloc(&L.vxB, (size_t)L.kbpB * NB * 64 * sizeof(uint16_t)));
+        PACK_CUDA(cudaMalloc(&L.wk2A, (size_t)(L.rpA / 128) * L.kbpA * 128 * sizeof(uint2)));
+        PACK_CUDA(cudaMalloc(&L.wk2B, (size_t)(L.rpB / 128) * L.kbpB * 128 * sizeof(uint2)));
     }
     if (want_prefill) {
         L.xs_rows = ((size_t)d.max_T * L.LP + 255) / 256 * 256;
@@ -233,8 +236,10 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
         PACK_RC(launch_kblock(L.wB, d.k, L.wordsB, L.wkB, L.rpB, L.padB / 64, st));
         PACK_RC(launch_vperm(L.VA, d.k, d.l, d.env_dtype, L.vpA, L.padA / 64, L.LP, st));
         PACK_RC(launch_vperm(L.VB, d.d_in, d.l, d.env_dtype, L.vpB, L.padB / 64, L.LP, st));
-        PACK_RC(launch_vtile(L.VA, d.k, d.l, d.env_dtype, L.vxA, L.padA / 64, L.LP < 16 ? 16 : L.LP, st));
-        PACK_RC(launch_vtile(L.VB, d.d_in, d.l, d.env_dtype, L.vxB, L.padB / 64, L.LP < 16 ? 16 : L.LP, st));
+        PACK_RC(launch_vtile(L.VA, d.k, d.l, d.env_dtype, L.vxA, L.kbpA, L.LP < 16 ? 16 : L.LP, st));
+        PACK_RC(launch_vtile(L.VB, d.d_in, d.l, d.env_dtype, L.vxB, L.kbpB, L.LP < 16 ? 16 : L.LP, st));
+        PACK_RC(launch_wk2(L.wA, d.d_out, L.wordsA, L.wk2A, L.rpA / 128, L.kbpA, st));
+        PACK_RC(launch_wk2(L.wB, d.k, L.wordsB, L.wk2B, L.rpB / 128, L.kbpB, st));
     }
     if (want_prefill) {
         PACK_RC(launch_vtrans(L.VB, d.d_in, d.l, d.env_dtype, L.vtB, L.padB, L.LP, st));
