@@ -39,10 +39,11 @@ namespace cg = cooperative_groups;
 
 namespace mdbf {
 
-constexpr int TX_GROUPS = 4;                           // expander groups of 4 warps; group g takes pairs g, g + 4, ...
+constexpr int TX_GROUPS = 2;                           // expander groups of 4 warps; group g takes pairs g, g + 4, ...
+constexpr int TX_ISSUERS = 4;                          // MMA issuer warps, one accumulator each (a thread issues ~1 MMA / 100+ clk here)
 constexpr int TX_EXPANDERS = TX_GROUPS * 128;
 constexpr int TX_W_ISSUER0 = TX_EXPANDERS / 32;
-constexpr int TX_THREADS = TX_EXPANDERS + TM_ISSUERS * 32 + 64;   // + sign loader warp + V loader warp
+constexpr int TX_THREADS = TX_EXPANDERS + TX_ISSUERS * 32 + 64;   // + sign loader warp + V loader warp
 constexpr int TX_MAX_SSTAGES = 16;                     // sign ring: 2 KB per stage (one pair of K blocks)
 constexpr int TX_MAX_ASTAGES = 7;                      // A / V stages: 64 TMEM columns + two V tiles each
 
@@ -105,9 +106,9 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
     const int pr0 = blockIdx.y * a.pairs_per_cta;
     const int npr = max(0, min(a.pairs_per_cta, a.npairs_total - pr0));
 
-    if (tid <= NB4) {       // s_full 1, s_empty 4, v_full 1, a_full 4, a_empty 1, acc_bar TM_ISSUERS
+    if (tid <= NB4) {       // s_full 1, s_empty 4, v_full 1, a_full 4, a_empty 1, acc_bar TX_ISSUERS
         const uint32_t count = tid < NB0 ? 1u : tid < NB1 ? 4u : tid < NB2 ? 1u : tid < NB3 ? 4u : tid < NB4 ? 1u
-                                                                                                      : (uint32_t)TM_ISSUERS;
+                                                                                                      : (uint32_t)TX_ISSUERS;
         mbar_init(smem_u32(&bars[tid]), count);
     }
     if (tid == 0) abort_flag_s = 0;
@@ -120,7 +121,7 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
-    const uint32_t tmem_a0 = tmem + (uint32_t)(TM_ISSUERS * NB);
+    const uint32_t tmem_a0 = tmem + (uint32_t)(TX_ISSUERS * NB);
 
     pdl_launch_dependents();
 
@@ -232,27 +233,34 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
         if (alive) alive = mbar_wait(acc_bar, 0u, abort_flag, a.status);
         tc_fence_after();
         if (alive) {
-            const int nacc = npr < TM_ISSUERS ? npr : TM_ISSUERS;
+            const int nacc = npr < TX_ISSUERS ? npr : TX_ISSUERS;
 #pragma unroll
             for (int cc = 0; cc < NB / 16; ++cc) {
-                uint32_t d[TM_ISSUERS][16];
+                float sum[16];
 #pragma unroll
-                for (int acc = 0; acc < TM_ISSUERS; ++acc)
-                    if (acc < nacc) tmem_ld16(tmem + lane_base + (uint32_t)(acc * NB + cc * 16), d[acc]);
-                tmem_ld_wait();
+                for (int j = 0; j < 16; ++j) sum[j] = 0.f;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    float sum = 0.f;
+                for (int a4 = 0; a4 < TX_ISSUERS; a4 += 4) {             // four accumulators per round of loads
+                    uint32_t d[4][16];
 #pragma unroll
-                    for (int acc = 0; acc < TM_ISSUERS; ++acc)
-                        if (acc < nacc) sum += __uint_as_float(d[acc][j]);
-                    if (cc * 16 + j < LP) outv += u[(cc * 16 + j) % LP] * sum;
+                    for (int q = 0; q < 4; ++q)
+                        if (a4 + q < nacc) tmem_ld16(tmem + lane_base + (uint32_t)((a4 + q) * NB + cc * 16), d[q]);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (a4 + q < nacc) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) sum[j] += __uint_as_float(d[q][j]);
+                        }
                 }
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (cc * 16 + j < LP) outv += u[(cc * 16 + j) % LP] * sum[j];
             }
         }
         if (grp == 0) part[row_l] = outv;
     }
-    else if (warp < TX_W_ISSUER0 + TM_ISSUERS) {
+    else if (warp < TX_W_ISSUER0 + TX_ISSUERS) {
         // ================================== MMA issuers ===================================
         const int w = warp - TX_W_ISSUER0;
         const uint32_t idesc = make_idesc(NB);
@@ -261,7 +269,14 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
         int it = 0;
         int as = w % nas;
         uint32_t as_ph = (uint32_t)(w / nas) & 1u;
-        for (int pr = w; pr < npr; pr += TM_ISSUERS, ++it) {
+        // An issuer whose first pair already reuses a stage (w >= nas) has to see the earlier phases of
+        // that stage complete first: a parity test alone cannot tell phase n from phase n - 2.
+        if (w < npr)
+            for (int k = 0; k < w / nas && alive; ++k) {
+                alive = tx_wait(v_full + 8 * as, (uint32_t)k & 1u, abort_flag, a.status);
+                if (alive) alive = tx_wait(a_full + 8 * as, (uint32_t)k & 1u, abort_flag, a.status);
+            }
+        for (int pr = w; pr < npr && alive; pr += TX_ISSUERS, ++it) {
             alive = tx_wait(v_full + 8 * as, as_ph, abort_flag, a.status);
             if (!alive) break;
             alive = tx_wait(a_full + 8 * as, as_ph, abort_flag, a.status);
@@ -277,7 +292,7 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
                 umma_commit(a_empty + 8 * as);               // frees the A stage and the V stage together
             }
             __syncwarp();
-            as += TM_ISSUERS;
+            as += TX_ISSUERS;
             while (as >= nas) { as -= nas; as_ph ^= 1u; }
         }
         if (lane == 0) {
@@ -285,7 +300,7 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
             else mbar_arrive(acc_bar);
         }
         __syncwarp();
-    } else if (warp == TX_W_ISSUER0 + TM_ISSUERS) {
+    } else if (warp == TX_W_ISSUER0 + TX_ISSUERS) {
         // ============================== sign-word loader ================================
         if (lane == 0) {
             bool alive = true;
@@ -411,7 +426,7 @@ struct TxPlan {
 static bool plan_t1(int rows, int kb_pad, int LP, TxPlan *p) {
     const int NB = LP < 16 ? 16 : LP;
     const int rb = ceil_div(rows, 128), npairs = kb_pad / 2;
-    int nas = (512 - TM_ISSUERS * NB) / 64;
+    int nas = (512 - TX_ISSUERS * NB) / 64;                  // NB = 32 with 8 accumulators leaves 4 stages
     if (nas > TX_MAX_ASTAGES) nas = TX_MAX_ASTAGES;
     long best_cost = -1;
     int best_ks = 1;

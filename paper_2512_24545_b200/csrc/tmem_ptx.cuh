@@ -7,6 +7,7 @@ namespace mdbf {
 
 constexpr int TM_ISSUERS = 4;                          // MMA issuer warps, one accumulator each
 constexpr uint32_t TM_MAX_POLLS = 1u << 21;
+constexpr unsigned long long TM_MAX_WAIT_NS = 1000000000ull;   // one second per wait at most
 
 // ------------------------------------------------------------------ PTX wrappers
 namespace tm {
@@ -29,10 +30,23 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
+    return t;
+}
+// Bounded wait, in polls and in time (a failed try_wait may park the thread for a while, so the poll
+// count alone does not bound the time): false when it gave up (status word set, abort flag raised).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status) {
+    unsigned long long t0 = 0;
     for (uint32_t it = 0; it < TM_MAX_POLLS; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 255u && *abort_flag) return false;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > TM_MAX_WAIT_NS) break;
+        }
     }
     *abort_flag = 1;
     atomicExch(status, (int32_t)MDBF_ERR_TIMEOUT);
