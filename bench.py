@@ -39,6 +39,16 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
 
 
+def dominant_kernel(spec, T):
+    """Name of the kernel the library's dispatcher picks for this (l, T): the one the roofline line is about."""
+    lp = 1
+    while lp < spec.l:
+        lp *= 2
+    if T == 1:
+        return "tmem_t1_kernel"
+    return "gemm_stage_kernel"
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -275,7 +285,7 @@ def run_mdbf(args):
         "clocks": clocks,
         "roofline": {"bound": bound, "achieved": per_gpu, "peak": peak, "unit": unit,
                      "frac": per_gpu / peak, "peak_source": f"of {peak_kind}",
-                     "kernel": "decode_stage_kernel" if T <= 4 else "prefill_stage_kernel",
+                     "kernel": dominant_kernel(groups[0][0], T),
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -32,7 +32,11 @@
 // Every mbarrier wait is bounded: when it expires the kernel records MDBF_ERR_TIMEOUT in
 // the layer's status word, all roles fall through to the common exit, TMEM is released and
 // the kernel returns.  No TMA multicast is used anywhere.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace mdbf {
 
@@ -63,6 +67,7 @@ struct GemmArgs {
     int pad_next;
     // stage A only
     __nv_bfloat16 *y;        // [T][rows]
+    int kb_per_cta;          // K blocks per cluster rank (blockIdx.z); the ranks' partial outputs are reduced over DSMEM
     int32_t *status;
 };
 
@@ -97,6 +102,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     atomicExch(status, (int32_t)MDBF_ERR_TIMEOUT);
     return false;
 }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
@@ -171,7 +178,7 @@ __device__ __forceinline__ uint32_t sign_pair(uint32_t byte, int i) {
 }
 
 // ----------------------------------------------------------------- GEMM stage
-template <int LP, bool STAGE_A>
+template <int LP, bool STAGE_A, bool SPLIT>
 __global__ void __launch_bounds__(PF_THREADS, 1)
 gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs) {
     constexpr int TT = PF_BN / LP;              // tokens per CTA tile
@@ -191,7 +198,11 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
 
     const int row0 = blockIdx.x * PF_BM;
     const int tau0 = blockIdx.y * TT;
-    const int nkb = (a.cols + PF_BK - 1) / PF_BK;
+    const int nkb_total = (a.cols + PF_BK - 1) / PF_BK;
+    const int kb0 = SPLIT ? blockIdx.z * a.kb_per_cta : 0;   // this cluster rank's slice of the reduction
+    const int nkb = SPLIT ? max(0, min(a.kb_per_cta, nkb_total - kb0)) : nkb_total;
+    constexpr bool split = SPLIT;                            // the reduction is shared by the ranks of a cluster
+    cg::cluster_group cluster = cg::this_cluster();
 
     if (tid == 0) {
         for (int s = 0; s < PF_STAGES; ++s) {
@@ -210,12 +221,15 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_d = tmem_base_slot;
+    // Programmatic dependent launch: the next kernel may start its prologue now; whatever reads or
+    // overwrites data of the previous kernel (the Xs operand, z / Xs_next / y) waits for it below.
+    pdl_launch_dependents();
 
     if (warp < 4) {
         // ============================ sign-tile expanders ============================
         const int arow = tid;                                     // one row of the tile per thread
-        const uint2 *wp = a.wk + (size_t)row0 + arow;             // + kb * rows_pad
-        uint2 w_next = __ldg(wp);
+        const uint2 *wp = a.wk + (size_t)kb0 * a.rows_pad + (size_t)row0 + arow;   // + kb * rows_pad
+        uint2 w_next = nkb > 0 ? __ldg(wp) : make_uint2(0u, 0u);
         bool alive = true;
         for (int kb = 0; kb < nkb && alive; ++kb) {
             const int s = kb % PF_STAGES;
@@ -247,6 +261,22 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
         }
         if (alive) alive = mbar_wait(accum_bar, 0u, abort_flag, a.status);
         tc_fence_after();
+        pdl_wait();                                   // the stores below must follow the previous kernel's reads
+        // one finished output value: stored at once, or parked for the cluster reduction
+        float *part = reinterpret_cast<float *>(smem_gen);               // [token of the tile][128 rows]; the stages are idle now
+        auto emit = [&](int tau, float acc) {
+            if (egrow < a.rows && tau < a.T) {
+                if (STAGE_A) {
+                    a.y[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(acc);
+                } else {
+                    a.z[(size_t)tau * a.rows + egrow] = acc;
+                    __nv_bfloat16 *xo = a.xs_next + (size_t)tau * LP * a.pad_next + egrow;
+#pragma unroll
+                    for (int t2 = 0; t2 < LP; ++t2)
+                        xo[(size_t)t2 * a.pad_next] = __float2bfloat16_rn(vn[t2] * acc);
+                }
+            }
+        };
         if (alive) {
             float acc = 0.f;
 #pragma unroll 1
@@ -254,33 +284,46 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
                 const int col0 = ld * 32;
                 if (col0 >= a.n_eff) break;                              // warp-uniform
                 uint32_t v[32];
-                tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)col0, v);
-                tmem_ld_wait();
+                if (!SPLIT || nkb > 0) {
+                    tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)col0, v);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;              // an empty slice contributes nothing
+                }
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     const int t = j % LP;                // col0 is a multiple of 32 and LP divides 32
                     acc += u[t] * __uint_as_float(v[j]);
                     if (t == LP - 1) {
-                        const int tau = tau0 + (col0 + j) / LP;
-                        if (egrow < a.rows && tau < a.T) {
-                            if (STAGE_A) {
-                                a.y[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(acc);
-                            } else {
-                                a.z[(size_t)tau * a.rows + egrow] = acc;
-                                __nv_bfloat16 *xo = a.xs_next + (size_t)tau * LP * a.pad_next + egrow;
-#pragma unroll
-                                for (int t2 = 0; t2 < LP; ++t2)
-                                    xo[(size_t)t2 * a.pad_next] = __float2bfloat16_rn(vn[t2] * acc);
-                            }
-                        }
+                        const int tl = (col0 + j) / LP;
+                        if (split) part[tl * PF_BM + arow] = acc;
+                        else emit(tau0 + tl, acc);
                         acc = 0.f;
                     }
                 }
             }
         }
+        if (split) {
+            // the ranks of the cluster hold partial sums over their slices of the reduction: rank 0 adds
+            // them up in rank order (deterministic) through distributed shared memory and stores
+            tc_fence_before();
+            cluster.sync();
+            if (cluster.block_rank() == 0 && alive && !*abort_flag) {
+                const unsigned nranks = cluster.num_blocks();
+                const int ntl = a.n_eff / LP;
+                for (int tl = 0; tl < ntl; ++tl) {
+                    float acc = part[tl * PF_BM + arow];
+                    for (unsigned rk = 1; rk < nranks; ++rk) acc += cluster.map_shared_rank(part, rk)[tl * PF_BM + arow];
+                    emit(tau0 + tl, acc);
+                }
+            }
+            cluster.sync();
+        }
     } else if (warp == 4) {
         // ================================ TMA issuer =================================
         bool alive = true;
+        pdl_wait();                                   // Xs comes from the previous kernel
         for (int kb = 0; kb < nkb && alive; ++kb) {
             const int s = kb % PF_STAGES;
             const uint32_t ph = (uint32_t)(kb / PF_STAGES) & 1u;
@@ -289,7 +332,7 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
             if (lane == 0) {
                 mbar_arrive_expect_tx(full_bar + 8 * s, PF_B_BYTES);
                 tma_load_2d(smem_base + (uint32_t)s * PF_STAGE_BYTES + PF_A_BYTES, &tmap_xs,
-                            kb * PF_BK, tau0 * LP, full_bar + 8 * s);
+                            (kb0 + kb) * PF_BK, tau0 * LP, full_bar + 8 * s);
             }
             __syncwarp();
         }
@@ -315,8 +358,12 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
             }
             __syncwarp();
         }
-        if (lane == 0 && alive) umma_commit(accum_bar);
+        if (lane == 0 && alive) { if (nkb > 0) umma_commit(accum_bar); else mbar_arrive(accum_bar); }
         __syncwarp();
+    }
+    if (split && warp >= 4) {          // the expander warps run these two barriers inside their epilogue
+        cluster.sync();
+        cluster.sync();
     }
 
     tc_fence_before();
@@ -333,6 +380,8 @@ prescale_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ V
                 int T, int cols, int pad, int vec_ok) {
     const int chunks = pad / 8;
     const size_t total = (size_t)T * chunks;
+    pdl_launch_dependents();
+    pdl_wait();                                       // x may come from, and Xs may still be read by, earlier kernels
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (size_t)gridDim.x * blockDim.x) {
         const int tau = (int)(idx / chunks), c = (int)(idx % chunks) * 8;
@@ -440,16 +489,43 @@ mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows
 // ---------------------------------------------------------------------- launch
 template <int LP, bool STAGE_A>
 static mdbf_status_t launch_gemm(const GemmArgs &a, const CUtensorMap &tm, cudaStream_t st) {
-    auto kern = gemm_stage_kernel<LP, STAGE_A>;
     static bool attr_set = false;
     if (!attr_set) {
-        MDBF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
+        MDBF_CUDA(cudaFuncSetAttribute(gemm_stage_kernel<LP, STAGE_A, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
+        MDBF_CUDA(cudaFuncSetAttribute(gemm_stage_kernel<LP, STAGE_A, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
         attr_set = true;
     }
     const int TT = PF_BN / LP;
-    dim3 grid(ceil_div(a.rows, PF_BM), ceil_div(a.T, TT));
-    kern<<<grid, PF_THREADS, PF_SMEM_BYTES, st>>>(a, tm);
-    MDBF_CUDA(cudaGetLastError());
+    const int rb = ceil_div(a.rows, PF_BM), ntiles = ceil_div(a.T, TT), nkb = ceil_div(a.cols, PF_BK);
+    // Few tokens leave most SMs without a tile: split the reduction over a cluster of up to 8 CTAs
+    // (partial outputs reduced through DSMEM).  Cost model: waves x (K blocks per CTA + fixed part).
+    int best_ks = 1;
+    long best_cost = -1;
+    for (int ks = 1; ks <= 8; ks *= 2) {
+        const int per = ceil_div(nkb, ks);
+        if (ks > 1 && per * (ks - 1) >= nkb) continue;                 // an empty rank
+        const long waves = ceil_div((long)rb * ntiles * ks, 148);
+        const long cost = waves * (per + 10);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ks = ks; }
+    }
+    GemmArgs args = a;
+    args.kb_per_cta = ceil_div(nkb, best_ks);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(rb, ntiles, best_ks);
+    cfg.blockDim = dim3(PF_THREADS);
+    cfg.dynamicSmemBytes = PF_SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = best_ks;
+    cfg.attrs = attr;
+    cfg.numAttrs = best_ks > 1 ? 2 : 1;      // an unsplit launch keeps the plain block order (row blocks of a token tile run together)
+    if (best_ks > 1) MDBF_CUDA(cudaLaunchKernelEx(&cfg, gemm_stage_kernel<LP, STAGE_A, true>, args, tm));
+    else MDBF_CUDA(cudaLaunchKernelEx(&cfg, gemm_stage_kernel<LP, STAGE_A, false>, args, tm));
     return MDBF_OK;
 }
 
@@ -460,8 +536,19 @@ static mdbf_status_t run_prefill(Layer &L, const void *x, void *y, int T, cudaSt
     const int tok = T < TT ? T : TT;
     const int n_eff = ((tok * LP + 15) / 16) * 16;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(x) & 15u) == 0 && d.d_in % 8 == 0) ? 1 : 0;
-    prescale_kernel<LP><<<pf_grid((size_t)T * (L.padB / 8)), 256, 0, st>>>(
-        reinterpret_cast<const __nv_bfloat16 *>(x), L.vtB, L.xsB, T, d.d_in, L.padB, vec_ok);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(pf_grid((size_t)T * (L.padB / 8)));
+        cfg.blockDim = dim3(256);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        MDBF_CUDA(cudaLaunchKernelEx(&cfg, prescale_kernel<LP>, reinterpret_cast<const __nv_bfloat16 *>(x),
+                                     (const float *)L.vtB, L.xsB, T, d.d_in, L.padB, vec_ok));
+    }
     MDBF_CUDA(cudaGetLastError());
 
     GemmArgs b = {};

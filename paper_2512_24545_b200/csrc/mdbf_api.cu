@@ -176,7 +176,7 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     L.padA = ceil_div(d.k, 64) * 64; L.padB = ceil_div(d.d_in, 64) * 64;
     L.rpA = ceil_div(d.d_out, 128) * 128; L.rpB = ceil_div(d.k, 128) * 128;
     // the large-T kernel takes 16-bit envelopes and l <= 32; its scratch is sized by max_T
-    const bool want_prefill = d.env_dtype != MDBF_F32 && d.l <= 32 && d.max_T > kDecodeMaxT;
+    const bool want_prefill = d.env_dtype != MDBF_F32 && d.l <= 32 && d.max_T >= 2;
     const bool want_tc = d.env_dtype != MDBF_F32 && d.l <= 32;
     if (want_tc) {
         PACK_CUDA(cudaMalloc(&L.wkA, (size_t)(L.padA / 64) * L.rpA * sizeof(uint2)));
@@ -325,10 +325,13 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
     int kernel = h->kernel;
     const bool tc_ok = (act_dtype == MDBF_BF16) && (L.d.env_dtype != MDBF_F32) && L.d.l <= 32;
     if (kernel == MDBF_KERNEL_AUTO) {
+        // one token: TMEM-operand kernel; more: the tcgen05 GEMM (it splits the reduction over a
+        // cluster when few tokens would leave SMs idle); the others remain selectable
         if (!tc_ok) kernel = MDBF_KERNEL_ALU;
+        else if (T == 1 && tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
+        else if (L.xsB) kernel = MDBF_KERNEL_PREFILL;
         else if (tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
-        else if (T <= kDecodeMaxT) kernel = MDBF_KERNEL_DECODE;
-        else kernel = MDBF_KERNEL_PREFILL;
+        else kernel = MDBF_KERNEL_DECODE;
     }
     if (kernel != MDBF_KERNEL_ALU && !tc_ok) {
         set_error("mdbf_linear_forward: the tensor-core kernels need bf16 activations, 16-bit envelopes and l <= 32");
