@@ -373,18 +373,21 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
 
 // ------------------------------------------------------------------- pre-scale
 // Xs[(tau*LP + t) * pad + c] = bf16( Vt[t][c] * x[tau][c] ), zero for c >= cols.
-// One thread per (tau, 8 columns).
-template <int LP>
+// One thread per (tau, 8 columns) and, with TS > 1 (few tokens: more threads to cover the load
+// latency), per mode: thread handles LP / TS modes.
+template <int LP, int TS>
 __global__ void __launch_bounds__(256)
 prescale_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ Vt, __nv_bfloat16 *__restrict__ xs,
                 int T, int cols, int pad, int vec_ok) {
     const int chunks = pad / 8;
-    const size_t total = (size_t)T * chunks;
+    constexpr int MODES = LP / TS;
+    const size_t total = (size_t)T * chunks * TS;
     pdl_launch_dependents();
     pdl_wait();                                       // x may come from, and Xs may still be read by, earlier kernels
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (size_t)gridDim.x * blockDim.x) {
-        const int tau = (int)(idx / chunks), c = (int)(idx % chunks) * 8;
+        const int c = (int)(idx % chunks) * 8;
+        const int tg = (int)((idx / chunks) % TS), tau = (int)(idx / ((size_t)chunks * TS));
         float xv[8];
         if (vec_ok && c + 8 <= cols) {
             const uint4 r = __ldg(reinterpret_cast<const uint4 *>(x + (size_t)tau * cols + c));
@@ -399,7 +402,8 @@ prescale_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ V
             for (int i = 0; i < 8; ++i) xv[i] = (c + i < cols) ? __bfloat162float(x[(size_t)tau * cols + c + i]) : 0.f;
         }
 #pragma unroll
-        for (int t = 0; t < LP; ++t) {
+        for (int tm = 0; tm < MODES; ++tm) {
+            const int t = tg * MODES + tm;
             const float4 v0 = __ldg(reinterpret_cast<const float4 *>(Vt + (size_t)t * pad + c));
             const float4 v1 = __ldg(reinterpret_cast<const float4 *>(Vt + (size_t)t * pad + c + 4));
             uint4 o;
@@ -537,8 +541,9 @@ static mdbf_status_t run_prefill(Layer &L, const void *x, void *y, int T, cudaSt
     const int n_eff = ((tok * LP + 15) / 16) * 16;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(x) & 15u) == 0 && d.d_in % 8 == 0) ? 1 : 0;
     {
+        const bool few = (size_t)T * (L.padB / 8) < (size_t)148 * 256 * 4;     // few tokens: one thread per mode
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(pf_grid((size_t)T * (L.padB / 8)));
+        cfg.gridDim = dim3(pf_grid((size_t)T * (L.padB / 8) * (few ? LP : 1)));
         cfg.blockDim = dim3(256);
         cfg.stream = st;
         cudaLaunchAttribute attr[1];
@@ -546,8 +551,12 @@ static mdbf_status_t run_prefill(Layer &L, const void *x, void *y, int T, cudaSt
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        MDBF_CUDA(cudaLaunchKernelEx(&cfg, prescale_kernel<LP>, reinterpret_cast<const __nv_bfloat16 *>(x),
-                                     (const float *)L.vtB, L.xsB, T, d.d_in, L.padB, vec_ok));
+        if (few)
+            MDBF_CUDA(cudaLaunchKernelEx(&cfg, prescale_kernel<LP, LP>, reinterpret_cast<const __nv_bfloat16 *>(x),
+                                         (const float *)L.vtB, L.xsB, T, d.d_in, L.padB, vec_ok));
+        else
+            MDBF_CUDA(cudaLaunchKernelEx(&cfg, prescale_kernel<LP, 1>, reinterpret_cast<const __nv_bfloat16 *>(x),
+                                         (const float *)L.vtB, L.xsB, T, d.d_in, L.padB, vec_ok));
     }
     MDBF_CUDA(cudaGetLastError());
 
