@@ -54,7 +54,7 @@ struct Layer {
     float *vtB;                   // V_B transposed, fp32 [LP][padB]
     __nv_bfloat16 *xsB, *xsA;     // pre-scaled operands [xs_rows][padB], [xs_rows][padA]
     size_t xs_rows;               // max_T * LP rounded up to 256
-    CUtensorMap tmB, tmA;         // tensor maps of xsB / xsA
+    CUtensorMap tmB[3], tmA[3];   // tensor maps of xsB / xsA with boxes of 64, 128 and 256 rows (few tokens load a narrow box)
     // scratch
     float *z;                     // [kMaxKSplit][zT][k] stage-B partial sums of the small-T kernel
     size_t zstride;               // zT * k
@@ -106,7 +106,7 @@ mdbf_status_t launch_vfrag(const void *V, int cols, int l, int env_dtype, uint2 
 mdbf_status_t launch_kblock(const uint32_t *canon, int rows, int nwords, uint2 *out, int rows_pad, int kblocks,
                             cudaStream_t st);
 mdbf_status_t launch_vtrans(const void *V, int cols, int l, int env_dtype, float *out, int pad, int LP, cudaStream_t st);
-mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad);
+mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad, int box_rows);
 mdbf_status_t launch_reconstruct(const Layer &L, float *W, cudaStream_t st);
 mdbf_status_t launch_forward_alu(Layer &L, const void *x, void *y, int T, int act_dtype,
                                  cudaStream_t st, int *launches);

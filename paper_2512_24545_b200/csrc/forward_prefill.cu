@@ -67,6 +67,7 @@ struct GemmArgs {
     int pad_next;
     // stage A only
     __nv_bfloat16 *y;        // [T][rows]
+    int box_rows;            // rows of the TMA box of the Xs operand: 64, 128 or 256 (>= n_eff)
     int kb_per_cta;          // K blocks per cluster rank (blockIdx.z); the ranks' partial outputs are reduced over DSMEM
     int32_t *status;
 };
@@ -330,7 +331,7 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
             alive = mbar_wait(empty_bar + 8 * s, ph ^ 1u, abort_flag, a.status);
             if (!alive) break;
             if (lane == 0) {
-                mbar_arrive_expect_tx(full_bar + 8 * s, PF_B_BYTES);
+                mbar_arrive_expect_tx(full_bar + 8 * s, (uint32_t)a.box_rows * PF_BK * 2);
                 tma_load_2d(smem_base + (uint32_t)s * PF_STAGE_BYTES + PF_A_BYTES, &tmap_xs,
                             (kb0 + kb) * PF_BK, tau0 * LP, full_bar + 8 * s);
             }
@@ -461,7 +462,7 @@ mdbf_status_t launch_vtrans(const void *V, int cols, int l, int env_dtype, float
 }
 
 // Tensor map of a pre-scaled operand: bf16 [rows][pad] row-major, box 64 x 256, 128B swizzle.
-mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad) {
+mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad, int box_rows) {
     typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -478,7 +479,7 @@ mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows
     }
     const cuuint64_t gdim[2] = {(cuuint64_t)pad, (cuuint64_t)rows};
     const cuuint64_t gstride[1] = {(cuuint64_t)pad * 2};
-    const cuuint32_t box[2] = {PF_BK, PF_BN};
+    const cuuint32_t box[2] = {PF_BK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -564,14 +565,17 @@ static mdbf_status_t run_prefill(Layer &L, const void *x, void *y, int T, cudaSt
     b.wk = L.wkB; b.rows_pad = L.rpB; b.rows = d.k; b.cols = d.d_in;
     b.U = L.UB; b.env_dtype = d.env_dtype; b.l = d.l; b.T = T; b.n_eff = n_eff;
     b.z = L.zsum; b.Vnext = L.VA; b.xs_next = L.xsA; b.pad_next = L.padA; b.status = L.status;
-    mdbf_status_t rc = launch_gemm<LP, false>(b, L.tmB, st);
+    const int bi = n_eff <= 64 ? 0 : n_eff <= 128 ? 1 : 2;    // narrowest TMA box that covers the used columns
+    b.box_rows = 64 << bi;
+    mdbf_status_t rc = launch_gemm<LP, false>(b, L.tmB[bi], st);
     if (rc) return rc;
 
     GemmArgs a = {};
     a.wk = L.wkA; a.rows_pad = L.rpA; a.rows = d.d_out; a.cols = d.k;
     a.U = L.UA; a.env_dtype = d.env_dtype; a.l = d.l; a.T = T; a.n_eff = n_eff;
     a.y = reinterpret_cast<__nv_bfloat16 *>(y); a.status = L.status;
-    return launch_gemm<LP, true>(a, L.tmA, st);
+    a.box_rows = 64 << bi;
+    return launch_gemm<LP, true>(a, L.tmA[bi], st);
 }
 
 mdbf_status_t launch_forward_prefill(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches) {

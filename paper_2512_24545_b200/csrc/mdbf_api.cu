@@ -197,8 +197,10 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
         PACK_CUDA(cudaMalloc(&L.xsA, L.xs_rows * L.padA * 2));
         PACK_CUDA(cudaMemsetAsync(L.xsB, 0, L.xs_rows * L.padB * 2, st));
         PACK_CUDA(cudaMemsetAsync(L.xsA, 0, L.xs_rows * L.padA * 2, st));
-        PACK_RC(make_xs_tensor_map(&L.tmB, L.xsB, L.xs_rows, L.padB));
-        PACK_RC(make_xs_tensor_map(&L.tmA, L.xsA, L.xs_rows, L.padA));
+        for (int i = 0; i < 3; ++i) {
+            PACK_RC(make_xs_tensor_map(&L.tmB[i], L.xsB, L.xs_rows, L.padB, 64 << i));
+            PACK_RC(make_xs_tensor_map(&L.tmA[i], L.xsA, L.xs_rows, L.padA, 64 << i));
+        }
     }
     L.zstride = (size_t)decode_scratch_T(d) * d.k;
     PACK_CUDA(cudaMalloc(&L.z, (size_t)kMaxKSplit * L.zstride * sizeof(float)));
