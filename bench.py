@@ -36,7 +36,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that workload).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {
+    "decode_qproj": 1083648,                # tmem_t1_kernel, k = 1664 layer, either stage
+    "prefill_4096_l16_bpw10": 370142976,     # gemm_stage_kernel stage B: 269.4 MB read + 100.7 MB written
+}
 
 
 def dominant_kernel(spec, T):

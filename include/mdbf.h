@@ -60,11 +60,11 @@ typedef enum { MDBF_F32 = 0, MDBF_F16 = 1, MDBF_BF16 = 2 } mdbf_dtype_t;
 
 /* Kernel selector for mdbf_set_kernel. */
 typedef enum {
-    MDBF_KERNEL_AUTO = 0,   /* choose by (l, T, dtypes)                                         */
+    MDBF_KERNEL_AUTO = 0,   /* T = 1: TMEM path; T >= 2: PREFILL; fp32 / l > 32: ALU             */
     MDBF_KERNEL_ALU = 1,    /* fp32 CUDA-core path, sign applied by XOR of the IEEE sign bit      */
-    MDBF_KERNEL_DECODE = 2, /* small-T path: register bit->bf16 expansion + warp-level MMA        */
-    MDBF_KERNEL_PREFILL = 3, /* large-T path: tcgen05 MMA with TMEM accumulators                  */
-    MDBF_KERNEL_TMEM = 4    /* small-T path: tcgen05 MMA, sign operand expanded into TMEM         */
+    MDBF_KERNEL_DECODE = 2, /* T <= 4: register bit->bf16 expansion + warp-level MMA              */
+    MDBF_KERNEL_PREFILL = 3, /* T >= 2 (max_T >= 2): tcgen05 GEMM, TMEM accumulator, TMA operand   */
+    MDBF_KERNEL_TMEM = 4    /* l*T <= 64: tcgen05 MMA with the sign operand expanded into TMEM    */
 } mdbf_kernel_t;
 
 typedef struct {
