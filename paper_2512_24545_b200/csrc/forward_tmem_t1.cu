@@ -32,6 +32,7 @@
 // 32*(p/32) + (p%32)/2 + 16*(p%2).  Every mbarrier wait is bounded (MDBF_ERR_TIMEOUT in the
 // status word, all roles fall through, TMEM released).  No TMA multicast.
 #include <cooperative_groups.h>
+#include <cstdlib>
 
 #include "tmem_ptx.cuh"
 
@@ -421,6 +422,18 @@ struct TxPlan {
     size_t smem;
 };
 
+// Fixed part of a CTA's time (set-up, cluster reduction) in units of one K block of streaming;
+// MDBF_T1_FIXED_COST overrides it for experiments.
+static int fixed_cost() {
+    static int v = -1;
+    if (v < 0) {
+        const char *e = getenv("MDBF_T1_FIXED_COST");
+        v = e ? atoi(e) : 48;
+        if (v < 0) v = 16;
+    }
+    return v;
+}
+
 // Cluster size along the reduction: one CTA per SM (all of TMEM), as few waves as possible, the
 // per-CTA prologue (about 16 K blocks' worth of time) weighed against its share of the reduction.
 static bool plan_t1(int rows, int kb_pad, int LP, TxPlan *p) {
@@ -430,11 +443,13 @@ static bool plan_t1(int rows, int kb_pad, int LP, TxPlan *p) {
     if (nas > TX_MAX_ASTAGES) nas = TX_MAX_ASTAGES;
     long best_cost = -1;
     int best_ks = 1;
-    for (int ks = 1; ks <= 8; ks *= 2) {
+    static int max_ks = 0;
+    if (!max_ks) { const char *e = getenv("MDBF_T1_MAX_KS"); max_ks = e ? atoi(e) : 8; if (max_ks < 1 || max_ks > 8) max_ks = 8; }
+    for (int ks = 1; ks <= max_ks; ks *= 2) {
         const int per = ceil_div(npairs, ks);
         if (ks > 1 && per * (ks - 1) >= npairs) continue;              // an empty rank: pointless split
         const long waves = ceil_div(rb * ks, 148);
-        const long cost = waves * (2 * per + 16);
+        const long cost = waves * (2 * per + fixed_cost());
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ks = ks; }
     }
     p->ks = best_ks;
