@@ -74,7 +74,7 @@ __device__ __forceinline__ bool tx_wait(uint32_t bar, uint32_t parity, volatile 
 //   vring [nastages][2 * NB * 128 B]   V tile images of a pair (B operand)
 //   sring [nsstages][2048 B]           packed sign words of a pair: [2][128 rows] uint2
 //   xp    [pairs_per_cta * 64] u32     activation pairs in MMA k order (bf16x2)
-//   part  [128] float                  partial outputs (cluster reduction)
+//   part  [8][128] float               partial outputs pushed by the other cluster ranks (rank 0 only reads)
 template <int LP>
 __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) {
     using namespace tm;
@@ -259,7 +259,6 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
                     if (cc * 16 + j < LP) outv += u[(cc * 16 + j) % LP] * sum[j];
             }
         }
-        if (grp == 0) part[row_l] = outv;
     }
     else if (warp < TX_W_ISSUER0 + TX_ISSUERS) {
         // ================================== MMA issuers ===================================
@@ -338,22 +337,24 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
     }
 
     // ------------------------------ cluster reduction and store ------------------------------
+    // The other ranks push their partial outputs into rank 0's shared memory; one cluster barrier
+    // (release / acquire) later rank 0 adds them up in rank order and stores.  Nobody reads a remote
+    // CTA's memory after the barrier, so every CTA may leave as soon as it has passed it.
     tc_fence_before();
+    const unsigned crank = cluster.block_rank();
+    if (warp < 4 && crank != 0) cluster.map_shared_rank(part, 0)[crank * 128 + row_l] = outv;
     cluster.sync();
-    if (warp < 4 && cluster.block_rank() == 0) {
+    if (warp < 4 && crank == 0) {
         const unsigned nranks = cluster.num_blocks();
-        float rv[8];
 #pragma unroll
-        for (unsigned rk = 1; rk < 8; ++rk) rv[rk] = rk < nranks ? cluster.map_shared_rank(part, rk)[row_l] : 0.f;
-#pragma unroll
-        for (unsigned rk = 1; rk < 8; ++rk) outv += rv[rk];
+        for (unsigned rk = 1; rk < 8; ++rk)
+            if (rk < nranks) outv += part[rk * 128 + row_l];
         const int grow = row0 + row_l;
         if (grow < a.rows && !*abort_flag) {
             if (stage_a) reinterpret_cast<__nv_bfloat16 *>(a.out)[grow] = __float2bfloat16_rn(outv);
             else reinterpret_cast<float *>(a.out)[grow] = outv;
         }
     }
-    cluster.sync();
     if (warp == TX_W_ISSUER0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
 }
 
@@ -458,7 +459,7 @@ static bool plan_t1(int rows, int kb_pad, int LP, TxPlan *p) {
     p->nsstages = p->pairs_per_cta < TX_MAX_SSTAGES ? p->pairs_per_cta : TX_MAX_SSTAGES;
     if (p->nsstages < 1) p->nsstages = 1;
     p->tmem_cols = 512;
-    p->smem = 1024 + (size_t)nas * 2 * NB * 128 + (size_t)p->nsstages * 2048 + (size_t)p->pairs_per_cta * 256 + 512;
+    p->smem = 1024 + (size_t)nas * 2 * NB * 128 + (size_t)p->nsstages * 2048 + (size_t)p->pairs_per_cta * 256 + 4096;
     return nas >= 2 && p->smem <= 220 * 1024;
 }
 
