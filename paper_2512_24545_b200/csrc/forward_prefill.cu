@@ -49,7 +49,8 @@ constexpr int PF_THREADS = PF_EXPANDERS + 64;
 constexpr int PF_A_BYTES = PF_BM * PF_BK * 2;      // 16 KB
 constexpr int PF_B_BYTES = PF_BN * PF_BK * 2;      // 32 KB
 constexpr int PF_STAGE_BYTES = PF_A_BYTES + PF_B_BYTES;
-constexpr int PF_SMEM_BYTES = PF_STAGES * PF_STAGE_BYTES + 1024;   // + alignment slack
+constexpr int PF_PART_BYTES = 32 * 1024;           // partial outputs pushed by the ranks of a split cluster: [rank][token][128] fp32
+constexpr int PF_SMEM_BYTES = PF_STAGES * PF_STAGE_BYTES + PF_PART_BYTES + 1024;   // + alignment slack
 constexpr uint32_t PF_MAX_POLLS = 1u << 20;
 
 struct GemmArgs {
@@ -264,7 +265,12 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
         tc_fence_after();
         pdl_wait();                                   // the stores below must follow the previous kernel's reads
         // one finished output value: stored at once, or parked for the cluster reduction
-        float *part = reinterpret_cast<float *>(smem_gen);               // [token of the tile][128 rows]; the stages are idle now
+        // [rank][token of the tile][128 rows], a region of its own: other ranks write into it while this
+        // CTA's pipeline stages may still be busy
+        float *part = reinterpret_cast<float *>(smem_gen + PF_STAGES * PF_STAGE_BYTES);
+        const unsigned crank = SPLIT ? cluster.block_rank() : 0u;
+        const int ntl = ((a.n_eff + 31) / 32 * 32) / LP;      // token slots the read-out loop below produces (32 columns at a time)
+        float *part_dst = SPLIT ? cluster.map_shared_rank(part, 0) : part;
         auto emit = [&](int tau, float acc) {
             if (egrow < a.rows && tau < a.T) {
                 if (STAGE_A) {
@@ -298,7 +304,7 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
                     acc += u[t] * __uint_as_float(v[j]);
                     if (t == LP - 1) {
                         const int tl = (col0 + j) / LP;
-                        if (split) part[tl * PF_BM + arow] = acc;
+                        if (split) part_dst[((int)crank * ntl + tl) * PF_BM + arow] = acc;
                         else emit(tau0 + tl, acc);
                         acc = 0.f;
                     }
@@ -306,20 +312,18 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
             }
         }
         if (split) {
-            // the ranks of the cluster hold partial sums over their slices of the reduction: rank 0 adds
-            // them up in rank order (deterministic) through distributed shared memory and stores
+            // every rank has pushed its partial sums into rank 0's shared memory ([rank][token][row]);
+            // after one cluster barrier rank 0 adds them up in rank order (deterministic) and stores
             tc_fence_before();
             cluster.sync();
-            if (cluster.block_rank() == 0 && alive && !*abort_flag) {
+            if (crank == 0 && alive && !*abort_flag) {
                 const unsigned nranks = cluster.num_blocks();
-                const int ntl = a.n_eff / LP;
                 for (int tl = 0; tl < ntl; ++tl) {
-                    float acc = part[tl * PF_BM + arow];
-                    for (unsigned rk = 1; rk < nranks; ++rk) acc += cluster.map_shared_rank(part, rk)[tl * PF_BM + arow];
+                    float acc = 0.f;
+                    for (unsigned rk = 0; rk < nranks; ++rk) acc += part[((int)rk * ntl + tl) * PF_BM + arow];
                     emit(tau0 + tl, acc);
                 }
             }
-            cluster.sync();
         }
     } else if (warp == 4) {
         // ================================ TMA issuer =================================
@@ -362,10 +366,7 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
         if (lane == 0 && alive) { if (nkb > 0) umma_commit(accum_bar); else mbar_arrive(accum_bar); }
         __syncwarp();
     }
-    if (split && warp >= 4) {          // the expander warps run these two barriers inside their epilogue
-        cluster.sync();
-        cluster.sync();
-    }
+    if (split && warp >= 4) cluster.sync();          // the expander warps run this barrier inside their epilogue
 
     tc_fence_before();
     __syncthreads();
@@ -509,6 +510,7 @@ static mdbf_status_t launch_gemm(const GemmArgs &a, const CUtensorMap &tm, cudaS
     for (int ks = 1; ks <= 8; ks *= 2) {
         const int per = ceil_div(nkb, ks);
         if (ks > 1 && per * (ks - 1) >= nkb) continue;                 // an empty rank
+        if (ks > 1 && (size_t)ks * (((a.n_eff + 31) / 32 * 32) / LP) * PF_BM * sizeof(float) > PF_PART_BYTES) continue;   // partials must fit
         const long waves = ceil_div((long)rb * ntiles * ks, 148);
         const long cost = waves * (per + 10);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ks = ks; }
