@@ -16,11 +16,13 @@
 //   gemm_stage_kernel<B> z, and in the same epilogue Xs_A = bf16(V_A * z) for the next stage
 //   gemm_stage_kernel<A> y
 //
-// GEMM CTA = 128 rows of S x 256 columns (256/LP tokens x LP modes), 6 warps:
-//   warps 0-3  expand 64 packed sign bits per row and K block into the 128B-swizzled bf16 A tile
-//              (+-1.0; three integer ops per pair of elements), later run the epilogue
-//   warp 4     one lane issues the TMA load of the 256 x 64 Xs tile (tensor map, 128B swizzle)
-//   warp 5     one lane issues 4 tcgen05.mma (K = 16 each) per K block and commits the stage
+// GEMM CTA = 128 rows of S x 256 columns (256/LP tokens x LP modes), 10 warps:
+//   warps 0-7  two groups of four; group g expands, for the K blocks g, g+2, ..., 64 packed sign
+//              bits per row into the 128B-swizzled bf16 A tile (+-1.0; three integer ops per pair
+//              of elements); later both groups run the epilogue on alternate 32-column chunks
+//   warp 8     one lane issues the TMA load of the Xs tile (tensor map, 128B swizzle; box of 64,
+//              128 or 256 rows)
+//   warp 9     one lane issues 4 tcgen05.mma (K = 16 each) per K block and commits the stage
 // in a 4-stage mbarrier ring.  The epilogue reads the 128 x 256 fp32 accumulator from TMEM
 // (tcgen05.ld), contracts the LP modes of every token with U in registers and stores.
 //
@@ -44,8 +46,11 @@ constexpr int PF_BM = 128;
 constexpr int PF_BN = 256;
 constexpr int PF_BK = 64;
 constexpr int PF_STAGES = 4;
-constexpr int PF_EXPANDERS = 128;
-constexpr int PF_THREADS = PF_EXPANDERS + 64;
+constexpr int PF_EXPANDERS = 128;                  // threads that fill one A tile (one per row)
+constexpr int PF_GROUPS = 2;                       // expander groups: group g fills the tiles of K blocks g, g + 2, ...
+constexpr int PF_W_TMA = PF_GROUPS * 4;            // warp indices of the two single-lane roles
+constexpr int PF_W_MMA = PF_W_TMA + 1;
+constexpr int PF_THREADS = PF_GROUPS * PF_EXPANDERS + 64;
 constexpr int PF_A_BYTES = PF_BM * PF_BK * 2;      // 16 KB
 constexpr int PF_B_BYTES = PF_BN * PF_BK * 2;      // 32 KB
 constexpr int PF_STAGE_BYTES = PF_A_BYTES + PF_B_BYTES;
@@ -215,7 +220,7 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
         abort_flag_s = 0;
         fence_barrier_init();
     }
-    if (warp == 5) {
+    if (warp == PF_W_MMA) {
         tmem_alloc(smem_u32(&tmem_base_slot), PF_BN);
         tmem_relinquish();
     }
@@ -227,17 +232,21 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
     // overwrites data of the previous kernel (the Xs operand, z / Xs_next / y) waits for it below.
     pdl_launch_dependents();
 
-    if (warp < 4) {
+    if (warp < PF_W_TMA) {
         // ============================ sign-tile expanders ============================
-        const int arow = tid;                                     // one row of the tile per thread
+        // Two groups of four warps work on alternate K blocks: one warp's walk through a block is a
+        // chain of fixed latencies (barrier test, loads, shared stores, fence), so two blocks in
+        // flight nearly double the rate at which tiles reach the tensor core.
+        const int grp = warp >> 2;
+        const int arow = tid & (PF_EXPANDERS - 1);                // one row of the tile per thread
         const uint2 *wp = a.wk + (size_t)kb0 * a.rows_pad + (size_t)row0 + arow;   // + kb * rows_pad
-        uint2 w_next = nkb > 0 ? __ldg(wp) : make_uint2(0u, 0u);
+        uint2 w_next = grp < nkb ? __ldg(wp + (size_t)grp * a.rows_pad) : make_uint2(0u, 0u);
         bool alive = true;
-        for (int kb = 0; kb < nkb && alive; ++kb) {
+        for (int kb = grp; kb < nkb && alive; kb += PF_GROUPS) {
             const int s = kb % PF_STAGES;
             const uint32_t ph = (uint32_t)(kb / PF_STAGES) & 1u;
             const uint2 w = w_next;
-            if (kb + 1 < nkb) w_next = __ldg(wp + (size_t)(kb + 1) * a.rows_pad);
+            if (kb + PF_GROUPS < nkb) w_next = __ldg(wp + (size_t)(kb + PF_GROUPS) * a.rows_pad);
             alive = mbar_wait(empty_bar + 8 * s, ph ^ 1u, abort_flag, a.status);
             if (!alive) break;
             unsigned char *sA = smem_gen + (size_t)s * PF_STAGE_BYTES + arow * 128;
@@ -287,12 +296,12 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
         if (alive) {
             float acc = 0.f;
 #pragma unroll 1
-            for (int ld = 0; ld < PF_BN / 32; ++ld) {
+            for (int ld = grp; ld < PF_BN / 32; ld += PF_GROUPS) {      // the groups share a lane quadrant: alternate chunks
                 const int col0 = ld * 32;
                 if (col0 >= a.n_eff) break;                              // warp-uniform
                 uint32_t v[32];
                 if (!SPLIT || nkb > 0) {
-                    tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)col0, v);
+                    tmem_ld32(tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)col0, v);
                     tmem_ld_wait();
                 } else {
 #pragma unroll
@@ -318,14 +327,14 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
             cluster.sync();
             if (crank == 0 && alive && !*abort_flag) {
                 const unsigned nranks = cluster.num_blocks();
-                for (int tl = 0; tl < ntl; ++tl) {
+                for (int tl = grp; tl < ntl; tl += PF_GROUPS) {
                     float acc = 0.f;
                     for (unsigned rk = 0; rk < nranks; ++rk) acc += part[((int)rk * ntl + tl) * PF_BM + arow];
                     emit(tau0 + tl, acc);
                 }
             }
         }
-    } else if (warp == 4) {
+    } else if (warp == PF_W_TMA) {
         // ================================ TMA issuer =================================
         bool alive = true;
         pdl_wait();                                   // Xs comes from the previous kernel
@@ -366,11 +375,11 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
         if (lane == 0 && alive) { if (nkb > 0) umma_commit(accum_bar); else mbar_arrive(accum_bar); }
         __syncwarp();
     }
-    if (split && warp >= 4) cluster.sync();          // the expander warps run this barrier inside their epilogue
+    if (split && warp >= PF_W_TMA) cluster.sync();          // the expander warps run this barrier inside their epilogue
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) tmem_dealloc(tmem_d, PF_BN);
+    if (warp == PF_W_MMA) tmem_dealloc(tmem_d, PF_BN);
 }
 
 // ------------------------------------------------------------------- pre-scale
