@@ -205,6 +205,13 @@ mdbf_status_t mdbf_reconstruct(mdbf_handle_t h, float *W, void *stream);
  * Synchronises the device.  Reading clears the word. */
 mdbf_status_t mdbf_poll_status(mdbf_handle_t h, int32_t *device_status);
 
+/* Self-test of the bounded device-side wait the tcgen05 kernels use (no counterpart in the paper):
+ * launches one warp that waits on a barrier nothing arrives at.  After the time limit (about one
+ * second) the kernel records MDBF_ERR_TIMEOUT in the handle's status word and returns normally; the
+ * context stays usable and mdbf_poll_status reports (and clears) the code.  Asynchronous on
+ * `stream`. */
+mdbf_status_t mdbf_selftest_wait_timeout(mdbf_handle_t h, void *stream);
+
 /* Number of kernels the last forward on this handle launched. */
 mdbf_status_t mdbf_last_launch_count(mdbf_handle_t h, int32_t *count);
 

@@ -123,6 +123,7 @@ mdbf_status_t launch_wk2(const uint32_t *canon, int rows, int nwords, uint2 *out
                          cudaStream_t st);
 mdbf_status_t launch_vtile(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int NB,
                            cudaStream_t st);
+mdbf_status_t launch_wait_timeout_selftest(Layer &L, cudaStream_t st);
 mdbf_status_t launch_zsum(Layer &L, int T, cudaStream_t st);
 
 // host-side canonical packer (pack.cu)

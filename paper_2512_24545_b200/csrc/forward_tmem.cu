@@ -546,4 +546,26 @@ mdbf_status_t launch_forward_tmem(Layer &L, const void *x, void *y, int T, cudaS
     return MDBF_OK;
 }
 
+// ------------------------------------------------------------------ self-test of the bounded wait
+// One warp waits on an mbarrier that nothing ever arrives at, with the same bounded wait the
+// forward kernels use: after the time limit it must record MDBF_ERR_TIMEOUT in the status word and
+// return normally (no trap, the context stays usable).
+__global__ void wait_timeout_selftest_kernel(int32_t *status) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag_s;
+    if (threadIdx.x == 0) {
+        tm::mbar_init(tm::smem_u32(&bar), 1);
+        abort_flag_s = 0;
+        tm::fence_barrier_init();
+    }
+    __syncthreads();
+    tm::mbar_wait(tm::smem_u32(&bar), 0u, &abort_flag_s, status);
+}
+
+mdbf_status_t launch_wait_timeout_selftest(Layer &L, cudaStream_t st) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(L.status);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}
+
 }  // namespace mdbf

@@ -415,6 +415,12 @@ mdbf_status_t mdbf_poll_status(mdbf_handle_t h, int32_t *device_status) {
     return MDBF_OK;
 }
 
+mdbf_status_t mdbf_selftest_wait_timeout(mdbf_handle_t h, void *stream) {
+    mdbf_status_t rc = check_handle(h, "mdbf_selftest_wait_timeout");
+    if (rc) return rc;
+    return launch_wait_timeout_selftest(h->L, (cudaStream_t)stream);
+}
+
 mdbf_status_t mdbf_last_launch_count(mdbf_handle_t h, int32_t *count) {
     mdbf_status_t rc = check_handle(h, "mdbf_last_launch_count");
     if (rc) return rc;

@@ -29,7 +29,8 @@ EXPORTS = (
     "mdbf_pack_signs", "mdbf_unpack_signs", "mdbf_pack", "mdbf_get_packed", "mdbf_get_envelope",
     "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host",
     "mdbf_linear_forward_static",
-    "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_poll_status", "mdbf_last_launch_count",
+    "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_poll_status", "mdbf_selftest_wait_timeout",
+    "mdbf_last_launch_count",
     "mdbf_destroy", "mdbf_last_error", "mdbf_version",
 )
 
@@ -73,6 +74,7 @@ def lib() -> ctypes.CDLL:
     L.mdbf_get_intermediate.argtypes = [vp, vp, i32, ctypes.c_int, vp]
     L.mdbf_reconstruct.argtypes = [vp, vp, vp]
     L.mdbf_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
+    L.mdbf_selftest_wait_timeout.argtypes = [vp, vp]
     L.mdbf_last_launch_count.argtypes = [vp, ctypes.POINTER(i32)]
     L.mdbf_destroy.argtypes = [vp]
     for name in EXPORTS:
@@ -179,6 +181,11 @@ def mdbf_poll_status(h: int) -> int:
     v = ctypes.c_int32()
     _check(lib().mdbf_poll_status(h, ctypes.byref(v)))
     return v.value
+
+
+def mdbf_selftest_wait_timeout(h: int, stream: int = 0) -> None:
+    """Launch the bounded-wait self-test: about a second later the handle's status word reads ERR_TIMEOUT."""
+    _check(lib().mdbf_selftest_wait_timeout(h, stream))
 
 
 def mdbf_last_launch_count(h: int) -> int:

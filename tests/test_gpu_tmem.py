@@ -106,3 +106,22 @@ def test_tmem_kernel_rejects_wide_batches():
             g.forward(x, kernel=M.KERNEL_TMEM)                   # 16 modes x 8 tokens > 64 columns
         assert e.value.status == M.ERR_SHAPE
         assert rel_err(g.forward(x), g.oracle_forward(x)) <= TOL["bf16"]      # AUTO -> large-T kernel
+
+
+def test_bounded_wait_times_out_and_the_context_survives():
+    """A device-side wait that can never complete gives up after its time limit, reports
+    MDBF_ERR_TIMEOUT through the status word, and leaves the context usable."""
+    import time
+    spec = spec_of(128, 128, 128, 16)
+    x = inputs.make_activations(spec, 1)
+    with GpuLayer(spec, 1) as g:
+        assert M.mdbf_poll_status(g.h) == 0
+        t0 = time.perf_counter()
+        M.mdbf_selftest_wait_timeout(g.h, torch.cuda.current_stream().cuda_stream)
+        status = M.mdbf_poll_status(g.h)                           # synchronises
+        dt = time.perf_counter() - t0
+        assert status == M.ERR_TIMEOUT
+        assert 0.5 < dt < 10.0
+        assert M.mdbf_poll_status(g.h) == 0                        # reading cleared it
+        assert rel_err(g.forward(x), g.oracle_forward(x)) <= TOL["bf16"]       # still works
+        assert M.mdbf_poll_status(g.h) == 0
