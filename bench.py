@@ -89,6 +89,18 @@ def workload_specs(name):
         T = int(name.split("_T")[1]) if "_T" in name else 1
         return [(s, 4 if T <= 16 else 1) for s in inputs.block70b()], T, "hbm" if T <= 16 else "tensor", \
             f"70B-class decoder block, 7 linears, l=16 ~1.0 bpw, T={T}"
+    if name.startswith("sum_qproj"):
+        # sum_qproj_l<l>P<P>: P terms of envelope rank l on the 4096^2 shape, together ~1.0 bpw; the
+        # residual-compensation format ((l, P) = (1, 2) is the two-DBF-term case); T = 1
+        import re as _re
+        m = _re.match(r"sum_qproj_l(\d+)P(\d+)", name)
+        l, P = (int(m.group(1)), int(m.group(2))) if m else (1, 2)
+        bits = (1.0 / P) * 4096 * 4096                    # budget per term; k = largest multiple of 128 that meets it
+        k = int((bits - 16 * l * 8192) / (8192 + 32 * l)) // 128 * 128
+        base = inputs.qproj(1664)
+        terms = [(inputs.scaled(base, name=f"sum_qproj_l{l}_term{p}", k=k, l=l, seed=6 + 37 * p,
+                                env_std=0.02 * 0.6 ** p), 64) for p in range(P)]
+        return terms, 1, "hbm", f"sum of {P} terms 4096x4096 l={l} k={k} (~1.0 bpw together) T=1, 64 distinct sums"
     if name.startswith("prefill"):
         # prefill_<d_out>_l<l>_<bpw10|bpw15>
         parts = name.split("_")
@@ -177,13 +189,17 @@ def run_mdbf(args):
     stream = torch.cuda.Stream()
     st = stream.cuda_stream
 
+    P_sum = len(groups) if args.workload.startswith("sum_") else 0     # > 0: every P_sum consecutive layers are one sum
+    if P_sum:
+        ncopies = args.copies if args.copies > 0 else groups[0][1]
+        groups = [(inputs.scaled(sp, seed=sp.seed + 1000 * c), 1) for c in range(ncopies) for (sp, _n) in groups]
     layers = []          # (handle, spec, x_dev, y_dev, x_host, y_host)
     total_bytes = 0
     total_flops = 0.0
     weight_bytes = 0
     xs = {}
     for spec, copies in groups:
-        for c in range(args.copies if args.copies > 0 else copies):
+        for c in range(1 if P_sum else (args.copies if args.copies > 0 else copies)):
             sp = inputs.scaled(spec, seed=spec.seed + 1000 * (c + 1)) if c else spec
             lay = inputs.make_layer(sp)
             h = M.mdbf_pack(sp.d_out, sp.d_in, sp.k, sp.l, M.DTYPES[sp.env_dtype], T,
@@ -204,7 +220,14 @@ def run_mdbf(args):
     if weight_bytes < 2 * 126e6:       # rotation too small to defeat L2: flush between steps
         flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
 
+    acc = torch.zeros((T, max(sp.d_out for (_h, sp, *_r) in layers)), dtype=torch.float32, device="cuda") if P_sum else None
+
     def step():
+        if P_sum:
+            for i in range(0, len(layers), P_sum):
+                hs = [layers[i + p][0] for p in range(P_sum)]
+                M.mdbf_linear_forward_sum(hs, layers[i][2].data_ptr(), layers[i][3].data_ptr(), acc.data_ptr(), T, M.BF16, st)
+            return
         for (h, sp, xd, yd, _, _) in layers:
             M.mdbf_linear_forward(h, xd.data_ptr(), yd.data_ptr(), T, M.BF16, st)
 
@@ -242,7 +265,7 @@ def run_mdbf(args):
         barrier()
         clocks = sampler.stop()
         ms = sum(e0.elapsed_time(e1) for e0, e1 in ev)
-    launches = sum(M.mdbf_last_launch_count(h) for (h, *_rest) in layers) * args.steps
+    launches = (sum(M.mdbf_last_launch_count(h) for (h, *_rest) in layers) + (len(layers) // P_sum if P_sum else 0)) * args.steps
 
     # end to end: host buffers through the C-ABI, copies inside the timed region
     e2e_steps = max(1, min(args.steps, 10))

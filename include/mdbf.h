@@ -141,6 +141,18 @@ mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel /* mdbf_kernel_t *
 mdbf_status_t mdbf_linear_forward(mdbf_handle_t h, const void *x, void *y, int32_t T,
                                   int32_t act_dtype, void *stream);
 
+/* Sum of P layers on the same input, y = (W_hat^(1) + ... + W_hat^(P)) x: the residual-compensation
+ * form (Eq. dbf-residual-comp: a DBF term plus a DBF term fitted to the residual, (l, P) = (1, 2);
+ * the paper's (l, P) sweep uses the same sum with MDBF terms).  Every term is evaluated by the same
+ * kernels as mdbf_linear_forward with an fp32 output: term 1 stores into `acc`, the others add to
+ * it, and one pass rounds `acc` to y - so y carries a single rounding whatever P is.
+ *   terms  P handles of equal d_out and d_in (k, l and env_dtype may differ), all distinct
+ *   x, y   device, T x d_in read, T x d_out written, of act_dtype
+ *   acc    device, T x d_out float32 scratch owned by the caller, overwritten
+ * Asynchronous on `stream`, allocates nothing.  Errors: INVALID_ARG, SHAPE, DTYPE, CUDA. */
+mdbf_status_t mdbf_linear_forward_sum(const mdbf_handle_t *terms, int32_t P, const void *x, void *y, float *acc,
+                                      int32_t T, int32_t act_dtype, void *stream);
+
 /* Same computation with HOST buffers: copies x to a handle-owned device
  * staging buffer, runs the forward, copies y back, all on `stream`, and
  * synchronises the stream before returning.  x_host / y_host should be pinned

@@ -28,7 +28,8 @@ pattern of a 4x4x2 instance against the scalar-loop C twin, gauge flips,
 demodulation rank and isometry (Eq. me-dbf-envelope-rank, Lemma sign-mask
 isometry), a hand-worked example (tests/golden/), the bit-packing definition
 against numpy.packbits, the exact-projection error against the singular-value
-tail (Theorem 1).  No function here is "parity unpinned".
+tail (Theorem 1); the sum of terms against the two-term product of Eq. dbf-residual-comp written
+out per entry and against the sum of single-term forwards.  No function here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -36,7 +37,7 @@ import numpy as np
 
 __all__ = [
     "envelope", "modulated_factor", "reconstruct", "reconstruct_rows", "forward",
-    "forward_staged", "rel_frobenius", "pack_signs", "unpack_signs",
+    "forward_staged", "reconstruct_sum", "forward_sum", "rel_frobenius", "pack_signs", "unpack_signs",
     "bits_per_weight", "largest_inner_rank", "project_fixed_mask", "msvid",
 ]
 
@@ -130,6 +131,32 @@ def forward_staged(S_A, S_B, U_A, V_A, U_B, V_B, X):
     if vec:
         return Y[:, 0], Z[:, 0]
     return Y, Z
+
+
+def reconstruct_sum(terms):
+    """Dense sum of P layers, W_hat = sum_p W_hat^(p): the residual-compensation form
+    (Eq. dbf-residual-comp writes it for two DBF terms, i.e. l = 1, P = 2; the paper's (l, P) sweep
+    uses MDBF terms).  `terms` is a sequence of (S_A, S_B, U_A, V_A, U_B, V_B) tuples of equal
+    d_out and d_in; inner rank and envelope rank may differ between terms."""
+    terms = list(terms)
+    if not terms:
+        raise ValueError("at least one term")
+    W = reconstruct(*terms[0])
+    for t in terms[1:]:
+        Wp = reconstruct(*t)
+        if Wp.shape != W.shape:
+            raise ValueError("terms must share d_out and d_in")
+        W = W + Wp
+    return W
+
+
+def forward_sum(terms, X):
+    """Y = (sum_p W_hat^(p)) X with the sum materialised densely first."""
+    X = _f64(X)
+    W = reconstruct_sum(terms)
+    if X.shape[0] != W.shape[1]:
+        raise ValueError("activation rows must equal d_in")
+    return W @ X
 
 
 def rel_frobenius(A, B):

@@ -62,6 +62,7 @@ struct Layer {
     void *xstage, *ystage;        // device staging for the host-buffer entry point
     int32_t *status;              // device status word
     int last_ksplit;              // how many partials the last forward wrote (0 = zsum valid)
+    int out_mode;                 // set per call: 0 y in the activation type; 1 / 2: fp32 y stored / added (a term of a sum)
 };
 
 // thread-local error string
@@ -124,6 +125,7 @@ mdbf_status_t launch_wk2(const uint32_t *canon, int rows, int nwords, uint2 *out
 mdbf_status_t launch_vtile(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int NB,
                            cudaStream_t st);
 mdbf_status_t launch_wait_timeout_selftest(Layer &L, cudaStream_t st);
+mdbf_status_t launch_cast(const float *acc, void *y, size_t n, int act_dtype, cudaStream_t st);
 mdbf_status_t launch_zsum(Layer &L, int T, cudaStream_t st);
 
 // host-side canonical packer (pack.cu)

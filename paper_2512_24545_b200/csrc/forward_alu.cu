@@ -22,7 +22,7 @@ template <typename InT, typename OutT>
 __global__ void __launch_bounds__(256)
 alu_stage_kernel(const uint32_t *__restrict__ words, int nwords, int rows, int cols,
                  const void *__restrict__ U, const void *__restrict__ V, int l, int env_dtype,
-                 const InT *__restrict__ in, OutT *__restrict__ out, int T) {
+                 const InT *__restrict__ in, OutT *__restrict__ out, int T, int add) {
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (r >= rows) return;
@@ -74,7 +74,10 @@ alu_stage_kernel(const uint32_t *__restrict__ words, int nwords, int rows, int c
         if (lane == 0) {
 #pragma unroll
             for (int b = 0; b < ALU_TT; ++b)
-                if (tau0 + b < T) act_store<OutT>(out, (size_t)(tau0 + b) * rows + r, res[b]);
+                if (tau0 + b < T) {
+                    const size_t o = (size_t)(tau0 + b) * rows + r;
+                    act_store<OutT>(out, o, add ? act_load<OutT>(out, o) + res[b] : res[b]);      // add: a further term of a sum
+                }
         }
     }
 }
@@ -84,11 +87,16 @@ static mdbf_status_t run(Layer &L, const void *x, void *y, int T, cudaStream_t s
     const int wpb = 8;
     alu_stage_kernel<ActT, float><<<ceil_div(L.d.k, wpb), wpb * 32, 0, st>>>(
         L.wB, L.wordsB, L.d.k, L.d.d_in, L.UB, L.VB, L.d.l, L.d.env_dtype,
-        reinterpret_cast<const ActT *>(x), L.zsum, T);
+        reinterpret_cast<const ActT *>(x), L.zsum, T, 0);
     MDBF_CUDA(cudaGetLastError());
-    alu_stage_kernel<float, ActT><<<ceil_div(L.d.d_out, wpb), wpb * 32, 0, st>>>(
-        L.wA, L.wordsA, L.d.d_out, L.d.k, L.UA, L.VA, L.d.l, L.d.env_dtype,
-        L.zsum, reinterpret_cast<ActT *>(y), T);
+    if (L.out_mode == 0)
+        alu_stage_kernel<float, ActT><<<ceil_div(L.d.d_out, wpb), wpb * 32, 0, st>>>(
+            L.wA, L.wordsA, L.d.d_out, L.d.k, L.UA, L.VA, L.d.l, L.d.env_dtype,
+            L.zsum, reinterpret_cast<ActT *>(y), T, 0);
+    else                                   // a term of a sum of layers: fp32 output, stored or added
+        alu_stage_kernel<float, float><<<ceil_div(L.d.d_out, wpb), wpb * 32, 0, st>>>(
+            L.wA, L.wordsA, L.d.d_out, L.d.k, L.UA, L.VA, L.d.l, L.d.env_dtype,
+            L.zsum, reinterpret_cast<float *>(y), T, L.out_mode == 2 ? 1 : 0);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
@@ -102,6 +110,24 @@ mdbf_status_t launch_forward_alu(Layer &L, const void *x, void *y, int T, int ac
     else { set_error("mdbf_linear_forward: unsupported activation dtype %d", act_dtype); return MDBF_ERR_DTYPE; }
     if (rc == MDBF_OK) { L.last_ksplit = 0; *launches = 2; }
     return rc;
+}
+
+// fp32 accumulator of a sum of layers -> activation type (one rounding)
+template <typename OutT>
+__global__ void cast_kernel(const float *__restrict__ acc, OutT *__restrict__ y, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        act_store<OutT>(y, i, acc[i]);
+}
+
+mdbf_status_t launch_cast(const float *acc, void *y, size_t n, int act_dtype, cudaStream_t st) {
+    int grid = (int)((n + 255) / 256);
+    if (grid > 148 * 16) grid = 148 * 16;
+    if (grid < 1) grid = 1;
+    if (act_dtype == MDBF_F32) cast_kernel<float><<<grid, 256, 0, st>>>(acc, reinterpret_cast<float *>(y), n);
+    else if (act_dtype == MDBF_BF16) cast_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(acc, reinterpret_cast<__nv_bfloat16 *>(y), n);
+    else cast_kernel<__half><<<grid, 256, 0, st>>>(acc, reinterpret_cast<__half *>(y), n);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
 }
 
 // sum the stage-B partials into zsum (inspection only)

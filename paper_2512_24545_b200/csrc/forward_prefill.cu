@@ -73,6 +73,8 @@ struct GemmArgs {
     int pad_next;
     // stage A only
     __nv_bfloat16 *y;        // [T][rows]
+    float *y32;              // [T][rows]: fp32 output when the layer is a term of a sum (y_mode 1: store, 2: add)
+    int y_mode;
     int box_rows;            // rows of the TMA box of the Xs operand: 64, 128 or 256 (>= n_eff)
     int kb_per_cta;          // K blocks per cluster rank (blockIdx.z); the ranks' partial outputs are reduced over DSMEM
     int32_t *status;
@@ -283,7 +285,9 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
         auto emit = [&](int tau, float acc) {
             if (egrow < a.rows && tau < a.T) {
                 if (STAGE_A) {
-                    a.y[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(acc);
+                    if (a.y_mode == 0) a.y[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(acc);
+                    else if (a.y_mode == 1) a.y32[(size_t)tau * a.rows + egrow] = acc;
+                    else a.y32[(size_t)tau * a.rows + egrow] += acc;
                 } else {
                     a.z[(size_t)tau * a.rows + egrow] = acc;
                     __nv_bfloat16 *xo = a.xs_next + (size_t)tau * LP * a.pad_next + egrow;
@@ -584,7 +588,7 @@ static mdbf_status_t run_prefill(Layer &L, const void *x, void *y, int T, cudaSt
     GemmArgs a = {};
     a.wk = L.wkA; a.rows_pad = L.rpA; a.rows = d.d_out; a.cols = d.k;
     a.U = L.UA; a.env_dtype = d.env_dtype; a.l = d.l; a.T = T; a.n_eff = n_eff;
-    a.y = reinterpret_cast<__nv_bfloat16 *>(y); a.status = L.status;
+    a.y = reinterpret_cast<__nv_bfloat16 *>(y); a.y32 = reinterpret_cast<float *>(y); a.y_mode = L.out_mode; a.status = L.status;
     a.box_rows = 64 << bi;
     return launch_gemm<LP, true>(a, L.tmA[bi], st);
 }

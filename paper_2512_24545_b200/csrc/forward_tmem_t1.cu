@@ -60,7 +60,7 @@ struct TxArgs {
     int npairs_total;         // pairs of K blocks along the reduction
     int pairs_per_cta;        // pairs per cluster rank
     int nastages, nsstages, tmem_cols;
-    int stage_a;              // 0: stage B (bf16 in, fp32 out), 1: stage A (fp32 in, bf16 out)
+    int stage_a;              // 0: stage B (bf16 in, fp32 out); stage A (fp32 in): 1 bf16 out, 2 fp32 out, 3 added to fp32 out
     int32_t *status;
 };
 
@@ -351,7 +351,8 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
             if (rk < nranks) outv += part[rk * 128 + row_l];
         const int grow = row0 + row_l;
         if (grow < a.rows && !*abort_flag) {
-            if (stage_a) reinterpret_cast<__nv_bfloat16 *>(a.out)[grow] = __float2bfloat16_rn(outv);
+            if (a.stage_a == 1) reinterpret_cast<__nv_bfloat16 *>(a.out)[grow] = __float2bfloat16_rn(outv);
+            else if (a.stage_a == 3) reinterpret_cast<float *>(a.out)[grow] += outv;      // a further term of a sum of layers
             else reinterpret_cast<float *>(a.out)[grow] = outv;
         }
     }
@@ -508,7 +509,7 @@ static mdbf_status_t run_t1(Layer &L, const void *x, void *y, cudaStream_t st) {
     TxArgs s = {};
     s.wk2 = L.wk2A; s.kb_pad = L.kbpA; s.rows = d.d_out; s.cols = d.k;
     s.vtile = L.vxA; s.U = L.UA; s.env_dtype = d.env_dtype; s.l = d.l;
-    s.in = L.zsum; s.out = y; s.stage_a = 1;
+    s.in = L.zsum; s.out = y; s.stage_a = 1 + L.out_mode;
     s.npairs_total = L.kbpA / 2; s.pairs_per_cta = pa.pairs_per_cta;
     s.nastages = pa.nastages; s.nsstages = pa.nsstages; s.tmem_cols = pa.tmem_cols; s.status = L.status;
     return launch_t1<LP>(s, pa, st);

@@ -317,8 +317,9 @@ mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel) {
 }
 
 static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32_t T, int32_t act_dtype,
-                                  cudaStream_t st) {
+                                  cudaStream_t st, int out_mode = 0) {
     Layer &L = h->L;
+    L.out_mode = out_mode;
     if (T < 1 || T > L.d.max_T) {
         set_error("mdbf_linear_forward: T=%d outside [1, max_T=%d]", T, L.d.max_T);
         return MDBF_ERR_SHAPE;
@@ -344,6 +345,10 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
                   kDecodeMaxT, T, L.d.l);
         return MDBF_ERR_SHAPE;
     }
+    if (out_mode != 0 && (kernel == MDBF_KERNEL_DECODE || (kernel == MDBF_KERNEL_TMEM && T > 1))) {
+        set_error("mdbf_linear_forward_sum: the forced kernel has no fp32-accumulate output");
+        return MDBF_ERR_INVALID_ARG;
+    }
     int launches = 0;
     mdbf_status_t rc;
     if (kernel == MDBF_KERNEL_ALU) rc = launch_forward_alu(L, x, y, T, act_dtype, st, &launches);
@@ -360,6 +365,29 @@ mdbf_status_t mdbf_linear_forward(mdbf_handle_t h, const void *x, void *y, int32
     if (rc) return rc;
     if (!x || !y) { set_error("mdbf_linear_forward: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
     return forward_impl(h, x, y, T, act_dtype, (cudaStream_t)stream);
+}
+
+mdbf_status_t mdbf_linear_forward_sum(const mdbf_handle_t *terms, int32_t P, const void *x, void *y, float *acc,
+                                      int32_t T, int32_t act_dtype, void *stream) {
+    if (!terms || !x || !y || !acc) { set_error("mdbf_linear_forward_sum: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    if (P < 1 || P > 64) { set_error("mdbf_linear_forward_sum: P=%d outside [1, 64]", P); return MDBF_ERR_SHAPE; }
+    for (int p = 0; p < P; ++p) {
+        mdbf_status_t rc = check_handle(terms[p], "mdbf_linear_forward_sum");
+        if (rc) return rc;
+        if (terms[p]->L.d.d_out != terms[0]->L.d.d_out || terms[p]->L.d.d_in != terms[0]->L.d.d_in) {
+            set_error("mdbf_linear_forward_sum: term %d is %d x %d, term 0 is %d x %d", p, terms[p]->L.d.d_out,
+                      terms[p]->L.d.d_in, terms[0]->L.d.d_out, terms[0]->L.d.d_in);
+            return MDBF_ERR_SHAPE;
+        }
+        for (int q = 0; q < p; ++q)
+            if (terms[q] == terms[p]) { set_error("mdbf_linear_forward_sum: term %d repeats term %d", p, q); return MDBF_ERR_INVALID_ARG; }
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    for (int p = 0; p < P; ++p) {            // term 0 stores its fp32 output into acc, the others add to it (stream order)
+        mdbf_status_t rc = forward_impl(terms[p], x, acc, T, act_dtype, st, p == 0 ? 1 : 2);
+        if (rc) return rc;
+    }
+    return launch_cast(acc, y, (size_t)T * terms[0]->L.d.d_out, act_dtype, st);
 }
 
 mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T,

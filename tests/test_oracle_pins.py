@@ -209,9 +209,34 @@ def pin_packing(o):
     assert int(o.pack_signs(alt)[0, 0]) == 0xAAAAAAAA
 
 
+def pin_sum_of_terms(o):
+    """Residual compensation (Eq. dbf-residual-comp): for l = 1, P = 2 the sum of terms is
+    D_a1 S_a1 D_m1 S_b1^T D_b1 + D_a2 S_a2 D_m2 S_b2^T D_b2, written out per entry here; for general
+    terms (different k and l) it is the sum of the single-term results."""
+    rng = np.random.default_rng(21)
+    d_out, d_in = 5, 6
+    t1 = rand_layer(rng, d_out, d_in, 4, 1)
+    t2 = rand_layer(rng, d_out, d_in, 3, 1)
+    W = np.zeros((d_out, d_in))
+    for (S_A, S_B, U_A, V_A, U_B, V_B) in (t1, t2):
+        a, m, b = U_A[:, 0], V_A[:, 0] * U_B[:, 0], V_B[:, 0]
+        for n in range(d_out):
+            for i in range(d_in):
+                W[n, i] += a[n] * sum(S_A[n, j] * m[j] * S_B[j, i] for j in range(S_A.shape[1])) * b[i]
+    assert real.rel_frobenius(o.reconstruct_sum([t1, t2]), W) < 1e-13
+    X = rng.standard_normal((d_in, 2))
+    assert real.rel_frobenius(o.forward_sum([t1, t2], X), W @ X) < 1e-13
+    t3 = rand_layer(rng, d_out, d_in, 7, 3)                   # a third term of another rank
+    ref = sum(real.forward(*t, X) for t in (t1, t2, t3))
+    assert real.rel_frobenius(o.forward_sum([t1, t2, t3], X), ref) < 1e-13
+    assert real.rel_frobenius(o.reconstruct_sum([t3]), real.reconstruct(*t3)) == 0.0
+    with pytest.raises(ValueError):
+        o.reconstruct_sum([t1, rand_layer(rng, d_out + 1, d_in, 2, 1)])
+
+
 ALL_PINS = [pin_worked_example, pin_sum_of_dbf, pin_l1_is_dbf, pin_all_plus_signs,
             pin_gauge_and_flips, pin_demodulation_and_isometry, pin_linearity_and_duality,
-            pin_metric, pin_packing]
+            pin_metric, pin_packing, pin_sum_of_terms]
 
 
 @pytest.mark.parametrize("pin", ALL_PINS, ids=lambda f: f.__name__)
@@ -378,6 +403,11 @@ def _mutants():
         bits = np.pad((S == -1).astype(np.uint8), ((0, 0), (0, pad)))
         return np.packbits(bits, axis=1, bitorder="big").view(">u4").astype(np.uint32)
     m["pack MSB first"] = ns(pack_signs=pack_msb)
+    m["sum keeps only the first term"] = ns(reconstruct_sum=lambda ts: real.reconstruct(*list(ts)[0]),
+                                            forward_sum=lambda ts, X: real.forward(*list(ts)[0], X))
+    m["second term subtracted"] = ns(
+        reconstruct_sum=lambda ts: real.reconstruct(*list(ts)[0]) - sum(real.reconstruct(*t) for t in list(ts)[1:]),
+        forward_sum=lambda ts, X: real.forward_sum(ts, X))
     return m
 
 
