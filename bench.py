@@ -198,8 +198,11 @@ def run_mdbf(args):
     total_flops = 0.0
     weight_bytes = 0
     xs = {}
+    if args.workload.startswith("block70b"):       # block by block: q, k, v, o, gate, up, down of copy 0, then copy 1, ...
+        nc = args.copies if args.copies > 0 else groups[0][1]
+        groups = [(inputs.scaled(sp, seed=sp.seed + 1000 * c) if c else sp, 1) for c in range(nc) for (sp, _n) in groups]
     for spec, copies in groups:
-        for c in range(1 if P_sum else (args.copies if args.copies > 0 else copies)):
+        for c in range(1 if (P_sum or args.workload.startswith("block70b")) else (args.copies if args.copies > 0 else copies)):
             sp = inputs.scaled(spec, seed=spec.seed + 1000 * (c + 1)) if c else spec
             lay = inputs.make_layer(sp)
             h = M.mdbf_pack(sp.d_out, sp.d_in, sp.k, sp.l, M.DTYPES[sp.env_dtype], T,
@@ -222,7 +225,28 @@ def run_mdbf(args):
 
     acc = torch.zeros((T, max(sp.d_out for (_h, sp, *_r) in layers)), dtype=torch.float32, device="cuda") if P_sum else None
 
+    # the 70B-class block at one token: q/k/v share the hidden input and gate/up share the MLP input, so they
+    # go through the sibling entry point (one pair of launches per group); o and down stand alone
+    sib_groups = None
+    if args.workload.startswith("block70b") and T == 1 and not args.no_siblings:
+        sib_groups = []
+        for b0 in range(0, len(layers), 7):
+            blk = layers[b0:b0 + 7]
+            if len(blk) == 7:
+                sib_groups += [blk[0:3], blk[3:4], blk[4:6], blk[6:7]]
+            else:
+                sib_groups += [[l] for l in blk]
+
     def step():
+        if sib_groups is not None:
+            for grp in sib_groups:
+                if len(grp) == 1:
+                    (h, sp, xd, yd, _, _) = grp[0]
+                    M.mdbf_linear_forward(h, xd.data_ptr(), yd.data_ptr(), T, M.BF16, st)
+                else:
+                    M.mdbf_linear_forward_siblings([g[0] for g in grp], grp[0][2].data_ptr(), [g[3].data_ptr() for g in grp],
+                                                   T, M.BF16, st)
+            return
         if P_sum:
             for i in range(0, len(layers), P_sum):
                 hs = [layers[i + p][0] for p in range(P_sum)]
@@ -408,6 +432,7 @@ def main():
     ap.add_argument("--impl", default="mdbf", choices=["mdbf", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every forward from the host")
+    ap.add_argument("--no-siblings", action="store_true", help="block workloads: one forward per layer instead of fused q/k/v and gate/up")
     ap.add_argument("--copies", type=int, default=0, help="distinct layers per shape (0 = workload default); small values for ncu captures")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -153,6 +153,18 @@ mdbf_status_t mdbf_linear_forward(mdbf_handle_t h, const void *x, void *y, int32
 mdbf_status_t mdbf_linear_forward_sum(const mdbf_handle_t *terms, int32_t P, const void *x, void *y, float *acc,
                                       int32_t T, int32_t act_dtype, void *stream);
 
+/* Sibling projections: n layers applied to the same input, ys[i] = W_hat_i x (q/k/v, or gate/up, of a
+ * decoder block; the paper quantises each linear layer separately, so this is n forwards of
+ * Eq. DBF-inference-form / Eq. me-dbf-expand on a shared x).  With one token, bf16 activations and
+ * layers of equal envelope-rank bucket the stages of up to four layers share a launch (their row
+ * blocks side by side in one grid): two launches instead of 2n, and small layers no longer leave
+ * most SMs idle.  Otherwise the layers run one after the other, exactly as n calls of
+ * mdbf_linear_forward.
+ *   layers  n distinct handles of equal d_in          ys  n device pointers, ys[i] is T x d_out_i
+ * Asynchronous on `stream`, allocates nothing.  Errors: INVALID_ARG, SHAPE, DTYPE, CUDA. */
+mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t n, const void *x, void *const *ys,
+                                           int32_t T, int32_t act_dtype, void *stream);
+
 /* Same computation with HOST buffers: copies x to a handle-owned device
  * staging buffer, runs the forward, copies y back, all on `stream`, and
  * synchronises the stream before returning.  x_host / y_host should be pinned

@@ -64,6 +64,16 @@ struct TxArgs {
     int32_t *status;
 };
 
+// One launch may serve several layers that share their input (sibling projections: q/k/v, gate/up):
+// the row blocks of the layers are laid side by side along blockIdx.x, the cluster size, ring depths
+// and TMEM plan are common, everything else is per layer.
+constexpr int TX_MAX_LAYERS = 4;
+struct TxMulti {
+    TxArgs layer[TX_MAX_LAYERS];
+    int rb_start[TX_MAX_LAYERS + 1];   // first row block of each layer; rb_start[nlayers] = gridDim.x
+    int nlayers;
+};
+
 // First test inline (the common case: the barrier has completed), bounded loop otherwise.
 __device__ __forceinline__ bool tx_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status) {
     if (tm::mbar_try_wait(bar, parity)) return true;
@@ -76,7 +86,7 @@ __device__ __forceinline__ bool tx_wait(uint32_t bar, uint32_t parity, volatile 
 //   xp    [pairs_per_cta * 64] u32     activation pairs in MMA k order (bf16x2)
 //   part  [8][128] float               partial outputs pushed by the other cluster ranks (rank 0 only reads)
 template <int LP>
-__global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) {
+__device__ __forceinline__ void tmem_t1_body(const TxArgs &a, const int rb) {
     using namespace tm;
     constexpr int NB = LP < 16 ? 16 : LP;                    // MMA N
     constexpr int VBYTES = 2 * NB * 128;                     // two tiles
@@ -103,7 +113,7 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
     const uint32_t s_full = smem_u32(&bars[0]), s_empty = smem_u32(&bars[NB0]), v_full = smem_u32(&bars[NB1]),
                    a_full = smem_u32(&bars[NB2]), a_empty = smem_u32(&bars[NB3]), acc_bar = smem_u32(&bars[NB4]);
 
-    const int row0 = blockIdx.x * 128;
+    const int row0 = rb * 128;
     const int pr0 = blockIdx.y * a.pairs_per_cta;
     const int npr = max(0, min(a.pairs_per_cta, a.npairs_total - pr0));
 
@@ -306,7 +316,7 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
             bool alive = true;
             int rs = 0;
             uint32_t ph = 0;
-            const uint2 *src = a.wk2 + ((size_t)blockIdx.x * a.kb_pad + (size_t)pr0 * 2) * 128;
+            const uint2 *src = a.wk2 + ((size_t)rb * a.kb_pad + (size_t)pr0 * 2) * 128;
             for (int pr = 0; pr < npr; ++pr) {
                 alive = tx_wait(s_empty + 8 * rs, ph ^ 1u, abort_flag, a.status);
                 if (!alive) break;
@@ -357,6 +367,23 @@ __global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) 
         }
     }
     if (warp == TX_W_ISSUER0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
+}
+
+// One layer per launch: the arguments are plain kernel parameters (fastest for the small layers).
+template <int LP>
+__global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) {
+    tmem_t1_body<LP>(a, (int)blockIdx.x);
+}
+
+// Several sibling layers per launch: each CTA picks its layer by its position in the grid.
+template <int LP>
+__global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_multi_kernel(const __grid_constant__ TxMulti m) {
+    int li = 0;
+#pragma unroll
+    for (int i = 1; i < TX_MAX_LAYERS; ++i)
+        if (i < m.nlayers && (int)blockIdx.x >= m.rb_start[i]) li = i;
+    const TxArgs a = m.layer[li];                             // by value: one indexed read of the parameter block
+    tmem_t1_body<LP>(a, (int)blockIdx.x - m.rb_start[li]);
 }
 
 // ----------------------------------------------------------- pack-time private copies
@@ -420,7 +447,8 @@ mdbf_status_t launch_wk2(const uint32_t *canon, int rows, int nwords, uint2 *out
 
 // ---------------------------------------------------------------------- launch
 struct TxPlan {
-    int ks, pairs_per_cta, nastages, nsstages, tmem_cols;
+    int ks, nastages, tmem_cols;
+    int pairs_per_cta[TX_MAX_LAYERS], nsstages;
     size_t smem;
 };
 
@@ -431,49 +459,56 @@ static int fixed_cost() {
     if (v < 0) {
         const char *e = getenv("MDBF_T1_FIXED_COST");
         v = e ? atoi(e) : 48;
-        if (v < 0) v = 16;
+        if (v < 0) v = 48;
     }
     return v;
 }
 
-// Cluster size along the reduction: one CTA per SM (all of TMEM), as few waves as possible, the
-// per-CTA prologue (about 16 K blocks' worth of time) weighed against its share of the reduction.
-static bool plan_t1(int rows, int kb_pad, int LP, TxPlan *p) {
+// One plan for all the layers of a launch.  Cluster size along the reduction: one CTA per SM (all of
+// TMEM), as few waves as possible, the per-CTA fixed part weighed against its share of the reduction.
+static bool plan_t1(int n, const int *rows, const int *kb_pad, int LP, TxPlan *p) {
     const int NB = LP < 16 ? 16 : LP;
-    const int rb = ceil_div(rows, 128), npairs = kb_pad / 2;
-    int nas = (512 - TX_ISSUERS * NB) / 64;                  // NB = 32 with 8 accumulators leaves 4 stages
+    int nas = (512 - TX_ISSUERS * NB) / 64;
     if (nas > TX_MAX_ASTAGES) nas = TX_MAX_ASTAGES;
-    long best_cost = -1;
-    int best_ks = 1;
     static int max_ks = 0;
     if (!max_ks) { const char *e = getenv("MDBF_T1_MAX_KS"); max_ks = e ? atoi(e) : 8; if (max_ks < 1 || max_ks > 8) max_ks = 8; }
+    int rb = 0, max_pairs = 0, min_pairs = 1 << 30;
+    for (int i = 0; i < n; ++i) {
+        rb += ceil_div(rows[i], 128);
+        max_pairs = max(max_pairs, kb_pad[i] / 2);
+        min_pairs = min(min_pairs, kb_pad[i] / 2);
+    }
+    long best_cost = -1;
+    int best_ks = 1;
     for (int ks = 1; ks <= max_ks; ks *= 2) {
-        const int per = ceil_div(npairs, ks);
-        if (ks > 1 && per * (ks - 1) >= npairs) continue;              // an empty rank: pointless split
+        if (ks > 1 && ceil_div(min_pairs, ks) * (ks - 1) >= min_pairs) continue;     // an empty rank in some layer
         const long waves = ceil_div(rb * ks, 148);
-        const long cost = waves * (2 * per + fixed_cost());
+        const long cost = waves * (2 * ceil_div(max_pairs, ks) + fixed_cost());
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ks = ks; }
     }
     p->ks = best_ks;
-    p->pairs_per_cta = ceil_div(npairs, best_ks);
+    int max_per = 1;
+    for (int i = 0; i < n; ++i) {
+        p->pairs_per_cta[i] = ceil_div(kb_pad[i] / 2, best_ks);
+        max_per = max(max_per, p->pairs_per_cta[i]);
+    }
     p->nastages = nas;
-    p->nsstages = p->pairs_per_cta < TX_MAX_SSTAGES ? p->pairs_per_cta : TX_MAX_SSTAGES;
-    if (p->nsstages < 1) p->nsstages = 1;
+    p->nsstages = max_per < TX_MAX_SSTAGES ? max_per : TX_MAX_SSTAGES;
     p->tmem_cols = 512;
-    p->smem = 1024 + (size_t)nas * 2 * NB * 128 + (size_t)p->nsstages * 2048 + (size_t)p->pairs_per_cta * 256 + 4096;
+    p->smem = 1024 + (size_t)nas * 2 * NB * 128 + (size_t)p->nsstages * 2048 + (size_t)max_per * 256 + 4096;
     return nas >= 2 && p->smem <= 220 * 1024;
 }
 
 template <int LP>
-static mdbf_status_t launch_t1(const TxArgs &a, const TxPlan &p, cudaStream_t st) {
-    auto kern = tmem_t1_kernel<LP>;
+static mdbf_status_t launch_t1(const TxMulti &m, const TxPlan &p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        MDBF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_kernel<LP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_multi_kernel<LP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
         attr_set = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(ceil_div(a.rows, 128), p.ks, 1);
+    cfg.gridDim = dim3(m.rb_start[m.nlayers], p.ks, 1);
     cfg.blockDim = dim3(TX_THREADS);
     cfg.dynamicSmemBytes = p.smem;
     cfg.stream = st;
@@ -486,47 +521,68 @@ static mdbf_status_t launch_t1(const TxArgs &a, const TxPlan &p, cudaStream_t st
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    MDBF_CUDA(cudaLaunchKernelEx(&cfg, kern, a));
+    if (m.nlayers == 1) MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_kernel<LP>, m.layer[0]));
+    else MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_multi_kernel<LP>, m));
     return MDBF_OK;
 }
 
+// Both stages of n layers that read the same x (n = 1: a single layer): one launch per stage.
 template <int LP>
-static mdbf_status_t run_t1(Layer &L, const void *x, void *y, cudaStream_t st) {
-    const mdbf_desc_t &d = L.d;
+static mdbf_status_t run_t1(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st) {
+    int rowsB[TX_MAX_LAYERS], kbB[TX_MAX_LAYERS], rowsA[TX_MAX_LAYERS], kbA[TX_MAX_LAYERS];
+    for (int i = 0; i < n; ++i) {
+        rowsB[i] = Ls[i]->d.k; kbB[i] = Ls[i]->kbpB;
+        rowsA[i] = Ls[i]->d.d_out; kbA[i] = Ls[i]->kbpA;
+    }
     TxPlan pb, pa;
-    if (!plan_t1(d.k, L.kbpB, LP, &pb) || !plan_t1(d.d_out, L.kbpA, LP, &pa)) {
+    if (!plan_t1(n, rowsB, kbB, LP, &pb) || !plan_t1(n, rowsA, kbA, LP, &pa)) {
         set_error("mdbf_linear_forward: the one-token TMEM kernel does not fit this shape");
         return MDBF_ERR_SHAPE;
     }
-    TxArgs b = {};
-    b.wk2 = L.wk2B; b.kb_pad = L.kbpB; b.rows = d.k; b.cols = d.d_in;
-    b.vtile = L.vxB; b.U = L.UB; b.env_dtype = d.env_dtype; b.l = d.l;
-    b.in = x; b.out = L.zsum; b.stage_a = 0;
-    b.npairs_total = L.kbpB / 2; b.pairs_per_cta = pb.pairs_per_cta;
-    b.nastages = pb.nastages; b.nsstages = pb.nsstages; b.tmem_cols = pb.tmem_cols; b.status = L.status;
-    mdbf_status_t rc = launch_t1<LP>(b, pb, st);
+    TxMulti mb = {}, ma = {};
+    mb.nlayers = ma.nlayers = n;
+    for (int i = 0; i < n; ++i) {
+        Layer &L = *Ls[i];
+        const mdbf_desc_t &d = L.d;
+        TxArgs &b = mb.layer[i];
+        b.wk2 = L.wk2B; b.kb_pad = L.kbpB; b.rows = d.k; b.cols = d.d_in;
+        b.vtile = L.vxB; b.U = L.UB; b.env_dtype = d.env_dtype; b.l = d.l;
+        b.in = x; b.out = L.zsum; b.stage_a = 0;
+        b.npairs_total = L.kbpB / 2; b.pairs_per_cta = pb.pairs_per_cta[i];
+        b.nastages = pb.nastages; b.nsstages = pb.nsstages; b.tmem_cols = pb.tmem_cols; b.status = L.status;
+        mb.rb_start[i + 1] = mb.rb_start[i] + ceil_div(d.k, 128);
+        TxArgs &s = ma.layer[i];
+        s.wk2 = L.wk2A; s.kb_pad = L.kbpA; s.rows = d.d_out; s.cols = d.k;
+        s.vtile = L.vxA; s.U = L.UA; s.env_dtype = d.env_dtype; s.l = d.l;
+        s.in = L.zsum; s.out = ys[i]; s.stage_a = 1 + L.out_mode;
+        s.npairs_total = L.kbpA / 2; s.pairs_per_cta = pa.pairs_per_cta[i];
+        s.nastages = pa.nastages; s.nsstages = pa.nsstages; s.tmem_cols = pa.tmem_cols; s.status = L.status;
+        ma.rb_start[i + 1] = ma.rb_start[i] + ceil_div(d.d_out, 128);
+    }
+    mdbf_status_t rc = launch_t1<LP>(mb, pb, st);
     if (rc) return rc;
-    TxArgs s = {};
-    s.wk2 = L.wk2A; s.kb_pad = L.kbpA; s.rows = d.d_out; s.cols = d.k;
-    s.vtile = L.vxA; s.U = L.UA; s.env_dtype = d.env_dtype; s.l = d.l;
-    s.in = L.zsum; s.out = y; s.stage_a = 1 + L.out_mode;
-    s.npairs_total = L.kbpA / 2; s.pairs_per_cta = pa.pairs_per_cta;
-    s.nastages = pa.nastages; s.nsstages = pa.nsstages; s.tmem_cols = pa.tmem_cols; s.status = L.status;
-    return launch_t1<LP>(s, pa, st);
+    return launch_t1<LP>(ma, pa, st);
+}
+
+// n <= TX_MAX_LAYERS layers with the same LP, all prepared for the one-token kernel.
+mdbf_status_t launch_forward_tmem_t1_multi(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st) {
+    switch (Ls[0]->LP) {
+        case 1: return run_t1<1>(Ls, n, x, ys, st);
+        case 2: return run_t1<2>(Ls, n, x, ys, st);
+        case 4: return run_t1<4>(Ls, n, x, ys, st);
+        case 8: return run_t1<8>(Ls, n, x, ys, st);
+        case 16: return run_t1<16>(Ls, n, x, ys, st);
+        case 32: return run_t1<32>(Ls, n, x, ys, st);
+        default:
+            set_error("mdbf_linear_forward: the one-token TMEM kernel handles l <= 32 (got %d)", Ls[0]->d.l);
+            return MDBF_ERR_SHAPE;
+    }
 }
 
 mdbf_status_t launch_forward_tmem_t1(Layer &L, const void *x, void *y, cudaStream_t st) {
-    switch (L.LP) {
-        case 1: return run_t1<1>(L, x, y, st);
-        case 2: return run_t1<2>(L, x, y, st);
-        case 4: return run_t1<4>(L, x, y, st);
-        case 8: return run_t1<8>(L, x, y, st);
-        case 16: return run_t1<16>(L, x, y, st);
-        case 32: return run_t1<32>(L, x, y, st);
-        default:
-            set_error("mdbf_linear_forward: the one-token TMEM kernel handles l <= 32 (got %d)", L.d.l);
-            return MDBF_ERR_SHAPE;
-    }
+    Layer *one[1] = {&L};
+    void *ys[1] = {y};
+    return launch_forward_tmem_t1_multi(one, 1, x, ys, st);
 }
 
 }  // namespace mdbf

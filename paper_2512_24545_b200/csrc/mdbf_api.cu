@@ -390,6 +390,54 @@ mdbf_status_t mdbf_linear_forward_sum(const mdbf_handle_t *terms, int32_t P, con
     return launch_cast(acc, y, (size_t)T * terms[0]->L.d.d_out, act_dtype, st);
 }
 
+mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t n, const void *x, void *const *ys,
+                                           int32_t T, int32_t act_dtype, void *stream) {
+    if (!layers || !x || !ys) { set_error("mdbf_linear_forward_siblings: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    if (n < 1 || n > 64) { set_error("mdbf_linear_forward_siblings: n=%d outside [1, 64]", n); return MDBF_ERR_SHAPE; }
+    bool fusable = T == 1 && act_dtype == MDBF_BF16;
+    for (int i = 0; i < n; ++i) {
+        mdbf_status_t rc = check_handle(layers[i], "mdbf_linear_forward_siblings");
+        if (rc) return rc;
+        if (!ys[i]) { set_error("mdbf_linear_forward_siblings: NULL output %d", i); return MDBF_ERR_INVALID_ARG; }
+        const Layer &L = layers[i]->L;
+        if (L.d.d_in != layers[0]->L.d.d_in) {
+            set_error("mdbf_linear_forward_siblings: layer %d has d_in=%d, layer 0 has %d", i, L.d.d_in, layers[0]->L.d.d_in);
+            return MDBF_ERR_SHAPE;
+        }
+        if (T < 1 || T > L.d.max_T) {
+            set_error("mdbf_linear_forward_siblings: T=%d outside [1, max_T=%d] of layer %d", T, L.d.max_T, i);
+            return MDBF_ERR_SHAPE;
+        }
+        for (int q = 0; q < i; ++q)
+            if (layers[q] == layers[i]) { set_error("mdbf_linear_forward_siblings: layer %d repeats layer %d", i, q); return MDBF_ERR_INVALID_ARG; }
+        fusable = fusable && L.vxA && L.vxB && L.LP == layers[0]->L.LP && layers[i]->kernel == MDBF_KERNEL_AUTO;
+    }
+    if (!valid_dtype(act_dtype)) { set_error("mdbf_linear_forward_siblings: bad act_dtype %d", act_dtype); return MDBF_ERR_DTYPE; }
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!fusable) {                          // more than one token, mixed envelope ranks, fp32 layers: one after the other
+        for (int i = 0; i < n; ++i) {
+            mdbf_status_t rc = forward_impl(layers[i], x, ys[i], T, act_dtype, st);
+            if (rc) return rc;
+        }
+        return MDBF_OK;
+    }
+    for (int i0 = 0; i0 < n; i0 += kMaxSiblings) {      // groups of up to kMaxSiblings layers per pair of launches
+        const int m = n - i0 < kMaxSiblings ? n - i0 : kMaxSiblings;
+        Layer *Ls[kMaxSiblings];
+        void *outs[kMaxSiblings];
+        for (int i = 0; i < m; ++i) {
+            Ls[i] = &layers[i0 + i]->L;
+            Ls[i]->out_mode = 0;
+            Ls[i]->last_ksplit = 0;
+            outs[i] = ys[i0 + i];
+            layers[i0 + i]->last_launches = i == 0 ? 2 : 0;
+        }
+        mdbf_status_t rc = launch_forward_tmem_t1_multi(Ls, m, x, outs, st);
+        if (rc) return rc;
+    }
+    return MDBF_OK;
+}
+
 mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T,
                                        int32_t act_dtype, void *stream) {
     mdbf_status_t rc = check_handle(h, "mdbf_linear_forward_host");

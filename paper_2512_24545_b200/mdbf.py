@@ -28,7 +28,7 @@ DTYPES = {"f32": F32, "f16": F16, "bf16": BF16}
 EXPORTS = (
     "mdbf_pack_signs", "mdbf_unpack_signs", "mdbf_pack", "mdbf_get_packed", "mdbf_get_envelope",
     "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host",
-    "mdbf_linear_forward_static", "mdbf_linear_forward_sum",
+    "mdbf_linear_forward_static", "mdbf_linear_forward_sum", "mdbf_linear_forward_siblings",
     "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_poll_status", "mdbf_selftest_wait_timeout",
     "mdbf_last_launch_count",
     "mdbf_destroy", "mdbf_last_error", "mdbf_version",
@@ -72,6 +72,7 @@ def lib() -> ctypes.CDLL:
     L.mdbf_linear_forward_host.argtypes = [vp, vp, vp, i32, i32, vp]
     L.mdbf_linear_forward_static.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, vp]
     L.mdbf_linear_forward_sum.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp]
+    L.mdbf_linear_forward_siblings.argtypes = [vp, i32, vp, vp, i32, i32, vp]
     L.mdbf_get_intermediate.argtypes = [vp, vp, i32, ctypes.c_int, vp]
     L.mdbf_reconstruct.argtypes = [vp, vp, vp]
     L.mdbf_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
@@ -157,6 +158,14 @@ def mdbf_linear_forward_sum(handles, x, y, acc, T: int, act_dtype: int, stream: 
     arr = (ctypes.c_void_p * len(handles))(*handles)
     _check(lib().mdbf_linear_forward_sum(ctypes.cast(arr, ctypes.c_void_p), len(handles), _addr(x), _addr(y), _addr(acc),
                                          T, act_dtype, stream))
+
+
+def mdbf_linear_forward_siblings(handles, x, ys, T: int, act_dtype: int, stream: int = 0) -> None:
+    """ys[i] = W_hat_i x for layers that share the input x (q/k/v, gate/up); ys are device addresses."""
+    hs = (ctypes.c_void_p * len(handles))(*handles)
+    outs = (ctypes.c_void_p * len(ys))(*[_addr(y) for y in ys])
+    _check(lib().mdbf_linear_forward_siblings(ctypes.cast(hs, ctypes.c_void_p), len(handles), _addr(x),
+                                              ctypes.cast(outs, ctypes.c_void_p), T, act_dtype, stream))
 
 
 def mdbf_linear_forward_host(h: int, x_host, y_host, T: int, act_dtype: int, stream: int = 0) -> None:
