@@ -42,13 +42,12 @@ NCU_TRAFFIC_BYTES_PER_LAUNCH = {
 }
 
 
-def dominant_kernel(spec, T):
+def dominant_kernel(spec, T, forced="auto"):
     """Name of the kernel the library's dispatcher picks for this (l, T): the one the roofline line is about."""
-    lp = 1
-    while lp < spec.l:
-        lp *= 2
     if T == 1:
         return "tmem_t1_kernel"
+    if forced == "mat":
+        return "mat_stage_kernel"
     return "gemm_stage_kernel"
 
 
@@ -72,6 +71,11 @@ def algorithmic_bytes(spec, T):
 
 def expanded_flops(spec, T):
     return 2.0 * spec.l * T * spec.k * (spec.d_in + spec.d_out)
+
+
+def materialised_flops(spec, T):
+    """Tensor FLOPs when the factor tiles are rebuilt on the fly: rank-l envelope product + one GEMM of width T."""
+    return (2.0 * T + 2.0 * spec.l) * spec.k * (spec.d_in + spec.d_out)
 
 
 # ---------------------------------------------------------------- workloads
@@ -196,6 +200,7 @@ def run_mdbf(args):
     layers = []          # (handle, spec, x_dev, y_dev, x_host, y_host)
     total_bytes = 0
     total_flops = 0.0
+    total_mat_flops = 0.0
     weight_bytes = 0
     xs = {}
     if args.workload.startswith("block70b"):       # block by block: q, k, v, o, gate, up, down of copy 0, then copy 1, ...
@@ -207,6 +212,8 @@ def run_mdbf(args):
             lay = inputs.make_layer(sp)
             h = M.mdbf_pack(sp.d_out, sp.d_in, sp.k, sp.l, M.DTYPES[sp.env_dtype], T,
                             *[np.ascontiguousarray(lay[n]) for n in ("S_A", "S_B", "U_A", "V_A", "U_B", "V_B")])
+            if T > 1 and args.kernel != "auto":
+                M.mdbf_set_kernel(h, {"prefill": M.KERNEL_PREFILL, "mat": M.KERNEL_MAT}[args.kernel])
             if sp.d_in not in xs:
                 xh = torch.from_numpy(inputs.make_activations(sp, T)).to(torch.bfloat16).pin_memory()
                 xs[sp.d_in] = (xh, xh.cuda())
@@ -216,6 +223,7 @@ def run_mdbf(args):
             layers.append((h, sp, xd, yd, xh, yh))
             total_bytes += algorithmic_bytes(sp, T)
             total_flops += expanded_flops(sp, T)
+            total_mat_flops += materialised_flops(sp, T)
             weight_bytes += algorithmic_bytes(sp, 0)
     torch.cuda.synchronize()
 
@@ -313,8 +321,11 @@ def run_mdbf(args):
         per_step = total_bytes / 1e9
         peak = peaks["hbm_gbs"]
     else:
-        metric, unit = "prefill_expanded_TFLOPs", "TFLOP/s"
-        per_step = total_flops / 1e12
+        # the expanded-order kernel is rated in FLOPs of the expanded contraction (which it executes); the
+        # materialised-order kernel executes l x fewer and is rated in those, never in expanded FLOPs
+        mat = args.kernel == "mat" and T > 1
+        metric, unit = ("prefill_executed_TFLOPs" if mat else "prefill_expanded_TFLOPs"), "TFLOP/s"
+        per_step = (total_mat_flops if mat else total_flops) / 1e12
         peak = peaks["bf16_tflops"] if sec < 1.0 else peaks["bf16_tflops_sustained"]
     value = replicas.aggregate_throughput(per_step * args.steps, world, sec)
     per_gpu = per_step * args.steps / sec
@@ -329,14 +340,17 @@ def run_mdbf(args):
                    "l2_policy": ("rotation of distinct layers larger than L2" if flush is None
                                  else "256 MiB L2 flush between steps"),
                    "launch": "CUDA graph replay per step" if graph is not None else "stream launches",
+                   "kernel": args.kernel,
+                   "GFLOP_expanded_per_step": round(total_flops / 1e9, 1),
+                   "GFLOP_materialised_per_step": round(total_mat_flops / 1e9, 1),
                    "replicas": world},
         "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
         "clocks": clocks,
         "roofline": {"bound": bound, "achieved": per_gpu, "peak": peak, "unit": unit,
                      "frac": per_gpu / peak, "peak_source": f"of {peak_kind}",
-                     "kernel": dominant_kernel(groups[0][0], T),
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)},
+                     "kernel": dominant_kernel(groups[0][0], T, args.kernel),
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload) if args.kernel == "auto" else None},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(groups[0][0], T, bound, budget_s=20.0)
@@ -432,6 +446,8 @@ def main():
     ap.add_argument("--impl", default="mdbf", choices=["mdbf", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every forward from the host")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "prefill", "mat"],
+                    help="T > 1: force the expanded-order (prefill) or the materialised-order (mat) kernel")
     ap.add_argument("--no-siblings", action="store_true", help="block workloads: one forward per layer instead of fused q/k/v and gate/up")
     ap.add_argument("--copies", type=int, default=0, help="distinct layers per shape (0 = workload default); small values for ncu captures")
     args = ap.parse_args()

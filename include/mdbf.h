@@ -64,7 +64,8 @@ typedef enum {
     MDBF_KERNEL_ALU = 1,    /* fp32 CUDA-core path, sign applied by XOR of the IEEE sign bit      */
     MDBF_KERNEL_DECODE = 2, /* T <= 4: register bit->bf16 expansion + warp-level MMA              */
     MDBF_KERNEL_PREFILL = 3, /* T >= 2 (max_T >= 2): tcgen05 GEMM, TMEM accumulator, TMA operand   */
-    MDBF_KERNEL_TMEM = 4    /* l*T <= 64: tcgen05 MMA with the sign operand expanded into TMEM    */
+    MDBF_KERNEL_TMEM = 4,   /* l*T <= 64: tcgen05 MMA with the sign operand expanded into TMEM    */
+    MDBF_KERNEL_MAT = 5     /* T >= 2: W_hat tiles rebuilt on the fly (rank-l mini-MMA + sign XOR), one GEMM of width T */
 } mdbf_kernel_t;
 
 typedef struct {

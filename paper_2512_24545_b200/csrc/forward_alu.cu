@@ -141,7 +141,8 @@ __global__ void zsum_kernel(const float *__restrict__ z, float *__restrict__ zsu
 }
 
 mdbf_status_t launch_zsum(Layer &L, int T, cudaStream_t st) {
-    if (L.last_ksplit <= 0) return MDBF_OK;
+    if (L.last_ksplit < 0) return launch_zb_to_zsum(L, T, st);   // the materialised-envelope kernel keeps z in bf16
+    if (L.last_ksplit == 0) return MDBF_OK;
     const size_t n = (size_t)T * L.d.k;
     const size_t stride = L.zstride;
     zsum_kernel<<<(int)min((size_t)1024, (n + 255) / 256), 256, 0, st>>>(L.z, L.zsum, L.last_ksplit, n, stride);

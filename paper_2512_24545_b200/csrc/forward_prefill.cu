@@ -475,8 +475,9 @@ mdbf_status_t launch_vtrans(const void *V, int cols, int l, int env_dtype, float
     return MDBF_OK;
 }
 
-// Tensor map of a pre-scaled operand: bf16 [rows][pad] row-major, box 64 x 256, 128B swizzle.
-mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad, int box_rows) {
+// Tensor map of a bf16 activation matrix [rows][cols] whose rows are `stride` elements apart: box of 64
+// columns x box_rows rows, 128B swizzle, zero fill outside the matrix.
+mdbf_status_t make_act_tensor_map(CUtensorMap *out, const void *base, size_t rows, int cols, int stride, int box_rows) {
     typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -491,8 +492,8 @@ mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows
         }
         fn = reinterpret_cast<encode_fn>(p);
     }
-    const cuuint64_t gdim[2] = {(cuuint64_t)pad, (cuuint64_t)rows};
-    const cuuint64_t gstride[1] = {(cuuint64_t)pad * 2};
+    const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)stride * 2};
     const cuuint32_t box[2] = {PF_BK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
@@ -503,6 +504,10 @@ mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows
         return MDBF_ERR_CUDA;
     }
     return MDBF_OK;
+}
+// Tensor map of a pre-scaled operand: bf16 [rows][pad] row-major.
+mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad, int box_rows) {
+    return make_act_tensor_map(out, base, rows, pad, pad, box_rows);
 }
 
 // ---------------------------------------------------------------------- launch

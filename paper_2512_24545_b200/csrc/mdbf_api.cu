@@ -58,7 +58,7 @@ static mdbf_status_t check_handle(mdbf_handle_t h, const char *fn) {
 }
 
 static void free_layer(Layer &L) {
-    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.vpA, L.vpB, L.vxA, L.vxB, L.wk2A, L.wk2B, L.wkA, L.wkB, L.vtB, L.xsB, L.xsA, L.z, L.zsum, L.xstage, L.ystage, L.status};
+    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.vpA, L.vpB, L.vxA, L.vxB, L.wk2A, L.wk2B, L.wkA, L.wkB, L.uiA, L.uiB, L.viA, L.viB, L.vtB, L.xsB, L.xsA, L.z, L.zsum, L.xstage, L.ystage, L.status};
     for (void *p : ptrs)
         if (p) cudaFree(p);
 }
@@ -197,6 +197,13 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
         PACK_CUDA(cudaMalloc(&L.xsA, L.xs_rows * L.padA * 2));
         PACK_CUDA(cudaMemsetAsync(L.xsB, 0, L.xs_rows * L.padB * 2, st));
         PACK_CUDA(cudaMemsetAsync(L.xsA, 0, L.xs_rows * L.padA * 2, st));
+        // the materialised-envelope kernel keeps its bf16 intermediate [max_T][padA] in the same scratch
+        L.zb = L.xsA;
+        L.kcm = d.l <= 16 ? 2 : 4;
+        PACK_CUDA(cudaMalloc(&L.uiA, (size_t)(L.rpA / 128) * L.kcm * 1024 * sizeof(uint16_t)));
+        PACK_CUDA(cudaMalloc(&L.uiB, (size_t)(L.rpB / 128) * L.kcm * 1024 * sizeof(uint16_t)));
+        PACK_CUDA(cudaMalloc(&L.viA, (size_t)(L.padA / 64) * L.kcm * 512 * sizeof(uint16_t)));
+        PACK_CUDA(cudaMalloc(&L.viB, (size_t)(L.padB / 64) * L.kcm * 512 * sizeof(uint16_t)));
         for (int i = 0; i < 3; ++i) {
             PACK_RC(make_xs_tensor_map(&L.tmB[i], L.xsB, L.xs_rows, L.padB, 64 << i));
             PACK_RC(make_xs_tensor_map(&L.tmA[i], L.xsA, L.xs_rows, L.padA, 64 << i));
@@ -245,6 +252,10 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     }
     if (want_prefill) {
         PACK_RC(launch_vtrans(L.VB, d.d_in, d.l, d.env_dtype, L.vtB, L.padB, L.LP, st));
+        PACK_RC(launch_uimg(L.UA, d.d_out, d.l, d.env_dtype, L.uiA, L.rpA / 128, L.kcm, st));
+        PACK_RC(launch_uimg(L.UB, d.k, d.l, d.env_dtype, L.uiB, L.rpB / 128, L.kcm, st));
+        PACK_RC(launch_vimg(L.VA, d.k, d.l, d.env_dtype, L.viA, L.padA / 64, L.kcm, st));
+        PACK_RC(launch_vimg(L.VB, d.d_in, d.l, d.env_dtype, L.viB, L.padB / 64, L.kcm, st));
     }
     PACK_CUDA(cudaStreamSynchronize(st));
     for (void *p : temps) cudaFree(p);
@@ -308,7 +319,7 @@ mdbf_status_t mdbf_get_desc(mdbf_handle_t h, mdbf_desc_t *out) {
 mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel) {
     mdbf_status_t rc = check_handle(h, "mdbf_set_kernel");
     if (rc) return rc;
-    if (kernel < MDBF_KERNEL_AUTO || kernel > MDBF_KERNEL_TMEM) {
+    if (kernel < MDBF_KERNEL_AUTO || kernel > MDBF_KERNEL_MAT) {
         set_error("mdbf_set_kernel: unknown kernel %d", kernel);
         return MDBF_ERR_INVALID_ARG;
     }
@@ -354,6 +365,7 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
     if (kernel == MDBF_KERNEL_ALU) rc = launch_forward_alu(L, x, y, T, act_dtype, st, &launches);
     else if (kernel == MDBF_KERNEL_DECODE) rc = launch_forward_decode(L, x, y, T, st, &launches);
     else if (kernel == MDBF_KERNEL_TMEM) rc = launch_forward_tmem(L, x, y, T, st, &launches);
+    else if (kernel == MDBF_KERNEL_MAT) rc = launch_forward_mat(L, x, y, T, st, &launches);
     else rc = launch_forward_prefill(L, x, y, T, st, &launches);
     if (rc == MDBF_OK) h->last_launches = launches;
     return rc;

@@ -1,0 +1,83 @@
+"""Parity of the materialised-envelope kernel (W_hat tiles rebuilt on the fly from Eq. me-dbf-basis,
+one GEMM of width T) with the CPU oracle: shapes that span several 128-row tiles, several K
+blocks, several token tiles and ragged tails in every dimension."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mdbf_oracle as orc
+from paper_2512_24545_b200 import inputs, mdbf as M
+from helpers import GpuLayer, TOL, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    from paper_2512_24545_b200 import build
+    build.build()
+    assert torch.cuda.is_available()
+
+
+def spec_of(d_out, d_in, k, l, **kw):
+    return inputs.scaled(inputs.qproj(1664), name="mat", d_out=d_out, d_in=d_in, k=k, l=l, outliers=False, **kw)
+
+
+@pytest.mark.parametrize("l,T", [(16, 16), (16, 48), (16, 5), (16, 2), (4, 64), (4, 100), (1, 256), (1, 300),
+                                 (3, 40), (8, 33), (20, 9), (32, 11), (16, 600)])
+def test_mat_kernel_small_shapes(l, T):
+    spec = spec_of(384, 576, 256, l)
+    x = inputs.make_activations(spec, T)
+    with GpuLayer(spec, T) as g:
+        ref = g.oracle_forward(x)
+        y = g.forward(x, kernel=M.KERNEL_MAT)
+        assert M.mdbf_poll_status(g.h) == 0
+        assert np.all(np.isfinite(y))
+        assert rel_err(y, ref) <= TOL["bf16"]
+        _, z_ref = orc.forward_staged(*g.oracle_args(), x.T.astype(np.float64))
+        assert rel_err(g.intermediate(T), z_ref.T) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("shape", [(1, 8, 1, 1), (100, 72, 50, 2), (129, 72, 130, 16), (300, 1000, 260, 5),
+                                   (130, 64, 65, 17)])
+def test_mat_kernel_ragged_shapes(shape):
+    d_out, d_in, k, l = shape
+    spec = spec_of(d_out, d_in, k, l)
+    x = inputs.make_activations(spec, 19)
+    with GpuLayer(spec, 19) as g:
+        y = g.forward(x, kernel=M.KERNEL_MAT)
+        assert M.mdbf_poll_status(g.h) == 0
+        # a one-term layer has nothing to average: worst case of the path's four bf16 roundings
+        # (W_hat of either stage, z, y), each at most 2^-8 relative
+        tol = 4 * 2.0 ** -8 if k == 1 else TOL["bf16"]
+        assert rel_err(y, g.oracle_forward(x)) <= tol
+
+
+@pytest.mark.parametrize("env_dtype", ["f16", "bf16"])
+def test_mat_kernel_envelope_types_and_other_kernels(env_dtype):
+    spec = spec_of(256, 512, 256, 16, env_dtype=env_dtype)
+    x = inputs.make_activations(spec, 64)
+    with GpuLayer(spec, 64) as g:
+        ref = g.oracle_forward(x)
+        y_mat = g.forward(x, kernel=M.KERNEL_MAT)
+        y_pf = g.forward(x, kernel=M.KERNEL_PREFILL)
+        assert rel_err(y_mat, ref) <= TOL["bf16"] and rel_err(y_pf, ref) <= TOL["bf16"]
+        assert rel_err(y_mat, y_pf) <= 2 * TOL["bf16"]
+        # repeated calls give the same bits
+        np.testing.assert_array_equal(y_mat, g.forward(x, kernel=M.KERNEL_MAT))
+
+
+def test_mat_kernel_rejects_what_it_cannot_take():
+    spec = spec_of(128, 100, 64, 4)                       # d_in not a multiple of 8: no tensor map over x
+    x = inputs.make_activations(spec, 8)
+    with GpuLayer(spec, 8) as g:
+        with pytest.raises(M.MdbfError) as e:
+            g.forward(x, kernel=M.KERNEL_MAT)
+        assert e.value.status == M.ERR_SHAPE
+        assert rel_err(g.forward(x), g.oracle_forward(x)) <= TOL["bf16"]       # AUTO still serves it
+    spec = spec_of(128, 128, 64, 4)
+    x1 = inputs.make_activations(spec, 1)
+    with GpuLayer(spec, 8) as g:
+        with pytest.raises(M.MdbfError) as e:
+            g.forward(x1, kernel=M.KERNEL_MAT)                                  # one token
+        assert e.value.status == M.ERR_SHAPE
