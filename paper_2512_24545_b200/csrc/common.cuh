@@ -57,7 +57,7 @@ struct Layer {
     CUtensorMap tmB[3], tmA[3];   // tensor maps of xsB / xsA with boxes of 64, 128 and 256 rows (few tokens load a narrow box)
     // materialised-envelope kernel: 16-bit envelope images in mini-MMA operand order (see forward_mat.cu)
     uint16_t *uiA, *uiB;          // U images [row blocks][kcm][16][8][8]
-    uint16_t *viA, *viB;          // V images [K blocks][kcm][8][8][8]
+    uint16_t *viA, *viB;          // V images [pairs of K blocks][kcm][16][8][8]
     int kcm;                      // 16-byte chunks of the mode axis: 2 (l <= 16) or 4 (l <= 32)
     __nv_bfloat16 *zb;            // bf16 intermediate [max_T][padA]
     // scratch
@@ -115,7 +115,6 @@ mdbf_status_t launch_vtrans(const void *V, int cols, int l, int env_dtype, float
 mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad, int box_rows);
 mdbf_status_t make_act_tensor_map(CUtensorMap *out, const void *base, size_t rows, int cols, int stride, int box_rows);
 mdbf_status_t launch_uimg(const void *U, int rows, int l, int env_dtype, uint16_t *out, int rblocks, int kc, cudaStream_t st);
-mdbf_status_t launch_vimg(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int kc, cudaStream_t st);
 mdbf_status_t launch_forward_mat(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches);
 bool mat_path_supports(const Layer &L, const void *x, int T);
 mdbf_status_t launch_zb_to_zsum(Layer &L, int T, cudaStream_t st);

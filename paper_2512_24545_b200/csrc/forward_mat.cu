@@ -13,20 +13,21 @@
 // two launches per forward.  The result differs from the expanded order only in rounding:
 // W_hat is rounded to bf16 once per entry, the activations are not rounded at all.
 //
-// CTA = 128 rows of W_hat x up to 256 tokens, 12 warps:
-//   warps 0-7  two groups of four on alternate K blocks (64 columns).  Per block a thread (= row =
-//              TMEM lane) reads its 64 fp32 envelope values with tcgen05.ld, packs pairs to bf16,
-//              XORs the sign bits of its 64 packed bits in, and writes the 128B-swizzled A tile.
-//              Afterwards both groups run the epilogue on alternate 32-token chunks.
-//   warp 8     one lane issues the TMA load of the activation tile [tokens x 64]
-//   warp 9     one lane issues the 4 main MMAs of a K block and commits the stage
-//   warp 10    one lane bulk-copies the envelope images (U once, V per K block, ring of 6 or 8)
-//   warp 11    one lane issues the mini-MMAs (U image x V image, no swizzle) into a ring of four
-//              64-column TMEM buffers, as far ahead of the main MMAs as the ring allows.  A warp of
-//              its own: one thread's chain of barrier tests, MMAs and commits would otherwise cap
-//              the rate of the main MMAs.
-// Ring: stages of (A 16 KB + activation tile), 4 deep at 256 tokens per tile and up to 10 deep with
-// narrower tiles.  TMEM: 256 accumulator + 4 x 64 envelope columns.
+// CTA = 128 rows of W_hat x up to 256 tokens, 20 warps; the unit of the pipeline is a PAIR of K blocks
+// (2 x 64 columns), because every barrier test, MMA and commit costs the issuing thread 60-150 cycles:
+//   warps 0-15 tile builders: warp = (half of a block's 64 columns, block of the pair, 32-row quadrant).
+//              Per pair a thread (= row = TMEM lane) reads its 32 fp32 envelope values with tcgen05.ld,
+//              packs pairs to bf16, XORs the sign bits of its 32 packed bits in, and writes 16 TMEM
+//              columns of the W_hat tile with tcgen05.st (the A operand of the main MMA lives in TMEM:
+//              no shared-memory round trip, no proxy fence).  Afterwards they run the epilogue.
+//   warp 16    one lane issues the TMA loads of the activation tiles [tokens x 64] of a pair
+//   warp 17    one lane issues the 8 main MMAs of a pair (A from TMEM, B from shared memory); one commit
+//              frees the TMEM slot, one the pair of activation tiles
+//   warp 18    one lane bulk-copies the envelope images (U once, V per pair, ring of 3 or 4)
+//   warp 19    one lane issues the mini-MMA of a pair (U image x V image, 128 columns, no swizzle)
+// Shared memory holds only activation tiles (ring of 6 at 256 tokens per tile: the L2 latency of a
+// 32 KB tile is about one pair of MMA time, so the ring must run two pairs ahead) and the images.
+// TMEM: 256 accumulator + 128 envelope + 2 x 64 W_hat columns.
 //
 // Every mbarrier wait is bounded; when one expires the kernel records MDBF_ERR_TIMEOUT in the
 // layer's status word, all roles fall through to the common exit, TMEM is released and the kernel
@@ -38,19 +39,15 @@ namespace mdbf {
 constexpr int MT_BM = 128;
 constexpr int MT_BN = 256;
 constexpr int MT_BK = 64;
-constexpr int MT_STAGES = 4;
-constexpr int MT_GROUPS = 2;
-constexpr int MT_W_TMA = MT_GROUPS * 4;
+constexpr int MT_XWARPS = 16;            // tile builders: (block of the pair) x (half of its 64 columns) x (32-row quadrant)
+constexpr int MT_W_TMA = MT_XWARPS;
 constexpr int MT_W_MMA = MT_W_TMA + 1;
 constexpr int MT_W_ENV = MT_W_TMA + 2;
 constexpr int MT_W_MINI = MT_W_TMA + 3;
 constexpr int MT_THREADS = (MT_W_MINI + 1) * 32;
-constexpr int MT_A_BYTES = MT_BM * MT_BK * 2;
-constexpr int MT_B_BYTES = MT_BN * MT_BK * 2;
-constexpr int MT_MAX_NS = 10;            // ring depth: 4 stages at 256 tokens per tile, more with narrower tiles
-constexpr int MT_RING_BYTES = MT_STAGES * (MT_A_BYTES + MT_B_BYTES);
-constexpr int MT_NE = 4;                 // envelope buffers in TMEM
-constexpr int MT_MAX_NV = 8;             // V-image ring depth (8 with l <= 16, 6 with l <= 32)
+constexpr int MT_MAX_NS = 12;            // activation-tile ring depth: 6 tiles of 256 tokens, more with narrower tiles
+constexpr int MT_NA = 2;                 // W_hat tile slots in TMEM, a pair of K blocks (2 x 32 columns) each
+constexpr int MT_MAX_NV = 4;             // V-image ring depth in pairs of K blocks (4 with l <= 16, 3 with l <= 32)
 constexpr int MT_TMEM_COLS = 512;
 
 struct MatArgs {
@@ -58,13 +55,13 @@ struct MatArgs {
     int rows_pad;
     int rows, cols;
     const uint16_t *uimg;    // [row block][KC][16][8][8] 16-bit envelope values (see uimg_kernel)
-    const uint16_t *vimg;    // [K block][KC][8][8][8]
+    const uint16_t *vimg;    // [pair of K blocks][KC][16][8][8]: the same layout with the 128 columns of the pair as rows
     int kc;                  // 16-byte chunks of the mode axis: 2 (l <= 16) or 4 (l <= 32)
     uint32_t env_fmt;        // 0: f16 envelopes, 1: bf16
-    int nv;                  // V-image ring depth
+    int nv;                  // V-image ring depth (pairs of K blocks)
     int T;
     int bn;                  // tokens per CTA tile = MMA N = rows of the TMA box (multiple of 16, <= 256)
-    int ns;                  // ring depth (stages of A tile + activation tile)
+    int ns;                  // activation-tile ring depth, even
     __nv_bfloat16 *zb;       // stage B: bf16 intermediate [T][zstride]
     int zstride;
     __nv_bfloat16 *y;        // stage A: [T][rows]
@@ -90,22 +87,6 @@ __global__ void uimg_kernel(const void *__restrict__ U, int rows, int l, int env
         out[idx] = v;
     }
 }
-// V of one K block as the B operand: column 64*kb + 8*g + i, mode 8*c + e at ((c*8 + g)*8 + i)*8 + e.
-__global__ void vimg_kernel(const void *__restrict__ V, int cols, int l, int env_dtype, uint16_t *__restrict__ out,
-                            int kblocks, int kc) {
-    const size_t per = (size_t)kc * 8 * 64;
-    const size_t total = (size_t)kblocks * per;
-    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
-        const int kb = (int)(idx / per);
-        const int rem = (int)(idx % per);
-        const int e = rem & 7, i = (rem >> 3) & 7, g = (rem >> 6) & 7, c = rem >> 9;
-        const int col = kb * 64 + g * 8 + i, t = c * 8 + e;
-        uint16_t v = 0;
-        if (col < cols && t < l) v = reinterpret_cast<const uint16_t *>(V)[(size_t)col * l + t];
-        out[idx] = v;
-    }
-}
-
 static int mt_grid(size_t items) {
     size_t g = (items + 255) / 256;
     if (g < 1) g = 1;
@@ -117,30 +98,40 @@ mdbf_status_t launch_uimg(const void *U, int rows, int l, int env_dtype, uint16_
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
-mdbf_status_t launch_vimg(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int kc, cudaStream_t st) {
-    vimg_kernel<<<mt_grid((size_t)kblocks * kc * 512), 256, 0, st>>>(V, cols, l, env_dtype, out, kblocks, kc);
-    MDBF_CUDA(cudaGetLastError());
-    return MDBF_OK;
-}
-
 // 32 columns of one row of the A tile: envelope values -> bf16 pairs, sign bits XOR-ed in.
-// `word` holds the row's 32 sign bits of these columns (bit set = -1); chunk c4 of 8 columns goes
-// to the 16-byte slot (cbase + c4) ^ (row & 7) of the row (128B swizzle).
-__device__ __forceinline__ void mt_expand_half(const uint32_t (&v)[32], uint32_t word, unsigned char *srow, int arow, int cbase) {
+// `word` holds the row's 32 sign bits of these columns (bit set = -1).
+__device__ __forceinline__ void mt_expand_half(const uint32_t (&v)[32], uint32_t word, uint32_t (&o)[16]) {
 #pragma unroll
     for (int c4 = 0; c4 < 4; ++c4) {
         const uint32_t byte = (word >> (8 * c4)) & 0xFFu;   // 8 bits: the two shifted copies in the product below cannot overlap
-        uint32_t o[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int col = c4 * 8 + 2 * i;
             const uint32_t e = tm::pack_bf16x2(__uint_as_float(v[col]), __uint_as_float(v[col + 1]));
             // bit 0 of the shifted byte -> bit 15, bit 1 -> bit 31; the other product bits fall outside the mask
             const uint32_t m = ((byte >> (2 * i)) * 0x40008000u) & 0x80008000u;
-            o[i] = e ^ m;
+            o[c4 * 4 + i] = e ^ m;
         }
-        *reinterpret_cast<uint4 *>(srow + (((cbase + c4) ^ (arow & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
     }
+}
+// Barriers tested together, so that the latencies of the tests overlap.
+__device__ __forceinline__ bool mt_wait2(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
+                                         volatile int *abort_flag, int32_t *status) {
+    const uint32_t oa = tm::mbar_try_wait(bar_a, par_a), ob = tm::mbar_try_wait(bar_b, par_b);
+    if (oa & ob) return true;
+    if (!oa && !tm::mbar_wait(bar_a, par_a, abort_flag, status)) return false;
+    if (!ob && !tm::mbar_wait(bar_b, par_b, abort_flag, status)) return false;
+    return true;
+}
+__device__ __forceinline__ bool mt_wait3(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b, uint32_t bar_c,
+                                         uint32_t par_c, volatile int *abort_flag, int32_t *status) {
+    const uint32_t oa = tm::mbar_try_wait(bar_a, par_a), ob = tm::mbar_try_wait(bar_b, par_b),
+                   oc = tm::mbar_try_wait(bar_c, par_c);
+    if (oa & ob & oc) return true;
+    if (!oa && !tm::mbar_wait(bar_a, par_a, abort_flag, status)) return false;
+    if (!ob && !tm::mbar_wait(bar_b, par_b, abort_flag, status)) return false;
+    if (!oc && !tm::mbar_wait(bar_c, par_c, abort_flag, status)) return false;
+    return true;
 }
 
 template <bool STAGE_A>
@@ -148,25 +139,25 @@ __global__ void __launch_bounds__(MT_THREADS, 1)
 mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in) {
     using namespace tm;
     extern __shared__ unsigned char mt_smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * MT_MAX_NS + 2 * MT_NE + 2 * MT_MAX_NV + 2];
+    __shared__ __align__(8) uint64_t bars[MT_MAX_NS + MT_MAX_NS / 2 + 2 * MT_NA + 2 + 2 * MT_MAX_NV + 2];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
     volatile int *abort_flag = &abort_flag_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = (smem_u32(mt_smem_raw) + 1023u) & ~1023u;
-    unsigned char *smem_gen = mt_smem_raw + (smem_base - smem_u32(mt_smem_raw));
-    const int ns = a.ns, nv = a.nv;
-    const uint32_t b_bytes = (uint32_t)a.bn * MT_BK * 2;
-    const uint32_t stage_bytes = MT_A_BYTES + b_bytes;              // A tile, then the activation tile
-    const uint32_t u_smem = smem_base + (uint32_t)ns * stage_bytes;
-    const uint32_t u_bytes = (uint32_t)a.kc * 2048u, v_bytes = (uint32_t)a.kc * 1024u;
-    const uint32_t v_smem = u_smem + u_bytes;                       // + vb * v_bytes
-    const uint32_t full_bar = smem_u32(&bars[0]);
-    const uint32_t empty_bar = full_bar + 8 * MT_MAX_NS;
-    const uint32_t efull_bar = empty_bar + 8 * MT_MAX_NS;
-    const uint32_t eempty_bar = efull_bar + 8 * MT_NE;
-    const uint32_t vfull_bar = eempty_bar + 8 * MT_NE;
+    const int nbp = a.ns / 2, nv = a.nv;                            // activation-tile slots in pairs, V-image slots
+    const uint32_t b_bytes = (uint32_t)a.bn * MT_BK * 2;            // one activation tile
+    const uint32_t u_smem = smem_base + (uint32_t)a.ns * b_bytes;
+    const uint32_t img_bytes = (uint32_t)a.kc * 2048u;              // U image of a row block, V image of a pair of K blocks
+    const uint32_t v_smem = u_smem + img_bytes;                     // + vb * img_bytes
+    const uint32_t bfull_bar = smem_u32(&bars[0]);                  // per activation tile
+    const uint32_t bempty_bar = bfull_bar + 8 * MT_MAX_NS;          // per pair of activation tiles
+    const uint32_t afull_bar = bempty_bar + 8 * (MT_MAX_NS / 2);    // per pair of W_hat tiles in TMEM
+    const uint32_t aempty_bar = afull_bar + 8 * MT_NA;
+    const uint32_t efull_bar = aempty_bar + 8 * MT_NA;
+    const uint32_t eempty_bar = efull_bar + 8;
+    const uint32_t vfull_bar = eempty_bar + 8;
     const uint32_t vempty_bar = vfull_bar + 8 * MT_MAX_NV;
     const uint32_t accum_bar = vempty_bar + 8 * MT_MAX_NV;
     const uint32_t u_bar = accum_bar + 8;
@@ -175,16 +166,17 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in) {
     const int row0 = rb * MT_BM;
     const int tau0 = blockIdx.y * a.bn;
     const int nkb = (a.cols + MT_BK - 1) / MT_BK;
+    const int npr = (nkb + 1) / 2;                                  // pairs of K blocks; the last one may hold one block
 
     if (tid == 0) {
-        for (int s = 0; s < MT_MAX_NS; ++s) {
-            mbar_init(full_bar + 8 * s, 128 + 1);       // one expander group + the TMA issuer's expect_tx
-            mbar_init(empty_bar + 8 * s, 1);
+        for (int s = 0; s < MT_MAX_NS; ++s) mbar_init(bfull_bar + 8 * s, 1);
+        for (int s = 0; s < MT_MAX_NS / 2; ++s) mbar_init(bempty_bar + 8 * s, 1);
+        for (int s = 0; s < MT_NA; ++s) {
+            mbar_init(afull_bar + 8 * s, MT_XWARPS);                // one arrival per builder warp
+            mbar_init(aempty_bar + 8 * s, 1);
         }
-        for (int e = 0; e < MT_NE; ++e) {
-            mbar_init(efull_bar + 8 * e, 1);
-            mbar_init(eempty_bar + 8 * e, 128);
-        }
+        mbar_init(efull_bar, 1);
+        mbar_init(eempty_bar, MT_XWARPS);
         for (int v = 0; v < MT_MAX_NV; ++v) {
             mbar_init(vfull_bar + 8 * v, 1);
             mbar_init(vempty_bar + 8 * v, 1);
@@ -201,45 +193,55 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in) {
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_d = tmem_base_slot;              // accumulator: columns 0 .. 255
-    const uint32_t tmem_e = tmem_base_slot + MT_BN;      // envelope buffers: 64 columns each
+    const uint32_t tmem_d = tmem_base_slot;                   // accumulator: columns 0 .. 255
+    const uint32_t tmem_e = tmem_base_slot + MT_BN;           // envelope values of a pair of K blocks: 128 columns
+    const uint32_t tmem_a = tmem_e + 2 * MT_BK;               // W_hat tiles: MT_NA pairs x (2 blocks x 32 columns of bf16 pairs)
     pdl_launch_dependents();
 
     if (warp < MT_W_TMA) {
         // ============================ W_hat tile builders ============================
-        const int grp = warp >> 2;
+        // warp = (half of the 64 columns, block of the pair, 32-row quadrant); every warp works on every pair
+        const int grp = (warp >> 2) & 1, half = warp >> 3;
         const int arow = tid & 127;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint2 *wp = a.wk + (size_t)row0 + arow;                       // + kb * rows_pad
-        uint2 w_next = grp < nkb ? __ldg(wp + (size_t)grp * a.rows_pad) : make_uint2(0u, 0u);
-        uint2 w_next2 = grp + MT_GROUPS < nkb ? __ldg(wp + (size_t)(grp + MT_GROUPS) * a.rows_pad) : make_uint2(0u, 0u);
+        const uint32_t *wp = reinterpret_cast<const uint32_t *>(a.wk + (size_t)row0 + arow) + half;   // + kb * rows_pad * 2
+        const size_t wstride = (size_t)a.rows_pad * 2;
+        uint32_t w_next = grp < nkb ? __ldg(wp + (size_t)grp * wstride) : 0u;
+        uint32_t w_next2 = grp + 2 < nkb ? __ldg(wp + (size_t)(grp + 2) * wstride) : 0u;
         bool alive = true;
-        int s = grp;                                      // ring slot and phase of K block kb (ns >= 4 > grp)
-        uint32_t ph = 0;
-        for (int kb = grp; kb < nkb && alive; kb += MT_GROUPS) {
-            const int eb = kb & (MT_NE - 1);
-            const uint32_t eph = (uint32_t)(kb / MT_NE) & 1u;
-            const uint2 w = w_next;
+        for (int p = 0; p < npr && alive; ++p) {          // (the second block of an odd tail pair is built from zeros and not used)
+            const int kb = 2 * p + grp;
+            const int as = p & (MT_NA - 1);
+            const uint32_t aph = (uint32_t)(p / MT_NA) & 1u;
+            const uint32_t w = w_next;
             w_next = w_next2;
-            if (kb + 2 * MT_GROUPS < nkb) w_next2 = __ldg(wp + (size_t)(kb + 2 * MT_GROUPS) * a.rows_pad);
-            alive = mbar_wait(efull_bar + 8 * eb, eph, abort_flag, a.status);
+            w_next2 = kb + 4 < nkb ? __ldg(wp + (size_t)(kb + 4) * wstride) : 0u;
+            alive = mbar_wait(efull_bar, (uint32_t)p & 1u, abort_flag, a.status);
             if (!alive) break;
             tc_fence_after();
-            uint32_t v0[32], v1[32];
-            tmem_ld32(tmem_e + (uint32_t)(eb * 64) + lane_base, v0);
-            tmem_ld32(tmem_e + (uint32_t)(eb * 64 + 32) + lane_base, v1);
+            uint32_t v[32];
+            tmem_ld32(tmem_e + (uint32_t)(grp * 64 + half * 32) + lane_base, v);
             tmem_ld_wait();
             tc_fence_before();
-            mbar_arrive(eempty_bar + 8 * eb);                                // the buffer may be overwritten
-            alive = mbar_wait(empty_bar + 8 * s, ph ^ 1u, abort_flag, a.status);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(eempty_bar);                          // the buffer may be overwritten
+            // the row is finished in registers before the tile slot is claimed: only the stores follow the wait
+            uint32_t o[16];
+            mt_expand_half(v, w, o);
+            alive = mbar_wait(aempty_bar + 8 * as, aph ^ 1u, abort_flag, a.status);
             if (!alive) break;
-            unsigned char *srow = smem_gen + (size_t)s * stage_bytes + arow * 128;
-            mt_expand_half(v0, w.x, srow, arow, 0);
-            mt_expand_half(v1, w.y, srow, arow, 4);
-            fence_proxy_async();
-            mbar_arrive(full_bar + 8 * s);
-            s += MT_GROUPS;
-            if (s >= ns) { s -= ns; ph ^= 1u; }
+            tc_fence_after();
+            const uint32_t a_col = tmem_a + (uint32_t)(as * 64 + grp * 32 + half * 16) + lane_base;
+            {
+                const uint32_t (&lo)[8] = *reinterpret_cast<const uint32_t (*)[8]>(&o[0]);
+                const uint32_t (&hi)[8] = *reinterpret_cast<const uint32_t (*)[8]>(&o[8]);
+                tmem_st8(a_col, lo);
+                tmem_st8(a_col + 8, hi);
+            }
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(afull_bar + 8 * as);
         }
 
         // ================================= epilogue ==================================
@@ -249,7 +251,7 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in) {
         pdl_wait();                                   // the stores below must follow the previous kernel's reads
         if (alive) {
 #pragma unroll 1
-            for (int ld = grp; ld * 32 < a.bn; ld += MT_GROUPS) {
+            for (int ld = warp >> 2; ld * 32 < a.bn; ld += MT_XWARPS / 4) {      // four warps share a lane quadrant: alternate chunks
                 const int col0 = ld * 32;
                 uint32_t v[32];
                 tmem_ld32(tmem_d + lane_base + (uint32_t)col0, v);
@@ -272,92 +274,95 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in) {
         }
     } else if (warp == MT_W_TMA) {
         // ============================ activation-tile loader ===========================
-        bool alive = true;
-        pdl_wait();                                   // the activations come from the previous kernel
-        int s = 0;
-        uint32_t ph = 0;
-        for (int kb = 0; kb < nkb && alive; ++kb) {
-            alive = mbar_wait(empty_bar + 8 * s, ph ^ 1u, abort_flag, a.status);
-            if (!alive) break;
-            if (lane == 0) {
-                mbar_arrive_expect_tx(full_bar + 8 * s, b_bytes);
-                tma_load_2d(smem_base + (uint32_t)s * stage_bytes + MT_A_BYTES, &tmap_in, kb * MT_BK, tau0,
-                            full_bar + 8 * s);
+        if (lane == 0) {
+            bool alive = true;
+            pdl_wait();                               // the activations come from the previous kernel
+            int bp = 0;
+            uint32_t ph = 0;
+            for (int p = 0; p < npr && alive; ++p) {
+                alive = mbar_wait(bempty_bar + 8 * bp, ph ^ 1u, abort_flag, a.status);
+                if (!alive) break;
+                for (int h = 0; h < 2 && 2 * p + h < nkb; ++h) {
+                    const int s = 2 * bp + h;
+                    mbar_arrive_expect_tx(bfull_bar + 8 * s, b_bytes);
+                    tma_load_2d(smem_base + (uint32_t)s * b_bytes, &tmap_in, (2 * p + h) * MT_BK, tau0, bfull_bar + 8 * s);
+                }
+                if (++bp == nbp) { bp = 0; ph ^= 1u; }
             }
-            __syncwarp();
-            if (++s == ns) { s = 0; ph ^= 1u; }
+            if (!alive) drain_delay();
         }
-        if (!alive) drain_delay();
+        __syncwarp();
     } else if (warp == MT_W_ENV) {
         // ============================= envelope-image loader ===========================
-        bool alive = true;
         if (lane == 0) {
-            mbar_arrive_expect_tx(u_bar, u_bytes);
-            bulk_load(u_smem, a.uimg + (size_t)rb * (u_bytes / 2), u_bytes, u_bar);
-        }
-        int vb = 0;
-        uint32_t vph = 0;
-        for (int kb = 0; kb < nkb && alive; ++kb) {
-            alive = mbar_wait(vempty_bar + 8 * vb, vph ^ 1u, abort_flag, a.status);
-            if (!alive) break;
-            if (lane == 0) {
-                mbar_arrive_expect_tx(vfull_bar + 8 * vb, v_bytes);
-                bulk_load(v_smem + (uint32_t)vb * v_bytes, a.vimg + (size_t)kb * (v_bytes / 2), v_bytes, vfull_bar + 8 * vb);
+            bool alive = true;
+            mbar_arrive_expect_tx(u_bar, img_bytes);
+            bulk_load(u_smem, a.uimg + (size_t)rb * (img_bytes / 2), img_bytes, u_bar);
+            int vb = 0;
+            uint32_t vph = 0;
+            for (int p = 0; p < npr && alive; ++p) {
+                alive = mbar_wait(vempty_bar + 8 * vb, vph ^ 1u, abort_flag, a.status);
+                if (!alive) break;
+                mbar_arrive_expect_tx(vfull_bar + 8 * vb, img_bytes);
+                bulk_load(v_smem + (uint32_t)vb * img_bytes, a.vimg + (size_t)p * (img_bytes / 2), img_bytes, vfull_bar + 8 * vb);
+                if (++vb == nv) { vb = 0; vph ^= 1u; }
             }
-            __syncwarp();
-            if (++vb == nv) { vb = 0; vph ^= 1u; }
+            if (!alive) drain_delay();
         }
-        if (!alive) drain_delay();
+        __syncwarp();
     } else if (warp == MT_W_MINI) {
-        // ===================== envelope mini-MMA issuer: E(j) = U image x V image(j)^T =====================
-        // runs as far ahead of the main MMAs as the four TMEM buffers allow
-        const uint32_t idesc_mini = make_idesc_fmt(MT_BK, a.env_fmt);
-        bool alive = mbar_wait(u_bar, 0u, abort_flag, a.status);
-        int vb = 0;
-        uint32_t vph = 0;
-        for (int j = 0; j < nkb && alive; ++j) {
-            const int eb = j & (MT_NE - 1);
-            alive = mbar_wait(vfull_bar + 8 * vb, vph, abort_flag, a.status);
-            if (!alive) break;
-            alive = mbar_wait(eempty_bar + 8 * eb, ((uint32_t)(j / MT_NE) & 1u) ^ 1u, abort_flag, a.status);
-            if (!alive) break;
-            tc_fence_after();
-            if (lane == 0) {
+        // ============ envelope mini-MMA issuer: E(pair p) = U image x V image(p)^T, 128 columns ============
+        if (lane == 0) {
+            const uint32_t idesc_mini = make_idesc_fmt(2 * MT_BK, a.env_fmt);
+            bool alive = mbar_wait(u_bar, 0u, abort_flag, a.status);
+            int vb = 0;
+            uint32_t vph = 0;
+            for (int p = 0; p < npr && alive; ++p) {
+                alive = mt_wait2(vfull_bar + 8 * vb, vph, eempty_bar, ((uint32_t)p & 1u) ^ 1u, abort_flag, a.status);
+                if (!alive) break;
+                tc_fence_after();
                 for (int q = 0; q < a.kc / 2; ++q) {
                     const uint64_t ud = make_smem_desc_plain(u_smem + (uint32_t)q * 4096u, 2048u, 128u);
-                    const uint64_t vd = make_smem_desc_plain(v_smem + (uint32_t)vb * v_bytes + (uint32_t)q * 2048u, 1024u, 128u);
-                    umma_ss(tmem_e + (uint32_t)(eb * 64), ud, vd, idesc_mini, q > 0 ? 1u : 0u);
+                    const uint64_t vd = make_smem_desc_plain(v_smem + (uint32_t)vb * img_bytes + (uint32_t)q * 4096u, 2048u, 128u);
+                    umma_ss(tmem_e, ud, vd, idesc_mini, q > 0 ? 1u : 0u);
                 }
-                umma_commit(efull_bar + 8 * eb);
+                umma_commit(efull_bar);
                 umma_commit(vempty_bar + 8 * vb);
+                if (++vb == nv) { vb = 0; vph ^= 1u; }
             }
-            __syncwarp();
-            if (++vb == nv) { vb = 0; vph ^= 1u; }
         }
+        __syncwarp();
     } else {
         // ================================ main MMA issuer =================================
-        const uint32_t idesc_main = make_idesc(a.bn);
-        bool alive = true;
-        int s = 0;
-        uint32_t ph = 0;
-        for (int kb = 0; kb < nkb && alive; ++kb) {
-            alive = mbar_wait(full_bar + 8 * s, ph, abort_flag, a.status);
-            if (!alive) break;
-            tc_fence_after();
-            if (lane == 0) {
-                const uint32_t sA = smem_base + (uint32_t)s * stage_bytes;
-                const uint64_t adesc = make_smem_desc(sA);
-                const uint64_t bdesc = make_smem_desc(sA + MT_A_BYTES);
+        // a pair of K blocks per step: W_hat tiles from TMEM, activation tiles from shared memory, 8 MMAs,
+        // one commit frees the TMEM slot and one the pair of activation tiles
+        if (lane == 0) {
+            const uint32_t idesc_main = make_idesc(a.bn);
+            bool alive = true;
+            int bp = 0;
+            uint32_t ph = 0;
+            for (int p = 0; p < npr && alive; ++p) {
+                const int s0 = 2 * bp, as = p & (MT_NA - 1);
+                const uint32_t aph = (uint32_t)(p / MT_NA) & 1u;
+                const bool two = 2 * p + 1 < nkb;
+                alive = two ? mt_wait3(afull_bar + 8 * as, aph, bfull_bar + 8 * s0, ph, bfull_bar + 8 * (s0 + 1), ph, abort_flag, a.status)
+                            : mt_wait2(afull_bar + 8 * as, aph, bfull_bar + 8 * s0, ph, abort_flag, a.status);
+                if (!alive) break;
+                tc_fence_after();
+                for (int h = 0; h < (two ? 2 : 1); ++h) {
+                    const uint64_t bdesc = make_smem_desc(smem_base + (uint32_t)(s0 + h) * b_bytes);
+                    const uint32_t a_t = tmem_a + (uint32_t)(as * 64 + h * 32);
 #pragma unroll
-                for (int k4 = 0; k4 < MT_BK / 16; ++k4)
-                    umma_ss(tmem_d, adesc + (uint64_t)(2 * k4), bdesc + (uint64_t)(2 * k4), idesc_main,
-                            (kb > 0 || k4 > 0) ? 1u : 0u);
-                umma_commit(empty_bar + 8 * s);
+                    for (int k4 = 0; k4 < MT_BK / 16; ++k4)
+                        umma_ts(tmem_d, a_t + (uint32_t)(8 * k4), bdesc + (uint64_t)(2 * k4), idesc_main,
+                                (p > 0 || h > 0 || k4 > 0) ? 1u : 0u);
+                }
+                umma_commit(aempty_bar + 8 * as);
+                umma_commit(bempty_bar + 8 * bp);
+                if (++bp == nbp) { bp = 0; ph ^= 1u; }
             }
-            __syncwarp();
-            if (++s == ns) { s = 0; ph ^= 1u; }
+            if (alive) { if (nkb > 0) umma_commit(accum_bar); else mbar_arrive(accum_bar); }
         }
-        if (lane == 0 && alive) { if (nkb > 0) umma_commit(accum_bar); else mbar_arrive(accum_bar); }
         __syncwarp();
     }
 
@@ -385,12 +390,14 @@ bool mat_path_supports(const Layer &L, const void *x, int T) {
     return L.uiA && L.zb && T >= 2 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && L.d.d_in % 8 == 0;
 }
 
-static int mt_ring(int bn) {
-    const int n = MT_RING_BYTES / (MT_A_BYTES + bn * MT_BK * 2);
+// shared memory: ring of activation tiles, U image, ring of V images, alignment slack
+static int mt_ring(int kc, int nv, int bn) {
+    const size_t avail = 227 * 1024 - 1024 - 1024 - (size_t)(1 + nv) * kc * 2048;    // 1 KB static, 1 KB slack
+    const int n = (int)(avail / ((size_t)bn * MT_BK * 2)) / 2 * 2;
     return n < MT_MAX_NS ? n : MT_MAX_NS;
 }
 static size_t mt_smem_bytes(int kc, int nv, int bn) {
-    return (size_t)mt_ring(bn) * (MT_A_BYTES + bn * MT_BK * 2) + (size_t)kc * 2048 + (size_t)nv * kc * 1024 + 1024;
+    return (size_t)mt_ring(kc, nv, bn) * bn * MT_BK * 2 + (size_t)(1 + nv) * kc * 2048 + 1024;
 }
 
 template <bool STAGE_A>
@@ -398,7 +405,7 @@ static mdbf_status_t launch_mat(const MatArgs &a, const CUtensorMap &tm, cudaStr
     static bool attr_set = false;
     if (!attr_set) {
         MDBF_CUDA(cudaFuncSetAttribute(mat_stage_kernel<STAGE_A>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)mt_smem_bytes(4, 6, MT_BN)));
+                                       (int)mt_smem_bytes(4, 3, MT_BN)));
         attr_set = true;
     }
     cudaLaunchConfig_t cfg = {};
@@ -432,8 +439,8 @@ mdbf_status_t launch_forward_mat(Layer &L, const void *x, void *y, int T, cudaSt
     MatArgs b = {};
     b.wk = L.wkB; b.rows_pad = L.rpB; b.rows = d.k; b.cols = d.d_in;
     b.uimg = L.uiB; b.vimg = L.viB; b.kc = L.kcm; b.env_fmt = d.env_dtype == MDBF_BF16 ? 1u : 0u;
-    b.nv = L.kcm == 2 ? 8 : 6;
-    b.T = T; b.bn = bn; b.ns = mt_ring(bn); b.zb = L.zb; b.zstride = L.padA; b.status = L.status;
+    b.nv = L.kcm == 2 ? 4 : 3;
+    b.T = T; b.bn = bn; b.ns = mt_ring(b.kc, b.nv, bn); b.zb = L.zb; b.zstride = L.padA; b.status = L.status;
     rc = launch_mat<false>(b, tmx, st);
     if (rc) return rc;
 

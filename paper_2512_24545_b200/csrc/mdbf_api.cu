@@ -202,8 +202,8 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
         L.kcm = d.l <= 16 ? 2 : 4;
         PACK_CUDA(cudaMalloc(&L.uiA, (size_t)(L.rpA / 128) * L.kcm * 1024 * sizeof(uint16_t)));
         PACK_CUDA(cudaMalloc(&L.uiB, (size_t)(L.rpB / 128) * L.kcm * 1024 * sizeof(uint16_t)));
-        PACK_CUDA(cudaMalloc(&L.viA, (size_t)(L.padA / 64) * L.kcm * 512 * sizeof(uint16_t)));
-        PACK_CUDA(cudaMalloc(&L.viB, (size_t)(L.padB / 64) * L.kcm * 512 * sizeof(uint16_t)));
+        PACK_CUDA(cudaMalloc(&L.viA, (size_t)ceil_div(L.padA, 128) * L.kcm * 1024 * sizeof(uint16_t)));
+        PACK_CUDA(cudaMalloc(&L.viB, (size_t)ceil_div(L.padB, 128) * L.kcm * 1024 * sizeof(uint16_t)));
         for (int i = 0; i < 3; ++i) {
             PACK_RC(make_xs_tensor_map(&L.tmB[i], L.xsB, L.xs_rows, L.padB, 64 << i));
             PACK_RC(make_xs_tensor_map(&L.tmA[i], L.xsA, L.xs_rows, L.padA, 64 << i));
@@ -254,8 +254,8 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
         PACK_RC(launch_vtrans(L.VB, d.d_in, d.l, d.env_dtype, L.vtB, L.padB, L.LP, st));
         PACK_RC(launch_uimg(L.UA, d.d_out, d.l, d.env_dtype, L.uiA, L.rpA / 128, L.kcm, st));
         PACK_RC(launch_uimg(L.UB, d.k, d.l, d.env_dtype, L.uiB, L.rpB / 128, L.kcm, st));
-        PACK_RC(launch_vimg(L.VA, d.k, d.l, d.env_dtype, L.viA, L.padA / 64, L.kcm, st));
-        PACK_RC(launch_vimg(L.VB, d.d_in, d.l, d.env_dtype, L.viB, L.padB / 64, L.kcm, st));
+        PACK_RC(launch_uimg(L.VA, d.k, d.l, d.env_dtype, L.viA, ceil_div(L.padA, 128), L.kcm, st));     // V: columns of a pair of K blocks as rows
+        PACK_RC(launch_uimg(L.VB, d.d_in, d.l, d.env_dtype, L.viB, ceil_div(L.padB, 128), L.kcm, st));
     }
     PACK_CUDA(cudaStreamSynchronize(st));
     for (void *p : temps) cudaFree(p);
