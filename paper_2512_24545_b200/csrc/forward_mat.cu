@@ -67,6 +67,7 @@ struct MatArgs {
     __nv_bfloat16 *y;        // stage A: [T][rows]
     float *y32;              // stage A, fp32 output modes (y_mode 1: store, 2: add)
     int y_mode;
+    int tma_out;             // 1: bf16 output staged in shared memory and written by TMA (16-byte aligned base and pitch)
     int32_t *status;
 };
 
@@ -136,7 +137,7 @@ __device__ __forceinline__ bool mt_wait3(uint32_t bar_a, uint32_t par_a, uint32_
 
 template <bool STAGE_A>
 __global__ void __launch_bounds__(MT_THREADS, 1)
-mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in) {
+mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out) {
     using namespace tm;
     extern __shared__ unsigned char mt_smem_raw[];
     __shared__ __align__(8) uint64_t bars[MT_MAX_NS + MT_MAX_NS / 2 + 2 * MT_NA + 2 + 2 * MT_MAX_NV + 2];
@@ -146,6 +147,7 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in) {
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = (smem_u32(mt_smem_raw) + 1023u) & ~1023u;
+    unsigned char *smem_gen = mt_smem_raw + (smem_base - smem_u32(mt_smem_raw));
     const int nbp = a.ns / 2, nv = a.nv;                            // activation-tile slots in pairs, V-image slots
     const uint32_t b_bytes = (uint32_t)a.bn * MT_BK * 2;            // one activation tile
     const uint32_t u_smem = smem_base + (uint32_t)a.ns * b_bytes;
@@ -249,7 +251,34 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in) {
         if (alive) alive = mbar_wait(accum_bar, 0u, abort_flag, a.status);
         tc_fence_after();
         pdl_wait();                                   // the stores below must follow the previous kernel's reads
-        if (alive) {
+        // one decision per group of four warps (they meet at a barrier below): all of them arrive here, and a
+        // wait that expired in any thread has raised the abort flag before that thread arrived
+        asm volatile("bar.sync %0, 128;\n" ::"r"(1 + (warp >> 2)) : "memory");
+        alive = !*abort_flag;
+        if (alive && a.tma_out) {
+            // The four warps of group g = warp / 4 cover all 128 rows; they take tokens [64g, 64g + 64): accumulator ->
+            // bf16 [token][128 rows] in the (now idle) activation ring -> one TMA store per group, which clips
+            // rows and tokens outside the output.
+            const int g = warp >> 2;
+            if (g * 64 < a.bn) {
+                unsigned char *stg = smem_gen + g * (64 * MT_BM * 2);
+                for (int c = 0; c < 2 && g * 64 + c * 32 < a.bn; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_d + lane_base + (uint32_t)(g * 64 + c * 32), v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        *reinterpret_cast<__nv_bfloat16 *>(stg + (c * 32 + j) * (MT_BM * 2) + arow * 2) =
+                            __float2bfloat16_rn(__uint_as_float(v[j]));
+                }
+                fence_proxy_async();
+                asm volatile("bar.sync %0, 128;\n" ::"r"(1 + g) : "memory");
+                if ((tid & 127) == 0 && tau0 + g * 64 < a.T) {
+                    tma_store_2d(&tmap_out, row0, tau0 + g * 64, smem_base + (uint32_t)g * (64 * MT_BM * 2));
+                    bulk_commit_wait_all();
+                }
+            }
+        } else if (alive) {
 #pragma unroll 1
             for (int ld = warp >> 2; ld * 32 < a.bn; ld += MT_XWARPS / 4) {      // four warps share a lane quadrant: alternate chunks
                 const int col0 = ld * 32;
@@ -400,8 +429,38 @@ static size_t mt_smem_bytes(int kc, int nv, int bn) {
     return (size_t)mt_ring(kc, nv, bn) * bn * MT_BK * 2 + (size_t)(1 + nv) * kc * 2048 + 1024;
 }
 
+// Tensor map of a bf16 output [T][rows] with rows `pitch` elements apart: box of 128 rows x 64 tokens, no swizzle.
+static mdbf_status_t make_out_tensor_map(CUtensorMap *out, const void *base, int T, int rows, int pitch) {
+    typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static encode_fn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        MDBF_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q));
+        if (!p || q != cudaDriverEntryPointSuccess) {
+            set_error("cuTensorMapEncodeTiled is not available from the driver");
+            return MDBF_ERR_CUDA;
+        }
+        fn = reinterpret_cast<encode_fn>(p);
+    }
+    const cuuint64_t gdim[2] = {(cuuint64_t)rows, (cuuint64_t)T};
+    const cuuint64_t gstride[1] = {(cuuint64_t)pitch * 2};
+    const cuuint32_t box[2] = {MT_BM, 64};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled (output) failed with CUresult %d", (int)r);
+        return MDBF_ERR_CUDA;
+    }
+    return MDBF_OK;
+}
+
 template <bool STAGE_A>
-static mdbf_status_t launch_mat(const MatArgs &a, const CUtensorMap &tm, cudaStream_t st) {
+static mdbf_status_t launch_mat(const MatArgs &a, const CUtensorMap &tm, const CUtensorMap &tmo, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
         MDBF_CUDA(cudaFuncSetAttribute(mat_stage_kernel<STAGE_A>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -418,7 +477,7 @@ static mdbf_status_t launch_mat(const MatArgs &a, const CUtensorMap &tm, cudaStr
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    MDBF_CUDA(cudaLaunchKernelEx(&cfg, mat_stage_kernel<STAGE_A>, a, tm));
+    MDBF_CUDA(cudaLaunchKernelEx(&cfg, mat_stage_kernel<STAGE_A>, a, tm, tmo));
     return MDBF_OK;
 }
 
@@ -430,18 +489,28 @@ mdbf_status_t launch_forward_mat(Layer &L, const void *x, void *y, int T, cudaSt
         return MDBF_ERR_SHAPE;
     }
     const int bn = T >= MT_BN ? MT_BN : ((T + 15) / 16) * 16;
-    CUtensorMap tmx, tmz;
+    CUtensorMap tmx, tmz, tmzo, tmyo;
     mdbf_status_t rc = make_act_tensor_map(&tmx, x, (size_t)T, d.d_in, d.d_in, bn);
     if (rc) return rc;
     rc = make_act_tensor_map(&tmz, L.zb, (size_t)T, d.k, L.padA, bn);
     if (rc) return rc;
+    rc = make_out_tensor_map(&tmzo, L.zb, T, d.k, L.padA);
+    if (rc) return rc;
+    // y goes out by TMA when its base and row pitch are 16-byte aligned and it is bf16; otherwise by plain stores
+    const bool y_tma = L.out_mode == 0 && (reinterpret_cast<uintptr_t>(y) & 15u) == 0 && d.d_out % 8 == 0;
+    tmyo = tmzo;
+    if (y_tma) {
+        rc = make_out_tensor_map(&tmyo, y, T, d.d_out, d.d_out);
+        if (rc) return rc;
+    }
 
     MatArgs b = {};
     b.wk = L.wkB; b.rows_pad = L.rpB; b.rows = d.k; b.cols = d.d_in;
     b.uimg = L.uiB; b.vimg = L.viB; b.kc = L.kcm; b.env_fmt = d.env_dtype == MDBF_BF16 ? 1u : 0u;
     b.nv = L.kcm == 2 ? 4 : 3;
     b.T = T; b.bn = bn; b.ns = mt_ring(b.kc, b.nv, bn); b.zb = L.zb; b.zstride = L.padA; b.status = L.status;
-    rc = launch_mat<false>(b, tmx, st);
+    b.tma_out = 1;
+    rc = launch_mat<false>(b, tmx, tmzo, st);
     if (rc) return rc;
 
     MatArgs a = {};
@@ -449,7 +518,8 @@ mdbf_status_t launch_forward_mat(Layer &L, const void *x, void *y, int T, cudaSt
     a.uimg = L.uiA; a.vimg = L.viA; a.kc = L.kcm; a.env_fmt = b.env_fmt; a.nv = b.nv;
     a.T = T; a.bn = bn; a.ns = b.ns;
     a.y = reinterpret_cast<__nv_bfloat16 *>(y); a.y32 = reinterpret_cast<float *>(y); a.y_mode = L.out_mode; a.status = L.status;
-    rc = launch_mat<true>(a, tmz, st);
+    a.tma_out = y_tma ? 1 : 0;
+    rc = launch_mat<true>(a, tmz, tmyo, st);
     if (rc) return rc;
     L.last_ksplit = -1;
     *launches = 2;
