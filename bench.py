@@ -37,8 +37,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that workload).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    "decode_qproj": 1083648,                # tmem_t1_kernel, k = 1664 layer, either stage
-    "prefill_4096_l16_bpw10": 370142976,     # gemm_stage_kernel stage B: 269.4 MB read + 100.7 MB written
+    ("decode_qproj", "tmem_t1_kernel"): 1083648,                   # k = 1664 layer, either stage
+    ("prefill_4096_l16_bpw10", "gemm_stage_kernel"): 370142976,    # stage B: 269.4 MB read + 100.7 MB written
 }
 
 
@@ -71,6 +71,14 @@ def algorithmic_bytes(spec, T):
 
 def expanded_flops(spec, T):
     return 2.0 * spec.l * T * spec.k * (spec.d_in + spec.d_out)
+
+
+def rated_materialised(spec, T, forced="auto"):
+    """Whether a tensor-bound workload is rated in FLOPs of the materialised order: mirrors the library's
+    dispatch (T >= 64, or 128 for the rank-1 envelope, runs the materialised-order kernel)."""
+    if forced != "auto":
+        return forced == "mat"
+    return T >= (128 if spec.l == 1 else 64)
 
 
 def materialised_flops(spec, T):
@@ -323,7 +331,8 @@ def run_mdbf(args):
     else:
         # the expanded-order kernel is rated in FLOPs of the expanded contraction (which it executes); the
         # materialised-order kernel executes l x fewer and is rated in those, never in expanded FLOPs
-        mat = args.kernel == "mat" and T > 1
+        mat = M.mdbf_last_kernel(layers[0][0]) == M.KERNEL_MAT
+        assert mat == rated_materialised(groups[0][0], T, args.kernel), "bench.py's copy of the dispatch rule is stale"
         metric, unit = ("prefill_executed_TFLOPs" if mat else "prefill_expanded_TFLOPs"), "TFLOP/s"
         per_step = (total_mat_flops if mat else total_flops) / 1e12
         peak = peaks["bf16_tflops"] if sec < 1.0 else peaks["bf16_tflops_sustained"]
@@ -349,11 +358,12 @@ def run_mdbf(args):
         "clocks": clocks,
         "roofline": {"bound": bound, "achieved": per_gpu, "peak": peak, "unit": unit,
                      "frac": per_gpu / peak, "peak_source": f"of {peak_kind}",
-                     "kernel": dominant_kernel(groups[0][0], T, args.kernel),
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload) if args.kernel == "auto" else None},
+                     "kernel": dominant_kernel(groups[0][0], T, "mat" if M.mdbf_last_kernel(layers[0][0]) == M.KERNEL_MAT else "prefill"),
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.workload, dominant_kernel(groups[0][0], T, "mat" if M.mdbf_last_kernel(layers[0][0]) == M.KERNEL_MAT else "prefill")))},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(groups[0][0], T, bound, budget_s=20.0)
+        out["cpu_baseline"] = cpu_baseline(groups[0][0], T, bound, budget_s=20.0,
+                                           mat=bound != "hbm" and M.mdbf_last_kernel(layers[0][0]) == M.KERNEL_MAT)
     for (h, *_r) in layers:
         M.mdbf_destroy(h)
     if dist:
@@ -381,7 +391,7 @@ def oracle_sample(spec, T, rows_frac):
     return dt, n / spec.d_out
 
 
-def cpu_baseline(spec, T, bound, budget_s=15.0):
+def cpu_baseline(spec, T, bound, budget_s=15.0, mat=False):
     cores = len(os.sched_getaffinity(0))
     dt, frac = oracle_sample(spec, T, 1.0 / 64)          # probe
     frac_target = min(1.0, max(1.0 / 64, frac * budget_s / max(dt, 1e-3) * 0.5))
@@ -395,7 +405,7 @@ def cpu_baseline(spec, T, bound, budget_s=15.0):
     if bound == "hbm":
         v, unit = algorithmic_bytes(spec, T) * frac / 1e9 / dt, "GB/s"
     else:
-        v, unit = expanded_flops(spec, T) * frac / 1e12 / dt, "TFLOP/s"
+        v, unit = (materialised_flops if mat else expanded_flops)(spec, T) * frac / 1e12 / dt, "TFLOP/s"
     return {"value": v, "unit": unit, "cores": cores, "kind": "oracle",
             "sample": f"fp64 dense definition on the first {frac:.3f} of the output rows of one "
                       f"{spec.name} layer, T={T}, {reps} repetitions of {dt:.2f} s"}
@@ -421,8 +431,9 @@ def run_reference(args):
         metric, unit = "decode_algorithmic_GBps", "GB/s"
         per = algorithmic_bytes(spec, T) * fr / 1e9
     else:
-        metric, unit = "prefill_expanded_TFLOPs", "TFLOP/s"
-        per = expanded_flops(spec, T) * fr / 1e12
+        mat = rated_materialised(spec, T, args.kernel)    # same work unit as the arm it is compared with
+        metric, unit = ("prefill_executed_TFLOPs" if mat else "prefill_expanded_TFLOPs"), "TFLOP/s"
+        per = (materialised_flops if mat else expanded_flops)(spec, T) * fr / 1e12
     value = per * args.steps / total
     sample = (f"fp64 dense definition on the first {fr:.3f} of the output rows of one {spec.name} "
               f"layer per step, T={T}")

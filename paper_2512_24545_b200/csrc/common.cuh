@@ -150,5 +150,6 @@ struct mdbf_handle_s {
     uint32_t magic;
     int32_t kernel;
     int32_t last_launches;
+    int32_t last_kernel;
     mdbf::Layer L;
 };

@@ -343,6 +343,9 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         // cluster when few tokens would leave SMs idle); the others remain selectable
         if (!tc_ok) kernel = MDBF_KERNEL_ALU;
         else if (T == 1 && tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
+        // many tokens: rebuilding W_hat tiles and running one GEMM of width T beats the l sign GEMMs of the
+        // expanded order (measured crossover: 64 tokens, 128 for the rank-1 envelope)
+        else if (T >= (L.d.l == 1 ? 128 : 64) && mat_path_supports(L, x, T)) kernel = MDBF_KERNEL_MAT;
         else if (L.xsB) kernel = MDBF_KERNEL_PREFILL;
         else if (tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
         else kernel = MDBF_KERNEL_DECODE;
@@ -367,7 +370,7 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
     else if (kernel == MDBF_KERNEL_TMEM) rc = launch_forward_tmem(L, x, y, T, st, &launches);
     else if (kernel == MDBF_KERNEL_MAT) rc = launch_forward_mat(L, x, y, T, st, &launches);
     else rc = launch_forward_prefill(L, x, y, T, st, &launches);
-    if (rc == MDBF_OK) h->last_launches = launches;
+    if (rc == MDBF_OK) { h->last_launches = launches; h->last_kernel = kernel; }
     return rc;
 }
 
@@ -443,6 +446,7 @@ mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t 
             Ls[i]->last_ksplit = 0;
             outs[i] = ys[i0 + i];
             layers[i0 + i]->last_launches = i == 0 ? 2 : 0;
+            layers[i0 + i]->last_kernel = MDBF_KERNEL_TMEM;
         }
         mdbf_status_t rc = launch_forward_tmem_t1_multi(Ls, m, x, outs, st);
         if (rc) return rc;
@@ -514,6 +518,14 @@ mdbf_status_t mdbf_last_launch_count(mdbf_handle_t h, int32_t *count) {
     if (rc) return rc;
     if (!count) { set_error("mdbf_last_launch_count: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
     *count = h->last_launches;
+    return MDBF_OK;
+}
+
+mdbf_status_t mdbf_last_kernel(mdbf_handle_t h, int32_t *kernel) {
+    mdbf_status_t rc = check_handle(h, "mdbf_last_kernel");
+    if (rc) return rc;
+    if (!kernel) { set_error("mdbf_last_kernel: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    *kernel = h->last_kernel;
     return MDBF_OK;
 }
 

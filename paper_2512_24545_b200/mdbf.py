@@ -31,6 +31,7 @@ EXPORTS = (
     "mdbf_linear_forward_static", "mdbf_linear_forward_sum", "mdbf_linear_forward_siblings",
     "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_poll_status", "mdbf_selftest_wait_timeout",
     "mdbf_last_launch_count",
+    "mdbf_last_kernel",
     "mdbf_destroy", "mdbf_last_error", "mdbf_version",
 )
 
@@ -78,6 +79,7 @@ def lib() -> ctypes.CDLL:
     L.mdbf_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
     L.mdbf_selftest_wait_timeout.argtypes = [vp, vp]
     L.mdbf_last_launch_count.argtypes = [vp, ctypes.POINTER(i32)]
+    L.mdbf_last_kernel.argtypes = [vp, ctypes.POINTER(i32)]
     L.mdbf_destroy.argtypes = [vp]
     for name in EXPORTS:
         getattr(L, name).restype = i32
@@ -208,6 +210,13 @@ def mdbf_selftest_wait_timeout(h: int, stream: int = 0) -> None:
 def mdbf_last_launch_count(h: int) -> int:
     v = ctypes.c_int32()
     _check(lib().mdbf_last_launch_count(h, ctypes.byref(v)))
+    return v.value
+
+
+def mdbf_last_kernel(h: int) -> int:
+    """The KERNEL_* constant of the kernel the last forward on this handle ran (0 before the first)."""
+    v = ctypes.c_int32()
+    _check(lib().mdbf_last_kernel(h, ctypes.byref(v)))
     return v.value
 
 

@@ -85,7 +85,7 @@ def test_host_packer_rejects_bad_values_and_args():
 
 def test_handle_calls_reject_null_and_garbage():
     for fn, args in [(M.mdbf_destroy, ()), (M.mdbf_get_desc, ()), (M.mdbf_set_kernel, (0,)),
-                     (M.mdbf_poll_status, ()), (M.mdbf_last_launch_count, ())]:
+                     (M.mdbf_poll_status, ()), (M.mdbf_last_launch_count, ()), (M.mdbf_last_kernel, ())]:
         with pytest.raises(M.MdbfError) as e:
             fn(0, *args)
         assert e.value.status == M.ERR_INVALID_ARG
