@@ -75,10 +75,10 @@ def expanded_flops(spec, T):
 
 def rated_materialised(spec, T, forced="auto"):
     """Whether a tensor-bound workload is rated in FLOPs of the materialised order: mirrors the library's
-    dispatch (T >= 64, or 128 for the rank-1 envelope, runs the materialised-order kernel)."""
+    dispatch (T >= 32, or any T >= 2 for the rank-1 envelope, runs the materialised-order kernel)."""
     if forced != "auto":
         return forced == "mat"
-    return T >= (128 if spec.l == 1 else 64)
+    return T >= 32 or (spec.l == 1 and T >= 2)
 
 
 def materialised_flops(spec, T):

@@ -32,7 +32,11 @@
 // Every mbarrier wait is bounded; when one expires the kernel records MDBF_ERR_TIMEOUT in the
 // layer's status word, all roles fall through to the common exit, TMEM is released and the kernel
 // returns.  No TMA multicast is used.
+#include <cooperative_groups.h>
+
 #include "tmem_ptx.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace mdbf {
 
@@ -67,6 +71,8 @@ struct MatArgs {
     __nv_bfloat16 *y;        // stage A: [T][rows]
     float *y32;              // stage A, fp32 output modes (y_mode 1: store, 2: add)
     int y_mode;
+    int ppc;                 // split launches: pairs of K blocks per cluster rank (blockIdx.z)
+    int tpr;                 // split launches: tokens each rank reduces and stores, ceil(bn / ranks)
     int tma_out;             // 1: bf16 output staged in shared memory and written by TMA (16-byte aligned base and pitch)
     int32_t *status;
 };
@@ -135,7 +141,7 @@ __device__ __forceinline__ bool mt_wait3(uint32_t bar_a, uint32_t par_a, uint32_
     return true;
 }
 
-template <bool STAGE_A>
+template <bool STAGE_A, bool SPLIT>
 __global__ void __launch_bounds__(MT_THREADS, 1)
 mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out) {
     using namespace tm;
@@ -167,7 +173,13 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
     const int rb = blockIdx.x;
     const int row0 = rb * MT_BM;
     const int tau0 = blockIdx.y * a.bn;
-    const int nkb = (a.cols + MT_BK - 1) / MT_BK;
+    // a split launch shares the reduction among the ranks of a cluster (blockIdx.z): rank r takes the pairs
+    // [r * ppc, (r + 1) * ppc) of K blocks; all loops below count blocks and pairs from this rank's first one
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned crank = SPLIT ? cluster.block_rank() : 0u;
+    const int nkb_total = (a.cols + MT_BK - 1) / MT_BK;
+    const int kb0 = SPLIT ? (int)crank * 2 * a.ppc : 0;
+    const int nkb = SPLIT ? max(0, min(2 * a.ppc, nkb_total - kb0)) : nkb_total;
     const int npr = (nkb + 1) / 2;                                  // pairs of K blocks; the last one may hold one block
 
     if (tid == 0) {
@@ -199,6 +211,9 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
     const uint32_t tmem_e = tmem_base_slot + MT_BN;           // envelope values of a pair of K blocks: 128 columns
     const uint32_t tmem_a = tmem_e + 2 * MT_BK;               // W_hat tiles: MT_NA pairs x (2 blocks x 32 columns of bf16 pairs)
     pdl_launch_dependents();
+    // remote shared memory may only be written once its CTA runs: every thread arrives here and waits, much
+    // later, just before the first remote store
+    if (SPLIT) cluster.barrier_arrive();
 
     if (warp < MT_W_TMA) {
         // ============================ W_hat tile builders ============================
@@ -206,8 +221,8 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
         const int grp = (warp >> 2) & 1, half = warp >> 3;
         const int arow = tid & 127;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t *wp = reinterpret_cast<const uint32_t *>(a.wk + (size_t)row0 + arow) + half;   // + kb * rows_pad * 2
         const size_t wstride = (size_t)a.rows_pad * 2;
+        const uint32_t *wp = reinterpret_cast<const uint32_t *>(a.wk + (size_t)row0 + arow) + half + (size_t)kb0 * wstride;   // + kb * wstride
         uint32_t w_next = grp < nkb ? __ldg(wp + (size_t)grp * wstride) : 0u;
         uint32_t w_next2 = grp + 2 < nkb ? __ldg(wp + (size_t)(grp + 2) * wstride) : 0u;
         bool alive = true;
@@ -255,7 +270,55 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
         // wait that expired in any thread has raised the abort flag before that thread arrived
         asm volatile("bar.sync %0, 128;\n" ::"r"(1 + (warp >> 2)) : "memory");
         alive = !*abort_flag;
-        if (alive && a.tma_out) {
+        if (SPLIT) {
+            // Partial sums of the ranks meet in shared memory: rank r owns the tokens [r * tpr, (r + 1) * tpr) of the
+            // tile, every rank pushes its partial values of those tokens into rank r's region [rank][token][128 rows]
+            // (a region of its own: the owner's pipeline may still be running), and after one cluster barrier each
+            // rank adds its tokens up in rank order (deterministic) and stores them.
+            float *part = reinterpret_cast<float *>(smem_gen + (v_smem - smem_base) + (size_t)nv * img_bytes);
+            cluster.barrier_wait();
+            if (alive) {
+#pragma unroll 1
+                for (int ld = warp >> 2; ld * 32 < a.bn; ld += MT_XWARPS / 4) {
+                    const int col0 = ld * 32;
+                    uint32_t v[32];
+                    if (nkb > 0) {
+                        tmem_ld32(tmem_d + lane_base + (uint32_t)col0, v);
+                        tmem_ld_wait();
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = 0u;          // an empty slice contributes nothing
+                    }
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int t = col0 + j;
+                        if (t < a.bn) {
+                            const int owner = t / a.tpr, slot = t - owner * a.tpr;
+                            float *dst = cluster.map_shared_rank(part, owner);
+                            dst[((int)crank * a.tpr + slot) * MT_BM + arow] = __uint_as_float(v[j]);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            cluster.sync();
+            if (alive && !*abort_flag) {
+                const int nranks = (int)cluster.num_blocks();
+                for (int slot = warp >> 2; slot < a.tpr; slot += MT_XWARPS / 4) {
+                    const int tau = tau0 + (int)crank * a.tpr + slot;
+                    if ((int)crank * a.tpr + slot >= a.bn || tau >= a.T || egrow >= a.rows) continue;
+                    float acc = 0.f;
+                    for (int rk = 0; rk < nranks; ++rk) acc += part[(rk * a.tpr + slot) * MT_BM + arow];
+                    if (STAGE_A) {
+                        if (a.y_mode == 0) a.y[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(acc);
+                        else if (a.y_mode == 1) a.y32[(size_t)tau * a.rows + egrow] = acc;
+                        else a.y32[(size_t)tau * a.rows + egrow] += acc;
+                    } else {
+                        a.zb[(size_t)tau * a.zstride + egrow] = __float2bfloat16_rn(acc);
+                    }
+                }
+            }
+        } else if (alive && a.tma_out) {
             // The four warps of group g = warp / 4 cover all 128 rows; they take tokens [64g, 64g + 64): accumulator ->
             // bf16 [token][128 rows] in the (now idle) activation ring -> one TMA store per group, which clips
             // rows and tokens outside the output.
@@ -314,7 +377,7 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
                 for (int h = 0; h < 2 && 2 * p + h < nkb; ++h) {
                     const int s = 2 * bp + h;
                     mbar_arrive_expect_tx(bfull_bar + 8 * s, b_bytes);
-                    tma_load_2d(smem_base + (uint32_t)s * b_bytes, &tmap_in, (2 * p + h) * MT_BK, tau0, bfull_bar + 8 * s);
+                    tma_load_2d(smem_base + (uint32_t)s * b_bytes, &tmap_in, (kb0 + 2 * p + h) * MT_BK, tau0, bfull_bar + 8 * s);
                 }
                 if (++bp == nbp) { bp = 0; ph ^= 1u; }
             }
@@ -333,7 +396,7 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
                 alive = mbar_wait(vempty_bar + 8 * vb, vph ^ 1u, abort_flag, a.status);
                 if (!alive) break;
                 mbar_arrive_expect_tx(vfull_bar + 8 * vb, img_bytes);
-                bulk_load(v_smem + (uint32_t)vb * img_bytes, a.vimg + (size_t)p * (img_bytes / 2), img_bytes, vfull_bar + 8 * vb);
+                bulk_load(v_smem + (uint32_t)vb * img_bytes, a.vimg + (size_t)(kb0 / 2 + p) * (img_bytes / 2), img_bytes, vfull_bar + 8 * vb);
                 if (++vb == nv) { vb = 0; vph ^= 1u; }
             }
             if (!alive) drain_delay();
@@ -395,6 +458,11 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
         __syncwarp();
     }
 
+    if (SPLIT && warp >= MT_W_TMA) {                    // the builder warps run these barriers inside their epilogue
+        cluster.barrier_wait();
+        cluster.sync();
+    }
+
     tc_fence_before();
     __syncthreads();
     if (warp == MT_W_MMA) tmem_dealloc(tmem_d, MT_TMEM_COLS);
@@ -419,14 +487,18 @@ bool mat_path_supports(const Layer &L, const void *x, int T) {
     return L.uiA && L.zb && T >= 2 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && L.d.d_in % 8 == 0;
 }
 
-// shared memory: ring of activation tiles, U image, ring of V images, alignment slack
-static int mt_ring(int kc, int nv, int bn) {
-    const size_t avail = 227 * 1024 - 1024 - 1024 - (size_t)(1 + nv) * kc * 2048;    // 1 KB static, 1 KB slack
+// shared memory: ring of activation tiles, U image, ring of V images, (split launches) partial sums, slack
+static int mt_ring(int kc, int nv, int bn, size_t part_bytes) {
+    const size_t avail = 227 * 1024 - 1024 - 1024 - (size_t)(1 + nv) * kc * 2048 - part_bytes;    // 1 KB static, 1 KB slack
     const int n = (int)(avail / ((size_t)bn * MT_BK * 2)) / 2 * 2;
     return n < MT_MAX_NS ? n : MT_MAX_NS;
 }
-static size_t mt_smem_bytes(int kc, int nv, int bn) {
-    return (size_t)mt_ring(kc, nv, bn) * bn * MT_BK * 2 + (size_t)(1 + nv) * kc * 2048 + 1024;
+static size_t mt_smem_bytes(int kc, int nv, int bn, size_t part_bytes) {
+    return (size_t)mt_ring(kc, nv, bn, part_bytes) * bn * MT_BK * 2 + (size_t)(1 + nv) * kc * 2048 + part_bytes + 1024;
+}
+static int mt_env_int(const char *name, int dflt) {
+    const char *v = getenv(name);
+    return v && *v ? atoi(v) : dflt;
 }
 
 // Tensor map of a bf16 output [T][rows] with rows `pitch` elements apart: box of 128 rows x 64 tokens, no swizzle.
@@ -460,24 +532,54 @@ static mdbf_status_t make_out_tensor_map(CUtensorMap *out, const void *base, int
 }
 
 template <bool STAGE_A>
-static mdbf_status_t launch_mat(const MatArgs &a, const CUtensorMap &tm, const CUtensorMap &tmo, cudaStream_t st) {
+static mdbf_status_t launch_mat(const MatArgs &a0, const CUtensorMap &tm, const CUtensorMap &tmo, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        MDBF_CUDA(cudaFuncSetAttribute(mat_stage_kernel<STAGE_A>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)mt_smem_bytes(4, 3, MT_BN)));
+        MDBF_CUDA(cudaFuncSetAttribute(mat_stage_kernel<STAGE_A, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)mt_smem_bytes(4, 3, MT_BN, 0)));
+        MDBF_CUDA(cudaFuncSetAttribute(mat_stage_kernel<STAGE_A, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)mt_smem_bytes(4, 3, MT_BN, 0)));
         attr_set = true;
     }
+    MatArgs a = a0;
+    const int rb = ceil_div(a.rows, MT_BM), npr = ceil_div(ceil_div(a.cols, MT_BK), 2);
+    // One token tile of at most 64 tokens leaves most SMs without work and every CTA with a long serial
+    // chain of K blocks: split the reduction over a cluster of up to 8 CTAs.
+    // Cost model: waves x (pairs per CTA + fixed part, in pairs).
+    int ks = 1;
+    if (a.T <= 64) {
+        const int fixed = mt_env_int("MDBF_MAT_FIXED_COST", 8), max_ks = mt_env_int("MDBF_MAT_MAX_KS", 8);
+        long best = -1;
+        for (int c = 1; c <= 8 && c <= max_ks; ++c) {
+            const int per = ceil_div(npr, c);
+            if (c > 1 && per * (c - 1) >= npr) continue;               // an empty rank
+            const long cost = (long)ceil_div(rb * c, 148) * (per + fixed);
+            if (best < 0 || cost < best) { best = cost; ks = c; }
+        }
+    }
+    size_t part_bytes = 0;
+    if (ks > 1) {
+        a.ppc = ceil_div(npr, ks);
+        a.tpr = ceil_div(a.bn, ks);
+        part_bytes = (size_t)ks * a.tpr * MT_BM * sizeof(float);
+    }
+    a.ns = mt_ring(a.kc, a.nv, a.bn, part_bytes);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(ceil_div(a.rows, MT_BM), ceil_div(a.T, a.bn), 1);
+    cfg.gridDim = dim3(rb, ceil_div(a.T, a.bn), ks);
     cfg.blockDim = dim3(MT_THREADS);
-    cfg.dynamicSmemBytes = mt_smem_bytes(a.kc, a.nv, a.bn);
+    cfg.dynamicSmemBytes = mt_smem_bytes(a.kc, a.nv, a.bn, part_bytes);
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = ks;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    MDBF_CUDA(cudaLaunchKernelEx(&cfg, mat_stage_kernel<STAGE_A>, a, tm, tmo));
+    cfg.numAttrs = ks > 1 ? 2 : 1;
+    if (ks > 1) MDBF_CUDA(cudaLaunchKernelEx(&cfg, mat_stage_kernel<STAGE_A, true>, a, tm, tmo));
+    else MDBF_CUDA(cudaLaunchKernelEx(&cfg, mat_stage_kernel<STAGE_A, false>, a, tm, tmo));
     return MDBF_OK;
 }
 
@@ -508,7 +610,7 @@ mdbf_status_t launch_forward_mat(Layer &L, const void *x, void *y, int T, cudaSt
     b.wk = L.wkB; b.rows_pad = L.rpB; b.rows = d.k; b.cols = d.d_in;
     b.uimg = L.uiB; b.vimg = L.viB; b.kc = L.kcm; b.env_fmt = d.env_dtype == MDBF_BF16 ? 1u : 0u;
     b.nv = L.kcm == 2 ? 4 : 3;
-    b.T = T; b.bn = bn; b.ns = mt_ring(b.kc, b.nv, bn); b.zb = L.zb; b.zstride = L.padA; b.status = L.status;
+    b.T = T; b.bn = bn;  b.zb = L.zb; b.zstride = L.padA; b.status = L.status;
     b.tma_out = 1;
     rc = launch_mat<false>(b, tmx, tmzo, st);
     if (rc) return rc;
@@ -516,7 +618,7 @@ mdbf_status_t launch_forward_mat(Layer &L, const void *x, void *y, int T, cudaSt
     MatArgs a = {};
     a.wk = L.wkA; a.rows_pad = L.rpA; a.rows = d.d_out; a.cols = d.k;
     a.uimg = L.uiA; a.vimg = L.viA; a.kc = L.kcm; a.env_fmt = b.env_fmt; a.nv = b.nv;
-    a.T = T; a.bn = bn; a.ns = b.ns;
+    a.T = T; a.bn = bn; 
     a.y = reinterpret_cast<__nv_bfloat16 *>(y); a.y32 = reinterpret_cast<float *>(y); a.y_mode = L.out_mode; a.status = L.status;
     a.tma_out = y_tma ? 1 : 0;
     rc = launch_mat<true>(a, tmz, tmyo, st);

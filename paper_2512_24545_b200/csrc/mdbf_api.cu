@@ -343,9 +343,9 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         // cluster when few tokens would leave SMs idle); the others remain selectable
         if (!tc_ok) kernel = MDBF_KERNEL_ALU;
         else if (T == 1 && tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
-        // many tokens: rebuilding W_hat tiles and running one GEMM of width T beats the l sign GEMMs of the
-        // expanded order (measured crossover: 64 tokens, 128 for the rank-1 envelope)
-        else if (T >= (L.d.l == 1 ? 128 : 64) && mat_path_supports(L, x, T)) kernel = MDBF_KERNEL_MAT;
+        // rebuilding W_hat tiles and running one GEMM of width T beats the l sign GEMMs of the expanded order
+        // from 32 tokens on, and at every T >= 2 for the rank-1 envelope (measured crossovers)
+        else if ((T >= 32 || L.d.l == 1) && mat_path_supports(L, x, T)) kernel = MDBF_KERNEL_MAT;
         else if (L.xsB) kernel = MDBF_KERNEL_PREFILL;
         else if (tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
         else kernel = MDBF_KERNEL_DECODE;

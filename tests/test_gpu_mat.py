@@ -53,6 +53,19 @@ def test_mat_kernel_ragged_shapes(shape):
         assert rel_err(y, g.oracle_forward(x)) <= tol
 
 
+@pytest.mark.parametrize("shape", [(128, 2048, 1024, 8, 8), (256, 1100 * 8, 520, 16, 40), (200, 4096, 136, 3, 2)])
+def test_mat_kernel_split_reduction(shape):
+    """Few tokens and few row blocks: the reduction is split over a cluster and summed through shared memory."""
+    d_out, d_in, k, l, T = shape
+    spec = spec_of(d_out, d_in, k, l)
+    x = inputs.make_activations(spec, T)
+    with GpuLayer(spec, T) as g:
+        y = g.forward(x, kernel=M.KERNEL_MAT)
+        assert M.mdbf_poll_status(g.h) == 0
+        assert rel_err(y, g.oracle_forward(x)) <= TOL["bf16"]
+        np.testing.assert_array_equal(y, g.forward(x, kernel=M.KERNEL_MAT))     # deterministic summation order
+
+
 @pytest.mark.parametrize("env_dtype", ["f16", "bf16"])
 def test_mat_kernel_envelope_types_and_other_kernels(env_dtype):
     spec = spec_of(256, 512, 256, 16, env_dtype=env_dtype)
