@@ -37,7 +37,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that workload).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    ("decode_qproj", "tmem_t1_kernel"): 1083648,                   # k = 1664 layer, either stage
+    ("decode_qproj", "tmem_t1_kernel"): 1082112,                   # k = 1664 layer, stage B (stage A: 1080320)
+    ("prefill_4096_l16_bpw10", "mat_stage_kernel"): 17858048,      # stage B: x read once + signs + images; nothing reaches DRAM on the way out
     ("prefill_4096_l16_bpw10", "gemm_stage_kernel"): 370142976,    # stage B: 269.4 MB read + 100.7 MB written
 }
 
