@@ -48,7 +48,7 @@ def dominant_kernel(spec, T, forced="auto"):
     if T == 1:
         return "tmem_t1_kernel"
     if forced == "mat":
-        return "mat_stage_kernel"
+        return "mat_stage_kernel" if T > 64 else "mat_small_kernel"
     return "gemm_stage_kernel"
 
 
@@ -76,10 +76,10 @@ def expanded_flops(spec, T):
 
 def rated_materialised(spec, T, forced="auto"):
     """Whether a tensor-bound workload is rated in FLOPs of the materialised order: mirrors the library's
-    dispatch (T >= 32, or any T >= 2 for the rank-1 envelope, runs the materialised-order kernel)."""
+    dispatch (every T >= 2 runs the materialised-order kernel; the bench shapes all qualify for it)."""
     if forced != "auto":
         return forced == "mat"
-    return T >= 32 or (spec.l == 1 and T >= 2)
+    return T >= 2
 
 
 def materialised_flops(spec, T):

@@ -60,7 +60,7 @@ typedef enum { MDBF_F32 = 0, MDBF_F16 = 1, MDBF_BF16 = 2 } mdbf_dtype_t;
 
 /* Kernel selector for mdbf_set_kernel. */
 typedef enum {
-    MDBF_KERNEL_AUTO = 0,   /* T = 1: TMEM; T >= 32 (l = 1: T >= 2): MAT; other T >= 2: PREFILL; fp32 / l > 32: ALU */
+    MDBF_KERNEL_AUTO = 0,   /* T = 1: TMEM; T >= 2: MAT (PREFILL where MAT cannot run); fp32 / l > 32: ALU */
     MDBF_KERNEL_ALU = 1,    /* fp32 CUDA-core path, sign applied by XOR of the IEEE sign bit      */
     MDBF_KERNEL_DECODE = 2, /* T <= 4: register bit->bf16 expansion + warp-level MMA              */
     MDBF_KERNEL_PREFILL = 3, /* T >= 2 (max_T >= 2): tcgen05 GEMM, TMEM accumulator, TMA operand   */

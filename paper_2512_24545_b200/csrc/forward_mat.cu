@@ -141,7 +141,7 @@ __device__ __forceinline__ bool mt_wait3(uint32_t bar_a, uint32_t par_a, uint32_
     return true;
 }
 
-template <bool STAGE_A, bool SPLIT>
+template <bool STAGE_A>
 __global__ void __launch_bounds__(MT_THREADS, 1)
 mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out) {
     using namespace tm;
@@ -173,13 +173,7 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
     const int rb = blockIdx.x;
     const int row0 = rb * MT_BM;
     const int tau0 = blockIdx.y * a.bn;
-    // a split launch shares the reduction among the ranks of a cluster (blockIdx.z): rank r takes the pairs
-    // [r * ppc, (r + 1) * ppc) of K blocks; all loops below count blocks and pairs from this rank's first one
-    cg::cluster_group cluster = cg::this_cluster();
-    const unsigned crank = SPLIT ? cluster.block_rank() : 0u;
-    const int nkb_total = (a.cols + MT_BK - 1) / MT_BK;
-    const int kb0 = SPLIT ? (int)crank * 2 * a.ppc : 0;
-    const int nkb = SPLIT ? max(0, min(2 * a.ppc, nkb_total - kb0)) : nkb_total;
+    const int nkb = (a.cols + MT_BK - 1) / MT_BK;
     const int npr = (nkb + 1) / 2;                                  // pairs of K blocks; the last one may hold one block
 
     if (tid == 0) {
@@ -211,9 +205,6 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
     const uint32_t tmem_e = tmem_base_slot + MT_BN;           // envelope values of a pair of K blocks: 128 columns
     const uint32_t tmem_a = tmem_e + 2 * MT_BK;               // W_hat tiles: MT_NA pairs x (2 blocks x 32 columns of bf16 pairs)
     pdl_launch_dependents();
-    // remote shared memory may only be written once its CTA runs: every thread arrives here and waits, much
-    // later, just before the first remote store
-    if (SPLIT) cluster.barrier_arrive();
 
     if (warp < MT_W_TMA) {
         // ============================ W_hat tile builders ============================
@@ -222,7 +213,7 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
         const int arow = tid & 127;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const size_t wstride = (size_t)a.rows_pad * 2;
-        const uint32_t *wp = reinterpret_cast<const uint32_t *>(a.wk + (size_t)row0 + arow) + half + (size_t)kb0 * wstride;   // + kb * wstride
+        const uint32_t *wp = reinterpret_cast<const uint32_t *>(a.wk + (size_t)row0 + arow) + half;   // + kb * wstride
         uint32_t w_next = grp < nkb ? __ldg(wp + (size_t)grp * wstride) : 0u;
         uint32_t w_next2 = grp + 2 < nkb ? __ldg(wp + (size_t)(grp + 2) * wstride) : 0u;
         bool alive = true;
@@ -270,55 +261,7 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
         // wait that expired in any thread has raised the abort flag before that thread arrived
         asm volatile("bar.sync %0, 128;\n" ::"r"(1 + (warp >> 2)) : "memory");
         alive = !*abort_flag;
-        if (SPLIT) {
-            // Partial sums of the ranks meet in shared memory: rank r owns the tokens [r * tpr, (r + 1) * tpr) of the
-            // tile, every rank pushes its partial values of those tokens into rank r's region [rank][token][128 rows]
-            // (a region of its own: the owner's pipeline may still be running), and after one cluster barrier each
-            // rank adds its tokens up in rank order (deterministic) and stores them.
-            float *part = reinterpret_cast<float *>(smem_gen + (v_smem - smem_base) + (size_t)nv * img_bytes);
-            cluster.barrier_wait();
-            if (alive) {
-#pragma unroll 1
-                for (int ld = warp >> 2; ld * 32 < a.bn; ld += MT_XWARPS / 4) {
-                    const int col0 = ld * 32;
-                    uint32_t v[32];
-                    if (nkb > 0) {
-                        tmem_ld32(tmem_d + lane_base + (uint32_t)col0, v);
-                        tmem_ld_wait();
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = 0u;          // an empty slice contributes nothing
-                    }
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int t = col0 + j;
-                        if (t < a.bn) {
-                            const int owner = t / a.tpr, slot = t - owner * a.tpr;
-                            float *dst = cluster.map_shared_rank(part, owner);
-                            dst[((int)crank * a.tpr + slot) * MT_BM + arow] = __uint_as_float(v[j]);
-                        }
-                    }
-                }
-            }
-            tc_fence_before();
-            cluster.sync();
-            if (alive && !*abort_flag) {
-                const int nranks = (int)cluster.num_blocks();
-                for (int slot = warp >> 2; slot < a.tpr; slot += MT_XWARPS / 4) {
-                    const int tau = tau0 + (int)crank * a.tpr + slot;
-                    if ((int)crank * a.tpr + slot >= a.bn || tau >= a.T || egrow >= a.rows) continue;
-                    float acc = 0.f;
-                    for (int rk = 0; rk < nranks; ++rk) acc += part[(rk * a.tpr + slot) * MT_BM + arow];
-                    if (STAGE_A) {
-                        if (a.y_mode == 0) a.y[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(acc);
-                        else if (a.y_mode == 1) a.y32[(size_t)tau * a.rows + egrow] = acc;
-                        else a.y32[(size_t)tau * a.rows + egrow] += acc;
-                    } else {
-                        a.zb[(size_t)tau * a.zstride + egrow] = __float2bfloat16_rn(acc);
-                    }
-                }
-            }
-        } else if (alive && a.tma_out) {
+        if (alive && a.tma_out) {
             // The four warps of group g = warp / 4 cover all 128 rows; they take tokens [64g, 64g + 64): accumulator ->
             // bf16 [token][128 rows] in the (now idle) activation ring -> one TMA store per group, which clips
             // rows and tokens outside the output.
@@ -377,7 +320,7 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
                 for (int h = 0; h < 2 && 2 * p + h < nkb; ++h) {
                     const int s = 2 * bp + h;
                     mbar_arrive_expect_tx(bfull_bar + 8 * s, b_bytes);
-                    tma_load_2d(smem_base + (uint32_t)s * b_bytes, &tmap_in, (kb0 + 2 * p + h) * MT_BK, tau0, bfull_bar + 8 * s);
+                    tma_load_2d(smem_base + (uint32_t)s * b_bytes, &tmap_in, (2 * p + h) * MT_BK, tau0, bfull_bar + 8 * s);
                 }
                 if (++bp == nbp) { bp = 0; ph ^= 1u; }
             }
@@ -396,7 +339,7 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
                 alive = mbar_wait(vempty_bar + 8 * vb, vph ^ 1u, abort_flag, a.status);
                 if (!alive) break;
                 mbar_arrive_expect_tx(vfull_bar + 8 * vb, img_bytes);
-                bulk_load(v_smem + (uint32_t)vb * img_bytes, a.vimg + (size_t)(kb0 / 2 + p) * (img_bytes / 2), img_bytes, vfull_bar + 8 * vb);
+                bulk_load(v_smem + (uint32_t)vb * img_bytes, a.vimg + (size_t)p * (img_bytes / 2), img_bytes, vfull_bar + 8 * vb);
                 if (++vb == nv) { vb = 0; vph ^= 1u; }
             }
             if (!alive) drain_delay();
@@ -458,14 +401,309 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
         __syncwarp();
     }
 
-    if (SPLIT && warp >= MT_W_TMA) {                    // the builder warps run these barriers inside their epilogue
+    tc_fence_before();
+    __syncthreads();
+    if (warp == MT_W_MMA) tmem_dealloc(tmem_d, MT_TMEM_COLS);
+}
+
+// ------------------------------------------------------------------ tiles of at most 64 tokens
+// With few tokens the tensor pipe is idle and the per-pair chains of the single-thread roles and of the
+// builders set the pace, so this variant runs TWO pipelines side by side: pairs of K blocks alternate
+// between two halves g = pair & 1, each with its own envelope buffer (128 TMEM columns), W_hat tile slot,
+// group of 8 builder warps (a warp: one block of the pair, 32 rows, all 64 columns), main-MMA issuer and
+// accumulator; the epilogue adds the two accumulators.  Loaders and the mini-MMA issuer are shared.
+// TMEM: D0 0..63, D1 64..127, W_hat slots 128 + 64 g, envelope buffers 256 + 128 g.
+constexpr int MS_W_TMA = MT_XWARPS;
+constexpr int MS_W_MMA0 = MT_XWARPS + 1;
+constexpr int MS_W_ENV = MT_XWARPS + 2;
+constexpr int MS_W_MINI = MT_XWARPS + 3;
+constexpr int MS_W_MMA1 = MT_XWARPS + 4;
+constexpr int MS_THREADS = (MS_W_MMA1 + 1) * 32;
+constexpr int MS_BN = 64;
+
+template <bool STAGE_A, bool SPLIT>
+__global__ void __launch_bounds__(MS_THREADS, 1)
+mat_small_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in) {
+    using namespace tm;
+    extern __shared__ unsigned char mt_smem_raw[];
+    __shared__ __align__(8) uint64_t bars[MT_MAX_NS + MT_MAX_NS / 2 + 8 + 2 * MT_MAX_NV + 2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag_s;
+    volatile int *abort_flag = &abort_flag_s;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t smem_base = (smem_u32(mt_smem_raw) + 1023u) & ~1023u;
+    unsigned char *smem_gen = mt_smem_raw + (smem_base - smem_u32(mt_smem_raw));
+    const int nbp = a.ns / 2, nv = a.nv;
+    const uint32_t b_bytes = (uint32_t)a.bn * MT_BK * 2;
+    const uint32_t u_smem = smem_base + (uint32_t)a.ns * b_bytes;
+    const uint32_t img_bytes = (uint32_t)a.kc * 2048u;
+    const uint32_t v_smem = u_smem + img_bytes;
+    const uint32_t bfull_bar = smem_u32(&bars[0]);                  // per activation tile
+    const uint32_t bempty_bar = bfull_bar + 8 * MT_MAX_NS;          // per pair of activation tiles
+    const uint32_t afull_bar = bempty_bar + 8 * (MT_MAX_NS / 2);    // [2] per half
+    const uint32_t aempty_bar = afull_bar + 16;
+    const uint32_t efull_bar = aempty_bar + 16;
+    const uint32_t eempty_bar = efull_bar + 16;
+    const uint32_t vfull_bar = eempty_bar + 16;
+    const uint32_t vempty_bar = vfull_bar + 8 * MT_MAX_NV;
+    const uint32_t accum_bar = vempty_bar + 8 * MT_MAX_NV;
+    const uint32_t u_bar = accum_bar + 8;
+
+    const int rb = blockIdx.x;
+    const int row0 = rb * MT_BM;
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned crank = SPLIT ? cluster.block_rank() : 0u;
+    const int nkb_total = (a.cols + MT_BK - 1) / MT_BK;
+    const int kb0 = SPLIT ? (int)crank * 2 * a.ppc : 0;
+    const int nkb = SPLIT ? max(0, min(2 * a.ppc, nkb_total - kb0)) : nkb_total;
+    const int npr = (nkb + 1) / 2;
+
+    if (tid == 0) {
+        for (int s = 0; s < MT_MAX_NS; ++s) mbar_init(bfull_bar + 8 * s, 1);
+        for (int s = 0; s < MT_MAX_NS / 2; ++s) mbar_init(bempty_bar + 8 * s, 1);
+        for (int g = 0; g < 2; ++g) {
+            mbar_init(afull_bar + 8 * g, MT_XWARPS / 2);            // one arrival per builder warp of the half
+            mbar_init(aempty_bar + 8 * g, 1);
+            mbar_init(efull_bar + 8 * g, 1);
+            mbar_init(eempty_bar + 8 * g, MT_XWARPS / 2);
+        }
+        for (int v = 0; v < MT_MAX_NV; ++v) {
+            mbar_init(vfull_bar + 8 * v, 1);
+            mbar_init(vempty_bar + 8 * v, 1);
+        }
+        mbar_init(accum_bar, 2);                                    // both main-MMA issuers
+        mbar_init(u_bar, 1);
+        abort_flag_s = 0;
+        fence_barrier_init();
+    }
+    if (warp == MS_W_MMA0) {
+        tmem_alloc(smem_u32(&tmem_base_slot), MT_TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = tmem_base_slot;                   // + 64 g
+    const uint32_t tmem_a = tmem_base_slot + 2 * MS_BN;       // + 64 g
+    const uint32_t tmem_e = tmem_base_slot + 256;             // + 128 g
+    pdl_launch_dependents();
+    if (SPLIT) cluster.barrier_arrive();                      // see mat_stage_kernel
+
+    if (warp < MS_W_TMA) {
+        // ============================ W_hat tile builders ============================
+        const int g = warp >> 3, blk = (warp >> 2) & 1;
+        const int arow = tid & 127;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint2 *wp = a.wk + (size_t)kb0 * a.rows_pad + (size_t)row0 + arow;     // + kb * rows_pad
+        const int kbf = 2 * g + blk;                                                   // this warp's first block
+        uint2 w_next = kbf < nkb ? __ldg(wp + (size_t)kbf * a.rows_pad) : make_uint2(0u, 0u);
+        uint2 w_next2 = kbf + 4 < nkb ? __ldg(wp + (size_t)(kbf + 4) * a.rows_pad) : make_uint2(0u, 0u);
+        bool alive = true;
+        for (int i = 0; 2 * i + g < npr && alive; ++i) {
+            const int kb = 2 * (2 * i + g) + blk;
+            const uint32_t ph = (uint32_t)i & 1u;
+            const uint2 w = w_next;
+            w_next = w_next2;
+            w_next2 = kb + 8 < nkb ? __ldg(wp + (size_t)(kb + 8) * a.rows_pad) : make_uint2(0u, 0u);
+            alive = mbar_wait(efull_bar + 8 * g, ph, abort_flag, a.status);
+            if (!alive) break;
+            tc_fence_after();
+            uint32_t o0[16], o1[16];
+            {
+                uint32_t v[32];
+                tmem_ld32(tmem_e + (uint32_t)(g * 128 + blk * 64) + lane_base, v);
+                tmem_ld_wait();
+                mt_expand_half(v, w.x, o0);
+                tmem_ld32(tmem_e + (uint32_t)(g * 128 + blk * 64 + 32) + lane_base, v);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(eempty_bar + 8 * g);
+                mt_expand_half(v, w.y, o1);
+            }
+            alive = mbar_wait(aempty_bar + 8 * g, ph ^ 1u, abort_flag, a.status);
+            if (!alive) break;
+            tc_fence_after();
+            const uint32_t a_col = tmem_a + (uint32_t)(g * 64 + blk * 32) + lane_base;
+            tmem_st8(a_col, *reinterpret_cast<const uint32_t (*)[8]>(&o0[0]));
+            tmem_st8(a_col + 8, *reinterpret_cast<const uint32_t (*)[8]>(&o0[8]));
+            tmem_st8(a_col + 16, *reinterpret_cast<const uint32_t (*)[8]>(&o1[0]));
+            tmem_st8(a_col + 24, *reinterpret_cast<const uint32_t (*)[8]>(&o1[8]));
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(afull_bar + 8 * g);
+        }
+
+        // ================================= epilogue ==================================
+        // the four warps of a lane quadrant take 16 tokens each; out = D0 + D1
+        const int egrow = row0 + arow;
+        const int chunk = warp >> 2;
+        if (alive) alive = mbar_wait(accum_bar, 0u, abort_flag, a.status);
+        tc_fence_after();
+        pdl_wait();                                   // the stores below must follow the previous kernel's reads
+        float acc[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+        if (alive && chunk * 16 < a.bn) {
+            uint32_t v[16];
+            if (npr > 0) {
+                tmem_ld16(tmem_d + lane_base + (uint32_t)(chunk * 16), v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) acc[j] = __uint_as_float(v[j]);
+            }
+            if (npr > 1) {
+                tmem_ld16(tmem_d + MS_BN + lane_base + (uint32_t)(chunk * 16), v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) acc[j] += __uint_as_float(v[j]);
+            }
+        }
+        auto emit = [&](int tau, float val) {
+            if (STAGE_A) {
+                if (a.y_mode == 0) a.y[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(val);
+                else if (a.y_mode == 1) a.y32[(size_t)tau * a.rows + egrow] = val;
+                else a.y32[(size_t)tau * a.rows + egrow] += val;
+            } else {
+                a.zb[(size_t)tau * a.zstride + egrow] = __float2bfloat16_rn(val);
+            }
+        };
+        if (SPLIT) {
+            // partial sums reduce-scattered by token through distributed shared memory (see mat_stage_kernel)
+            float *part = reinterpret_cast<float *>(smem_gen + (v_smem - smem_base) + (size_t)nv * img_bytes);
+            cluster.barrier_wait();
+            if (alive && chunk * 16 < a.bn) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int t = chunk * 16 + j;
+                    if (t < a.bn) {
+                        const int owner = t / a.tpr, slot = t - owner * a.tpr;
+                        float *dst = cluster.map_shared_rank(part, owner);
+                        dst[((int)crank * a.tpr + slot) * MT_BM + arow] = acc[j];
+                    }
+                }
+            }
+            tc_fence_before();
+            cluster.sync();
+            if (alive && !*abort_flag) {
+                const int nranks = (int)cluster.num_blocks();
+                for (int slot = chunk; slot < a.tpr; slot += 4) {
+                    const int t = (int)crank * a.tpr + slot;
+                    if (t >= a.bn || t >= a.T || egrow >= a.rows) continue;
+                    float sum = 0.f;
+                    for (int rk = 0; rk < nranks; ++rk) sum += part[(rk * a.tpr + slot) * MT_BM + arow];
+                    emit(t, sum);
+                }
+            }
+        } else if (alive && egrow < a.rows) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int t = chunk * 16 + j;
+                if (t < a.bn && t < a.T) emit(t, acc[j]);
+            }
+        }
+    } else if (warp == MS_W_TMA) {
+        // ============================ activation-tile loader ===========================
+        if (lane == 0) {
+            bool alive = true;
+            pdl_wait();
+            int bp = 0;
+            uint32_t ph = 0;
+            for (int p = 0; p < npr && alive; ++p) {
+                alive = mbar_wait(bempty_bar + 8 * bp, ph ^ 1u, abort_flag, a.status);
+                if (!alive) break;
+                for (int h = 0; h < 2 && 2 * p + h < nkb; ++h) {
+                    const int s = 2 * bp + h;
+                    mbar_arrive_expect_tx(bfull_bar + 8 * s, b_bytes);
+                    tma_load_2d(smem_base + (uint32_t)s * b_bytes, &tmap_in, (kb0 + 2 * p + h) * MT_BK, 0, bfull_bar + 8 * s);
+                }
+                if (++bp == nbp) { bp = 0; ph ^= 1u; }
+            }
+            if (!alive) drain_delay();
+        }
+        __syncwarp();
+    } else if (warp == MS_W_ENV) {
+        // ============================= envelope-image loader ===========================
+        if (lane == 0) {
+            bool alive = true;
+            mbar_arrive_expect_tx(u_bar, img_bytes);
+            bulk_load(u_smem, a.uimg + (size_t)rb * (img_bytes / 2), img_bytes, u_bar);
+            int vb = 0;
+            uint32_t vph = 0;
+            for (int p = 0; p < npr && alive; ++p) {
+                alive = mbar_wait(vempty_bar + 8 * vb, vph ^ 1u, abort_flag, a.status);
+                if (!alive) break;
+                mbar_arrive_expect_tx(vfull_bar + 8 * vb, img_bytes);
+                bulk_load(v_smem + (uint32_t)vb * img_bytes, a.vimg + (size_t)(kb0 / 2 + p) * (img_bytes / 2), img_bytes, vfull_bar + 8 * vb);
+                if (++vb == nv) { vb = 0; vph ^= 1u; }
+            }
+            if (!alive) drain_delay();
+        }
+        __syncwarp();
+    } else if (warp == MS_W_MINI) {
+        // ======================= envelope mini-MMA issuer, buffers alternate =======================
+        if (lane == 0) {
+            const uint32_t idesc_mini = make_idesc_fmt(2 * MT_BK, a.env_fmt);
+            bool alive = mbar_wait(u_bar, 0u, abort_flag, a.status);
+            int vb = 0;
+            uint32_t vph = 0;
+            for (int p = 0; p < npr && alive; ++p) {
+                const int g = p & 1;
+                alive = mt_wait2(vfull_bar + 8 * vb, vph, eempty_bar + 8 * g, ((uint32_t)(p >> 1) & 1u) ^ 1u, abort_flag, a.status);
+                if (!alive) break;
+                tc_fence_after();
+                for (int q = 0; q < a.kc / 2; ++q) {
+                    const uint64_t ud = make_smem_desc_plain(u_smem + (uint32_t)q * 4096u, 2048u, 128u);
+                    const uint64_t vd = make_smem_desc_plain(v_smem + (uint32_t)vb * img_bytes + (uint32_t)q * 4096u, 2048u, 128u);
+                    umma_ss(tmem_e + (uint32_t)(g * 128), ud, vd, idesc_mini, q > 0 ? 1u : 0u);
+                }
+                umma_commit(efull_bar + 8 * g);
+                umma_commit(vempty_bar + 8 * vb);
+                if (++vb == nv) { vb = 0; vph ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ===================== main MMA issuers: issuer g takes the pairs p = g, g + 2, ... =====================
+        const int g = warp == MS_W_MMA0 ? 0 : 1;
+        if (lane == 0) {
+            const uint32_t idesc_main = make_idesc(a.bn);
+            bool alive = true;
+            int it = 0;
+            for (int p = g; p < npr && alive; p += 2, ++it) {
+                const int bp = p % nbp;
+                const uint32_t bph = (uint32_t)(p / nbp) & 1u, aph = (uint32_t)it & 1u;
+                const int s0 = 2 * bp;
+                const bool two = 2 * p + 1 < nkb;
+                alive = two ? mt_wait3(afull_bar + 8 * g, aph, bfull_bar + 8 * s0, bph, bfull_bar + 8 * (s0 + 1), bph, abort_flag, a.status)
+                            : mt_wait2(afull_bar + 8 * g, aph, bfull_bar + 8 * s0, bph, abort_flag, a.status);
+                if (!alive) break;
+                tc_fence_after();
+                for (int h = 0; h < (two ? 2 : 1); ++h) {
+                    const uint64_t bdesc = make_smem_desc(smem_base + (uint32_t)(s0 + h) * b_bytes);
+                    const uint32_t a_t = tmem_a + (uint32_t)(g * 64 + h * 32);
+#pragma unroll
+                    for (int k4 = 0; k4 < MT_BK / 16; ++k4)
+                        umma_ts(tmem_d + (uint32_t)(g * MS_BN), a_t + (uint32_t)(8 * k4), bdesc + (uint64_t)(2 * k4), idesc_main,
+                                (it > 0 || h > 0 || k4 > 0) ? 1u : 0u);
+                }
+                umma_commit(aempty_bar + 8 * g);
+                umma_commit(bempty_bar + 8 * bp);
+            }
+            if (alive && it > 0) umma_commit(accum_bar); else mbar_arrive(accum_bar);
+        }
+        __syncwarp();
+    }
+    if (SPLIT && warp >= MS_W_TMA) {                    // the builder warps run these barriers inside their epilogue
         cluster.barrier_wait();
         cluster.sync();
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == MT_W_MMA) tmem_dealloc(tmem_d, MT_TMEM_COLS);
+    if (warp == MS_W_MMA0) tmem_dealloc(tmem_base_slot, MT_TMEM_COLS);
 }
 
 // bf16 intermediate -> the fp32 inspection buffer
@@ -535,20 +773,21 @@ template <bool STAGE_A>
 static mdbf_status_t launch_mat(const MatArgs &a0, const CUtensorMap &tm, const CUtensorMap &tmo, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        MDBF_CUDA(cudaFuncSetAttribute(mat_stage_kernel<STAGE_A, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)mt_smem_bytes(4, 3, MT_BN, 0)));
-        MDBF_CUDA(cudaFuncSetAttribute(mat_stage_kernel<STAGE_A, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)mt_smem_bytes(4, 3, MT_BN, 0)));
+        const int max_smem = (int)mt_smem_bytes(4, 3, MT_BN, 0);
+        MDBF_CUDA(cudaFuncSetAttribute(mat_stage_kernel<STAGE_A>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        MDBF_CUDA(cudaFuncSetAttribute(mat_small_kernel<STAGE_A, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        MDBF_CUDA(cudaFuncSetAttribute(mat_small_kernel<STAGE_A, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
         attr_set = true;
     }
     MatArgs a = a0;
     const int rb = ceil_div(a.rows, MT_BM), npr = ceil_div(ceil_div(a.cols, MT_BK), 2);
+    const bool small = a.T <= MS_BN;
     // One token tile of at most 64 tokens leaves most SMs without work and every CTA with a long serial
     // chain of K blocks: split the reduction over a cluster of up to 8 CTAs.
     // Cost model: waves x (pairs per CTA + fixed part, in pairs).
     int ks = 1;
-    if (a.T <= 64) {
-        const int fixed = mt_env_int("MDBF_MAT_FIXED_COST", 8), max_ks = mt_env_int("MDBF_MAT_MAX_KS", 8);
+    if (small) {
+        const int fixed = mt_env_int("MDBF_MAT_FIXED_COST", 12), max_ks = mt_env_int("MDBF_MAT_MAX_KS", 8);
         long best = -1;
         for (int c = 1; c <= 8 && c <= max_ks; ++c) {
             const int per = ceil_div(npr, c);
@@ -566,7 +805,7 @@ static mdbf_status_t launch_mat(const MatArgs &a0, const CUtensorMap &tm, const 
     a.ns = mt_ring(a.kc, a.nv, a.bn, part_bytes);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(rb, ceil_div(a.T, a.bn), ks);
-    cfg.blockDim = dim3(MT_THREADS);
+    cfg.blockDim = dim3(small ? MS_THREADS : MT_THREADS);
     cfg.dynamicSmemBytes = mt_smem_bytes(a.kc, a.nv, a.bn, part_bytes);
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
@@ -578,8 +817,9 @@ static mdbf_status_t launch_mat(const MatArgs &a0, const CUtensorMap &tm, const 
     attr[1].val.clusterDim.z = ks;
     cfg.attrs = attr;
     cfg.numAttrs = ks > 1 ? 2 : 1;
-    if (ks > 1) MDBF_CUDA(cudaLaunchKernelEx(&cfg, mat_stage_kernel<STAGE_A, true>, a, tm, tmo));
-    else MDBF_CUDA(cudaLaunchKernelEx(&cfg, mat_stage_kernel<STAGE_A, false>, a, tm, tmo));
+    if (!small) MDBF_CUDA(cudaLaunchKernelEx(&cfg, mat_stage_kernel<STAGE_A>, a, tm, tmo));
+    else if (ks > 1) MDBF_CUDA(cudaLaunchKernelEx(&cfg, mat_small_kernel<STAGE_A, true>, a, tm));
+    else MDBF_CUDA(cudaLaunchKernelEx(&cfg, mat_small_kernel<STAGE_A, false>, a, tm));
     return MDBF_OK;
 }
 

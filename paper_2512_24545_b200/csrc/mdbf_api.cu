@@ -343,9 +343,10 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         // cluster when few tokens would leave SMs idle); the others remain selectable
         if (!tc_ok) kernel = MDBF_KERNEL_ALU;
         else if (T == 1 && tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
-        // rebuilding W_hat tiles and running one GEMM of width T beats the l sign GEMMs of the expanded order
-        // from 32 tokens on, and at every T >= 2 for the rank-1 envelope (measured crossovers)
-        else if ((T >= 32 || L.d.l == 1) && mat_path_supports(L, x, T)) kernel = MDBF_KERNEL_MAT;
+        // more tokens: rebuilding W_hat tiles and running one GEMM of width T (measured faster than, or equal
+        // to, the l sign GEMMs of the expanded order at every T >= 2); the expanded order serves the layers
+        // the tensor map over x cannot take (d_in not a multiple of 8, unaligned x)
+        else if (mat_path_supports(L, x, T)) kernel = MDBF_KERNEL_MAT;
         else if (L.xsB) kernel = MDBF_KERNEL_PREFILL;
         else if (tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
         else kernel = MDBF_KERNEL_DECODE;
