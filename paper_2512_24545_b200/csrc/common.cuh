@@ -27,6 +27,14 @@ struct TiledSigns {
     int ktiles;             // ceil(cols / 128)
 };
 
+// tensor maps of the last materialised-order forward (they depend only on the pointers and T)
+struct MatMaps {
+    bool valid;
+    const void *x, *y;
+    int T;
+    CUtensorMap tmx, tmz, tmzo, tmyo;
+};
+
 struct Layer {
     mdbf_desc_t d;
     int device;
@@ -60,6 +68,7 @@ struct Layer {
     uint16_t *viA, *viB;          // V images [pairs of K blocks][kcm][16][8][8]
     int kcm;                      // 16-byte chunks of the mode axis: 2 (l <= 16) or 4 (l <= 32)
     __nv_bfloat16 *zb;            // bf16 intermediate [max_T][padA]
+    MatMaps mat_maps;
     // scratch
     float *z;                     // [kMaxKSplit][zT][k] stage-B partial sums of the small-T kernel
     size_t zstride;               // zT * k

@@ -831,20 +831,30 @@ mdbf_status_t launch_forward_mat(Layer &L, const void *x, void *y, int T, cudaSt
         return MDBF_ERR_SHAPE;
     }
     const int bn = T >= MT_BN ? MT_BN : ((T + 15) / 16) * 16;
-    CUtensorMap tmx, tmz, tmzo, tmyo;
-    mdbf_status_t rc = make_act_tensor_map(&tmx, x, (size_t)T, d.d_in, d.d_in, bn);
-    if (rc) return rc;
-    rc = make_act_tensor_map(&tmz, L.zb, (size_t)T, d.k, L.padA, bn);
-    if (rc) return rc;
-    rc = make_out_tensor_map(&tmzo, L.zb, T, d.k, L.padA);
-    if (rc) return rc;
-    // y goes out by TMA when its base and row pitch are 16-byte aligned and it is bf16; otherwise by plain stores
-    const bool y_tma = L.out_mode == 0 && (reinterpret_cast<uintptr_t>(y) & 15u) == 0 && d.d_out % 8 == 0;
-    tmyo = tmzo;
-    if (y_tma) {
-        rc = make_out_tensor_map(&tmyo, y, T, d.d_out, d.d_out);
+    // y goes out by TMA when its base and row pitch are 16-byte aligned and it is bf16; otherwise by plain stores.
+    // Small tiles (T <= 64) always use plain stores and need no output maps.
+    const bool small = T <= MS_BN;
+    const bool y_tma = !small && L.out_mode == 0 && (reinterpret_cast<uintptr_t>(y) & 15u) == 0 && d.d_out % 8 == 0;
+    // The tensor maps depend only on (x, y, T): a caller that repeats a call (a decoding loop, a replayed
+    // graph being captured again) reuses the encoded maps of the last call.
+    MatMaps &m = L.mat_maps;
+    mdbf_status_t rc;
+    if (!(m.valid && m.x == x && m.T == T)) {
+        m.valid = false;
+        rc = make_act_tensor_map(&m.tmx, x, (size_t)T, d.d_in, d.d_in, bn);
         if (rc) return rc;
+        rc = make_act_tensor_map(&m.tmz, L.zb, (size_t)T, d.k, L.padA, bn);
+        if (rc) return rc;
+        rc = make_out_tensor_map(&m.tmzo, L.zb, T, d.k, L.padA);
+        if (rc) return rc;
+        m.x = x; m.T = T; m.y = nullptr; m.valid = true;
     }
+    if (y_tma && m.y != y) {
+        rc = make_out_tensor_map(&m.tmyo, y, T, d.d_out, d.d_out);
+        if (rc) return rc;
+        m.y = y;
+    }
+    const CUtensorMap &tmx = m.tmx, &tmz = m.tmz, &tmzo = m.tmzo, &tmyo = y_tma ? m.tmyo : m.tmzo;
 
     MatArgs b = {};
     b.wk = L.wkB; b.rows_pad = L.rpB; b.rows = d.k; b.cols = d.d_in;
