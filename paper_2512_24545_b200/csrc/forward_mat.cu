@@ -115,8 +115,9 @@ __device__ __forceinline__ void mt_expand_half(const uint32_t (&v)[32], uint32_t
         for (int i = 0; i < 4; ++i) {
             const int col = c4 * 8 + 2 * i;
             const uint32_t e = tm::pack_bf16x2(__uint_as_float(v[col]), __uint_as_float(v[col + 1]));
-            // bit 0 of the shifted byte -> bit 15, bit 1 -> bit 31; the other product bits fall outside the mask
-            const uint32_t m = ((byte >> (2 * i)) * 0x40008000u) & 0x80008000u;
+            // bit 2i of the byte -> bit 15, bit 2i+1 -> bit 31; the other product bits fall outside the mask and the
+            // two shifted copies cannot overlap.  A multiply (idle FMA pipe) instead of a shift on the busy ALU pipe.
+            const uint32_t m = (byte * (0x40008000u >> (2 * i))) & 0x80008000u;
             o[c4 * 4 + i] = e ^ m;
         }
     }
@@ -281,7 +282,7 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
                 asm volatile("bar.sync %0, 128;\n" ::"r"(1 + g) : "memory");
                 if ((tid & 127) == 0 && tau0 + g * 64 < a.T) {
                     tma_store_2d(&tmap_out, row0, tau0 + g * 64, smem_base + (uint32_t)g * (64 * MT_BM * 2));
-                    bulk_commit_wait_all();
+                    bulk_commit_wait_read();
                 }
             }
         } else if (alive) {

@@ -110,9 +110,11 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *tmap, int x, int
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];\n"
                  ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(src) : "memory");
 }
-__device__ __forceinline__ void bulk_commit_wait_all() {
+// closes the bulk async-group and waits until its stores have read their shared-memory source (the
+// writes to global memory complete before the grid does)
+__device__ __forceinline__ void bulk_commit_wait_read() {
     asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
-    asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory");
 }
 // K-major shared-memory operand without swizzle: 8-row x 16-byte core matrices of 128 contiguous
 // bytes; `lbo` bytes between core matrices adjacent along K, `sbo` bytes between 8-row groups.
