@@ -126,18 +126,25 @@ mdbf_status_t mdbf_get_envelope(mdbf_handle_t h, int which, float *out, int out_
 /* Read the layer's descriptor back. */
 mdbf_status_t mdbf_get_desc(mdbf_handle_t h, mdbf_desc_t *out);
 
-/* Force a kernel for later forwards on this handle (tests, benchmarks). */
+/* Force a kernel for later forwards on this handle (tests, benchmarks).  MDBF_KERNEL_PREFILL
+ * allocates that kernel's scratch (max_T * l * (d_in + k) * 2 bytes of pre-scaled operands) on the
+ * first request, which synchronises the device; a forward that falls back to it without this call
+ * allocates on its first use, so make that first use outside stream capture. */
 mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel /* mdbf_kernel_t */);
 
 /* ---------------------------------------------------------------- forward
- * y = W_hat x (Eq. DBF-inference-form with Eq. me-dbf-expand; steps: scale by
- * V_B, sign contraction with S_B, contract modes with U_B, scale by V_A, sign
- * contraction with S_A, contract modes with U_A).
+ * y = W_hat x, evaluated stage by stage, z = (S_B (.) U_B V_B^T) x, y = (S_A (.) U_A V_A^T) z
+ * (Eq. DBF-inference-form).  One token and the selectable expanded-order kernels follow
+ * Eq. me-dbf-expand (scale by V, sign contraction with S, contract the l modes with U); from two
+ * tokens on the default kernels rebuild each factor S (.) U V^T of Eq. me-dbf-basis tile by tile
+ * and multiply it by the activations once.  Both orders compute the same y up to rounding.
  *   x  device, T x d_in  of act_dtype (token-contiguous), read only
  *   y  device, T x d_out of act_dtype, written (round-to-nearest-even)
  *   act_dtype  MDBF_BF16 or MDBF_F32 (MDBF_F16 is accepted by the ALU path)
- * Accumulation is fp32.  Asynchronous on `stream`; allocates nothing, does not
- * synchronise.  x and y must not alias.
+ * Accumulation is fp32.  Asynchronous on `stream`; allocates nothing and does not synchronise,
+ * except for the first forward of a handle that has to run the expanded order for T >= 2 without
+ * a prior mdbf_set_kernel(PREFILL): layers with d_in % 8 != 0 get that scratch at pack time, so
+ * this concerns only an x that is not 16-byte aligned.  x and y must not alias.
  * Errors: INVALID_ARG, SHAPE (T < 1 or T > max_T), DTYPE, CUDA. */
 mdbf_status_t mdbf_linear_forward(mdbf_handle_t h, const void *x, void *y, int32_t T,
                                   int32_t act_dtype, void *stream);

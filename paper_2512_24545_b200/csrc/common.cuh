@@ -60,7 +60,7 @@ struct Layer {
     int rpA, rpB;                 // rows padded to 128
     int padA, padB;               // reduction length (k, d_in) padded to 64
     float *vtB;                   // V_B transposed, fp32 [LP][padB]
-    __nv_bfloat16 *xsB, *xsA;     // pre-scaled operands [xs_rows][padB], [xs_rows][padA]
+    __nv_bfloat16 *xsB, *xsA;     // pre-scaled operands [xs_rows][padB], [xs_rows][padA]; allocated on first use of the expanded order
     size_t xs_rows;               // max_T * LP rounded up to 256
     CUtensorMap tmB[3], tmA[3];   // tensor maps of xsB / xsA with boxes of 64, 128 and 256 rows (few tokens load a narrow box)
     // materialised-envelope kernel: 16-bit envelope images in mini-MMA operand order (see forward_mat.cu)
@@ -122,6 +122,7 @@ mdbf_status_t launch_kblock(const uint32_t *canon, int rows, int nwords, uint2 *
                             cudaStream_t st);
 mdbf_status_t launch_vtrans(const void *V, int cols, int l, int env_dtype, float *out, int pad, int LP, cudaStream_t st);
 mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad, int box_rows);
+mdbf_status_t ensure_prefill_scratch(Layer &L);
 mdbf_status_t make_act_tensor_map(CUtensorMap *out, const void *base, size_t rows, int cols, int stride, int box_rows);
 mdbf_status_t launch_uimg(const void *U, int rows, int l, int env_dtype, uint16_t *out, int rblocks, int kc, cudaStream_t st);
 mdbf_status_t launch_forward_mat(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches);

@@ -598,11 +598,34 @@ static mdbf_status_t run_prefill(Layer &L, const void *x, void *y, int T, cudaSt
     return launch_gemm<LP, true>(a, L.tmA[bi], st);
 }
 
+// Scratch of the expanded order: the pre-scaled operands and their tensor maps.  Allocated on first use
+// (mdbf_pack does it only for layers the materialised order cannot serve), which synchronises the device.
+mdbf_status_t ensure_prefill_scratch(Layer &L) {
+    if (L.xsB) return MDBF_OK;
+    L.xs_rows = ((size_t)L.d.max_T * L.LP + 255) / 256 * 256;
+    __nv_bfloat16 *b = nullptr, *a = nullptr;
+    MDBF_CUDA(cudaMalloc(&b, L.xs_rows * L.padB * 2));
+    cudaError_t e = cudaMalloc(&a, L.xs_rows * L.padA * 2);
+    if (e == cudaSuccess) e = cudaMemset(b, 0, L.xs_rows * L.padB * 2);
+    if (e == cudaSuccess) e = cudaMemset(a, 0, L.xs_rows * L.padA * 2);
+    if (e != cudaSuccess) { cudaFree(b); cudaFree(a); return cuda_fail(e, "scratch of the expanded order"); }
+    for (int i = 0; i < 3; ++i) {
+        mdbf_status_t rc = make_xs_tensor_map(&L.tmB[i], b, L.xs_rows, L.padB, 64 << i);
+        if (rc == MDBF_OK) rc = make_xs_tensor_map(&L.tmA[i], a, L.xs_rows, L.padA, 64 << i);
+        if (rc) { cudaFree(b); cudaFree(a); return rc; }
+    }
+    L.xsB = b; L.xsA = a;
+    return MDBF_OK;
+}
+
 mdbf_status_t launch_forward_prefill(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches) {
-    if (!L.xsB) {
-        set_error("mdbf_linear_forward: this layer was packed with max_T <= %d and holds no large-T scratch",
-                  kDecodeMaxT);
+    if (!L.vtB) {
+        set_error("mdbf_linear_forward: this layer was packed with max_T = 1 and holds nothing for the expanded order");
         return MDBF_ERR_SHAPE;
+    }
+    {
+        mdbf_status_t rc0 = ensure_prefill_scratch(L);
+        if (rc0) return rc0;
     }
     mdbf_status_t rc;
     switch (L.LP) {

@@ -58,7 +58,7 @@ static mdbf_status_t check_handle(mdbf_handle_t h, const char *fn) {
 }
 
 static void free_layer(Layer &L) {
-    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.vpA, L.vpB, L.vxA, L.vxB, L.wk2A, L.wk2B, L.wkA, L.wkB, L.uiA, L.uiB, L.viA, L.viB, L.vtB, L.xsB, L.xsA, L.z, L.zsum, L.xstage, L.ystage, L.status};
+    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.vpA, L.vpB, L.vxA, L.vxB, L.wk2A, L.wk2B, L.wkA, L.wkB, L.uiA, L.uiB, L.viA, L.viB, L.vtB, L.xsB, L.xsA, L.zb, L.z, L.zsum, L.xstage, L.ystage, L.status};
     for (void *p : ptrs)
         if (p) cudaFree(p);
 }
@@ -193,21 +193,17 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     if (want_prefill) {
         L.xs_rows = ((size_t)d.max_T * L.LP + 255) / 256 * 256;
         PACK_CUDA(cudaMalloc(&L.vtB, (size_t)L.LP * L.padB * sizeof(float)));
-        PACK_CUDA(cudaMalloc(&L.xsB, L.xs_rows * L.padB * 2));
-        PACK_CUDA(cudaMalloc(&L.xsA, L.xs_rows * L.padA * 2));
-        PACK_CUDA(cudaMemsetAsync(L.xsB, 0, L.xs_rows * L.padB * 2, st));
-        PACK_CUDA(cudaMemsetAsync(L.xsA, 0, L.xs_rows * L.padA * 2, st));
-        // the materialised-envelope kernel keeps its bf16 intermediate [max_T][padA] in the same scratch
-        L.zb = L.xsA;
+        // The pre-scaled operands of the expanded order (max_T * LP * (d_in + k) * 2 bytes) are allocated on
+        // its first use (ensure_prefill_scratch): the default path for T >= 2 does not need them.
+        // bf16 intermediate of the materialised-envelope kernels, [max_T][padA]; the padding columns stay zero
+        PACK_CUDA(cudaMalloc(&L.zb, (size_t)d.max_T * L.padA * 2));
+        PACK_CUDA(cudaMemsetAsync(L.zb, 0, (size_t)d.max_T * L.padA * 2, st));
         L.kcm = d.l <= 16 ? 2 : 4;
         PACK_CUDA(cudaMalloc(&L.uiA, (size_t)(L.rpA / 128) * L.kcm * 1024 * sizeof(uint16_t)));
         PACK_CUDA(cudaMalloc(&L.uiB, (size_t)(L.rpB / 128) * L.kcm * 1024 * sizeof(uint16_t)));
         PACK_CUDA(cudaMalloc(&L.viA, (size_t)ceil_div(L.padA, 128) * L.kcm * 1024 * sizeof(uint16_t)));
         PACK_CUDA(cudaMalloc(&L.viB, (size_t)ceil_div(L.padB, 128) * L.kcm * 1024 * sizeof(uint16_t)));
-        for (int i = 0; i < 3; ++i) {
-            PACK_RC(make_xs_tensor_map(&L.tmB[i], L.xsB, L.xs_rows, L.padB, 64 << i));
-            PACK_RC(make_xs_tensor_map(&L.tmA[i], L.xsA, L.xs_rows, L.padA, 64 << i));
-        }
+        if (d.d_in % 8 != 0) PACK_RC(ensure_prefill_scratch(L));     // no tensor map over x: the expanded order will run
     }
     L.zstride = (size_t)decode_scratch_T(d) * d.k;
     PACK_CUDA(cudaMalloc(&L.z, (size_t)kMaxKSplit * L.zstride * sizeof(float)));
@@ -323,6 +319,10 @@ mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel) {
         set_error("mdbf_set_kernel: unknown kernel %d", kernel);
         return MDBF_ERR_INVALID_ARG;
     }
+    if (kernel == MDBF_KERNEL_PREFILL && h->L.vtB) {      // allocate its scratch here rather than inside a forward
+        rc = ensure_prefill_scratch(h->L);
+        if (rc) return rc;
+    }
     h->kernel = kernel;
     return MDBF_OK;
 }
@@ -347,7 +347,7 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         // to, the l sign GEMMs of the expanded order at every T >= 2); the expanded order serves the layers
         // the tensor map over x cannot take (d_in not a multiple of 8, unaligned x)
         else if (mat_path_supports(L, x, T)) kernel = MDBF_KERNEL_MAT;
-        else if (L.xsB) kernel = MDBF_KERNEL_PREFILL;
+        else if (L.vtB) kernel = MDBF_KERNEL_PREFILL;
         else if (tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
         else kernel = MDBF_KERNEL_DECODE;
     }

@@ -94,3 +94,31 @@ def test_mat_kernel_rejects_what_it_cannot_take():
         with pytest.raises(M.MdbfError) as e:
             g.forward(x1, kernel=M.KERNEL_MAT)                                  # one token
         assert e.value.status == M.ERR_SHAPE
+
+
+def test_auto_dispatch_reports_its_kernel_and_serves_unaligned_x():
+    spec = spec_of(256, 512, 256, 16)
+    with GpuLayer(spec, 64) as g:
+        assert M.mdbf_last_kernel(g.h) == 0
+        x1 = inputs.make_activations(spec, 1)
+        g.forward(x1)
+        assert M.mdbf_last_kernel(g.h) == M.KERNEL_TMEM
+        x8 = inputs.make_activations(spec, 8)
+        y8 = g.forward(x8)
+        assert M.mdbf_last_kernel(g.h) == M.KERNEL_MAT
+        ref = g.oracle_forward(x8)
+        assert rel_err(y8, ref) <= TOL["bf16"]
+        # x two bytes off a 16-byte boundary: no tensor map over it, the expanded order runs (and allocates
+        # its scratch on this first use)
+        buf = torch.zeros(8 * spec.d_in + 8, dtype=torch.bfloat16, device="cuda")
+        xd = buf[1:1 + 8 * spec.d_in].view(8, spec.d_in)
+        xd.copy_(torch.from_numpy(x8).to(torch.bfloat16))
+        assert xd.data_ptr() % 16 == 2
+        yd = torch.zeros((8, spec.d_out), dtype=torch.bfloat16, device="cuda")
+        M.mdbf_linear_forward(g.h, xd.data_ptr(), yd.data_ptr(), 8, M.BF16, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert M.mdbf_last_kernel(g.h) == M.KERNEL_PREFILL
+        assert rel_err(yd.to(torch.float32).cpu().numpy(), ref) <= TOL["bf16"]
+    with GpuLayer(inputs.tiny(), 8) as g:                                      # fp32 layer
+        g.forward(inputs.make_activations(inputs.tiny(), 8))
+        assert M.mdbf_last_kernel(g.h) == M.KERNEL_ALU
