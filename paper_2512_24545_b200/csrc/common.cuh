@@ -123,6 +123,7 @@ mdbf_status_t launch_kblock(const uint32_t *canon, int rows, int nwords, uint2 *
 mdbf_status_t launch_vtrans(const void *V, int cols, int l, int env_dtype, float *out, int pad, int LP, cudaStream_t st);
 mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad, int box_rows);
 mdbf_status_t ensure_prefill_scratch(Layer &L);
+mdbf_status_t ensure_kernel_layouts(Layer &L, int kernel, int T);
 mdbf_status_t make_act_tensor_map(CUtensorMap *out, const void *base, size_t rows, int cols, int stride, int box_rows);
 mdbf_status_t launch_uimg(const void *U, int rows, int l, int env_dtype, uint16_t *out, int rblocks, int kc, cudaStream_t st);
 mdbf_status_t launch_forward_mat(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches);

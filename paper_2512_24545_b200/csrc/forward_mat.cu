@@ -55,8 +55,8 @@ constexpr int MT_MAX_NV = 4;             // V-image ring depth in pairs of K blo
 constexpr int MT_TMEM_COLS = 512;
 
 struct MatArgs {
-    const uint2 *wk;         // K-blocked sign words [kblocks][rows_pad], 64 bits per row and block
-    int rows_pad;
+    const uint2 *wk2;        // sign words, row-block major [row block][kb_pad][128 rows], 64 bits per row and K block
+    int kb_pad;              // K blocks per row block in wk2 (even, zero padded)
     int rows, cols;
     const uint16_t *uimg;    // [row block][KC][16][8][8] 16-bit envelope values (see uimg_kernel)
     const uint16_t *vimg;    // [pair of K blocks][KC][16][8][8]: the same layout with the 128 columns of the pair as rows
@@ -213,8 +213,8 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
         const int grp = (warp >> 2) & 1, half = warp >> 3;
         const int arow = tid & 127;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const size_t wstride = (size_t)a.rows_pad * 2;
-        const uint32_t *wp = reinterpret_cast<const uint32_t *>(a.wk + (size_t)row0 + arow) + half;   // + kb * wstride
+        const size_t wstride = 2 * MT_BM;                                  // 32-bit words from one K block to the next
+        const uint32_t *wp = reinterpret_cast<const uint32_t *>(a.wk2 + (size_t)rb * a.kb_pad * MT_BM + arow) + half;   // + kb * wstride
         uint32_t w_next = grp < nkb ? __ldg(wp + (size_t)grp * wstride) : 0u;
         uint32_t w_next2 = grp + 2 < nkb ? __ldg(wp + (size_t)(grp + 2) * wstride) : 0u;
         bool alive = true;
@@ -496,17 +496,17 @@ mat_small_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in) {
         const int g = warp >> 3, blk = (warp >> 2) & 1;
         const int arow = tid & 127;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint2 *wp = a.wk + (size_t)kb0 * a.rows_pad + (size_t)row0 + arow;     // + kb * rows_pad
+        const uint2 *wp = a.wk2 + ((size_t)rb * a.kb_pad + kb0) * MT_BM + arow;       // + kb * 128
         const int kbf = 2 * g + blk;                                                   // this warp's first block
-        uint2 w_next = kbf < nkb ? __ldg(wp + (size_t)kbf * a.rows_pad) : make_uint2(0u, 0u);
-        uint2 w_next2 = kbf + 4 < nkb ? __ldg(wp + (size_t)(kbf + 4) * a.rows_pad) : make_uint2(0u, 0u);
+        uint2 w_next = kbf < nkb ? __ldg(wp + (size_t)kbf * MT_BM) : make_uint2(0u, 0u);
+        uint2 w_next2 = kbf + 4 < nkb ? __ldg(wp + (size_t)(kbf + 4) * MT_BM) : make_uint2(0u, 0u);
         bool alive = true;
         for (int i = 0; 2 * i + g < npr && alive; ++i) {
             const int kb = 2 * (2 * i + g) + blk;
             const uint32_t ph = (uint32_t)i & 1u;
             const uint2 w = w_next;
             w_next = w_next2;
-            w_next2 = kb + 8 < nkb ? __ldg(wp + (size_t)(kb + 8) * a.rows_pad) : make_uint2(0u, 0u);
+            w_next2 = kb + 8 < nkb ? __ldg(wp + (size_t)(kb + 8) * MT_BM) : make_uint2(0u, 0u);
             alive = mbar_wait(efull_bar + 8 * g, ph, abort_flag, a.status);
             if (!alive) break;
             tc_fence_after();
@@ -858,7 +858,7 @@ mdbf_status_t launch_forward_mat(Layer &L, const void *x, void *y, int T, cudaSt
     const CUtensorMap &tmx = m.tmx, &tmz = m.tmz, &tmzo = m.tmzo, &tmyo = y_tma ? m.tmyo : m.tmzo;
 
     MatArgs b = {};
-    b.wk = L.wkB; b.rows_pad = L.rpB; b.rows = d.k; b.cols = d.d_in;
+    b.wk2 = L.wk2B; b.kb_pad = L.kbpB; b.rows = d.k; b.cols = d.d_in;
     b.uimg = L.uiB; b.vimg = L.viB; b.kc = L.kcm; b.env_fmt = d.env_dtype == MDBF_BF16 ? 1u : 0u;
     b.nv = L.kcm == 2 ? 4 : 3;
     b.T = T; b.bn = bn;  b.zb = L.zb; b.zstride = L.padA; b.status = L.status;
@@ -867,7 +867,7 @@ mdbf_status_t launch_forward_mat(Layer &L, const void *x, void *y, int T, cudaSt
     if (rc) return rc;
 
     MatArgs a = {};
-    a.wk = L.wkA; a.rows_pad = L.rpA; a.rows = d.d_out; a.cols = d.k;
+    a.wk2 = L.wk2A; a.kb_pad = L.kbpA; a.rows = d.d_out; a.cols = d.k;
     a.uimg = L.uiA; a.vimg = L.viA; a.kc = L.kcm; a.env_fmt = b.env_fmt; a.nv = b.nv;
     a.T = T; a.bn = bn; 
     a.y = reinterpret_cast<__nv_bfloat16 *>(y); a.y32 = reinterpret_cast<float *>(y); a.y_mode = L.out_mode; a.status = L.status;

@@ -619,13 +619,9 @@ mdbf_status_t ensure_prefill_scratch(Layer &L) {
 }
 
 mdbf_status_t launch_forward_prefill(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches) {
-    if (!L.vtB) {
-        set_error("mdbf_linear_forward: this layer was packed with max_T = 1 and holds nothing for the expanded order");
+    if (!L.xsB || !L.vtB || !L.wkB) {
+        set_error("mdbf_linear_forward: the expanded-order kernel needs a layer packed with max_T >= 2");
         return MDBF_ERR_SHAPE;
-    }
-    {
-        mdbf_status_t rc0 = ensure_prefill_scratch(L);
-        if (rc0) return rc0;
     }
     mdbf_status_t rc;
     switch (L.LP) {

@@ -462,7 +462,7 @@ static bool plan_stage(int rows, int cols, int LP, int T, TmPlan *p) {
 }
 
 bool tmem_path_supports(const Layer &L, int T) {
-    if (!L.vpA || !L.vpB || L.d.l > 32) return false;
+    if (!L.wk2A || L.d.l > 32) return false;      // 16-bit envelopes, l <= 32 (the generic kernel's V copy is built on first use)
     TmPlan pb, pa;
     return plan_stage(L.d.k, L.d.d_in, L.LP, T, &pb) && plan_stage(L.d.d_out, L.d.k, L.LP, T, &pa);
 }
@@ -519,7 +519,7 @@ static mdbf_status_t run_tm(Layer &L, const void *x, void *y, int T, cudaStream_
 }
 
 mdbf_status_t launch_forward_tmem(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches) {
-    if (!L.vpA || !L.vpB) {
+    if (!L.wk2A || (T > 1 && (!L.vpA || !L.wkA))) {
         set_error("mdbf_linear_forward: this layer holds no TMEM-operand copies (fp32 envelopes or l > 32)");
         return MDBF_ERR_SHAPE;
     }

@@ -66,6 +66,75 @@ static void free_layer(Layer &L) {
 // number of tokens the small-T kernel's partial-sum scratch is sized for
 static int decode_scratch_T(const mdbf_desc_t &d) { return d.max_T < kDecodeMaxT ? d.max_T : kDecodeMaxT; }
 
+// mdbf_pack builds what the default dispatch uses (canonical words, the row-block-major sign copy, the
+// one-token V tiles, the envelope images).  The private layouts and scratch of the other kernels are built
+// here on their first use (or by mdbf_set_kernel): on the default stream, followed by a synchronisation.
+#define ENS_CUDA(call)                                                   \
+    do {                                                                 \
+        cudaError_t e__ = (call);                                        \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #call);            \
+    } while (0)
+#define ENS_RC(call)                                 \
+    do {                                             \
+        mdbf_status_t r__ = (call);                  \
+        if (r__ != MDBF_OK) return r__;              \
+    } while (0)
+static mdbf_status_t ensure_kblock_words(Layer &L) {
+    const mdbf_desc_t &d = L.d;
+    if (L.wkA) return MDBF_OK;
+    uint2 *a = nullptr, *b = nullptr;
+    ENS_CUDA(cudaMalloc(&a, (size_t)(L.padA / 64) * L.rpA * sizeof(uint2)));
+    cudaError_t e = cudaMalloc(&b, (size_t)(L.padB / 64) * L.rpB * sizeof(uint2));
+    if (e != cudaSuccess) { cudaFree(a); return cuda_fail(e, "K-blocked sign words"); }
+    L.wkA = a; L.wkB = b;
+    ENS_RC(launch_kblock(L.wA, d.d_out, L.wordsA, L.wkA, L.rpA, L.padA / 64, 0));
+    ENS_RC(launch_kblock(L.wB, d.k, L.wordsB, L.wkB, L.rpB, L.padB / 64, 0));
+    return MDBF_OK;
+}
+mdbf_status_t ensure_kernel_layouts(Layer &L, int kernel, int T) {
+    const mdbf_desc_t &d = L.d;
+    bool built = false;
+    if (kernel == MDBF_KERNEL_DECODE && !L.tA) {
+        ENS_CUDA(cudaMalloc(&L.tA, (size_t)L.rtA * L.ktA * 512));
+        ENS_CUDA(cudaMalloc(&L.tB, (size_t)L.rtB * L.ktB * 512));
+        ENS_CUDA(cudaMalloc(&L.vfA, (size_t)L.ktA * 8 * L.NT * 256));
+        ENS_CUDA(cudaMalloc(&L.vfB, (size_t)L.ktB * 8 * L.NT * 256));
+        ENS_CUDA(cudaMalloc(&L.z, (size_t)kMaxKSplit * L.zstride * sizeof(float)));
+        ENS_RC(launch_tile(L.wA, d.d_out, L.wordsA, L.tA, L.rtA, L.ktA, 0));
+        ENS_RC(launch_tile(L.wB, d.k, L.wordsB, L.tB, L.rtB, L.ktB, 0));
+        ENS_RC(launch_vfrag(L.VA, d.k, d.l, d.env_dtype, L.vfA, L.ktA, L.NT, 0));
+        ENS_RC(launch_vfrag(L.VB, d.d_in, d.l, d.env_dtype, L.vfB, L.ktB, L.NT, 0));
+        built = true;
+    }
+    if (kernel == MDBF_KERNEL_TMEM && T > 1 && L.wk2A && !L.vpA) {
+        ENS_RC(ensure_kblock_words(L));
+        ENS_CUDA(cudaMalloc(&L.vpA, (size_t)(L.padA / 64) * L.LP * 64 * sizeof(uint16_t)));
+        ENS_CUDA(cudaMalloc(&L.vpB, (size_t)(L.padB / 64) * L.LP * 64 * sizeof(uint16_t)));
+        ENS_RC(launch_vperm(L.VA, d.k, d.l, d.env_dtype, L.vpA, L.padA / 64, L.LP, 0));
+        ENS_RC(launch_vperm(L.VB, d.d_in, d.l, d.env_dtype, L.vpB, L.padB / 64, L.LP, 0));
+        built = true;
+    }
+    if (kernel == MDBF_KERNEL_PREFILL && L.zb && !L.xsB) {
+        ENS_RC(ensure_kblock_words(L));
+        if (!L.vtB) {
+            ENS_CUDA(cudaMalloc(&L.vtB, (size_t)L.LP * L.padB * sizeof(float)));
+            ENS_RC(launch_vtrans(L.VB, d.d_in, d.l, d.env_dtype, L.vtB, L.padB, L.LP, 0));
+        }
+        ENS_RC(ensure_prefill_scratch(L));
+        built = true;
+    }
+    if (built) ENS_CUDA(cudaStreamSynchronize(0));
+    return MDBF_OK;
+}
+static mdbf_status_t ensure_host_staging(Layer &L) {
+    if (L.xstage) return MDBF_OK;
+    ENS_CUDA(cudaMalloc(&L.xstage, (size_t)L.d.max_T * L.d.d_in * 4));
+    ENS_CUDA(cudaMalloc(&L.ystage, (size_t)L.d.max_T * L.d.d_out * 4));
+    return MDBF_OK;
+}
+#undef ENS_CUDA
+#undef ENS_RC
+
 }  // namespace mdbf
 
 using namespace mdbf;
@@ -162,15 +231,11 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
 
     PACK_CUDA(cudaMalloc(&L.wA, (size_t)d.d_out * L.wordsA * 4));
     PACK_CUDA(cudaMalloc(&L.wB, (size_t)d.k * L.wordsB * 4));
-    PACK_CUDA(cudaMalloc(&L.tA, (size_t)L.rtA * L.ktA * 512));
-    PACK_CUDA(cudaMalloc(&L.tB, (size_t)L.rtB * L.ktB * 512));
     PACK_CUDA(cudaMalloc(&L.UA, nUA * es));
     PACK_CUDA(cudaMalloc(&L.VA, nVA * es));
     PACK_CUDA(cudaMalloc(&L.UB, nUB * es));
     PACK_CUDA(cudaMalloc(&L.VB, nVB * es));
     L.NT = d.l <= 8 ? 1 : d.l <= 16 ? 2 : d.l <= 32 ? 4 : 8;
-    PACK_CUDA(cudaMalloc(&L.vfA, (size_t)L.ktA * 8 * L.NT * 256));
-    PACK_CUDA(cudaMalloc(&L.vfB, (size_t)L.ktB * 8 * L.NT * 256));
     L.LP = 1;
     while (L.LP < d.l) L.LP *= 2;
     L.padA = ceil_div(d.k, 64) * 64; L.padB = ceil_div(d.d_in, 64) * 64;
@@ -179,10 +244,6 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     const bool want_prefill = d.env_dtype != MDBF_F32 && d.l <= 32 && d.max_T >= 2;
     const bool want_tc = d.env_dtype != MDBF_F32 && d.l <= 32;
     if (want_tc) {
-        PACK_CUDA(cudaMalloc(&L.wkA, (size_t)(L.padA / 64) * L.rpA * sizeof(uint2)));
-        PACK_CUDA(cudaMalloc(&L.wkB, (size_t)(L.padB / 64) * L.rpB * sizeof(uint2)));
-        PACK_CUDA(cudaMalloc(&L.vpA, (size_t)(L.padA / 64) * L.LP * 64 * sizeof(uint16_t)));
-        PACK_CUDA(cudaMalloc(&L.vpB, (size_t)(L.padB / 64) * L.LP * 64 * sizeof(uint16_t)));
         const int NB = L.LP < 16 ? 16 : L.LP;
         L.kbpA = ceil_div(L.padA / 64, 2) * 2; L.kbpB = ceil_div(L.padB / 64, 2) * 2;
         PACK_CUDA(cudaMalloc(&L.vxA, (size_t)L.kbpA * NB * 64 * sizeof(uint16_t)));
@@ -191,8 +252,6 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
         PACK_CUDA(cudaMalloc(&L.wk2B, (size_t)(L.rpB / 128) * L.kbpB * 128 * sizeof(uint2)));
     }
     if (want_prefill) {
-        L.xs_rows = ((size_t)d.max_T * L.LP + 255) / 256 * 256;
-        PACK_CUDA(cudaMalloc(&L.vtB, (size_t)L.LP * L.padB * sizeof(float)));
         // The pre-scaled operands of the expanded order (max_T * LP * (d_in + k) * 2 bytes) are allocated on
         // its first use (ensure_prefill_scratch): the default path for T >= 2 does not need them.
         // bf16 intermediate of the materialised-envelope kernels, [max_T][padA]; the padding columns stay zero
@@ -203,13 +262,9 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
         PACK_CUDA(cudaMalloc(&L.uiB, (size_t)(L.rpB / 128) * L.kcm * 1024 * sizeof(uint16_t)));
         PACK_CUDA(cudaMalloc(&L.viA, (size_t)ceil_div(L.padA, 128) * L.kcm * 1024 * sizeof(uint16_t)));
         PACK_CUDA(cudaMalloc(&L.viB, (size_t)ceil_div(L.padB, 128) * L.kcm * 1024 * sizeof(uint16_t)));
-        if (d.d_in % 8 != 0) PACK_RC(ensure_prefill_scratch(L));     // no tensor map over x: the expanded order will run
     }
     L.zstride = (size_t)decode_scratch_T(d) * d.k;
-    PACK_CUDA(cudaMalloc(&L.z, (size_t)kMaxKSplit * L.zstride * sizeof(float)));
     PACK_CUDA(cudaMalloc(&L.zsum, (size_t)d.max_T * d.k * sizeof(float)));
-    PACK_CUDA(cudaMalloc(&L.xstage, (size_t)d.max_T * d.d_in * 4));
-    PACK_CUDA(cudaMalloc(&L.ystage, (size_t)d.max_T * d.d_out * 4));
     PACK_CUDA(cudaMalloc(&L.status, sizeof(int32_t)));
     PACK_CUDA(cudaMemsetAsync(L.status, 0, sizeof(int32_t), st));
     PACK_CUDA(cudaMemsetAsync(L.zsum, 0, (size_t)d.max_T * d.k * sizeof(float), st));
@@ -228,26 +283,17 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     }
     PACK_RC(launch_pack((const int8_t *)dsrc[0], d.d_out, d.k, L.wA, st));
     PACK_RC(launch_pack((const int8_t *)dsrc[1], d.k, d.d_in, L.wB, st));
-    PACK_RC(launch_tile(L.wA, d.d_out, L.wordsA, L.tA, L.rtA, L.ktA, st));
-    PACK_RC(launch_tile(L.wB, d.k, L.wordsB, L.tB, L.rtB, L.ktB, st));
     PACK_RC(launch_env_round((const float *)dsrc[2], L.UA, nUA, d.env_dtype, st));
     PACK_RC(launch_env_round((const float *)dsrc[3], L.VA, nVA, d.env_dtype, st));
     PACK_RC(launch_env_round((const float *)dsrc[4], L.UB, nUB, d.env_dtype, st));
     PACK_RC(launch_env_round((const float *)dsrc[5], L.VB, nVB, d.env_dtype, st));
-    PACK_RC(launch_vfrag(L.VA, d.k, d.l, d.env_dtype, L.vfA, L.ktA, L.NT, st));
-    PACK_RC(launch_vfrag(L.VB, d.d_in, d.l, d.env_dtype, L.vfB, L.ktB, L.NT, st));
     if (want_tc) {
-        PACK_RC(launch_kblock(L.wA, d.d_out, L.wordsA, L.wkA, L.rpA, L.padA / 64, st));
-        PACK_RC(launch_kblock(L.wB, d.k, L.wordsB, L.wkB, L.rpB, L.padB / 64, st));
-        PACK_RC(launch_vperm(L.VA, d.k, d.l, d.env_dtype, L.vpA, L.padA / 64, L.LP, st));
-        PACK_RC(launch_vperm(L.VB, d.d_in, d.l, d.env_dtype, L.vpB, L.padB / 64, L.LP, st));
         PACK_RC(launch_vtile(L.VA, d.k, d.l, d.env_dtype, L.vxA, L.kbpA, L.LP < 16 ? 16 : L.LP, st));
         PACK_RC(launch_vtile(L.VB, d.d_in, d.l, d.env_dtype, L.vxB, L.kbpB, L.LP < 16 ? 16 : L.LP, st));
         PACK_RC(launch_wk2(L.wA, d.d_out, L.wordsA, L.wk2A, L.rpA / 128, L.kbpA, st));
         PACK_RC(launch_wk2(L.wB, d.k, L.wordsB, L.wk2B, L.rpB / 128, L.kbpB, st));
     }
     if (want_prefill) {
-        PACK_RC(launch_vtrans(L.VB, d.d_in, d.l, d.env_dtype, L.vtB, L.padB, L.LP, st));
         PACK_RC(launch_uimg(L.UA, d.d_out, d.l, d.env_dtype, L.uiA, L.rpA / 128, L.kcm, st));
         PACK_RC(launch_uimg(L.UB, d.k, d.l, d.env_dtype, L.uiB, L.rpB / 128, L.kcm, st));
         PACK_RC(launch_uimg(L.VA, d.k, d.l, d.env_dtype, L.viA, ceil_div(L.padA, 128), L.kcm, st));     // V: columns of a pair of K blocks as rows
@@ -256,6 +302,8 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     PACK_CUDA(cudaStreamSynchronize(st));
     for (void *p : temps) cudaFree(p);
     temps.clear();
+    // a layer the materialised order can never serve (no tensor map over x) will run the expanded order
+    if (want_prefill && d.d_in % 8 != 0) PACK_RC(ensure_kernel_layouts(L, MDBF_KERNEL_PREFILL, 2));
 #undef PACK_CUDA
 #undef PACK_RC
     h->magic = kHandleMagic;
@@ -319,8 +367,10 @@ mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel) {
         set_error("mdbf_set_kernel: unknown kernel %d", kernel);
         return MDBF_ERR_INVALID_ARG;
     }
-    if (kernel == MDBF_KERNEL_PREFILL && h->L.vtB) {      // allocate its scratch here rather than inside a forward
-        rc = ensure_prefill_scratch(h->L);
+    // build the kernel's private layouts and scratch here rather than inside a forward
+    const bool tc_layer = h->L.wk2A != nullptr;
+    if (kernel == MDBF_KERNEL_DECODE || ((kernel == MDBF_KERNEL_TMEM || kernel == MDBF_KERNEL_PREFILL) && tc_layer)) {
+        rc = ensure_kernel_layouts(h->L, kernel, 2);
         if (rc) return rc;
     }
     h->kernel = kernel;
@@ -347,7 +397,7 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         // to, the l sign GEMMs of the expanded order at every T >= 2); the expanded order serves the layers
         // the tensor map over x cannot take (d_in not a multiple of 8, unaligned x)
         else if (mat_path_supports(L, x, T)) kernel = MDBF_KERNEL_MAT;
-        else if (L.vtB) kernel = MDBF_KERNEL_PREFILL;
+        else if (L.zb) kernel = MDBF_KERNEL_PREFILL;
         else if (tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
         else kernel = MDBF_KERNEL_DECODE;
     }
@@ -365,7 +415,8 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         return MDBF_ERR_INVALID_ARG;
     }
     int launches = 0;
-    mdbf_status_t rc;
+    mdbf_status_t rc = ensure_kernel_layouts(L, kernel, T);      // no-op for the default kernels
+    if (rc) return rc;
     if (kernel == MDBF_KERNEL_ALU) rc = launch_forward_alu(L, x, y, T, act_dtype, st, &launches);
     else if (kernel == MDBF_KERNEL_DECODE) rc = launch_forward_decode(L, x, y, T, st, &launches);
     else if (kernel == MDBF_KERNEL_TMEM) rc = launch_forward_tmem(L, x, y, T, st, &launches);
@@ -468,6 +519,8 @@ mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void
     if (!valid_dtype(act_dtype)) { set_error("mdbf_linear_forward_host: bad act_dtype %d", act_dtype); return MDBF_ERR_DTYPE; }
     cudaStream_t st = (cudaStream_t)stream;
     const size_t es = dtype_size(act_dtype);
+    rc = ensure_host_staging(L);
+    if (rc) return rc;
     MDBF_CUDA(cudaMemcpyAsync(L.xstage, x_host, (size_t)T * L.d.d_in * es, cudaMemcpyHostToDevice, st));
     rc = forward_impl(h, L.xstage, L.ystage, T, act_dtype, st);
     if (rc) return rc;
