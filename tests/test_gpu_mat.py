@@ -24,7 +24,7 @@ def spec_of(d_out, d_in, k, l, **kw):
 
 
 @pytest.mark.parametrize("l,T", [(16, 16), (16, 48), (16, 5), (16, 2), (4, 64), (4, 100), (1, 256), (1, 300),
-                                 (3, 40), (8, 33), (20, 9), (32, 11), (16, 600)])
+                                 (3, 40), (8, 33), (20, 9), (32, 11), (16, 600), (32, 130), (20, 300), (2, 65)])
 def test_mat_kernel_small_shapes(l, T):
     spec = spec_of(384, 576, 256, l)
     x = inputs.make_activations(spec, T)
@@ -66,11 +66,11 @@ def test_mat_kernel_split_reduction(shape):
         np.testing.assert_array_equal(y, g.forward(x, kernel=M.KERNEL_MAT))     # deterministic summation order
 
 
-@pytest.mark.parametrize("env_dtype", ["f16", "bf16"])
-def test_mat_kernel_envelope_types_and_other_kernels(env_dtype):
+@pytest.mark.parametrize("env_dtype,T", [("f16", 64), ("bf16", 64), ("f16", 200), ("bf16", 200)])
+def test_mat_kernel_envelope_types_and_other_kernels(env_dtype, T):
     spec = spec_of(256, 512, 256, 16, env_dtype=env_dtype)
-    x = inputs.make_activations(spec, 64)
-    with GpuLayer(spec, 64) as g:
+    x = inputs.make_activations(spec, T)
+    with GpuLayer(spec, T) as g:
         ref = g.oracle_forward(x)
         y_mat = g.forward(x, kernel=M.KERNEL_MAT)
         y_pf = g.forward(x, kernel=M.KERNEL_PREFILL)
