@@ -122,3 +122,32 @@ def test_auto_dispatch_reports_its_kernel_and_serves_unaligned_x():
     with GpuLayer(inputs.tiny(), 8) as g:                                      # fp32 layer
         g.forward(inputs.make_activations(inputs.tiny(), 8))
         assert M.mdbf_last_kernel(g.h) == M.KERNEL_ALU
+
+
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        d_out = int(rng.integers(1, 700))
+        d_in = 8 * int(rng.integers(1, 90))                      # the tensor map over x needs a multiple of 8
+        k = int(rng.integers(1, 500))
+        l = int(rng.choice([1, 2, 3, 5, 8, 13, 16, 17, 24, 32]))
+        T = int(rng.choice([2, 3, 7, 16, 17, 31, 48, 64, 65, 100, 255, 256, 257, 400]))
+        out.append((d_out, d_in, k, l, T))
+    return out
+
+
+@pytest.mark.parametrize("shape", _random_shapes(24, seed=2512))
+def test_mat_kernels_seeded_random_shapes(shape):
+    """Ragged sizes in every dimension at once, through AUTO (small-tile kernel up to 64 tokens, large-tile above)."""
+    d_out, d_in, k, l, T = shape
+    spec = spec_of(d_out, d_in, k, l)
+    x = inputs.make_activations(spec, T)
+    with GpuLayer(spec, T) as g:
+        y = g.forward(x)
+        assert M.mdbf_last_kernel(g.h) == M.KERNEL_MAT
+        assert M.mdbf_poll_status(g.h) == 0
+        assert np.all(np.isfinite(y))
+        # few terms per output (small k) do not average the roundings: worst case of four bf16 roundings
+        tol = TOL["bf16"] if k >= 32 else 4 * 2.0 ** -8
+        assert rel_err(y, g.oracle_forward(x)) <= tol
