@@ -40,11 +40,10 @@ namespace cg = cooperative_groups;
 
 namespace mdbf {
 
-constexpr int TX_GROUPS = 2;                           // expander groups of 4 warps; group g takes pairs g, g + 4, ...
+// expander groups of 4 warps (template parameter G of the kernel; group g takes the pairs g, g + G, ...): 2 for
+// CTAs with few pairs (all latency, fewer warps start faster), 3 for long CTAs (+5 % on 70B-class layers; 4: worse)
 constexpr int TX_ISSUERS = 4;                          // MMA issuer warps, one accumulator each (a thread issues ~1 MMA / 100+ clk here)
-constexpr int TX_EXPANDERS = TX_GROUPS * 128;
-constexpr int TX_W_ISSUER0 = TX_EXPANDERS / 32;
-constexpr int TX_THREADS = TX_EXPANDERS + TX_ISSUERS * 32 + 64;   // + sign loader warp + V loader warp
+constexpr int tx_threads(int groups) { return groups * 128 + TX_ISSUERS * 32 + 64; }   // + sign loader warp + V loader warp
 constexpr int TX_MAX_SSTAGES = 16;                     // sign ring: 2 KB per stage (one pair of K blocks)
 constexpr int TX_MAX_ASTAGES = 7;                      // A / V stages: 64 TMEM columns + two V tiles each
 
@@ -85,9 +84,11 @@ __device__ __forceinline__ bool tx_wait(uint32_t bar, uint32_t parity, volatile 
 //   sring [nsstages][2048 B]           packed sign words of a pair: [2][128 rows] uint2
 //   xp    [pairs_per_cta * 64] u32     activation pairs in MMA k order (bf16x2)
 //   part  [8][128] float               partial outputs pushed by the other cluster ranks (rank 0 only reads)
-template <int LP>
+template <int LP, int TX_GROUPS>
 __device__ __forceinline__ void tmem_t1_body(const TxArgs &a, const int rb) {
     using namespace tm;
+    constexpr int TX_EXPANDERS = TX_GROUPS * 128;
+    constexpr int TX_W_ISSUER0 = TX_EXPANDERS / 32;
     constexpr int NB = LP < 16 ? 16 : LP;                    // MMA N
     constexpr int VBYTES = 2 * NB * 128;                     // two tiles
     extern __shared__ unsigned char tx_smem_raw[];
@@ -370,20 +371,20 @@ __device__ __forceinline__ void tmem_t1_body(const TxArgs &a, const int rb) {
 }
 
 // One layer per launch: the arguments are plain kernel parameters (fastest for the small layers).
-template <int LP>
-__global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_kernel(const TxArgs a) {
-    tmem_t1_body<LP>(a, (int)blockIdx.x);
+template <int LP, int G>
+__global__ void __launch_bounds__(tx_threads(G), 1) tmem_t1_kernel(const TxArgs a) {
+    tmem_t1_body<LP, G>(a, (int)blockIdx.x);
 }
 
 // Several sibling layers per launch: each CTA picks its layer by its position in the grid.
-template <int LP>
-__global__ void __launch_bounds__(TX_THREADS, 1) tmem_t1_multi_kernel(const __grid_constant__ TxMulti m) {
+template <int LP, int G>
+__global__ void __launch_bounds__(tx_threads(G), 1) tmem_t1_multi_kernel(const __grid_constant__ TxMulti m) {
     int li = 0;
 #pragma unroll
     for (int i = 1; i < TX_MAX_LAYERS; ++i)
         if (i < m.nlayers && (int)blockIdx.x >= m.rb_start[i]) li = i;
     const TxArgs a = m.layer[li];                             // by value: one indexed read of the parameter block
-    tmem_t1_body<LP>(a, (int)blockIdx.x - m.rb_start[li]);
+    tmem_t1_body<LP, G>(a, (int)blockIdx.x - m.rb_start[li]);
 }
 
 // ----------------------------------------------------------- pack-time private copies
@@ -499,17 +500,17 @@ static bool plan_t1(int n, const int *rows, const int *kb_pad, int LP, TxPlan *p
     return nas >= 2 && p->smem <= 220 * 1024;
 }
 
-template <int LP>
-static mdbf_status_t launch_t1(const TxMulti &m, const TxPlan &p, cudaStream_t st) {
+template <int LP, int G>
+static mdbf_status_t launch_t1g(const TxMulti &m, const TxPlan &p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_kernel<LP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
-        MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_multi_kernel<LP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_kernel<LP, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_multi_kernel<LP, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
         attr_set = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(m.rb_start[m.nlayers], p.ks, 1);
-    cfg.blockDim = dim3(TX_THREADS);
+    cfg.blockDim = dim3(tx_threads(G));
     cfg.dynamicSmemBytes = p.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
@@ -521,9 +522,19 @@ static mdbf_status_t launch_t1(const TxMulti &m, const TxPlan &p, cudaStream_t s
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (m.nlayers == 1) MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_kernel<LP>, m.layer[0]));
-    else MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_multi_kernel<LP>, m));
+    if (m.nlayers == 1) MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_kernel<LP, G>, m.layer[0]));
+    else MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_multi_kernel<LP, G>, m));
     return MDBF_OK;
+}
+// Two expander groups for CTAs with few pairs of K blocks, three from `long_cta` pairs per CTA on (16: the
+// 4096 x 4096 layers keep two groups, the 11008- and 70B-class layers get three).
+template <int LP>
+static mdbf_status_t launch_t1(const TxMulti &m, const TxPlan &p, cudaStream_t st) {
+    static int long_cta = 0;
+    if (!long_cta) { const char *e = getenv("MDBF_T1_LONG_CTA"); long_cta = e ? atoi(e) : 16; if (long_cta < 1) long_cta = 1; }
+    int max_per = 0;
+    for (int i = 0; i < m.nlayers; ++i) max_per = max(max_per, p.pairs_per_cta[i]);
+    return max_per >= long_cta ? launch_t1g<LP, 3>(m, p, st) : launch_t1g<LP, 2>(m, p, st);
 }
 
 // Both stages of n layers that read the same x (n = 1: a single layer): one launch per stage.
