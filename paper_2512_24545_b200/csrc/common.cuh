@@ -142,6 +142,7 @@ mdbf_status_t launch_vperm(const void *V, int cols, int l, int env_dtype, uint16
                            cudaStream_t st);
 mdbf_status_t launch_forward_tmem_t1(Layer &L, const void *x, void *y, cudaStream_t st);
 constexpr int kMaxSiblings = 4;   // layers one launch of the one-token kernel can serve
+int last_t1_launch_count();
 mdbf_status_t launch_forward_tmem_t1_multi(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st);
 mdbf_status_t launch_wk2(const uint32_t *canon, int rows, int nwords, uint2 *out, int rblocks, int kb_pad,
                          cudaStream_t st);

@@ -529,7 +529,7 @@ mdbf_status_t launch_forward_tmem(Layer &L, const void *x, void *y, int T, cudaS
         rc = launch_forward_tmem_t1(L, x, y, st);
         if (rc) return rc;
         L.last_ksplit = 0;
-        *launches = 2;
+        *launches = last_t1_launch_count();
         return MDBF_OK;
     }
 #define MDBF_TM_CASE(lp) case lp: rc = bf ? run_tm<lp, true>(L, x, y, T, st) : run_tm<lp, false>(L, x, y, T, st); break;

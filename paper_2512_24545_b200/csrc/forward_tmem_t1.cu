@@ -51,6 +51,7 @@ struct TxArgs {
     const uint2 *wk2;         // sign words, row-block major: [row block][kb_pad][128 rows], 64 bits each
     int kb_pad;               // K blocks per row block in wk2 / vtile (even, zero padded)
     int rows, cols;
+    int rb0;                  // first row block this launch serves in this layer (a launch may cover a slice of the row blocks)
     const uint16_t *vtile;    // bf16 V tile images [kb_pad][NB * 64], 128B-swizzled, NB = max(LP, 16)
     const void *U;            // [rows][l] env_dtype
     int env_dtype, l;
@@ -373,7 +374,7 @@ __device__ __forceinline__ void tmem_t1_body(const TxArgs &a, const int rb) {
 // One layer per launch: the arguments are plain kernel parameters (fastest for the small layers).
 template <int LP, int G>
 __global__ void __launch_bounds__(tx_threads(G), 1) tmem_t1_kernel(const TxArgs a) {
-    tmem_t1_body<LP, G>(a, (int)blockIdx.x);
+    tmem_t1_body<LP, G>(a, (int)blockIdx.x + a.rb0);
 }
 
 // Several sibling layers per launch: each CTA picks its layer by its position in the grid.
@@ -384,7 +385,7 @@ __global__ void __launch_bounds__(tx_threads(G), 1) tmem_t1_multi_kernel(const _
     for (int i = 1; i < TX_MAX_LAYERS; ++i)
         if (i < m.nlayers && (int)blockIdx.x >= m.rb_start[i]) li = i;
     const TxArgs a = m.layer[li];                             // by value: one indexed read of the parameter block
-    tmem_t1_body<LP, G>(a, (int)blockIdx.x - m.rb_start[li]);
+    tmem_t1_body<LP, G>(a, (int)blockIdx.x - m.rb_start[li] + a.rb0);
 }
 
 // ----------------------------------------------------------- pack-time private copies
@@ -500,6 +501,9 @@ static bool plan_t1(int n, const int *rows, const int *kb_pad, int LP, TxPlan *p
     return nas >= 2 && p->smem <= 220 * 1024;
 }
 
+static thread_local int g_t1_launches = 0;      // kernels the last one-token forward of this thread launched
+int last_t1_launch_count() { return g_t1_launches; }
+
 template <int LP, int G>
 static mdbf_status_t launch_t1g(const TxMulti &m, const TxPlan &p, cudaStream_t st) {
     static bool attr_set = false;
@@ -524,6 +528,7 @@ static mdbf_status_t launch_t1g(const TxMulti &m, const TxPlan &p, cudaStream_t 
     cfg.numAttrs = 2;
     if (m.nlayers == 1) MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_kernel<LP, G>, m.layer[0]));
     else MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_multi_kernel<LP, G>, m));
+    ++g_t1_launches;
     return MDBF_OK;
 }
 // Two expander groups for CTAs with few pairs of K blocks, three from `long_cta` pairs per CTA on (16: the
@@ -537,6 +542,47 @@ static mdbf_status_t launch_t1(const TxMulti &m, const TxPlan &p, cudaStream_t s
     return max_per >= long_cta ? launch_t1g<LP, 3>(m, p, st) : launch_t1g<LP, 2>(m, p, st);
 }
 
+// One stage.  When the grid ends in a wave with only a few CTAs (448 row blocks on 148 SMs: the last 4 would
+// cost a whole wave), those row blocks go to a second, short launch that splits their reduction over a
+// cluster instead; both launches read the same input and write disjoint rows.
+template <int LP>
+static mdbf_status_t launch_stage(const TxMulti &full, const TxPlan &p, const int *kb_pad, cudaStream_t st) {
+    const int n = full.nlayers, R = full.rb_start[n];
+    int max_per = 0;
+    for (int i = 0; i < n; ++i) max_per = max(max_per, p.pairs_per_cta[i]);
+    const int tail = R % 148;                                   // CTAs of the last wave (cluster size 1)
+    if (!(p.ks == 1 && R > 148 && tail > 0 && 4 * tail <= 148 && max_per >= 16)) return launch_t1<LP>(full, p, st);
+
+    TxMulti part[2] = {};
+    int rows_tail[TX_MAX_LAYERS], kb_tail[TX_MAX_LAYERS], src_tail[TX_MAX_LAYERS];
+    const int cut = R - tail;                                   // global row blocks [0, cut) stay in the main launch
+    for (int i = 0; i < n; ++i) {
+        const int lo = full.rb_start[i], hi = full.rb_start[i + 1];
+        for (int h = 0; h < 2; ++h) {
+            const int a = max(lo, h ? cut : 0), b = min(hi, h ? R : cut);
+            if (a >= b) continue;
+            TxMulti &m = part[h];
+            TxArgs &t = m.layer[m.nlayers];
+            t = full.layer[i];
+            t.rb0 = a - lo;
+            if (h) { rows_tail[m.nlayers] = (b - a) * 128; kb_tail[m.nlayers] = kb_pad[i]; src_tail[m.nlayers] = i; }
+            m.rb_start[m.nlayers + 1] = m.rb_start[m.nlayers] + (b - a);
+            ++m.nlayers;
+        }
+    }
+    TxPlan pt;
+    if (!plan_t1(part[1].nlayers, rows_tail, kb_tail, LP, &pt)) return launch_t1<LP>(full, p, st);
+    for (int j = 0; j < part[1].nlayers; ++j) {
+        TxArgs &t = part[1].layer[j];
+        t.pairs_per_cta = pt.pairs_per_cta[j];
+        t.nastages = pt.nastages; t.nsstages = pt.nsstages; t.tmem_cols = pt.tmem_cols;
+        (void)src_tail[j];
+    }
+    mdbf_status_t rc = launch_t1<LP>(part[0], p, st);
+    if (rc) return rc;
+    return launch_t1<LP>(part[1], pt, st);
+}
+
 // Both stages of n layers that read the same x (n = 1: a single layer): one launch per stage.
 template <int LP>
 static mdbf_status_t run_t1(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st) {
@@ -545,6 +591,7 @@ static mdbf_status_t run_t1(Layer *const *Ls, int n, const void *x, void *const 
         rowsB[i] = Ls[i]->d.k; kbB[i] = Ls[i]->kbpB;
         rowsA[i] = Ls[i]->d.d_out; kbA[i] = Ls[i]->kbpA;
     }
+    g_t1_launches = 0;
     TxPlan pb, pa;
     if (!plan_t1(n, rowsB, kbB, LP, &pb) || !plan_t1(n, rowsA, kbA, LP, &pa)) {
         set_error("mdbf_linear_forward: the one-token TMEM kernel does not fit this shape");
@@ -570,9 +617,9 @@ static mdbf_status_t run_t1(Layer *const *Ls, int n, const void *x, void *const 
         s.nastages = pa.nastages; s.nsstages = pa.nsstages; s.tmem_cols = pa.tmem_cols; s.status = L.status;
         ma.rb_start[i + 1] = ma.rb_start[i] + ceil_div(d.d_out, 128);
     }
-    mdbf_status_t rc = launch_t1<LP>(mb, pb, st);
+    mdbf_status_t rc = launch_stage<LP>(mb, pb, kbB, st);
     if (rc) return rc;
-    return launch_t1<LP>(ma, pa, st);
+    return launch_stage<LP>(ma, pa, kbA, st);
 }
 
 // n <= TX_MAX_LAYERS layers with the same LP, all prepared for the one-token kernel.

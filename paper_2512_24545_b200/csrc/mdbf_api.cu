@@ -502,6 +502,7 @@ mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t 
         }
         mdbf_status_t rc = launch_forward_tmem_t1_multi(Ls, m, x, outs, st);
         if (rc) return rc;
+        layers[i0]->last_launches = last_t1_launch_count();
     }
     return MDBF_OK;
 }

@@ -55,6 +55,28 @@ def test_fused_siblings_one_token(shapes):
         assert rel_err(got, single) <= 1e-3                   # same arithmetic up to the order of the cluster reduction
 
 
+@pytest.mark.parametrize("shapes", [[(9600, 2048), (9600, 2048)],       # 150 row blocks on 148 SMs: two go to the short launch
+                                    [(19300, 2100)]])                    # one layer, 151 row blocks, ragged last block
+def test_last_partial_wave_goes_to_a_second_launch(shapes):
+    """Stage A has a few more row blocks than SMs: the row blocks of the last, nearly empty wave run in a
+    second launch with the reduction split over a cluster.  Every output row must still be written once."""
+    specs = sib_specs(256, shapes)
+    x = inputs.make_activations(specs[0], 1)
+    for (got, ref, single), sp in zip(run_siblings(specs, x), specs):
+        assert np.all(np.isfinite(got))
+        assert rel_err(got, ref) <= TOL["bf16"]
+        assert rel_err(got[:, -400:], ref[:, -400:]) <= TOL["bf16"]      # the rows the second launch wrote
+        assert rel_err(got, single) <= 1e-3
+
+
+def test_second_launch_is_counted():
+    spec = sib_specs(256, [(19300, 2100)])[0]
+    x = inputs.make_activations(spec, 1)
+    with GpuLayer(spec, 1) as g:
+        g.forward(x)
+        assert M.mdbf_last_launch_count(g.h) == 3             # stage B, stage A main part, stage A last row blocks
+
+
 def test_siblings_fall_back_to_separate_forwards():
     specs = sib_specs(256, [(128, 128), (64, 96)])
     x = inputs.make_activations(specs[0], 3)                  # three tokens: not fused
