@@ -31,7 +31,7 @@
 //
 // Every mbarrier wait is bounded; when one expires the kernel records MDBF_ERR_TIMEOUT in the
 // layer's status word, all roles fall through to the common exit, TMEM is released and the kernel
-// returns.  No TMA multicast is used.
+// returns.  Every TMA and bulk copy targets the issuing CTA's own shared memory only.
 #include <cooperative_groups.h>
 
 #include "tmem_ptx.cuh"

@@ -33,7 +33,7 @@
 //
 // Every mbarrier wait is bounded: when it expires the kernel records MDBF_ERR_TIMEOUT in
 // the layer's status word, all roles fall through to the common exit, TMEM is released and
-// the kernel returns.  No TMA multicast is used anywhere.
+// the kernel returns.  Every TMA and bulk copy targets the issuing CTA's own shared memory only.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -137,7 +137,7 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
 }
-// 2-D tiled TMA load into this CTA's shared memory, completion on an mbarrier (no multicast).
+// 2-D tiled TMA load into this CTA's shared memory, completion on an mbarrier (one destination CTA).
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int x, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"

@@ -36,7 +36,7 @@
 //
 // Every mbarrier wait is bounded; when one expires the kernel records MDBF_ERR_TIMEOUT, every role
 // falls through to the common exit (cluster barriers included), TMEM is released and the kernel
-// returns.  No TMA multicast is used.
+// returns.  Every TMA and bulk copy targets the issuing CTA's own shared memory only.
 #include <cooperative_groups.h>
 
 #include "tmem_ptx.cuh"

@@ -30,7 +30,7 @@
 // reduce their partial outputs through distributed shared memory (deterministic, no atomics).
 // Column order inside a K block as in forward_tmem.cu: MMA k index p is canonical column
 // 32*(p/32) + (p%32)/2 + 16*(p%2).  Every mbarrier wait is bounded (MDBF_ERR_TIMEOUT in the
-// status word, all roles fall through, TMEM released).  No TMA multicast.
+// status word, all roles fall through, TMEM released).  Every bulk copy targets the issuing CTA's own shared memory only.
 #include <cooperative_groups.h>
 #include <cstdlib>
 

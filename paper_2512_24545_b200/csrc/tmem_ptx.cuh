@@ -88,7 +88,7 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-// 2-D tiled TMA load into this CTA's shared memory, completion on an mbarrier (no multicast).
+// 2-D tiled TMA load into this CTA's shared memory, completion on an mbarrier (one destination CTA).
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int x, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
@@ -136,7 +136,7 @@ __device__ __forceinline__ uint32_t make_idesc_fmt(int n, uint32_t fmt) {
     d |= (uint32_t)(128 >> 4) << 24;
     return d;
 }
-// contiguous global -> this CTA's shared memory, completion on an mbarrier (no multicast)
+// contiguous global -> this CTA's shared memory, completion on an mbarrier (one destination CTA)
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
