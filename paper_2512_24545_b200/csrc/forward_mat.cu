@@ -13,6 +13,9 @@
 // two launches per forward.  The result differs from the expanded order only in rounding:
 // W_hat is rounded to bf16 once per entry, the activations are not rounded at all.
 //
+// Two kernels: mat_stage_kernel for more than 64 tokens (described here) and mat_small_kernel for one tile of
+// at most 64 tokens (further down).
+//
 // CTA = 128 rows of W_hat x up to 256 tokens, 20 warps; the unit of the pipeline is a PAIR of K blocks
 // (2 x 64 columns), because every barrier test, MMA and commit costs the issuing thread 60-150 cycles:
 //   warps 0-15 tile builders: warp = (half of a block's 64 columns, block of the pair, 32-row quadrant).
