@@ -76,7 +76,9 @@ struct Layer {
     void *xstage, *ystage;        // device staging for the host-buffer entry point
     int32_t *status;              // device status word
     int last_ksplit;              // how many partials the last forward wrote (0 = zsum valid, -1 = the intermediate is in zb)
-    int out_mode;                 // set per call: 0 y in the activation type; 1 / 2: fp32 y stored / added (a term of a sum)
+    int out_mode;                 // set per call: 0 y in the activation type; 1 / 2: fp32 y stored / added (a term of a sum);
+                                  // 3 (one-token kernel only): last term, sum_y = bf16(fp32 y + this term)
+    void *sum_y;                  // set per call with out_mode 3
 };
 
 // thread-local error string

@@ -57,10 +57,12 @@ struct TxArgs {
     int env_dtype, l;
     const void *in;           // stage B: bf16 x [cols]; stage A: fp32 z [cols]
     void *out;                // stage B: fp32 z [rows]; stage A: bf16 y [rows]
+    void *out_final;          // stage A, mode 4: bf16 y [rows] that receives round(out[] + this term)
     int npairs_total;         // pairs of K blocks along the reduction
     int pairs_per_cta;        // pairs per cluster rank
     int nastages, nsstages, tmem_cols;
-    int stage_a;              // 0: stage B (bf16 in, fp32 out); stage A (fp32 in): 1 bf16 out, 2 fp32 out, 3 added to fp32 out
+    int stage_a;              // 0: stage B (bf16 in, fp32 out); stage A (fp32 in): 1 bf16 out, 2 fp32 out, 3 added to fp32 out,
+                              // 4 last term of a sum: out_final = bf16(fp32 out + this term)
     int32_t *status;
 };
 
@@ -85,7 +87,7 @@ __device__ __forceinline__ bool tx_wait(uint32_t bar, uint32_t parity, volatile 
 //   sring [nsstages][2048 B]           packed sign words of a pair: [2][128 rows] uint2
 //   xp    [pairs_per_cta * 64] u32     activation pairs in MMA k order (bf16x2)
 //   part  [8][128] float               partial outputs pushed by the other cluster ranks (rank 0 only reads)
-template <int LP, int TX_GROUPS>
+template <int LP, int TX_GROUPS, bool SUM_LAST = false>
 __device__ __forceinline__ void tmem_t1_body(const TxArgs &a, const int rb) {
     using namespace tm;
     constexpr int TX_EXPANDERS = TX_GROUPS * 128;
@@ -365,6 +367,8 @@ __device__ __forceinline__ void tmem_t1_body(const TxArgs &a, const int rb) {
         if (grow < a.rows && !*abort_flag) {
             if (a.stage_a == 1) reinterpret_cast<__nv_bfloat16 *>(a.out)[grow] = __float2bfloat16_rn(outv);
             else if (a.stage_a == 3) reinterpret_cast<float *>(a.out)[grow] += outv;      // a further term of a sum of layers
+            else if (SUM_LAST && a.stage_a == 4)                                           // its last term: one rounding of the whole sum
+                reinterpret_cast<__nv_bfloat16 *>(a.out_final)[grow] = __float2bfloat16_rn(reinterpret_cast<const float *>(a.out)[grow] + outv);
             else reinterpret_cast<float *>(a.out)[grow] = outv;
         }
     }
@@ -375,6 +379,13 @@ __device__ __forceinline__ void tmem_t1_body(const TxArgs &a, const int rb) {
 template <int LP, int G>
 __global__ void __launch_bounds__(tx_threads(G), 1) tmem_t1_kernel(const TxArgs a) {
     tmem_t1_body<LP, G>(a, (int)blockIdx.x + a.rb0);
+}
+
+// The last term of a sum of layers (mode 4 of the epilogue), an instantiation of its own so that the plain kernel
+// carries no trace of it.
+template <int LP, int G>
+__global__ void __launch_bounds__(tx_threads(G), 1) tmem_t1_sumlast_kernel(const TxArgs a) {
+    tmem_t1_body<LP, G, true>(a, (int)blockIdx.x + a.rb0);
 }
 
 // Several sibling layers per launch: each CTA picks its layer by its position in the grid.
@@ -510,6 +521,7 @@ static mdbf_status_t launch_t1g(const TxMulti &m, const TxPlan &p, cudaStream_t 
     if (!attr_set) {
         MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_kernel<LP, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
         MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_multi_kernel<LP, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_sumlast_kernel<LP, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
         attr_set = true;
     }
     cudaLaunchConfig_t cfg = {};
@@ -526,7 +538,8 @@ static mdbf_status_t launch_t1g(const TxMulti &m, const TxPlan &p, cudaStream_t 
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (m.nlayers == 1) MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_kernel<LP, G>, m.layer[0]));
+    if (m.nlayers == 1 && m.layer[0].stage_a == 4) MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_sumlast_kernel<LP, G>, m.layer[0]));
+    else if (m.nlayers == 1) MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_kernel<LP, G>, m.layer[0]));
     else MDBF_CUDA(cudaLaunchKernelEx(&cfg, tmem_t1_multi_kernel<LP, G>, m));
     ++g_t1_launches;
     return MDBF_OK;
@@ -612,7 +625,7 @@ static mdbf_status_t run_t1(Layer *const *Ls, int n, const void *x, void *const 
         TxArgs &s = ma.layer[i];
         s.wk2 = L.wk2A; s.kb_pad = L.kbpA; s.rows = d.d_out; s.cols = d.k;
         s.vtile = L.vxA; s.U = L.UA; s.env_dtype = d.env_dtype; s.l = d.l;
-        s.in = L.zsum; s.out = ys[i]; s.stage_a = 1 + L.out_mode;
+        s.in = L.zsum; s.out = ys[i]; s.out_final = L.sum_y; s.stage_a = 1 + L.out_mode;
         s.npairs_total = L.kbpA / 2; s.pairs_per_cta = pa.pairs_per_cta[i];
         s.nastages = pa.nastages; s.nsstages = pa.nsstages; s.tmem_cols = pa.tmem_cols; s.status = L.status;
         ma.rb_start[i + 1] = ma.rb_start[i] + ceil_div(d.d_out, 128);

@@ -450,10 +450,19 @@ mdbf_status_t mdbf_linear_forward_sum(const mdbf_handle_t *terms, int32_t P, con
             if (terms[q] == terms[p]) { set_error("mdbf_linear_forward_sum: term %d repeats term %d", p, q); return MDBF_ERR_INVALID_ARG; }
     }
     cudaStream_t st = (cudaStream_t)stream;
-    for (int p = 0; p < P; ++p) {            // term 0 stores its fp32 output into acc, the others add to it (stream order)
-        mdbf_status_t rc = forward_impl(terms[p], x, acc, T, act_dtype, st, p == 0 ? 1 : 2);
+    // term 0 stores its fp32 output into acc, the others add to it (stream order).  When the last term runs the
+    // one-token kernel, its epilogue adds and rounds into y itself; otherwise a cast pass follows.
+    Layer &last = terms[P - 1]->L;
+    const bool fused_cast = P >= 2 && T == 1 && act_dtype == MDBF_BF16 && last.d.env_dtype != MDBF_F32 && last.d.l <= 32 &&
+                            (terms[P - 1]->kernel == MDBF_KERNEL_AUTO || terms[P - 1]->kernel == MDBF_KERNEL_TMEM) &&
+                            tmem_path_supports(last, 1);
+    for (int p = 0; p < P; ++p) {
+        int mode = p == 0 ? 1 : 2;
+        if (fused_cast && p == P - 1) { mode = 3; last.sum_y = y; }
+        mdbf_status_t rc = forward_impl(terms[p], x, acc, T, act_dtype, st, mode);
         if (rc) return rc;
     }
+    if (fused_cast) return MDBF_OK;
     return launch_cast(acc, y, (size_t)T * terms[0]->L.d.d_out, act_dtype, st);
 }
 
