@@ -153,7 +153,10 @@ mdbf_status_t mdbf_linear_forward(mdbf_handle_t h, const void *x, void *y, int32
  * form (Eq. dbf-residual-comp: a DBF term plus a DBF term fitted to the residual, (l, P) = (1, 2);
  * the paper's (l, P) sweep uses the same sum with MDBF terms).  Every term is evaluated by the same
  * kernels as mdbf_linear_forward with an fp32 output: term 1 stores into `acc`, the others add to
- * it, and one pass rounds `acc` to y - so y carries a single rounding whatever P is.
+ * it, and one pass rounds `acc` to y - so y carries a single rounding whatever P is.  With one
+ * token, bf16 activations and at most four terms of one envelope-rank bucket, the first stage of
+ * all terms shares a launch and the last term's epilogue does the final add and rounding
+ * (P + 1 launches instead of 2P + 1, same result).
  *   terms  P handles of equal d_out and d_in (k, l and env_dtype may differ), all distinct
  *   x, y   device, T x d_in read, T x d_out written, of act_dtype
  *   acc    device, T x d_out float32 scratch owned by the caller, overwritten

@@ -76,9 +76,7 @@ struct Layer {
     void *xstage, *ystage;        // device staging for the host-buffer entry point
     int32_t *status;              // device status word
     int last_ksplit;              // how many partials the last forward wrote (0 = zsum valid, -1 = the intermediate is in zb)
-    int out_mode;                 // set per call: 0 y in the activation type; 1 / 2: fp32 y stored / added (a term of a sum);
-                                  // 3 (one-token kernel only): last term, sum_y = bf16(fp32 y + this term)
-    void *sum_y;                  // set per call with out_mode 3
+    int out_mode;                 // set per call: 0 y in the activation type; 1 / 2: fp32 y stored / added (a term of a sum)
 };
 
 // thread-local error string
@@ -145,6 +143,7 @@ mdbf_status_t launch_vperm(const void *V, int cols, int l, int env_dtype, uint16
 mdbf_status_t launch_forward_tmem_t1(Layer &L, const void *x, void *y, cudaStream_t st);
 constexpr int kMaxSiblings = 4;   // layers one launch of the one-token kernel can serve
 int last_t1_launch_count();
+mdbf_status_t launch_forward_tmem_t1_sum(Layer *const *Ls, int n, const void *x, float *acc, void *y, cudaStream_t st);
 mdbf_status_t launch_forward_tmem_t1_multi(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st);
 mdbf_status_t launch_wk2(const uint32_t *canon, int rows, int nwords, uint2 *out, int rblocks, int kb_pad,
                          cudaStream_t st);

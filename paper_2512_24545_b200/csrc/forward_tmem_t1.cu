@@ -597,8 +597,12 @@ static mdbf_status_t launch_stage(const TxMulti &full, const TxPlan &p, const in
 }
 
 // Both stages of n layers that read the same x (n = 1: a single layer): one launch per stage.
+// sum != nullptr: the n layers are the terms of a sum; stage B of all terms shares one launch (they read the
+// same x), the stage-A launches follow one another: term 0 stores its fp32 output into sum_acc, the middle
+// terms add to it, the last one adds and rounds into sum_y.
 template <int LP>
-static mdbf_status_t run_t1(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st) {
+static mdbf_status_t run_t1(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st,
+                            float *sum_acc = nullptr, void *sum_y = nullptr) {
     int rowsB[TX_MAX_LAYERS], kbB[TX_MAX_LAYERS], rowsA[TX_MAX_LAYERS], kbA[TX_MAX_LAYERS];
     for (int i = 0; i < n; ++i) {
         rowsB[i] = Ls[i]->d.k; kbB[i] = Ls[i]->kbpB;
@@ -625,14 +629,34 @@ static mdbf_status_t run_t1(Layer *const *Ls, int n, const void *x, void *const 
         TxArgs &s = ma.layer[i];
         s.wk2 = L.wk2A; s.kb_pad = L.kbpA; s.rows = d.d_out; s.cols = d.k;
         s.vtile = L.vxA; s.U = L.UA; s.env_dtype = d.env_dtype; s.l = d.l;
-        s.in = L.zsum; s.out = ys[i]; s.out_final = L.sum_y; s.stage_a = 1 + L.out_mode;
+        s.in = L.zsum; s.out = ys[i]; s.out_final = nullptr; s.stage_a = 1 + L.out_mode;
         s.npairs_total = L.kbpA / 2; s.pairs_per_cta = pa.pairs_per_cta[i];
         s.nastages = pa.nastages; s.nsstages = pa.nsstages; s.tmem_cols = pa.tmem_cols; s.status = L.status;
         ma.rb_start[i + 1] = ma.rb_start[i] + ceil_div(d.d_out, 128);
     }
     mdbf_status_t rc = launch_stage<LP>(mb, pb, kbB, st);
     if (rc) return rc;
-    return launch_stage<LP>(ma, pa, kbA, st);
+    if (!sum_acc) return launch_stage<LP>(ma, pa, kbA, st);
+    for (int i = 0; i < n; ++i) {
+        TxMulti one = {};
+        one.nlayers = 1;
+        one.rb_start[1] = ceil_div(rowsA[i], 128);
+        TxPlan p1;
+        if (!plan_t1(1, &rowsA[i], &kbA[i], LP, &p1)) {
+            set_error("mdbf_linear_forward_sum: the one-token TMEM kernel does not fit this shape");
+            return MDBF_ERR_SHAPE;
+        }
+        TxArgs &s = one.layer[0];
+        s = ma.layer[i];
+        s.out = n == 1 ? sum_y : (void *)sum_acc;
+        s.out_final = sum_y;
+        s.stage_a = n == 1 ? 1 : i == 0 ? 2 : i == n - 1 ? 4 : 3;
+        s.pairs_per_cta = p1.pairs_per_cta[0];
+        s.nastages = p1.nastages; s.nsstages = p1.nsstages; s.tmem_cols = p1.tmem_cols;
+        rc = launch_stage<LP>(one, p1, &kbA[i], st);
+        if (rc) return rc;
+    }
+    return MDBF_OK;
 }
 
 // n <= TX_MAX_LAYERS layers with the same LP, all prepared for the one-token kernel.
@@ -646,6 +670,22 @@ mdbf_status_t launch_forward_tmem_t1_multi(Layer *const *Ls, int n, const void *
         case 32: return run_t1<32>(Ls, n, x, ys, st);
         default:
             set_error("mdbf_linear_forward: the one-token TMEM kernel handles l <= 32 (got %d)", Ls[0]->d.l);
+            return MDBF_ERR_SHAPE;
+    }
+}
+
+// The terms of a sum of layers (same LP, at most TX_MAX_LAYERS) at one token: y = bf16(sum of the terms' outputs).
+mdbf_status_t launch_forward_tmem_t1_sum(Layer *const *Ls, int n, const void *x, float *acc, void *y, cudaStream_t st) {
+    void *ys[TX_MAX_LAYERS] = {};
+    switch (Ls[0]->LP) {
+        case 1: return run_t1<1>(Ls, n, x, ys, st, acc, y);
+        case 2: return run_t1<2>(Ls, n, x, ys, st, acc, y);
+        case 4: return run_t1<4>(Ls, n, x, ys, st, acc, y);
+        case 8: return run_t1<8>(Ls, n, x, ys, st, acc, y);
+        case 16: return run_t1<16>(Ls, n, x, ys, st, acc, y);
+        case 32: return run_t1<32>(Ls, n, x, ys, st, acc, y);
+        default:
+            set_error("mdbf_linear_forward_sum: the one-token TMEM kernel handles l <= 32 (got %d)", Ls[0]->d.l);
             return MDBF_ERR_SHAPE;
     }
 }

@@ -450,19 +450,34 @@ mdbf_status_t mdbf_linear_forward_sum(const mdbf_handle_t *terms, int32_t P, con
             if (terms[q] == terms[p]) { set_error("mdbf_linear_forward_sum: term %d repeats term %d", p, q); return MDBF_ERR_INVALID_ARG; }
     }
     cudaStream_t st = (cudaStream_t)stream;
-    // term 0 stores its fp32 output into acc, the others add to it (stream order).  When the last term runs the
-    // one-token kernel, its epilogue adds and rounds into y itself; otherwise a cast pass follows.
-    Layer &last = terms[P - 1]->L;
-    const bool fused_cast = P >= 2 && T == 1 && act_dtype == MDBF_BF16 && last.d.env_dtype != MDBF_F32 && last.d.l <= 32 &&
-                            (terms[P - 1]->kernel == MDBF_KERNEL_AUTO || terms[P - 1]->kernel == MDBF_KERNEL_TMEM) &&
-                            tmem_path_supports(last, 1);
+    // One token, bf16, every term ready for the one-token kernel with the same envelope-rank bucket: stage B of
+    // all terms shares a launch, the last term's stage-A epilogue adds the fp32 sum of the others and rounds
+    // into y (P + 1 launches, no cast pass).
+    bool fused = T == 1 && act_dtype == MDBF_BF16 && P <= kMaxSiblings;
+    for (int p = 0; p < P && fused; ++p) {
+        const Layer &L = terms[p]->L;
+        fused = L.d.env_dtype != MDBF_F32 && L.d.l <= 32 && L.vxA && L.vxB && L.LP == terms[0]->L.LP &&
+                terms[p]->kernel == MDBF_KERNEL_AUTO && tmem_path_supports(L, 1);
+    }
+    if (fused) {
+        Layer *Ls[kMaxSiblings];
+        for (int p = 0; p < P; ++p) {
+            Ls[p] = &terms[p]->L;
+            Ls[p]->out_mode = 0;
+            Ls[p]->last_ksplit = 0;
+            terms[p]->last_kernel = MDBF_KERNEL_TMEM;
+            terms[p]->last_launches = 0;
+        }
+        mdbf_status_t rc = launch_forward_tmem_t1_sum(Ls, P, x, acc, y, st);
+        if (rc) return rc;
+        terms[0]->last_launches = last_t1_launch_count();
+        return MDBF_OK;
+    }
+    // otherwise: term 0 stores its fp32 output into acc, the others add to it (stream order), a cast pass follows
     for (int p = 0; p < P; ++p) {
-        int mode = p == 0 ? 1 : 2;
-        if (fused_cast && p == P - 1) { mode = 3; last.sum_y = y; }
-        mdbf_status_t rc = forward_impl(terms[p], x, acc, T, act_dtype, st, mode);
+        mdbf_status_t rc = forward_impl(terms[p], x, acc, T, act_dtype, st, p == 0 ? 1 : 2);
         if (rc) return rc;
     }
-    if (fused_cast) return MDBF_OK;
     return launch_cast(acc, y, (size_t)T * terms[0]->L.d.d_out, act_dtype, st);
 }
 
