@@ -65,6 +65,19 @@ def test_three_mdbf_terms_of_different_rank(T):
     assert rel_err(y, ref) <= rel_err(sum(singles), ref) + 1e-4
 
 
+@pytest.mark.parametrize("P", [1, 3, 4, 5])
+def test_terms_of_one_envelope_rank_at_one_token(P):
+    """Up to four terms of one envelope-rank bucket share the first-stage launch and the last term rounds the
+    sum into y (store, add, ..., add-and-round); five terms take the term-by-term path with a cast pass."""
+    specs = term_specs(300, 1000, [257, 200, 130, 64, 40][:P], [8] * P)
+    x = inputs.make_activations(specs[0], 1)
+    y, ref, singles = run_sum(specs, x)
+    assert np.all(np.isfinite(y))
+    assert rel_err(y, ref) <= TOL["bf16"]
+    if P == 1:
+        np.testing.assert_array_equal(y, singles[0])
+
+
 def test_fp32_terms_and_single_term():
     t = inputs.tiny()
     specs = [inputs.scaled(t, name="a", seed=1), inputs.scaled(t, name="b", seed=2, env_std=t.env_std * 0.5)]
