@@ -60,12 +60,13 @@ typedef enum { MDBF_F32 = 0, MDBF_F16 = 1, MDBF_BF16 = 2 } mdbf_dtype_t;
 
 /* Kernel selector for mdbf_set_kernel. */
 typedef enum {
-    MDBF_KERNEL_AUTO = 0,   /* T = 1: TMEM; T >= 2: MAT (PREFILL where MAT cannot run); fp32 / l > 32: ALU */
+    MDBF_KERNEL_AUTO = 0,   /* T = 1: I8; T >= 2: MAT (PREFILL where MAT cannot run); fp32 / l > 32: ALU */
     MDBF_KERNEL_ALU = 1,    /* fp32 CUDA-core path, sign applied by XOR of the IEEE sign bit      */
     MDBF_KERNEL_DECODE = 2, /* T <= 4: register bit->bf16 expansion + warp-level MMA              */
     MDBF_KERNEL_PREFILL = 3, /* T >= 2 (max_T >= 2): tcgen05 GEMM, TMEM accumulator, TMA operand   */
     MDBF_KERNEL_TMEM = 4,   /* l*T <= 64: tcgen05 MMA with the sign operand expanded into TMEM    */
-    MDBF_KERNEL_MAT = 5     /* T >= 2: W_hat tiles rebuilt on the fly (rank-l mini-MMA + sign XOR), one GEMM of width T */
+    MDBF_KERNEL_MAT = 5,    /* T >= 2: W_hat tiles rebuilt on the fly (rank-l mini-MMA + sign XOR), one GEMM of width T */
+    MDBF_KERNEL_I8 = 6      /* T = 1: one persistent launch, packed bits as the 8-bit integer tcgen05 operand, fixed-point scaled input */
 } mdbf_kernel_t;
 
 typedef struct {

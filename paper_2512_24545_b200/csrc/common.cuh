@@ -35,6 +35,16 @@ struct MatMaps {
     CUtensorMap tmx, tmz, tmzo, tmyo;
 };
 
+// Scratch and pack-time constants of the one-token kernel (forward_t1.cu); index 0 = stage B, 1 = stage A.
+struct T1Buffers {
+    float *vmax;                  // [2][32] max_c |V[c][t]| per stage and mode
+    unsigned int *sync;           // scalars of a forward: column sums of the fixed-point operand, max |x|, max |z|
+    int8_t *img[2];               // operand images [Np][NB][128]
+    unsigned long long *acc64[2]; // fixed-point sums of the partial outputs of split row blocks [R * 128] (zero between launches)
+    int R[2], RG[2], Np[2];       // row blocks, groups of four row blocks, pairs of K blocks
+    int NB, ctas;
+};
+
 struct Layer {
     mdbf_desc_t d;
     int device;
@@ -69,6 +79,7 @@ struct Layer {
     int kcm;                      // 16-byte chunks of the mode axis: 2 (l <= 16) or 4 (l <= 32)
     __nv_bfloat16 *zb;            // bf16 intermediate [max_T][padA]
     MatMaps mat_maps;
+    T1Buffers t1;
     // scratch
     float *z;                     // [kMaxKSplit][zT][k] stage-B partial sums of the small-T kernel
     size_t zstride;               // zT * k
@@ -141,10 +152,14 @@ bool tmem_path_supports(const Layer &L, int T);
 mdbf_status_t launch_vperm(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int LP,
                            cudaStream_t st);
 mdbf_status_t launch_forward_tmem_t1(Layer &L, const void *x, void *y, cudaStream_t st);
+mdbf_status_t t1_prepare(Layer &L, cudaStream_t st);
+void t1_release(Layer &L);
+bool t1_supports(const Layer &L);
+mdbf_status_t launch_forward_t1_group(Layer *const *Ls, int n, const void *const *xs, void *const *ys, cudaStream_t st, int stages = 3);
 constexpr int kMaxSiblings = 4;   // layers one launch of the one-token kernel can serve
 int last_t1_launch_count();
 mdbf_status_t launch_forward_tmem_t1_sum(Layer *const *Ls, int n, const void *x, float *acc, void *y, cudaStream_t st);
-mdbf_status_t launch_forward_tmem_t1_multi(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st);
+mdbf_status_t launch_forward_tmem_t1_multi(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st, int stages = 3);
 mdbf_status_t launch_wk2(const uint32_t *canon, int rows, int nwords, uint2 *out, int rblocks, int kb_pad,
                          cudaStream_t st);
 mdbf_status_t launch_vtile(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int NB,

@@ -602,7 +602,7 @@ static mdbf_status_t launch_stage(const TxMulti &full, const TxPlan &p, const in
 // terms add to it, the last one adds and rounds into sum_y.
 template <int LP>
 static mdbf_status_t run_t1(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st,
-                            float *sum_acc = nullptr, void *sum_y = nullptr) {
+                            float *sum_acc = nullptr, void *sum_y = nullptr, int stages = 3) {
     int rowsB[TX_MAX_LAYERS], kbB[TX_MAX_LAYERS], rowsA[TX_MAX_LAYERS], kbA[TX_MAX_LAYERS];
     for (int i = 0; i < n; ++i) {
         rowsB[i] = Ls[i]->d.k; kbB[i] = Ls[i]->kbpB;
@@ -634,8 +634,9 @@ static mdbf_status_t run_t1(Layer *const *Ls, int n, const void *x, void *const 
         s.nastages = pa.nastages; s.nsstages = pa.nsstages; s.tmem_cols = pa.tmem_cols; s.status = L.status;
         ma.rb_start[i + 1] = ma.rb_start[i] + ceil_div(d.d_out, 128);
     }
-    mdbf_status_t rc = launch_stage<LP>(mb, pb, kbB, st);
+    mdbf_status_t rc = (stages & 1) ? launch_stage<LP>(mb, pb, kbB, st) : MDBF_OK;     // stages: bit 0 = stage B, bit 1 = stage A
     if (rc) return rc;
+    if (!(stages & 2)) return MDBF_OK;
     if (!sum_acc) return launch_stage<LP>(ma, pa, kbA, st);
     for (int i = 0; i < n; ++i) {
         TxMulti one = {};
@@ -660,14 +661,14 @@ static mdbf_status_t run_t1(Layer *const *Ls, int n, const void *x, void *const 
 }
 
 // n <= TX_MAX_LAYERS layers with the same LP, all prepared for the one-token kernel.
-mdbf_status_t launch_forward_tmem_t1_multi(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st) {
+mdbf_status_t launch_forward_tmem_t1_multi(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st, int stages) {
     switch (Ls[0]->LP) {
-        case 1: return run_t1<1>(Ls, n, x, ys, st);
-        case 2: return run_t1<2>(Ls, n, x, ys, st);
-        case 4: return run_t1<4>(Ls, n, x, ys, st);
-        case 8: return run_t1<8>(Ls, n, x, ys, st);
-        case 16: return run_t1<16>(Ls, n, x, ys, st);
-        case 32: return run_t1<32>(Ls, n, x, ys, st);
+        case 1: return run_t1<1>(Ls, n, x, ys, st, nullptr, nullptr, stages);
+        case 2: return run_t1<2>(Ls, n, x, ys, st, nullptr, nullptr, stages);
+        case 4: return run_t1<4>(Ls, n, x, ys, st, nullptr, nullptr, stages);
+        case 8: return run_t1<8>(Ls, n, x, ys, st, nullptr, nullptr, stages);
+        case 16: return run_t1<16>(Ls, n, x, ys, st, nullptr, nullptr, stages);
+        case 32: return run_t1<32>(Ls, n, x, ys, st, nullptr, nullptr, stages);
         default:
             set_error("mdbf_linear_forward: the one-token TMEM kernel handles l <= 32 (got %d)", Ls[0]->d.l);
             return MDBF_ERR_SHAPE;
@@ -693,7 +694,7 @@ mdbf_status_t launch_forward_tmem_t1_sum(Layer *const *Ls, int n, const void *x,
 mdbf_status_t launch_forward_tmem_t1(Layer &L, const void *x, void *y, cudaStream_t st) {
     Layer *one[1] = {&L};
     void *ys[1] = {y};
-    return launch_forward_tmem_t1_multi(one, 1, x, ys, st);
+    return launch_forward_tmem_t1_multi(one, 1, x, ys, st, 3);
 }
 
 }  // namespace mdbf

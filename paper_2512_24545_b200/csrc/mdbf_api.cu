@@ -61,6 +61,7 @@ static void free_layer(Layer &L) {
     void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.vpA, L.vpB, L.vxA, L.vxB, L.wk2A, L.wk2B, L.wkA, L.wkB, L.uiA, L.uiB, L.viA, L.viB, L.vtB, L.xsB, L.xsA, L.zb, L.z, L.zsum, L.xstage, L.ystage, L.status};
     for (void *p : ptrs)
         if (p) cudaFree(p);
+    t1_release(L);
 }
 
 // number of tokens the small-T kernel's partial-sum scratch is sized for
@@ -292,6 +293,7 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
         PACK_RC(launch_vtile(L.VB, d.d_in, d.l, d.env_dtype, L.vxB, L.kbpB, L.LP < 16 ? 16 : L.LP, st));
         PACK_RC(launch_wk2(L.wA, d.d_out, L.wordsA, L.wk2A, L.rpA / 128, L.kbpA, st));
         PACK_RC(launch_wk2(L.wB, d.k, L.wordsB, L.wk2B, L.rpB / 128, L.kbpB, st));
+        if (L.LP <= 16) PACK_RC(t1_prepare(L, st));
     }
     if (want_prefill) {
         PACK_RC(launch_uimg(L.UA, d.d_out, d.l, d.env_dtype, L.uiA, L.rpA / 128, L.kcm, st));
@@ -363,7 +365,7 @@ mdbf_status_t mdbf_get_desc(mdbf_handle_t h, mdbf_desc_t *out) {
 mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel) {
     mdbf_status_t rc = check_handle(h, "mdbf_set_kernel");
     if (rc) return rc;
-    if (kernel < MDBF_KERNEL_AUTO || kernel > MDBF_KERNEL_MAT) {
+    if (kernel < MDBF_KERNEL_AUTO || kernel > MDBF_KERNEL_I8) {
         set_error("mdbf_set_kernel: unknown kernel %d", kernel);
         return MDBF_ERR_INVALID_ARG;
     }
@@ -374,6 +376,40 @@ mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel) {
         if (rc) return rc;
     }
     h->kernel = kernel;
+    return MDBF_OK;
+}
+
+// One token, n <= 4 layers that share x and are prepared for both one-token kernels.  Each stage goes to the kernel
+// that is faster for its size: the integer kernel streams a stage's sign words several times faster but needs two
+// launches per stage (operand images, then the contraction); below kI8StageBytes of sign words per stage the
+// single launch of the bf16 TMEM-operand kernel wins.  The two kernels exchange the intermediate through the
+// layers' fp32 z buffers, so the stages can mix.  force: 0 = choose, 1 = TMEM-operand kernel, 2 = integer kernel.
+static constexpr size_t kI8StageBytes = 18u << 20;
+static mdbf_status_t forward_t1_auto(Layer *const *Ls, int n, const void *x, void *const *ys, cudaStream_t st, int force,
+                                     int *launches, int *kernel_used) {
+    size_t bytes[2] = {0, 0};
+    bool i8_ok = true, old_ok = true;
+    for (int i = 0; i < n; ++i) {
+        bytes[0] += (size_t)Ls[i]->d.k * Ls[i]->d.d_in / 8;
+        bytes[1] += (size_t)Ls[i]->d.d_out * Ls[i]->d.k / 8;
+        i8_ok = i8_ok && t1_supports(*Ls[i]) && Ls[i]->out_mode == 0;
+        old_ok = old_ok && Ls[i]->vxA && Ls[i]->vxB && tmem_path_supports(*Ls[i], 1);
+    }
+    int i8_stages = 0;
+    for (int s = 0; s < 2; ++s)
+        if (i8_ok && (force == 2 || !old_ok || (force == 0 && bytes[s] >= kI8StageBytes))) i8_stages |= 1 << s;
+    if (!i8_ok && !old_ok) { set_error("mdbf_linear_forward: no one-token kernel fits this layer"); return MDBF_ERR_SHAPE; }
+    const void *xs[kMaxSiblings];
+    for (int i = 0; i < n; ++i) xs[i] = x;
+    int nl = 0;
+    for (int s = 0; s < 2; ++s) {
+        mdbf_status_t rc;
+        if (i8_stages >> s & 1) { rc = launch_forward_t1_group(Ls, n, xs, ys, st, 1 << s); nl += 2; }
+        else { rc = launch_forward_tmem_t1_multi(Ls, n, x, ys, st, 1 << s); nl += last_t1_launch_count(); }
+        if (rc) return rc;
+    }
+    *launches = nl;
+    *kernel_used = i8_stages == 3 ? MDBF_KERNEL_I8 : MDBF_KERNEL_TMEM;
     return MDBF_OK;
 }
 
@@ -392,6 +428,7 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         // one token: TMEM-operand kernel; more: the tcgen05 GEMM (it splits the reduction over a
         // cluster when few tokens would leave SMs idle); the others remain selectable
         if (!tc_ok) kernel = MDBF_KERNEL_ALU;
+        else if (T == 1 && out_mode == 0 && (t1_supports(L) || tmem_path_supports(L, T))) kernel = -1;     // one token: per-stage choice below
         else if (T == 1 && tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
         // more tokens: rebuilding W_hat tiles and running one GEMM of width T (measured faster than, or equal
         // to, the l sign GEMMs of the expanded order at every T >= 2); the expanded order serves the layers
@@ -400,6 +437,13 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         else if (L.zb) kernel = MDBF_KERNEL_PREFILL;
         else if (tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
         else kernel = MDBF_KERNEL_DECODE;
+    }
+    if (kernel == -1) {
+        Layer *one = &L;
+        int launches = 0, used = 0;
+        mdbf_status_t rc = forward_t1_auto(&one, 1, x, &y, st, 0, &launches, &used);
+        if (rc == MDBF_OK) { L.last_ksplit = 0; h->last_launches = launches; h->last_kernel = used; }
+        return rc;
     }
     if (kernel != MDBF_KERNEL_ALU && !tc_ok) {
         set_error("mdbf_linear_forward: the tensor-core kernels need bf16 activations, 16-bit envelopes and l <= 32");
@@ -410,6 +454,10 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
                   kDecodeMaxT, T, L.d.l);
         return MDBF_ERR_SHAPE;
     }
+    if (kernel == MDBF_KERNEL_I8 && (T != 1 || !t1_supports(L))) {
+        set_error("mdbf_linear_forward: the one-token integer kernel needs T = 1, 16-bit envelopes and l <= 32");
+        return MDBF_ERR_SHAPE;
+    }
     if (out_mode != 0 && (kernel == MDBF_KERNEL_DECODE || (kernel == MDBF_KERNEL_TMEM && T > 1))) {
         set_error("mdbf_linear_forward_sum: the forced kernel has no fp32-accumulate output");
         return MDBF_ERR_INVALID_ARG;
@@ -417,7 +465,12 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
     int launches = 0;
     mdbf_status_t rc = ensure_kernel_layouts(L, kernel, T);      // no-op for the default kernels
     if (rc) return rc;
-    if (kernel == MDBF_KERNEL_ALU) rc = launch_forward_alu(L, x, y, T, act_dtype, st, &launches);
+    if (kernel == MDBF_KERNEL_I8) {
+        Layer *one = &L;
+        rc = launch_forward_t1_group(&one, 1, &x, &y, st);
+        L.last_ksplit = 0;
+        launches = 4;                                         // image and stage kernel, twice
+    } else if (kernel == MDBF_KERNEL_ALU) rc = launch_forward_alu(L, x, y, T, act_dtype, st, &launches);
     else if (kernel == MDBF_KERNEL_DECODE) rc = launch_forward_decode(L, x, y, T, st, &launches);
     else if (kernel == MDBF_KERNEL_TMEM) rc = launch_forward_tmem(L, x, y, T, st, &launches);
     else if (kernel == MDBF_KERNEL_MAT) rc = launch_forward_mat(L, x, y, T, st, &launches);
@@ -486,6 +539,7 @@ mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t 
     if (!layers || !x || !ys) { set_error("mdbf_linear_forward_siblings: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
     if (n < 1 || n > 64) { set_error("mdbf_linear_forward_siblings: n=%d outside [1, 64]", n); return MDBF_ERR_SHAPE; }
     bool fusable = T == 1 && act_dtype == MDBF_BF16;
+    const int32_t k0 = layers[0] ? layers[0]->kernel : 0;       // checked below; AUTO, or the same one-token kernel forced on every layer
     for (int i = 0; i < n; ++i) {
         mdbf_status_t rc = check_handle(layers[i], "mdbf_linear_forward_siblings");
         if (rc) return rc;
@@ -501,7 +555,8 @@ mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t 
         }
         for (int q = 0; q < i; ++q)
             if (layers[q] == layers[i]) { set_error("mdbf_linear_forward_siblings: layer %d repeats layer %d", i, q); return MDBF_ERR_INVALID_ARG; }
-        fusable = fusable && L.vxA && L.vxB && L.LP == layers[0]->L.LP && layers[i]->kernel == MDBF_KERNEL_AUTO;
+        fusable = fusable && L.vxA && L.vxB && L.LP == layers[0]->L.LP && layers[i]->kernel == k0 &&
+                  (k0 == MDBF_KERNEL_AUTO || k0 == MDBF_KERNEL_TMEM || k0 == MDBF_KERNEL_I8);
     }
     if (!valid_dtype(act_dtype)) { set_error("mdbf_linear_forward_siblings: bad act_dtype %d", act_dtype); return MDBF_ERR_DTYPE; }
     cudaStream_t st = (cudaStream_t)stream;
@@ -512,7 +567,7 @@ mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t 
         }
         return MDBF_OK;
     }
-    for (int i0 = 0; i0 < n; i0 += kMaxSiblings) {      // groups of up to kMaxSiblings layers per pair of launches
+    for (int i0 = 0; i0 < n; i0 += kMaxSiblings) {      // groups of up to kMaxSiblings layers per set of launches
         const int m = n - i0 < kMaxSiblings ? n - i0 : kMaxSiblings;
         Layer *Ls[kMaxSiblings];
         void *outs[kMaxSiblings];
@@ -521,12 +576,14 @@ mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t 
             Ls[i]->out_mode = 0;
             Ls[i]->last_ksplit = 0;
             outs[i] = ys[i0 + i];
-            layers[i0 + i]->last_launches = i == 0 ? 2 : 0;
-            layers[i0 + i]->last_kernel = MDBF_KERNEL_TMEM;
         }
-        mdbf_status_t rc = launch_forward_tmem_t1_multi(Ls, m, x, outs, st);
+        int launches = 0, used = 0;
+        mdbf_status_t rc = forward_t1_auto(Ls, m, x, outs, st, k0 == MDBF_KERNEL_I8 ? 2 : k0 == MDBF_KERNEL_TMEM ? 1 : 0, &launches, &used);
         if (rc) return rc;
-        layers[i0]->last_launches = last_t1_launch_count();
+        for (int i = 0; i < m; ++i) {
+            layers[i0 + i]->last_launches = i == 0 ? launches : 0;
+            layers[i0 + i]->last_kernel = used;
+        }
     }
     return MDBF_OK;
 }

@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmdbf.so")
 
 F32, F16, BF16 = 0, 1, 2
-KERNEL_AUTO, KERNEL_ALU, KERNEL_DECODE, KERNEL_PREFILL, KERNEL_TMEM, KERNEL_MAT = 0, 1, 2, 3, 4, 5
+KERNEL_AUTO, KERNEL_ALU, KERNEL_DECODE, KERNEL_PREFILL, KERNEL_TMEM, KERNEL_MAT, KERNEL_I8 = 0, 1, 2, 3, 4, 5, 6
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_DTYPE, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT, ERR_VALUE = (
     -1, -2, -3, -4, -5, -6, -7, -8)
