@@ -310,6 +310,8 @@ def run_mdbf(args):
 
     # end to end: host buffers through the C-ABI, copies inside the timed region
     e2e_steps = max(1, min(args.steps, 10))
+    for (h, *_r) in layers:
+        M.mdbf_prepare_host_staging(h)
     for _ in range(2):
         for (h, sp, _, _, xh, yh) in layers:
             M.mdbf_linear_forward_host(h, xh.data_ptr(), yh.data_ptr(), T, M.BF16, st)

@@ -60,11 +60,11 @@ typedef enum { MDBF_F32 = 0, MDBF_F16 = 1, MDBF_BF16 = 2 } mdbf_dtype_t;
 
 /* Kernel selector for mdbf_set_kernel. */
 typedef enum {
-    MDBF_KERNEL_AUTO = 0,   /* T = 1: I8; T >= 2: MAT (PREFILL where MAT cannot run); fp32 / l > 32: ALU */
+    MDBF_KERNEL_AUTO = 0,   /* T = 1: TMEM or I8 per stage, by size; T >= 2: MAT (PREFILL / ALU where MAT cannot run); fp32 / l > 32: ALU */
     MDBF_KERNEL_ALU = 1,    /* fp32 CUDA-core path, sign applied by XOR of the IEEE sign bit      */
-    MDBF_KERNEL_DECODE = 2, /* T <= 4: register bit->bf16 expansion + warp-level MMA              */
-    MDBF_KERNEL_PREFILL = 3, /* T >= 2 (max_T >= 2): tcgen05 GEMM, TMEM accumulator, TMA operand   */
-    MDBF_KERNEL_TMEM = 4,   /* l*T <= 64: tcgen05 MMA with the sign operand expanded into TMEM    */
+                            /* 2: retired (a warp-level MMA kernel for T <= 4)                     */
+    MDBF_KERNEL_PREFILL = 3, /* T >= 2 (max_T >= 2): expanded order, tcgen05 GEMM of width l*T, TMEM accumulator, TMA operand */
+    MDBF_KERNEL_TMEM = 4,   /* T = 1: tcgen05 MMA, sign (.) activation as bf16 operand in TMEM, one launch per stage */
     MDBF_KERNEL_MAT = 5,    /* T >= 2: W_hat tiles rebuilt on the fly (rank-l mini-MMA + sign XOR), one GEMM of width T */
     MDBF_KERNEL_I8 = 6      /* T = 1: one persistent launch, packed bits as the 8-bit integer tcgen05 operand, fixed-point scaled input */
 } mdbf_kernel_t;
@@ -105,10 +105,12 @@ mdbf_status_t mdbf_unpack_signs(const uint32_t *p, int64_t rows, int64_t cols, i
  *   (round-to-nearest-even) to desc->env_dtype — the rounded values are the
  *   layer and can be read back with mdbf_get_envelope.
  * inputs_on_device: 0 = all seven pointers are host memory, 1 = all device.
- * The handle owns device copies of the canonical words, of a kernel-private
- * tiled copy of them, of the envelopes, and scratch for the k x T
- * intermediate sized for max_T: one forward per handle may be in flight at a
- * time.  Synchronises `stream` before returning.
+ * The handle owns one device copy of the sign words (in the layout its kernels
+ * read; canonical words are produced on request by mdbf_get_packed), the
+ * envelopes with their operand layouts, and scratch for the k x T
+ * intermediate sized for max_T: about one bit per sign plus the envelopes.
+ * One forward per handle may be in flight at a time.  Synchronises `stream`
+ * before returning.
  * Errors: INVALID_ARG (NULL), SHAPE, DTYPE, VALUE (host inputs only), ALLOC,
  * CUDA, ARCH. */
 mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t *S_B,
@@ -129,8 +131,8 @@ mdbf_status_t mdbf_get_desc(mdbf_handle_t h, mdbf_desc_t *out);
 
 /* Force a kernel for later forwards on this handle (tests, benchmarks).  MDBF_KERNEL_PREFILL
  * allocates that kernel's scratch (max_T * l * (d_in + k) * 2 bytes of pre-scaled operands) on the
- * first request, which synchronises the device; a forward that falls back to it without this call
- * allocates on its first use, so make that first use outside stream capture. */
+ * first request, which synchronises the device; no forward ever does (a forward that is forced to
+ * that kernel on a handle without the scratch returns MDBF_ERR_INVALID_ARG). */
 mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel /* mdbf_kernel_t */);
 
 /* ---------------------------------------------------------------- forward
@@ -142,10 +144,18 @@ mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel /* mdbf_kernel_t *
  *   x  device, T x d_in  of act_dtype (token-contiguous), read only
  *   y  device, T x d_out of act_dtype, written (round-to-nearest-even)
  *   act_dtype  MDBF_BF16 or MDBF_F32 (MDBF_F16 is accepted by the ALU path)
- * Accumulation is fp32.  Asynchronous on `stream`; allocates nothing and does not synchronise,
- * except for the first forward of a handle that has to run the expanded order for T >= 2 without
- * a prior mdbf_set_kernel(PREFILL): layers with d_in % 8 != 0 get that scratch at pack time, so
- * this concerns only an x that is not 16-byte aligned.  x and y must not alias.
+ * Precision.  Accumulation is fp32 (one token, integer kernel: exact int32 sums of 21-bit fixed-point
+ * operands).  What is rounded to bf16 on the way, besides y itself: T >= 2, default order: every
+ * entry of the two rebuilt factors and the intermediate z (four roundings with y); T >= 2, expanded
+ * order: the pre-scaled x and z (three); one token, TMEM-operand kernel: V_B, z and V_A (four);
+ * one token, integer kernel: nothing (one).  fp16 envelopes are re-rounded to bf16 where they become
+ * bf16 MMA operands.  Measured against the fp64 definition: 1.6e-3 to 3.7e-3 relative Frobenius
+ * error on the 7B- and 70B-class shapes, bound 5e-3.
+ * Asynchronous on `stream`; never allocates and never synchronises.  With the library choosing the
+ * kernel, an x that the default kernels cannot take (T >= 2 and x not 16-byte aligned) is served
+ * by the expanded order if mdbf_set_kernel(PREFILL) has prepared its scratch on this handle, else
+ * by the CUDA-core kernel.  x and y must not alias; the current device must be the one the layer
+ * was packed on.
  * Errors: INVALID_ARG, SHAPE (T < 1 or T > max_T), DTYPE, CUDA. */
 mdbf_status_t mdbf_linear_forward(mdbf_handle_t h, const void *x, void *y, int32_t T,
                                   int32_t act_dtype, void *stream);
@@ -177,10 +187,14 @@ mdbf_status_t mdbf_linear_forward_sum(const mdbf_handle_t *terms, int32_t P, con
 mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t n, const void *x, void *const *ys,
                                            int32_t T, int32_t act_dtype, void *stream);
 
-/* Same computation with HOST buffers: copies x to a handle-owned device
- * staging buffer, runs the forward, copies y back, all on `stream`, and
- * synchronises the stream before returning.  x_host / y_host should be pinned
- * for full copy bandwidth. */
+/* Device staging buffers for mdbf_linear_forward_host (max_T * (d_in + d_out) * 4 bytes): allocated
+ * here, once, so that the host-buffer forward itself allocates nothing.  Errors: ALLOC, CUDA. */
+mdbf_status_t mdbf_prepare_host_staging(mdbf_handle_t h);
+
+/* Same computation with HOST buffers: copies x to the handle's device staging buffer, runs the
+ * forward, copies y back, all on `stream`, and synchronises the stream before returning.  x_host /
+ * y_host should be pinned for full copy bandwidth.  Needs mdbf_prepare_host_staging once per handle
+ * (MDBF_ERR_INVALID_ARG otherwise). */
 mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T,
                                        int32_t act_dtype, void *stream);
 
@@ -213,7 +227,10 @@ mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void
  * library routine.
  *
  * The first call on each device looks the array's device address up (with
- * that device current); make that first call outside any stream capture.
+ * that device current) and keeps it for the life of the process; make that
+ * first call outside any stream capture.  cudaDeviceReset() destroys the
+ * array with the context: do not call this function again on that device
+ * afterwards (the kept address would be stale).
  * Every call on a device shares the one array, which keeps whatever the
  * previous call left in it: each call overwrites all the entries it later
  * reads, so nothing has to be cleared, but two calls that overlap on the GPU

@@ -13,19 +13,6 @@ namespace mdbf {
 
 constexpr uint32_t kHandleMagic = 0x4D444246u;  // "MDBF"
 constexpr int kMaxL = 64;
-constexpr int kMaxKSplit = 8;          // stage-B partial sums kept per handle
-constexpr int kDecodeMaxT = 4;         // tokens per call the small-T kernel takes
-
-// Kernel-private tiled copy of a packed sign matrix (see pack.cu):
-// tiles of 32 rows x 128 columns, 512 bytes each, tile (rt, kt) at
-// ((rt * ktiles) + kt) * 128 words; inside a tile lane L = 4*g + q of a warp
-// owns the uint4 { w(g, q), w(g+8, q), w(g+16, q), w(g+24, q) } where
-// w(r, q) is canonical word q of row r of the tile.
-struct TiledSigns {
-    const uint32_t *words;  // device
-    int rtiles;             // ceil(rows / 32)
-    int ktiles;             // ceil(cols / 128)
-};
 
 // tensor maps of the last materialised-order forward (they depend only on the pointers and T)
 struct MatMaps {
@@ -48,19 +35,12 @@ struct T1Buffers {
 struct Layer {
     mdbf_desc_t d;
     int device;
-    // canonical words
+    // canonical words: kept only by layers without the row-block-major copy below (fp32 envelopes, l > 32)
     uint32_t *wA, *wB;
     int wordsA, wordsB;           // words per row
-    // tiled words
-    uint32_t *tA, *tB;
-    int rtA, ktA, rtB, ktB;
     // envelopes in env_dtype, row-major [rows][l]
     void *UA, *VA, *UB, *VB;
-    // kernel-private bf16 copies of V_A / V_B in MMA B-fragment order (see forward_decode.cu)
-    uint2 *vfA, *vfB;
-    int NT;                       // 8-column mode tiles in the fragment copies: 1, 2, 4 or 8
-    // TMEM-operand small-T kernel (16-bit envelopes, l <= 32): V in MMA k order, 16-bit, [kblocks][LP][64]
-    uint16_t *vpA, *vpB;
+    // one-token kernels (16-bit envelopes, l <= 32)
     uint16_t *vxA, *vxB;          // bf16 V tile images for the one-token kernel: [kb_pad][max(LP,16)][64], swizzled
     uint2 *wk2A, *wk2B;           // sign words, row-block major [row block][kb_pad][128] (one-token kernel)
     int kbpA, kbpB;               // K blocks per row block in wk2 / vx (even, zero padded)
@@ -81,14 +61,29 @@ struct Layer {
     MatMaps mat_maps;
     T1Buffers t1;
     // scratch
-    float *z;                     // [kMaxKSplit][zT][k] stage-B partial sums of the small-T kernel
-    size_t zstride;               // zT * k
-    float *zsum;                  // [max_T][k] summed intermediate (ALU path, inspection)
+    float *zsum;                  // [max_T][k] fp32 intermediate (ALU and one-token kernels; inspection copy otherwise)
     void *xstage, *ystage;        // device staging for the host-buffer entry point
     int32_t *status;              // device status word
-    int last_ksplit;              // how many partials the last forward wrote (0 = zsum valid, -1 = the intermediate is in zb)
+    int last_ksplit;              // where the last forward left the intermediate: 0 = zsum, -1 = zb (bf16)
     int out_mode;                 // set per call: 0 y in the activation type; 1 / 2: fp32 y stored / added (a term of a sum)
 };
+
+// A packed sign matrix as the kernels that are not tied to one layout read it: the canonical words (layers that only
+// the CUDA-core kernels serve), or - tensor-core layers keep a single copy of their signs - the row-block-major
+// copy of the one-token kernels, [row block of 128][kb_pad K blocks of 64 columns][128 rows] with 64 bits per entry.
+struct SignView {
+    const uint32_t *canon;
+    const uint2 *wk2;
+    int nwords;                   // 32-bit words per row in the canonical layout
+    int kb_pad;
+    __device__ __forceinline__ uint32_t word(int row, int w) const {
+        if (canon) return canon[(size_t)row * nwords + w];
+        const uint2 v = wk2[((size_t)(row >> 7) * kb_pad + (w >> 1)) * 128 + (row & 127)];
+        return (w & 1) ? v.y : v.x;
+    }
+};
+struct Layer;
+SignView sign_view(const Layer &L, int which);      // 0: S_A, 1: S_B
 
 // thread-local error string
 void set_error(const char *fmt, ...);
@@ -118,19 +113,28 @@ template <> __device__ __forceinline__ void act_store<__half>(__half *p, size_t 
 template <> __device__ __forceinline__ void act_store<__nv_bfloat16>(__nv_bfloat16 *p, size_t i, float v) { p[i] = __float2bfloat16_rn(v); }
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// cudaFuncSetAttribute is per device: one flag per (call site, device).  Returns true the first time it is asked
+// about the current device (the caller then sets its attributes), false afterwards or when the device is unknown.
+struct PerDeviceOnce {
+    bool done[64] = {};
+    bool first() {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;     // unknown device: set again, it is cheap
+        if (done[dev]) return false;
+        done[dev] = true;
+        return true;
+    }
+};
 inline size_t dtype_size(int dt) { return dt == MDBF_F32 ? 4 : 2; }
 
 // --- launchers (each returns after enqueueing on `st`) ------------------------
 mdbf_status_t launch_pack(const int8_t *s, int64_t rows, int64_t cols, uint32_t *out, cudaStream_t st);
 mdbf_status_t launch_unpack(const uint32_t *p, int64_t rows, int64_t cols, int8_t *out, cudaStream_t st);
-mdbf_status_t launch_tile(const uint32_t *canon, int rows, int words, uint32_t *tiled, int rtiles,
-                          int ktiles, cudaStream_t st);
 mdbf_status_t launch_env_round(const float *src, void *dst, size_t n, int dtype, cudaStream_t st);
 mdbf_status_t launch_env_read(const void *src, float *dst, size_t n, int dtype, cudaStream_t st);
-mdbf_status_t launch_vfrag(const void *V, int cols, int l, int env_dtype, uint2 *out, int ktiles, int NT,
-                           cudaStream_t st);
-mdbf_status_t launch_kblock(const uint32_t *canon, int rows, int nwords, uint2 *out, int rows_pad, int kblocks,
-                            cudaStream_t st);
+mdbf_status_t launch_kblock(const SignView &sv, int rows, uint2 *out, int rows_pad, int kblocks, cudaStream_t st);
+mdbf_status_t launch_canon(const SignView &sv, int rows, uint32_t *out, cudaStream_t st);
 mdbf_status_t launch_vtrans(const void *V, int cols, int l, int env_dtype, float *out, int pad, int LP, cudaStream_t st);
 mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows, int pad, int box_rows);
 mdbf_status_t ensure_prefill_scratch(Layer &L);
@@ -143,14 +147,10 @@ mdbf_status_t launch_zb_to_zsum(Layer &L, int T, cudaStream_t st);
 mdbf_status_t launch_reconstruct(const Layer &L, float *W, cudaStream_t st);
 mdbf_status_t launch_forward_alu(Layer &L, const void *x, void *y, int T, int act_dtype,
                                  cudaStream_t st, int *launches);
-mdbf_status_t launch_forward_decode(Layer &L, const void *x, void *y, int T, cudaStream_t st,
-                                    int *launches);
 mdbf_status_t launch_forward_prefill(Layer &L, const void *x, void *y, int T, cudaStream_t st,
                                      int *launches);
 mdbf_status_t launch_forward_tmem(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches);
 bool tmem_path_supports(const Layer &L, int T);
-mdbf_status_t launch_vperm(const void *V, int cols, int l, int env_dtype, uint16_t *out, int kblocks, int LP,
-                           cudaStream_t st);
 mdbf_status_t launch_forward_tmem_t1(Layer &L, const void *x, void *y, cudaStream_t st);
 mdbf_status_t t1_prepare(Layer &L, cudaStream_t st);
 void t1_release(Layer &L);

@@ -20,13 +20,13 @@ constexpr int ALU_TT = 8;   // tokens per pass
 
 template <typename InT, typename OutT>
 __global__ void __launch_bounds__(256)
-alu_stage_kernel(const uint32_t *__restrict__ words, int nwords, int rows, int cols,
+alu_stage_kernel(const SignView words, int rows, int cols,
                  const void *__restrict__ U, const void *__restrict__ V, int l, int env_dtype,
                  const InT *__restrict__ in, OutT *__restrict__ out, int T, int add) {
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (r >= rows) return;
-    const uint32_t *wrow = words + (size_t)r * nwords;
+    const int nwords = words.nwords;
 
     for (int tau0 = 0; tau0 < T; tau0 += ALU_TT) {
         float res[ALU_TT];
@@ -39,7 +39,7 @@ alu_stage_kernel(const uint32_t *__restrict__ words, int nwords, int rows, int c
 #pragma unroll
                 for (int b = 0; b < ALU_TT; ++b) acc[a][b] = 0.f;
             for (int w = lane; w < nwords; w += 32) {
-                const uint32_t word = wrow[w];
+                const uint32_t word = words.word(r, w);
                 const int cmax = min(32, cols - w * 32);
                 for (int bit = 0; bit < cmax; ++bit) {
                     const int c = w * 32 + bit;
@@ -86,16 +86,16 @@ template <typename ActT>
 static mdbf_status_t run(Layer &L, const void *x, void *y, int T, cudaStream_t st) {
     const int wpb = 8;
     alu_stage_kernel<ActT, float><<<ceil_div(L.d.k, wpb), wpb * 32, 0, st>>>(
-        L.wB, L.wordsB, L.d.k, L.d.d_in, L.UB, L.VB, L.d.l, L.d.env_dtype,
+        sign_view(L, 1), L.d.k, L.d.d_in, L.UB, L.VB, L.d.l, L.d.env_dtype,
         reinterpret_cast<const ActT *>(x), L.zsum, T, 0);
     MDBF_CUDA(cudaGetLastError());
     if (L.out_mode == 0)
         alu_stage_kernel<float, ActT><<<ceil_div(L.d.d_out, wpb), wpb * 32, 0, st>>>(
-            L.wA, L.wordsA, L.d.d_out, L.d.k, L.UA, L.VA, L.d.l, L.d.env_dtype,
+            sign_view(L, 0), L.d.d_out, L.d.k, L.UA, L.VA, L.d.l, L.d.env_dtype,
             L.zsum, reinterpret_cast<ActT *>(y), T, 0);
     else                                   // a term of a sum of layers: fp32 output, stored or added
         alu_stage_kernel<float, float><<<ceil_div(L.d.d_out, wpb), wpb * 32, 0, st>>>(
-            L.wA, L.wordsA, L.d.d_out, L.d.k, L.UA, L.VA, L.d.l, L.d.env_dtype,
+            sign_view(L, 0), L.d.d_out, L.d.k, L.UA, L.VA, L.d.l, L.d.env_dtype,
             L.zsum, reinterpret_cast<float *>(y), T, L.out_mode == 2 ? 1 : 0);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
@@ -130,23 +130,9 @@ mdbf_status_t launch_cast(const float *acc, void *y, size_t n, int act_dtype, cu
     return MDBF_OK;
 }
 
-// sum the stage-B partials into zsum (inspection only)
-__global__ void zsum_kernel(const float *__restrict__ z, float *__restrict__ zsum, int ksplit, size_t n,
-                            size_t stride) {
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        float s = 0.f;
-        for (int p = 0; p < ksplit; ++p) s += z[p * stride + i];
-        zsum[i] = s;
-    }
-}
-
+// make the fp32 copy of the intermediate current (inspection only): the materialised-envelope kernels keep z in bf16
 mdbf_status_t launch_zsum(Layer &L, int T, cudaStream_t st) {
-    if (L.last_ksplit < 0) return launch_zb_to_zsum(L, T, st);   // the materialised-envelope kernel keeps z in bf16
-    if (L.last_ksplit == 0) return MDBF_OK;
-    const size_t n = (size_t)T * L.d.k;
-    const size_t stride = L.zstride;
-    zsum_kernel<<<(int)min((size_t)1024, (n + 255) / 256), 256, 0, st>>>(L.z, L.zsum, L.last_ksplit, n, stride);
-    MDBF_CUDA(cudaGetLastError());
+    if (L.last_ksplit < 0) return launch_zb_to_zsum(L, T, st);
     return MDBF_OK;
 }
 

@@ -738,11 +738,6 @@ static int mt_ring(int kc, int nv, int bn, size_t part_bytes) {
 static size_t mt_smem_bytes(int kc, int nv, int bn, size_t part_bytes) {
     return (size_t)mt_ring(kc, nv, bn, part_bytes) * bn * MT_BK * 2 + (size_t)(1 + nv) * kc * 2048 + part_bytes + 1024;
 }
-static int mt_env_int(const char *name, int dflt) {
-    const char *v = getenv(name);
-    return v && *v ? atoi(v) : dflt;
-}
-
 // Tensor map of a bf16 output [T][rows] with rows `pitch` elements apart: box of 128 rows x 64 tokens, no swizzle.
 static mdbf_status_t make_out_tensor_map(CUtensorMap *out, const void *base, int T, int rows, int pitch) {
     typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -775,13 +770,12 @@ static mdbf_status_t make_out_tensor_map(CUtensorMap *out, const void *base, int
 
 template <bool STAGE_A>
 static mdbf_status_t launch_mat(const MatArgs &a0, const CUtensorMap &tm, const CUtensorMap &tmo, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce once;
+    if (once.first()) {
         const int max_smem = (int)mt_smem_bytes(4, 3, MT_BN, 0);
         MDBF_CUDA(cudaFuncSetAttribute(mat_stage_kernel<STAGE_A>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
         MDBF_CUDA(cudaFuncSetAttribute(mat_small_kernel<STAGE_A, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
         MDBF_CUDA(cudaFuncSetAttribute(mat_small_kernel<STAGE_A, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
-        attr_set = true;
     }
     MatArgs a = a0;
     const int rb = ceil_div(a.rows, MT_BM), npr = ceil_div(ceil_div(a.cols, MT_BK), 2);
@@ -791,7 +785,7 @@ static mdbf_status_t launch_mat(const MatArgs &a0, const CUtensorMap &tm, const 
     // Cost model: waves x (pairs per CTA + fixed part, in pairs).
     int ks = 1;
     if (small) {
-        const int fixed = mt_env_int("MDBF_MAT_FIXED_COST", 12), max_ks = mt_env_int("MDBF_MAT_MAX_KS", 8);
+        const int fixed = 12, max_ks = 8;                                  // fixed part of a CTA in pairs (swept on four shapes); portable cluster size
         long best = -1;
         for (int c = 1; c <= 8 && c <= max_ks; ++c) {
             const int per = ceil_div(npr, c);

@@ -433,15 +433,15 @@ prescale_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ V
 
 // --------------------------------------------------------- pack-time private copies
 // K-blocked sign words: out[kb * rows_pad + r] = words (2kb, 2kb+1) of row r, zero outside the matrix.
-__global__ void kblock_kernel(const uint32_t *__restrict__ canon, int rows, int nwords, uint2 *__restrict__ out,
-                              int rows_pad, int kblocks) {
+__global__ void kblock_kernel(const SignView sv, int rows, uint2 *__restrict__ out, int rows_pad, int kblocks) {
+    const int nwords = sv.nwords;
     const size_t total = (size_t)kblocks * rows_pad;
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
         const int kb = (int)(idx / rows_pad), r = (int)(idx % rows_pad);
         uint2 v = make_uint2(0u, 0u);
         if (r < rows) {
-            if (2 * kb < nwords) v.x = canon[(size_t)r * nwords + 2 * kb];
-            if (2 * kb + 1 < nwords) v.y = canon[(size_t)r * nwords + 2 * kb + 1];
+            if (2 * kb < nwords) v.x = sv.word(r, 2 * kb);
+            if (2 * kb + 1 < nwords) v.y = sv.word(r, 2 * kb + 1);
         }
         out[idx] = v;
     }
@@ -463,9 +463,19 @@ static int pf_grid(size_t items) {
     return (int)g;
 }
 
-mdbf_status_t launch_kblock(const uint32_t *canon, int rows, int nwords, uint2 *out, int rows_pad, int kblocks,
-                            cudaStream_t st) {
-    kblock_kernel<<<pf_grid((size_t)kblocks * rows_pad), 256, 0, st>>>(canon, rows, nwords, out, rows_pad, kblocks);
+mdbf_status_t launch_kblock(const SignView &sv, int rows, uint2 *out, int rows_pad, int kblocks, cudaStream_t st) {
+    kblock_kernel<<<pf_grid((size_t)kblocks * rows_pad), 256, 0, st>>>(sv, rows, out, rows_pad, kblocks);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}
+// canonical words of a sign matrix from whichever copy the layer keeps (mdbf_get_packed)
+__global__ void canon_kernel(const SignView sv, int rows, uint32_t *__restrict__ out) {
+    const size_t total = (size_t)rows * sv.nwords;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x)
+        out[idx] = sv.word((int)(idx / sv.nwords), (int)(idx % sv.nwords));
+}
+mdbf_status_t launch_canon(const SignView &sv, int rows, uint32_t *out, cudaStream_t st) {
+    canon_kernel<<<pf_grid((size_t)rows * sv.nwords), 256, 0, st>>>(sv, rows, out);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
@@ -513,11 +523,10 @@ mdbf_status_t make_xs_tensor_map(CUtensorMap *out, const void *base, size_t rows
 // ---------------------------------------------------------------------- launch
 template <int LP, bool STAGE_A>
 static mdbf_status_t launch_gemm(const GemmArgs &a, const CUtensorMap &tm, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce once;
+    if (once.first()) {
         MDBF_CUDA(cudaFuncSetAttribute(gemm_stage_kernel<LP, STAGE_A, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
         MDBF_CUDA(cudaFuncSetAttribute(gemm_stage_kernel<LP, STAGE_A, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
-        attr_set = true;
     }
     const int TT = PF_BN / LP;
     const int rb = ceil_div(a.rows, PF_BM), ntiles = ceil_div(a.T, TT), nkb = ceil_div(a.cols, PF_BK);

@@ -881,13 +881,8 @@ static mdbf_status_t t1_launch(const t1::Group &grp, int ctas, cudaStream_t st, 
     auto stage_kern = t1::t1_stage_kernel<LP>;
     auto image_kern = t1::t1_image_kernel<LP>;
     const size_t smem = t1::Cfg<LP>::SMEM;
-    static bool attr_set[64] = {};
-    int dev = 0;
-    MDBF_CUDA(cudaGetDevice(&dev));
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        MDBF_CUDA(cudaFuncSetAttribute(stage_kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_set[dev] = true;
-    }
+    static PerDeviceOnce once;
+    if (once.first()) MDBF_CUDA(cudaFuncSetAttribute(stage_kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     for (int s = 0; s < 2; ++s) {
         if (!(stages >> s & 1)) continue;
         mdbf_status_t rc = t1_launch_one(image_kern, grp.items[s], t1::kImgThreads, 0, st, grp, s);

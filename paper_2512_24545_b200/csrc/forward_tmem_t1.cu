@@ -28,7 +28,7 @@
 //
 // CTA = 128 sign rows x a slice of the reduction; the KS CTAs of a row block form a cluster and
 // reduce their partial outputs through distributed shared memory (deterministic, no atomics).
-// Column order inside a K block as in forward_tmem.cu: MMA k index p is canonical column
+// Column order inside a K block: MMA k index p is canonical column
 // 32*(p/32) + (p%32)/2 + 16*(p%2).  Every mbarrier wait is bounded (MDBF_ERR_TIMEOUT in the
 // status word, all roles fall through, TMEM released).  Every bulk copy targets the issuing CTA's own shared memory only.
 #include <cooperative_groups.h>
@@ -465,17 +465,9 @@ struct TxPlan {
     size_t smem;
 };
 
-// Fixed part of a CTA's time (set-up, cluster reduction) in units of one K block of streaming;
-// MDBF_T1_FIXED_COST overrides it for experiments.
-static int fixed_cost() {
-    static int v = -1;
-    if (v < 0) {
-        const char *e = getenv("MDBF_T1_FIXED_COST");
-        v = e ? atoi(e) : 48;
-        if (v < 0) v = 48;
-    }
-    return v;
-}
+// Fixed part of a CTA's time (set-up, cluster reduction) in units of one K block of streaming (swept on the
+// 7B- and 70B-class shapes).
+static int fixed_cost() { return 48; }
 
 // One plan for all the layers of a launch.  Cluster size along the reduction: one CTA per SM (all of
 // TMEM), as few waves as possible, the per-CTA fixed part weighed against its share of the reduction.
@@ -483,8 +475,7 @@ static bool plan_t1(int n, const int *rows, const int *kb_pad, int LP, TxPlan *p
     const int NB = LP < 16 ? 16 : LP;
     int nas = (512 - TX_ISSUERS * NB) / 64;
     if (nas > TX_MAX_ASTAGES) nas = TX_MAX_ASTAGES;
-    static int max_ks = 0;
-    if (!max_ks) { const char *e = getenv("MDBF_T1_MAX_KS"); max_ks = e ? atoi(e) : 8; if (max_ks < 1 || max_ks > 8) max_ks = 8; }
+    const int max_ks = 8;                                     // portable cluster size
     int rb = 0, max_pairs = 0, min_pairs = 1 << 30;
     for (int i = 0; i < n; ++i) {
         rb += ceil_div(rows[i], 128);
@@ -517,12 +508,11 @@ int last_t1_launch_count() { return g_t1_launches; }
 
 template <int LP, int G>
 static mdbf_status_t launch_t1g(const TxMulti &m, const TxPlan &p, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce once;
+    if (once.first()) {
         MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_kernel<LP, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
         MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_multi_kernel<LP, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
         MDBF_CUDA(cudaFuncSetAttribute(tmem_t1_sumlast_kernel<LP, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
-        attr_set = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(m.rb_start[m.nlayers], p.ks, 1);
@@ -548,8 +538,7 @@ static mdbf_status_t launch_t1g(const TxMulti &m, const TxPlan &p, cudaStream_t 
 // 4096 x 4096 layers keep two groups, the 11008- and 70B-class layers get three).
 template <int LP>
 static mdbf_status_t launch_t1(const TxMulti &m, const TxPlan &p, cudaStream_t st) {
-    static int long_cta = 0;
-    if (!long_cta) { const char *e = getenv("MDBF_T1_LONG_CTA"); long_cta = e ? atoi(e) : 16; if (long_cta < 1) long_cta = 1; }
+    const int long_cta = 16;
     int max_per = 0;
     for (int i = 0; i < m.nlayers; ++i) max_per = max(max_per, p.pairs_per_cta[i]);
     return max_per >= long_cta ? launch_t1g<LP, 3>(m, p, st) : launch_t1g<LP, 2>(m, p, st);
@@ -689,6 +678,48 @@ mdbf_status_t launch_forward_tmem_t1_sum(Layer *const *Ls, int n, const void *x,
             set_error("mdbf_linear_forward_sum: the one-token TMEM kernel handles l <= 32 (got %d)", Ls[0]->d.l);
             return MDBF_ERR_SHAPE;
     }
+}
+
+// Whether the one-token TMEM-operand kernel can run this layer (16-bit envelopes, l <= 32, both stages plannable).
+bool tmem_path_supports(const Layer &L, int T) {
+    if (T != 1 || !L.wk2A || !L.vxA || !L.vxB || L.d.l > 32) return false;
+    const int rowsB = L.d.k, rowsA = L.d.d_out;
+    TxPlan pb, pa;
+    return plan_t1(1, &rowsB, &L.kbpB, L.LP, &pb) && plan_t1(1, &rowsA, &L.kbpA, L.LP, &pa);
+}
+
+// ------------------------------------------------------------------ self-test of the bounded wait
+// One warp waits on an mbarrier that nothing ever arrives at, with the same bounded wait the
+// forward kernels use: after the time limit it must record MDBF_ERR_TIMEOUT in the status word and
+// return normally (no trap, the context stays usable).
+__global__ void wait_timeout_selftest_kernel(int32_t *status) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag_s;
+    if (threadIdx.x == 0) {
+        tm::mbar_init(tm::smem_u32(&bar), 1);
+        abort_flag_s = 0;
+        tm::fence_barrier_init();
+    }
+    __syncthreads();
+    tm::mbar_wait(tm::smem_u32(&bar), 0u, &abort_flag_s, status);
+}
+
+mdbf_status_t launch_wait_timeout_selftest(Layer &L, cudaStream_t st) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(L.status);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}
+
+mdbf_status_t launch_forward_tmem(Layer &L, const void *x, void *y, int T, cudaStream_t st, int *launches) {
+    if (T != 1 || !L.wk2A || !L.vxA || !L.vxB) {
+        set_error("mdbf_linear_forward: the TMEM-operand kernel takes one token, 16-bit envelopes and l <= 32");
+        return MDBF_ERR_SHAPE;
+    }
+    mdbf_status_t rc = launch_forward_tmem_t1(L, x, y, st);
+    if (rc) return rc;
+    L.last_ksplit = 0;
+    *launches = last_t1_launch_count();
+    return MDBF_OK;
 }
 
 mdbf_status_t launch_forward_tmem_t1(Layer &L, const void *x, void *y, cudaStream_t st) {

@@ -57,15 +57,34 @@ static mdbf_status_t check_handle(mdbf_handle_t h, const char *fn) {
     return MDBF_OK;
 }
 
+// A layer lives on the device it was packed on; its kernels must be launched there.
+static mdbf_status_t check_device(const Layer &L, const char *fn) {
+    int dev = -1;
+    MDBF_CUDA(cudaGetDevice(&dev));
+    if (dev != L.device) {
+        set_error("%s: the layer was packed on device %d, the current device is %d", fn, L.device, dev);
+        return MDBF_ERR_INVALID_ARG;
+    }
+    return MDBF_OK;
+}
+
+}  // namespace mdbf
+mdbf::SignView mdbf::sign_view(const Layer &L, int which) {
+    SignView v;
+    v.canon = which == 0 ? L.wA : L.wB;
+    v.wk2 = which == 0 ? L.wk2A : L.wk2B;
+    v.nwords = which == 0 ? L.wordsA : L.wordsB;
+    v.kb_pad = which == 0 ? L.kbpA : L.kbpB;
+    return v;
+}
+namespace mdbf {
+
 static void free_layer(Layer &L) {
-    void *ptrs[] = {L.wA, L.wB, L.tA, L.tB, L.UA, L.VA, L.UB, L.VB, L.vfA, L.vfB, L.vpA, L.vpB, L.vxA, L.vxB, L.wk2A, L.wk2B, L.wkA, L.wkB, L.uiA, L.uiB, L.viA, L.viB, L.vtB, L.xsB, L.xsA, L.zb, L.z, L.zsum, L.xstage, L.ystage, L.status};
+    void *ptrs[] = {L.wA, L.wB, L.UA, L.VA, L.UB, L.VB, L.vxA, L.vxB, L.wk2A, L.wk2B, L.wkA, L.wkB, L.uiA, L.uiB, L.viA, L.viB, L.vtB, L.xsB, L.xsA, L.zb, L.zsum, L.xstage, L.ystage, L.status};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     t1_release(L);
 }
-
-// number of tokens the small-T kernel's partial-sum scratch is sized for
-static int decode_scratch_T(const mdbf_desc_t &d) { return d.max_T < kDecodeMaxT ? d.max_T : kDecodeMaxT; }
 
 // mdbf_pack builds what the default dispatch uses (canonical words, the row-block-major sign copy, the
 // one-token V tiles, the envelope images).  The private layouts and scratch of the other kernels are built
@@ -87,50 +106,38 @@ static mdbf_status_t ensure_kblock_words(Layer &L) {
     ENS_CUDA(cudaMalloc(&a, (size_t)(L.padA / 64) * L.rpA * sizeof(uint2)));
     cudaError_t e = cudaMalloc(&b, (size_t)(L.padB / 64) * L.rpB * sizeof(uint2));
     if (e != cudaSuccess) { cudaFree(a); return cuda_fail(e, "K-blocked sign words"); }
+    mdbf_status_t rc = launch_kblock(sign_view(L, 0), d.d_out, a, L.rpA, L.padA / 64, 0);
+    if (rc == MDBF_OK) rc = launch_kblock(sign_view(L, 1), d.k, b, L.rpB, L.padB / 64, 0);
+    if (rc) { cudaFree(a); cudaFree(b); return rc; }
     L.wkA = a; L.wkB = b;
-    ENS_RC(launch_kblock(L.wA, d.d_out, L.wordsA, L.wkA, L.rpA, L.padA / 64, 0));
-    ENS_RC(launch_kblock(L.wB, d.k, L.wordsB, L.wkB, L.rpB, L.padB / 64, 0));
     return MDBF_OK;
 }
+// Scratch and private layouts of the expanded-order kernel (K-blocked sign words, transposed V_B, the pre-scaled
+// operands): built by mdbf_pack for layers that can only run that order, else by mdbf_set_kernel(PREFILL) - never
+// by a forward.  Every buffer is published to the layer only once it is complete.
 mdbf_status_t ensure_kernel_layouts(Layer &L, int kernel, int T) {
+    (void)T;
     const mdbf_desc_t &d = L.d;
-    bool built = false;
-    if (kernel == MDBF_KERNEL_DECODE && !L.tA) {
-        ENS_CUDA(cudaMalloc(&L.tA, (size_t)L.rtA * L.ktA * 512));
-        ENS_CUDA(cudaMalloc(&L.tB, (size_t)L.rtB * L.ktB * 512));
-        ENS_CUDA(cudaMalloc(&L.vfA, (size_t)L.ktA * 8 * L.NT * 256));
-        ENS_CUDA(cudaMalloc(&L.vfB, (size_t)L.ktB * 8 * L.NT * 256));
-        ENS_CUDA(cudaMalloc(&L.z, (size_t)kMaxKSplit * L.zstride * sizeof(float)));
-        ENS_RC(launch_tile(L.wA, d.d_out, L.wordsA, L.tA, L.rtA, L.ktA, 0));
-        ENS_RC(launch_tile(L.wB, d.k, L.wordsB, L.tB, L.rtB, L.ktB, 0));
-        ENS_RC(launch_vfrag(L.VA, d.k, d.l, d.env_dtype, L.vfA, L.ktA, L.NT, 0));
-        ENS_RC(launch_vfrag(L.VB, d.d_in, d.l, d.env_dtype, L.vfB, L.ktB, L.NT, 0));
-        built = true;
+    if (kernel != MDBF_KERNEL_PREFILL || !L.zb || L.xsB) return MDBF_OK;
+    ENS_RC(ensure_kblock_words(L));
+    if (!L.vtB) {
+        float *vt = nullptr;
+        ENS_CUDA(cudaMalloc(&vt, (size_t)L.LP * L.padB * sizeof(float)));
+        mdbf_status_t rc = launch_vtrans(L.VB, d.d_in, d.l, d.env_dtype, vt, L.padB, L.LP, 0);
+        if (rc) { cudaFree(vt); return rc; }
+        L.vtB = vt;
     }
-    if (kernel == MDBF_KERNEL_TMEM && T > 1 && L.wk2A && !L.vpA) {
-        ENS_RC(ensure_kblock_words(L));
-        ENS_CUDA(cudaMalloc(&L.vpA, (size_t)(L.padA / 64) * L.LP * 64 * sizeof(uint16_t)));
-        ENS_CUDA(cudaMalloc(&L.vpB, (size_t)(L.padB / 64) * L.LP * 64 * sizeof(uint16_t)));
-        ENS_RC(launch_vperm(L.VA, d.k, d.l, d.env_dtype, L.vpA, L.padA / 64, L.LP, 0));
-        ENS_RC(launch_vperm(L.VB, d.d_in, d.l, d.env_dtype, L.vpB, L.padB / 64, L.LP, 0));
-        built = true;
-    }
-    if (kernel == MDBF_KERNEL_PREFILL && L.zb && !L.xsB) {
-        ENS_RC(ensure_kblock_words(L));
-        if (!L.vtB) {
-            ENS_CUDA(cudaMalloc(&L.vtB, (size_t)L.LP * L.padB * sizeof(float)));
-            ENS_RC(launch_vtrans(L.VB, d.d_in, d.l, d.env_dtype, L.vtB, L.padB, L.LP, 0));
-        }
-        ENS_RC(ensure_prefill_scratch(L));
-        built = true;
-    }
-    if (built) ENS_CUDA(cudaStreamSynchronize(0));
+    ENS_RC(ensure_prefill_scratch(L));
+    ENS_CUDA(cudaStreamSynchronize(0));
     return MDBF_OK;
 }
 static mdbf_status_t ensure_host_staging(Layer &L) {
     if (L.xstage) return MDBF_OK;
-    ENS_CUDA(cudaMalloc(&L.xstage, (size_t)L.d.max_T * L.d.d_in * 4));
-    ENS_CUDA(cudaMalloc(&L.ystage, (size_t)L.d.max_T * L.d.d_out * 4));
+    void *xs = nullptr, *ys = nullptr;
+    ENS_CUDA(cudaMalloc(&xs, (size_t)L.d.max_T * L.d.d_in * 4));
+    cudaError_t e = cudaMalloc(&ys, (size_t)L.d.max_T * L.d.d_out * 4);
+    if (e != cudaSuccess) { cudaFree(xs); return cuda_fail(e, "host-entry staging"); }
+    L.xstage = xs; L.ystage = ys;
     return MDBF_OK;
 }
 #undef ENS_CUDA
@@ -206,8 +213,6 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     L.device = dev;
     L.wordsA = ceil_div(d.k, 32);
     L.wordsB = ceil_div(d.d_in, 32);
-    L.rtA = ceil_div(d.d_out, 32); L.ktA = ceil_div(d.k, 128);
-    L.rtB = ceil_div(d.k, 32);     L.ktB = ceil_div(d.d_in, 128);
     const size_t es = dtype_size(d.env_dtype);
     const size_t nUA = (size_t)d.d_out * d.l, nVA = (size_t)d.k * d.l, nUB = nVA, nVB = (size_t)d.d_in * d.l;
     const size_t nSA = (size_t)d.d_out * d.k, nSB = (size_t)d.k * d.d_in;
@@ -236,7 +241,6 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     PACK_CUDA(cudaMalloc(&L.VA, nVA * es));
     PACK_CUDA(cudaMalloc(&L.UB, nUB * es));
     PACK_CUDA(cudaMalloc(&L.VB, nVB * es));
-    L.NT = d.l <= 8 ? 1 : d.l <= 16 ? 2 : d.l <= 32 ? 4 : 8;
     L.LP = 1;
     while (L.LP < d.l) L.LP *= 2;
     L.padA = ceil_div(d.k, 64) * 64; L.padB = ceil_div(d.d_in, 64) * 64;
@@ -264,7 +268,6 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
         PACK_CUDA(cudaMalloc(&L.viA, (size_t)ceil_div(L.padA, 128) * L.kcm * 1024 * sizeof(uint16_t)));
         PACK_CUDA(cudaMalloc(&L.viB, (size_t)ceil_div(L.padB, 128) * L.kcm * 1024 * sizeof(uint16_t)));
     }
-    L.zstride = (size_t)decode_scratch_T(d) * d.k;
     PACK_CUDA(cudaMalloc(&L.zsum, (size_t)d.max_T * d.k * sizeof(float)));
     PACK_CUDA(cudaMalloc(&L.status, sizeof(int32_t)));
     PACK_CUDA(cudaMemsetAsync(L.status, 0, sizeof(int32_t), st));
@@ -304,6 +307,10 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     PACK_CUDA(cudaStreamSynchronize(st));
     for (void *p : temps) cudaFree(p);
     temps.clear();
+    if (want_tc) {                                    // one copy of the signs per layer: the row-block-major one serves every kernel
+        cudaFree(L.wA); cudaFree(L.wB);
+        L.wA = nullptr; L.wB = nullptr;
+    }
     // a layer the materialised order can never serve (no tensor map over x) will run the expanded order
     if (want_prefill && d.d_in % 8 != 0) PACK_RC(ensure_kernel_layouts(L, MDBF_KERNEL_PREFILL, 2));
 #undef PACK_CUDA
@@ -319,11 +326,25 @@ mdbf_status_t mdbf_get_packed(mdbf_handle_t h, int which, uint32_t *out, int out
     if (rc) return rc;
     if (!out || (which != 0 && which != 1)) { set_error("mdbf_get_packed: bad argument"); return MDBF_ERR_INVALID_ARG; }
     const Layer &L = h->L;
-    const size_t bytes = which == 0 ? (size_t)L.d.d_out * L.wordsA * 4 : (size_t)L.d.k * L.wordsB * 4;
+    const int rows = which == 0 ? L.d.d_out : L.d.k;
+    const size_t bytes = (size_t)rows * (which == 0 ? L.wordsA : L.wordsB) * 4;
     cudaStream_t st = (cudaStream_t)stream;
-    MDBF_CUDA(cudaMemcpyAsync(out, which == 0 ? L.wA : L.wB, bytes,
-                              out_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
-    MDBF_CUDA(cudaStreamSynchronize(st));
+    const SignView sv = sign_view(L, which);
+    if (out_on_device) {
+        rc = launch_canon(sv, rows, out, st);
+        if (rc) return rc;
+        MDBF_CUDA(cudaStreamSynchronize(st));
+        return MDBF_OK;
+    }
+    uint32_t *tmp = nullptr;                          // check path: a temporary device copy in canonical order
+    MDBF_CUDA(cudaMalloc(&tmp, bytes));
+    rc = launch_canon(sv, rows, tmp, st);
+    cudaError_t e = cudaSuccess;
+    if (rc == MDBF_OK) e = cudaMemcpyAsync(out, tmp, bytes, cudaMemcpyDeviceToHost, st);
+    if (rc == MDBF_OK && e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(tmp);
+    if (rc) return rc;
+    if (e != cudaSuccess) return cuda_fail(e, "mdbf_get_packed copy");
     return MDBF_OK;
 }
 
@@ -365,13 +386,12 @@ mdbf_status_t mdbf_get_desc(mdbf_handle_t h, mdbf_desc_t *out) {
 mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel) {
     mdbf_status_t rc = check_handle(h, "mdbf_set_kernel");
     if (rc) return rc;
-    if (kernel < MDBF_KERNEL_AUTO || kernel > MDBF_KERNEL_I8) {
+    if (kernel < MDBF_KERNEL_AUTO || kernel > MDBF_KERNEL_I8 || kernel == 2) {
         set_error("mdbf_set_kernel: unknown kernel %d", kernel);
         return MDBF_ERR_INVALID_ARG;
     }
-    // build the kernel's private layouts and scratch here rather than inside a forward
-    const bool tc_layer = h->L.wk2A != nullptr;
-    if (kernel == MDBF_KERNEL_DECODE || ((kernel == MDBF_KERNEL_TMEM || kernel == MDBF_KERNEL_PREFILL) && tc_layer)) {
+    // the expanded-order kernel's layouts and scratch are built here, never inside a forward
+    if (kernel == MDBF_KERNEL_PREFILL && h->L.wk2A != nullptr) {
         rc = ensure_kernel_layouts(h->L, kernel, 2);
         if (rc) return rc;
     }
@@ -422,6 +442,10 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         return MDBF_ERR_SHAPE;
     }
     if (!valid_dtype(act_dtype)) { set_error("mdbf_linear_forward: bad act_dtype %d", act_dtype); return MDBF_ERR_DTYPE; }
+    {
+        mdbf_status_t rcd = check_device(L, "mdbf_linear_forward");
+        if (rcd) return rcd;
+    }
     int kernel = h->kernel;
     const bool tc_ok = (act_dtype == MDBF_BF16) && (L.d.env_dtype != MDBF_F32) && L.d.l <= 32;
     if (kernel == MDBF_KERNEL_AUTO) {
@@ -434,9 +458,8 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         // to, the l sign GEMMs of the expanded order at every T >= 2); the expanded order serves the layers
         // the tensor map over x cannot take (d_in not a multiple of 8, unaligned x)
         else if (mat_path_supports(L, x, T)) kernel = MDBF_KERNEL_MAT;
-        else if (L.zb) kernel = MDBF_KERNEL_PREFILL;
-        else if (tmem_path_supports(L, T)) kernel = MDBF_KERNEL_TMEM;
-        else kernel = MDBF_KERNEL_DECODE;
+        else if (L.xsB) kernel = MDBF_KERNEL_PREFILL;           // its scratch exists (d_in % 8 != 0 layers get it at pack time)
+        else kernel = MDBF_KERNEL_ALU;                          // e.g. an x that is not 16-byte aligned: no allocation here, ever
     }
     if (kernel == -1) {
         Layer *one = &L;
@@ -449,29 +472,26 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         set_error("mdbf_linear_forward: the tensor-core kernels need bf16 activations, 16-bit envelopes and l <= 32");
         return MDBF_ERR_DTYPE;
     }
-    if (kernel == MDBF_KERNEL_DECODE && (T > kDecodeMaxT || L.d.l > 32)) {
-        set_error("mdbf_linear_forward: the small-T kernel handles T <= %d and l <= 32 (got T=%d, l=%d)",
-                  kDecodeMaxT, T, L.d.l);
-        return MDBF_ERR_SHAPE;
+    if (kernel == MDBF_KERNEL_PREFILL && !L.xsB) {
+        set_error("mdbf_linear_forward: the expanded-order kernel has no scratch on this handle; call mdbf_set_kernel(handle, MDBF_KERNEL_PREFILL) first (it allocates)");
+        return MDBF_ERR_INVALID_ARG;
     }
     if (kernel == MDBF_KERNEL_I8 && (T != 1 || !t1_supports(L))) {
         set_error("mdbf_linear_forward: the one-token integer kernel needs T = 1, 16-bit envelopes and l <= 32");
         return MDBF_ERR_SHAPE;
     }
-    if (out_mode != 0 && (kernel == MDBF_KERNEL_DECODE || (kernel == MDBF_KERNEL_TMEM && T > 1))) {
+    if (out_mode != 0 && kernel == MDBF_KERNEL_I8) {
         set_error("mdbf_linear_forward_sum: the forced kernel has no fp32-accumulate output");
         return MDBF_ERR_INVALID_ARG;
     }
     int launches = 0;
-    mdbf_status_t rc = ensure_kernel_layouts(L, kernel, T);      // no-op for the default kernels
-    if (rc) return rc;
+    mdbf_status_t rc = MDBF_OK;
     if (kernel == MDBF_KERNEL_I8) {
         Layer *one = &L;
         rc = launch_forward_t1_group(&one, 1, &x, &y, st);
         L.last_ksplit = 0;
         launches = 4;                                         // image and stage kernel, twice
     } else if (kernel == MDBF_KERNEL_ALU) rc = launch_forward_alu(L, x, y, T, act_dtype, st, &launches);
-    else if (kernel == MDBF_KERNEL_DECODE) rc = launch_forward_decode(L, x, y, T, st, &launches);
     else if (kernel == MDBF_KERNEL_TMEM) rc = launch_forward_tmem(L, x, y, T, st, &launches);
     else if (kernel == MDBF_KERNEL_MAT) rc = launch_forward_mat(L, x, y, T, st, &launches);
     else rc = launch_forward_prefill(L, x, y, T, st, &launches);
@@ -493,6 +513,8 @@ mdbf_status_t mdbf_linear_forward_sum(const mdbf_handle_t *terms, int32_t P, con
     if (P < 1 || P > 64) { set_error("mdbf_linear_forward_sum: P=%d outside [1, 64]", P); return MDBF_ERR_SHAPE; }
     for (int p = 0; p < P; ++p) {
         mdbf_status_t rc = check_handle(terms[p], "mdbf_linear_forward_sum");
+        if (rc) return rc;
+        rc = check_device(terms[p]->L, "mdbf_linear_forward_sum");
         if (rc) return rc;
         if (terms[p]->L.d.d_out != terms[0]->L.d.d_out || terms[p]->L.d.d_in != terms[0]->L.d.d_in) {
             set_error("mdbf_linear_forward_sum: term %d is %d x %d, term 0 is %d x %d", p, terms[p]->L.d.d_out,
@@ -545,6 +567,8 @@ mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t 
         if (rc) return rc;
         if (!ys[i]) { set_error("mdbf_linear_forward_siblings: NULL output %d", i); return MDBF_ERR_INVALID_ARG; }
         const Layer &L = layers[i]->L;
+        rc = check_device(L, "mdbf_linear_forward_siblings");
+        if (rc) return rc;
         if (L.d.d_in != layers[0]->L.d.d_in) {
             set_error("mdbf_linear_forward_siblings: layer %d has d_in=%d, layer 0 has %d", i, L.d.d_in, layers[0]->L.d.d_in);
             return MDBF_ERR_SHAPE;
@@ -601,14 +625,24 @@ mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void
     if (!valid_dtype(act_dtype)) { set_error("mdbf_linear_forward_host: bad act_dtype %d", act_dtype); return MDBF_ERR_DTYPE; }
     cudaStream_t st = (cudaStream_t)stream;
     const size_t es = dtype_size(act_dtype);
-    rc = ensure_host_staging(L);
-    if (rc) return rc;
+    if (!L.xstage) {
+        set_error("mdbf_linear_forward_host: no staging buffers on this handle; call mdbf_prepare_host_staging(handle) once first (it allocates)");
+        return MDBF_ERR_INVALID_ARG;
+    }
     MDBF_CUDA(cudaMemcpyAsync(L.xstage, x_host, (size_t)T * L.d.d_in * es, cudaMemcpyHostToDevice, st));
     rc = forward_impl(h, L.xstage, L.ystage, T, act_dtype, st);
     if (rc) return rc;
     MDBF_CUDA(cudaMemcpyAsync(y_host, L.ystage, (size_t)T * L.d.d_out * es, cudaMemcpyDeviceToHost, st));
     MDBF_CUDA(cudaStreamSynchronize(st));
     return MDBF_OK;
+}
+
+mdbf_status_t mdbf_prepare_host_staging(mdbf_handle_t h) {
+    mdbf_status_t rc = check_handle(h, "mdbf_prepare_host_staging");
+    if (rc) return rc;
+    rc = check_device(h->L, "mdbf_prepare_host_staging");
+    if (rc) return rc;
+    return ensure_host_staging(h->L);
 }
 
 mdbf_status_t mdbf_get_intermediate(mdbf_handle_t h, float *z, int32_t T, int out_on_device, void *stream) {

@@ -66,24 +66,6 @@ __global__ void unpack_kernel(const uint32_t *__restrict__ p, int64_t rows, int6
     }
 }
 
-// canonical -> tiled (layout documented at TiledSigns)
-__global__ void tile_kernel(const uint32_t *__restrict__ canon, int rows, int words,
-                            uint32_t *__restrict__ tiled, int rtiles, int ktiles) {
-    const int64_t total = (int64_t)rtiles * ktiles * 128;
-    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t tile = idx >> 7;
-        const int within = (int)(idx & 127);
-        const int lane = within >> 2, comp = within & 3;
-        const int g = lane >> 2, q = lane & 3;
-        const int rt = (int)(tile / ktiles), kt = (int)(tile - (int64_t)rt * ktiles);
-        const int row = rt * 32 + g + 8 * comp;
-        const int word = kt * 4 + q;
-        uint32_t v = 0;
-        if (row < rows && word < words) v = canon[(int64_t)row * words + word];
-        tiled[idx] = v;
-    }
-}
 
 __global__ void env_round_kernel(const float *__restrict__ src, void *__restrict__ dst, size_t n, int dtype) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
@@ -120,13 +102,6 @@ mdbf_status_t launch_unpack(const uint32_t *p, int64_t rows, int64_t cols, int8_
     return MDBF_OK;
 }
 
-mdbf_status_t launch_tile(const uint32_t *canon, int rows, int words, uint32_t *tiled, int rtiles,
-                          int ktiles, cudaStream_t st) {
-    tile_kernel<<<grid_for((int64_t)rtiles * ktiles * 128, 256), 256, 0, st>>>(canon, rows, words, tiled,
-                                                                             rtiles, ktiles);
-    MDBF_CUDA(cudaGetLastError());
-    return MDBF_OK;
-}
 
 mdbf_status_t launch_env_round(const float *src, void *dst, size_t n, int dtype, cudaStream_t st) {
     env_round_kernel<<<grid_for((int64_t)n, 256), 256, 0, st>>>(src, dst, n, dtype);

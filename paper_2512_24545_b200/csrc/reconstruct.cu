@@ -10,7 +10,7 @@ constexpr int RT = 64;   // output tile (rows and columns)
 constexpr int RJ = 16;   // inner-rank chunk
 
 __global__ void __launch_bounds__(256)
-reconstruct_kernel(const uint32_t *__restrict__ wA, int wordsA, const uint32_t *__restrict__ wB, int wordsB,
+reconstruct_kernel(const SignView wA, const SignView wB,
                    const void *__restrict__ UA, const void *__restrict__ VA,
                    const void *__restrict__ UB, const void *__restrict__ VB,
                    int d_out, int d_in, int k, int l, int env_dtype, float *__restrict__ W) {
@@ -35,7 +35,7 @@ reconstruct_kernel(const uint32_t *__restrict__ wA, int wordsA, const uint32_t *
                     for (int t = 0; t < l; ++t)
                         v += (double)env_load(UA, (size_t)n * l + t, env_dtype) *
                              (double)env_load(VA, (size_t)j * l + t, env_dtype);
-                    if ((wA[(size_t)n * wordsA + (j >> 5)] >> (j & 31)) & 1u) v = -v;
+                    if ((wA.word(n, j >> 5) >> (j & 31)) & 1u) v = -v;
                 }
                 sU[cj][rn] = v;
             }
@@ -47,7 +47,7 @@ reconstruct_kernel(const uint32_t *__restrict__ wA, int wordsA, const uint32_t *
                     for (int s = 0; s < l; ++s)
                         v += (double)env_load(UB, (size_t)j * l + s, env_dtype) *
                              (double)env_load(VB, (size_t)i * l + s, env_dtype);
-                    if ((wB[(size_t)j * wordsB + (i >> 5)] >> (i & 31)) & 1u) v = -v;
+                    if ((wB.word(j, i >> 5) >> (i & 31)) & 1u) v = -v;
                 }
                 sV[cj][ci] = v;
             }
@@ -81,7 +81,7 @@ reconstruct_kernel(const uint32_t *__restrict__ wA, int wordsA, const uint32_t *
 
 mdbf_status_t launch_reconstruct(const Layer &L, float *W, cudaStream_t st) {
     dim3 grid(ceil_div(L.d.d_in, RT), ceil_div(L.d.d_out, RT));
-    reconstruct_kernel<<<grid, 256, 0, st>>>(L.wA, L.wordsA, L.wB, L.wordsB, L.UA, L.VA, L.UB, L.VB,
+    reconstruct_kernel<<<grid, 256, 0, st>>>(sign_view(L, 0), sign_view(L, 1), L.UA, L.VA, L.UB, L.VB,
                                              L.d.d_out, L.d.d_in, L.d.k, L.d.l, L.d.env_dtype, W);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;

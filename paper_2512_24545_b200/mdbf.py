@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmdbf.so")
 
 F32, F16, BF16 = 0, 1, 2
-KERNEL_AUTO, KERNEL_ALU, KERNEL_DECODE, KERNEL_PREFILL, KERNEL_TMEM, KERNEL_MAT, KERNEL_I8 = 0, 1, 2, 3, 4, 5, 6
+KERNEL_AUTO, KERNEL_ALU, KERNEL_PREFILL, KERNEL_TMEM, KERNEL_MAT, KERNEL_I8 = 0, 1, 3, 4, 5, 6
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_DTYPE, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT, ERR_VALUE = (
     -1, -2, -3, -4, -5, -6, -7, -8)
@@ -27,7 +27,7 @@ DTYPES = {"f32": F32, "f16": F16, "bf16": BF16}
 
 EXPORTS = (
     "mdbf_pack_signs", "mdbf_unpack_signs", "mdbf_pack", "mdbf_get_packed", "mdbf_get_envelope",
-    "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host",
+    "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host", "mdbf_prepare_host_staging",
     "mdbf_linear_forward_static", "mdbf_linear_forward_sum", "mdbf_linear_forward_siblings",
     "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_poll_status", "mdbf_selftest_wait_timeout",
     "mdbf_last_launch_count",
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
     L.mdbf_set_kernel.argtypes = [vp, i32]
     L.mdbf_linear_forward.argtypes = [vp, vp, vp, i32, i32, vp]
     L.mdbf_linear_forward_host.argtypes = [vp, vp, vp, i32, i32, vp]
+    L.mdbf_prepare_host_staging.argtypes = [vp]
     L.mdbf_linear_forward_static.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, vp]
     L.mdbf_linear_forward_sum.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp]
     L.mdbf_linear_forward_siblings.argtypes = [vp, i32, vp, vp, i32, i32, vp]
@@ -168,6 +169,11 @@ def mdbf_linear_forward_siblings(handles, x, ys, T: int, act_dtype: int, stream:
     outs = (ctypes.c_void_p * len(ys))(*[_addr(y) for y in ys])
     _check(lib().mdbf_linear_forward_siblings(ctypes.cast(hs, ctypes.c_void_p), len(handles), _addr(x),
                                               ctypes.cast(outs, ctypes.c_void_p), T, act_dtype, stream))
+
+
+def mdbf_prepare_host_staging(h: int) -> None:
+    """Allocate the handle's device staging buffers for mdbf_linear_forward_host (once per handle)."""
+    _check(lib().mdbf_prepare_host_staging(h))
 
 
 def mdbf_linear_forward_host(h: int, x_host, y_host, T: int, act_dtype: int, stream: int = 0) -> None:

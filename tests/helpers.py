@@ -86,24 +86,27 @@ def rel_err(got: np.ndarray, ref: np.ndarray) -> float:
     return orc.rel_frobenius(got, ref)
 
 
-def magnitude_bound(g: "GpuLayer", x: np.ndarray) -> np.ndarray:
-    """|U_hat| (|V_hat^T| |x|) as a (T, d_out) array: what |y| could be if nothing cancelled.  Every rounding on a
+def magnitude_bound(g: "GpuLayer", x: np.ndarray, rows=None) -> np.ndarray:
+    """|U_hat| (|V_hat^T| |x|) as a (T, d_out) array (or its columns `rows`): what |y| could be if nothing cancelled.  Every rounding on a
     bf16 path perturbs a y element by at most 2^-8 of this (a relative error of one operand or partial result
     propagates through sums of absolute values), whatever the shape - also where k is too small for errors to
     average out."""
     L = g.lay
-    Uh = np.abs(orc.modulated_factor(L["S_A"], L["U_A"], L["V_A"]))       # d_out x k
-    Vh = np.abs(orc.modulated_factor(L["S_B"], L["U_B"], L["V_B"]))       # k x d_in
+    sel = slice(None) if rows is None else rows
+    Uh = np.abs(orc.modulated_factor(L["S_A"][sel], L["U_A"][sel], L["V_A"]))     # (rows of) d_out x k
+    Vh = np.abs(orc.modulated_factor(L["S_B"], L["U_B"], L["V_B"]))               # k x d_in
     return (Uh @ (Vh @ np.abs(x.T.astype(np.float64)))).T
 
 
 def check_parity(g: "GpuLayer", x: np.ndarray, got: np.ndarray, ref: np.ndarray | None = None, roundings: int = 4,
-                 act: str | None = None) -> float:
+                 act: str | None = None, averaging: bool = True) -> float:
     """The three parity assertions of a forward against the oracle; returns the whole-array error.
       1. whole array: relative Frobenius error <= 5e-3 (bf16 activations, fp32 accumulation) / 1e-5 (fp32 path);
       2. every block of 128 output rows on its own: the same bound, so that one wrong tile cannot hide in the norm;
       3. every element: |y - y_ref| <= (roundings + 1) * 2^-8 * |U_hat| (|V_hat^T| |x|) (fp32 path: 1e-5 of it),
-         `roundings` = bf16 roundings on the path that produced y."""
+         `roundings` = bf16 roundings on the path that produced y.
+    averaging=False (layers with a handful of terms per output, where rounding errors cannot average out and the
+    Frobenius ratio is no sharper than the per-element bound) keeps assertion 3 only."""
     act = act or g.spec.act_dtype
     tol = TOL[act]
     if ref is None:
@@ -117,10 +120,14 @@ def check_parity(g: "GpuLayer", x: np.ndarray, got: np.ndarray, ref: np.ndarray 
     assert excess[worst] <= 1e-30, (f"element {worst}: |y - y_ref| = {abs(got[worst] - ref[worst]):.3e} exceeds "
                                     f"{unit:.2e} * {bound[worst]:.3e}")
     err = rel_err(got, ref)
+    if not averaging:
+        return err
     assert err <= tol, f"relative Frobenius error {err:.3e} > {tol}"
     ref_rms = np.sqrt(np.mean(ref ** 2))
     for r0 in range(0, ref.shape[1], 128):
         blk = slice(r0, min(r0 + 128, ref.shape[1]))
+        if blk.stop - blk.start < 128:                                   # a ragged tail of a few rows is too small a sample for a
+            continue                                                     # norm ratio: the per-element bound above covers it
         if np.sqrt(np.mean(ref[:, blk] ** 2)) < 1e-3 * ref_rms:          # a block of (nearly) zero rows has no relative error
             continue
         e = rel_err(got[:, blk], ref[:, blk])

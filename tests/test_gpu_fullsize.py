@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_2512_24545_b200 import inputs, mdbf as M
-from helpers import GpuLayer, TOL, rel_err
+from helpers import GpuLayer, TOL, magnitude_bound, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -54,9 +54,23 @@ def test_mlp_small_batch_full_size(which, T):
         assert rel_err(y0, y[:1]) <= 2 * TOL["bf16"]
 
 
-@pytest.mark.parametrize("d_out,l,bpw", [(4096, 16, 1.0), (4096, 4, 1.5), (4096, 1, 1.0), (11008, 16, 1.5),
-                                         (11008, 1, 1.5)])
+PREFILL_POINTS = [(d_out, l, bpw) for d_out in (4096, 11008) for l in (1, 4, 16) for bpw in (1.0, 1.5)]
+
+
+def check_tokens_rows(g, x, y, rows, tok):
+    ref = g.oracle_forward_rows(x[tok], rows)
+    assert np.all(np.isfinite(y))
+    got = y[np.ix_(tok, rows)]
+    assert rel_err(got, ref) <= TOL["bf16"]
+    # every sampled element on its own (no token or row hides in the norm): four bf16 roundings at most on any path
+    bound = magnitude_bound(g, x[tok], rows)
+    assert np.all(np.abs(got - ref) <= 5 * 2.0 ** -8 * bound)
+
+
+@pytest.mark.parametrize("d_out,l,bpw", PREFILL_POINTS)
 def test_prefill_full_size(d_out, l, bpw):
+    """All twelve points of the prefill sweep (both shapes, l in {1, 4, 16}, ~1.0 and ~1.5 bpw) at T = 2048
+    under the library's own choice of kernel."""
     spec = inputs.prefill(d_out, l, bpw)
     T = 2048
     x = inputs.make_activations(spec, T)
@@ -64,20 +78,65 @@ def test_prefill_full_size(d_out, l, bpw):
         y = g.forward(x)
         assert M.mdbf_poll_status(g.h) == 0
         tok = np.array([0, 1, 15, 16, 255, 256, 1000, 2047])       # sampled tokens x sampled rows
-        rows = sampled_rows(spec.d_out, n=24)
-        ref = g.oracle_forward_rows(x[tok], rows)
-        assert rel_err(y[np.ix_(tok, rows)], ref) <= TOL["bf16"]
-        assert np.all(np.isfinite(y))
+        check_tokens_rows(g, x, y, sampled_rows(spec.d_out, n=24), tok)
         # linearity at full size: a power-of-two scale is exact
         y2 = g.forward(2.0 * x[:64])
         np.testing.assert_array_equal(y2, 2.0 * g.forward(x[:64]))
 
 
-@pytest.mark.parametrize("idx", [1, 4])      # k_proj 1024x8192 and gate 28672x8192
-def test_block70b_layers_full_size(idx):
+@pytest.mark.parametrize("d_out,l,bpw", [(4096, 16, 1.0), (11008, 1, 1.5), (4096, 4, 1.5)])
+def test_prefill_full_size_expanded_order(d_out, l, bpw):
+    """The expanded-order kernel (pre-scale, l sign GEMMs of width l T, mode contraction in the epilogue) at T = 2048."""
+    spec = inputs.prefill(d_out, l, bpw)
+    T = 2048
+    x = inputs.make_activations(spec, T)
+    with GpuLayer(spec, T) as g:
+        y = g.forward(x, kernel=M.KERNEL_PREFILL)
+        assert M.mdbf_poll_status(g.h) == 0
+        assert M.mdbf_last_kernel(g.h) == M.KERNEL_PREFILL
+        tok = np.array([0, 1, 15, 16, 255, 256, 1000, 2047])
+        check_tokens_rows(g, x, y, sampled_rows(spec.d_out, n=24), tok)
+
+
+@pytest.mark.parametrize("idx", range(7))      # q, k, v, o, gate, up, down of the 70B-class block
+def test_block70b_layers_full_size_one_token(idx):
     spec = inputs.block70b()[idx]
     x = inputs.make_activations(spec, 1)
     with GpuLayer(spec, 1) as g:
         y = g.forward(x)
         assert M.mdbf_poll_status(g.h) == 0
         check_rows(g, x, y, sampled_rows(spec.d_out, n=16), TOL["bf16"])
+        y8 = g.forward(x, kernel=M.KERNEL_I8)                       # both one-token kernels at full size
+        check_rows(g, x, y8, sampled_rows(spec.d_out, n=16), TOL["bf16"])
+
+
+def test_block70b_siblings_full_size_one_token():
+    """q/k/v and gate/up through the sibling entry point, as bench.py runs the block."""
+    specs = inputs.block70b()
+    for group in ([0, 1, 2], [4, 5]):
+        layers = [GpuLayer(specs[i], 1) for i in group]
+        try:
+            x = inputs.make_activations(specs[group[0]], 1)
+            xd = torch.from_numpy(x).to(torch.bfloat16).cuda()
+            ys = [torch.full((1, specs[i].d_out), float("nan"), dtype=torch.bfloat16, device="cuda") for i in group]
+            M.mdbf_linear_forward_siblings([g.h for g in layers], xd.data_ptr(), [y.data_ptr() for y in ys], 1, M.BF16,
+                                           torch.cuda.current_stream().cuda_stream)
+            torch.cuda.synchronize()
+            for g, y in zip(layers, ys):
+                assert M.mdbf_poll_status(g.h) == 0
+                check_rows(g, x, y.to(torch.float32).cpu().numpy(), sampled_rows(g.spec.d_out, n=12), TOL["bf16"])
+        finally:
+            for g in layers:
+                g.close()
+
+
+@pytest.mark.parametrize("idx", range(7))
+def test_block70b_layers_full_size_2048_tokens(idx):
+    spec = inputs.block70b()[idx]
+    T = 2048
+    x = inputs.make_activations(spec, T)
+    with GpuLayer(spec, T) as g:
+        y = g.forward(x)
+        assert M.mdbf_poll_status(g.h) == 0
+        tok = np.array([0, 255, 256, 1033, 2047])
+        check_tokens_rows(g, x, y, sampled_rows(spec.d_out, n=8), tok)

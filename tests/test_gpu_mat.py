@@ -7,7 +7,7 @@ import torch
 
 from oracle import mdbf_oracle as orc
 from paper_2512_24545_b200 import inputs, mdbf as M
-from helpers import GpuLayer, TOL, rel_err
+from helpers import check_parity, GpuLayer, rel_err, TOL
 
 pytestmark = pytest.mark.gpu
 
@@ -32,8 +32,7 @@ def test_mat_kernel_small_shapes(l, T):
         ref = g.oracle_forward(x)
         y = g.forward(x, kernel=M.KERNEL_MAT)
         assert M.mdbf_poll_status(g.h) == 0
-        assert np.all(np.isfinite(y))
-        assert rel_err(y, ref) <= TOL["bf16"]
+        check_parity(g, x, y, ref)                               # whole array, every 128-row block, every element
         _, z_ref = orc.forward_staged(*g.oracle_args(), x.T.astype(np.float64))
         assert rel_err(g.intermediate(T), z_ref.T) <= TOL["bf16"]
 
@@ -47,10 +46,9 @@ def test_mat_kernel_ragged_shapes(shape):
     with GpuLayer(spec, 19) as g:
         y = g.forward(x, kernel=M.KERNEL_MAT)
         assert M.mdbf_poll_status(g.h) == 0
-        # a one-term layer has nothing to average: worst case of the path's four bf16 roundings
-        # (W_hat of either stage, z, y), each at most 2^-8 relative
-        tol = 4 * 2.0 ** -8 if k == 1 else TOL["bf16"]
-        assert rel_err(y, g.oracle_forward(x)) <= tol
+        # a layer with a few terms per output cannot average its four bf16 roundings (W_hat of either stage, z, y):
+        # there the per-element bound is the assertion
+        check_parity(g, x, y, averaging=k >= 8)
 
 
 @pytest.mark.parametrize("shape", [(128, 2048, 1024, 8, 8), (256, 1100 * 8, 520, 16, 40), (200, 4096, 136, 3, 2)])
@@ -62,7 +60,7 @@ def test_mat_kernel_split_reduction(shape):
     with GpuLayer(spec, T) as g:
         y = g.forward(x, kernel=M.KERNEL_MAT)
         assert M.mdbf_poll_status(g.h) == 0
-        assert rel_err(y, g.oracle_forward(x)) <= TOL["bf16"]
+        check_parity(g, x, y)
         np.testing.assert_array_equal(y, g.forward(x, kernel=M.KERNEL_MAT))     # deterministic summation order
 
 
@@ -108,13 +106,21 @@ def test_auto_dispatch_reports_its_kernel_and_serves_unaligned_x():
         assert M.mdbf_last_kernel(g.h) == M.KERNEL_MAT
         ref = g.oracle_forward(x8)
         assert rel_err(y8, ref) <= TOL["bf16"]
-        # x two bytes off a 16-byte boundary: no tensor map over it, the expanded order runs (and allocates
-        # its scratch on this first use)
+        # x two bytes off a 16-byte boundary: no tensor map over it and no scratch for the expanded order on this
+        # handle: the CUDA-core kernel serves the call (a forward never allocates); after mdbf_set_kernel(PREFILL)
+        # has built that scratch, the library's own choice for such an x is the expanded order
         buf = torch.zeros(8 * spec.d_in + 8, dtype=torch.bfloat16, device="cuda")
         xd = buf[1:1 + 8 * spec.d_in].view(8, spec.d_in)
         xd.copy_(torch.from_numpy(x8).to(torch.bfloat16))
         assert xd.data_ptr() % 16 == 2
         yd = torch.zeros((8, spec.d_out), dtype=torch.bfloat16, device="cuda")
+        M.mdbf_linear_forward(g.h, xd.data_ptr(), yd.data_ptr(), 8, M.BF16, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert M.mdbf_last_kernel(g.h) == M.KERNEL_ALU
+        assert rel_err(yd.to(torch.float32).cpu().numpy(), ref) <= TOL["bf16"]
+        M.mdbf_set_kernel(g.h, M.KERNEL_PREFILL)
+        M.mdbf_set_kernel(g.h, M.KERNEL_AUTO)
+        yd.zero_()
         M.mdbf_linear_forward(g.h, xd.data_ptr(), yd.data_ptr(), 8, M.BF16, torch.cuda.current_stream().cuda_stream)
         torch.cuda.synchronize()
         assert M.mdbf_last_kernel(g.h) == M.KERNEL_PREFILL
@@ -148,6 +154,4 @@ def test_mat_kernels_seeded_random_shapes(shape):
         assert M.mdbf_last_kernel(g.h) == M.KERNEL_MAT
         assert M.mdbf_poll_status(g.h) == 0
         assert np.all(np.isfinite(y))
-        # few terms per output (small k) do not average the roundings: worst case of four bf16 roundings
-        tol = TOL["bf16"] if k >= 32 else 4 * 2.0 ** -8
-        assert rel_err(y, g.oracle_forward(x)) <= tol
+        check_parity(g, x, y, averaging=k >= 32)                # few terms per output: the per-element bound alone

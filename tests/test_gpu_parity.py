@@ -10,7 +10,7 @@ import torch
 
 from oracle import mdbf_oracle as orc
 from paper_2512_24545_b200 import inputs, mdbf as M
-from helpers import GpuLayer, TOL, TOL_RECONSTRUCT, rel_err
+from helpers import GpuLayer, TOL, TOL_RECONSTRUCT, check_parity, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -88,7 +88,7 @@ def test_tiny_config_fp32(T):
         y = g.forward(x)
         assert M.mdbf_last_launch_count(g.h) == 2
         ref = g.oracle_forward(x)
-        assert rel_err(y, ref) <= TOL["f32"]
+        check_parity(g, x, y, ref)
         z = g.intermediate(T)
         _, z_ref = orc.forward_staged(*g.oracle_args(), x.T.astype(np.float64))
         assert rel_err(z, z_ref.T) <= TOL["f32"]
@@ -100,39 +100,37 @@ def test_alu_path_ragged_shapes_fp32(shape):
     spec = inputs.scaled(inputs.tiny(), d_out=d_out, d_in=d_in, k=k, l=l)
     x = inputs.make_activations(spec, 3)
     with GpuLayer(spec, 3) as g:
-        assert rel_err(g.forward(x), g.oracle_forward(x)) <= TOL["f32"]
+        check_parity(g, x, g.forward(x), averaging=k >= 8)
 
 
-# ------------------------------------------------------- forward, small-T kernel
+# ------------------------------------------------------- forward, few tokens, library's choice of kernel
 @pytest.mark.parametrize("T", [1, 2, 3, 4])
 @pytest.mark.parametrize("l", [1, 4, 16, 24])
-def test_decode_kernel_small_shapes(T, l):
+def test_few_tokens_small_shapes(T, l):
     spec = small_spec(l=l)
     x = inputs.make_activations(spec, T)
     with GpuLayer(spec, 4) as g:
         ref = g.oracle_forward(x)
-        y = g.forward(x, kernel=M.KERNEL_DECODE)
-        assert np.all(np.isfinite(y))
-        assert rel_err(y, ref) <= TOL["bf16"]
+        y = g.forward(x)
+        check_parity(g, x, y, ref)
         _, z_ref = orc.forward_staged(*g.oracle_args(), x.T.astype(np.float64))
         assert rel_err(g.intermediate(T), z_ref.T) <= TOL["bf16"]
         y_alu = g.forward(x, kernel=M.KERNEL_ALU)
-        assert rel_err(y_alu, ref) <= TOL["bf16"]
+        check_parity(g, x, y_alu, ref, roundings=1)
         assert rel_err(y, y_alu) <= 2 * TOL["bf16"]
 
 
 @pytest.mark.parametrize("shape", [(1, 1, 1, 1), (31, 127, 33, 2), (32, 128, 128, 16), (129, 1025, 257, 9),
                                    (1000, 2100, 1300, 16)])
-def test_decode_kernel_edge_shapes(shape):
+def test_few_tokens_edge_shapes(shape):
     d_out, d_in, k, l = shape
     spec = small_spec(d_out=d_out, d_in=d_in, k=k, l=l)
     x = inputs.make_activations(spec, 2)
     with GpuLayer(spec, 2) as g:
-        y = g.forward(x, kernel=M.KERNEL_DECODE)
-        assert rel_err(y, g.oracle_forward(x)) <= TOL["bf16"]
+        check_parity(g, x, g.forward(x), averaging=k >= 8)
 
 
-def test_decode_kernel_bf16_envelopes_and_repeat_calls():
+def test_bf16_envelopes_and_repeat_calls():
     spec = small_spec(env_dtype="bf16")
     x = inputs.make_activations(spec, 1)
     with GpuLayer(spec, 1) as g:
@@ -212,7 +210,7 @@ def test_forward_error_paths():
     with GpuLayer(spec32, 1) as g:
         xb = inputs.round_to(inputs.make_activations(spec32, 1), "bf16")
         with pytest.raises(M.MdbfError) as e:
-            g.forward(xb, kernel=M.KERNEL_DECODE)
+            g.forward(xb, kernel=M.KERNEL_TMEM)
         assert e.value.status == M.ERR_DTYPE
         assert rel_err(g.forward(xb), g.oracle_forward(xb)) <= TOL["bf16"]     # AUTO -> fp32 path
 
@@ -223,6 +221,10 @@ def test_host_buffer_entry_point():
     with GpuLayer(spec, 2) as g:
         xh = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
         yh = torch.zeros((2, spec.d_out), dtype=torch.bfloat16).pin_memory()
+        with pytest.raises(M.MdbfError) as e:                      # no staging buffers yet: the call never allocates
+            M.mdbf_linear_forward_host(g.h, xh.data_ptr(), yh.data_ptr(), 2, M.BF16, torch.cuda.current_stream().cuda_stream)
+        assert e.value.status == M.ERR_INVALID_ARG
+        M.mdbf_prepare_host_staging(g.h)
         M.mdbf_linear_forward_host(g.h, xh.data_ptr(), yh.data_ptr(), 2, M.BF16,
                                    torch.cuda.current_stream().cuda_stream)
         y_dev = g.forward(x)

@@ -6,7 +6,7 @@ import torch
 
 from oracle import mdbf_oracle as orc
 from paper_2512_24545_b200 import inputs, mdbf as M
-from helpers import GpuLayer, TOL, rel_err
+from helpers import check_parity, GpuLayer, rel_err, TOL
 
 pytestmark = pytest.mark.gpu
 
@@ -31,8 +31,7 @@ def test_prefill_kernel_small_shapes(l, T):
         ref = g.oracle_forward(x)
         y = g.forward(x, kernel=M.KERNEL_PREFILL)
         assert M.mdbf_poll_status(g.h) == 0
-        assert np.all(np.isfinite(y))
-        assert rel_err(y, ref) <= TOL["bf16"]
+        check_parity(g, x, y, ref, roundings=3)
         _, z_ref = orc.forward_staged(*g.oracle_args(), x.T.astype(np.float64))
         assert rel_err(g.intermediate(T), z_ref.T) <= TOL["bf16"]
 
@@ -45,12 +44,10 @@ def test_prefill_kernel_ragged_shapes(shape):
     with GpuLayer(spec, 19) as g:
         y = g.forward(x, kernel=M.KERNEL_PREFILL)
         assert M.mdbf_poll_status(g.h) == 0
-        # 5e-3 is a bound on the Frobenius (RMS) error of many independently rounded terms; the
-        # one-term layer has nothing to average, so it gets a worst-case style bound instead: its
-        # bf16 roundings (scaled x, scaled z, y; z itself stays fp32) are each at most 2^-8 relative
-        # and at most 2^-9 on average over the mantissa range, hence 4 * 2^-9 with margin.
-        tol = 4 * 2.0 ** -9 if k == 1 else TOL["bf16"]
-        assert rel_err(y, g.oracle_forward(x)) <= tol
+        # 5e-3 bounds the Frobenius (RMS) error of many independently rounded terms; a layer with a few terms per
+        # output has nothing to average, so there the per-element bound (three bf16 roundings: scaled x, scaled z, y)
+        # is the assertion
+        check_parity(g, x, y, roundings=3, averaging=k >= 8)
 
 
 def test_prefill_agrees_with_small_T_kernel_and_auto_dispatch():
@@ -59,9 +56,9 @@ def test_prefill_agrees_with_small_T_kernel_and_auto_dispatch():
     with GpuLayer(spec, 64) as g:
         ref = g.oracle_forward(x)
         y_pf = g.forward(x, kernel=M.KERNEL_PREFILL)
-        y_dec = g.forward(x, kernel=M.KERNEL_DECODE)
-        assert rel_err(y_pf, ref) <= TOL["bf16"] and rel_err(y_dec, ref) <= TOL["bf16"]
-        assert rel_err(y_pf, y_dec) <= 2 * TOL["bf16"]
+        y_alu = g.forward(x, kernel=M.KERNEL_ALU)
+        assert rel_err(y_pf, ref) <= TOL["bf16"] and rel_err(y_alu, ref) <= TOL["bf16"]
+        assert rel_err(y_pf, y_alu) <= 2 * TOL["bf16"]
         x64 = inputs.make_activations(spec, 64)
         y_auto = g.forward(x64)                       # T >= 2 -> materialised-order kernel
         assert M.mdbf_last_kernel(g.h) == M.KERNEL_MAT

@@ -64,6 +64,12 @@ def test_static_forward_matches_handle_forward_twice(case):
             got, ref = y.float().cpu().numpy(), y_ref.float().cpu().numpy()
             assert np.all(np.isfinite(got))
             assert _rel(got, ref) <= TOL[act], f"call {call}"
+            # and against the CPU oracle itself, on the values as stored (envelopes rounded to the layer's type)
+            from oracle import mdbf_oracle as orc
+            stored = [e.float().cpu().numpy().astype(np.float64) for e in env]
+            y_orc = orc.forward(lay["S_A"], lay["S_B"], stored[0], stored[1], stored[2], stored[3],
+                                x.float().cpu().numpy().T.astype(np.float64)).T
+            assert _rel(got, y_orc) <= TOL[act], f"call {call} against the oracle"
     finally:
         M.mdbf_destroy(h)
 
