@@ -43,11 +43,12 @@ NCU_TRAFFIC_BYTES_PER_LAUNCH = {
 }
 
 
-def dominant_kernel(spec, T, forced="auto"):
-    """Name of the kernel the library's dispatcher picks for this (l, T): the one the roofline line is about."""
+def dominant_kernel(workload, T, kernels_used, M):
+    """Name of the kernel that takes most of the step's device time (the one the roofline line is about)."""
     if T == 1:
-        return "tmem_t1_kernel"
-    if forced == "mat":
+        # the integer kernel streams the large stages (gate/up stage A and down stage B of the 70B-class block)
+        return "t1_stage_kernel" if workload.startswith("block70b") or M.KERNEL_I8 in kernels_used else "tmem_t1_kernel"
+    if M.KERNEL_MAT in kernels_used:
         return "mat_stage_kernel" if T > 64 else "mat_small_kernel"
     return "gemm_stage_kernel"
 
@@ -126,54 +127,96 @@ def workload_specs(name):
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons sampled during the timed region."""
+    """SM clock and throttle reasons sampled during the timed region: NVML polled every few milliseconds (a timed
+    region of some tens of milliseconds still gets a handful of samples), nvidia-smi as the fallback.  Read-only."""
 
     def __init__(self, index):
         self.index = index
-        self.samples = []
+        self.samples = []          # (sm_mhz, max_mhz, reasons bitmask)
+        self.stop_flag = False
+        self.thread = None
+        self.nvml = None
         self.proc = None
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nvml = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            self.thread = threading.Thread(target=self._poll_nvml, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread = threading.Thread(target=self._read_smi, daemon=True)
             self.thread.start()
         except OSError:
             self.proc = None
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.samples.append(line.strip())
+    def _poll_nvml(self):
+        n = self.nvml
+        while not self.stop_flag:
+            try:
+                sm = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
+                try:
+                    reasons = int(n.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                except Exception:
+                    reasons = int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                self.samples.append((sm, self.max_mhz, reasons))
+            except Exception:
+                break
+            time.sleep(0.002)
 
-    def stop(self):
-        if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=2)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
+    def _read_smi(self):
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for s in self.samples:
-            f = [x.strip() for x in s.split(",")]
+        bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+        for line in self.proc.stdout:
+            f = [x.strip() for x in line.split(",")]
             if len(f) < 7:
                 continue
             try:
-                sm.append(float(f[0])); mx.append(float(f[1]))
+                sm, mx = float(f[0]), float(f[1])
             except ValueError:
                 continue
-            for n, v in zip(names, f[3:7]):
+            mask = 0
+            for nm, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
-                    reasons.add(n)
+                    mask |= bits[nm]
+            self.samples.append((sm, mx, mask))
+
+    def stop(self):
+        self.stop_flag = True
+        if self.nvml is None and self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is not None:
+            time.sleep(0.05)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        if self.thread is not None:
+            self.thread.join(timeout=1.0)
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+        sm = [x[0] for x in self.samples]
+        mx = [x[1] for x in self.samples]
+        reasons = set()
+        for (_s, _m, mask) in self.samples:
+            for bit, nm in names.items():
+                if mask & bit:
+                    reasons.add(nm)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm),
+                "source": "nvml" if self.nvml is not None else "nvidia-smi"}
 
 
 def dist_setup(n_gpus):
@@ -191,20 +234,19 @@ def dist_setup(n_gpus):
 
 
 # ------------------------------------------------------------------ mdbf arm
-def run_mdbf(args):
+def measure(workload, kernel, steps, warmup, dist, world, local, no_graph=False, no_siblings=False, copies=0,
+            want_e2e=True):
+    """Time `steps` steps of one workload (after >= 3 untimed ones) and return the measured fields."""
     import torch
-    from paper_2512_24545_b200 import build, inputs, mdbf as M, replicas
-    build.build()
-    dist, rank, world, local = dist_setup(args.gpus)
-    torch.cuda.set_device(local)
+    from paper_2512_24545_b200 import inputs, mdbf as M, replicas
     peaks, peak_kind = load_peaks()
-    groups, T, bound, desc = workload_specs(args.workload)
+    groups, T, bound, desc = workload_specs(workload)
     stream = torch.cuda.Stream()
     st = stream.cuda_stream
 
-    P_sum = len(groups) if args.workload.startswith("sum_") else 0     # > 0: every P_sum consecutive layers are one sum
+    P_sum = len(groups) if workload.startswith("sum_") else 0     # > 0: every P_sum consecutive layers are one sum
     if P_sum:
-        ncopies = args.copies if args.copies > 0 else groups[0][1]
+        ncopies = copies if copies > 0 else groups[0][1]
         groups = [(inputs.scaled(sp, seed=sp.seed + 1000 * c), 1) for c in range(ncopies) for (sp, _n) in groups]
     layers = []          # (handle, spec, x_dev, y_dev, x_host, y_host)
     total_bytes = 0
@@ -212,17 +254,19 @@ def run_mdbf(args):
     total_mat_flops = 0.0
     weight_bytes = 0
     xs = {}
-    if args.workload.startswith("block70b"):       # block by block: q, k, v, o, gate, up, down of copy 0, then copy 1, ...
-        nc = args.copies if args.copies > 0 else groups[0][1]
+    if workload.startswith("block70b"):       # block by block: q, k, v, o, gate, up, down of copy 0, then copy 1, ...
+        nc = copies if copies > 0 else groups[0][1]
         groups = [(inputs.scaled(sp, seed=sp.seed + 1000 * c) if c else sp, 1) for c in range(nc) for (sp, _n) in groups]
     for spec, copies in groups:
-        for c in range(1 if (P_sum or args.workload.startswith("block70b")) else (args.copies if args.copies > 0 else copies)):
+        for c in range(1 if (P_sum or workload.startswith("block70b")) else (copies if copies > 0 else copies)):
             sp = inputs.scaled(spec, seed=spec.seed + 1000 * (c + 1)) if c else spec
             lay = inputs.make_layer(sp)
             h = M.mdbf_pack(sp.d_out, sp.d_in, sp.k, sp.l, M.DTYPES[sp.env_dtype], T,
                             *[np.ascontiguousarray(lay[n]) for n in ("S_A", "S_B", "U_A", "V_A", "U_B", "V_B")])
-            if T > 1 and args.kernel != "auto":
-                M.mdbf_set_kernel(h, {"prefill": M.KERNEL_PREFILL, "mat": M.KERNEL_MAT}[args.kernel])
+            if T > 1 and kernel in ("prefill", "mat"):
+                M.mdbf_set_kernel(h, {"prefill": M.KERNEL_PREFILL, "mat": M.KERNEL_MAT}[kernel])
+            if T == 1 and kernel in ("tmem", "i8"):
+                M.mdbf_set_kernel(h, {"tmem": M.KERNEL_TMEM, "i8": M.KERNEL_I8}[kernel])
             if sp.d_in not in xs:
                 xh = torch.from_numpy(inputs.make_activations(sp, T)).to(torch.bfloat16).pin_memory()
                 xs[sp.d_in] = (xh, xh.cuda())
@@ -245,7 +289,7 @@ def run_mdbf(args):
     # the 70B-class block at one token: q/k/v share the hidden input and gate/up share the MLP input, so they
     # go through the sibling entry point (one pair of launches per group); o and down stand alone
     sib_groups = None
-    if args.workload.startswith("block70b") and T == 1 and not args.no_siblings:
+    if workload.startswith("block70b") and T == 1 and not no_siblings:
         sib_groups = []
         for b0 in range(0, len(layers), 7):
             blk = layers[b0:b0 + 7]
@@ -282,7 +326,7 @@ def run_mdbf(args):
     with torch.cuda.stream(stream):
         step()                       # first call sets kernel attributes (not capturable state)
         torch.cuda.synchronize()
-        if not args.no_graph:
+        if not no_graph:
             # one CUDA graph per step: removes the host launch cost of the back-to-back forwards
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph, stream=stream):
@@ -290,13 +334,13 @@ def run_mdbf(args):
             run_step = graph.replay
         else:
             run_step = step
-        for _ in range(max(3, args.warmup)):
+        for _ in range(max(3, warmup)):
             run_step()
         barrier()
         sampler = ClockSampler(local)
         sampler.start()
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-              for _ in range(args.steps)]
+              for _ in range(steps)]
         for (e0, e1) in ev:
             if flush is not None:
                 flush.fill_(1)
@@ -306,22 +350,26 @@ def run_mdbf(args):
         barrier()
         clocks = sampler.stop()
         ms = sum(e0.elapsed_time(e1) for e0, e1 in ev)
-    launches = (sum(M.mdbf_last_launch_count(h) for (h, *_rest) in layers) + (len(layers) // P_sum if (P_sum and T > 1) else 0)) * args.steps     # the cast pass of a sum runs only for T > 1
+    launches = (sum(M.mdbf_last_launch_count(h) for (h, *_rest) in layers) + (len(layers) // P_sum if (P_sum and T > 1) else 0)) * steps     # the cast pass of a sum runs only for T > 1
+    kernels_used = sorted({M.mdbf_last_kernel(h) for (h, *_r) in layers})
+    mat = M.KERNEL_MAT in kernels_used
 
     # end to end: host buffers through the C-ABI, copies inside the timed region
-    e2e_steps = max(1, min(args.steps, 10))
-    for (h, *_r) in layers:
-        M.mdbf_prepare_host_staging(h)
-    for _ in range(2):
-        for (h, sp, _, _, xh, yh) in layers:
-            M.mdbf_linear_forward_host(h, xh.data_ptr(), yh.data_ptr(), T, M.BF16, st)
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        for (h, sp, _, _, xh, yh) in layers:
-            M.mdbf_linear_forward_host(h, xh.data_ptr(), yh.data_ptr(), T, M.BF16, st)
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
+    e2e_steps = max(1, min(steps, 10))
+    e2e_s = 0.0
+    if want_e2e:
+        for (h, *_r) in layers:
+            M.mdbf_prepare_host_staging(h)
+        for _ in range(2):
+            for (h, sp, _, _, xh, yh) in layers:
+                M.mdbf_linear_forward_host(h, xh.data_ptr(), yh.data_ptr(), T, M.BF16, st)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            for (h, sp, _, _, xh, yh) in layers:
+                M.mdbf_linear_forward_host(h, xh.data_ptr(), yh.data_ptr(), T, M.BF16, st)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
     h2d = sum(T * sp.d_in * 2 for (_, sp, *_r) in layers)
     d2h = sum(T * sp.d_out * 2 for (_, sp, *_r) in layers)
 
@@ -334,41 +382,76 @@ def run_mdbf(args):
     else:
         # the expanded-order kernel is rated in FLOPs of the expanded contraction (which it executes); the
         # materialised-order kernel executes l x fewer and is rated in those, never in expanded FLOPs
-        mat = M.mdbf_last_kernel(layers[0][0]) == M.KERNEL_MAT
-        assert mat == rated_materialised(groups[0][0], T, args.kernel), "bench.py's copy of the dispatch rule is stale"
+        assert mat == rated_materialised(groups[0][0], T, kernel), "bench.py's copy of the dispatch rule is stale"
         metric, unit = ("prefill_executed_TFLOPs" if mat else "prefill_expanded_TFLOPs"), "TFLOP/s"
         per_step = (total_mat_flops if mat else total_flops) / 1e12
         peak = peaks["bf16_tflops"] if sec < 1.0 else peaks["bf16_tflops_sustained"]
-    value = replicas.aggregate_throughput(per_step * args.steps, world, sec)
-    per_gpu = per_step * args.steps / sec
-    e2e_value = replicas.aggregate_throughput(per_step * e2e_steps, world, e2e_ms_max / 1e3)
+    value = replicas.aggregate_throughput(per_step * steps, world, sec)
+    per_gpu = per_step * steps / sec
+    e2e_value = replicas.aggregate_throughput(per_step * e2e_steps, world, e2e_ms_max / 1e3) if want_e2e else None
 
+    dom = dominant_kernel(workload, T, kernels_used, M)
     out = {
-        "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
-        "warmup": max(3, args.warmup), "ms_per_step": ms_max / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "description": desc, "layers": len(layers), "T": T,
+        "metric": metric, "value": value, "unit": unit, "steps": steps, "warmup": max(3, warmup),
+        "ms_per_step": ms_max / steps,
+        "config": {"workload": workload, "description": desc, "layers": len(layers), "T": T,
                    "weights_MB": round(weight_bytes / 1e6, 1),
                    "l2_policy": ("rotation of distinct layers larger than L2" if flush is None
                                  else "256 MiB L2 flush between steps"),
                    "launch": "CUDA graph replay per step" if graph is not None else "stream launches",
-                   "kernel": args.kernel,
+                   "kernel": kernel,
                    "GFLOP_expanded_per_step": round(total_flops / 1e9, 1),
                    "GFLOP_materialised_per_step": round(total_mat_flops / 1e9, 1),
                    "replicas": world},
-        "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h} if want_e2e else None,
         "gpu_launches": launches,
         "clocks": clocks,
         "roofline": {"bound": bound, "achieved": per_gpu, "peak": peak, "unit": unit,
-                     "frac": per_gpu / peak, "peak_source": f"of {peak_kind}",
-                     "kernel": dominant_kernel(groups[0][0], T, "mat" if M.mdbf_last_kernel(layers[0][0]) == M.KERNEL_MAT else "prefill"),
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.workload, dominant_kernel(groups[0][0], T, "mat" if M.mdbf_last_kernel(layers[0][0]) == M.KERNEL_MAT else "prefill")))},
+                     "frac": per_gpu / peak, "peak_source": f"of {peak_kind}", "kernel": dom,
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((workload, dom))},
     }
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(groups[0][0], T, bound, budget_s=20.0,
-                                           mat=bound != "hbm" and M.mdbf_last_kernel(layers[0][0]) == M.KERNEL_MAT)
+    cpu_args = (groups[0][0], T, bound, bound != "hbm" and mat)
     for (h, *_r) in layers:
         M.mdbf_destroy(h)
+    del layers, xs, flush
+    torch.cuda.empty_cache()
+    return out, cpu_args
+
+
+# workloads the default line reports beside the headline one: the largest decode configuration, the MLP shapes at one
+# and at sixteen tokens, the prefill point under the library's own choice and under the expanded order (the metric's
+# own unit), the block prefill
+ALSO = [("block70b_T1", "auto"), ("decode_mlp_T1", "auto"), ("decode_mlp_T16", "auto"), ("prefill_4096_l16_bpw10", "auto"),
+        ("prefill_4096_l16_bpw10", "prefill"), ("block70b_T2048", "auto")]
+
+
+def run_mdbf(args):
+    import torch
+    from paper_2512_24545_b200 import build
+    build.build()
+    dist, rank, world, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    main, cpu_args = measure(args.workload, args.kernel, args.steps, args.warmup, dist, world, local,
+                             no_graph=args.no_graph, no_siblings=args.no_siblings, copies=args.copies)
+    out = {
+        "metric": main["metric"], "value": main["value"], "unit": main["unit"], "n_gpus": world, "steps": main["steps"],
+        "warmup": main["warmup"], "ms_per_step": main["ms_per_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": main["config"], "e2e": main["e2e"], "gpu_launches": main["gpu_launches"], "clocks": main["clocks"],
+        "roofline": main["roofline"],
+    }
+    if world == 1 and args.also and args.workload == "decode_qproj" and args.kernel == "auto":
+        also = {}
+        for (wl, kern) in ALSO:
+            m, _ = measure(wl, kern, max(3, min(args.steps, 10)), args.warmup, None, 1, local, want_e2e=False)
+            also[wl if kern == "auto" else f"{wl}:{kern}"] = {
+                "metric": m["metric"], "value": m["value"], "unit": m["unit"], "ms_per_step": m["ms_per_step"],
+                "steps": m["steps"], "gpu_launches": m["gpu_launches"], "clocks": m["clocks"], "roofline": m["roofline"],
+                "config": {k: m["config"][k] for k in ("layers", "T", "weights_MB", "l2_policy", "kernel")}}
+        out["also"] = also
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        spec0, T, bound, mat0 = cpu_args
+        out["cpu_baseline"] = cpu_baseline(spec0, T, bound, budget_s=20.0, mat=mat0)
     if dist:
         dist.destroy_process_group()
     if rank == 0:
@@ -460,8 +543,11 @@ def main():
     ap.add_argument("--impl", default="mdbf", choices=["mdbf", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every forward from the host")
-    ap.add_argument("--kernel", default="auto", choices=["auto", "prefill", "mat"],
-                    help="T > 1: force the expanded-order (prefill) or the materialised-order (mat) kernel")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "prefill", "mat", "tmem", "i8"],
+                    help="T > 1: force the expanded-order (prefill) or the materialised-order (mat) kernel; "
+                         "T = 1: force the bf16 TMEM-operand (tmem) or the integer (i8) kernel")
+    ap.add_argument("--no-also", dest="also", action="store_false",
+                    help="default workload only: skip the extra workloads reported under \"also\"")
     ap.add_argument("--no-siblings", action="store_true", help="block workloads: one forward per layer instead of fused q/k/v and gate/up")
     ap.add_argument("--copies", type=int, default=0, help="distinct layers per shape (0 = workload default); small values for ncu captures")
     args = ap.parse_args()
