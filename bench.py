@@ -235,7 +235,7 @@ def dist_setup(n_gpus):
 
 # ------------------------------------------------------------------ mdbf arm
 def measure(workload, kernel, steps, warmup, dist, world, local, no_graph=False, no_siblings=False, copies=0,
-            want_e2e=True):
+            want_e2e=True, fuse_block=False):
     """Time `steps` steps of one workload (after >= 3 untimed ones) and return the measured fields."""
     import torch
     from paper_2512_24545_b200 import inputs, mdbf as M, replicas
@@ -299,6 +299,14 @@ def measure(workload, kernel, steps, warmup, dist, world, local, no_graph=False,
                 sib_groups += [[l] for l in blk]
 
     def step():
+        if fuse_block and workload.startswith("block70b") and T == 1:
+            # the seven layers of a block as independent forwards (their inputs are seeded, not produced by one another):
+            # one set of launches per block through the group entry point
+            for b0 in range(0, len(layers), 7):
+                blk = layers[b0:b0 + 7]
+                M.mdbf_linear_forward_group([g[0] for g in blk], [g[2].data_ptr() for g in blk], [g[3].data_ptr() for g in blk],
+                                            T, M.BF16, st)
+            return
         if sib_groups is not None:
             for grp in sib_groups:
                 if len(grp) == 1:
@@ -399,7 +407,7 @@ def measure(workload, kernel, steps, warmup, dist, world, local, no_graph=False,
                    "l2_policy": ("rotation of distinct layers larger than L2" if flush is None
                                  else "256 MiB L2 flush between steps"),
                    "launch": "CUDA graph replay per step" if graph is not None else "stream launches",
-                   "kernel": kernel,
+                   "kernel": kernel, "grouping": ("seven independent forwards per set of launches" if fuse_block else "q/k/v and gate/up as siblings, o and down alone" if sib_groups is not None else "one forward per layer"),
                    "GFLOP_expanded_per_step": round(total_flops / 1e9, 1),
                    "GFLOP_materialised_per_step": round(total_mat_flops / 1e9, 1),
                    "replicas": world},
@@ -421,7 +429,7 @@ def measure(workload, kernel, steps, warmup, dist, world, local, no_graph=False,
 # workloads the default line reports beside the headline one: the largest decode configuration, the MLP shapes at one
 # and at sixteen tokens, the prefill point under the library's own choice and under the expanded order (the metric's
 # own unit), the block prefill
-ALSO = [("block70b_T1", "auto"), ("decode_mlp_T1", "auto"), ("decode_mlp_T16", "auto"), ("prefill_4096_l16_bpw10", "auto"),
+ALSO = [("block70b_T1", "auto"), ("block70b_T1", "fused"), ("decode_mlp_T1", "auto"), ("decode_mlp_T16", "auto"), ("prefill_4096_l16_bpw10", "auto"),
         ("prefill_4096_l16_bpw10", "prefill"), ("block70b_T2048", "auto")]
 
 
@@ -432,7 +440,7 @@ def run_mdbf(args):
     dist, rank, world, local = dist_setup(args.gpus)
     torch.cuda.set_device(local)
     main, cpu_args = measure(args.workload, args.kernel, args.steps, args.warmup, dist, world, local,
-                             no_graph=args.no_graph, no_siblings=args.no_siblings, copies=args.copies)
+                             no_graph=args.no_graph, no_siblings=args.no_siblings, copies=args.copies, fuse_block=args.fuse_block)
     out = {
         "metric": main["metric"], "value": main["value"], "unit": main["unit"], "n_gpus": world, "steps": main["steps"],
         "warmup": main["warmup"], "ms_per_step": main["ms_per_step"], "higher_is_better": True,
@@ -443,11 +451,12 @@ def run_mdbf(args):
     if world == 1 and args.also and args.workload == "decode_qproj" and args.kernel == "auto":
         also = {}
         for (wl, kern) in ALSO:
-            m, _ = measure(wl, kern, max(3, min(args.steps, 10)), args.warmup, None, 1, local, want_e2e=False)
+            m, _ = measure(wl, "auto" if kern == "fused" else kern, max(3, min(args.steps, 10)), args.warmup, None, 1, local,
+                           want_e2e=False, fuse_block=kern == "fused")
             also[wl if kern == "auto" else f"{wl}:{kern}"] = {
                 "metric": m["metric"], "value": m["value"], "unit": m["unit"], "ms_per_step": m["ms_per_step"],
                 "steps": m["steps"], "gpu_launches": m["gpu_launches"], "clocks": m["clocks"], "roofline": m["roofline"],
-                "config": {k: m["config"][k] for k in ("layers", "T", "weights_MB", "l2_policy", "kernel")}}
+                "config": {k: m["config"][k] for k in ("layers", "T", "weights_MB", "l2_policy", "kernel", "grouping")}}
         out["also"] = also
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         spec0, T, bound, mat0 = cpu_args
@@ -546,6 +555,8 @@ def main():
     ap.add_argument("--kernel", default="auto", choices=["auto", "prefill", "mat", "tmem", "i8"],
                     help="T > 1: force the expanded-order (prefill) or the materialised-order (mat) kernel; "
                          "T = 1: force the bf16 TMEM-operand (tmem) or the integer (i8) kernel")
+    ap.add_argument("--fuse-block", action="store_true",
+                    help="block workloads at one token: the seven layers as independent forwards in one set of launches")
     ap.add_argument("--no-also", dest="also", action="store_false",
                     help="default workload only: skip the extra workloads reported under \"also\"")
     ap.add_argument("--no-siblings", action="store_true", help="block workloads: one forward per layer instead of fused q/k/v and gate/up")

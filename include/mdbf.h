@@ -187,6 +187,18 @@ mdbf_status_t mdbf_linear_forward_sum(const mdbf_handle_t *terms, int32_t P, con
 mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t n, const void *x, void *const *ys,
                                            int32_t T, int32_t act_dtype, void *stream);
 
+/* Independent layers, each with its own input: ys[i] = W_hat_i xs[i] for n layers whose forwards do not depend on
+ * one another (projections of different requests, or of different places of a model whose inputs are all at hand).
+ * The arithmetic is n forwards of Eq. DBF-inference-form / Eq. me-dbf-expand; only the launch structure changes:
+ * with one token, bf16 activations and layers of equal envelope-rank bucket (l <= 16, 16-bit envelopes) up to
+ * eight layers share the four launches of the integer one-token kernel (operand images and contraction, per stage),
+ * every CTA walking its share of every layer, so that the fixed cost of a forward is paid once and small layers no
+ * longer leave SMs idle.  Otherwise the layers run one after the other, exactly as n calls of mdbf_linear_forward.
+ *   layers  n distinct handles          xs, ys  n device pointers each: xs[i] is T x d_in_i, ys[i] is T x d_out_i
+ * Asynchronous on `stream`, allocates nothing.  Errors: INVALID_ARG, SHAPE, DTYPE, CUDA. */
+mdbf_status_t mdbf_linear_forward_group(const mdbf_handle_t *layers, int32_t n, const void *const *xs, void *const *ys,
+                                        int32_t T, int32_t act_dtype, void *stream);
+
 /* Device staging buffers for mdbf_linear_forward_host (max_T * (d_in + d_out) * 4 bytes): allocated
  * here, once, so that the host-buffer forward itself allocates nothing.  Errors: ALLOC, CUDA. */
 mdbf_status_t mdbf_prepare_host_staging(mdbf_handle_t h);

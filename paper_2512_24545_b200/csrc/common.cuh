@@ -25,8 +25,9 @@ struct MatMaps {
 // Scratch and pack-time constants of the one-token kernel (forward_t1.cu); index 0 = stage B, 1 = stage A.
 struct T1Buffers {
     float *vmax;                  // [2][32] max_c |V[c][t]| per stage and mode
-    unsigned int *sync;           // scalars of a forward: column sums of the fixed-point operand, max |x|, max |z|
+    unsigned int *sync;           // scalars of a forward: max |x|, max |z|
     int8_t *img[2];               // operand images [Np][NB][128]
+    int *colsum[2];               // column sums of the images' fixed-point values [Np][32]
     unsigned long long *acc64[2]; // fixed-point sums of the partial outputs of split row blocks [R * 128] (zero between launches)
     int R[2], RG[2], Np[2];       // row blocks, groups of four row blocks, pairs of K blocks
     int NB, ctas;

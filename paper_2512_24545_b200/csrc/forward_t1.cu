@@ -18,8 +18,8 @@
 //
 //     sum_c S[r][c] q[c][t] = sum_c q[c][t]  -  2 * sum_c b[r][c] q[c][t]
 //
-// the row-independent first term (column sums of q, accumulated as 64-bit integers while the operand is
-// built) is added when a row is finalised.  The accumulators are int32 and exact, so the only roundings
+// the row-independent first term (column sums of q, stored per pair of K blocks beside the images) is added by
+// every segment for the pairs it covers.  The accumulators are int32 and exact, so the only roundings
 // of the path are the fixed-point step (2^-21 of the operand's range) and the final store.  The B operand
 // ("image" of a pair of K blocks: N rows x 128 bytes, K-major, 128B swizzle) is built once per stage and
 // shared by every row block.
@@ -70,14 +70,11 @@ constexpr int kSignSlots = 8;                      // sign ring: 8 KB per slot (
 constexpr int kImgSlots = 8;                       // image ring
 constexpr int kIssuers = 8;                        // two per row block of the unit: even and odd units
 constexpr int kThreads = (4 * 4 + 4 + kIssuers + 2) * 32;
-constexpr int kImgThreads = 256;                   // image kernel: 128 builders + 128 more for the pass over the input
+constexpr int kImgThreads = 512;                   // image kernel: 128 builders, all of them for the pass over the input
 
 // word offsets inside a layer's scalar block (uint32 words)
-constexpr int kSyCacc = 0;                         // [2][32] int64: column sums of q per stage and mode while the image kernel adds to them
-constexpr int kSyCtot = 128;                       // [2][32] int64: the finished sums of the last image kernel of the stage
-constexpr int kSyAmax = 256;                       // [2] float bits: max |input| of the stage (stage B: max |x|, stage A: max |z|)
-constexpr int kSyCount = 258;                      // [2] image CTAs of the stage that have finished
-constexpr int kSyWords = 260;
+constexpr int kSyAmax = 0;                         // [2] float bits: max |input| of the stage (stage B: max |x|, stage A: max |z|)
+constexpr int kSyWords = 2;
 
 struct Stage {
     const uint2 *wk2;          // sign words [R][kb_pad][128 rows], 64 bits each
@@ -85,11 +82,11 @@ struct Stage {
     const void *U;             // [rows][l] 16-bit envelope factor the modes are contracted with
     const float *vmax;         // [32] max_c |V[c][t]|
     int8_t *img;               // [Np][NB][128] operand images (scratch, rewritten by every launch)
+    int *colsum;               // [Np][32] column sums of q per pair and mode (scratch, rewritten with the images)
     unsigned long long *acc64; // [R * 128] fixed-point sums of the partial outputs of split groups (zero between launches)
     int rows, cols;
     int R, RG, Np, kb_pad;
-    int chunk;                 // units of this stage of this layer per CTA (each CTA walks its share of every layer, in layer order)
-    int rot;                   // CTA that takes the first share (the next layer starts where this one ended)
+    int unit0;                 // first unit of this stage of this layer among the launch's units of the stage
     int item0;                 // first image of this stage of this layer among the launch's images of the stage
 };
 
@@ -107,6 +104,8 @@ struct Group {
     LayerArgs layer[kMaxLayers];
     int nlayers;
     int items[2];              // images per stage, all layers
+    int units[2], chunk[2];    // units per stage, all layers; units per CTA
+    unsigned shl_mul[8];       // 2^(7 - i): the expanders' left shifts as multiplies by a kernel parameter (FMA pipe, not the ALU pipe)
 };
 
 // ------------------------------------------------------------------ small device helpers
@@ -136,31 +135,32 @@ __device__ __forceinline__ uint32_t make_idesc_i8(int n) {
     return d;
 }
 
-// The segments (group of four row blocks, range of pairs) of one stage that a CTA owns, in order: its share
-// of layer 0, then of layer 1, ...  Share v of a layer is units [v * chunk, (v + 1) * chunk) of its
-// RG x Np units (group-major); CTA c holds share (c - rot) mod C.
+// The segments (group of four row blocks, range of pairs) of one stage that a CTA owns, in order.  The units of the
+// stage, layer after layer and group-major inside a layer, are cut into equal contiguous shares: a CTA meets a
+// segment boundary only where its share crosses from one group of row blocks into the next.
 struct Seg {
     int li, rg, p0, p1, segidx, nseg, nrb;
 };
 struct SegIter {
-    int stage, cta, ncta, li, u, u1, v;
-    __device__ __forceinline__ SegIter(const Group &g, int stage_, int cta_, int ncta_) : stage(stage_), cta(cta_), ncta(ncta_), li(-1), u(0), u1(0), v(0) {}
+    int stage, cta, chunk, u, u1;
+    __device__ __forceinline__ SegIter(const Group &g, int stage_, int cta_, int) : stage(stage_), cta(cta_) {
+        chunk = g.chunk[stage];
+        const int units = g.units[stage];
+        u = min(cta * chunk, units);
+        u1 = min(u + chunk, units);
+    }
     __device__ __forceinline__ bool next(const Group &g, Seg &s) {
-        while (u >= u1) {
-            if (++li >= g.nlayers) return false;
-            const Stage &S = g.layer[li].st[stage];
-            v = cta - S.rot;
-            if (v < 0) v += ncta;
-            const int units = S.RG * S.Np;
-            u = min(v * S.chunk, units);
-            u1 = min(u + S.chunk, units);
-        }
+        if (u >= u1) return false;
+        int li = 0;
+        while (li + 1 < g.nlayers && u >= g.layer[li + 1].st[stage].unit0) ++li;
         const Stage &S = g.layer[li].st[stage];
-        const int rg = u / S.Np;
-        const int p0 = u - rg * S.Np;
+        const int local = u - S.unit0;
+        const int rg = local / S.Np;
+        const int p0 = local - rg * S.Np;
         const int len = min(S.Np - p0, u1 - u);
-        const int first = (rg * S.Np) / S.chunk, last = (rg * S.Np + S.Np - 1) / S.chunk;
-        s.li = li; s.rg = rg; s.p0 = p0; s.p1 = p0 + len; s.segidx = v - first; s.nseg = last - first + 1;
+        const int gstart = S.unit0 + rg * S.Np;
+        const int first = gstart / chunk, last = (gstart + S.Np - 1) / chunk;
+        s.li = li; s.rg = rg; s.p0 = p0; s.p1 = p0 + len; s.segidx = cta - first; s.nseg = last - first + 1;
         s.nrb = min(kRBG, S.R - kRBG * rg);
         u += len;
         return true;
@@ -255,13 +255,13 @@ __device__ __forceinline__ void load_image_inputs(const LayerArgs &L, int s, int
     }
 }
 // tile: where the image goes (the layer's image buffer in global memory, or an image slot of this CTA's
-// shared memory); add_colsum: the one build per pair that feeds the stage's column sums
+// shared memory); cs_out: where the pair's column sums go ([32] ints), or null
 template <int LP>
 __device__ __forceinline__ void build_image(const LayerArgs &L, int s, const float (&in)[4], float amax, int atid, const ImgFactors<LP> &f,
-                                            int8_t *tile, bool add_colsum) {
+                                            int8_t *tile, int *cs_out) {
     constexpr int MT = ImgFactors<LP>::MT;
     const int mg = atid >> 5, lane = atid & 31, wq = lane >> 3, i = lane & 7;
-    long long csum[MT];
+    int csum[MT];                                 // |sum| <= 128 * 2^20
 #pragma unroll
     for (int m = 0; m < MT; ++m) csum[m] = 0;
     if (mg * MT >= LP) return;                    // whole warps only (LP < 4)
@@ -298,14 +298,13 @@ __device__ __forceinline__ void build_image(const LayerArgs &L, int s, const flo
             const int off = n * 128 + (((2 * wq + (i >> 2)) ^ (n & 7)) << 4) + ((i & 3) << 2);
             *reinterpret_cast<uint32_t *>(tile + off) = w[m][j];
         }
-    if (!add_colsum) return;
+    if (!cs_out) return;
 #pragma unroll
     for (int m = 0; m < MT; ++m) {
-        long long v = csum[m];
+        int v = csum[m];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0)
-            atomicAdd(reinterpret_cast<unsigned long long *>(L.sync + kSyCacc) + s * 32 + mg * MT + m, (unsigned long long)v);
+        if (lane == 0) cs_out[mg * MT + m] = v;
     }
 }
 
@@ -368,7 +367,6 @@ template <int LP>
 __global__ void __launch_bounds__(kImgThreads) t1_image_kernel(const __grid_constant__ Group g, const int s) {
     constexpr int IMG = Cfg<LP>::IMG;
     __shared__ float redw[kImgThreads / 32];
-    __shared__ int last_s;
     const int tid = threadIdx.x;
     const int m = blockIdx.x;
     int li = 0;
@@ -384,24 +382,7 @@ __global__ void __launch_bounds__(kImgThreads) t1_image_kernel(const __grid_cons
     if (tid < 128) {
         float in[4];
         load_image_inputs(L, s, p, tid, in);
-        build_image<LP>(L, s, in, amax, tid, fac, L.st[s].img + (size_t)p * IMG, true);
-    }
-    // The CTA of the layer that finishes last moves the column sums to where the stage kernel reads them and clears the
-    // accumulators and the count for the next forward.
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const unsigned old = atomicAdd(L.sync + kSyCount + s, 1u);
-        last_s = old == (unsigned)(L.st[s].Np - 1);
-        __threadfence();
-    }
-    __syncthreads();
-    if (last_s) {
-        if (tid < 32) {
-            unsigned long long *acc = reinterpret_cast<unsigned long long *>(L.sync + kSyCacc) + s * 32 + tid;
-            reinterpret_cast<unsigned long long *>(L.sync + kSyCtot)[s * 32 + tid] = atomicExch(acc, 0ull);
-        }
-        if (tid == 0) L.sync[kSyCount + s] = 0u;
+        build_image<LP>(L, s, in, amax, tid, fac, L.st[s].img + (size_t)p * IMG, L.st[s].colsum + p * 32);
     }
 }
 
@@ -423,6 +404,7 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
     __shared__ __align__(8) uint64_t bars[NBARS];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
+    __shared__ unsigned long long cs_s[32];
     volatile int *abort_flag = &abort_flag_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -495,7 +477,7 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) v[q][i] = (ws[q] << (7 - i)) & 0x80808080u;      // bit 8e + i -> top bit of byte e
+                    for (int i = 0; i < 8; ++i) v[q][i] = (ws[q] * g.shl_mul[i]) & 0x80808080u;   // bit 8e + i -> top bit of byte e
                 // A stage qn % NAG: whatever this row block last put there was consumed by unit qn - NAG at the latest, and
                 // every issuer releases a unit's image with a commit, i.e. after all its earlier MMAs have retired: one
                 // commit per unit and issuer serves both rings.
@@ -551,7 +533,18 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
             float scale[LP];
 #pragma unroll
             for (int t = 0; t < LP; ++t) scale[t] = S.vmax[t];
-            if (nseg_done == 0) pdl_wait();                      // the scalars below are the previous kernel's
+            if (nseg_done == 0) pdl_wait();                      // what follows is the previous kernel's output
+            // column sums of q over the pairs of this segment: warp w takes every fourth pair, lane = mode
+            {
+                aux_sync();                                      // cs_s may still be read from the previous segment
+                if (atid < 32) cs_s[atid] = 0ull;
+                aux_sync();
+                long long v = 0;
+                if ((atid & 31) < LP)
+                    for (int p = sg.p0 + (atid >> 5); p < sg.p1; p += 4) v += __ldcg(S.colsum + p * 32 + (atid & 31));
+                if ((atid & 31) < LP) atomicAdd(&cs_s[atid & 31], (unsigned long long)v);
+                aux_sync();
+            }
             const float am = __uint_as_float(__ldcg(L.sync + kSyAmax + s)) * (1.f / kQmax);
 #pragma unroll
             for (int t = 0; t < LP; ++t) scale[t] *= am;
@@ -560,31 +553,33 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
             if (*abort_flag) { alive = false; break; }
             tc_fence_after();
             if (warp == W_AUX) TR(4);
-            float part[kRBG];
+            // First only what needs the accumulators: per row block the three digits of every mode combined into one float,
+            // f[j][t] = -2 * sum_c b q[c][t] (the A bytes are 128 b: -2 * 128^digit / 128), and the accumulator cleared; then
+            // the issuers may start the next segment while the contraction with U and the hand-over run here.
+            float f[kRBG][LP];
 #pragma unroll
             for (int j = 0; j < kRBG; ++j) {
-                part[j] = 0.f;
+#pragma unroll
+                for (int t = 0; t < LP; ++t) f[j][t] = 0.f;
                 if (j < sg.nrb) {
-                    // f[t] = -2 * sum_c b q[c][t] = sum over the three digits of -2 * 128^digit / 128 * D (the A bytes are 128 b)
-                    float f[Cfg<LP>::NB];
 #pragma unroll
                     for (int c16 = 0; c16 < NB / 16; ++c16) {
                         uint32_t d[16];
                         tmem_ld16(tmem + lane_base + (uint32_t)(j * NB + c16 * 16), d);
                         tmem_ld_wait();
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) f[c16 * 16 + e] = (float)(int)d[e];
                         const uint32_t zero[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
                         tmem_st8(tmem + lane_base + (uint32_t)(j * NB + c16 * 16), zero);
                         tmem_st8(tmem + lane_base + (uint32_t)(j * NB + c16 * 16 + 8), zero);
-                    }
-                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int t = 0; t < LP; ++t) {
-                        const float ft = fmaf(-256.f, f[2 * LP + t], fmaf(-2.f, f[LP + t], -0.015625f * f[t]));
-                        acc[t & 3] = fmaf(env16_to_float(urow[j].get(t), L.env_dtype) * scale[t], ft, acc[t & 3]);
+                        for (int e = 0; e < 16; ++e) {
+                            const int col = c16 * 16 + e;
+                            if (col < 3 * LP) {
+                                const int jd = col / LP, t = col % LP;
+                                const float wgt = jd == 0 ? -0.015625f : jd == 1 ? -2.f : -256.f;
+                                f[j][t] = fmaf(wgt, (float)(int)d[e], f[j][t]);
+                            }
+                        }
                     }
-                    part[j] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
                 }
             }
             if (warp == W_AUX) TR(24);
@@ -593,6 +588,16 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty);               // read and cleared: the issuers may start the next segment
             ++nseg_done;
+
+            float part[kRBG];
+#pragma unroll
+            for (int j = 0; j < kRBG; ++j) {
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int t = 0; t < LP; ++t)                     // contraction with U; + sum_c q over the segment's pairs (S = 1 - 2 b)
+                    acc[t & 3] = fmaf(env16_to_float(urow[j].get(t), L.env_dtype) * scale[t], f[j][t] + (float)(long long)cs_s[t], acc[t & 3]);
+                part[j] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+            }
 
             // A group split over several CTAs.  Every segment adds, per row, its partial output as a fixed-point number in
             // the upper 56 bits of the row's 64-bit accumulator and 1 in the lower 8 (integer addition: the order of
@@ -633,30 +638,10 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                     }
             }
             if (warp == W_AUX) TR(25);
-            // the row-independent term: column sums of q, complete since the image kernel ended
-            if (fin[0] || fin[1] || fin[2] || fin[3]) {
-                const unsigned long long *ct = reinterpret_cast<const unsigned long long *>(L.sync + kSyCtot) + s * 32;
-                float cs[LP];
-#pragma unroll
-                for (int t = 0; t < LP; ++t) cs[t] = (float)(long long)__ldcg(ct + t);
-#pragma unroll
-                for (int t = 0; t < LP; ++t) cs[t] *= scale[t];
-#pragma unroll
-                for (int j = 0; j < kRBG; ++j)
-#pragma unroll
-                    for (int t = 0; t < LP; ++t) part[j] = fmaf(env16_to_float(urow[j].get(t), L.env_dtype), cs[t], part[j]);
-            }
             if (s == 0) {
-                float m = 0.f;
 #pragma unroll
                 for (int j = 0; j < kRBG; ++j)
-                    if (fin[j]) {
-                        L.z[(sg.rg * kRBG + j) * 128 + atid] = part[j];
-                        m = fmaxf(m, fabsf(part[j]));
-                    }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-                (void)m;
+                    if (fin[j]) L.z[(sg.rg * kRBG + j) * 128 + atid] = part[j];
             } else {
 #pragma unroll
                 for (int j = 0; j < kRBG; ++j)
@@ -840,6 +825,8 @@ mdbf_status_t t1_prepare(Layer &L, cudaStream_t st) {
     for (int s = 0; s < 2; ++s) {
         MDBF_CUDA(cudaMalloc(&b.img[s], (size_t)b.Np[s] * NB * 128));
         MDBF_CUDA(cudaMemsetAsync(b.img[s], 0, (size_t)b.Np[s] * NB * 128, st));      // the padding rows stay zero
+        MDBF_CUDA(cudaMalloc(&b.colsum[s], (size_t)b.Np[s] * 32 * sizeof(int)));
+        MDBF_CUDA(cudaMemsetAsync(b.colsum[s], 0, (size_t)b.Np[s] * 32 * sizeof(int), st));
         MDBF_CUDA(cudaMalloc(&b.acc64[s], (size_t)b.R[s] * 128 * sizeof(unsigned long long)));
         MDBF_CUDA(cudaMemsetAsync(b.acc64[s], 0, (size_t)b.R[s] * 128 * sizeof(unsigned long long), st));
     }
@@ -852,7 +839,7 @@ mdbf_status_t t1_prepare(Layer &L, cudaStream_t st) {
 
 void t1_release(Layer &L) {
     T1Buffers &b = L.t1;
-    void *ptrs[] = {b.vmax, b.sync, b.img[0], b.img[1], b.acc64[0], b.acc64[1]};
+    void *ptrs[] = {b.vmax, b.sync, b.img[0], b.img[1], b.colsum[0], b.colsum[1], b.acc64[0], b.acc64[1]};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     b = T1Buffers{};
@@ -901,8 +888,8 @@ mdbf_status_t launch_forward_t1_group(Layer *const *Ls, int n, const void *const
     if (n < 1 || n > t1::kMaxLayers) { set_error("one-token kernel: %d layers in one launch (at most %d)", n, t1::kMaxLayers); return MDBF_ERR_SHAPE; }
     t1::Group grp = {};
     grp.nlayers = n;
+    for (int i = 0; i < 8; ++i) grp.shl_mul[i] = 128u >> i;
     const int C = Ls[0]->t1.ctas;
-    int rot[2] = {0, 0};
     for (int i = 0; i < n; ++i) {
         Layer &L = *Ls[i];
         if (!t1_supports(L) || L.LP != Ls[0]->LP || L.t1.ctas != C) { set_error("one-token kernel: layer %d was not prepared for it", i); return MDBF_ERR_INVALID_ARG; }
@@ -915,15 +902,15 @@ mdbf_status_t launch_forward_t1_group(Layer *const *Ls, int n, const void *const
             S.U = s ? L.UA : L.UB;
             S.vmax = b.vmax + 32 * s;
             S.img = b.img[s];
+            S.colsum = b.colsum[s];
             S.acc64 = b.acc64[s];
             S.rows = s ? L.d.d_out : L.d.k;
             S.cols = s ? L.d.k : L.d.d_in;
             S.R = b.R[s]; S.RG = b.RG[s]; S.Np = b.Np[s];
             S.kb_pad = s ? L.kbpA : L.kbpB;
-            S.chunk = ceil_div(S.RG * S.Np, C);
-            S.rot = rot[s];
-            rot[s] = (rot[s] + ceil_div(S.RG * S.Np, S.chunk)) % C;
+            S.unit0 = grp.units[s];
             S.item0 = grp.items[s];
+            grp.units[s] += S.RG * S.Np;
             grp.items[s] += S.Np;
         }
         a.x = xs[i];
@@ -933,6 +920,7 @@ mdbf_status_t launch_forward_t1_group(Layer *const *Ls, int n, const void *const
         a.status = L.status;
         a.l = L.d.l; a.env_dtype = L.d.env_dtype; a.out_mode = L.out_mode;
     }
+    for (int s = 0; s < 2; ++s) grp.chunk[s] = ceil_div(grp.units[s], C);
     switch (Ls[0]->LP) {
         case 1: return t1_launch<1>(grp, C, st, stages);
         case 2: return t1_launch<2>(grp, C, st, stages);

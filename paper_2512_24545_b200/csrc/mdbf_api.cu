@@ -637,6 +637,52 @@ mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void
     return MDBF_OK;
 }
 
+mdbf_status_t mdbf_linear_forward_group(const mdbf_handle_t *layers, int32_t n, const void *const *xs, void *const *ys,
+                                        int32_t T, int32_t act_dtype, void *stream) {
+    if (!layers || !xs || !ys) { set_error("mdbf_linear_forward_group: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    if (n < 1 || n > 64) { set_error("mdbf_linear_forward_group: n=%d outside [1, 64]", n); return MDBF_ERR_SHAPE; }
+    if (!valid_dtype(act_dtype)) { set_error("mdbf_linear_forward_group: bad act_dtype %d", act_dtype); return MDBF_ERR_DTYPE; }
+    bool fusable = T == 1 && act_dtype == MDBF_BF16;
+    for (int i = 0; i < n; ++i) {
+        mdbf_status_t rc = check_handle(layers[i], "mdbf_linear_forward_group");
+        if (rc) return rc;
+        if (!xs[i] || !ys[i]) { set_error("mdbf_linear_forward_group: NULL input or output %d", i); return MDBF_ERR_INVALID_ARG; }
+        const Layer &L = layers[i]->L;
+        rc = check_device(L, "mdbf_linear_forward_group");
+        if (rc) return rc;
+        if (T < 1 || T > L.d.max_T) {
+            set_error("mdbf_linear_forward_group: T=%d outside [1, max_T=%d] of layer %d", T, L.d.max_T, i);
+            return MDBF_ERR_SHAPE;
+        }
+        for (int q = 0; q < i; ++q)
+            if (layers[q] == layers[i]) { set_error("mdbf_linear_forward_group: layer %d repeats layer %d", i, q); return MDBF_ERR_INVALID_ARG; }
+        fusable = fusable && t1_supports(L) && L.LP == layers[0]->L.LP &&
+                  (layers[i]->kernel == MDBF_KERNEL_AUTO || layers[i]->kernel == MDBF_KERNEL_I8);
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!fusable || n == 1) {
+        for (int i = 0; i < n; ++i) {
+            mdbf_status_t rc = forward_impl(layers[i], xs[i], ys[i], T, act_dtype, st);
+            if (rc) return rc;
+        }
+        return MDBF_OK;
+    }
+    for (int i0 = 0; i0 < n; i0 += 8) {                  // up to eight layers per set of four launches
+        const int m = n - i0 < 8 ? n - i0 : 8;
+        Layer *Ls[8];
+        for (int i = 0; i < m; ++i) {
+            Ls[i] = &layers[i0 + i]->L;
+            Ls[i]->out_mode = 0;
+            Ls[i]->last_ksplit = 0;
+            layers[i0 + i]->last_launches = i == 0 ? 4 : 0;
+            layers[i0 + i]->last_kernel = MDBF_KERNEL_I8;
+        }
+        mdbf_status_t rc = launch_forward_t1_group(Ls, m, xs + i0, ys + i0, st, 3);
+        if (rc) return rc;
+    }
+    return MDBF_OK;
+}
+
 mdbf_status_t mdbf_prepare_host_staging(mdbf_handle_t h) {
     mdbf_status_t rc = check_handle(h, "mdbf_prepare_host_staging");
     if (rc) return rc;

@@ -28,7 +28,7 @@ DTYPES = {"f32": F32, "f16": F16, "bf16": BF16}
 EXPORTS = (
     "mdbf_pack_signs", "mdbf_unpack_signs", "mdbf_pack", "mdbf_get_packed", "mdbf_get_envelope",
     "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host", "mdbf_prepare_host_staging",
-    "mdbf_linear_forward_static", "mdbf_linear_forward_sum", "mdbf_linear_forward_siblings",
+    "mdbf_linear_forward_static", "mdbf_linear_forward_sum", "mdbf_linear_forward_siblings", "mdbf_linear_forward_group",
     "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_poll_status", "mdbf_selftest_wait_timeout",
     "mdbf_last_launch_count",
     "mdbf_last_kernel",
@@ -75,6 +75,7 @@ def lib() -> ctypes.CDLL:
     L.mdbf_linear_forward_static.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, vp]
     L.mdbf_linear_forward_sum.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp]
     L.mdbf_linear_forward_siblings.argtypes = [vp, i32, vp, vp, i32, i32, vp]
+    L.mdbf_linear_forward_group.argtypes = [vp, i32, vp, vp, i32, i32, vp]
     L.mdbf_get_intermediate.argtypes = [vp, vp, i32, ctypes.c_int, vp]
     L.mdbf_reconstruct.argtypes = [vp, vp, vp]
     L.mdbf_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
@@ -169,6 +170,15 @@ def mdbf_linear_forward_siblings(handles, x, ys, T: int, act_dtype: int, stream:
     outs = (ctypes.c_void_p * len(ys))(*[_addr(y) for y in ys])
     _check(lib().mdbf_linear_forward_siblings(ctypes.cast(hs, ctypes.c_void_p), len(handles), _addr(x),
                                               ctypes.cast(outs, ctypes.c_void_p), T, act_dtype, stream))
+
+
+def mdbf_linear_forward_group(handles, xs, ys, T: int, act_dtype: int, stream: int = 0) -> None:
+    """ys[i] = W_hat_i xs[i] for independent layers (own inputs); xs, ys are device addresses."""
+    hs = (ctypes.c_void_p * len(handles))(*handles)
+    ins = (ctypes.c_void_p * len(xs))(*[_addr(x) for x in xs])
+    outs = (ctypes.c_void_p * len(ys))(*[_addr(y) for y in ys])
+    _check(lib().mdbf_linear_forward_group(ctypes.cast(hs, ctypes.c_void_p), len(handles), ctypes.cast(ins, ctypes.c_void_p),
+                                           ctypes.cast(outs, ctypes.c_void_p), T, act_dtype, stream))
 
 
 def mdbf_prepare_host_staging(h: int) -> None:

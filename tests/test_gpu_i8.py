@@ -133,3 +133,45 @@ def test_stages_mix_kernels(big_stage):
         y8 = g.forward(x, kernel=M.KERNEL_I8)
         assert rel_err(y8[:, rows], ref) <= TOL["bf16"]
         assert rel_err(y, y8) <= 2 * TOL["bf16"]
+
+
+def test_group_of_independent_layers():
+    """mdbf_linear_forward_group: layers with their own inputs (different d_in) in one set of four launches; each
+    output is that layer's forward, bit for bit what the layer gives alone through the same kernel."""
+    shapes = [(300, 640, 200), (1024, 384, 512), (130, 2048, 131), (700, 640, 1100), (64, 128, 64)]
+    specs = [inputs.scaled(inputs.qproj(1664), name=f"grp{i}", d_out=do, d_in=di, k=k, l=16, seed=90 + i)
+             for i, (do, di, k) in enumerate(shapes)]
+    layers = [GpuLayer(sp, 1) for sp in specs]
+    try:
+        xs = [inputs.make_activations(sp, 1) for sp in specs]
+        xd = [torch.from_numpy(x).to(torch.bfloat16).cuda() for x in xs]
+        ys = [torch.full((1, sp.d_out), float("nan"), dtype=torch.bfloat16, device="cuda") for sp in specs]
+        M.mdbf_linear_forward_group([g.h for g in layers], [x.data_ptr() for x in xd], [y.data_ptr() for y in ys], 1, M.BF16,
+                                    torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert M.mdbf_last_launch_count(layers[0].h) == 4 and M.mdbf_last_kernel(layers[0].h) == M.KERNEL_I8
+        for g, x, y in zip(layers, xs, ys):
+            assert M.mdbf_poll_status(g.h) == 0
+            got = y.to(torch.float32).cpu().numpy()
+            check_parity(g, x, got, roundings=1)
+            np.testing.assert_array_equal(got, g.forward(x, kernel=M.KERNEL_I8))
+        # three tokens: the same call runs the layers one after the other
+        layers3 = [GpuLayer(sp, 3) for sp in specs[:2]]
+        try:
+            x3 = [inputs.make_activations(sp, 3) for sp in specs[:2]]
+            xd3 = [torch.from_numpy(x).to(torch.bfloat16).cuda() for x in x3]
+            y3 = [torch.zeros((3, sp.d_out), dtype=torch.bfloat16, device="cuda") for sp in specs[:2]]
+            M.mdbf_linear_forward_group([g.h for g in layers3], [x.data_ptr() for x in xd3], [y.data_ptr() for y in y3], 3, M.BF16,
+                                        torch.cuda.current_stream().cuda_stream)
+            torch.cuda.synchronize()
+            for g, x, y in zip(layers3, x3, y3):
+                check_parity(g, x, y.to(torch.float32).cpu().numpy())
+        finally:
+            for g in layers3:
+                g.close()
+        with pytest.raises(M.MdbfError) as e:
+            M.mdbf_linear_forward_group([layers[0].h, layers[0].h], [xd[0].data_ptr()] * 2, [ys[0].data_ptr()] * 2, 1, M.BF16)
+        assert e.value.status == M.ERR_INVALID_ARG
+    finally:
+        for g in layers:
+            g.close()
