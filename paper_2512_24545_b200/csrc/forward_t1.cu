@@ -450,6 +450,7 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         bool alive = true;
         int qn = 0;                                              // units this CTA has walked
+        int prev_as = -1;                                        // A stage whose stores are still to be published
         TRC_DECL;
         SegIter it(g, s, cta, (int)gridDim.x);
         Seg sg;
@@ -469,15 +470,22 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(s_empty + 8 * rs);
+                if (prev_as >= 0) {                              // publish the previous unit: its stores had a unit's time to land
+                    tmem_st_wait();                              // (before the validity test: the row block may not exist in this unit)
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(a_full + 8 * (grp * NAG + prev_as));
+                    prev_as = -1;
+                }
                 if (!valid) continue;
                 // the 32 operand words of this row are finished in registers before the A stage is claimed (the MMAs of
                 // the unit that used the stage two units ago may still run): only the stores follow the wait
                 const uint32_t ws[4] = {w0.x, w0.y, w1.x, w1.y};
-                uint32_t v[4][8];
+                uint32_t v[32];                                  // sign word q -> TMEM columns 8q .. 8q+7
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) v[q][i] = (ws[q] * g.shl_mul[i]) & 0x80808080u;   // bit 8e + i -> top bit of byte e
+                    for (int i = 0; i < 8; ++i) v[8 * q + i] = (ws[q] * g.shl_mul[i]) & 0x80808080u;   // bit 8e + i -> top bit of byte e
                 // A stage qn % NAG: whatever this row block last put there was consumed by unit qn - NAG at the latest, and
                 // every issuer releases a unit's image with a commit, i.e. after all its earlier MMAs have retired: one
                 // commit per unit and issuer serves both rings.
@@ -491,15 +499,17 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                 TRC(2);
                 tc_fence_after();
                 const uint32_t a_col = tmem_a0 + lane_base + (uint32_t)((grp * NAG + as) * 32);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) tmem_st8(a_col + (uint32_t)(8 * q), v[q]);          // sign word q -> TMEM columns 8q .. 8q+7
-                tmem_st_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(a_full + 8 * (grp * NAG + as));
+                tmem_st32(a_col, v);                             // one store of the whole row: a tcgen05.st holds the warp for ~140 clocks whatever its width
+                prev_as = as;
             }
         }
-        if (warp == 0) { TR(11); }
+        if (prev_as >= 0) {
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (alive && lane == 0) mbar_arrive(a_full + 8 * (grp * NAG + prev_as));
+        }
+        if (warp == 0) { TR(11); TRC_OUT(28); }
     } else if (warp < W_ISS) {
         // ============================ epilogue warps: contraction with U, row finalisation ============================
         const int atid = tid - W_AUX * 32;                       // 0 .. 127 = row of the tile = TMEM lane
@@ -711,7 +721,7 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
             __syncwarp();
             ++nseg_done;
         }
-        if (warp == W_ISS) TRC_OUT(28);
+        if (warp == W_ISS) { }
     } else if (warp == W_SLOAD) {
         // ================================= sign-word loader ==================================
         // Lane l owns ring slot l: it waits for the slot, then issues the (up to) four bulk copies of its unit.  Sign

@@ -99,7 +99,8 @@ def run_siblings(specs, x, kernel):
         raise
 
 
-@pytest.mark.parametrize("shapes", [[(300, 200), (128, 64)], [(1024, 512), (130, 128), (131, 64), (700, 1100)]])
+@pytest.mark.parametrize("shapes", [[(300, 200), (128, 64)], [(1024, 512), (130, 128), (131, 64), (700, 1100)],
+                                    [(640, 640), (2048, 384), (1400, 896), (512, 1152)]])   # row blocks not a multiple of four between full groups
 def test_i8_kernel_several_layers_per_launch(shapes):
     """Sibling layers in one set of launches: every CTA walks its share of every layer; layers of different d_out and k."""
     specs = [inputs.scaled(inputs.qproj(1664), name=f"i8s{i}", d_out=do, d_in=640, k=k, l=16, seed=70 + i)
