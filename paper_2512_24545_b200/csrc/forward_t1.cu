@@ -139,30 +139,48 @@ __device__ __forceinline__ uint32_t make_idesc_i8(int n) {
 // stage, layer after layer and group-major inside a layer, are cut into equal contiguous shares: a CTA meets a
 // segment boundary only where its share crosses from one group of row blocks into the next.
 struct Seg {
-    int li, rg, p0, p1, segidx, nseg, nrb;
+    int li, rg, p0, p1, nseg, nrb;
 };
+// A CTA's share [u, u1) of the stage's units, cut at the group boundaries it contains.  The last segment's epilogue
+// is the only one nothing hides, and a segment's epilogue cannot start before the previous one's has ended: when the
+// share ends in a segment shorter than the one it starts with, the CTA walks its share backwards, so that the short
+// segment's epilogue runs under the long one's streaming.  (Partial sums are added as integers: any order will do.)
 struct SegIter {
-    int stage, cta, chunk, u, u1;
-    __device__ __forceinline__ SegIter(const Group &g, int stage_, int cta_, int) : stage(stage_), cta(cta_) {
+    int stage, chunk, u, u1;
+    bool backwards;
+    struct Where { int li, rg, p, gstart, Np, R; };
+    __device__ __forceinline__ Where locate(const Group &g, int unit) const {
+        int li = 0;
+        while (li + 1 < g.nlayers && unit >= g.layer[li + 1].st[stage].unit0) ++li;
+        const Stage &S = g.layer[li].st[stage];
+        const int local = unit - S.unit0;
+        Where w;
+        w.li = li; w.Np = S.Np; w.R = S.R;
+        w.rg = local / S.Np;
+        w.p = local - w.rg * S.Np;
+        w.gstart = S.unit0 + w.rg * S.Np;
+        return w;
+    }
+    __device__ __forceinline__ SegIter(const Group &g, int stage_, int cta, int) : stage(stage_) {
         chunk = g.chunk[stage];
         const int units = g.units[stage];
         u = min(cta * chunk, units);
         u1 = min(u + chunk, units);
+        backwards = false;
+        if (u < u1) {
+            const Where a = locate(g, u), b = locate(g, u1 - 1);
+            const int first_len = min(a.gstart + a.Np, u1) - u, last_len = u1 - max(b.gstart, u);
+            backwards = last_len < first_len;
+        }
     }
     __device__ __forceinline__ bool next(const Group &g, Seg &s) {
         if (u >= u1) return false;
-        int li = 0;
-        while (li + 1 < g.nlayers && u >= g.layer[li + 1].st[stage].unit0) ++li;
-        const Stage &S = g.layer[li].st[stage];
-        const int local = u - S.unit0;
-        const int rg = local / S.Np;
-        const int p0 = local - rg * S.Np;
-        const int len = min(S.Np - p0, u1 - u);
-        const int gstart = S.unit0 + rg * S.Np;
-        const int first = gstart / chunk, last = (gstart + S.Np - 1) / chunk;
-        s.li = li; s.rg = rg; s.p0 = p0; s.p1 = p0 + len; s.segidx = cta - first; s.nseg = last - first + 1;
-        s.nrb = min(kRBG, S.R - kRBG * rg);
-        u += len;
+        const Where w = locate(g, backwards ? u1 - 1 : u);
+        const int lo = max(w.gstart, u), hi = min(w.gstart + w.Np, u1);     // the part of this group inside the share
+        const int first = w.gstart / chunk, last = (w.gstart + w.Np - 1) / chunk;
+        s.li = w.li; s.rg = w.rg; s.p0 = lo - w.gstart; s.p1 = hi - w.gstart; s.nseg = last - first + 1;
+        s.nrb = min(kRBG, w.R - kRBG * w.rg);
+        if (backwards) u1 = lo; else u = hi;
         return true;
     }
 };
@@ -360,11 +378,13 @@ __device__ __forceinline__ float amax_f32_block(const float *z, int n, float *re
 }
 
 // ------------------------------------------------------------------------ image kernel
-// One CTA per pair of K blocks of every layer of the launch (stage s): the operand images of the stage.
-// Every CTA makes its own pass over the stage's input (x, or the intermediate z) for its largest magnitude: a few
-// KB out of L2, cheaper than a reduction across CTAs, and independent of which kernel produced the input.
+// One CTA per pair of K blocks of every layer of the launch (stage s): the operand images of the stage (four pairs
+// per CTA measured 2-9 % slower on the 70B-class block).
+// Every CTA makes its own pass over the stage's input (x, or an intermediate z that another kernel produced) for its
+// largest magnitude: a few KB out of L2, cheaper than a reduction across CTAs.  The stage kernel of this file leaves
+// max |z| behind (one atomic maximum per warp of finished rows), so stage A after it skips the pass.
 template <int LP>
-__global__ void __launch_bounds__(kImgThreads) t1_image_kernel(const __grid_constant__ Group g, const int s) {
+__global__ void __launch_bounds__(kImgThreads) t1_image_kernel(const __grid_constant__ Group g, const int s, const int have_amax) {
     constexpr int IMG = Cfg<LP>::IMG;
     __shared__ float redw[kImgThreads / 32];
     const int tid = threadIdx.x;
@@ -372,18 +392,24 @@ __global__ void __launch_bounds__(kImgThreads) t1_image_kernel(const __grid_cons
     int li = 0;
     while (li + 1 < g.nlayers && m >= g.layer[li + 1].st[s].item0) ++li;
     const LayerArgs &L = g.layer[li];
+    const int atid = tid & 127;
     const int p = m - L.st[s].item0;
+    const bool builds = tid < 128;
     tm::pdl_launch_dependents();
     ImgFactors<LP> fac;
-    if (tid < 128) load_image_factors<LP>(L, s, p, tid, fac);    // immutable: in flight while the previous kernel drains
+    if (builds) load_image_factors<LP>(L, s, p, atid, fac);      // immutable: in flight while the previous kernel drains
     tm::pdl_wait();
-    const float amax = s == 0 ? amax_bf16_block(L.x, L.st[0].cols, redw) : amax_f32_block(L.z, L.st[1].cols, redw);
-    if (p == 0 && tid == 0) L.sync[kSyAmax + s] = __float_as_uint(amax);
-    if (tid < 128) {
-        float in[4];
-        load_image_inputs(L, s, p, tid, in);
-        build_image<LP>(L, s, in, amax, tid, fac, L.st[s].img + (size_t)p * IMG, L.st[s].colsum + p * 32);
+    float in[4] = {0.f, 0.f, 0.f, 0.f};
+    if (builds) load_image_inputs(L, s, p, atid, in);            // requested before the pass below: one round trip, not two
+    float amax;
+    if (have_amax) {                                             // stage A after this file's stage B: its epilogue left max |z|
+        amax = __uint_as_float(__ldcg(L.sync + kSyAmax + 1));
+    } else {
+        amax = s == 0 ? amax_bf16_block(L.x, L.st[0].cols, redw) : amax_f32_block(L.z, L.st[1].cols, redw);
+        if (p == 0 && atid == 0) L.sync[kSyAmax + s] = __float_as_uint(amax);
     }
+    if (s == 0 && p == 0 && atid == 0) L.sync[kSyAmax + 1] = 0u; // stage B's epilogue takes the maximum into it
+    if (builds) build_image<LP>(L, s, in, amax, atid, fac, L.st[s].img + (size_t)p * IMG, L.st[s].colsum + p * 32);
 }
 
 // ------------------------------------------------------------------------ stage kernel
@@ -510,6 +536,9 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
             if (alive && lane == 0) mbar_arrive(a_full + 8 * (grp * NAG + prev_as));
         }
         if (warp == 0) { TR(11); TRC_OUT(28); }
+#ifdef MDBF_T1_TRACE
+        if (warp == 0 && lane == 0) g_t1_trace[cta * 32 + 27] = (unsigned long long)qn;
+#endif
     } else if (warp < W_ISS) {
         // ============================ epilogue warps: contraction with U, row finalisation ============================
         const int atid = tid - W_AUX * 32;                       // 0 .. 127 = row of the tile = TMEM lane
@@ -649,9 +678,16 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
             }
             if (warp == W_AUX) TR(25);
             if (s == 0) {
+                float zmax = 0.f;
 #pragma unroll
                 for (int j = 0; j < kRBG; ++j)
-                    if (fin[j]) L.z[(sg.rg * kRBG + j) * 128 + atid] = part[j];
+                    if (fin[j]) {
+                        L.z[(sg.rg * kRBG + j) * 128 + atid] = part[j];
+                        zmax = fmaxf(zmax, fabsf(part[j]));
+                    }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+                if (lane == 0 && zmax > 0.f) atomicMax(L.sync + kSyAmax + 1, __float_as_uint(zmax));   // non-negative floats order like their bits
             } else {
 #pragma unroll
                 for (int j = 0; j < kRBG; ++j)
@@ -664,6 +700,9 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
             }
             if (warp == W_AUX) TR(5);
         }
+#ifdef MDBF_T1_TRACE
+        if (warp == W_AUX && lane == 0) g_t1_trace[cta * 32 + 26] = (unsigned long long)nseg_done;
+#endif
     } else if (warp < W_SLOAD) {
         // ==================================== MMA issuers ====================================
         // Two issuers per row block of the unit, one for the even and one for the odd units (= A stage 0 / 1): while one
@@ -857,8 +896,8 @@ void t1_release(Layer &L) {
 
 bool t1_supports(const Layer &L) { return L.t1.sync != nullptr && L.wk2A != nullptr && L.LP <= 16 && L.d.d_in <= (1 << 17) && L.d.k <= (1 << 17); }
 
-template <typename Kern>
-static mdbf_status_t t1_launch_one(Kern kern, int grid, int block, size_t smem, cudaStream_t st, const t1::Group &grp, int stage) {
+template <typename Kern, typename... Args>
+static mdbf_status_t t1_launch_one(Kern kern, int grid, int block, size_t smem, cudaStream_t st, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(block);
@@ -869,7 +908,7 @@ static mdbf_status_t t1_launch_one(Kern kern, int grid, int block, size_t smem, 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    MDBF_CUDA(cudaLaunchKernelEx(&cfg, kern, grp, stage));
+    MDBF_CUDA(cudaLaunchKernelEx(&cfg, kern, args...));
     return MDBF_OK;
 }
 
@@ -882,7 +921,8 @@ static mdbf_status_t t1_launch(const t1::Group &grp, int ctas, cudaStream_t st, 
     if (once.first()) MDBF_CUDA(cudaFuncSetAttribute(stage_kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     for (int s = 0; s < 2; ++s) {
         if (!(stages >> s & 1)) continue;
-        mdbf_status_t rc = t1_launch_one(image_kern, grp.items[s], t1::kImgThreads, 0, st, grp, s);
+        // stage A right after this file's stage B: max |z| is already there
+        mdbf_status_t rc = t1_launch_one(image_kern, grp.items[s], t1::kImgThreads, 0, st, grp, s, (int)(s == 1 && stages == 3));
         if (rc) return rc;
         rc = t1_launch_one(stage_kern, ctas, t1::kThreads, smem, st, grp, s);
         if (rc) return rc;
