@@ -53,7 +53,9 @@ enum {
     MDBF_ERR_CUDA = -5,        /* a CUDA runtime call failed (see last_error)     */
     MDBF_ERR_ARCH = -6,        /* no CUDA device, or not compute capability 10.x  */
     MDBF_ERR_TIMEOUT = -7,     /* a bounded device-side wait expired              */
-    MDBF_ERR_VALUE = -8        /* a sign that is neither +1 nor -1                */
+    MDBF_ERR_VALUE = -8,       /* a sign that is neither +1 nor -1                */
+    MDBF_ERR_BOUNDS = -9       /* bounds-checked build only: a kernel computed a   */
+                               /* store index outside its buffer (store skipped)  */
 };
 
 typedef enum { MDBF_F32 = 0, MDBF_F16 = 1, MDBF_BF16 = 2 } mdbf_dtype_t;
@@ -269,6 +271,12 @@ mdbf_status_t mdbf_reconstruct(mdbf_handle_t h, float *W, void *stream);
  * wait inside a kernel expired; the kernel then returns without completing y).
  * Synchronises the device.  Reading clears the word. */
 mdbf_status_t mdbf_poll_status(mdbf_handle_t h, int32_t *device_status);
+
+/* Test hook (no counterpart in the paper): the `nth` device allocation that the calling thread makes
+ * inside this library from now on fails with MDBF_ERR_ALLOC without touching the device; nth <= 0
+ * cancels a pending request.  A call that fails this way frees what it had allocated, publishes
+ * nothing half-built to the handle and leaves the handle (if any) as usable as before. */
+void mdbf_debug_fail_alloc(int nth);
 
 /* Self-test of the bounded device-side wait the tcgen05 kernels use (no counterpart in the paper):
  * launches one warp that waits on a barrier nothing arrives at.  After the time limit (about one

@@ -69,6 +69,21 @@ struct Layer {
     int out_mode;                 // set per call: 0 y in the activation type; 1 / 2: fp32 y stored / added (a term of a sum)
 };
 
+// Bounds-checked build (-DMDBF_BOUNDS_CHECK; `python -m paper_2512_24545_b200.build --bounds-check`): every store of
+// a tensor-core forward kernel into the caller's output or into a handle's scratch compares its flat index with the
+// extent of the buffer, re-derived from the launch arguments and not from the tile logic that guards the store.  An
+// index outside records MDBF_ERR_BOUNDS in the status word and the store is skipped (no trap: the context stays
+// usable and the tests read the status).  The normal build compiles the check away.
+#ifdef MDBF_BOUNDS_CHECK
+__device__ __forceinline__ bool store_in_bounds(size_t idx, size_t extent, int32_t *status) {
+    if (idx < extent) return true;
+    atomicExch(status, (int32_t)MDBF_ERR_BOUNDS);
+    return false;
+}
+#else
+__device__ __forceinline__ bool store_in_bounds(size_t, size_t, int32_t *) { return true; }
+#endif
+
 // A packed sign matrix as the kernels that are not tied to one layout read it: the canonical words (layers that only
 // the CUDA-core kernels serve), or - tensor-core layers keep a single copy of their signs - the row-block-major
 // copy of the one-token kernels, [row block of 128][kb_pad K blocks of 64 columns][128 rows] with 64 bits per entry.
@@ -89,6 +104,11 @@ SignView sign_view(const Layer &L, int which);      // 0: S_A, 1: S_B
 // thread-local error string
 void set_error(const char *fmt, ...);
 mdbf_status_t cuda_fail(cudaError_t e, const char *what);
+// Every device allocation of the library goes through here: cudaMalloc, or - after mdbf_debug_fail_alloc(n) on the
+// calling thread - cudaErrorMemoryAllocation for the n-th call from now on without touching the device (the tests
+// inject allocation failures this way, on the host).
+cudaError_t dev_malloc(void **p, size_t bytes);
+template <typename T> inline cudaError_t dev_malloc(T **p, size_t bytes) { return dev_malloc(reinterpret_cast<void **>(p), bytes); }
 
 #define MDBF_CUDA(call)                                                        \
     do {                                                                       \

@@ -283,7 +283,10 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
                 }
                 fence_proxy_async();
                 asm volatile("bar.sync %0, 128;\n" ::"r"(1 + g) : "memory");
-                if ((tid & 127) == 0 && tau0 + g * 64 < a.T) {
+                // the tensor map clips the tile at the extent of the output; its origin has to lie inside and start on
+                // a 16-byte boundary (8 entries of 16 bits)
+                const bool origin_ok = row0 >= 0 && row0 < a.rows && (row0 & 7) == 0 && tau0 + g * 64 >= 0;
+                if ((tid & 127) == 0 && tau0 + g * 64 < a.T && store_in_bounds(origin_ok ? 0 : 1, 1, a.status)) {
                     tma_store_2d(&tmap_out, row0, tau0 + g * 64, smem_base + (uint32_t)g * (64 * MT_BM * 2));
                     bulk_commit_wait_read();
                 }
@@ -301,11 +304,14 @@ mat_stage_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in, c
                     if (egrow < a.rows && col0 + j < a.bn && tau < a.T) {
                         const float acc = __uint_as_float(v[j]);
                         if (STAGE_A) {
-                            if (a.y_mode == 0) a.y[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(acc);
-                            else if (a.y_mode == 1) a.y32[(size_t)tau * a.rows + egrow] = acc;
-                            else a.y32[(size_t)tau * a.rows + egrow] += acc;
+                            const size_t o = (size_t)tau * a.rows + egrow;
+                            if (!store_in_bounds(o, (size_t)a.T * a.rows, a.status)) continue;
+                            if (a.y_mode == 0) a.y[o] = __float2bfloat16_rn(acc);
+                            else if (a.y_mode == 1) a.y32[o] = acc;
+                            else a.y32[o] += acc;
                         } else {
-                            a.zb[(size_t)tau * a.zstride + egrow] = __float2bfloat16_rn(acc);
+                            const size_t o = (size_t)tau * a.zstride + egrow;
+                            if (store_in_bounds(o, (size_t)a.T * a.zstride, a.status)) a.zb[o] = __float2bfloat16_rn(acc);
                         }
                     }
                 }
@@ -567,11 +573,14 @@ mat_small_kernel(const MatArgs a, const __grid_constant__ CUtensorMap tmap_in) {
         }
         auto emit = [&](int tau, float val) {
             if (STAGE_A) {
-                if (a.y_mode == 0) a.y[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(val);
-                else if (a.y_mode == 1) a.y32[(size_t)tau * a.rows + egrow] = val;
-                else a.y32[(size_t)tau * a.rows + egrow] += val;
+                const size_t o = (size_t)tau * a.rows + egrow;
+                if (!store_in_bounds(o, (size_t)a.T * a.rows, a.status)) return;
+                if (a.y_mode == 0) a.y[o] = __float2bfloat16_rn(val);
+                else if (a.y_mode == 1) a.y32[o] = val;
+                else a.y32[o] += val;
             } else {
-                a.zb[(size_t)tau * a.zstride + egrow] = __float2bfloat16_rn(val);
+                const size_t o = (size_t)tau * a.zstride + egrow;
+                if (store_in_bounds(o, (size_t)a.T * a.zstride, a.status)) a.zb[o] = __float2bfloat16_rn(val);
             }
         };
         if (SPLIT) {

@@ -284,12 +284,16 @@ gemm_stage_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap_xs)
         float *part_dst = SPLIT ? cluster.map_shared_rank(part, 0) : part;
         auto emit = [&](int tau, float acc) {
             if (egrow < a.rows && tau < a.T) {
+                const size_t o = (size_t)tau * a.rows + egrow;
+                if (!store_in_bounds(o, (size_t)a.T * a.rows, a.status)) return;
                 if (STAGE_A) {
-                    if (a.y_mode == 0) a.y[(size_t)tau * a.rows + egrow] = __float2bfloat16_rn(acc);
-                    else if (a.y_mode == 1) a.y32[(size_t)tau * a.rows + egrow] = acc;
-                    else a.y32[(size_t)tau * a.rows + egrow] += acc;
+                    if (a.y_mode == 0) a.y[o] = __float2bfloat16_rn(acc);
+                    else if (a.y_mode == 1) a.y32[o] = acc;
+                    else a.y32[o] += acc;
                 } else {
-                    a.z[(size_t)tau * a.rows + egrow] = acc;
+                    a.z[o] = acc;
+                    // pre-scaled operand of stage A: [(tau, mode)][pad_next] entries, this row's column
+                    if (!store_in_bounds((size_t)(tau * LP + LP - 1) * a.pad_next + egrow, (size_t)a.T * LP * a.pad_next, a.status)) return;
                     __nv_bfloat16 *xo = a.xs_next + (size_t)tau * LP * a.pad_next + egrow;
 #pragma unroll
                     for (int t2 = 0; t2 < LP; ++t2)
@@ -613,8 +617,8 @@ mdbf_status_t ensure_prefill_scratch(Layer &L) {
     if (L.xsB) return MDBF_OK;
     L.xs_rows = ((size_t)L.d.max_T * L.LP + 255) / 256 * 256;
     __nv_bfloat16 *b = nullptr, *a = nullptr;
-    MDBF_CUDA(cudaMalloc(&b, L.xs_rows * L.padB * 2));
-    cudaError_t e = cudaMalloc(&a, L.xs_rows * L.padA * 2);
+    MDBF_CUDA(dev_malloc(&b, L.xs_rows * L.padB * 2));
+    cudaError_t e = dev_malloc(&a, L.xs_rows * L.padA * 2);
     if (e == cudaSuccess) e = cudaMemset(b, 0, L.xs_rows * L.padB * 2);
     if (e == cudaSuccess) e = cudaMemset(a, 0, L.xs_rows * L.padA * 2);
     if (e != cudaSuccess) { cudaFree(b); cudaFree(a); return cuda_fail(e, "scratch of the expanded order"); }

@@ -664,7 +664,9 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                 }
 #pragma unroll
                 for (int j = 0; j < kRBG; ++j)
-                    if (fin[j]) old[j] = atomicAdd(S.acc64 + (sg.rg * kRBG + j) * 128 + atid, mine[j]);
+                    if (fin[j] && store_in_bounds((size_t)((sg.rg * kRBG + j) * 128 + atid), (size_t)S.R * 128, L.status))
+                        old[j] = atomicAdd(S.acc64 + (sg.rg * kRBG + j) * 128 + atid, mine[j]);
+                    else fin[j] = false;
 #pragma unroll
                 for (int j = 0; j < kRBG; ++j)
                     if (fin[j]) {
@@ -681,7 +683,7 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                 float zmax = 0.f;
 #pragma unroll
                 for (int j = 0; j < kRBG; ++j)
-                    if (fin[j]) {
+                    if (fin[j] && store_in_bounds((size_t)((sg.rg * kRBG + j) * 128 + atid), (size_t)S.rows, L.status)) {
                         L.z[(sg.rg * kRBG + j) * 128 + atid] = part[j];
                         zmax = fmaxf(zmax, fabsf(part[j]));
                     }
@@ -693,6 +695,7 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                 for (int j = 0; j < kRBG; ++j)
                     if (fin[j]) {
                         const int grow = (sg.rg * kRBG + j) * 128 + atid;
+                        if (!store_in_bounds((size_t)grow, (size_t)S.rows, L.status)) continue;
                         if (L.out_mode == 0) reinterpret_cast<__nv_bfloat16 *>(L.y)[grow] = __float2bfloat16_rn(part[j]);
                         else if (L.out_mode == 1) reinterpret_cast<float *>(L.y)[grow] = part[j];
                         else reinterpret_cast<float *>(L.y)[grow] += part[j];
@@ -868,15 +871,15 @@ mdbf_status_t t1_prepare(Layer &L, cudaStream_t st) {
     b.R[0] = L.rpB / 128; b.Np[0] = L.kbpB / 2;
     b.R[1] = L.rpA / 128; b.Np[1] = L.kbpA / 2;
     for (int s = 0; s < 2; ++s) b.RG[s] = ceil_div(b.R[s], t1::kRBG);
-    MDBF_CUDA(cudaMalloc(&b.vmax, 64 * sizeof(float)));
-    MDBF_CUDA(cudaMalloc(&b.sync, (size_t)t1::kSyWords * 4));
+    MDBF_CUDA(dev_malloc(&b.vmax, 64 * sizeof(float)));
+    MDBF_CUDA(dev_malloc(&b.sync, (size_t)t1::kSyWords * 4));
     MDBF_CUDA(cudaMemsetAsync(b.sync, 0, (size_t)t1::kSyWords * 4, st));
     for (int s = 0; s < 2; ++s) {
-        MDBF_CUDA(cudaMalloc(&b.img[s], (size_t)b.Np[s] * NB * 128));
+        MDBF_CUDA(dev_malloc(&b.img[s], (size_t)b.Np[s] * NB * 128));
         MDBF_CUDA(cudaMemsetAsync(b.img[s], 0, (size_t)b.Np[s] * NB * 128, st));      // the padding rows stay zero
-        MDBF_CUDA(cudaMalloc(&b.colsum[s], (size_t)b.Np[s] * 32 * sizeof(int)));
+        MDBF_CUDA(dev_malloc(&b.colsum[s], (size_t)b.Np[s] * 32 * sizeof(int)));
         MDBF_CUDA(cudaMemsetAsync(b.colsum[s], 0, (size_t)b.Np[s] * 32 * sizeof(int), st));
-        MDBF_CUDA(cudaMalloc(&b.acc64[s], (size_t)b.R[s] * 128 * sizeof(unsigned long long)));
+        MDBF_CUDA(dev_malloc(&b.acc64[s], (size_t)b.R[s] * 128 * sizeof(unsigned long long)));
         MDBF_CUDA(cudaMemsetAsync(b.acc64[s], 0, (size_t)b.R[s] * 128 * sizeof(unsigned long long), st));
     }
     MDBF_CUDA(cudaMemsetAsync(b.vmax, 0, 64 * sizeof(float), st));

@@ -364,7 +364,7 @@ __device__ __forceinline__ void tmem_t1_body(const TxArgs &a, const int rb) {
         for (unsigned rk = 1; rk < 8; ++rk)
             if (rk < nranks) outv += part[rk * 128 + row_l];
         const int grow = row0 + row_l;
-        if (grow < a.rows && !*abort_flag) {
+        if (grow < a.rows && !*abort_flag && store_in_bounds((size_t)grow, (size_t)a.rows, a.status)) {
             if (a.stage_a == 1) reinterpret_cast<__nv_bfloat16 *>(a.out)[grow] = __float2bfloat16_rn(outv);
             else if (a.stage_a == 3) reinterpret_cast<float *>(a.out)[grow] += outv;      // a further term of a sum of layers
             else if (SUM_LAST && a.stage_a == 4)                                           // its last term: one rounding of the whole sum

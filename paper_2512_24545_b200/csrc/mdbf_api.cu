@@ -103,8 +103,8 @@ static mdbf_status_t ensure_kblock_words(Layer &L) {
     const mdbf_desc_t &d = L.d;
     if (L.wkA) return MDBF_OK;
     uint2 *a = nullptr, *b = nullptr;
-    ENS_CUDA(cudaMalloc(&a, (size_t)(L.padA / 64) * L.rpA * sizeof(uint2)));
-    cudaError_t e = cudaMalloc(&b, (size_t)(L.padB / 64) * L.rpB * sizeof(uint2));
+    ENS_CUDA(dev_malloc(&a, (size_t)(L.padA / 64) * L.rpA * sizeof(uint2)));
+    cudaError_t e = dev_malloc(&b, (size_t)(L.padB / 64) * L.rpB * sizeof(uint2));
     if (e != cudaSuccess) { cudaFree(a); return cuda_fail(e, "K-blocked sign words"); }
     mdbf_status_t rc = launch_kblock(sign_view(L, 0), d.d_out, a, L.rpA, L.padA / 64, 0);
     if (rc == MDBF_OK) rc = launch_kblock(sign_view(L, 1), d.k, b, L.rpB, L.padB / 64, 0);
@@ -122,7 +122,7 @@ mdbf_status_t ensure_kernel_layouts(Layer &L, int kernel, int T) {
     ENS_RC(ensure_kblock_words(L));
     if (!L.vtB) {
         float *vt = nullptr;
-        ENS_CUDA(cudaMalloc(&vt, (size_t)L.LP * L.padB * sizeof(float)));
+        ENS_CUDA(dev_malloc(&vt, (size_t)L.LP * L.padB * sizeof(float)));
         mdbf_status_t rc = launch_vtrans(L.VB, d.d_in, d.l, d.env_dtype, vt, L.padB, L.LP, 0);
         if (rc) { cudaFree(vt); return rc; }
         L.vtB = vt;
@@ -134,8 +134,8 @@ mdbf_status_t ensure_kernel_layouts(Layer &L, int kernel, int T) {
 static mdbf_status_t ensure_host_staging(Layer &L) {
     if (L.xstage) return MDBF_OK;
     void *xs = nullptr, *ys = nullptr;
-    ENS_CUDA(cudaMalloc(&xs, (size_t)L.d.max_T * L.d.d_in * 4));
-    cudaError_t e = cudaMalloc(&ys, (size_t)L.d.max_T * L.d.d_out * 4);
+    ENS_CUDA(dev_malloc(&xs, (size_t)L.d.max_T * L.d.d_in * 4));
+    cudaError_t e = dev_malloc(&ys, (size_t)L.d.max_T * L.d.d_out * 4);
     if (e != cudaSuccess) { cudaFree(xs); return cuda_fail(e, "host-entry staging"); }
     L.xstage = xs; L.ystage = ys;
     return MDBF_OK;
@@ -143,14 +143,31 @@ static mdbf_status_t ensure_host_staging(Layer &L) {
 #undef ENS_CUDA
 #undef ENS_RC
 
+static thread_local int g_fail_alloc_in = 0;       // > 0: that many dev_malloc calls from now, the last of them fails
+cudaError_t dev_malloc(void **p, size_t bytes) {
+    if (g_fail_alloc_in > 0 && --g_fail_alloc_in == 0) {
+        *p = nullptr;
+        return cudaErrorMemoryAllocation;
+    }
+    return cudaMalloc(p, bytes);
+}
+
 }  // namespace mdbf
 
 using namespace mdbf;
 
 extern "C" {
 
+void mdbf_debug_fail_alloc(int nth) { g_fail_alloc_in = nth > 0 ? nth : 0; }
+
 const char *mdbf_last_error(void) { return g_err; }
-const char *mdbf_version(void) { return "libmdbf 0.1 (sm_100a)"; }
+const char *mdbf_version(void) {
+#ifdef MDBF_BOUNDS_CHECK
+    return "libmdbf 0.2 (sm_100a) +bounds-check";
+#else
+    return "libmdbf 0.2 (sm_100a)";
+#endif
+}
 
 mdbf_status_t mdbf_pack_signs(const int8_t *s, int64_t rows, int64_t cols, uint32_t *out, int on_device,
                               void *stream) {
@@ -235,12 +252,12 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
         if (r__ != MDBF_OK) return fail(r__);        \
     } while (0)
 
-    PACK_CUDA(cudaMalloc(&L.wA, (size_t)d.d_out * L.wordsA * 4));
-    PACK_CUDA(cudaMalloc(&L.wB, (size_t)d.k * L.wordsB * 4));
-    PACK_CUDA(cudaMalloc(&L.UA, nUA * es));
-    PACK_CUDA(cudaMalloc(&L.VA, nVA * es));
-    PACK_CUDA(cudaMalloc(&L.UB, nUB * es));
-    PACK_CUDA(cudaMalloc(&L.VB, nVB * es));
+    PACK_CUDA(dev_malloc(&L.wA, (size_t)d.d_out * L.wordsA * 4));
+    PACK_CUDA(dev_malloc(&L.wB, (size_t)d.k * L.wordsB * 4));
+    PACK_CUDA(dev_malloc(&L.UA, nUA * es));
+    PACK_CUDA(dev_malloc(&L.VA, nVA * es));
+    PACK_CUDA(dev_malloc(&L.UB, nUB * es));
+    PACK_CUDA(dev_malloc(&L.VB, nVB * es));
     L.LP = 1;
     while (L.LP < d.l) L.LP *= 2;
     L.padA = ceil_div(d.k, 64) * 64; L.padB = ceil_div(d.d_in, 64) * 64;
@@ -251,25 +268,25 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     if (want_tc) {
         const int NB = L.LP < 16 ? 16 : L.LP;
         L.kbpA = ceil_div(L.padA / 64, 2) * 2; L.kbpB = ceil_div(L.padB / 64, 2) * 2;
-        PACK_CUDA(cudaMalloc(&L.vxA, (size_t)L.kbpA * NB * 64 * sizeof(uint16_t)));
-        PACK_CUDA(cudaMalloc(&L.vxB, (size_t)L.kbpB * NB * 64 * sizeof(uint16_t)));
-        PACK_CUDA(cudaMalloc(&L.wk2A, (size_t)(L.rpA / 128) * L.kbpA * 128 * sizeof(uint2)));
-        PACK_CUDA(cudaMalloc(&L.wk2B, (size_t)(L.rpB / 128) * L.kbpB * 128 * sizeof(uint2)));
+        PACK_CUDA(dev_malloc(&L.vxA, (size_t)L.kbpA * NB * 64 * sizeof(uint16_t)));
+        PACK_CUDA(dev_malloc(&L.vxB, (size_t)L.kbpB * NB * 64 * sizeof(uint16_t)));
+        PACK_CUDA(dev_malloc(&L.wk2A, (size_t)(L.rpA / 128) * L.kbpA * 128 * sizeof(uint2)));
+        PACK_CUDA(dev_malloc(&L.wk2B, (size_t)(L.rpB / 128) * L.kbpB * 128 * sizeof(uint2)));
     }
     if (want_prefill) {
         // The pre-scaled operands of the expanded order (max_T * LP * (d_in + k) * 2 bytes) are allocated on
         // its first use (ensure_prefill_scratch): the default path for T >= 2 does not need them.
         // bf16 intermediate of the materialised-envelope kernels, [max_T][padA]; the padding columns stay zero
-        PACK_CUDA(cudaMalloc(&L.zb, (size_t)d.max_T * L.padA * 2));
+        PACK_CUDA(dev_malloc(&L.zb, (size_t)d.max_T * L.padA * 2));
         PACK_CUDA(cudaMemsetAsync(L.zb, 0, (size_t)d.max_T * L.padA * 2, st));
         L.kcm = d.l <= 16 ? 2 : 4;
-        PACK_CUDA(cudaMalloc(&L.uiA, (size_t)(L.rpA / 128) * L.kcm * 1024 * sizeof(uint16_t)));
-        PACK_CUDA(cudaMalloc(&L.uiB, (size_t)(L.rpB / 128) * L.kcm * 1024 * sizeof(uint16_t)));
-        PACK_CUDA(cudaMalloc(&L.viA, (size_t)ceil_div(L.padA, 128) * L.kcm * 1024 * sizeof(uint16_t)));
-        PACK_CUDA(cudaMalloc(&L.viB, (size_t)ceil_div(L.padB, 128) * L.kcm * 1024 * sizeof(uint16_t)));
+        PACK_CUDA(dev_malloc(&L.uiA, (size_t)(L.rpA / 128) * L.kcm * 1024 * sizeof(uint16_t)));
+        PACK_CUDA(dev_malloc(&L.uiB, (size_t)(L.rpB / 128) * L.kcm * 1024 * sizeof(uint16_t)));
+        PACK_CUDA(dev_malloc(&L.viA, (size_t)ceil_div(L.padA, 128) * L.kcm * 1024 * sizeof(uint16_t)));
+        PACK_CUDA(dev_malloc(&L.viB, (size_t)ceil_div(L.padB, 128) * L.kcm * 1024 * sizeof(uint16_t)));
     }
-    PACK_CUDA(cudaMalloc(&L.zsum, (size_t)d.max_T * d.k * sizeof(float)));
-    PACK_CUDA(cudaMalloc(&L.status, sizeof(int32_t)));
+    PACK_CUDA(dev_malloc(&L.zsum, (size_t)d.max_T * d.k * sizeof(float)));
+    PACK_CUDA(dev_malloc(&L.status, sizeof(int32_t)));
     PACK_CUDA(cudaMemsetAsync(L.status, 0, sizeof(int32_t), st));
     PACK_CUDA(cudaMemsetAsync(L.zsum, 0, (size_t)d.max_T * d.k * sizeof(float), st));
 
@@ -280,7 +297,7 @@ mdbf_status_t mdbf_pack(const mdbf_desc_t *desc, const int8_t *S_A, const int8_t
     for (int i = 0; i < 6; ++i) {
         if (inputs_on_device) { dsrc[i] = src[i]; continue; }
         void *tmp = nullptr;
-        PACK_CUDA(cudaMalloc(&tmp, bytes[i]));
+        PACK_CUDA(dev_malloc(&tmp, bytes[i]));
         temps.push_back(tmp);
         PACK_CUDA(cudaMemcpyAsync(tmp, src[i], bytes[i], cudaMemcpyHostToDevice, st));
         dsrc[i] = tmp;
@@ -337,7 +354,7 @@ mdbf_status_t mdbf_get_packed(mdbf_handle_t h, int which, uint32_t *out, int out
         return MDBF_OK;
     }
     uint32_t *tmp = nullptr;                          // check path: a temporary device copy in canonical order
-    MDBF_CUDA(cudaMalloc(&tmp, bytes));
+    MDBF_CUDA(dev_malloc(&tmp, bytes));
     rc = launch_canon(sv, rows, tmp, st);
     cudaError_t e = cudaSuccess;
     if (rc == MDBF_OK) e = cudaMemcpyAsync(out, tmp, bytes, cudaMemcpyDeviceToHost, st);
@@ -364,7 +381,7 @@ mdbf_status_t mdbf_get_envelope(mdbf_handle_t h, int which, float *out, int out_
         return MDBF_OK;
     }
     float *tmp = nullptr;
-    MDBF_CUDA(cudaMalloc(&tmp, n[which] * 4));
+    MDBF_CUDA(dev_malloc(&tmp, n[which] * 4));
     rc = launch_env_read(src[which], tmp, n[which], L.d.env_dtype, st);
     cudaError_t e = cudaSuccess;
     if (rc == MDBF_OK) e = cudaMemcpyAsync(out, tmp, n[which] * 4, cudaMemcpyDeviceToHost, st);
@@ -473,7 +490,7 @@ static mdbf_status_t forward_impl(mdbf_handle_t h, const void *x, void *y, int32
         return MDBF_ERR_DTYPE;
     }
     if (kernel == MDBF_KERNEL_PREFILL && !L.xsB) {
-        set_error("mdbf_linear_forward: the expanded-order kernel has no scratch on this handle; call mdbf_set_kernel(handle, MDBF_KERNEL_PREFILL) first (it allocates)");
+        set_error("mdbf_linear_forward: the expanded-order kernel has no scratch on this handle; call mdbf_set_kernel(handle, MDBF_KERNEL_PREFILL) first (it allocates; a handle packed with max_T = 1 never has any)");
         return MDBF_ERR_INVALID_ARG;
     }
     if (kernel == MDBF_KERNEL_I8 && (T != 1 || !t1_supports(L))) {

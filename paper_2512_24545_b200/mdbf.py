@@ -21,15 +21,15 @@ LIB_PATH = os.path.join(_HERE, "libmdbf.so")
 F32, F16, BF16 = 0, 1, 2
 KERNEL_AUTO, KERNEL_ALU, KERNEL_PREFILL, KERNEL_TMEM, KERNEL_MAT, KERNEL_I8 = 0, 1, 3, 4, 5, 6
 OK = 0
-ERR_INVALID_ARG, ERR_SHAPE, ERR_DTYPE, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT, ERR_VALUE = (
-    -1, -2, -3, -4, -5, -6, -7, -8)
+ERR_INVALID_ARG, ERR_SHAPE, ERR_DTYPE, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT, ERR_VALUE, ERR_BOUNDS = (
+    -1, -2, -3, -4, -5, -6, -7, -8, -9)
 DTYPES = {"f32": F32, "f16": F16, "bf16": BF16}
 
 EXPORTS = (
     "mdbf_pack_signs", "mdbf_unpack_signs", "mdbf_pack", "mdbf_get_packed", "mdbf_get_envelope",
     "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host", "mdbf_prepare_host_staging",
     "mdbf_linear_forward_static", "mdbf_linear_forward_sum", "mdbf_linear_forward_siblings", "mdbf_linear_forward_group",
-    "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_poll_status", "mdbf_selftest_wait_timeout",
+    "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_poll_status", "mdbf_selftest_wait_timeout", "mdbf_debug_fail_alloc",
     "mdbf_last_launch_count",
     "mdbf_last_kernel",
     "mdbf_destroy", "mdbf_last_error", "mdbf_version",
@@ -80,6 +80,7 @@ def lib() -> ctypes.CDLL:
     L.mdbf_reconstruct.argtypes = [vp, vp, vp]
     L.mdbf_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
     L.mdbf_selftest_wait_timeout.argtypes = [vp, vp]
+    L.mdbf_debug_fail_alloc.argtypes = [i32]
     L.mdbf_last_launch_count.argtypes = [vp, ctypes.POINTER(i32)]
     L.mdbf_last_kernel.argtypes = [vp, ctypes.POINTER(i32)]
     L.mdbf_destroy.argtypes = [vp]
@@ -89,6 +90,7 @@ def lib() -> ctypes.CDLL:
     L.mdbf_last_error.argtypes = []
     L.mdbf_version.restype = ctypes.c_char_p
     L.mdbf_version.argtypes = []
+    L.mdbf_debug_fail_alloc.restype = None
     _lib = L
     return L
 
@@ -216,6 +218,11 @@ def mdbf_poll_status(h: int) -> int:
     v = ctypes.c_int32()
     _check(lib().mdbf_poll_status(h, ctypes.byref(v)))
     return v.value
+
+
+def mdbf_debug_fail_alloc(nth: int) -> None:
+    """Test hook: the nth device allocation this thread makes inside the library from now on fails (nth <= 0: cancel)."""
+    lib().mdbf_debug_fail_alloc(nth)
 
 
 def mdbf_selftest_wait_timeout(h: int, stream: int = 0) -> None:

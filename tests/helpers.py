@@ -13,6 +13,10 @@ TOL = {"bf16": 5e-3, "f16": 5e-3, "f32": 1e-5}     # relative Frobenius bounds o
 TOL_RECONSTRUCT = 1e-6
 
 
+GUARD_BYTES = 4096          # on either side of every output buffer of GpuLayer.forward (a multiple of 16: y stays aligned)
+GUARD_PATTERN = 0xA5
+
+
 class GpuLayer:
     """A packed layer plus the host copies of what went in."""
 
@@ -48,12 +52,29 @@ class GpuLayer:
         act = act_dtype or self.spec.act_dtype
         T = x.shape[0]
         xd = torch.from_numpy(np.ascontiguousarray(x)).to(TORCH_DT[act]).cuda()
-        yd = torch.full((T, self.spec.d_out), float("nan"), dtype=TORCH_DT[act], device="cuda")
+        # the output sits between two guard regions filled with a byte pattern no kernel writes: a store before the
+        # first or past the last element of y shows up here (no memory checker runs on the GPU tests)
+        n = T * self.spec.d_out
+        esz = torch.empty((), dtype=TORCH_DT[act]).element_size()
+        guard = GUARD_BYTES // esz
+        raw = torch.empty(guard + n + guard, dtype=TORCH_DT[act], device="cuda")
+        raw.view(torch.uint8).fill_(GUARD_PATTERN)
+        yd = raw[guard:guard + n].view(T, self.spec.d_out)
+        yd.fill_(float("nan"))
         M.mdbf_set_kernel(self.h, kernel)
-        M.mdbf_linear_forward(self.h, xd.data_ptr(), yd.data_ptr(), T, M.DTYPES[act],
-                              torch.cuda.current_stream().cuda_stream)
-        torch.cuda.synchronize()
-        M.mdbf_set_kernel(self.h, M.KERNEL_AUTO)
+        try:
+            M.mdbf_linear_forward(self.h, xd.data_ptr(), yd.data_ptr(), T, M.DTYPES[act],
+                                  torch.cuda.current_stream().cuda_stream)
+            torch.cuda.synchronize()
+        finally:
+            M.mdbf_set_kernel(self.h, M.KERNEL_AUTO)
+        lo = raw[:guard].view(torch.uint8)
+        hi = raw[guard + n:].view(torch.uint8)
+        assert bool((lo == GUARD_PATTERN).all()) and bool((hi == GUARD_PATTERN).all()), "a kernel wrote outside y"
+        # the device status word: MDBF_ERR_TIMEOUT after a bounded wait expired and, in the bounds-checked build
+        # (MDBF_BOUNDS_CHECK=1), MDBF_ERR_BOUNDS after a kernel computed a store index outside its buffer
+        status = M.mdbf_poll_status(self.h)
+        assert status == 0, f"device status {status} after a forward"
         return yd.to(torch.float32).cpu().numpy()
 
     def intermediate(self, T: int) -> np.ndarray:
