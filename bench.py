@@ -38,8 +38,13 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # captures summarised under profiles/ (None until a capture exists for that workload).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     ("decode_qproj", "tmem_t1_kernel"): 1082112,                   # k = 1664 layer, stage B (stage A: 1080320)
+    ("block70b_T1", "t1_stage_kernel"): 46402560,                  # gate/up stage A in one launch (45.3 MB algorithmic); down stage B: 23289856
+    ("decode_mlp_T1", "tmem_t1_kernel"): 5998592,                  # up / gate, either stage (down: 2342400)
+    ("decode_mlp_T16", "mat_small_kernel"): 6340000,               # up stage B (stage A: 6.11 MB, down stage A: 2.47 MB)
     ("prefill_4096_l16_bpw10", "mat_stage_kernel"): 17858048,      # stage B: x read once + signs + images; nothing reaches DRAM on the way out
     ("prefill_4096_l16_bpw10", "gemm_stage_kernel"): 370142976,    # stage B: 269.4 MB read + 100.7 MB written
+    ("block70b_T2048", "mat_stage_kernel"): 197116928,             # its largest launch, down stage B (185.9 MB read: 117 MB of x, partly twice,
+                                                                   # + signs; 11.3 MB written); gate / up stage A: 123.3 MB
 }
 
 
@@ -257,8 +262,8 @@ def measure(workload, kernel, steps, warmup, dist, world, local, no_graph=False,
     if workload.startswith("block70b"):       # block by block: q, k, v, o, gate, up, down of copy 0, then copy 1, ...
         nc = copies if copies > 0 else groups[0][1]
         groups = [(inputs.scaled(sp, seed=sp.seed + 1000 * c) if c else sp, 1) for c in range(nc) for (sp, _n) in groups]
-    for spec, copies in groups:
-        for c in range(1 if (P_sum or workload.startswith("block70b")) else (copies if copies > 0 else copies)):
+    for spec, default_copies in groups:
+        for c in range(1 if (P_sum or workload.startswith("block70b")) else (copies if copies > 0 else default_copies)):
             sp = inputs.scaled(spec, seed=spec.seed + 1000 * (c + 1)) if c else spec
             lay = inputs.make_layer(sp)
             h = M.mdbf_pack(sp.d_out, sp.d_in, sp.k, sp.l, M.DTYPES[sp.env_dtype], T,

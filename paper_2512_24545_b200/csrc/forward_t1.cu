@@ -5,7 +5,7 @@
 // Eq. me-dbf-expand); stage B (S_B, V_B, U_B) maps x -> z, stage A (S_A, V_A, U_A) maps z -> y
 // (Eq. DBF-inference-form, column convention).
 //
-// The scaled operand w[c][t] = V[c][t] * in[c] (steps a1 / a4 of the path: the pre-scale by the envelope
+// The scaled operand w[c][t] = V[c][t] * in[c] (the first step of a stage: the pre-scale by the envelope
 // factor) is turned into a 21-bit fixed-point number per mode t,  w ~ delta_t * q,  |q| <= 2^20 - 2,
 // q = q0 + 2^7 q1 + 2^14 q2  with three signed 8-bit digits, delta_t from max|in| * max_c |V[c][t]|.
 // The contraction with the signs is then an exact integer matrix product
@@ -31,9 +31,10 @@
 // image kernel: one CTA per pair of K blocks of every layer: max |input|, fixed-point digits, column sums.
 // stage kernel: a fixed grid of CTAs (one per SM), each walking its share of the units (group of four row
 // blocks of 128 rows) x (pair of K blocks) of every layer, in layer order.  Roles of a CTA: four groups of
-// four expander warps (group = row block of the unit, thread = row = TMEM lane), four MMA issuer warps
-// (issuer = row block, own accumulator and own double-buffered A stages), one warp bulk-copying sign words
-// (ring of 8 units = 64 KB, lane = ring slot), one bulk-copying images (ring of 8), and four epilogue
+// four expander warps (group = row block of the unit, thread = row = TMEM lane), eight MMA issuer warps (two
+// per row block, one for the even and one for the odd units, i.e. one per A stage of the row block; both add
+// into the row block's accumulator), one warp bulk-copying sign words (ring of 8 units = 64 KB, lane = ring
+// slot), one bulk-copying images (ring of 8), and four epilogue
 // warps (tcgen05.ld, contraction with U).  A group of row blocks split over several CTAs is summed through
 // one 64-bit integer atomic per row (order-independent, hence deterministic): the thread whose addition
 // completes the row's count finalises the row.  No CTA ever waits for another one; every mbarrier wait is
@@ -42,23 +43,6 @@
 #include <cstdlib>
 
 #include "tmem_ptx.cuh"
-
-#ifdef MDBF_T1_TRACE
-__device__ unsigned long long g_t1_trace[160 * 32];
-#define TR(slot) do { if (lane == 0) g_t1_trace[cta * 32 + (slot)] = tm_trace_ns(); } while (0)
-__device__ __forceinline__ unsigned long long tm_trace_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t)); return t; }
-extern "C" int mdbf_debug_t1_trace(unsigned long long *out) {
-    return (int)cudaMemcpyFromSymbol(out, g_t1_trace, sizeof(g_t1_trace));
-}
-#define TRC_DECL long long trc_t = clock64(), trc_a[4] = {0, 0, 0, 0}; int trc_n = 0
-#define TRC(k) do { const long long trc_now = clock64(); trc_a[k] += trc_now - trc_t; trc_t = trc_now; } while (0)
-#define TRC_OUT(base) do { if (lane == 0) { for (int q_ = 0; q_ < 4; ++q_) g_t1_trace[cta * 32 + (base) + q_] = (unsigned long long)trc_a[q_]; g_t1_trace[cta * 32 + 23] = trc_n; } } while (0)
-#else
-#define TR(slot) do { } while (0)
-#define TRC_DECL do { } while (0)
-#define TRC(k) do { } while (0)
-#define TRC_OUT(base) do { } while (0)
-#endif
 
 namespace mdbf {
 namespace t1 {
@@ -435,7 +419,6 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
-    if (warp == 0) TR(0);
     const uint32_t smem_base = (smem_u32(t1_smem_raw) + 1023u) & ~1023u;
     unsigned char *smem_gen = t1_smem_raw + (smem_base - smem_u32(t1_smem_raw));
     const uint32_t off_s = (uint32_t)(NIM * IMG);                // sign ring after the image ring
@@ -467,7 +450,6 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
     const uint32_t tmem_a0 = tmem + (uint32_t)(4 * NB);         // A stages: [row block j][NAG][32 columns]
 
     pdl_launch_dependents();
-    if (warp == 0) TR(1);
 
     if (warp < W_AUX) {
         // ===================================== expanders =====================================
@@ -477,17 +459,14 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
         bool alive = true;
         int qn = 0;                                              // units this CTA has walked
         int prev_as = -1;                                        // A stage whose stores are still to be published
-        TRC_DECL;
         SegIter it(g, s, cta, (int)gridDim.x);
         Seg sg;
         while (alive && it.next(g, sg)) {
             const bool valid = grp < sg.nrb;
             for (int p = sg.p0; p < sg.p1; ++p, ++qn) {
                 const int rs = qn % NSQ;
-                TRC(3);
                 alive = bwait(s_full + 8 * rs, (uint32_t)(qn / NSQ) & 1u, abort_flag, status0);
                 if (!alive) break;
-                TRC(0);
                 uint2 w0 = make_uint2(0u, 0u), w1 = w0;
                 if (valid) {
                     const unsigned char *sw = smem_gen + off_s + rs * 8192 + grp * 2048 + row_l * 8;
@@ -516,13 +495,11 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                 // every issuer releases a unit's image with a commit, i.e. after all its earlier MMAs have retired: one
                 // commit per unit and issuer serves both rings.
                 const int as = qn % NAG;
-                TRC(1);
                 if (qn >= NAG) {
                     const int qp = qn - NAG;
                     alive = bwait(i_empty + 8 * (qp % NIM), (uint32_t)(qp / NIM) & 1u, abort_flag, status0);
                     if (!alive) break;
                 }
-                TRC(2);
                 tc_fence_after();
                 const uint32_t a_col = tmem_a0 + lane_base + (uint32_t)((grp * NAG + as) * 32);
                 tmem_st32(a_col, v);                             // one store of the whole row: a tcgen05.st holds the warp for ~140 clocks whatever its width
@@ -535,10 +512,6 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
             __syncwarp();
             if (alive && lane == 0) mbar_arrive(a_full + 8 * (grp * NAG + prev_as));
         }
-        if (warp == 0) { TR(11); TRC_OUT(28); }
-#ifdef MDBF_T1_TRACE
-        if (warp == 0 && lane == 0) g_t1_trace[cta * 32 + 27] = (unsigned long long)qn;
-#endif
     } else if (warp < W_ISS) {
         // ============================ epilogue warps: contraction with U, row finalisation ============================
         const int atid = tid - W_AUX * 32;                       // 0 .. 127 = row of the tile = TMEM lane
@@ -591,7 +564,6 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
             aux_sync();                                          // one decision for the whole group
             if (*abort_flag) { alive = false; break; }
             tc_fence_after();
-            if (warp == W_AUX) TR(4);
             // First only what needs the accumulators: per row block the three digits of every mode combined into one float,
             // f[j][t] = -2 * sum_c b q[c][t] (the A bytes are 128 b: -2 * 128^digit / 128), and the accumulator cleared; then
             // the issuers may start the next segment while the contraction with U and the hand-over run here.
@@ -621,7 +593,6 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                     }
                 }
             }
-            if (warp == W_AUX) TR(24);
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
@@ -678,7 +649,6 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                         }
                     }
             }
-            if (warp == W_AUX) TR(25);
             if (s == 0) {
                 float zmax = 0.f;
 #pragma unroll
@@ -701,11 +671,7 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                         else reinterpret_cast<float *>(L.y)[grow] += part[j];
                     }
             }
-            if (warp == W_AUX) TR(5);
         }
-#ifdef MDBF_T1_TRACE
-        if (warp == W_AUX && lane == 0) g_t1_trace[cta * 32 + 26] = (unsigned long long)nseg_done;
-#endif
     } else if (warp < W_SLOAD) {
         // ==================================== MMA issuers ====================================
         // Two issuers per row block of the unit, one for the even and one for the odd units (= A stage 0 / 1): while one
@@ -718,7 +684,6 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
         bool alive = true;
         int qn = 0, nseg_done = 0;
         uint32_t ause = 0u;                                      // uses of this issuer's A stage so far
-        TRC_DECL;
         SegIter it(g, s, cta, (int)gridDim.x);
         Seg sg;
         while (alive && it.next(g, sg)) {
@@ -729,10 +694,8 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
             for (int p = sg.p0; p < sg.p1 && alive; ++p, ++qn) {
                 if ((qn & 1) != par) continue;
                 const int is = qn % NIM;
-                TRC(3);
                 alive = bwait(i_full + 8 * is, (uint32_t)(qn / NIM) & 1u, abort_flag, status0);
                 if (!alive) break;
-                TRC(0);
                 if (!valid) {                                    // no such row block: only release the image (after this issuer's earlier MMAs)
                     if (lane == 0) umma_commit(i_empty + 8 * is);
                     __syncwarp();
@@ -740,9 +703,7 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                 }
                 alive = bwait(a_full + 8 * (k * NAG + par), ause & 1u, abort_flag, status0);
                 if (!alive) break;
-                TRC(1);
                 tc_fence_after();
-                if (warp == W_ISS && nseg_done == 0 && issued == 0) TR(12);
                 if (lane == 0) {
                     const uint64_t bdesc = make_smem_desc(smem_base + (uint32_t)(is * IMG));
                     const uint32_t a_t = tmem_a0 + (uint32_t)((k * NAG + par) * 32);
@@ -752,7 +713,6 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
                     umma_commit(i_empty + 8 * is);               // one of the four releases of the image; with all four the A stages of the unit are free too
                 }
                 __syncwarp();
-                TRC(2);
                 ++issued;
                 ++ause;
             }
@@ -763,7 +723,6 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
             __syncwarp();
             ++nseg_done;
         }
-        if (warp == W_ISS) { }
     } else if (warp == W_SLOAD) {
         // ================================= sign-word loader ==================================
         // Lane l owns ring slot l: it waits for the slot, then issues the (up to) four bulk copies of its unit.  Sign
@@ -815,7 +774,6 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
     }
 
     // ------------------------------ leave ------------------------------
-    if (warp == 0) TR(20);
     tc_fence_before();
     __syncthreads();
     if (warp == W_ISS) tmem_dealloc(tmem, (uint32_t)TMEM_COLS);
@@ -824,7 +782,6 @@ __global__ void __launch_bounds__(kThreads, 1) t1_stage_kernel(const __grid_cons
         if (abort_flag_s)
             for (int li = 0; li < g.nlayers; ++li) atomicExch(g.layer[li].status, (int32_t)MDBF_ERR_TIMEOUT);
     }
-    if (warp == 0) TR(22);
 }
 
 // max_c |V[c][t]| per mode (pack time): one block per mode
