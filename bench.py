@@ -240,8 +240,10 @@ def dist_setup(n_gpus):
 
 # ------------------------------------------------------------------ mdbf arm
 def measure(workload, kernel, steps, warmup, dist, world, local, no_graph=False, no_siblings=False, copies=0,
-            want_e2e=True, fuse_block=False):
-    """Time `steps` steps of one workload (after >= 3 untimed ones) and return the measured fields."""
+            want_e2e=True, fuse_block=False, min_timed_ms=0.0):
+    """Time `steps` steps of one workload (after >= 3 untimed ones) and return the measured fields.  min_timed_ms > 0
+    raises `steps` (the returned dict says to what) until the timed region lasts about that long, so that the
+    clock record of a short workload holds more than a sample or two."""
     import torch
     from paper_2512_24545_b200 import inputs, mdbf as M, replicas
     peaks, peak_kind = load_peaks()
@@ -350,6 +352,15 @@ def measure(workload, kernel, steps, warmup, dist, world, local, no_graph=False,
         for _ in range(max(3, warmup)):
             run_step()
         barrier()
+        if min_timed_ms > 0:
+            w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if flush is not None:
+                flush.fill_(1)
+            w0.record(stream)
+            run_step()
+            w1.record(stream)
+            torch.cuda.synchronize()
+            steps = max(steps, min(2000, int(min_timed_ms / max(w0.elapsed_time(w1), 1e-3)) + 1))
         sampler = ClockSampler(local)
         sampler.start()
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
@@ -457,7 +468,7 @@ def run_mdbf(args):
         also = {}
         for (wl, kern) in ALSO:
             m, _ = measure(wl, "auto" if kern == "fused" else kern, max(3, min(args.steps, 10)), args.warmup, None, 1, local,
-                           want_e2e=False, fuse_block=kern == "fused")
+                           want_e2e=False, fuse_block=kern == "fused", min_timed_ms=60.0)
             also[wl if kern == "auto" else f"{wl}:{kern}"] = {
                 "metric": m["metric"], "value": m["value"], "unit": m["unit"], "ms_per_step": m["ms_per_step"],
                 "steps": m["steps"], "gpu_launches": m["gpu_launches"], "clocks": m["clocks"], "roofline": m["roofline"],
