@@ -212,6 +212,15 @@ mdbf_status_t mdbf_prepare_host_staging(mdbf_handle_t h);
 mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T,
                                        int32_t act_dtype, void *stream);
 
+/* The same without the final synchronisation: the two copies and the kernels are enqueued on
+ * `stream` and the call returns; y_host holds the result once the caller has synchronised the
+ * stream (or an event recorded after the call).  x_host must stay unchanged and both buffers
+ * allocated until then; pageable buffers make the copies synchronous, so use pinned memory.  Calls
+ * on different handles pipeline on one stream: the next layer's input copy overlaps this layer's
+ * kernels.  Two calls on the SAME handle share its staging buffers and are ordered by the stream. */
+mdbf_status_t mdbf_linear_forward_host_async(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T,
+                                             int32_t act_dtype, void *stream);
+
 /* ------------------------------------------------- forward without allocation
  * (The paper has no counterpart: this entry point exists for deployment, not
  * for the method.)

@@ -629,8 +629,8 @@ mdbf_status_t mdbf_linear_forward_siblings(const mdbf_handle_t *layers, int32_t 
     return MDBF_OK;
 }
 
-mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T,
-                                       int32_t act_dtype, void *stream) {
+static mdbf_status_t forward_host_impl(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T, int32_t act_dtype, void *stream,
+                                       bool wait) {
     mdbf_status_t rc = check_handle(h, "mdbf_linear_forward_host");
     if (rc) return rc;
     if (!x_host || !y_host) { set_error("mdbf_linear_forward_host: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
@@ -650,8 +650,18 @@ mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void
     rc = forward_impl(h, L.xstage, L.ystage, T, act_dtype, st);
     if (rc) return rc;
     MDBF_CUDA(cudaMemcpyAsync(y_host, L.ystage, (size_t)T * L.d.d_out * es, cudaMemcpyDeviceToHost, st));
-    MDBF_CUDA(cudaStreamSynchronize(st));
+    if (wait) MDBF_CUDA(cudaStreamSynchronize(st));
     return MDBF_OK;
+}
+
+mdbf_status_t mdbf_linear_forward_host(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T,
+                                       int32_t act_dtype, void *stream) {
+    return forward_host_impl(h, x_host, y_host, T, act_dtype, stream, true);
+}
+
+mdbf_status_t mdbf_linear_forward_host_async(mdbf_handle_t h, const void *x_host, void *y_host, int32_t T,
+                                             int32_t act_dtype, void *stream) {
+    return forward_host_impl(h, x_host, y_host, T, act_dtype, stream, false);
 }
 
 mdbf_status_t mdbf_linear_forward_group(const mdbf_handle_t *layers, int32_t n, const void *const *xs, void *const *ys,

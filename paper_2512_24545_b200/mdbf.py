@@ -27,7 +27,7 @@ DTYPES = {"f32": F32, "f16": F16, "bf16": BF16}
 
 EXPORTS = (
     "mdbf_pack_signs", "mdbf_unpack_signs", "mdbf_pack", "mdbf_get_packed", "mdbf_get_envelope",
-    "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host", "mdbf_prepare_host_staging",
+    "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host", "mdbf_linear_forward_host_async", "mdbf_prepare_host_staging",
     "mdbf_linear_forward_static", "mdbf_linear_forward_sum", "mdbf_linear_forward_siblings", "mdbf_linear_forward_group",
     "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_poll_status", "mdbf_selftest_wait_timeout", "mdbf_debug_fail_alloc",
     "mdbf_last_launch_count",
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
     L.mdbf_set_kernel.argtypes = [vp, i32]
     L.mdbf_linear_forward.argtypes = [vp, vp, vp, i32, i32, vp]
     L.mdbf_linear_forward_host.argtypes = [vp, vp, vp, i32, i32, vp]
+    L.mdbf_linear_forward_host_async.argtypes = [vp, vp, vp, i32, i32, vp]
     L.mdbf_prepare_host_staging.argtypes = [vp]
     L.mdbf_linear_forward_static.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, vp]
     L.mdbf_linear_forward_sum.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp]
@@ -190,6 +191,11 @@ def mdbf_prepare_host_staging(h: int) -> None:
 
 def mdbf_linear_forward_host(h: int, x_host, y_host, T: int, act_dtype: int, stream: int = 0) -> None:
     _check(lib().mdbf_linear_forward_host(h, _addr(x_host), _addr(y_host), T, act_dtype, stream))
+
+
+def mdbf_linear_forward_host_async(h: int, x_host, y_host, T: int, act_dtype: int, stream: int = 0) -> None:
+    """Host buffers, no synchronisation: y_host is valid once the caller has synchronised `stream`."""
+    _check(lib().mdbf_linear_forward_host_async(h, _addr(x_host), _addr(y_host), T, act_dtype, stream))
 
 
 STATIC_MAX_KT = 262144

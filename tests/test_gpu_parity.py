@@ -229,3 +229,10 @@ def test_host_buffer_entry_point():
                                    torch.cuda.current_stream().cuda_stream)
         y_dev = g.forward(x)
         np.testing.assert_array_equal(yh.to(torch.float32).numpy(), y_dev)
+        # without the final synchronisation: valid once the caller has synchronised the stream
+        yh.zero_()
+        st = torch.cuda.current_stream().cuda_stream
+        M.mdbf_linear_forward_host_async(g.h, xh.data_ptr(), yh.data_ptr(), 2, M.BF16, st)
+        M.mdbf_linear_forward_host_async(g.h, xh.data_ptr(), yh.data_ptr(), 2, M.BF16, st)   # same handle: ordered by the stream
+        torch.cuda.current_stream().synchronize()
+        np.testing.assert_array_equal(yh.to(torch.float32).numpy(), y_dev)
