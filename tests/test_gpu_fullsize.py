@@ -140,3 +140,35 @@ def test_block70b_layers_full_size_2048_tokens(idx):
         assert M.mdbf_poll_status(g.h) == 0
         tok = np.array([0, 255, 256, 1033, 2047])
         check_tokens_rows(g, x, y, sampled_rows(spec.d_out, n=8), tok)
+
+
+SECOND_SEED = 90001
+
+
+@pytest.mark.parametrize("case", ["qproj1664", "qproj2560", "up_T1", "down_T16", "gate_T1", "down70b_T1", "prefill4096", "prefill11008"])
+def test_second_seed_with_outlier_channels(case):
+    """The margin under the 5e-3 bound does not hinge on the seeds of the workload table: every config once more with
+    other seeds, and with the 1 % outlier channels (x20) switched on for the prefill shapes as well."""
+    if case.startswith("qproj"):
+        spec, T = inputs.qproj(int(case[5:])), 1
+    elif case == "up_T1":
+        spec, T = inputs.mlp("up"), 1
+    elif case == "down_T16":
+        spec, T = inputs.mlp("down"), 16
+    elif case == "gate_T1":
+        spec, T = inputs.block70b()[4], 1
+    elif case == "down70b_T1":
+        spec, T = inputs.block70b()[6], 1
+    elif case == "prefill4096":
+        spec, T = inputs.prefill(4096, 16, 1.0), 2048
+    else:
+        spec, T = inputs.prefill(11008, 4, 1.5), 2048
+    spec = inputs.scaled(spec, seed=spec.seed + SECOND_SEED, outliers=True)
+    x = inputs.make_activations(spec, T)
+    rows = sampled_rows(spec.d_out, n=16, seed=1)
+    tok = np.unique(np.array([0, T // 3, T - 1]))
+    with GpuLayer(spec, T) as g:
+        kernels = [M.KERNEL_AUTO] + ([M.KERNEL_I8, M.KERNEL_TMEM] if T == 1 else [])
+        for kernel in kernels:
+            y = g.forward(x, kernel=kernel)
+            check_tokens_rows(g, x, y, rows, tok)
