@@ -68,7 +68,8 @@ typedef enum {
     MDBF_KERNEL_PREFILL = 3, /* T >= 2 (max_T >= 2): expanded order, tcgen05 GEMM of width l*T, TMEM accumulator, TMA operand */
     MDBF_KERNEL_TMEM = 4,   /* T = 1: tcgen05 MMA, sign (.) activation as bf16 operand in TMEM, one launch per stage */
     MDBF_KERNEL_MAT = 5,    /* T >= 2: W_hat tiles rebuilt on the fly (rank-l mini-MMA + sign XOR), one GEMM of width T */
-    MDBF_KERNEL_I8 = 6      /* T = 1: one persistent launch, packed bits as the 8-bit integer tcgen05 operand, fixed-point scaled input */
+    MDBF_KERNEL_I8 = 6      /* T = 1, l <= 16: packed bits as the 8-bit integer tcgen05 operand, 21-bit fixed-point scaled input;
+                             * two launches per stage (operand images, contraction on one CTA per SM) */
 } mdbf_kernel_t;
 
 typedef struct {
@@ -134,7 +135,8 @@ mdbf_status_t mdbf_get_desc(mdbf_handle_t h, mdbf_desc_t *out);
 /* Force a kernel for later forwards on this handle (tests, benchmarks).  MDBF_KERNEL_PREFILL
  * allocates that kernel's scratch (max_T * l * (d_in + k) * 2 bytes of pre-scaled operands) on the
  * first request, which synchronises the device; no forward ever does (a forward that is forced to
- * that kernel on a handle without the scratch returns MDBF_ERR_INVALID_ARG). */
+ * that kernel on a handle without the scratch returns MDBF_ERR_INVALID_ARG; a handle packed with
+ * max_T = 1 never has the scratch). */
 mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel /* mdbf_kernel_t */);
 
 /* ---------------------------------------------------------------- forward
