@@ -154,7 +154,9 @@ mdbf_status_t mdbf_set_kernel(mdbf_handle_t h, int32_t kernel /* mdbf_kernel_t *
  * order: the pre-scaled x and z (three); one token, TMEM-operand kernel: V_B, z and V_A (four);
  * one token, integer kernel: nothing (one).  fp16 envelopes are re-rounded to bf16 where they become
  * bf16 MMA operands.  Measured against the fp64 definition: 1.6e-3 to 3.7e-3 relative Frobenius
- * error on the 7B- and 70B-class shapes, bound 5e-3.
+ * error on the 7B- and 70B-class shapes, bound 5e-3.  x is expected to be finite: the integer
+ * kernel scales its operand by max|x| (and max|z|), so an Inf or NaN in x gives an unspecified y
+ * there, where the floating-point kernels would propagate it.
  * Asynchronous on `stream`; never allocates and never synchronises.  With the library choosing the
  * kernel, an x that the default kernels cannot take (T >= 2 and x not 16-byte aligned) is served
  * by the expanded order if mdbf_set_kernel(PREFILL) has prepared its scratch on this handle, else
