@@ -285,6 +285,31 @@ mdbf_status_t mdbf_reconstruct(mdbf_handle_t h, float *W, void *stream);
  * Synchronises the device.  Reading clears the word. */
 mdbf_status_t mdbf_poll_status(mdbf_handle_t h, int32_t *device_status);
 
+/* ---------------------------------------------------------------- quantizer, first step
+ * Multi-Envelope SVID of a device matrix (Eq. msvid-def):  MSVID_l[Z] = sign(Z) (.) TSVD_l(|Z|),  sign(0) = +1.
+ * It is the operator the paper applies to each balanced factor of W's truncated SVD to initialise MDBF
+ * (Eq. mesvid-init-compact); by Theorem 1 (Eq. rankl-error, Eq. Ustar) its result is the best approximation of Z
+ * among the matrices that keep Z's sign mask and have an envelope of rank <= l, with error
+ * (sum_{i > l} sigma_i(|Z|)^2)^(1/2).
+ *   Z         device, rows x cols fp32, row-major, read only
+ *   l         envelope rank, 1 <= l <= min(32, rows, cols)
+ *   n_iter    subspace iterations (two passes over Z each), >= 1; 2 already fixes the leading singular value,
+ *             8 leaves the squared error within about half a per cent of the optimum on Gaussian-like inputs
+ *   Q0        device, cols x l fp32: the start block of the iteration (e.g. i.i.d. Gaussian; the caller draws it,
+ *             so that a run is reproducible from its inputs alone); needs full column rank
+ *   S_packed  device, rows x ceil(cols / 32) uint32, written: the sign mask in the canonical packing of
+ *             mdbf_pack_signs (bit set <=> entry negative); exact
+ *   U, V      device, rows x l and cols x l fp32, written: balanced factors of the truncated envelope,
+ *             TSVD_l(|Z|) ~ U V^T, columns ordered by decreasing singular value (each pair is unique up to a
+ *             common sign only, and up to rotations inside a group of equal singular values)
+ *   sigma     device, l fp32, written: the estimated singular values; each is a lower bound of the exact one
+ * The truncated SVD is computed by block subspace iteration (hand-written CUDA-core kernels, fp32 with the small
+ * Gram matrices in fp64), not to machine precision: see n_iter.  Allocates its scratch ((rows + cols + cols *
+ * ceil(rows / 256)) * l floats) and synchronises `stream` before it returns.  Errors: INVALID_ARG, SHAPE, ALLOC,
+ * ARCH, CUDA. */
+mdbf_status_t mdbf_msvid(const float *Z, int64_t rows, int64_t cols, int32_t l, int32_t n_iter, const float *Q0,
+                         uint32_t *S_packed, float *U, float *V, float *sigma, void *stream);
+
 /* Test hook (no counterpart in the paper): the `nth` device allocation that the calling thread makes
  * inside this library from now on fails with MDBF_ERR_ALLOC without touching the device; nth <= 0
  * cancels a pending request.  A call that fails this way frees what it had allocated, publishes

@@ -104,6 +104,8 @@ SignView sign_view(const Layer &L, int which);      // 0: S_A, 1: S_B
 // thread-local error string
 void set_error(const char *fmt, ...);
 mdbf_status_t cuda_fail(cudaError_t e, const char *what);
+// MDBF_OK when the current device is one this library runs on (compute capability 10.x), MDBF_ERR_ARCH otherwise
+mdbf_status_t require_device(int *dev_out);
 // Every device allocation of the library goes through here: cudaMalloc, or - after mdbf_debug_fail_alloc(n) on the
 // calling thread - cudaErrorMemoryAllocation for the n-th call from now on without touching the device (the tests
 // inject allocation failures this way, on the host).

@@ -26,7 +26,7 @@ mdbf_status_t cuda_fail(cudaError_t e, const char *what) {
 }
 
 // The product has no CPU fallback: anything that computes needs an sm_100 device.
-static mdbf_status_t require_device(int *dev_out) {
+mdbf_status_t require_device(int *dev_out) {
     int n = 0;
     cudaError_t e = cudaGetDeviceCount(&n);
     if (e != cudaSuccess || n == 0) {

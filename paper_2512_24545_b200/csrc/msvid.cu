@@ -1,0 +1,408 @@
+// Multi-Envelope SVID on the GPU:  MSVID_l[Z] = sign(Z) (.) TSVD_l(|Z|)   (Eq. msvid-def), the operator the paper
+// applies to the balanced factors of a weight matrix to initialise MDBF (Eq. mesvid-init-compact) and, by
+// Theorem 1 (Eq. rankl-error / Eq. Ustar), the best approximation of Z among all matrices that keep Z's sign mask
+// and have an envelope of rank <= l.
+//
+// The sign mask is exact (bit set <=> entry negative, sign(0) = +1: the Notation section), written in the
+// library's canonical packing.  The truncated SVD of the demodulated envelope |Z| (N x M, never stored: every pass
+// takes the absolute value on the fly) is computed by block subspace iteration on a block of l columns:
+//
+//     Q  <- orth(Q0)                                 M x l start block, passed in by the caller
+//     repeat n_iter times:   Y <- orth(|Z| Q);   Q <- orth(|Z|^T Y)
+//     Y  <- |Z| Q;   Y^T Y = W diag(s^2) W^T        (l x l symmetric eigenproblem, Jacobi)
+//     U  <- Y W diag(s^-1/2),   V <- Q W diag(s^1/2)      balanced factors:  U V^T = Y Q^T ~ TSVD_l(|Z|)
+//
+// Two passes over Z per iteration, each a tall-skinny product on the CUDA cores (16 FMAs per 4 bytes of Z at
+// l = 16: the kernels are bound by HBM, not by arithmetic, so there is nothing for the tensor cores to win);
+// orth() is a Cholesky QR with the l x l Gram matrix accumulated and factorised in fp64.  What the iteration
+// leaves short of the exact TSVD is the mixing among the nearly equal singular values of the bulk: the largest
+// singular value converges in two iterations, the squared error of the envelope stays within a fraction of a
+// per cent of the optimum of Theorem 1 (the GPU tests bound it), and every Ritz value is a lower bound of the
+// singular value it estimates.
+#include <algorithm>
+#include <cmath>
+
+#include "common.cuh"
+
+namespace mdbf {
+namespace msv {
+
+constexpr int kMaxL = 32;
+
+// ------------------------------------------------------------------ sign mask
+// One warp per (row, word): bit c % 32 of word c / 32 is set <=> Z[r][c] is negative (a NaN counts as negative, as
+// in the comparison `not (z >= 0)` that defines sign() with sign(0) = +1); padding bits are 0.
+__global__ void sign_pack_kernel(const float *__restrict__ Z, long long p, long long q, int nwords, uint32_t *__restrict__ out) {
+    const long long total = p * nwords;
+    const int lane = threadIdx.x & 31;
+    for (long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < total; w += ((long long)gridDim.x * blockDim.x) >> 5) {
+        const long long r = w / nwords;
+        const long long c = (w - r * nwords) * 32 + lane;
+        const bool neg = c < q && !(Z[r * q + c] >= 0.f);
+        const uint32_t bits = __ballot_sync(0xffffffffu, neg);
+        if (lane == 0) out[w] = bits;
+    }
+}
+
+// ------------------------------------------------------------------ Y = |Z| Q
+// CTA = 4 warps x 4 rows.  Q (M x LP, zero beyond the l real columns) is staged tile by tile, transposed, in shared
+// memory; a lane owns the columns lane, lane + 32, ... of the tile and keeps 4 x LP partial sums in registers, so a
+// value of Q read from shared memory serves four rows.
+constexpr int AQ_WARPS = 4, AQ_ROWS = 4, AQ_TJ = 256;
+template <int LP>
+__global__ void __launch_bounds__(AQ_WARPS * 32) absz_q_kernel(const float *__restrict__ Z, int p, int q, const float *__restrict__ Q,
+                                                              float *__restrict__ Y) {
+    __shared__ float Qs[LP][AQ_TJ + 1];                // + 1: the transposing store hits LP different banks
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r0 = (blockIdx.x * AQ_WARPS + warp) * AQ_ROWS;
+    float acc[AQ_ROWS][LP];
+#pragma unroll
+    for (int r = 0; r < AQ_ROWS; ++r)
+#pragma unroll
+        for (int t = 0; t < LP; ++t) acc[r][t] = 0.f;
+    for (int j0 = 0; j0 < q; j0 += AQ_TJ) {
+        __syncthreads();
+        for (int e = threadIdx.x; e < AQ_TJ * LP; e += AQ_WARPS * 32) {
+            const int jj = e / LP, t = e - jj * LP;
+            Qs[t][jj] = j0 + jj < q ? Q[(size_t)(j0 + jj) * LP + t] : 0.f;
+        }
+        __syncthreads();
+        float z[AQ_ROWS][AQ_TJ / 32];
+#pragma unroll
+        for (int r = 0; r < AQ_ROWS; ++r)
+#pragma unroll
+            for (int s = 0; s < AQ_TJ / 32; ++s) {
+                const int j = j0 + s * 32 + lane;
+                z[r][s] = (r0 + r < p && j < q) ? fabsf(Z[(size_t)(r0 + r) * q + j]) : 0.f;
+            }
+#pragma unroll
+        for (int s = 0; s < AQ_TJ / 32; ++s)
+#pragma unroll
+            for (int t = 0; t < LP; ++t) {
+                const float qv = Qs[t][s * 32 + lane];
+#pragma unroll
+                for (int r = 0; r < AQ_ROWS; ++r) acc[r][t] = fmaf(z[r][s], qv, acc[r][t]);
+            }
+    }
+#pragma unroll
+    for (int r = 0; r < AQ_ROWS; ++r)
+#pragma unroll
+        for (int t = 0; t < LP; ++t) {
+            float v = acc[r][t];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (lane == 0 && r0 + r < p) Y[(size_t)(r0 + r) * LP + t] = v;
+        }
+}
+
+// ------------------------------------------------------------------ W = |Z|^T Y
+// CTA = 256 columns (thread = column) x a chunk of 256 rows; the chunk's rows of Y sit in shared memory and are read
+// by all threads at once (broadcast).  Partial sums per chunk go to P[chunk][column][LP]; a second kernel adds the
+// chunks in order (no atomics: the result does not depend on scheduling).
+constexpr int ZY_COLS = 256, ZY_ROWS = 256;
+template <int LP>
+__global__ void __launch_bounds__(ZY_COLS) abszT_y_kernel(const float *__restrict__ Z, int p, int q, const float *__restrict__ Y,
+                                                           float *__restrict__ P) {
+    __shared__ float Ys[ZY_ROWS][LP];
+    const int j = blockIdx.x * ZY_COLS + threadIdx.x;
+    const int i0 = blockIdx.y * ZY_ROWS;
+    const int nrows = min(ZY_ROWS, p - i0);
+    for (int e = threadIdx.x; e < ZY_ROWS * LP; e += ZY_COLS) {
+        const int i = e / LP, t = e - i * LP;
+        Ys[i][t] = i < nrows ? Y[(size_t)(i0 + i) * LP + t] : 0.f;
+    }
+    __syncthreads();
+    float acc[LP];
+#pragma unroll
+    for (int t = 0; t < LP; ++t) acc[t] = 0.f;
+    if (j < q) {
+        const float *zp = Z + (size_t)i0 * q + j;
+        int i = 0;
+        for (; i + 8 <= nrows; i += 8) {
+            float z[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) z[u] = fabsf(zp[(size_t)(i + u) * q]);
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+#pragma unroll
+                for (int t = 0; t < LP; ++t) acc[t] = fmaf(z[u], Ys[i + u][t], acc[t]);
+        }
+        for (; i < nrows; ++i) {
+            const float z = fabsf(zp[(size_t)i * q]);
+#pragma unroll
+            for (int t = 0; t < LP; ++t) acc[t] = fmaf(z, Ys[i][t], acc[t]);
+        }
+        float *out = P + ((size_t)blockIdx.y * q + j) * LP;
+#pragma unroll
+        for (int t = 0; t < LP; ++t) out[t] = acc[t];
+    }
+}
+__global__ void chunk_sum_kernel(const float *__restrict__ P, int nchunks, size_t n, float *__restrict__ out) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        float v = 0.f;
+        for (int c = 0; c < nchunks; ++c) v += P[(size_t)c * n + i];
+        out[i] = v;
+    }
+}
+
+// ------------------------------------------------------------------ orth(): Cholesky QR, Gram matrix in fp64
+// partial Gram matrices of chunks of 256 rows of a tall matrix A (n x LP)
+template <int LP>
+__global__ void __launch_bounds__(256) gram_kernel(const float *__restrict__ A, int n, double *__restrict__ Gp) {
+    __shared__ float As[256][LP + 1];
+    const int i0 = blockIdx.x * 256;
+    const int nrows = min(256, n - i0);
+    for (int e = threadIdx.x; e < 256 * LP; e += 256) {
+        const int i = e / LP, t = e - i * LP;
+        As[i][t] = i < nrows ? A[(size_t)(i0 + i) * LP + t] : 0.f;
+    }
+    __syncthreads();
+    for (int pr = threadIdx.x; pr < LP * LP; pr += 256) {
+        const int a = pr / LP, b = pr - a * LP;
+        double s = 0.0;
+        if (b <= a)
+            for (int i = 0; i < nrows; ++i) s += (double)As[i][a] * (double)As[i][b];
+        Gp[(size_t)blockIdx.x * LP * LP + pr] = s;
+    }
+}
+// One CTA: G = sum of the partial Gram matrices = L L^T; M[b][a] = (L^-1)[a][b], so that A M has orthonormal columns.
+// A zero (or numerically vanished) pivot - a padding column, or a block wider than the rank of the matrix - leaves
+// its column as it is instead of dividing by zero.
+template <int LP>
+__global__ void __launch_bounds__(LP * LP < 32 ? 32 : LP * LP) chol_kernel(const double *__restrict__ Gp, int nchunks, float *__restrict__ M) {
+    __shared__ double G[LP][LP + 1], Li[LP][LP + 1];
+    const int tid = threadIdx.x;
+    const int a = tid / LP, b = tid - a * LP;
+    if (tid < LP * LP) {
+        double s = 0.0;
+        for (int c = 0; c < nchunks; ++c) s += Gp[(size_t)c * LP * LP + tid];
+        G[a][b] = s;                                   // lower triangle (b <= a) holds the sums
+        Li[a][b] = 0.0;
+    }
+    __syncthreads();
+    double scale = 0.0;
+    if (tid == 0)
+        for (int k = 0; k < LP; ++k) scale = fmax(scale, G[k][k]);
+    // column-by-column Cholesky on the lower triangle, one thread per row
+    for (int k = 0; k < LP; ++k) {
+        if (tid == 0) {
+            const double d = G[k][k];
+            G[k][k] = d > 1e-24 * scale && d > 0.0 ? sqrt(d) : 0.0;
+        }
+        __syncthreads();
+        const double d = G[k][k];
+        if (tid > k && tid < LP) G[tid][k] = d > 0.0 ? G[tid][k] / d : 0.0;
+        __syncthreads();
+        if (tid > k && tid < LP)
+            for (int jj = k + 1; jj <= tid; ++jj) G[tid][jj] -= G[tid][k] * G[jj][k];
+        __syncthreads();
+    }
+    // inverse of the lower-triangular factor, one thread per column
+    if (tid < LP) {
+        const int c = tid;
+        for (int i = c; i < LP; ++i) {
+            double s = i == c ? 1.0 : 0.0;
+            for (int k = c; k < i; ++k) s -= G[i][k] * Li[k][c];
+            Li[i][c] = G[i][i] > 0.0 ? s / G[i][i] : (i == c ? 1.0 : 0.0);
+        }
+    }
+    __syncthreads();
+    if (tid < LP * LP) M[tid] = (float)Li[b][a];        // M[a][b] with a = row index of M: M[a][b] = Li[b][a]
+}
+// A <- A M, row by row (M is LP x LP, row-major)
+template <int LP>
+__global__ void __launch_bounds__(256) right_mul_kernel(float *__restrict__ A, int n, const float *__restrict__ M, float *__restrict__ out,
+                                                        int out_cols) {
+    __shared__ float Ms[LP][LP];
+    for (int e = threadIdx.x; e < LP * LP; e += 256) Ms[e / LP][e % LP] = M[e];
+    __syncthreads();
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= n) return;
+    float a[LP], o[LP];
+#pragma unroll
+    for (int t = 0; t < LP; ++t) { a[t] = A[(size_t)i * LP + t]; o[t] = 0.f; }
+#pragma unroll
+    for (int b = 0; b < LP; ++b)
+#pragma unroll
+        for (int t = 0; t < LP; ++t) o[t] = fmaf(a[b], Ms[b][t], o[t]);
+    if (out) {
+        for (int t = 0; t < out_cols; ++t) out[(size_t)i * out_cols + t] = o[t];     // compact result (the first out_cols columns)
+    } else {
+#pragma unroll
+        for (int t = 0; t < LP; ++t) A[(size_t)i * LP + t] = o[t];
+    }
+}
+
+// ------------------------------------------------------------------ the small eigenproblem
+// One thread: cyclic Jacobi on G = Y^T Y (l x l, fp64), eigenvalues sorted in descending order; writes the singular
+// values s_t = sqrt(lambda_t) and the two LP x LP matrices that turn (Y, Q) into the balanced factors:
+// MU[b][t] = W[b][t] s_t^-1/2, MV[b][t] = W[b][t] s_t^1/2 (zero columns beyond l and for vanished singular values).
+template <int LP>
+__global__ void jacobi_kernel(const double *__restrict__ Gp, int nchunks, int l, float *__restrict__ sigma, float *__restrict__ MU,
+                              float *__restrict__ MV) {
+    __shared__ double G[LP][LP], W[LP][LP];
+    if (threadIdx.x != 0) return;
+    for (int a = 0; a < LP; ++a)
+        for (int b = 0; b <= a; ++b) {
+            double s = 0.0;
+            for (int c = 0; c < nchunks; ++c) s += Gp[(size_t)c * LP * LP + a * LP + b];
+            G[a][b] = G[b][a] = s;
+        }
+    for (int a = 0; a < LP; ++a)
+        for (int b = 0; b < LP; ++b) W[a][b] = a == b ? 1.0 : 0.0;
+    for (int sweep = 0; sweep < 60; ++sweep) {
+        double off = 0.0, diag = 0.0;
+        for (int a = 0; a < l; ++a) {
+            diag += G[a][a] * G[a][a];
+            for (int b = 0; b < a; ++b) off += G[a][b] * G[a][b];
+        }
+        if (off <= 1e-30 * diag) break;
+        for (int pi = 0; pi < l - 1; ++pi)
+            for (int qi = pi + 1; qi < l; ++qi) {
+                const double apq = G[pi][qi];
+                if (apq == 0.0) continue;
+                const double theta = (G[qi][qi] - G[pi][pi]) / (2.0 * apq);
+                const double t = (theta >= 0.0 ? 1.0 : -1.0) / (fabs(theta) + sqrt(theta * theta + 1.0));
+                const double c = 1.0 / sqrt(t * t + 1.0), s = t * c;
+                for (int k = 0; k < l; ++k) {
+                    const double gkp = G[k][pi], gkq = G[k][qi];
+                    G[k][pi] = c * gkp - s * gkq;
+                    G[k][qi] = s * gkp + c * gkq;
+                }
+                for (int k = 0; k < l; ++k) {
+                    const double gpk = G[pi][k], gqk = G[qi][k];
+                    G[pi][k] = c * gpk - s * gqk;
+                    G[qi][k] = s * gpk + c * gqk;
+                }
+                for (int k = 0; k < l; ++k) {
+                    const double wkp = W[k][pi], wkq = W[k][qi];
+                    W[k][pi] = c * wkp - s * wkq;
+                    W[k][qi] = s * wkp + c * wkq;
+                }
+            }
+    }
+    int order[LP];
+    for (int t = 0; t < l; ++t) order[t] = t;
+    for (int t = 0; t < l; ++t)                        // selection sort, descending eigenvalues
+        for (int u = t + 1; u < l; ++u)
+            if (G[order[u]][order[u]] > G[order[t]][order[t]]) { const int x = order[t]; order[t] = order[u]; order[u] = x; }
+    const double top = l > 0 ? fmax(G[order[0]][order[0]], 0.0) : 0.0;
+    for (int t = 0; t < LP; ++t) {
+        double lam = t < l ? G[order[t]][order[t]] : 0.0;
+        if (!(lam > 1e-24 * top)) lam = 0.0;
+        const double sv = sqrt(lam), rs = sqrt(sv);
+        if (t < l) sigma[t] = (float)sv;
+        for (int b = 0; b < LP; ++b) {
+            const double w = (t < l && b < l) ? W[b][order[t]] : 0.0;
+            MU[b * LP + t] = (float)(rs > 0.0 ? w / rs : 0.0);
+            MV[b * LP + t] = (float)(w * rs);
+        }
+    }
+}
+
+// start block: Q0 (M x l, compact) -> Q (M x LP, zero padding)
+__global__ void pad_kernel(const float *__restrict__ src, size_t n, int l, int LP, float *__restrict__ dst) {
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n * LP; e += (size_t)gridDim.x * blockDim.x) {
+        const size_t i = e / LP;
+        const int t = (int)(e - i * LP);
+        dst[e] = t < l ? src[i * l + t] : 0.f;
+    }
+}
+
+struct Scratch {
+    float *Q = nullptr, *Y = nullptr, *P = nullptr, *M = nullptr, *MU = nullptr, *MV = nullptr;
+    double *Gp = nullptr;
+    ~Scratch() {
+        void *ptrs[] = {Q, Y, P, M, MU, MV, Gp};
+        for (void *x : ptrs)
+            if (x) cudaFree(x);
+    }
+};
+
+template <int LP>
+static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st) {
+    const int chunks = ceil_div(n, 256);
+    gram_kernel<LP><<<chunks, 256, 0, st>>>(A, n, w.Gp);
+    chol_kernel<LP><<<1, LP * LP < 32 ? 32 : LP * LP, 0, st>>>(w.Gp, chunks, w.M);
+    right_mul_kernel<LP><<<chunks, 256, 0, st>>>(A, n, w.M, nullptr, 0);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}
+
+template <int LP>
+static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const float *Q0, uint32_t *S, float *U, float *V, float *sigma,
+                         cudaStream_t st) {
+    Scratch w;
+    const int zy_chunks = ceil_div(p, ZY_ROWS);
+    const int gchunks = ceil_div(max(p, q), 256);
+    MDBF_CUDA(dev_malloc(&w.Q, (size_t)q * LP * sizeof(float)));
+    MDBF_CUDA(dev_malloc(&w.Y, (size_t)p * LP * sizeof(float)));
+    MDBF_CUDA(dev_malloc(&w.P, (size_t)zy_chunks * q * LP * sizeof(float)));
+    MDBF_CUDA(dev_malloc(&w.Gp, (size_t)gchunks * LP * LP * sizeof(double)));
+    MDBF_CUDA(dev_malloc(&w.M, (size_t)LP * LP * sizeof(float)));
+    MDBF_CUDA(dev_malloc(&w.MU, (size_t)LP * LP * sizeof(float)));
+    MDBF_CUDA(dev_malloc(&w.MV, (size_t)LP * LP * sizeof(float)));
+
+    const int nwords = ceil_div(q, 32);
+    sign_pack_kernel<<<(int)std::min<long long>(((long long)p * nwords * 32 + 255) / 256, 148LL * 16), 256, 0, st>>>(Z, p, q, nwords, S);
+    pad_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(Q0, (size_t)q, l, LP, w.Q);
+    MDBF_CUDA(cudaGetLastError());
+    mdbf_status_t rc = orth<LP>(w.Q, q, w, st);                        // twice: the start block may be badly conditioned
+    if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st);
+    if (rc) return rc;
+    const dim3 zy_grid(ceil_div(q, ZY_COLS), zy_chunks);
+    const int aq_grid = ceil_div(p, AQ_WARPS * AQ_ROWS);
+    for (int it = 0; it < n_iter; ++it) {
+        absz_q_kernel<LP><<<aq_grid, AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y);
+        rc = orth<LP>(w.Y, p, w, st);
+        if (rc) return rc;
+        abszT_y_kernel<LP><<<zy_grid, ZY_COLS, 0, st>>>(Z, p, q, w.Y, w.P);
+        chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, zy_chunks, (size_t)q * LP, w.Q);
+        MDBF_CUDA(cudaGetLastError());
+        rc = orth<LP>(w.Q, q, w, st);
+        if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st);               // the right block carries the result: orthonormal to fp32
+        if (rc) return rc;
+    }
+    absz_q_kernel<LP><<<aq_grid, AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y);
+    const int ychunks = ceil_div(p, 256);
+    gram_kernel<LP><<<ychunks, 256, 0, st>>>(w.Y, p, w.Gp);
+    jacobi_kernel<LP><<<1, 32, 0, st>>>(w.Gp, ychunks, l, sigma, w.MU, w.MV);
+    right_mul_kernel<LP><<<ychunks, 256, 0, st>>>(w.Y, p, w.MU, U, l);
+    right_mul_kernel<LP><<<ceil_div(q, 256), 256, 0, st>>>(w.Q, q, w.MV, V, l);
+    MDBF_CUDA(cudaGetLastError());
+    MDBF_CUDA(cudaStreamSynchronize(st));                              // the scratch is freed on return
+    return MDBF_OK;
+}
+
+}  // namespace msv
+}  // namespace mdbf
+
+using namespace mdbf;
+
+extern "C" mdbf_status_t mdbf_msvid(const float *Z, int64_t rows, int64_t cols, int32_t l, int32_t n_iter, const float *Q0,
+                                    uint32_t *S_packed, float *U, float *V, float *sigma, void *stream) {
+    if (!Z || !Q0 || !S_packed || !U || !V || !sigma) { set_error("mdbf_msvid: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    if (rows < 1 || cols < 1 || rows > (1 << 24) || cols > (1 << 24) || rows * cols > (1LL << 40)) {
+        set_error("mdbf_msvid: size %lld x %lld outside the supported range", (long long)rows, (long long)cols);
+        return MDBF_ERR_SHAPE;
+    }
+    if (l < 1 || l > msv::kMaxL || l > rows || l > cols) {
+        set_error("mdbf_msvid: l=%d outside [1, min(%d, rows, cols)]", l, msv::kMaxL);
+        return MDBF_ERR_SHAPE;
+    }
+    if (n_iter < 1 || n_iter > 1000) { set_error("mdbf_msvid: n_iter=%d outside [1, 1000]", n_iter); return MDBF_ERR_SHAPE; }
+    mdbf_status_t rc = require_device(nullptr);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int p = (int)rows, q = (int)cols;
+    int LP = 1;
+    while (LP < l) LP *= 2;
+    switch (LP) {
+        case 1: return msv::run<1>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
+        case 2: return msv::run<2>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
+        case 4: return msv::run<4>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
+        case 8: return msv::run<8>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
+        case 16: return msv::run<16>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
+        default: return msv::run<32>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
+    }
+}

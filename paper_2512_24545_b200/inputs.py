@@ -135,3 +135,28 @@ def block70b() -> List[LayerSpec]:
 def scaled(spec: LayerSpec, **kw) -> LayerSpec:
     """A copy of `spec` with some fields replaced (reduced shapes for quick tests)."""
     return replace(spec, **kw)
+
+
+# ---------------------------------------------------------------- inputs of the quantizer's first step
+def make_factor_matrix(rows: int, cols: int, seed: int, special_values: bool = True) -> np.ndarray:
+    """A dense fp32 matrix to hand to the Multi-Envelope SVID: Gaussian entries under log-normal row and column
+    scales (the envelope of a trained factor is not flat), a few exact zeros, a negative zero and a tiny negative
+    entry so that the sign convention sign(0) = +1 is exercised.  Stands in for the balanced SVD factors of a
+    checkpoint's weight matrix, which are not available here."""
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, rows, cols])))
+    Z = rng.standard_normal((rows, cols))
+    Z *= np.exp(0.5 * rng.standard_normal((rows, 1))) * np.exp(0.5 * rng.standard_normal((1, cols)))
+    Z = Z.astype(np.float32)
+    if special_values and rows * cols >= 8:
+        flat = Z.reshape(-1)
+        idx = rng.choice(flat.size, size=min(8, flat.size), replace=False)
+        flat[idx[:-2]] = 0.0
+        flat[idx[-2]] = -0.0
+        flat[idx[-1]] = -1e-30
+    return Z
+
+
+def make_start_block(cols: int, l: int, seed: int) -> np.ndarray:
+    """The cols x l Gaussian block a subspace iteration starts from (drawn here, passed in as an input)."""
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, cols, l, 7])))
+    return rng.standard_normal((cols, l)).astype(np.float32)

@@ -1,0 +1,129 @@
+"""Multi-Envelope SVID on the GPU (mdbf_msvid, Eq. msvid-def) against the oracle: the sign mask bit for bit, and the
+truncated envelope through what is unique about it - the singular values and the error of Theorem 1
+(Eq. rankl-error), which the exact TSVD attains and no rank-l envelope can beat.  The factors themselves are not
+compared: they are unique only up to signs and to rotations among equal singular values, and the GPU computes
+them by subspace iteration, not by a full SVD."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mdbf_oracle as orc
+from paper_2512_24545_b200 import inputs, mdbf as M
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    from paper_2512_24545_b200 import build
+    build.build()
+    assert torch.cuda.is_available()
+
+
+def run_msvid(Z, l, n_iter, Q0=None, seed=11):
+    rows, cols = Z.shape
+    Q0 = inputs.make_start_block(cols, l, seed) if Q0 is None else Q0
+    Zd = torch.from_numpy(np.ascontiguousarray(Z, dtype=np.float32)).cuda()
+    Qd = torch.from_numpy(np.ascontiguousarray(Q0, dtype=np.float32)).cuda()
+    nwords = (cols + 31) // 32
+    Sd = torch.full((rows, nwords), -1, dtype=torch.int32, device="cuda")
+    Ud = torch.full((rows, l), float("nan"), dtype=torch.float32, device="cuda")
+    Vd = torch.full((cols, l), float("nan"), dtype=torch.float32, device="cuda")
+    sd = torch.full((l,), float("nan"), dtype=torch.float32, device="cuda")
+    M.mdbf_msvid(Zd.data_ptr(), rows, cols, l, n_iter, Qd.data_ptr(), Sd.data_ptr(), Ud.data_ptr(), Vd.data_ptr(), sd.data_ptr(),
+                 torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    return (Sd.cpu().numpy().view(np.uint32), Ud.cpu().numpy().astype(np.float64), Vd.cpu().numpy().astype(np.float64),
+            sd.cpu().numpy().astype(np.float64))
+
+
+def envelope_error(Z, U, V):
+    return np.linalg.norm(np.abs(Z.astype(np.float64)) - U @ V.T)
+
+
+@pytest.mark.parametrize("shape", [(300, 517), (1024, 768), (129, 33), (64, 2000), (2000, 64), (33, 40)])
+@pytest.mark.parametrize("l", [1, 4, 16])
+def test_sign_mask_exact_and_envelope_near_the_optimum(shape, l):
+    rows, cols = shape
+    Z = inputs.make_factor_matrix(rows, cols, seed=5)
+    S_ref, _, _ = orc.msvid(Z, l)
+    sv = np.linalg.svd(np.abs(Z.astype(np.float64)), compute_uv=False)
+    tail = np.sqrt(np.sum(sv[l:] ** 2))                                    # Eq. rankl-error
+    Sp, U, V, s = run_msvid(Z, l, n_iter=8)
+    # the mask: integer work, bit for bit (sign(0) = sign(-0) = +1, the tiny negative entry is -1)
+    np.testing.assert_array_equal(Sp, orc.pack_signs(S_ref))
+    # singular values: the leading one has converged; every estimate is a lower bound of the exact value (Ritz
+    # values of a projection) and not far below it after eight iterations
+    assert np.all(np.isfinite(U)) and np.all(np.isfinite(V)) and np.all(np.isfinite(s))
+    assert abs(s[0] - sv[0]) <= 2e-5 * sv[0]
+    assert np.all(s <= sv[:l] * (1 + 2e-5))
+    assert np.all(s >= 0.80 * sv[:l])
+    assert np.all(np.diff(s) <= 1e-6 * sv[0])                              # descending
+    # the envelope: no rank-l matrix beats the tail of Theorem 1, and the iteration ends within 1 % of it
+    err = envelope_error(Z, U, V)
+    assert err >= tail * (1 - 1e-5)
+    assert err <= tail * 1.01 + 1e-5 * sv[0]
+    # remodulated with the mask the error is the same number (Eq. envelope-isometry)
+    S = orc.unpack_signs(Sp, cols).astype(np.float64)
+    assert abs(np.linalg.norm(Z.astype(np.float64) - S * (U @ V.T)) - err) <= 1e-9 * sv[0]
+    # balanced factors: both columns of a pair carry the square root of their singular value
+    np.testing.assert_allclose(np.linalg.norm(U, axis=0), np.sqrt(s), rtol=2e-4)
+    np.testing.assert_allclose(np.linalg.norm(V, axis=0), np.sqrt(s), rtol=2e-4)
+
+
+def test_error_decreases_with_envelope_rank_and_with_iterations():
+    Z = inputs.make_factor_matrix(700, 900, seed=6)
+    errs_l = [envelope_error(Z, *run_msvid(Z, l, n_iter=6)[1:3]) for l in (1, 2, 4, 8, 16, 32)]
+    assert all(b <= a * (1 + 1e-6) for a, b in zip(errs_l, errs_l[1:]))   # F_1(S) is inside F_l(S): Theorem 1's remark
+    errs_it = [envelope_error(Z, *run_msvid(Z, 16, n_iter=n)[1:3]) for n in (1, 2, 4, 8, 16)]
+    assert all(b <= a * (1 + 1e-6) for a, b in zip(errs_it, errs_it[1:]))
+    sv = np.linalg.svd(np.abs(Z.astype(np.float64)), compute_uv=False)
+    assert errs_it[-1] <= np.sqrt(np.sum(sv[16:] ** 2)) * 1.005
+
+
+def test_envelope_of_exact_low_rank_is_reproduced():
+    """|Z| of rank 3 and l = 4: the block is wider than the rank, the fourth singular value is zero, the first three
+    reproduce |Z| (and Z, with the mask) to fp32 accuracy."""
+    rng = np.random.default_rng(17)
+    E = np.abs(rng.standard_normal((257, 3))) @ np.abs(rng.standard_normal((3, 190)))
+    S = np.where(rng.random((257, 190)) < 0.5, -1.0, 1.0)
+    Z = (S * E).astype(np.float32)
+    Sp, U, V, s = run_msvid(Z, 4, n_iter=3)
+    np.testing.assert_array_equal(Sp, orc.pack_signs(np.where(Z >= 0, 1, -1).astype(np.int8)))
+    sv = np.linalg.svd(np.abs(Z.astype(np.float64)), compute_uv=False)
+    np.testing.assert_allclose(s[:3], sv[:3], rtol=2e-5)
+    assert s[3] <= 1e-3 * sv[0]
+    assert envelope_error(Z, U, V) <= 2e-5 * np.linalg.norm(Z)
+    Sm = orc.unpack_signs(Sp, 190).astype(np.float64)
+    assert np.linalg.norm(Z - Sm * (U @ V.T)) <= 2e-5 * np.linalg.norm(Z)
+
+
+def test_full_size_factor():
+    """4096 x 4096, l = 16: the mask against the oracle on every row, the singular values against the full SVD, the
+    envelope error through ||A - A Q Q^T||^2 = ||A||^2 - sum s_t^2 (Q orthonormal) against Theorem 1's tail."""
+    Z = inputs.make_factor_matrix(4096, 4096, seed=7)
+    Sp, U, V, s = run_msvid(Z, 16, n_iter=4)
+    np.testing.assert_array_equal(Sp, orc.pack_signs(np.where(Z >= 0, 1, -1).astype(np.int8)))
+    A = np.abs(Z.astype(np.float64))
+    sv = np.linalg.svd(A, compute_uv=False)
+    assert abs(s[0] - sv[0]) <= 2e-5 * sv[0]
+    assert np.all(s <= sv[:16] * (1 + 2e-5)) and np.all(s >= 0.8 * sv[:16])
+    tail2 = np.sum(sv[16:] ** 2)
+    err2 = np.sum(A * A) - np.sum(s ** 2)
+    assert tail2 * (1 - 1e-4) <= err2 <= tail2 * 1.01
+
+
+def test_argument_errors():
+    Z = torch.zeros((8, 8), dtype=torch.float32, device="cuda")
+    Q = torch.ones((8, 2), dtype=torch.float32, device="cuda")
+    S = torch.zeros((8, 1), dtype=torch.int32, device="cuda")
+    U = torch.zeros((8, 2), dtype=torch.float32, device="cuda")
+    s = torch.zeros((2,), dtype=torch.float32, device="cuda")
+    args = lambda: (Z.data_ptr(), 8, 8, 2, 2, Q.data_ptr(), S.data_ptr(), U.data_ptr(), U.data_ptr(), s.data_ptr())
+    for bad, status in (((0,), M.ERR_INVALID_ARG), ((1, 0), M.ERR_SHAPE), ((3, 0), M.ERR_SHAPE), ((3, 33), M.ERR_SHAPE),
+                        ((3, 9), M.ERR_SHAPE), ((4, 0), M.ERR_SHAPE)):
+        a = list(args())
+        a[bad[0]] = bad[1] if len(bad) > 1 else 0
+        with pytest.raises(M.MdbfError) as e:
+            M.mdbf_msvid(*a)
+        assert e.value.status == status
