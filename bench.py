@@ -445,6 +445,119 @@ def measure(workload, kernel, steps, warmup, dist, world, local, no_graph=False,
     return out, cpu_args
 
 
+# ------------------------------------------------------------ quantizer, first step (MSVID)
+def measure_msvid(workload, steps, warmup, dist, world, local, want_e2e=True, min_timed_ms=0.0):
+    """msvid_<rows>x<cols>_l<l>[_it<n>]: one step = one mdbf_msvid call on a resident rows x cols fp32 matrix (sign mask +
+    rank-l envelope, n subspace iterations).  Algorithmic bytes: the sign pass and the 2 n + 1 product passes each
+    read Z once (rows * cols * 4 bytes; |Z| is never stored), plus the mask and the factors written."""
+    import re
+    import torch
+    from paper_2512_24545_b200 import inputs, mdbf as M, replicas
+    m = re.match(r"msvid_(\d+)x(\d+)_l(\d+)(?:_it(\d+))?$", workload)
+    if not m:
+        raise SystemExit(f"unknown workload {workload}")
+    rows, cols, l = int(m.group(1)), int(m.group(2)), int(m.group(3))
+    n_iter = int(m.group(4)) if m.group(4) else 4
+    peaks, peak_kind = load_peaks()
+    stream = torch.cuda.Stream()
+    st = stream.cuda_stream
+    Zh = torch.from_numpy(inputs.make_factor_matrix(rows, cols, seed=8)).pin_memory()
+    Qh = torch.from_numpy(inputs.make_start_block(cols, l, seed=8)).pin_memory()
+    Zd, Qd = Zh.cuda(), Qh.cuda()
+    nwords = (cols + 31) // 32
+    Sd = torch.zeros((rows, nwords), dtype=torch.int32, device="cuda")
+    Ud = torch.zeros((rows, l), dtype=torch.float32, device="cuda")
+    Vd = torch.zeros((cols, l), dtype=torch.float32, device="cuda")
+    sd = torch.zeros((l,), dtype=torch.float32, device="cuda")
+    Sh, Uh, Vh = (torch.zeros_like(t, device="cpu").pin_memory() for t in (Sd, Ud, Vd))
+    ws_bytes = M.mdbf_msvid_workspace_bytes(rows, cols, l)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    passes = 2 * n_iter + 2
+    step_bytes = passes * rows * cols * 4 + rows * nwords * 4 + (rows + cols) * l * 4
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda") if rows * cols * 4 < 2 * 126e6 else None
+
+    def step():
+        M.mdbf_msvid(Zd.data_ptr(), rows, cols, l, n_iter, Qd.data_ptr(), Sd.data_ptr(), Ud.data_ptr(), Vd.data_ptr(), sd.data_ptr(),
+                     ws.data_ptr(), ws_bytes, st)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(3, warmup)):
+            step()
+        barrier()
+        if min_timed_ms > 0:
+            w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            w0.record(stream); step(); w1.record(stream)
+            torch.cuda.synchronize()
+            steps = max(steps, min(2000, int(min_timed_ms / max(w0.elapsed_time(w1), 1e-3)) + 1))
+        sampler = ClockSampler(local)
+        sampler.start()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for (e0, e1) in ev:
+            if flush is not None:
+                flush.fill_(1)
+            e0.record(stream)
+            step()
+            e1.record(stream)
+        barrier()
+        clocks = sampler.stop()
+        ms = sum(e0.elapsed_time(e1) for e0, e1 in ev)
+        e2e_steps = max(1, min(steps, 3))
+        e2e_s = 0.0
+        if want_e2e:
+            t0 = time.perf_counter()
+            for _ in range(e2e_steps):
+                Zd.copy_(Zh, non_blocking=True)
+                Qd.copy_(Qh, non_blocking=True)
+                step()
+                Sh.copy_(Sd, non_blocking=True); Uh.copy_(Ud, non_blocking=True); Vh.copy_(Vd, non_blocking=True)
+                stream.synchronize()
+            e2e_s = time.perf_counter() - t0
+    ms_max, e2e_ms_max = replicas.max_over_ranks([ms, e2e_s * 1e3], dist, device="cuda")
+    value = replicas.aggregate_throughput(step_bytes * steps / 1e9, world, ms_max / 1e3)
+    per_gpu = step_bytes * steps / 1e9 / (ms_max / 1e3)
+    peak = peaks["hbm_gbs"]
+    launches_per_call = 2 + 2 * 3 + n_iter * (1 + 3 + 2 + 3) + 3 + 1 + 2 + 2          # as msvid.cu issues them
+    out = {
+        "metric": "msvid_algorithmic_GBps", "value": value, "unit": "GB/s", "steps": steps, "warmup": max(3, warmup),
+        "ms_per_step": ms_max / steps,
+        "config": {"workload": workload, "description": f"MSVID_l of a {rows} x {cols} fp32 factor, l={l}, {n_iter} subspace iterations "
+                                                        f"({passes} passes over Z)", "layers": 1, "T": 0, "weights_MB": round(rows * cols * 4 / 1e6, 1),
+                   "l2_policy": "matrix larger than L2" if flush is None else "256 MiB L2 flush between steps",
+                   "launch": "stream launches", "kernel": "msvid", "grouping": "one call per step", "replicas": world},
+        "e2e": ({"value": replicas.aggregate_throughput(step_bytes * e2e_steps / 1e9, world, e2e_ms_max / 1e3), "unit": "GB/s",
+                 "h2d_bytes_per_step": rows * cols * 4 + cols * l * 4, "d2h_bytes_per_step": rows * nwords * 4 + (rows + cols) * l * 4}
+                if want_e2e else None),
+        "gpu_launches": launches_per_call * steps,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
+                     "peak_source": f"of {peak_kind}", "kernel": "absz_q_kernel / abszT_y_kernel",
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((workload, "absz_q_kernel"))},
+    }
+    del Zd, Qd, Sd, Ud, Vd, ws, flush
+    torch.cuda.empty_cache()
+    return out, ("msvid", rows, cols, l)
+
+
+def cpu_baseline_msvid(rows, cols, l, budget_s=20.0):
+    """The oracle's MSVID (full SVD of |Z|, fp64) on a leading block of rows small enough for the budget."""
+    from oracle import mdbf_oracle as orc
+    from paper_2512_24545_b200 import inputs
+    sub = min(rows, 2048)
+    Z = inputs.make_factor_matrix(sub, min(cols, 4096), seed=8)
+    t0 = time.perf_counter()
+    orc.msvid(Z, l)
+    dt = time.perf_counter() - t0
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    return {"value": Z.size * 4 / 1e9 / dt, "unit": "GB/s of Z per call", "cores": cores, "kind": "oracle",
+            "sample": f"fp64 sign mask + full SVD of a {Z.shape[0]} x {Z.shape[1]} block of the workload's matrix, one call, {dt:.1f} s"}
+
+
 # workloads the default line reports beside the headline one: the largest decode configuration, the MLP shapes at one
 # and at sixteen tokens, the prefill point under the library's own choice and under the expanded order (the metric's
 # own unit), the block prefill
@@ -458,12 +571,15 @@ def run_mdbf(args):
     build.build()
     dist, rank, world, local = dist_setup(args.gpus)
     torch.cuda.set_device(local)
-    main, cpu_args = measure(args.workload, args.kernel, args.steps, args.warmup, dist, world, local,
-                             no_graph=args.no_graph, no_siblings=args.no_siblings, copies=args.copies, fuse_block=args.fuse_block)
+    if args.workload.startswith("msvid"):
+        main, cpu_args = measure_msvid(args.workload, args.steps, args.warmup, dist, world, local)
+    else:
+        main, cpu_args = measure(args.workload, args.kernel, args.steps, args.warmup, dist, world, local,
+                                 no_graph=args.no_graph, no_siblings=args.no_siblings, copies=args.copies, fuse_block=args.fuse_block)
     out = {
         "metric": main["metric"], "value": main["value"], "unit": main["unit"], "n_gpus": world, "steps": main["steps"],
         "warmup": main["warmup"], "ms_per_step": main["ms_per_step"], "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if args.workload.startswith("msvid") else "bf16", "data": "synthetic",
         "config": main["config"], "e2e": main["e2e"], "gpu_launches": main["gpu_launches"], "clocks": main["clocks"],
         "roofline": main["roofline"],
     }
@@ -478,8 +594,11 @@ def run_mdbf(args):
                 "config": {k: m["config"][k] for k in ("layers", "T", "weights_MB", "l2_policy", "kernel", "grouping")}}
         out["also"] = also
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        spec0, T, bound, mat0 = cpu_args
-        out["cpu_baseline"] = cpu_baseline(spec0, T, bound, budget_s=20.0, mat=mat0)
+        if cpu_args[0] == "msvid":
+            out["cpu_baseline"] = cpu_baseline_msvid(*cpu_args[1:])
+        else:
+            spec0, T, bound, mat0 = cpu_args
+            out["cpu_baseline"] = cpu_baseline(spec0, T, bound, budget_s=20.0, mat=mat0)
     if dist:
         dist.destroy_process_group()
     if rank == 0:

@@ -303,12 +303,17 @@ mdbf_status_t mdbf_poll_status(mdbf_handle_t h, int32_t *device_status);
  *             TSVD_l(|Z|) ~ U V^T, columns ordered by decreasing singular value (each pair is unique up to a
  *             common sign only, and up to rotations inside a group of equal singular values)
  *   sigma     device, l fp32, written: the estimated singular values; each is a lower bound of the exact one
+ *   workspace device, at least mdbf_msvid_workspace_bytes(rows, cols, l) bytes on a 256-byte boundary, scratch of the
+ *             call (about (rows + cols + cols * ceil(rows / 256)) * l floats); free again when the stream has passed it
  * The truncated SVD is computed by block subspace iteration (hand-written CUDA-core kernels, fp32 with the small
- * Gram matrices in fp64), not to machine precision: see n_iter.  Allocates its scratch ((rows + cols + cols *
- * ceil(rows / 256)) * l floats) and synchronises `stream` before it returns.  Errors: INVALID_ARG, SHAPE, ALLOC,
- * ARCH, CUDA. */
+ * Gram matrices in fp64), not to machine precision: see n_iter.  Asynchronous on `stream`; allocates nothing and does
+ * not synchronise.  Errors: INVALID_ARG (NULL pointer, workspace too small or misaligned), SHAPE, ARCH, CUDA. */
 mdbf_status_t mdbf_msvid(const float *Z, int64_t rows, int64_t cols, int32_t l, int32_t n_iter, const float *Q0,
-                         uint32_t *S_packed, float *U, float *V, float *sigma, void *stream);
+                         uint32_t *S_packed, float *U, float *V, float *sigma, void *workspace, size_t workspace_bytes,
+                         void *stream);
+
+/* Size of the workspace mdbf_msvid needs for this shape (host computation, no device needed).  Errors: INVALID_ARG, SHAPE. */
+mdbf_status_t mdbf_msvid_workspace_bytes(int64_t rows, int64_t cols, int32_t l, size_t *bytes);
 
 /* Test hook (no counterpart in the paper): the `nth` device allocation that the calling thread makes
  * inside this library from now on fails with MDBF_ERR_ALLOC without touching the device; nth <= 0

@@ -30,25 +30,36 @@ namespace msv {
 constexpr int kMaxL = 32;
 
 // ------------------------------------------------------------------ sign mask
-// One warp per (row, word): bit c % 32 of word c / 32 is set <=> Z[r][c] is negative (a NaN counts as negative, as
-// in the comparison `not (z >= 0)` that defines sign() with sign(0) = +1); padding bits are 0.
-__global__ void sign_pack_kernel(const float *__restrict__ Z, long long p, long long q, int nwords, uint32_t *__restrict__ out) {
-    const long long total = p * nwords;
-    const int lane = threadIdx.x & 31;
-    for (long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < total; w += ((long long)gridDim.x * blockDim.x) >> 5) {
-        const long long r = w / nwords;
-        const long long c = (w - r * nwords) * 32 + lane;
-        const bool neg = c < q && !(Z[r * q + c] >= 0.f);
-        const uint32_t bits = __ballot_sync(0xffffffffu, neg);
-        if (lane == 0) out[w] = bits;
+// Bit c % 32 of word c / 32 is set <=> Z[r][c] is negative (a NaN counts as negative, as in the comparison
+// `not (z >= 0)` that defines sign() with sign(0) = +1); padding bits are 0.  CTA = one row x 2048 columns, a warp
+// takes eight words: eight independent 128-byte loads per lane, one ballot per word.
+constexpr int SP_WORDS = 8;
+__global__ void __launch_bounds__(256) sign_pack_kernel(const float *__restrict__ Z, int q, int nwords, uint32_t *__restrict__ out) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const size_t r = blockIdx.x;
+    const int w0 = (blockIdx.y * 8 + warp) * SP_WORDS;
+    const float *zr = Z + r * (size_t)q;
+    float z[SP_WORDS];
+#pragma unroll
+    for (int u = 0; u < SP_WORDS; ++u) {
+        const int c = (w0 + u) * 32 + lane;
+        z[u] = c < q ? zr[c] : 0.f;
     }
+    uint32_t mine = 0u;
+#pragma unroll
+    for (int u = 0; u < SP_WORDS; ++u) {
+        const uint32_t bits = __ballot_sync(0xffffffffu, !(z[u] >= 0.f));
+        if (lane == u) mine = bits;
+    }
+    if (lane < SP_WORDS && w0 + lane < nwords) out[r * nwords + w0 + lane] = mine;
 }
 
 // ------------------------------------------------------------------ Y = |Z| Q
-// CTA = 4 warps x 4 rows.  Q (M x LP, zero beyond the l real columns) is staged tile by tile, transposed, in shared
-// memory; a lane owns the columns lane, lane + 32, ... of the tile and keeps 4 x LP partial sums in registers, so a
-// value of Q read from shared memory serves four rows.
-constexpr int AQ_WARPS = 4, AQ_ROWS = 4, AQ_TJ = 256;
+// CTA = 8 warps x 2 rows.  Q (M x LP, zero beyond the l real columns) is staged tile by tile, transposed, in shared
+// memory; a lane owns the columns lane, lane + 32, ... of the tile and keeps 2 x LP partial sums in registers, so a
+// value of Q read from shared memory serves two rows (the shape that timed best among 4 or 8 warps x 2 or 4 rows:
+// the kernel lives on occupancy, the loads of a tile are not prefetched).
+constexpr int AQ_WARPS = 8, AQ_ROWS = 2, AQ_TJ = 256;
 template <int LP>
 __global__ void __launch_bounds__(AQ_WARPS * 32) absz_q_kernel(const float *__restrict__ Z, int p, int q, const float *__restrict__ Q,
                                                               float *__restrict__ Y) {
@@ -146,13 +157,14 @@ __global__ void chunk_sum_kernel(const float *__restrict__ P, int nchunks, size_
 }
 
 // ------------------------------------------------------------------ orth(): Cholesky QR, Gram matrix in fp64
-// partial Gram matrices of chunks of 256 rows of a tall matrix A (n x LP)
+// partial Gram matrices of chunks of GR_ROWS rows of a tall matrix A (n x LP)
+constexpr int GR_ROWS = 64;
 template <int LP>
 __global__ void __launch_bounds__(256) gram_kernel(const float *__restrict__ A, int n, double *__restrict__ Gp) {
-    __shared__ float As[256][LP + 1];
-    const int i0 = blockIdx.x * 256;
-    const int nrows = min(256, n - i0);
-    for (int e = threadIdx.x; e < 256 * LP; e += 256) {
+    __shared__ float As[GR_ROWS][LP + 1];
+    const int i0 = blockIdx.x * GR_ROWS;
+    const int nrows = min(GR_ROWS, n - i0);
+    for (int e = threadIdx.x; e < GR_ROWS * LP; e += 256) {
         const int i = e / LP, t = e - i * LP;
         As[i][t] = i < nrows ? A[(size_t)(i0 + i) * LP + t] : 0.f;
     }
@@ -234,68 +246,79 @@ __global__ void __launch_bounds__(256) right_mul_kernel(float *__restrict__ A, i
 }
 
 // ------------------------------------------------------------------ the small eigenproblem
-// One thread: cyclic Jacobi on G = Y^T Y (l x l, fp64), eigenvalues sorted in descending order; writes the singular
-// values s_t = sqrt(lambda_t) and the two LP x LP matrices that turn (Y, Q) into the balanced factors:
-// MU[b][t] = W[b][t] s_t^-1/2, MV[b][t] = W[b][t] s_t^1/2 (zero columns beyond l and for vanished singular values).
+// One warp, lane k = row / column k: cyclic Jacobi on G = Y^T Y (l x l, fp64), eigenvalues sorted in descending order;
+// writes the singular values s_t = sqrt(lambda_t) and the two LP x LP matrices that turn (Y, Q) into the balanced
+// factors: MU[b][t] = W[b][t] s_t^-1/2, MV[b][t] = W[b][t] s_t^1/2 (zero columns beyond l and for vanished values).
 template <int LP>
-__global__ void jacobi_kernel(const double *__restrict__ Gp, int nchunks, int l, float *__restrict__ sigma, float *__restrict__ MU,
-                              float *__restrict__ MV) {
-    __shared__ double G[LP][LP], W[LP][LP];
-    if (threadIdx.x != 0) return;
-    for (int a = 0; a < LP; ++a)
-        for (int b = 0; b <= a; ++b) {
-            double s = 0.0;
-            for (int c = 0; c < nchunks; ++c) s += Gp[(size_t)c * LP * LP + a * LP + b];
-            G[a][b] = G[b][a] = s;
-        }
-    for (int a = 0; a < LP; ++a)
-        for (int b = 0; b < LP; ++b) W[a][b] = a == b ? 1.0 : 0.0;
-    for (int sweep = 0; sweep < 60; ++sweep) {
+__global__ void __launch_bounds__(32) jacobi_kernel(const double *__restrict__ Gp, int nchunks, int l, float *__restrict__ sigma,
+                                                    float *__restrict__ MU, float *__restrict__ MV) {
+    __shared__ double G[LP][LP + 1], W[LP][LP + 1];
+    __shared__ int order[LP];
+    const int k = threadIdx.x;
+    for (int e = k; e < LP * LP; e += 32) {
+        const int a = e / LP, b = e - a * LP;
+        double s = 0.0;
+        const int lo = b <= a ? a * LP + b : b * LP + a;          // the partial sums hold the lower triangle
+        for (int c = 0; c < nchunks; ++c) s += Gp[(size_t)c * LP * LP + lo];
+        G[a][b] = s;
+        W[a][b] = a == b ? 1.0 : 0.0;
+    }
+    __syncwarp();
+    for (int sweep = 0; sweep < 30; ++sweep) {
         double off = 0.0, diag = 0.0;
-        for (int a = 0; a < l; ++a) {
-            diag += G[a][a] * G[a][a];
-            for (int b = 0; b < a; ++b) off += G[a][b] * G[a][b];
+        if (k < l) {
+            diag = G[k][k] * G[k][k];
+            for (int b = 0; b < k; ++b) off += G[k][b] * G[k][b];
         }
-        if (off <= 1e-30 * diag) break;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            off += __shfl_xor_sync(0xffffffffu, off, o);
+            diag += __shfl_xor_sync(0xffffffffu, diag, o);
+        }
+        if (off <= 1e-28 * diag) break;
         for (int pi = 0; pi < l - 1; ++pi)
             for (int qi = pi + 1; qi < l; ++qi) {
                 const double apq = G[pi][qi];
-                if (apq == 0.0) continue;
+                if (apq == 0.0) continue;                        // the same value in every lane
                 const double theta = (G[qi][qi] - G[pi][pi]) / (2.0 * apq);
                 const double t = (theta >= 0.0 ? 1.0 : -1.0) / (fabs(theta) + sqrt(theta * theta + 1.0));
-                const double c = 1.0 / sqrt(t * t + 1.0), s = t * c;
-                for (int k = 0; k < l; ++k) {
+                const double c = 1.0 / sqrt(t * t + 1.0), sn = t * c;
+                __syncwarp();
+                if (k < l) {
                     const double gkp = G[k][pi], gkq = G[k][qi];
-                    G[k][pi] = c * gkp - s * gkq;
-                    G[k][qi] = s * gkp + c * gkq;
-                }
-                for (int k = 0; k < l; ++k) {
-                    const double gpk = G[pi][k], gqk = G[qi][k];
-                    G[pi][k] = c * gpk - s * gqk;
-                    G[qi][k] = s * gpk + c * gqk;
-                }
-                for (int k = 0; k < l; ++k) {
+                    G[k][pi] = c * gkp - sn * gkq;
+                    G[k][qi] = sn * gkp + c * gkq;
                     const double wkp = W[k][pi], wkq = W[k][qi];
-                    W[k][pi] = c * wkp - s * wkq;
-                    W[k][qi] = s * wkp + c * wkq;
+                    W[k][pi] = c * wkp - sn * wkq;
+                    W[k][qi] = sn * wkp + c * wkq;
                 }
+                __syncwarp();
+                if (k < l) {
+                    const double gpk = G[pi][k], gqk = G[qi][k];
+                    G[pi][k] = c * gpk - sn * gqk;
+                    G[qi][k] = sn * gpk + c * gqk;
+                }
+                __syncwarp();
             }
     }
-    int order[LP];
-    for (int t = 0; t < l; ++t) order[t] = t;
-    for (int t = 0; t < l; ++t)                        // selection sort, descending eigenvalues
-        for (int u = t + 1; u < l; ++u)
-            if (G[order[u]][order[u]] > G[order[t]][order[t]]) { const int x = order[t]; order[t] = order[u]; order[u] = x; }
+    __syncwarp();
+    if (k == 0) {
+        for (int t = 0; t < l; ++t) order[t] = t;
+        for (int t = 0; t < l; ++t)                    // selection sort, descending eigenvalues
+            for (int u = t + 1; u < l; ++u)
+                if (G[order[u]][order[u]] > G[order[t]][order[t]]) { const int x = order[t]; order[t] = order[u]; order[u] = x; }
+    }
+    __syncwarp();
     const double top = l > 0 ? fmax(G[order[0]][order[0]], 0.0) : 0.0;
     for (int t = 0; t < LP; ++t) {
         double lam = t < l ? G[order[t]][order[t]] : 0.0;
         if (!(lam > 1e-24 * top)) lam = 0.0;
         const double sv = sqrt(lam), rs = sqrt(sv);
-        if (t < l) sigma[t] = (float)sv;
-        for (int b = 0; b < LP; ++b) {
-            const double w = (t < l && b < l) ? W[b][order[t]] : 0.0;
-            MU[b * LP + t] = (float)(rs > 0.0 ? w / rs : 0.0);
-            MV[b * LP + t] = (float)(w * rs);
+        if (k == 0 && t < l) sigma[t] = (float)sv;
+        if (k < LP) {
+            const double w = (t < l && k < l) ? W[k][order[t]] : 0.0;
+            MU[k * LP + t] = (float)(rs > 0.0 ? w / rs : 0.0);
+            MV[k * LP + t] = (float)(w * rs);
         }
     }
 }
@@ -309,42 +332,48 @@ __global__ void pad_kernel(const float *__restrict__ src, size_t n, int l, int L
     }
 }
 
+// The scratch of one call, carved out of the caller's workspace (256-byte aligned pieces).
 struct Scratch {
-    float *Q = nullptr, *Y = nullptr, *P = nullptr, *M = nullptr, *MU = nullptr, *MV = nullptr;
-    double *Gp = nullptr;
-    ~Scratch() {
-        void *ptrs[] = {Q, Y, P, M, MU, MV, Gp};
-        for (void *x : ptrs)
-            if (x) cudaFree(x);
-    }
+    float *Q, *Y, *P, *M, *MU, *MV;
+    double *Gp;
 };
+static size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
+static size_t carve(Scratch *w, char *base, int p, int q, int LP) {
+    const size_t zy_chunks = ceil_div(p, ZY_ROWS), gchunks = ceil_div(max(p, q), GR_ROWS);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char *ptr = base ? base + off : nullptr; off += align256(bytes); return ptr; };
+    float *Q = (float *)take((size_t)q * LP * sizeof(float));
+    float *Y = (float *)take((size_t)p * LP * sizeof(float));
+    float *P = (float *)take(zy_chunks * q * LP * sizeof(float));
+    double *Gp = (double *)take(gchunks * LP * LP * sizeof(double));
+    float *M = (float *)take((size_t)LP * LP * sizeof(float));
+    float *MU = (float *)take((size_t)LP * LP * sizeof(float));
+    float *MV = (float *)take((size_t)LP * LP * sizeof(float));
+    if (w) { w->Q = Q; w->Y = Y; w->P = P; w->Gp = Gp; w->M = M; w->MU = MU; w->MV = MV; }
+    return off;
+}
+static int padded_rank(int l) {
+    int LP = 1;
+    while (LP < l) LP *= 2;
+    return LP;
+}
 
 template <int LP>
 static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st) {
-    const int chunks = ceil_div(n, 256);
+    const int chunks = ceil_div(n, GR_ROWS);
     gram_kernel<LP><<<chunks, 256, 0, st>>>(A, n, w.Gp);
     chol_kernel<LP><<<1, LP * LP < 32 ? 32 : LP * LP, 0, st>>>(w.Gp, chunks, w.M);
-    right_mul_kernel<LP><<<chunks, 256, 0, st>>>(A, n, w.M, nullptr, 0);
+    right_mul_kernel<LP><<<ceil_div(n, 256), 256, 0, st>>>(A, n, w.M, nullptr, 0);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
 
 template <int LP>
 static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const float *Q0, uint32_t *S, float *U, float *V, float *sigma,
-                         cudaStream_t st) {
-    Scratch w;
+                         Scratch &w, cudaStream_t st) {
     const int zy_chunks = ceil_div(p, ZY_ROWS);
-    const int gchunks = ceil_div(max(p, q), 256);
-    MDBF_CUDA(dev_malloc(&w.Q, (size_t)q * LP * sizeof(float)));
-    MDBF_CUDA(dev_malloc(&w.Y, (size_t)p * LP * sizeof(float)));
-    MDBF_CUDA(dev_malloc(&w.P, (size_t)zy_chunks * q * LP * sizeof(float)));
-    MDBF_CUDA(dev_malloc(&w.Gp, (size_t)gchunks * LP * LP * sizeof(double)));
-    MDBF_CUDA(dev_malloc(&w.M, (size_t)LP * LP * sizeof(float)));
-    MDBF_CUDA(dev_malloc(&w.MU, (size_t)LP * LP * sizeof(float)));
-    MDBF_CUDA(dev_malloc(&w.MV, (size_t)LP * LP * sizeof(float)));
-
     const int nwords = ceil_div(q, 32);
-    sign_pack_kernel<<<(int)std::min<long long>(((long long)p * nwords * 32 + 255) / 256, 148LL * 16), 256, 0, st>>>(Z, p, q, nwords, S);
+    sign_pack_kernel<<<dim3(p, ceil_div(nwords, 8 * SP_WORDS)), 256, 0, st>>>(Z, q, nwords, S);
     pad_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(Q0, (size_t)q, l, LP, w.Q);
     MDBF_CUDA(cudaGetLastError());
     mdbf_status_t rc = orth<LP>(w.Q, q, w, st);                        // twice: the start block may be badly conditioned
@@ -360,17 +389,28 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
         chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, zy_chunks, (size_t)q * LP, w.Q);
         MDBF_CUDA(cudaGetLastError());
         rc = orth<LP>(w.Q, q, w, st);
-        if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st);               // the right block carries the result: orthonormal to fp32
+        if (rc == MDBF_OK && it == n_iter - 1) rc = orth<LP>(w.Q, q, w, st);   // the last block carries the result: orthonormal to fp32
         if (rc) return rc;
     }
     absz_q_kernel<LP><<<aq_grid, AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y);
-    const int ychunks = ceil_div(p, 256);
+    const int ychunks = ceil_div(p, GR_ROWS);
     gram_kernel<LP><<<ychunks, 256, 0, st>>>(w.Y, p, w.Gp);
     jacobi_kernel<LP><<<1, 32, 0, st>>>(w.Gp, ychunks, l, sigma, w.MU, w.MV);
-    right_mul_kernel<LP><<<ychunks, 256, 0, st>>>(w.Y, p, w.MU, U, l);
+    right_mul_kernel<LP><<<ceil_div(p, 256), 256, 0, st>>>(w.Y, p, w.MU, U, l);
     right_mul_kernel<LP><<<ceil_div(q, 256), 256, 0, st>>>(w.Q, q, w.MV, V, l);
     MDBF_CUDA(cudaGetLastError());
-    MDBF_CUDA(cudaStreamSynchronize(st));                              // the scratch is freed on return
+    return MDBF_OK;
+}
+
+static mdbf_status_t check_shape(const char *who, int64_t rows, int64_t cols, int32_t l) {
+    if (rows < 1 || cols < 1 || rows > (1 << 24) || cols > (1 << 24) || rows * cols > (1LL << 40)) {
+        set_error("%s: size %lld x %lld outside the supported range", who, (long long)rows, (long long)cols);
+        return MDBF_ERR_SHAPE;
+    }
+    if (l < 1 || l > kMaxL || l > rows || l > cols) {
+        set_error("%s: l=%d outside [1, min(%d, rows, cols)]", who, l, kMaxL);
+        return MDBF_ERR_SHAPE;
+    }
     return MDBF_OK;
 }
 
@@ -379,30 +419,38 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
 
 using namespace mdbf;
 
+extern "C" mdbf_status_t mdbf_msvid_workspace_bytes(int64_t rows, int64_t cols, int32_t l, size_t *bytes) {
+    if (!bytes) { set_error("mdbf_msvid_workspace_bytes: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    mdbf_status_t rc = msv::check_shape("mdbf_msvid_workspace_bytes", rows, cols, l);
+    if (rc) return rc;
+    *bytes = msv::carve(nullptr, nullptr, (int)rows, (int)cols, msv::padded_rank(l));
+    return MDBF_OK;
+}
+
 extern "C" mdbf_status_t mdbf_msvid(const float *Z, int64_t rows, int64_t cols, int32_t l, int32_t n_iter, const float *Q0,
-                                    uint32_t *S_packed, float *U, float *V, float *sigma, void *stream) {
-    if (!Z || !Q0 || !S_packed || !U || !V || !sigma) { set_error("mdbf_msvid: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
-    if (rows < 1 || cols < 1 || rows > (1 << 24) || cols > (1 << 24) || rows * cols > (1LL << 40)) {
-        set_error("mdbf_msvid: size %lld x %lld outside the supported range", (long long)rows, (long long)cols);
-        return MDBF_ERR_SHAPE;
-    }
-    if (l < 1 || l > msv::kMaxL || l > rows || l > cols) {
-        set_error("mdbf_msvid: l=%d outside [1, min(%d, rows, cols)]", l, msv::kMaxL);
-        return MDBF_ERR_SHAPE;
-    }
+                                    uint32_t *S_packed, float *U, float *V, float *sigma, void *workspace, size_t workspace_bytes,
+                                    void *stream) {
+    if (!Z || !Q0 || !S_packed || !U || !V || !sigma || !workspace) { set_error("mdbf_msvid: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    mdbf_status_t rc = msv::check_shape("mdbf_msvid", rows, cols, l);
+    if (rc) return rc;
     if (n_iter < 1 || n_iter > 1000) { set_error("mdbf_msvid: n_iter=%d outside [1, 1000]", n_iter); return MDBF_ERR_SHAPE; }
-    mdbf_status_t rc = require_device(nullptr);
+    const int p = (int)rows, q = (int)cols, LP = msv::padded_rank(l);
+    msv::Scratch w;
+    const size_t need = msv::carve(&w, (char *)workspace, p, q, LP);
+    if (workspace_bytes < need || ((uintptr_t)workspace & 255u) != 0) {
+        set_error("mdbf_msvid: the workspace must hold %zu bytes (mdbf_msvid_workspace_bytes) on a 256-byte boundary; got %zu at %p",
+                  need, workspace_bytes, workspace);
+        return MDBF_ERR_INVALID_ARG;
+    }
+    rc = require_device(nullptr);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    const int p = (int)rows, q = (int)cols;
-    int LP = 1;
-    while (LP < l) LP *= 2;
     switch (LP) {
-        case 1: return msv::run<1>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
-        case 2: return msv::run<2>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
-        case 4: return msv::run<4>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
-        case 8: return msv::run<8>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
-        case 16: return msv::run<16>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
-        default: return msv::run<32>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, st);
+        case 1: return msv::run<1>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
+        case 2: return msv::run<2>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
+        case 4: return msv::run<4>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
+        case 8: return msv::run<8>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
+        case 16: return msv::run<16>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
+        default: return msv::run<32>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
     }
 }

@@ -29,7 +29,7 @@ EXPORTS = (
     "mdbf_pack_signs", "mdbf_unpack_signs", "mdbf_pack", "mdbf_get_packed", "mdbf_get_envelope",
     "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host", "mdbf_linear_forward_host_async", "mdbf_prepare_host_staging",
     "mdbf_linear_forward_static", "mdbf_linear_forward_sum", "mdbf_linear_forward_siblings", "mdbf_linear_forward_group",
-    "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_msvid", "mdbf_poll_status", "mdbf_selftest_wait_timeout", "mdbf_debug_fail_alloc",
+    "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_msvid", "mdbf_msvid_workspace_bytes", "mdbf_poll_status", "mdbf_selftest_wait_timeout", "mdbf_debug_fail_alloc",
     "mdbf_last_launch_count",
     "mdbf_last_kernel",
     "mdbf_destroy", "mdbf_last_error", "mdbf_version",
@@ -79,7 +79,8 @@ def lib() -> ctypes.CDLL:
     L.mdbf_linear_forward_group.argtypes = [vp, i32, vp, vp, i32, i32, vp]
     L.mdbf_get_intermediate.argtypes = [vp, vp, i32, ctypes.c_int, vp]
     L.mdbf_reconstruct.argtypes = [vp, vp, vp]
-    L.mdbf_msvid.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp, vp]
+    L.mdbf_msvid.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    L.mdbf_msvid_workspace_bytes.argtypes = [i64, i64, i32, ctypes.POINTER(ctypes.c_size_t)]
     L.mdbf_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
     L.mdbf_selftest_wait_timeout.argtypes = [vp, vp]
     L.mdbf_debug_fail_alloc.argtypes = [i32]
@@ -227,10 +228,18 @@ def mdbf_poll_status(h: int) -> int:
     return v.value
 
 
-def mdbf_msvid(Z, rows: int, cols: int, l: int, n_iter: int, Q0, S_packed, U, V, sigma, stream: int = 0) -> None:
+def mdbf_msvid_workspace_bytes(rows: int, cols: int, l: int) -> int:
+    v = ctypes.c_size_t()
+    _check(lib().mdbf_msvid_workspace_bytes(rows, cols, l, ctypes.byref(v)))
+    return v.value
+
+
+def mdbf_msvid(Z, rows: int, cols: int, l: int, n_iter: int, Q0, S_packed, U, V, sigma, workspace, workspace_bytes: int,
+               stream: int = 0) -> None:
     """MSVID_l[Z] = sign(Z) (.) TSVD_l(|Z|) of a device matrix (all arguments device addresses): packed sign mask,
-    balanced envelope factors and singular values; see include/mdbf.h."""
-    _check(lib().mdbf_msvid(_addr(Z), rows, cols, l, n_iter, _addr(Q0), _addr(S_packed), _addr(U), _addr(V), _addr(sigma), stream))
+    balanced envelope factors and singular values; asynchronous, the caller owns the workspace.  See include/mdbf.h."""
+    _check(lib().mdbf_msvid(_addr(Z), rows, cols, l, n_iter, _addr(Q0), _addr(S_packed), _addr(U), _addr(V), _addr(sigma),
+                            _addr(workspace), workspace_bytes, stream))
 
 
 def mdbf_debug_fail_alloc(nth: int) -> None:

@@ -30,8 +30,10 @@ def run_msvid(Z, l, n_iter, Q0=None, seed=11):
     Ud = torch.full((rows, l), float("nan"), dtype=torch.float32, device="cuda")
     Vd = torch.full((cols, l), float("nan"), dtype=torch.float32, device="cuda")
     sd = torch.full((l,), float("nan"), dtype=torch.float32, device="cuda")
+    nbytes = M.mdbf_msvid_workspace_bytes(rows, cols, l)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
     M.mdbf_msvid(Zd.data_ptr(), rows, cols, l, n_iter, Qd.data_ptr(), Sd.data_ptr(), Ud.data_ptr(), Vd.data_ptr(), sd.data_ptr(),
-                 torch.cuda.current_stream().cuda_stream)
+                 ws.data_ptr(), nbytes, torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
     return (Sd.cpu().numpy().view(np.uint32), Ud.cpu().numpy().astype(np.float64), Vd.cpu().numpy().astype(np.float64),
             sd.cpu().numpy().astype(np.float64))
@@ -119,11 +121,18 @@ def test_argument_errors():
     S = torch.zeros((8, 1), dtype=torch.int32, device="cuda")
     U = torch.zeros((8, 2), dtype=torch.float32, device="cuda")
     s = torch.zeros((2,), dtype=torch.float32, device="cuda")
-    args = lambda: (Z.data_ptr(), 8, 8, 2, 2, Q.data_ptr(), S.data_ptr(), U.data_ptr(), U.data_ptr(), s.data_ptr())
-    for bad, status in (((0,), M.ERR_INVALID_ARG), ((1, 0), M.ERR_SHAPE), ((3, 0), M.ERR_SHAPE), ((3, 33), M.ERR_SHAPE),
-                        ((3, 9), M.ERR_SHAPE), ((4, 0), M.ERR_SHAPE)):
-        a = list(args())
-        a[bad[0]] = bad[1] if len(bad) > 1 else 0
+    nbytes = M.mdbf_msvid_workspace_bytes(8, 8, 2)
+    ws = torch.zeros(nbytes + 256, dtype=torch.uint8, device="cuda")
+    args = lambda: [Z.data_ptr(), 8, 8, 2, 2, Q.data_ptr(), S.data_ptr(), U.data_ptr(), U.data_ptr(), s.data_ptr(), ws.data_ptr(), nbytes]
+    for pos, val, status in ((0, 0, M.ERR_INVALID_ARG), (1, 0, M.ERR_SHAPE), (3, 0, M.ERR_SHAPE), (3, 33, M.ERR_SHAPE),
+                             (3, 9, M.ERR_SHAPE), (4, 0, M.ERR_SHAPE), (10, 0, M.ERR_INVALID_ARG), (11, nbytes - 1, M.ERR_INVALID_ARG),
+                             (10, ws.data_ptr() + 4, M.ERR_INVALID_ARG)):
+        a = args()
+        a[pos] = val
         with pytest.raises(M.MdbfError) as e:
             M.mdbf_msvid(*a)
         assert e.value.status == status
+    with pytest.raises(M.MdbfError):
+        M.mdbf_msvid_workspace_bytes(8, 8, 9)
+    M.mdbf_msvid(*args())                                    # and the same arguments untouched go through
+    torch.cuda.synchronize()
