@@ -522,7 +522,7 @@ def measure_msvid(workload, steps, warmup, dist, world, local, want_e2e=True, mi
     value = replicas.aggregate_throughput(step_bytes * steps / 1e9, world, ms_max / 1e3)
     per_gpu = step_bytes * steps / 1e9 / (ms_max / 1e3)
     peak = peaks["hbm_gbs"]
-    launches_per_call = 2 + 2 * 3 + n_iter * (1 + 3 + 2 + 3) + 3 + 1 + 2 + 2          # as msvid.cu issues them
+    launches_per_call = 2 + 2 * 4 + n_iter * (1 + 4 + 2 + 4) + 4 + 1 + 3 + 2          # as msvid.cu issues them
     out = {
         "metric": "msvid_algorithmic_GBps", "value": value, "unit": "GB/s", "steps": steps, "warmup": max(3, warmup),
         "ms_per_step": ms_max / steps,
@@ -560,9 +560,9 @@ def cpu_baseline_msvid(rows, cols, l, budget_s=20.0):
 
 # workloads the default line reports beside the headline one: the largest decode configuration, the MLP shapes at one
 # and at sixteen tokens, the prefill point under the library's own choice and under the expanded order (the metric's
-# own unit), the block prefill
+# own unit), the block prefill, and the quantizer's first step on a factor of the block's largest layer
 ALSO = [("block70b_T1", "auto"), ("block70b_T1", "fused"), ("decode_mlp_T1", "auto"), ("decode_mlp_T16", "auto"), ("prefill_4096_l16_bpw10", "auto"),
-        ("prefill_4096_l16_bpw10", "prefill"), ("block70b_T2048", "auto")]
+        ("prefill_4096_l16_bpw10", "prefill"), ("block70b_T2048", "auto"), ("msvid_28672x6016_l16", "auto")]
 
 
 def run_mdbf(args):
@@ -586,8 +586,11 @@ def run_mdbf(args):
     if world == 1 and args.also and args.workload == "decode_qproj" and args.kernel == "auto":
         also = {}
         for (wl, kern) in ALSO:
-            m, _ = measure(wl, "auto" if kern == "fused" else kern, max(3, min(args.steps, 10)), args.warmup, None, 1, local,
-                           want_e2e=False, fuse_block=kern == "fused", min_timed_ms=60.0)
+            if wl.startswith("msvid"):
+                m, _ = measure_msvid(wl, max(3, min(args.steps, 10)), args.warmup, None, 1, local, want_e2e=False, min_timed_ms=60.0)
+            else:
+                m, _ = measure(wl, "auto" if kern == "fused" else kern, max(3, min(args.steps, 10)), args.warmup, None, 1, local,
+                               want_e2e=False, fuse_block=kern == "fused", min_timed_ms=60.0)
             also[wl if kern == "auto" else f"{wl}:{kern}"] = {
                 "metric": m["metric"], "value": m["value"], "unit": m["unit"], "ms_per_step": m["ms_per_step"],
                 "steps": m["steps"], "gpu_launches": m["gpu_launches"], "clocks": m["clocks"], "roofline": m["roofline"],

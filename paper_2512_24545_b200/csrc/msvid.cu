@@ -177,6 +177,17 @@ __global__ void __launch_bounds__(256) gram_kernel(const float *__restrict__ A, 
         Gp[(size_t)blockIdx.x * LP * LP + pr] = s;
     }
 }
+// The chunks' partial Gram matrices added up: one warp per entry, lanes stride over the chunks, then a fixed
+// shuffle tree (the order of the additions does not depend on scheduling).
+__global__ void __launch_bounds__(256) gram_sum_kernel(const double *__restrict__ Gp, int nchunks, int nentries, double *__restrict__ G) {
+    const int e = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (e >= nentries) return;
+    double s = 0.0;
+    for (int c = lane; c < nchunks; c += 32) s += Gp[(size_t)c * nentries + e];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) G[e] = s;
+}
 // One CTA: G = sum of the partial Gram matrices = L L^T; M[b][a] = (L^-1)[a][b], so that A M has orthonormal columns.
 // A zero (or numerically vanished) pivot - a padding column, or a block wider than the rank of the matrix - leaves
 // its column as it is instead of dividing by zero.
@@ -187,6 +198,7 @@ __global__ void __launch_bounds__(LP * LP < 32 ? 32 : LP * LP) chol_kernel(const
     const int a = tid / LP, b = tid - a * LP;
     if (tid < LP * LP) {
         double s = 0.0;
+#pragma unroll 8
         for (int c = 0; c < nchunks; ++c) s += Gp[(size_t)c * LP * LP + tid];
         G[a][b] = s;                                   // lower triangle (b <= a) holds the sums
         Li[a][b] = 0.0;
@@ -259,6 +271,7 @@ __global__ void __launch_bounds__(32) jacobi_kernel(const double *__restrict__ G
         const int a = e / LP, b = e - a * LP;
         double s = 0.0;
         const int lo = b <= a ? a * LP + b : b * LP + a;          // the partial sums hold the lower triangle
+#pragma unroll 8
         for (int c = 0; c < nchunks; ++c) s += Gp[(size_t)c * LP * LP + lo];
         G[a][b] = s;
         W[a][b] = a == b ? 1.0 : 0.0;
@@ -275,7 +288,7 @@ __global__ void __launch_bounds__(32) jacobi_kernel(const double *__restrict__ G
             off += __shfl_xor_sync(0xffffffffu, off, o);
             diag += __shfl_xor_sync(0xffffffffu, diag, o);
         }
-        if (off <= 1e-28 * diag) break;
+        if (off <= 1e-24 * diag) break;                          // off-diagonal mass below 1e-12 of the diagonal's
         for (int pi = 0; pi < l - 1; ++pi)
             for (int qi = pi + 1; qi < l; ++qi) {
                 const double apq = G[pi][qi];
@@ -335,7 +348,7 @@ __global__ void pad_kernel(const float *__restrict__ src, size_t n, int l, int L
 // The scratch of one call, carved out of the caller's workspace (256-byte aligned pieces).
 struct Scratch {
     float *Q, *Y, *P, *M, *MU, *MV;
-    double *Gp;
+    double *Gp, *Gs;
 };
 static size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 static size_t carve(Scratch *w, char *base, int p, int q, int LP) {
@@ -346,10 +359,11 @@ static size_t carve(Scratch *w, char *base, int p, int q, int LP) {
     float *Y = (float *)take((size_t)p * LP * sizeof(float));
     float *P = (float *)take(zy_chunks * q * LP * sizeof(float));
     double *Gp = (double *)take(gchunks * LP * LP * sizeof(double));
+    double *Gs = (double *)take((size_t)LP * LP * sizeof(double));
     float *M = (float *)take((size_t)LP * LP * sizeof(float));
     float *MU = (float *)take((size_t)LP * LP * sizeof(float));
     float *MV = (float *)take((size_t)LP * LP * sizeof(float));
-    if (w) { w->Q = Q; w->Y = Y; w->P = P; w->Gp = Gp; w->M = M; w->MU = MU; w->MV = MV; }
+    if (w) { w->Q = Q; w->Y = Y; w->P = P; w->Gp = Gp; w->Gs = Gs; w->M = M; w->MU = MU; w->MV = MV; }
     return off;
 }
 static int padded_rank(int l) {
@@ -362,7 +376,8 @@ template <int LP>
 static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st) {
     const int chunks = ceil_div(n, GR_ROWS);
     gram_kernel<LP><<<chunks, 256, 0, st>>>(A, n, w.Gp);
-    chol_kernel<LP><<<1, LP * LP < 32 ? 32 : LP * LP, 0, st>>>(w.Gp, chunks, w.M);
+    gram_sum_kernel<<<ceil_div(LP * LP, 8), 256, 0, st>>>(w.Gp, chunks, LP * LP, w.Gs);
+    chol_kernel<LP><<<1, LP * LP < 32 ? 32 : LP * LP, 0, st>>>(w.Gs, 1, w.M);
     right_mul_kernel<LP><<<ceil_div(n, 256), 256, 0, st>>>(A, n, w.M, nullptr, 0);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
@@ -395,7 +410,8 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
     absz_q_kernel<LP><<<aq_grid, AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y);
     const int ychunks = ceil_div(p, GR_ROWS);
     gram_kernel<LP><<<ychunks, 256, 0, st>>>(w.Y, p, w.Gp);
-    jacobi_kernel<LP><<<1, 32, 0, st>>>(w.Gp, ychunks, l, sigma, w.MU, w.MV);
+    gram_sum_kernel<<<ceil_div(LP * LP, 8), 256, 0, st>>>(w.Gp, ychunks, LP * LP, w.Gs);
+    jacobi_kernel<LP><<<1, 32, 0, st>>>(w.Gs, 1, l, sigma, w.MU, w.MV);
     right_mul_kernel<LP><<<ceil_div(p, 256), 256, 0, st>>>(w.Y, p, w.MU, U, l);
     right_mul_kernel<LP><<<ceil_div(q, 256), 256, 0, st>>>(w.Q, q, w.MV, V, l);
     MDBF_CUDA(cudaGetLastError());
