@@ -258,14 +258,14 @@ __global__ void __launch_bounds__(256) right_mul_kernel(float *__restrict__ A, i
 }
 
 // ------------------------------------------------------------------ the small eigenproblem
-// One warp, lane k = row / column k: cyclic Jacobi on G = Y^T Y (l x l, fp64), eigenvalues sorted in descending order;
+// One warp, lane k = row / column k: Jacobi on G = Y^T Y (l x l, fp64), eigenvalues sorted in descending order;
 // writes the singular values s_t = sqrt(lambda_t) and the two LP x LP matrices that turn (Y, Q) into the balanced
 // factors: MU[b][t] = W[b][t] s_t^-1/2, MV[b][t] = W[b][t] s_t^1/2 (zero columns beyond l and for vanished values).
 template <int LP>
 __global__ void __launch_bounds__(32) jacobi_kernel(const double *__restrict__ Gp, int nchunks, int l, float *__restrict__ sigma,
                                                     float *__restrict__ MU, float *__restrict__ MV) {
-    __shared__ double G[LP][LP + 1], W[LP][LP + 1];
-    __shared__ int order[LP];
+    __shared__ double G[LP][LP + 1], W[LP][LP + 1], rc[LP], rs[LP];
+    __shared__ int order[LP], rp[LP], rq[LP];
     const int k = threadIdx.x;
     for (int e = k; e < LP * LP; e += 32) {
         const int a = e / LP, b = e - a * LP;
@@ -277,7 +277,11 @@ __global__ void __launch_bounds__(32) jacobi_kernel(const double *__restrict__ G
         W[a][b] = a == b ? 1.0 : 0.0;
     }
     __syncwarp();
-    for (int sweep = 0; sweep < 30; ++sweep) {
+    // Round-robin ordering: n - 1 rounds of n / 2 rotations on disjoint index pairs (n = l rounded up to even; a pair
+    // with the dummy index is skipped).  Lane i works out the rotation of pair i; then every lane applies all of the
+    // round's rotations to its row (columns p, q of G and of W), then to its column (rows p, q of G).
+    const int n = (l + 1) & ~1;
+    for (int sweep = 0; sweep < 30 && n >= 2; ++sweep) {
         double off = 0.0, diag = 0.0;
         if (k < l) {
             diag = G[k][k] * G[k][k];
@@ -289,15 +293,28 @@ __global__ void __launch_bounds__(32) jacobi_kernel(const double *__restrict__ G
             diag += __shfl_xor_sync(0xffffffffu, diag, o);
         }
         if (off <= 1e-24 * diag) break;                          // off-diagonal mass below 1e-12 of the diagonal's
-        for (int pi = 0; pi < l - 1; ++pi)
-            for (int qi = pi + 1; qi < l; ++qi) {
-                const double apq = G[pi][qi];
-                if (apq == 0.0) continue;                        // the same value in every lane
-                const double theta = (G[qi][qi] - G[pi][pi]) / (2.0 * apq);
-                const double t = (theta >= 0.0 ? 1.0 : -1.0) / (fabs(theta) + sqrt(theta * theta + 1.0));
-                const double c = 1.0 / sqrt(t * t + 1.0), sn = t * c;
-                __syncwarp();
-                if (k < l) {
+        for (int r = 0; r < n - 1; ++r) {
+            if (k < n / 2) {
+                const int a = k == 0 ? n - 1 : (r + k) % (n - 1), b = k == 0 ? r : (r - k + (n - 1)) % (n - 1);
+                const int pi = min(a, b), qi = max(a, b);
+                double c = 1.0, sn = 0.0;
+                if (qi < l) {
+                    const double apq = G[pi][qi];
+                    if (apq != 0.0) {
+                        const double theta = (G[qi][qi] - G[pi][pi]) / (2.0 * apq);
+                        const double t = (theta >= 0.0 ? 1.0 : -1.0) / (fabs(theta) + sqrt(theta * theta + 1.0));
+                        c = 1.0 / sqrt(t * t + 1.0);
+                        sn = t * c;
+                    }
+                }
+                rp[k] = pi; rq[k] = qi; rc[k] = c; rs[k] = sn;
+            }
+            __syncwarp();
+            if (k < l)
+                for (int i = 0; i < n / 2; ++i) {
+                    const double c = rc[i], sn = rs[i];
+                    if (sn == 0.0) continue;
+                    const int pi = rp[i], qi = rq[i];
                     const double gkp = G[k][pi], gkq = G[k][qi];
                     G[k][pi] = c * gkp - sn * gkq;
                     G[k][qi] = sn * gkp + c * gkq;
@@ -305,14 +322,18 @@ __global__ void __launch_bounds__(32) jacobi_kernel(const double *__restrict__ G
                     W[k][pi] = c * wkp - sn * wkq;
                     W[k][qi] = sn * wkp + c * wkq;
                 }
-                __syncwarp();
-                if (k < l) {
+            __syncwarp();
+            if (k < l)
+                for (int i = 0; i < n / 2; ++i) {
+                    const double c = rc[i], sn = rs[i];
+                    if (sn == 0.0) continue;
+                    const int pi = rp[i], qi = rq[i];
                     const double gpk = G[pi][k], gqk = G[qi][k];
                     G[pi][k] = c * gpk - sn * gqk;
                     G[qi][k] = sn * gpk + c * gqk;
                 }
-                __syncwarp();
-            }
+            __syncwarp();
+        }
     }
     __syncwarp();
     if (k == 0) {
