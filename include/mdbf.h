@@ -294,7 +294,7 @@ mdbf_status_t mdbf_poll_status(mdbf_handle_t h, int32_t *device_status);
  *   Z         device, rows x cols fp32, row-major, read only
  *   l         envelope rank, 1 <= l <= min(32, rows, cols)
  *   n_iter    subspace iterations (two passes over Z each), >= 1; 2 already fixes the leading singular value,
- *             8 leaves the squared error within about half a per cent of the optimum on Gaussian-like inputs
+ *             8 leaves the squared error within a fraction of a per cent to about one per cent of the optimum
  *   Q0        device, cols x l fp32: the start block of the iteration (e.g. i.i.d. Gaussian; the caller draws it,
  *             so that a run is reproducible from its inputs alone); needs full column rank
  *   S_packed  device, rows x ceil(cols / 32) uint32, written: the sign mask in the canonical packing of
