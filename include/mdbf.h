@@ -312,6 +312,16 @@ mdbf_status_t mdbf_msvid(const float *Z, int64_t rows, int64_t cols, int32_t l, 
                          uint32_t *S_packed, float *U, float *V, float *sigma, void *workspace, size_t workspace_bytes,
                          void *stream);
 
+/* Projection onto the matrices that share a GIVEN sign mask and have an envelope of rank <= l (Theorem 1, Eq. Ustar):
+ *   Pi(Z) = S (.) TSVD_l(S (.) Z),   error (sum_{i > l} sigma_i(S (.) Z)^2)^(1/2)   (Eq. rankl-error)
+ * - the step the paper's refinement repeats with the mask held fixed; mdbf_msvid is the special case S = sign(Z).
+ * Arguments as for mdbf_msvid, except that S_packed (rows x ceil(cols / 32) words, canonical packing, bit set <=> -1) is
+ * read, not written.  U V^T approximates the demodulated envelope S (.) Z, so the projection itself is S (.) (U V^T).
+ * The same workspace size serves.  Asynchronous on `stream`, allocates nothing.  Errors as for mdbf_msvid. */
+mdbf_status_t mdbf_project_fixed_mask(const float *Z, const uint32_t *S_packed, int64_t rows, int64_t cols, int32_t l,
+                                      int32_t n_iter, const float *Q0, float *U, float *V, float *sigma, void *workspace,
+                                      size_t workspace_bytes, void *stream);
+
 /* Size of the workspace mdbf_msvid needs for this shape (host computation, no device needed).  Errors: INVALID_ARG, SHAPE. */
 mdbf_status_t mdbf_msvid_workspace_bytes(int64_t rows, int64_t cols, int32_t l, size_t *bytes);
 

@@ -60,9 +60,10 @@ __global__ void __launch_bounds__(256) sign_pack_kernel(const float *__restrict_
 // value of Q read from shared memory serves two rows (the shape that timed best among 4 or 8 warps x 2 or 4 rows:
 // the kernel lives on occupancy, the loads of a tile are not prefetched).
 constexpr int AQ_WARPS = 8, AQ_ROWS = 2, AQ_TJ = 256;
-template <int LP>
+// MASKED: the envelope is S (.) Z for a given packed mask S (bit set <=> -1) instead of |Z| = sign(Z) (.) Z.
+template <int LP, bool MASKED>
 __global__ void __launch_bounds__(AQ_WARPS * 32) absz_q_kernel(const float *__restrict__ Z, int p, int q, const float *__restrict__ Q,
-                                                              float *__restrict__ Y) {
+                                                              float *__restrict__ Y, const uint32_t *__restrict__ S, int nwords) {
     __shared__ float Qs[LP][AQ_TJ + 1];                // + 1: the transposing store hits LP different banks
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r0 = (blockIdx.x * AQ_WARPS + warp) * AQ_ROWS;
@@ -84,7 +85,14 @@ __global__ void __launch_bounds__(AQ_WARPS * 32) absz_q_kernel(const float *__re
 #pragma unroll
             for (int s = 0; s < AQ_TJ / 32; ++s) {
                 const int j = j0 + s * 32 + lane;
-                z[r][s] = (r0 + r < p && j < q) ? fabsf(Z[(size_t)(r0 + r) * q + j]) : 0.f;
+                float v = (r0 + r < p && j < q) ? Z[(size_t)(r0 + r) * q + j] : 0.f;
+                if (MASKED) {
+                    const uint32_t w = (r0 + r < p && j0 + s * 32 < q) ? S[(size_t)(r0 + r) * nwords + ((j0 >> 5) + s)] : 0u;   // one word per warp
+                    v = __uint_as_float(__float_as_uint(v) ^ (((w >> lane) & 1u) << 31));
+                } else {
+                    v = fabsf(v);
+                }
+                z[r][s] = v;
             }
 #pragma unroll
         for (int s = 0; s < AQ_TJ / 32; ++s)
@@ -111,9 +119,9 @@ __global__ void __launch_bounds__(AQ_WARPS * 32) absz_q_kernel(const float *__re
 // by all threads at once (broadcast).  Partial sums per chunk go to P[chunk][column][LP]; a second kernel adds the
 // chunks in order (no atomics: the result does not depend on scheduling).
 constexpr int ZY_COLS = 256, ZY_ROWS = 256;
-template <int LP>
+template <int LP, bool MASKED>
 __global__ void __launch_bounds__(ZY_COLS) abszT_y_kernel(const float *__restrict__ Z, int p, int q, const float *__restrict__ Y,
-                                                           float *__restrict__ P) {
+                                                           float *__restrict__ P, const uint32_t *__restrict__ S, int nwords) {
     __shared__ float Ys[ZY_ROWS][LP];
     const int j = blockIdx.x * ZY_COLS + threadIdx.x;
     const int i0 = blockIdx.y * ZY_ROWS;
@@ -128,18 +136,23 @@ __global__ void __launch_bounds__(ZY_COLS) abszT_y_kernel(const float *__restric
     for (int t = 0; t < LP; ++t) acc[t] = 0.f;
     if (j < q) {
         const float *zp = Z + (size_t)i0 * q + j;
+        const uint32_t *sp = MASKED ? S + (size_t)i0 * nwords + (j >> 5) : nullptr;      // the lanes of a warp share each word
+        auto envelope = [&](int i) {
+            const float v = zp[(size_t)i * q];
+            return MASKED ? __uint_as_float(__float_as_uint(v) ^ (((sp[(size_t)i * nwords] >> (j & 31)) & 1u) << 31)) : fabsf(v);
+        };
         int i = 0;
         for (; i + 8 <= nrows; i += 8) {
             float z[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) z[u] = fabsf(zp[(size_t)(i + u) * q]);
+            for (int u = 0; u < 8; ++u) z[u] = envelope(i + u);
 #pragma unroll
             for (int u = 0; u < 8; ++u)
 #pragma unroll
                 for (int t = 0; t < LP; ++t) acc[t] = fmaf(z[u], Ys[i + u][t], acc[t]);
         }
         for (; i < nrows; ++i) {
-            const float z = fabsf(zp[(size_t)i * q]);
+            const float z = envelope(i);
 #pragma unroll
             for (int t = 0; t < LP; ++t) acc[t] = fmaf(z, Ys[i][t], acc[t]);
         }
@@ -404,12 +417,13 @@ static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st) {
     return MDBF_OK;
 }
 
-template <int LP>
+// MASKED = false: S is written (the mask of Z itself, Eq. msvid-def); MASKED = true: S is given (Eq. Ustar)
+template <int LP, bool MASKED>
 static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const float *Q0, uint32_t *S, float *U, float *V, float *sigma,
                          Scratch &w, cudaStream_t st) {
     const int zy_chunks = ceil_div(p, ZY_ROWS);
     const int nwords = ceil_div(q, 32);
-    sign_pack_kernel<<<dim3(p, ceil_div(nwords, 8 * SP_WORDS)), 256, 0, st>>>(Z, q, nwords, S);
+    if (!MASKED) sign_pack_kernel<<<dim3(p, ceil_div(nwords, 8 * SP_WORDS)), 256, 0, st>>>(Z, q, nwords, S);
     pad_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(Q0, (size_t)q, l, LP, w.Q);
     MDBF_CUDA(cudaGetLastError());
     mdbf_status_t rc = orth<LP>(w.Q, q, w, st);                        // twice: the start block may be badly conditioned
@@ -418,17 +432,17 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
     const dim3 zy_grid(ceil_div(q, ZY_COLS), zy_chunks);
     const int aq_grid = ceil_div(p, AQ_WARPS * AQ_ROWS);
     for (int it = 0; it < n_iter; ++it) {
-        absz_q_kernel<LP><<<aq_grid, AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y);
+        absz_q_kernel<LP, MASKED><<<aq_grid, AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y, S, nwords);
         rc = orth<LP>(w.Y, p, w, st);
         if (rc) return rc;
-        abszT_y_kernel<LP><<<zy_grid, ZY_COLS, 0, st>>>(Z, p, q, w.Y, w.P);
+        abszT_y_kernel<LP, MASKED><<<zy_grid, ZY_COLS, 0, st>>>(Z, p, q, w.Y, w.P, S, nwords);
         chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, zy_chunks, (size_t)q * LP, w.Q);
         MDBF_CUDA(cudaGetLastError());
         rc = orth<LP>(w.Q, q, w, st);
         if (rc == MDBF_OK && it == n_iter - 1) rc = orth<LP>(w.Q, q, w, st);   // the last block carries the result: orthonormal to fp32
         if (rc) return rc;
     }
-    absz_q_kernel<LP><<<aq_grid, AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y);
+    absz_q_kernel<LP, MASKED><<<aq_grid, AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y, S, nwords);
     const int ychunks = ceil_div(p, GR_ROWS);
     gram_kernel<LP><<<ychunks, 256, 0, st>>>(w.Y, p, w.Gp);
     gram_sum_kernel<<<ceil_div(LP * LP, 8), 256, 0, st>>>(w.Gp, ychunks, LP * LP, w.Gs);
@@ -464,30 +478,47 @@ extern "C" mdbf_status_t mdbf_msvid_workspace_bytes(int64_t rows, int64_t cols, 
     return MDBF_OK;
 }
 
-extern "C" mdbf_status_t mdbf_msvid(const float *Z, int64_t rows, int64_t cols, int32_t l, int32_t n_iter, const float *Q0,
-                                    uint32_t *S_packed, float *U, float *V, float *sigma, void *workspace, size_t workspace_bytes,
-                                    void *stream) {
-    if (!Z || !Q0 || !S_packed || !U || !V || !sigma || !workspace) { set_error("mdbf_msvid: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
-    mdbf_status_t rc = msv::check_shape("mdbf_msvid", rows, cols, l);
+static mdbf_status_t msvid_entry(const char *who, bool masked, const float *Z, int64_t rows, int64_t cols, int32_t l, int32_t n_iter,
+                                 const float *Q0, uint32_t *S_packed, float *U, float *V, float *sigma, void *workspace,
+                                 size_t workspace_bytes, void *stream) {
+    if (!Z || !Q0 || !S_packed || !U || !V || !sigma || !workspace) { set_error("%s: NULL pointer", who); return MDBF_ERR_INVALID_ARG; }
+    mdbf_status_t rc = msv::check_shape(who, rows, cols, l);
     if (rc) return rc;
-    if (n_iter < 1 || n_iter > 1000) { set_error("mdbf_msvid: n_iter=%d outside [1, 1000]", n_iter); return MDBF_ERR_SHAPE; }
+    if (n_iter < 1 || n_iter > 1000) { set_error("%s: n_iter=%d outside [1, 1000]", who, n_iter); return MDBF_ERR_SHAPE; }
     const int p = (int)rows, q = (int)cols, LP = msv::padded_rank(l);
     msv::Scratch w;
     const size_t need = msv::carve(&w, (char *)workspace, p, q, LP);
     if (workspace_bytes < need || ((uintptr_t)workspace & 255u) != 0) {
-        set_error("mdbf_msvid: the workspace must hold %zu bytes (mdbf_msvid_workspace_bytes) on a 256-byte boundary; got %zu at %p",
+        set_error("%s: the workspace must hold %zu bytes (mdbf_msvid_workspace_bytes) on a 256-byte boundary; got %zu at %p", who,
                   need, workspace_bytes, workspace);
         return MDBF_ERR_INVALID_ARG;
     }
     rc = require_device(nullptr);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+#define MSV_RUN(LPV)                                                                                              \
+    return masked ? msv::run<LPV, true>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st)                    \
+                  : msv::run<LPV, false>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st)
     switch (LP) {
-        case 1: return msv::run<1>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
-        case 2: return msv::run<2>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
-        case 4: return msv::run<4>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
-        case 8: return msv::run<8>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
-        case 16: return msv::run<16>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
-        default: return msv::run<32>(Z, p, q, l, n_iter, Q0, S_packed, U, V, sigma, w, st);
+        case 1: MSV_RUN(1);
+        case 2: MSV_RUN(2);
+        case 4: MSV_RUN(4);
+        case 8: MSV_RUN(8);
+        case 16: MSV_RUN(16);
+        default: MSV_RUN(32);
     }
+#undef MSV_RUN
+}
+
+extern "C" mdbf_status_t mdbf_msvid(const float *Z, int64_t rows, int64_t cols, int32_t l, int32_t n_iter, const float *Q0,
+                                    uint32_t *S_packed, float *U, float *V, float *sigma, void *workspace, size_t workspace_bytes,
+                                    void *stream) {
+    return msvid_entry("mdbf_msvid", false, Z, rows, cols, l, n_iter, Q0, S_packed, U, V, sigma, workspace, workspace_bytes, stream);
+}
+
+extern "C" mdbf_status_t mdbf_project_fixed_mask(const float *Z, const uint32_t *S_packed, int64_t rows, int64_t cols, int32_t l,
+                                                 int32_t n_iter, const float *Q0, float *U, float *V, float *sigma, void *workspace,
+                                                 size_t workspace_bytes, void *stream) {
+    return msvid_entry("mdbf_project_fixed_mask", true, Z, rows, cols, l, n_iter, Q0, const_cast<uint32_t *>(S_packed), U, V, sigma,
+                       workspace, workspace_bytes, stream);
 }

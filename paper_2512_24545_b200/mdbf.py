@@ -29,7 +29,7 @@ EXPORTS = (
     "mdbf_pack_signs", "mdbf_unpack_signs", "mdbf_pack", "mdbf_get_packed", "mdbf_get_envelope",
     "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host", "mdbf_linear_forward_host_async", "mdbf_prepare_host_staging",
     "mdbf_linear_forward_static", "mdbf_linear_forward_sum", "mdbf_linear_forward_siblings", "mdbf_linear_forward_group",
-    "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_msvid", "mdbf_msvid_workspace_bytes", "mdbf_poll_status", "mdbf_selftest_wait_timeout", "mdbf_debug_fail_alloc",
+    "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_msvid", "mdbf_msvid_workspace_bytes", "mdbf_project_fixed_mask", "mdbf_poll_status", "mdbf_selftest_wait_timeout", "mdbf_debug_fail_alloc",
     "mdbf_last_launch_count",
     "mdbf_last_kernel",
     "mdbf_destroy", "mdbf_last_error", "mdbf_version",
@@ -80,6 +80,7 @@ def lib() -> ctypes.CDLL:
     L.mdbf_get_intermediate.argtypes = [vp, vp, i32, ctypes.c_int, vp]
     L.mdbf_reconstruct.argtypes = [vp, vp, vp]
     L.mdbf_msvid.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    L.mdbf_project_fixed_mask.argtypes = [vp, vp, i64, i64, i32, i32, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     L.mdbf_msvid_workspace_bytes.argtypes = [i64, i64, i32, ctypes.POINTER(ctypes.c_size_t)]
     L.mdbf_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
     L.mdbf_selftest_wait_timeout.argtypes = [vp, vp]
@@ -240,6 +241,14 @@ def mdbf_msvid(Z, rows: int, cols: int, l: int, n_iter: int, Q0, S_packed, U, V,
     balanced envelope factors and singular values; asynchronous, the caller owns the workspace.  See include/mdbf.h."""
     _check(lib().mdbf_msvid(_addr(Z), rows, cols, l, n_iter, _addr(Q0), _addr(S_packed), _addr(U), _addr(V), _addr(sigma),
                             _addr(workspace), workspace_bytes, stream))
+
+
+def mdbf_project_fixed_mask(Z, S_packed, rows: int, cols: int, l: int, n_iter: int, Q0, U, V, sigma, workspace, workspace_bytes: int,
+                            stream: int = 0) -> None:
+    """S (.) TSVD_l(S (.) Z) for a given packed mask S (Theorem 1's minimiser): balanced factors of the envelope and its
+    singular values; device addresses throughout, asynchronous.  See include/mdbf.h."""
+    _check(lib().mdbf_project_fixed_mask(_addr(Z), _addr(S_packed), rows, cols, l, n_iter, _addr(Q0), _addr(U), _addr(V), _addr(sigma),
+                                         _addr(workspace), workspace_bytes, stream))
 
 
 def mdbf_debug_fail_alloc(nth: int) -> None:

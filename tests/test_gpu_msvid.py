@@ -115,6 +115,52 @@ def test_full_size_factor():
     assert tail2 * (1 - 1e-4) <= err2 <= tail2 * 1.01
 
 
+def run_projection(Z, S, l, n_iter, seed=11):
+    rows, cols = Z.shape
+    Zd = torch.from_numpy(np.ascontiguousarray(Z, dtype=np.float32)).cuda()
+    Qd = torch.from_numpy(inputs.make_start_block(cols, l, seed)).cuda()
+    Sd = torch.from_numpy(orc.pack_signs(S).view(np.int32)).cuda()
+    Ud = torch.full((rows, l), float("nan"), dtype=torch.float32, device="cuda")
+    Vd = torch.full((cols, l), float("nan"), dtype=torch.float32, device="cuda")
+    sd = torch.full((l,), float("nan"), dtype=torch.float32, device="cuda")
+    nbytes = M.mdbf_msvid_workspace_bytes(rows, cols, l)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    M.mdbf_project_fixed_mask(Zd.data_ptr(), Sd.data_ptr(), rows, cols, l, n_iter, Qd.data_ptr(), Ud.data_ptr(), Vd.data_ptr(), sd.data_ptr(),
+                              ws.data_ptr(), nbytes, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    return Ud.cpu().numpy().astype(np.float64), Vd.cpu().numpy().astype(np.float64), sd.cpu().numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("shape,l", [((300, 517), 4), ((1024, 768), 16), ((129, 33), 1), ((64, 2000), 8), ((700, 900), 32)])
+def test_projection_under_a_given_mask(shape, l):
+    """Theorem 1 with a mask that is NOT the sign of Z: the envelope S (.) Z has entries of both signs and no dominant
+    direction; the error of the projection is bounded below by Eq. rankl-error and the iteration ends close to it."""
+    rows, cols = shape
+    Z = inputs.make_factor_matrix(rows, cols, seed=9, special_values=False)
+    S = inputs.make_signs(rows, cols, seed=21, stream="S_A")
+    P_ref, sv = orc.project_fixed_mask(S, Z, l)
+    tail = np.sqrt(np.sum(sv[l:] ** 2))
+    U, V, s = run_projection(Z, S, l, n_iter=12)
+    assert np.all(np.isfinite(U)) and np.all(np.isfinite(V))
+    assert np.all(s <= sv[:l] * (1 + 2e-5)) and np.all(s >= 0.75 * sv[:l])
+    P = S * (U @ V.T)
+    err = np.linalg.norm(Z.astype(np.float64) - P)
+    assert abs(np.linalg.norm(Z.astype(np.float64) - P_ref) - tail) <= 1e-9 * sv[0]      # the oracle attains the bound
+    assert tail * (1 - 1e-5) <= err <= tail * 1.02
+    # the envelope error is the same number (Eq. envelope-isometry)
+    assert abs(np.linalg.norm(S * Z.astype(np.float64) - U @ V.T) - err) <= 1e-9 * sv[0]
+
+
+def test_projection_with_the_matrix_own_mask_is_msvid():
+    Z = inputs.make_factor_matrix(257, 390, seed=10)
+    S = np.where(Z >= 0, 1, -1).astype(np.int8)
+    _, U1, V1, s1 = run_msvid(Z, 8, n_iter=5)
+    U2, V2, s2 = run_projection(Z, S, 8, n_iter=5)
+    np.testing.assert_array_equal(s1, s2)                    # the same kernels on the same envelope: the same bits
+    np.testing.assert_array_equal(U1, U2)
+    np.testing.assert_array_equal(V1, V2)
+
+
 def test_argument_errors():
     Z = torch.zeros((8, 8), dtype=torch.float32, device="cuda")
     Q = torch.ones((8, 2), dtype=torch.float32, device="cuda")
