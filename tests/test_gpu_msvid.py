@@ -161,6 +161,48 @@ def test_projection_with_the_matrix_own_mask_is_msvid():
     np.testing.assert_array_equal(V1, V2)
 
 
+def test_msvid_of_both_factors_makes_a_layer():
+    """Eq. mesvid-init-compact from given balanced factors: MSVID_l of U0 (d_out x k) and of V0^T (k x d_in) on the GPU,
+    the two masks and envelopes packed into a layer, and that layer's dense reconstruction and forward compared with
+    the oracle's - whose own MSVID (exact SVD) sets the approximation error the GPU initialisation has to come close to."""
+    d_out, d_in, k, l = 384, 320, 128, 8
+    rng = np.random.default_rng(44)
+    W = (rng.standard_normal((d_out, 48)) @ rng.standard_normal((48, d_in)) / 7 + 0.3 * rng.standard_normal((d_out, d_in)))
+    Uw, sw, Vwt = np.linalg.svd(W, full_matrices=False)
+    U0 = (Uw[:, :k] * np.sqrt(sw[:k])).astype(np.float32)                  # Eq. mesvid-balanced, given as inputs
+    V0t = (np.sqrt(sw[:k])[:, None] * Vwt[:k]).astype(np.float32)
+    W_R = U0.astype(np.float64) @ V0t.astype(np.float64)
+    SpA, UA, VA, _ = run_msvid(U0, l, n_iter=12)
+    SpB, UB, VB, _ = run_msvid(V0t, l, n_iter=12)
+    S_A, S_B = orc.unpack_signs(SpA, k), orc.unpack_signs(SpB, d_in)
+    # the same construction in the oracle (exact truncated SVDs)
+    So_A, Uo_A, Vo_A = orc.msvid(U0, l)
+    So_B, Uo_B, Vo_B = orc.msvid(V0t, l)
+    np.testing.assert_array_equal(S_A, So_A)
+    np.testing.assert_array_equal(S_B, So_B)
+    W_gpu_init = orc.reconstruct(S_A, S_B, UA, VA, UB, VB)
+    W_orc_init = orc.reconstruct(So_A, So_B, Uo_A, Vo_A, Uo_B, Vo_B)
+    e_gpu = np.linalg.norm(W_R - W_gpu_init) / np.linalg.norm(W_R)
+    e_orc = np.linalg.norm(W_R - W_orc_init) / np.linalg.norm(W_R)
+    assert e_gpu <= e_orc * 1.03                                            # the initialisation is as good as the exact one, within 3 %
+    # the factors as a layer of the library (fp32 envelopes: no storage rounding in the way)
+    h = M.mdbf_pack(d_out, d_in, k, l, M.F32, 4, S_A, S_B, *[np.ascontiguousarray(a, dtype=np.float32) for a in (UA, VA, UB, VB)])
+    try:
+        Wd = torch.empty((d_out, d_in), dtype=torch.float32, device="cuda")
+        M.mdbf_reconstruct(h, Wd.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert orc.rel_frobenius(Wd.cpu().numpy(), W_gpu_init) <= 1e-6
+        x = rng.standard_normal((4, d_in)).astype(np.float32)
+        xd = torch.from_numpy(x).cuda()
+        yd = torch.empty((4, d_out), dtype=torch.float32, device="cuda")
+        M.mdbf_linear_forward(h, xd.data_ptr(), yd.data_ptr(), 4, M.F32, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        ref = (W_gpu_init @ x.T.astype(np.float64)).T
+        assert orc.rel_frobenius(yd.cpu().numpy(), ref) <= 1e-5
+    finally:
+        M.mdbf_destroy(h)
+
+
 def test_argument_errors():
     Z = torch.zeros((8, 8), dtype=torch.float32, device="cuda")
     Q = torch.ones((8, 2), dtype=torch.float32, device="cuda")
