@@ -43,9 +43,9 @@ NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     ("decode_mlp_T16", "mat_small_kernel"): 6340000,               # up stage B (stage A: 6.11 MB, down stage A: 2.47 MB)
     ("prefill_4096_l16_bpw10", "mat_stage_kernel"): 17858048,      # stage B: x read once + signs + images; nothing reaches DRAM on the way out
     ("prefill_4096_l16_bpw10", "gemm_stage_kernel"): 370142976,    # stage B: 269.4 MB read + 100.7 MB written
-    ("msvid_28672x6016_l16", "absz_q_kernel"): 701000000,         # Z once per pass (689.9 MB) + the skinny operand and result, scaled by
-                                                                   # rows x cols from the 8192 x 8192 capture (273.0 MB for 268.4 MB of Z)
-    ("msvid_8192x8192_l16", "absz_q_kernel"): 273003776,
+    ("msvid_28672x6016_l16", "absz_q_kernel"): 703000000,         # Z once per pass (689.9 MB) + the skinny operand and result, scaled by
+                                                                   # rows x cols from the 8192 x 8192 capture (273.6 MB for 268.4 MB of Z)
+    ("msvid_8192x8192_l16", "absz_q_kernel"): 273649664,
     ("block70b_T2048", "mat_stage_kernel"): 197116928,             # its largest launch, down stage B (185.9 MB read: 117 MB of x, partly twice,
                                                                    # + signs; 11.3 MB written); gate / up stage A: 123.3 MB
 }
