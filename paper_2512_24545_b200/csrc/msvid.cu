@@ -255,50 +255,44 @@ __global__ void __launch_bounds__(256) gram_sum_kernel(const double *__restrict_
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if (lane == 0) G[e] = s;
 }
-// One CTA: G = sum of the partial Gram matrices = L L^T; M[b][a] = (L^-1)[a][b], so that A M has orthonormal columns.
-// A zero (or numerically vanished) pivot - a padding column, or a block wider than the rank of the matrix - leaves
-// its column as it is instead of dividing by zero.
+// One warp, lane = row: G = L L^T (G: the summed Gram matrix, lower triangle); M[b][a] = (L^-1)[a][b], so that A M has
+// orthonormal columns.  A zero (or numerically vanished) pivot - a padding column, or a block wider than the rank of
+// the matrix - leaves its column as it is instead of dividing by zero.
 template <int LP>
-__global__ void __launch_bounds__(LP * LP < 32 ? 32 : LP * LP) chol_kernel(const double *__restrict__ Gp, int nchunks, float *__restrict__ M) {
+__global__ void __launch_bounds__(32) chol_kernel(const double *__restrict__ Gs, float *__restrict__ M) {
     __shared__ double G[LP][LP + 1], Li[LP][LP + 1];
-    const int tid = threadIdx.x;
-    const int a = tid / LP, b = tid - a * LP;
-    if (tid < LP * LP) {
-        double s = 0.0;
-#pragma unroll 8
-        for (int c = 0; c < nchunks; ++c) s += Gp[(size_t)c * LP * LP + tid];
-        G[a][b] = s;                                   // lower triangle (b <= a) holds the sums
-        Li[a][b] = 0.0;
+    const int k = threadIdx.x;
+    for (int e = k; e < LP * LP; e += 32) {
+        G[e / LP][e % LP] = Gs[e];
+        Li[e / LP][e % LP] = 0.0;
     }
-    __syncthreads();
+    __syncwarp();
     double scale = 0.0;
-    if (tid == 0)
-        for (int k = 0; k < LP; ++k) scale = fmax(scale, G[k][k]);
-    // column-by-column Cholesky on the lower triangle, one thread per row
-    for (int k = 0; k < LP; ++k) {
-        if (tid == 0) {
-            const double d = G[k][k];
-            G[k][k] = d > 1e-24 * scale && d > 0.0 ? sqrt(d) : 0.0;
+    for (int d = 0; d < LP; ++d) scale = fmax(scale, G[d][d]);
+    // column-by-column Cholesky on the lower triangle
+    for (int c = 0; c < LP; ++c) {
+        if (k == c) {
+            const double d = G[c][c];
+            G[c][c] = d > 1e-24 * scale && d > 0.0 ? sqrt(d) : 0.0;
         }
-        __syncthreads();
-        const double d = G[k][k];
-        if (tid > k && tid < LP) G[tid][k] = d > 0.0 ? G[tid][k] / d : 0.0;
-        __syncthreads();
-        if (tid > k && tid < LP)
-            for (int jj = k + 1; jj <= tid; ++jj) G[tid][jj] -= G[tid][k] * G[jj][k];
-        __syncthreads();
+        __syncwarp();
+        const double d = G[c][c];
+        if (k > c && k < LP) G[k][c] = d > 0.0 ? G[k][c] / d : 0.0;
+        __syncwarp();
+        if (k > c && k < LP)
+            for (int jj = c + 1; jj <= k; ++jj) G[k][jj] -= G[k][c] * G[jj][c];
+        __syncwarp();
     }
-    // inverse of the lower-triangular factor, one thread per column
-    if (tid < LP) {
-        const int c = tid;
-        for (int i = c; i < LP; ++i) {
-            double s = i == c ? 1.0 : 0.0;
-            for (int k = c; k < i; ++k) s -= G[i][k] * Li[k][c];
-            Li[i][c] = G[i][i] > 0.0 ? s / G[i][i] : (i == c ? 1.0 : 0.0);
+    // inverse of the lower-triangular factor, one lane per column
+    if (k < LP) {
+        for (int i = k; i < LP; ++i) {
+            double sum = i == k ? 1.0 : 0.0;
+            for (int m = k; m < i; ++m) sum -= G[i][m] * Li[m][k];
+            Li[i][k] = G[i][i] > 0.0 ? sum / G[i][i] : (i == k ? 1.0 : 0.0);
         }
     }
-    __syncthreads();
-    if (tid < LP * LP) M[tid] = (float)Li[b][a];        // M[a][b] with a = row index of M: M[a][b] = Li[b][a]
+    __syncwarp();
+    for (int e = k; e < LP * LP; e += 32) M[e] = (float)Li[e % LP][e / LP];      // M[a][b] = Li[b][a]
 }
 // A <- A M, row by row (M is LP x LP, row-major)
 template <int LP>
@@ -359,7 +353,8 @@ __global__ void __launch_bounds__(32) jacobi_kernel(const double *__restrict__ G
             off += __shfl_xor_sync(0xffffffffu, off, o);
             diag += __shfl_xor_sync(0xffffffffu, diag, o);
         }
-        if (off <= 1e-24 * diag) break;                          // off-diagonal mass below 1e-12 of the diagonal's
+        if (off <= 1e-20 * diag) break;                          // off-diagonal mass below 1e-10 of the diagonal's: the eigenvalues are then
+                                                                 // accurate to the square of that
         for (int r = 0; r < n - 1; ++r) {
             if (k < n / 2) {
                 const int a = k == 0 ? n - 1 : (r + k) % (n - 1), b = k == 0 ? r : (r - k + (n - 1)) % (n - 1);
@@ -465,7 +460,7 @@ static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st) {
     const int chunks = ceil_div(n, GR_ROWS);
     gram_kernel<LP><<<chunks, 256, 0, st>>>(A, n, w.Gp);
     gram_sum_kernel<<<ceil_div(LP * LP, 8), 256, 0, st>>>(w.Gp, chunks, LP * LP, w.Gs);
-    chol_kernel<LP><<<1, LP * LP < 32 ? 32 : LP * LP, 0, st>>>(w.Gs, 1, w.M);
+    chol_kernel<LP><<<1, 32, 0, st>>>(w.Gs, w.M);
     right_mul_kernel<LP><<<ceil_div(n, 256), 256, 0, st>>>(A, n, w.M, nullptr, 0);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
