@@ -121,3 +121,16 @@ def test_no_cpu_fallback_without_a_device():
     with pytest.raises(M.MdbfError) as e:
         M.mdbf_pack_signs(S, 4, 4, out, on_device=True)
     assert e.value.status == M.ERR_ARCH
+
+
+def test_msvid_workspace_size_is_a_host_computation():
+    """No device needed: the size grows with the shape and the envelope rank, bad shapes are refused."""
+    a = M.mdbf_msvid_workspace_bytes(1024, 768, 4)
+    b = M.mdbf_msvid_workspace_bytes(1024, 768, 16)
+    c = M.mdbf_msvid_workspace_bytes(4096, 768, 16)
+    assert 0 < a < b < c and a % 256 == 0
+    assert M.mdbf_msvid_workspace_bytes(1024, 768, 5) == M.mdbf_msvid_workspace_bytes(1024, 768, 8)   # rank padded to a power of two
+    for bad in ((0, 8, 1), (8, 0, 1), (8, 8, 0), (8, 8, 9), (8, 8, 33)):
+        with pytest.raises(M.MdbfError) as e:
+            M.mdbf_msvid_workspace_bytes(*bad)
+        assert e.value.status == M.ERR_SHAPE
