@@ -23,6 +23,7 @@
 #include <cmath>
 
 #include "common.cuh"
+#include "tmem_ptx.cuh"
 
 namespace mdbf {
 namespace msv {
@@ -166,6 +167,260 @@ __global__ void __launch_bounds__(AQ_WARPS * 32) absz_q_kernel(const float *__re
             for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
             if (lane == 0 && r0 + r < p) Y[(size_t)(r0 + r) * LP + t] = v;
         }
+}
+
+// ------------------------------------------------------------------ Y = |Z| Q on the tensor cores
+// The same product as absz_q_kernel with tcgen05 (kind::tf32, fp32 accumulators in tensor memory) and a three-term
+// split that keeps fp32 accuracy:  e = e_hi + e_lo,  q = q_hi + q_lo  (each part a TF32 number),
+//     e q  ~  e_hi q_hi + e_hi q_lo + e_lo q_hi                      (the dropped e_lo q_lo is below 2^-22 e q).
+// CTA = 128 rows x a range of K blocks of 32 columns (split over blockIdx.y, partial sums per range).  Per K block:
+//   one lane brings the raw 128 x 32 tile of Z into a ring of TC_RAW buffers by TMA (zero fill outside the matrix), so the
+//     bytes in flight do not depend on how many threads wait for them;
+//   8 converter warps (two groups on alternate K blocks; a quarter warp = one row's 128 bytes, so every shared-memory
+//     access touches each bank once) take the envelope (absolute value, or the sign flipped by the mask word - a K block
+//     is exactly one packed word), split it and write the operand tiles E_hi, E_lo (128 x 32 TF32, K-major, 128B swizzle);
+//   one lane bulk-copies the K block's image of Q: rows [0, LPP) = q_hi, [LPP, 2 LPP) = q_lo of the 32 columns,
+//     already in the operand layout (qimg_kernel builds the images once per pass);
+//   two lanes issue the MMAs, four K steps of 8 each: D1 (+)= E_hi [q_hi | q_lo] (N = 2 LPP), D2 (+)= E_lo q_hi (N = LPP).
+// Epilogue: thread = row = TMEM lane: y[t] = D1[t] + D1[LPP + t] + D2[t] into the range's partial sums.
+// Needs cols % 4 == 0 and Z on a 16-byte boundary (the tensor map's rules); other inputs take absz_q_kernel.
+// Every wait is bounded; on expiry the status word of the workspace is set and the call's outputs are NaN.
+constexpr int TC_KB = 32, TC_CONVERTERS = 256;
+constexpr int TC_W_ISSUE = 8, TC_W_RAW = 10, TC_W_IMG = 11, TC_THREADS = 12 * 32;
+constexpr int TC_TILE = 128 * TC_KB * 4;                        // bytes of a raw tile and of each operand tile
+template <int LP> struct TcCfg {
+    static constexpr int LPP = LP < 16 ? 16 : LP;              // MMA N is a multiple of 16
+    static constexpr int N1 = 2 * LPP, N2 = LPP;
+    static constexpr int IMG = N1 * 128;                        // bytes of one K block's image of Q
+    static constexpr int STAGE = 2 * TC_TILE + IMG;             // E_hi, E_lo, image
+    static constexpr int TMEM_COLS = N1 + N2 <= 64 ? 64 : 128;
+    // two CTAs per SM where their shared memory fits side by side (one's prologue and epilogue under the other's stream)
+    static constexpr int CTAS_PER_SM = LP <= 16 ? 2 : 1;
+    static constexpr int RAW = CTAS_PER_SM == 2 ? 2 : 4;       // raw tiles in flight per CTA
+    static constexpr int STAGES = CTAS_PER_SM == 2 ? 2 : 3;    // operand stages
+    static constexpr size_t SMEM = 1024 + (size_t)RAW * TC_TILE + (size_t)STAGES * STAGE;
+};
+__device__ __forceinline__ uint32_t tf32_round(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;\n" : "=r"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ void umma_ss_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// instruction descriptor: fp32 accumulator, A and B TF32, both K-major, M = 128
+__device__ __forceinline__ uint32_t make_idesc_tf32(int n) {
+    uint32_t d = 0;
+    d |= 1u << 4;                       // D: fp32
+    d |= 2u << 7;                       // A: tf32
+    d |= 2u << 10;                      // B: tf32
+    d |= (uint32_t)(n >> 3) << 17;      // N
+    d |= (uint32_t)(128 >> 4) << 24;    // M
+    return d;
+}
+// images of Q for one pass: K block kb holds rows n of 32 TF32 values, 128 bytes each, 128B swizzle
+template <int LP>
+__global__ void __launch_bounds__(256) qimg_kernel(const float *__restrict__ Q, int q, int nkb, uint32_t *__restrict__ img) {
+    constexpr int LPP = TcCfg<LP>::LPP, N1 = TcCfg<LP>::N1;
+    const size_t total = (size_t)nkb * N1 * 32;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+        const int kappa = (int)(e & 31);
+        const int n = (int)((e >> 5) % N1);
+        const int kb = (int)(e / ((size_t)N1 * 32));
+        const int t = n < LPP ? n : n - LPP;
+        const int col = kb * 32 + kappa;
+        const float v = (t < LP && col < q) ? Q[(size_t)col * LP + t] : 0.f;
+        const uint32_t hi = tf32_round(v);
+        const uint32_t out = n < LPP ? hi : tf32_round(v - __uint_as_float(hi));
+        img[(size_t)kb * (N1 * 32) + n * 32 + ((((kappa >> 2) ^ (n & 7)) << 2) | (kappa & 3))] = out;
+    }
+}
+template <int LP, bool MASKED>
+__global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) absz_q_tc_kernel(const __grid_constant__ CUtensorMap tmap_z, int p, int q,
+                                                                  const uint32_t *__restrict__ img, int kb_per_cta, float *__restrict__ P,
+                                                                  const uint32_t *__restrict__ S, int nwords, int32_t *__restrict__ status) {
+    using namespace tm;
+    using C = TcCfg<LP>;
+    constexpr int LPP = C::LPP, N1 = C::N1, N2 = C::N2, TC_RAW = C::RAW, TC_STAGES = C::STAGES;
+    extern __shared__ unsigned char tc_smem_raw[];
+    __shared__ __align__(8) uint64_t bars[2 * TC_STAGES + 2 * TC_RAW + 1];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag_s;
+    volatile int *abort_flag = &abort_flag_s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t smem_base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
+    unsigned char *smem_gen = tc_smem_raw + (smem_base - smem_u32(tc_smem_raw));
+    const uint32_t op_base = smem_base + (uint32_t)(TC_RAW * TC_TILE);
+    unsigned char *op_gen = smem_gen + TC_RAW * TC_TILE;
+    const uint32_t full_bar = smem_u32(&bars[0]), empty_bar = smem_u32(&bars[TC_STAGES]);
+    const uint32_t raw_full = smem_u32(&bars[2 * TC_STAGES]), raw_empty = smem_u32(&bars[2 * TC_STAGES + TC_RAW]);
+    const uint32_t accum_bar = smem_u32(&bars[2 * TC_STAGES + 2 * TC_RAW]);
+    const int row0 = blockIdx.x * 128;
+    const int nkb_total = (q + TC_KB - 1) / TC_KB;
+    const int kb0 = blockIdx.y * kb_per_cta;
+    const int nkb = max(0, min(kb_per_cta, nkb_total - kb0));
+    if (tid == 0) {
+        for (int s = 0; s < TC_STAGES; ++s) {
+            mbar_init(full_bar + 8 * s, 128 + 1);                // a converter group + the image's expect_tx
+            mbar_init(empty_bar + 8 * s, 2);                     // the two issuing lanes (commits)
+        }
+        for (int s = 0; s < TC_RAW; ++s) {
+            mbar_init(raw_full + 8 * s, 1);                      // the tile's expect_tx
+            mbar_init(raw_empty + 8 * s, 128);                   // the converter group that read it
+        }
+        mbar_init(accum_bar, 2);
+        abort_flag_s = 0;
+        fence_barrier_init();
+    }
+    if (warp == TC_W_ISSUE) {
+        tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_slot;
+
+    if (warp < TC_CONVERTERS / 32) {
+        // ============================ converters, then epilogue ============================
+        const int grp = warp >> 2;                               // K blocks grp, grp + 2, ...
+        const int rsub = (warp & 3) * 4 + (lane >> 3);           // rows rsub + 16 i, i = 0..7
+        const int chunk = lane & 7;
+        bool alive = true;
+        uint32_t word[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) word[i] = 0u;
+        if (MASKED && grp < nkb) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int gr = row0 + rsub + 16 * i;
+                if (gr < p) word[i] = S[(size_t)gr * nwords + kb0 + grp];
+            }
+        }
+        for (int kb = grp; kb < nkb && alive; kb += 2) {
+            const int s = kb % TC_STAGES, rs = kb % TC_RAW;
+            uint32_t word_next[8];
+            if (MASKED) {                                        // the next block's mask words travel while this one is converted
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int gr = row0 + rsub + 16 * i;
+                    word_next[i] = (kb + 2 < nkb && gr < p) ? S[(size_t)gr * nwords + kb0 + kb + 2] : 0u;
+                }
+            }
+            alive = mbar_wait(raw_full + 8 * rs, ((uint32_t)(kb / TC_RAW)) & 1u, abort_flag, status);
+            if (alive) alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(kb / TC_STAGES)) & 1u) ^ 1u, abort_flag, status);
+            alive = __all_sync(0xffffffffu, alive);
+            if (!alive) break;
+            const unsigned char *raw = smem_gen + (size_t)rs * TC_TILE;
+            unsigned char *stage = op_gen + (size_t)s * C::STAGE;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = rsub + 16 * i;
+                const float4 v = *reinterpret_cast<const float4 *>(raw + r * 128 + chunk * 16);
+                const float in[4] = {v.x, v.y, v.z, v.w};
+                uint32_t h[4], l[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float e = MASKED ? __uint_as_float(__float_as_uint(in[j]) ^ (((word[i] >> (4 * chunk + j)) & 1u) << 31)) : fabsf(in[j]);
+                    h[j] = tf32_round(e);
+                    l[j] = tf32_round(e - __uint_as_float(h[j]));
+                }
+                const int off = r * 128 + ((chunk ^ (r & 7)) << 4);
+                *reinterpret_cast<uint4 *>(stage + off) = make_uint4(h[0], h[1], h[2], h[3]);
+                *reinterpret_cast<uint4 *>(stage + TC_TILE + off) = make_uint4(l[0], l[1], l[2], l[3]);
+            }
+            mbar_arrive(raw_empty + 8 * rs);
+            fence_proxy_async();
+            mbar_arrive(full_bar + 8 * s);
+            if (MASKED) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) word[i] = word_next[i];
+            }
+        }
+        if (warp < 4) {
+            const int grow = row0 + tid;
+            if (alive) alive = mbar_wait(accum_bar, 0u, abort_flag, status);
+            alive = __all_sync(0xffffffffu, alive);
+            tc_fence_after();
+            const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+            float y[LPP];
+#pragma unroll
+            for (int t = 0; t < LPP; ++t) y[t] = 0.f;
+            if (alive && nkb > 0) {
+#pragma unroll
+                for (int c16 = 0; c16 < (N1 + N2) / 16; ++c16) {
+                    uint32_t d[16];
+                    tmem_ld16(tmem + lane_base + (uint32_t)(c16 * 16), d);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) y[(c16 * 16 + e) % LPP] += __uint_as_float(d[e]);      // columns t, LPP + t and N1 + t belong to mode t
+                }
+            }
+            if (grow < p) {
+                float *out = P + ((size_t)blockIdx.y * p + grow) * LP;
+#pragma unroll
+                for (int t = 0; t < LP; ++t) out[t] = alive ? y[t] : __int_as_float(0x7fc00000);
+            }
+        }
+    } else if (warp == TC_W_ISSUE || warp == TC_W_ISSUE + 1) {
+        // ================================== MMA issuers ===================================
+        const bool first = warp == TC_W_ISSUE;                   // first: D1 = E_hi [q_hi | q_lo]; second: D2 = E_lo q_hi
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_tf32(first ? N1 : N2);
+            const uint32_t d_tmem = tmem + (first ? 0u : (uint32_t)N1);
+            bool alive = true;
+            for (int kb = 0; kb < nkb && alive; ++kb) {
+                const int s = kb % TC_STAGES;
+                alive = mbar_wait(full_bar + 8 * s, ((uint32_t)(kb / TC_STAGES)) & 1u, abort_flag, status);
+                if (!alive) break;
+                tc_fence_after();
+                const uint32_t stage = op_base + (uint32_t)(s * C::STAGE);
+                const uint64_t adesc = make_smem_desc(stage + (first ? 0u : (uint32_t)TC_TILE));
+                const uint64_t bdesc = make_smem_desc(stage + 2u * TC_TILE);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)                   // 8 TF32 = 32 bytes per K step
+                    umma_ss_tf32(d_tmem, adesc + (uint64_t)(2 * ks), bdesc + (uint64_t)(2 * ks), idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+                umma_commit(empty_bar + 8 * s);
+            }
+            if (alive && nkb > 0) umma_commit(accum_bar);
+            else mbar_arrive(accum_bar);
+        }
+        __syncwarp();
+    } else if (warp == TC_W_RAW) {
+        // ================================ raw tile loader ================================
+        if (lane == 0) {
+            bool alive = true;
+            for (int kb = 0; kb < nkb && alive; ++kb) {
+                const int rs = kb % TC_RAW;
+                alive = mbar_wait(raw_empty + 8 * rs, (((uint32_t)(kb / TC_RAW)) & 1u) ^ 1u, abort_flag, status);
+                if (!alive) break;
+                mbar_arrive_expect_tx(raw_full + 8 * rs, (uint32_t)TC_TILE);
+                tma_load_2d(smem_base + (uint32_t)(rs * TC_TILE), &tmap_z, (kb0 + kb) * TC_KB, row0, raw_full + 8 * rs);
+            }
+        }
+        __syncwarp();
+    } else if (warp == TC_W_IMG) {
+        // ================================= image loader ==================================
+        if (lane == 0) {
+            bool alive = true;
+            for (int kb = 0; kb < nkb && alive; ++kb) {
+                const int s = kb % TC_STAGES;
+                alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(kb / TC_STAGES)) & 1u) ^ 1u, abort_flag, status);
+                if (!alive) break;
+                mbar_arrive_expect_tx(full_bar + 8 * s, (uint32_t)C::IMG);
+                bulk_load(op_base + (uint32_t)(s * C::STAGE) + 2u * TC_TILE, img + (size_t)(kb0 + kb) * (C::IMG / 4), (uint32_t)C::IMG, full_bar + 8 * s);
+            }
+        }
+        __syncwarp();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) drain_delay();                              // let copies in flight land before the shared memory goes back
+    if (warp == TC_W_ISSUE) tmem_dealloc(tmem, (uint32_t)C::TMEM_COLS);
 }
 
 // ------------------------------------------------------------------ W = |Z|^T Y
@@ -432,7 +687,25 @@ __global__ void pad_kernel(const float *__restrict__ src, size_t n, int l, int L
 struct Scratch {
     float *Q, *Y, *P, *M, *MU, *MV;
     double *Gp, *Gs;
+    uint32_t *img;          // operand images of Q for the tensor-core product
+    int32_t *status;        // set by a wait that ran out
 };
+// how the K blocks of the tensor-core product are split over blockIdx.y: the split that fills whole waves of resident CTAs best,
+// each CTA keeping at least 8 K blocks
+static int tc_split(int p, int q, int LP, int *kb_per_cta) {
+    const int slots = 148 * (LP <= 16 ? 2 : 1);
+    const int rb = ceil_div(p, 128), nkb = ceil_div(q, TC_KB);
+    int best = 1;
+    double best_eff = -1.0;
+    for (int ns = 1; ns <= 16 && nkb / ns >= 8; ++ns) {
+        const int per = ceil_div(nkb, ns), parts = ceil_div(nkb, per);
+        const int ctas = rb * parts, waves = ceil_div(ctas, slots);
+        const double eff = (double)rb * nkb / ((double)waves * slots * per);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = ns; }
+    }
+    *kb_per_cta = ceil_div(nkb, best);
+    return ceil_div(nkb, *kb_per_cta);
+}
 static size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 static size_t carve(Scratch *w, char *base, int p, int q, int LP) {
     const size_t zy_chunks = ceil_div(p, ZY_ROWS), gchunks = ceil_div(max(p, q), GR_ROWS);
@@ -440,13 +713,17 @@ static size_t carve(Scratch *w, char *base, int p, int q, int LP) {
     auto take = [&](size_t bytes) { char *ptr = base ? base + off : nullptr; off += align256(bytes); return ptr; };
     float *Q = (float *)take((size_t)q * LP * sizeof(float));
     float *Y = (float *)take((size_t)p * LP * sizeof(float));
-    float *P = (float *)take(zy_chunks * q * LP * sizeof(float));
+    int kb_per_cta = 0;
+    const size_t tc_parts = (size_t)tc_split(p, q, LP, &kb_per_cta);
+    float *P = (float *)take(std::max(zy_chunks * q, tc_parts * p) * LP * sizeof(float));
+    uint32_t *img = (uint32_t *)take((size_t)ceil_div(q, TC_KB) * 2 * (LP < 16 ? 16 : LP) * 128);
+    int32_t *status = (int32_t *)take(sizeof(int32_t));
     double *Gp = (double *)take(gchunks * LP * LP * sizeof(double));
     double *Gs = (double *)take((size_t)LP * LP * sizeof(double));
     float *M = (float *)take((size_t)LP * LP * sizeof(float));
     float *MU = (float *)take((size_t)LP * LP * sizeof(float));
     float *MV = (float *)take((size_t)LP * LP * sizeof(float));
-    if (w) { w->Q = Q; w->Y = Y; w->P = P; w->Gp = Gp; w->Gs = Gs; w->M = M; w->MU = MU; w->MV = MV; }
+    if (w) { w->Q = Q; w->Y = Y; w->P = P; w->Gp = Gp; w->Gs = Gs; w->M = M; w->MU = MU; w->MV = MV; w->img = img; w->status = status; }
     return off;
 }
 static int padded_rank(int l) {
@@ -466,6 +743,61 @@ static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st) {
     return MDBF_OK;
 }
 
+// Tensor map of the fp32 matrix Z [p][q]: box of 32 columns x 128 rows, no swizzle, zero fill outside the matrix.
+static mdbf_status_t make_z_tensor_map(CUtensorMap *out, const float *Z, int p, int q) {
+    typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static encode_fn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        MDBF_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &res));
+        if (!ptr || res != cudaDriverEntryPointSuccess) {
+            set_error("cuTensorMapEncodeTiled is not available from the driver");
+            return MDBF_ERR_CUDA;
+        }
+        fn = reinterpret_cast<encode_fn>(ptr);
+    }
+    const cuuint64_t gdim[2] = {(cuuint64_t)q, (cuuint64_t)p};
+    const cuuint64_t gstride[1] = {(cuuint64_t)q * sizeof(float)};
+    const cuuint32_t box[2] = {(cuuint32_t)TC_KB, 128u};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(Z), gdim, gstride, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled (Z) failed with CUresult %d", (int)r);
+        return MDBF_ERR_CUDA;
+    }
+    return MDBF_OK;
+}
+static bool tc_eligible(const float *Z, int q) { return (q & 3) == 0 && (reinterpret_cast<uintptr_t>(Z) & 15u) == 0; }
+
+// Y = E Q with E the envelope of Z (|Z|, or Z with the given mask's signs taken off)
+template <int LP, bool MASKED>
+static mdbf_status_t product(const float *Z, int p, int q, const uint32_t *S, int nwords, const CUtensorMap *tmz, Scratch &w, cudaStream_t st) {
+    using C = TcCfg<LP>;
+    if (!tmz) {
+        absz_q_kernel<LP, MASKED><<<ceil_div(p, AQ_WARPS * AQ_ROWS), AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y, S, nwords);
+        MDBF_CUDA(cudaGetLastError());
+        return MDBF_OK;
+    }
+    static bool attr_set = false;
+    if (!attr_set) {
+        MDBF_CUDA(cudaFuncSetAttribute(absz_q_tc_kernel<LP, MASKED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM));
+        attr_set = true;
+    }
+    int kb_per_cta = 0;
+    const int parts = tc_split(p, q, LP, &kb_per_cta);
+    const int nkb = ceil_div(q, TC_KB);
+    qimg_kernel<LP><<<std::min(ceil_div(nkb * C::N1 * 32, 256), 148 * 8), 256, 0, st>>>(w.Q, q, nkb, w.img);
+    absz_q_tc_kernel<LP, MASKED><<<dim3(ceil_div(p, 128), parts), TC_THREADS, C::SMEM, st>>>(*tmz, p, q, w.img, kb_per_cta, w.P, S, nwords, w.status);
+    chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)p * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, parts, (size_t)p * LP, w.Y);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}
+
 // MASKED = false: S is written (the mask of Z itself, Eq. msvid-def); MASKED = true: S is given (Eq. Ustar)
 template <int LP, bool MASKED>
 static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const float *Q0, uint32_t *S, float *U, float *V, float *sigma,
@@ -479,10 +811,17 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
     if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st);
     if (rc) return rc;
     const dim3 zy_grid(ceil_div(q, ZY_COLS), zy_chunks);
-    const int aq_grid = ceil_div(p, AQ_WARPS * AQ_ROWS);
+    MDBF_CUDA(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));
+    CUtensorMap tmap_z;
+    const CUtensorMap *tmz = nullptr;
+    if (tc_eligible(Z, q)) {
+        rc = make_z_tensor_map(&tmap_z, Z, p, q);
+        if (rc) return rc;
+        tmz = &tmap_z;
+    }
     for (int it = 0; it < n_iter; ++it) {
-        absz_q_kernel<LP, MASKED><<<aq_grid, AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y, S, nwords);
-        rc = orth<LP>(w.Y, p, w, st);
+        rc = product<LP, MASKED>(Z, p, q, S, nwords, tmz, w, st);
+        if (rc == MDBF_OK) rc = orth<LP>(w.Y, p, w, st);
         if (rc) return rc;
         abszT_y_kernel<LP, MASKED><<<zy_grid, ZY_COLS, 0, st>>>(Z, p, q, w.Y, w.P, S, nwords);
         chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, zy_chunks, (size_t)q * LP, w.Q);
@@ -491,7 +830,8 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
         if (rc == MDBF_OK && it == n_iter - 1) rc = orth<LP>(w.Q, q, w, st);   // the last block carries the result: orthonormal to fp32
         if (rc) return rc;
     }
-    absz_q_kernel<LP, MASKED><<<aq_grid, AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y, S, nwords);
+    rc = product<LP, MASKED>(Z, p, q, S, nwords, tmz, w, st);
+    if (rc) return rc;
     const int ychunks = ceil_div(p, GR_ROWS);
     gram_kernel<LP><<<ychunks, 256, 0, st>>>(w.Y, p, w.Gp);
     gram_sum_kernel<<<ceil_div(LP * LP, 8), 256, 0, st>>>(w.Gp, ychunks, LP * LP, w.Gs);
