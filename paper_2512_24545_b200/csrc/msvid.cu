@@ -239,8 +239,11 @@ __global__ void __launch_bounds__(256) qimg_kernel(const float *__restrict__ Q, 
         img[(size_t)kb * (N1 * 32) + n * 32 + ((((kappa >> 2) ^ (n & 7)) << 2) | (kappa & 3))] = out;
     }
 }
-template <int LP, bool MASKED>
-__global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) absz_q_tc_kernel(const __grid_constant__ CUtensorMap tmap_z, int p, int q,
+// TRANS = false: Y = E Q    (output rows = rows of Z, contraction over its columns; the tensor map's box is 32 columns x 128 rows)
+// TRANS = true:  W = E^T Y  (output rows = columns of Z, contraction over its rows; box of 128 columns x 32 rows, and the
+//                            converters transpose while they write the K-major operand tiles)
+template <int LP, bool MASKED, bool TRANS>
+__global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) envelope_product_tc_kernel(const __grid_constant__ CUtensorMap tmap_z, int p, int q,
                                                                   const uint32_t *__restrict__ img, int kb_per_cta, float *__restrict__ P,
                                                                   const uint32_t *__restrict__ S, int nwords, int32_t *__restrict__ status) {
     using namespace tm;
@@ -259,8 +262,9 @@ __global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) absz_q_tc_
     const uint32_t full_bar = smem_u32(&bars[0]), empty_bar = smem_u32(&bars[TC_STAGES]);
     const uint32_t raw_full = smem_u32(&bars[2 * TC_STAGES]), raw_empty = smem_u32(&bars[2 * TC_STAGES + TC_RAW]);
     const uint32_t accum_bar = smem_u32(&bars[2 * TC_STAGES + 2 * TC_RAW]);
-    const int row0 = blockIdx.x * 128;
-    const int nkb_total = (q + TC_KB - 1) / TC_KB;
+    const int m_ext = TRANS ? q : p, k_ext = TRANS ? p : q;
+    const int row0 = blockIdx.x * 128;                           // first output row (a row of Z, or a column when TRANS)
+    const int nkb_total = (k_ext + TC_KB - 1) / TC_KB;
     const int kb0 = blockIdx.y * kb_per_cta;
     const int nkb = max(0, min(kb_per_cta, nkb_total - kb0));
     if (tid == 0) {
@@ -288,57 +292,103 @@ __global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) absz_q_tc_
     if (warp < TC_CONVERTERS / 32) {
         // ============================ converters, then epilogue ============================
         const int grp = warp >> 2;                               // K blocks grp, grp + 2, ...
-        const int rsub = (warp & 3) * 4 + (lane >> 3);           // rows rsub + 16 i, i = 0..7
-        const int chunk = lane & 7;
         bool alive = true;
-        uint32_t word[8];
+        if (!TRANS) {
+            const int rsub = (warp & 3) * 4 + (lane >> 3);       // rows rsub + 16 i, i = 0..7
+            const int chunk = lane & 7;
+            uint32_t word[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) word[i] = 0u;
-        if (MASKED && grp < nkb) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int gr = row0 + rsub + 16 * i;
-                if (gr < p) word[i] = S[(size_t)gr * nwords + kb0 + grp];
-            }
-        }
-        for (int kb = grp; kb < nkb && alive; kb += 2) {
-            const int s = kb % TC_STAGES, rs = kb % TC_RAW;
-            uint32_t word_next[8];
-            if (MASKED) {                                        // the next block's mask words travel while this one is converted
+            for (int i = 0; i < 8; ++i) word[i] = 0u;
+            if (MASKED && grp < nkb) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int gr = row0 + rsub + 16 * i;
-                    word_next[i] = (kb + 2 < nkb && gr < p) ? S[(size_t)gr * nwords + kb0 + kb + 2] : 0u;
+                    if (gr < p) word[i] = S[(size_t)gr * nwords + kb0 + grp];
                 }
             }
-            alive = mbar_wait(raw_full + 8 * rs, ((uint32_t)(kb / TC_RAW)) & 1u, abort_flag, status);
-            if (alive) alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(kb / TC_STAGES)) & 1u) ^ 1u, abort_flag, status);
-            alive = __all_sync(0xffffffffu, alive);
-            if (!alive) break;
-            const unsigned char *raw = smem_gen + (size_t)rs * TC_TILE;
-            unsigned char *stage = op_gen + (size_t)s * C::STAGE;
+            for (int kb = grp; kb < nkb && alive; kb += 2) {
+                const int s = kb % TC_STAGES, rs = kb % TC_RAW;
+                uint32_t word_next[8];
+                if (MASKED) {                                    // the next block's mask words travel while this one is converted
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int r = rsub + 16 * i;
-                const float4 v = *reinterpret_cast<const float4 *>(raw + r * 128 + chunk * 16);
-                const float in[4] = {v.x, v.y, v.z, v.w};
-                uint32_t h[4], l[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float e = MASKED ? __uint_as_float(__float_as_uint(in[j]) ^ (((word[i] >> (4 * chunk + j)) & 1u) << 31)) : fabsf(in[j]);
-                    h[j] = tf32_round(e);
-                    l[j] = tf32_round(e - __uint_as_float(h[j]));
+                    for (int i = 0; i < 8; ++i) {
+                        const int gr = row0 + rsub + 16 * i;
+                        word_next[i] = (kb + 2 < nkb && gr < p) ? S[(size_t)gr * nwords + kb0 + kb + 2] : 0u;
+                    }
                 }
-                const int off = r * 128 + ((chunk ^ (r & 7)) << 4);
-                *reinterpret_cast<uint4 *>(stage + off) = make_uint4(h[0], h[1], h[2], h[3]);
-                *reinterpret_cast<uint4 *>(stage + TC_TILE + off) = make_uint4(l[0], l[1], l[2], l[3]);
-            }
-            mbar_arrive(raw_empty + 8 * rs);
-            fence_proxy_async();
-            mbar_arrive(full_bar + 8 * s);
-            if (MASKED) {
+                alive = mbar_wait(raw_full + 8 * rs, ((uint32_t)(kb / TC_RAW)) & 1u, abort_flag, status);
+                if (alive) alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(kb / TC_STAGES)) & 1u) ^ 1u, abort_flag, status);
+                alive = __all_sync(0xffffffffu, alive);
+                if (!alive) break;
+                const unsigned char *raw = smem_gen + (size_t)rs * TC_TILE;
+                unsigned char *stage = op_gen + (size_t)s * C::STAGE;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) word[i] = word_next[i];
+                for (int i = 0; i < 8; ++i) {
+                    const int r = rsub + 16 * i;
+                    const float4 v = *reinterpret_cast<const float4 *>(raw + r * 128 + chunk * 16);
+                    const float in[4] = {v.x, v.y, v.z, v.w};
+                    uint32_t h[4], l[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float e = MASKED ? __uint_as_float(__float_as_uint(in[j]) ^ (((word[i] >> (4 * chunk + j)) & 1u) << 31)) : fabsf(in[j]);
+                        h[j] = tf32_round(e);
+                        l[j] = tf32_round(e - __uint_as_float(h[j]));
+                    }
+                    const int off = r * 128 + ((chunk ^ (r & 7)) << 4);
+                    *reinterpret_cast<uint4 *>(stage + off) = make_uint4(h[0], h[1], h[2], h[3]);
+                    *reinterpret_cast<uint4 *>(stage + TC_TILE + off) = make_uint4(l[0], l[1], l[2], l[3]);
+                }
+                mbar_arrive(raw_empty + 8 * rs);
+                fence_proxy_async();
+                mbar_arrive(full_bar + 8 * s);
+                if (MASKED) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) word[i] = word_next[i];
+                }
+            }
+        } else {
+            // thread = output row j (a column of Z); a warp's 32 columns are exactly one packed mask word per row of Z:
+            // lane i holds the word of the K block's row i, handed round by shuffles
+            const int j = tid & 127;
+            const int wcol = (row0 >> 5) + (warp & 3);           // the warp's word column
+            auto mask_word = [&](int kb) -> uint32_t {
+                const int gr = (kb0 + kb) * TC_KB + lane;
+                return (MASKED && kb < nkb && gr < p && wcol < nwords) ? S[(size_t)gr * nwords + wcol] : 0u;
+            };
+            uint32_t myword = mask_word(grp);
+            for (int kb = grp; kb < nkb && alive; kb += 2) {
+                const int s = kb % TC_STAGES, rs = kb % TC_RAW;
+                const uint32_t myword_next = mask_word(kb + 2);
+                alive = mbar_wait(raw_full + 8 * rs, ((uint32_t)(kb / TC_RAW)) & 1u, abort_flag, status);
+                if (alive) alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(kb / TC_STAGES)) & 1u) ^ 1u, abort_flag, status);
+                alive = __all_sync(0xffffffffu, alive);
+                if (!alive) break;
+                const float *raw = reinterpret_cast<const float *>(smem_gen + (size_t)rs * TC_TILE);     // [32 rows of Z][128 columns]
+                unsigned char *stage = op_gen + (size_t)s * C::STAGE;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t h[4], l[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const float in = raw[(4 * c + u) * 128 + j];
+                        float e;
+                        if (MASKED) {
+                            const uint32_t w = __shfl_sync(0xffffffffu, myword, 4 * c + u);
+                            e = __uint_as_float(__float_as_uint(in) ^ (((w >> lane) & 1u) << 31));
+                        } else {
+                            e = fabsf(in);
+                        }
+                        h[u] = tf32_round(e);
+                        l[u] = tf32_round(e - __uint_as_float(h[u]));
+                    }
+                    const int off = j * 128 + ((c ^ (j & 7)) << 4);
+                    *reinterpret_cast<uint4 *>(stage + off) = make_uint4(h[0], h[1], h[2], h[3]);
+                    *reinterpret_cast<uint4 *>(stage + TC_TILE + off) = make_uint4(l[0], l[1], l[2], l[3]);
+                }
+                mbar_arrive(raw_empty + 8 * rs);
+                fence_proxy_async();
+                mbar_arrive(full_bar + 8 * s);
+                myword = myword_next;
             }
         }
         if (warp < 4) {
@@ -360,8 +410,8 @@ __global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) absz_q_tc_
                     for (int e = 0; e < 16; ++e) y[(c16 * 16 + e) % LPP] += __uint_as_float(d[e]);      // columns t, LPP + t and N1 + t belong to mode t
                 }
             }
-            if (grow < p) {
-                float *out = P + ((size_t)blockIdx.y * p + grow) * LP;
+            if (grow < m_ext) {
+                float *out = P + ((size_t)blockIdx.y * m_ext + grow) * LP;
 #pragma unroll
                 for (int t = 0; t < LP; ++t) out[t] = alive ? y[t] : __int_as_float(0x7fc00000);
             }
@@ -399,7 +449,8 @@ __global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) absz_q_tc_
                 alive = mbar_wait(raw_empty + 8 * rs, (((uint32_t)(kb / TC_RAW)) & 1u) ^ 1u, abort_flag, status);
                 if (!alive) break;
                 mbar_arrive_expect_tx(raw_full + 8 * rs, (uint32_t)TC_TILE);
-                tma_load_2d(smem_base + (uint32_t)(rs * TC_TILE), &tmap_z, (kb0 + kb) * TC_KB, row0, raw_full + 8 * rs);
+                if (TRANS) tma_load_2d(smem_base + (uint32_t)(rs * TC_TILE), &tmap_z, row0, (kb0 + kb) * TC_KB, raw_full + 8 * rs);
+                else tma_load_2d(smem_base + (uint32_t)(rs * TC_TILE), &tmap_z, (kb0 + kb) * TC_KB, row0, raw_full + 8 * rs);
             }
         }
         __syncwarp();
@@ -714,9 +765,9 @@ static size_t carve(Scratch *w, char *base, int p, int q, int LP) {
     float *Q = (float *)take((size_t)q * LP * sizeof(float));
     float *Y = (float *)take((size_t)p * LP * sizeof(float));
     int kb_per_cta = 0;
-    const size_t tc_parts = (size_t)tc_split(p, q, LP, &kb_per_cta);
-    float *P = (float *)take(std::max(zy_chunks * q, tc_parts * p) * LP * sizeof(float));
-    uint32_t *img = (uint32_t *)take((size_t)ceil_div(q, TC_KB) * 2 * (LP < 16 ? 16 : LP) * 128);
+    const size_t tc_parts = (size_t)tc_split(p, q, LP, &kb_per_cta), tc_parts_t = (size_t)tc_split(q, p, LP, &kb_per_cta);
+    float *P = (float *)take(std::max(std::max(zy_chunks, tc_parts_t) * q, tc_parts * p) * LP * sizeof(float));
+    uint32_t *img = (uint32_t *)take((size_t)ceil_div(std::max(p, q), TC_KB) * 2 * (LP < 16 ? 16 : LP) * 128);
     int32_t *status = (int32_t *)take(sizeof(int32_t));
     double *Gp = (double *)take(gchunks * LP * LP * sizeof(double));
     double *Gs = (double *)take((size_t)LP * LP * sizeof(double));
@@ -743,8 +794,8 @@ static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st) {
     return MDBF_OK;
 }
 
-// Tensor map of the fp32 matrix Z [p][q]: box of 32 columns x 128 rows, no swizzle, zero fill outside the matrix.
-static mdbf_status_t make_z_tensor_map(CUtensorMap *out, const float *Z, int p, int q) {
+// Tensor map of the fp32 matrix Z [p][q]: box of box_cols columns x box_rows rows, no swizzle, zero fill outside the matrix.
+static mdbf_status_t make_z_tensor_map(CUtensorMap *out, const float *Z, int p, int q, int box_cols, int box_rows) {
     typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -761,7 +812,7 @@ static mdbf_status_t make_z_tensor_map(CUtensorMap *out, const float *Z, int p, 
     }
     const cuuint64_t gdim[2] = {(cuuint64_t)q, (cuuint64_t)p};
     const cuuint64_t gstride[1] = {(cuuint64_t)q * sizeof(float)};
-    const cuuint32_t box[2] = {(cuuint32_t)TC_KB, 128u};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(Z), gdim, gstride, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -774,26 +825,48 @@ static mdbf_status_t make_z_tensor_map(CUtensorMap *out, const float *Z, int p, 
 }
 static bool tc_eligible(const float *Z, int q) { return (q & 3) == 0 && (reinterpret_cast<uintptr_t>(Z) & 15u) == 0; }
 
-// Y = E Q with E the envelope of Z (|Z|, or Z with the given mask's signs taken off)
-template <int LP, bool MASKED>
-static mdbf_status_t product(const float *Z, int p, int q, const uint32_t *S, int nwords, const CUtensorMap *tmz, Scratch &w, cudaStream_t st) {
+struct ZMaps {
+    bool use;               // the tensor-core kernels run (else the scalar ones)
+    CUtensorMap rows;       // box of 32 columns x 128 rows, for Y = E Q
+    CUtensorMap cols;       // box of 128 columns x 32 rows, for W = E^T Y
+};
+// out = E in (TRANS = false: out has p rows, in has q) or E^T in (TRANS = true: out has q rows, in has p), E the envelope
+// of Z (|Z|, or Z with the given mask's signs taken off), on the tensor cores
+template <int LP, bool MASKED, bool TRANS>
+static mdbf_status_t tc_product(const ZMaps &zm, int p, int q, const float *in, float *out, const uint32_t *S, int nwords, Scratch &w,
+                                cudaStream_t st) {
     using C = TcCfg<LP>;
-    if (!tmz) {
-        absz_q_kernel<LP, MASKED><<<ceil_div(p, AQ_WARPS * AQ_ROWS), AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y, S, nwords);
-        MDBF_CUDA(cudaGetLastError());
-        return MDBF_OK;
-    }
     static bool attr_set = false;
     if (!attr_set) {
-        MDBF_CUDA(cudaFuncSetAttribute(absz_q_tc_kernel<LP, MASKED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM));
+        MDBF_CUDA(cudaFuncSetAttribute(envelope_product_tc_kernel<LP, MASKED, TRANS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM));
         attr_set = true;
     }
+    const int m_ext = TRANS ? q : p, k_ext = TRANS ? p : q;
     int kb_per_cta = 0;
-    const int parts = tc_split(p, q, LP, &kb_per_cta);
-    const int nkb = ceil_div(q, TC_KB);
-    qimg_kernel<LP><<<std::min(ceil_div(nkb * C::N1 * 32, 256), 148 * 8), 256, 0, st>>>(w.Q, q, nkb, w.img);
-    absz_q_tc_kernel<LP, MASKED><<<dim3(ceil_div(p, 128), parts), TC_THREADS, C::SMEM, st>>>(*tmz, p, q, w.img, kb_per_cta, w.P, S, nwords, w.status);
-    chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)p * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, parts, (size_t)p * LP, w.Y);
+    const int parts = tc_split(m_ext, k_ext, LP, &kb_per_cta);
+    const int nkb = ceil_div(k_ext, TC_KB);
+    qimg_kernel<LP><<<std::min(ceil_div(nkb * C::N1 * 32, 256), 148 * 8), 256, 0, st>>>(in, k_ext, nkb, w.img);
+    envelope_product_tc_kernel<LP, MASKED, TRANS><<<dim3(ceil_div(m_ext, 128), parts), TC_THREADS, C::SMEM, st>>>(
+        TRANS ? zm.cols : zm.rows, p, q, w.img, kb_per_cta, w.P, S, nwords, w.status);
+    chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)m_ext * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, parts, (size_t)m_ext * LP, out);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}
+// Y = E Q
+template <int LP, bool MASKED>
+static mdbf_status_t product(const float *Z, int p, int q, const uint32_t *S, int nwords, const ZMaps &zm, Scratch &w, cudaStream_t st) {
+    if (zm.use) return tc_product<LP, MASKED, false>(zm, p, q, w.Q, w.Y, S, nwords, w, st);
+    absz_q_kernel<LP, MASKED><<<ceil_div(p, AQ_WARPS * AQ_ROWS), AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y, S, nwords);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}
+// Q = E^T Y
+template <int LP, bool MASKED>
+static mdbf_status_t product_t(const float *Z, int p, int q, const uint32_t *S, int nwords, const ZMaps &zm, Scratch &w, cudaStream_t st) {
+    if (zm.use) return tc_product<LP, MASKED, true>(zm, p, q, w.Y, w.Q, S, nwords, w, st);
+    const int zy_chunks = ceil_div(p, ZY_ROWS);
+    abszT_y_kernel<LP, MASKED><<<dim3(ceil_div(q, ZY_COLS), zy_chunks), ZY_COLS, 0, st>>>(Z, p, q, w.Y, w.P, S, nwords);
+    chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, zy_chunks, (size_t)q * LP, w.Q);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
@@ -802,7 +875,6 @@ static mdbf_status_t product(const float *Z, int p, int q, const uint32_t *S, in
 template <int LP, bool MASKED>
 static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const float *Q0, uint32_t *S, float *U, float *V, float *sigma,
                          Scratch &w, cudaStream_t st) {
-    const int zy_chunks = ceil_div(p, ZY_ROWS);
     const int nwords = ceil_div(q, 32);
     if (!MASKED) sign_pack_kernel<<<dim3(p, ceil_div(nwords, 8 * SP_WORDS)), 256, 0, st>>>(Z, q, nwords, S);
     pad_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(Q0, (size_t)q, l, LP, w.Q);
@@ -810,27 +882,23 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
     mdbf_status_t rc = orth<LP>(w.Q, q, w, st);                        // twice: the start block may be badly conditioned
     if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st);
     if (rc) return rc;
-    const dim3 zy_grid(ceil_div(q, ZY_COLS), zy_chunks);
     MDBF_CUDA(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));
-    CUtensorMap tmap_z;
-    const CUtensorMap *tmz = nullptr;
-    if (tc_eligible(Z, q)) {
-        rc = make_z_tensor_map(&tmap_z, Z, p, q);
+    ZMaps zm;
+    zm.use = tc_eligible(Z, q);
+    if (zm.use) {
+        rc = make_z_tensor_map(&zm.rows, Z, p, q, TC_KB, 128);
+        if (rc == MDBF_OK) rc = make_z_tensor_map(&zm.cols, Z, p, q, 128, TC_KB);
         if (rc) return rc;
-        tmz = &tmap_z;
     }
     for (int it = 0; it < n_iter; ++it) {
-        rc = product<LP, MASKED>(Z, p, q, S, nwords, tmz, w, st);
+        rc = product<LP, MASKED>(Z, p, q, S, nwords, zm, w, st);
         if (rc == MDBF_OK) rc = orth<LP>(w.Y, p, w, st);
-        if (rc) return rc;
-        abszT_y_kernel<LP, MASKED><<<zy_grid, ZY_COLS, 0, st>>>(Z, p, q, w.Y, w.P, S, nwords);
-        chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, zy_chunks, (size_t)q * LP, w.Q);
-        MDBF_CUDA(cudaGetLastError());
-        rc = orth<LP>(w.Q, q, w, st);
+        if (rc == MDBF_OK) rc = product_t<LP, MASKED>(Z, p, q, S, nwords, zm, w, st);
+        if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st);
         if (rc == MDBF_OK && it == n_iter - 1) rc = orth<LP>(w.Q, q, w, st);   // the last block carries the result: orthonormal to fp32
         if (rc) return rc;
     }
-    rc = product<LP, MASKED>(Z, p, q, S, nwords, tmz, w, st);
+    rc = product<LP, MASKED>(Z, p, q, S, nwords, zm, w, st);
     if (rc) return rc;
     const int ychunks = ceil_div(p, GR_ROWS);
     gram_kernel<LP><<<ychunks, 256, 0, st>>>(w.Y, p, w.Gp);
