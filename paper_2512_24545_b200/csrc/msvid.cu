@@ -169,48 +169,58 @@ __global__ void __launch_bounds__(AQ_WARPS * 32) absz_q_kernel(const float *__re
         }
 }
 
-// ------------------------------------------------------------------ Y = |Z| Q on the tensor cores
-// The same product as absz_q_kernel with tcgen05 (kind::tf32, fp32 accumulators in tensor memory) and a three-term
-// split that keeps fp32 accuracy:  e = e_hi + e_lo,  q = q_hi + q_lo  (each part a TF32 number),
-//     e q  ~  e_hi q_hi + e_hi q_lo + e_lo q_hi                      (the dropped e_lo q_lo is below 2^-22 e q).
-// CTA = 128 rows x a range of K blocks of 32 columns (split over blockIdx.y, partial sums per range).  Per K block:
-//   one lane brings the raw 128 x 32 tile of Z into a ring of TC_RAW buffers by TMA (zero fill outside the matrix), so the
+// ------------------------------------------------------------------ Y = |Z| Q and W = |Z|^T Y on the tensor cores
+// The two products of the subspace iteration with tcgen05 (kind::tf32, fp32 accumulators in tensor memory) and a
+// three-term split that keeps fp32 accuracy:  e = e_hi + e_lo,  q = q_hi + q_lo  (each part a TF32 number),
+//     e q  ~  e_hi q_hi + e_hi q_lo + e_lo q_hi                      (the dropped e_lo q_lo is below 2^-21 e q).
+// CTA = 128 output rows x a range of K blocks of 32 (split over blockIdx.y, partial sums per range).  Per K block:
+//   one lane brings the raw 128 x 32 tile of Z into a ring of buffers by TMA (zero fill outside the matrix), so the
 //     bytes in flight do not depend on how many threads wait for them;
-//   8 converter warps (two groups on alternate K blocks; a quarter warp = one row's 128 bytes, so every shared-memory
-//     access touches each bank once) take the envelope (absolute value, or the sign flipped by the mask word - a K block
-//     is exactly one packed word), split it and write the operand tiles E_hi, E_lo (128 x 32 TF32, K-major, 128B swizzle);
-//   one lane bulk-copies the K block's image of Q: rows [0, LPP) = q_hi, [LPP, 2 LPP) = q_lo of the 32 columns,
-//     already in the operand layout (qimg_kernel builds the images once per pass);
+//   8 converter warps (two groups on alternate K blocks, thread = output row = TMEM lane) read their row of the tile,
+//     take the envelope (absolute value, or the sign flipped by the given mask), split it and store E_hi and E_lo
+//     straight into tensor memory as the A operand: shared memory carries each byte of Z once in and once out,
+//     where operand tiles in shared memory would carry it six times and bound the kernel;
+//   one lane bulk-copies the K block's image of the other factor: rows [0, LPP) = q_hi, [LPP, 2 LPP) = q_lo of the 32
+//     contraction indices, already in the K-major 128B-swizzled operand layout (qimg_kernel builds the images once per pass);
 //   two lanes issue the MMAs, four K steps of 8 each: D1 (+)= E_hi [q_hi | q_lo] (N = 2 LPP), D2 (+)= E_lo q_hi (N = LPP).
-// Epilogue: thread = row = TMEM lane: y[t] = D1[t] + D1[LPP + t] + D2[t] into the range's partial sums.
-// Needs cols % 4 == 0 and Z on a 16-byte boundary (the tensor map's rules); other inputs take absz_q_kernel.
+// Epilogue: y[t] = D1[t] + D1[LPP + t] + D2[t] into the range's partial sums.
+// TRANS = false: Y = E Q    (output rows = rows of Z, contraction over its columns; TMA box of 32 columns x 128 rows,
+//                            128B-swizzled so that a thread's 16-byte reads of its own row spread over the banks)
+// TRANS = true:  W = E^T Y  (output rows = columns of Z, contraction over its rows; box of 128 columns x 32 rows)
+// Needs cols % 4 == 0 and Z on a 16-byte boundary (the tensor map's rules); other inputs take the scalar kernels.
 // Every wait is bounded; on expiry the status word of the workspace is set and the call's outputs are NaN.
 constexpr int TC_KB = 32, TC_CONVERTERS = 256;
 constexpr int TC_W_ISSUE = 8, TC_W_RAW = 10, TC_W_IMG = 11, TC_THREADS = 12 * 32;
-constexpr int TC_TILE = 128 * TC_KB * 4;                        // bytes of a raw tile and of each operand tile
+constexpr int TC_TILE = 128 * TC_KB * 4;                        // bytes of a raw tile
+constexpr int TC_RAW = 5;                                       // raw tiles in flight per CTA
 template <int LP> struct TcCfg {
     static constexpr int LPP = LP < 16 ? 16 : LP;              // MMA N is a multiple of 16
     static constexpr int N1 = 2 * LPP, N2 = LPP;
-    static constexpr int IMG = N1 * 128;                        // bytes of one K block's image of Q
-    static constexpr int STAGE = 2 * TC_TILE + IMG;             // E_hi, E_lo, image
-    static constexpr int TMEM_COLS = N1 + N2 <= 64 ? 64 : 128;
-    // two CTAs per SM where their shared memory fits side by side (one's prologue and epilogue under the other's stream)
-    static constexpr int CTAS_PER_SM = LP <= 16 ? 2 : 1;
-    static constexpr int RAW = CTAS_PER_SM == 2 ? 2 : 4;       // raw tiles in flight per CTA
-    static constexpr int STAGES = CTAS_PER_SM == 2 ? 2 : 3;    // operand stages
-    static constexpr size_t SMEM = 1024 + (size_t)RAW * TC_TILE + (size_t)STAGES * STAGE;
+    static constexpr int IMG = N1 * 128;                        // bytes of one K block's image of the other factor
+    static constexpr int ACC_COLS = N1 + N2 <= 64 ? 64 : 128;   // tensor memory: accumulators, then the A stages of 64 columns
+    static constexpr int STAGES = (256 - ACC_COLS) / 64;        // two CTAs share the SM's 512 columns
+    static constexpr int TMEM_COLS = 256;
+    static constexpr size_t SMEM = 1024 + (size_t)TC_RAW * TC_TILE + (size_t)STAGES * IMG;
 };
 __device__ __forceinline__ uint32_t tf32_round(float x) {
     uint32_t r;
     asm("cvt.rna.tf32.f32 %0, %1;\n" : "=r"(r) : "f"(x));
     return r;
 }
-__device__ __forceinline__ void umma_ss_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+// e = hi + lo with hi the TF32 truncation of e (the residual is then exact in fp32) and lo the residual rounded to
+// nearest TF32 by an integer half-ulp add: plain ALU work (the cvt instruction runs on the quarter-rate pipe).
+// |e - hi - lo| <= 2^-22 |e|.
+__device__ __forceinline__ void tf32_split(float e, uint32_t &hi, uint32_t &lo) {
+    hi = __float_as_uint(e) & 0xFFFFE000u;
+    lo = (__float_as_uint(e - __uint_as_float(hi)) + 0x1000u) & 0xFFFFE000u;
+}
+// D[tmem] (+)= A[tmem] * B[smem], TF32 operands
+__device__ __forceinline__ void umma_ts_tf32(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}\n"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 // instruction descriptor: fp32 accumulator, A and B TF32, both K-major, M = 128
 __device__ __forceinline__ uint32_t make_idesc_tf32(int n) {
@@ -222,7 +232,7 @@ __device__ __forceinline__ uint32_t make_idesc_tf32(int n) {
     d |= (uint32_t)(128 >> 4) << 24;    // M
     return d;
 }
-// images of Q for one pass: K block kb holds rows n of 32 TF32 values, 128 bytes each, 128B swizzle
+// images of a tall factor F (n x LP) for one pass: K block kb holds rows r of 32 TF32 values, 128 bytes each, 128B swizzle
 template <int LP>
 __global__ void __launch_bounds__(256) qimg_kernel(const float *__restrict__ Q, int q, int nkb, uint32_t *__restrict__ img) {
     constexpr int LPP = TcCfg<LP>::LPP, N1 = TcCfg<LP>::N1;
@@ -239,16 +249,13 @@ __global__ void __launch_bounds__(256) qimg_kernel(const float *__restrict__ Q, 
         img[(size_t)kb * (N1 * 32) + n * 32 + ((((kappa >> 2) ^ (n & 7)) << 2) | (kappa & 3))] = out;
     }
 }
-// TRANS = false: Y = E Q    (output rows = rows of Z, contraction over its columns; the tensor map's box is 32 columns x 128 rows)
-// TRANS = true:  W = E^T Y  (output rows = columns of Z, contraction over its rows; box of 128 columns x 32 rows, and the
-//                            converters transpose while they write the K-major operand tiles)
 template <int LP, bool MASKED, bool TRANS>
-__global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) envelope_product_tc_kernel(const __grid_constant__ CUtensorMap tmap_z, int p, int q,
+__global__ void __launch_bounds__(TC_THREADS, 2) envelope_product_tc_kernel(const __grid_constant__ CUtensorMap tmap_z, int p, int q,
                                                                   const uint32_t *__restrict__ img, int kb_per_cta, float *__restrict__ P,
                                                                   const uint32_t *__restrict__ S, int nwords, int32_t *__restrict__ status) {
     using namespace tm;
     using C = TcCfg<LP>;
-    constexpr int LPP = C::LPP, N1 = C::N1, N2 = C::N2, TC_RAW = C::RAW, TC_STAGES = C::STAGES;
+    constexpr int LPP = C::LPP, N1 = C::N1, N2 = C::N2, TC_STAGES = C::STAGES;
     extern __shared__ unsigned char tc_smem_raw[];
     __shared__ __align__(8) uint64_t bars[2 * TC_STAGES + 2 * TC_RAW + 1];
     __shared__ uint32_t tmem_base_slot;
@@ -257,8 +264,7 @@ __global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) envelope_p
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
     unsigned char *smem_gen = tc_smem_raw + (smem_base - smem_u32(tc_smem_raw));
-    const uint32_t op_base = smem_base + (uint32_t)(TC_RAW * TC_TILE);
-    unsigned char *op_gen = smem_gen + TC_RAW * TC_TILE;
+    const uint32_t img_base = smem_base + (uint32_t)(TC_RAW * TC_TILE);
     const uint32_t full_bar = smem_u32(&bars[0]), empty_bar = smem_u32(&bars[TC_STAGES]);
     const uint32_t raw_full = smem_u32(&bars[2 * TC_STAGES]), raw_empty = smem_u32(&bars[2 * TC_STAGES + TC_RAW]);
     const uint32_t accum_bar = smem_u32(&bars[2 * TC_STAGES + 2 * TC_RAW]);
@@ -269,12 +275,12 @@ __global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) envelope_p
     const int nkb = max(0, min(kb_per_cta, nkb_total - kb0));
     if (tid == 0) {
         for (int s = 0; s < TC_STAGES; ++s) {
-            mbar_init(full_bar + 8 * s, 128 + 1);                // a converter group + the image's expect_tx
+            mbar_init(full_bar + 8 * s, 4 + 1);                  // the four warps of a converter group + the image's expect_tx
             mbar_init(empty_bar + 8 * s, 2);                     // the two issuing lanes (commits)
         }
         for (int s = 0; s < TC_RAW; ++s) {
             mbar_init(raw_full + 8 * s, 1);                      // the tile's expect_tx
-            mbar_init(raw_empty + 8 * s, 128);                   // the converter group that read it
+            mbar_init(raw_empty + 8 * s, 4);                     // the four warps of the group that read it
         }
         mbar_init(accum_bar, 2);
         abort_flag_s = 0;
@@ -288,115 +294,71 @@ __global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) envelope_p
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
+    const uint32_t tmem_a0 = tmem + (uint32_t)C::ACC_COLS;       // A stage s: columns [64 s, 64 s + 32) = E_hi, the next 32 = E_lo
 
     if (warp < TC_CONVERTERS / 32) {
         // ============================ converters, then epilogue ============================
         const int grp = warp >> 2;                               // K blocks grp, grp + 2, ...
-        bool alive = true;
-        if (!TRANS) {
-            const int rsub = (warp & 3) * 4 + (lane >> 3);       // rows rsub + 16 i, i = 0..7
-            const int chunk = lane & 7;
-            uint32_t word[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) word[i] = 0u;
-            if (MASKED && grp < nkb) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int gr = row0 + rsub + 16 * i;
-                    if (gr < p) word[i] = S[(size_t)gr * nwords + kb0 + grp];
-                }
-            }
-            for (int kb = grp; kb < nkb && alive; kb += 2) {
-                const int s = kb % TC_STAGES, rs = kb % TC_RAW;
-                uint32_t word_next[8];
-                if (MASKED) {                                    // the next block's mask words travel while this one is converted
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int gr = row0 + rsub + 16 * i;
-                        word_next[i] = (kb + 2 < nkb && gr < p) ? S[(size_t)gr * nwords + kb0 + kb + 2] : 0u;
-                    }
-                }
-                alive = mbar_wait(raw_full + 8 * rs, ((uint32_t)(kb / TC_RAW)) & 1u, abort_flag, status);
-                if (alive) alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(kb / TC_STAGES)) & 1u) ^ 1u, abort_flag, status);
-                alive = __all_sync(0xffffffffu, alive);
-                if (!alive) break;
-                const unsigned char *raw = smem_gen + (size_t)rs * TC_TILE;
-                unsigned char *stage = op_gen + (size_t)s * C::STAGE;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int r = rsub + 16 * i;
-                    const float4 v = *reinterpret_cast<const float4 *>(raw + r * 128 + chunk * 16);
-                    const float in[4] = {v.x, v.y, v.z, v.w};
-                    uint32_t h[4], l[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float e = MASKED ? __uint_as_float(__float_as_uint(in[j]) ^ (((word[i] >> (4 * chunk + j)) & 1u) << 31)) : fabsf(in[j]);
-                        h[j] = tf32_round(e);
-                        l[j] = tf32_round(e - __uint_as_float(h[j]));
-                    }
-                    const int off = r * 128 + ((chunk ^ (r & 7)) << 4);
-                    *reinterpret_cast<uint4 *>(stage + off) = make_uint4(h[0], h[1], h[2], h[3]);
-                    *reinterpret_cast<uint4 *>(stage + TC_TILE + off) = make_uint4(l[0], l[1], l[2], l[3]);
-                }
-                mbar_arrive(raw_empty + 8 * rs);
-                fence_proxy_async();
-                mbar_arrive(full_bar + 8 * s);
-                if (MASKED) {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) word[i] = word_next[i];
-                }
-            }
-        } else {
-            // thread = output row j (a column of Z); a warp's 32 columns are exactly one packed mask word per row of Z:
-            // lane i holds the word of the K block's row i, handed round by shuffles
-            const int j = tid & 127;
-            const int wcol = (row0 >> 5) + (warp & 3);           // the warp's word column
-            auto mask_word = [&](int kb) -> uint32_t {
+        const int r = (warp & 3) * 32 + lane;                    // output row within the tile = TMEM lane
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const int wcol = (row0 >> 5) + (warp & 3);               // TRANS: the warp's 32 columns are one packed word per row of Z
+        // mask word(s) of K block kb: a thread's own row and the block's word (plain), or lane i = the block's row i (TRANS)
+        auto mask_word = [&](int kb) -> uint32_t {
+            if (!MASKED || kb >= nkb) return 0u;
+            if (TRANS) {
                 const int gr = (kb0 + kb) * TC_KB + lane;
-                return (MASKED && kb < nkb && gr < p && wcol < nwords) ? S[(size_t)gr * nwords + wcol] : 0u;
-            };
-            uint32_t myword = mask_word(grp);
-            for (int kb = grp; kb < nkb && alive; kb += 2) {
-                const int s = kb % TC_STAGES, rs = kb % TC_RAW;
-                const uint32_t myword_next = mask_word(kb + 2);
-                alive = mbar_wait(raw_full + 8 * rs, ((uint32_t)(kb / TC_RAW)) & 1u, abort_flag, status);
-                if (alive) alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(kb / TC_STAGES)) & 1u) ^ 1u, abort_flag, status);
-                alive = __all_sync(0xffffffffu, alive);
-                if (!alive) break;
-                const float *raw = reinterpret_cast<const float *>(smem_gen + (size_t)rs * TC_TILE);     // [32 rows of Z][128 columns]
-                unsigned char *stage = op_gen + (size_t)s * C::STAGE;
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    uint32_t h[4], l[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const float in = raw[(4 * c + u) * 128 + j];
-                        float e;
-                        if (MASKED) {
-                            const uint32_t w = __shfl_sync(0xffffffffu, myword, 4 * c + u);
-                            e = __uint_as_float(__float_as_uint(in) ^ (((w >> lane) & 1u) << 31));
-                        } else {
-                            e = fabsf(in);
-                        }
-                        h[u] = tf32_round(e);
-                        l[u] = tf32_round(e - __uint_as_float(h[u]));
-                    }
-                    const int off = j * 128 + ((c ^ (j & 7)) << 4);
-                    *reinterpret_cast<uint4 *>(stage + off) = make_uint4(h[0], h[1], h[2], h[3]);
-                    *reinterpret_cast<uint4 *>(stage + TC_TILE + off) = make_uint4(l[0], l[1], l[2], l[3]);
-                }
-                mbar_arrive(raw_empty + 8 * rs);
-                fence_proxy_async();
-                mbar_arrive(full_bar + 8 * s);
-                myword = myword_next;
+                return (gr < p && wcol < nwords) ? S[(size_t)gr * nwords + wcol] : 0u;
             }
+            return row0 + r < p ? S[(size_t)(row0 + r) * nwords + kb0 + kb] : 0u;
+        };
+        bool alive = true;
+        uint32_t word = mask_word(grp);
+        for (int kb = grp; kb < nkb && alive; kb += 2) {
+            const int s = kb % TC_STAGES, rs = kb % TC_RAW;
+            const uint32_t word_next = mask_word(kb + 2);        // travels while this block is converted
+            alive = mbar_wait(raw_full + 8 * rs, ((uint32_t)(kb / TC_RAW)) & 1u, abort_flag, status);
+            if (alive) alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(kb / TC_STAGES)) & 1u) ^ 1u, abort_flag, status);
+            alive = __all_sync(0xffffffffu, alive);
+            if (!alive) break;
+            tc_fence_after();
+            const unsigned char *raw = smem_gen + (size_t)rs * TC_TILE;
+            const uint32_t a_col = tmem_a0 + lane_base + (uint32_t)(s * 64);
+#pragma unroll
+            for (int c8 = 0; c8 < 4; ++c8) {                     // 8 contraction indices at a time
+                float in[8];
+                if (!TRANS) {                                    // chunk c of row r sits at position c ^ (r & 7)
+                    const float4 v0 = *reinterpret_cast<const float4 *>(raw + r * 128 + (((2 * c8) ^ (r & 7)) << 4));
+                    const float4 v1 = *reinterpret_cast<const float4 *>(raw + r * 128 + (((2 * c8 + 1) ^ (r & 7)) << 4));
+                    in[0] = v0.x; in[1] = v0.y; in[2] = v0.z; in[3] = v0.w; in[4] = v1.x; in[5] = v1.y; in[6] = v1.z; in[7] = v1.w;
+                } else {                                         // [32 rows of Z][128 columns]
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) in[u] = reinterpret_cast<const float *>(raw)[(8 * c8 + u) * 128 + r];
+                }
+                uint32_t h[8], l[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    float e;
+                    if (!MASKED) e = fabsf(in[u]);
+                    else if (!TRANS) e = __uint_as_float(__float_as_uint(in[u]) ^ (((word >> (8 * c8 + u)) & 1u) << 31));
+                    else e = __uint_as_float(__float_as_uint(in[u]) ^ (((__shfl_sync(0xffffffffu, word, 8 * c8 + u) >> lane) & 1u) << 31));
+                    tf32_split(e, h[u], l[u]);
+                }
+                tmem_st8(a_col + (uint32_t)(8 * c8), h);
+                tmem_st8(a_col + (uint32_t)(32 + 8 * c8), l);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(raw_empty + 8 * rs);
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full_bar + 8 * s);
+            word = word_next;
         }
         if (warp < 4) {
-            const int grow = row0 + tid;
+            const int grow = row0 + r;
             if (alive) alive = mbar_wait(accum_bar, 0u, abort_flag, status);
             alive = __all_sync(0xffffffffu, alive);
             tc_fence_after();
-            const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
             float y[LPP];
 #pragma unroll
             for (int t = 0; t < LPP; ++t) y[t] = 0.f;
@@ -428,13 +390,12 @@ __global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) envelope_p
                 alive = mbar_wait(full_bar + 8 * s, ((uint32_t)(kb / TC_STAGES)) & 1u, abort_flag, status);
                 if (!alive) break;
                 tc_fence_after();
-                const uint32_t stage = op_base + (uint32_t)(s * C::STAGE);
-                const uint64_t adesc = make_smem_desc(stage + (first ? 0u : (uint32_t)TC_TILE));
-                const uint64_t bdesc = make_smem_desc(stage + 2u * TC_TILE);
+                const uint32_t a_t = tmem_a0 + (uint32_t)(s * 64) + (first ? 0u : 32u);
+                const uint64_t bdesc = make_smem_desc(img_base + (uint32_t)(s * C::IMG));
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)                   // 8 TF32 = 32 bytes per K step
-                    umma_ss_tf32(d_tmem, adesc + (uint64_t)(2 * ks), bdesc + (uint64_t)(2 * ks), idesc, (kb > 0 || ks > 0) ? 1u : 0u);
-                umma_commit(empty_bar + 8 * s);
+                for (int ks = 0; ks < 4; ++ks)                   // 8 TF32 per K step: 8 TMEM columns of A, 32 bytes of B
+                    umma_ts_tf32(d_tmem, a_t + (uint32_t)(8 * ks), bdesc + (uint64_t)(2 * ks), idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+                umma_commit(empty_bar + 8 * s);                  // frees the A stage and the image together
             }
             if (alive && nkb > 0) umma_commit(accum_bar);
             else mbar_arrive(accum_bar);
@@ -463,7 +424,7 @@ __global__ void __launch_bounds__(TC_THREADS, TcCfg<LP>::CTAS_PER_SM) envelope_p
                 alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(kb / TC_STAGES)) & 1u) ^ 1u, abort_flag, status);
                 if (!alive) break;
                 mbar_arrive_expect_tx(full_bar + 8 * s, (uint32_t)C::IMG);
-                bulk_load(op_base + (uint32_t)(s * C::STAGE) + 2u * TC_TILE, img + (size_t)(kb0 + kb) * (C::IMG / 4), (uint32_t)C::IMG, full_bar + 8 * s);
+                bulk_load(img_base + (uint32_t)(s * C::IMG), img + (size_t)(kb0 + kb) * (C::IMG / 4), (uint32_t)C::IMG, full_bar + 8 * s);
             }
         }
         __syncwarp();
@@ -744,7 +705,8 @@ struct Scratch {
 // how the K blocks of the tensor-core product are split over blockIdx.y: the split that fills whole waves of resident CTAs best,
 // each CTA keeping at least 8 K blocks
 static int tc_split(int p, int q, int LP, int *kb_per_cta) {
-    const int slots = 148 * (LP <= 16 ? 2 : 1);
+    const int slots = 148 * 2;                                   // two CTAs per SM
+    (void)LP;
     const int rb = ceil_div(p, 128), nkb = ceil_div(q, TC_KB);
     int best = 1;
     double best_eff = -1.0;
@@ -794,8 +756,8 @@ static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st) {
     return MDBF_OK;
 }
 
-// Tensor map of the fp32 matrix Z [p][q]: box of box_cols columns x box_rows rows, no swizzle, zero fill outside the matrix.
-static mdbf_status_t make_z_tensor_map(CUtensorMap *out, const float *Z, int p, int q, int box_cols, int box_rows) {
+// Tensor map of the fp32 matrix Z [p][q]: box of box_cols columns x box_rows rows, zero fill outside the matrix.
+static mdbf_status_t make_z_tensor_map(CUtensorMap *out, const float *Z, int p, int q, int box_cols, int box_rows, bool swizzle128) {
     typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -815,7 +777,7 @@ static mdbf_status_t make_z_tensor_map(CUtensorMap *out, const float *Z, int p, 
     const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(Z), gdim, gstride, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         set_error("cuTensorMapEncodeTiled (Z) failed with CUresult %d", (int)r);
@@ -827,7 +789,7 @@ static bool tc_eligible(const float *Z, int q) { return (q & 3) == 0 && (reinter
 
 struct ZMaps {
     bool use;               // the tensor-core kernels run (else the scalar ones)
-    CUtensorMap rows;       // box of 32 columns x 128 rows, for Y = E Q
+    CUtensorMap rows;       // box of 32 columns x 128 rows, 128B swizzle, for Y = E Q
     CUtensorMap cols;       // box of 128 columns x 32 rows, for W = E^T Y
 };
 // out = E in (TRANS = false: out has p rows, in has q) or E^T in (TRANS = true: out has q rows, in has p), E the envelope
@@ -863,7 +825,7 @@ static mdbf_status_t product(const float *Z, int p, int q, const uint32_t *S, in
 // Q = E^T Y
 template <int LP, bool MASKED>
 static mdbf_status_t product_t(const float *Z, int p, int q, const uint32_t *S, int nwords, const ZMaps &zm, Scratch &w, cudaStream_t st) {
-    if (zm.use) return tc_product<LP, MASKED, true>(zm, p, q, w.Y, w.Q, S, nwords, w, st);
+    if (zm.use && LP >= 8) return tc_product<LP, MASKED, true>(zm, p, q, w.Y, w.Q, S, nwords, w, st);   // narrower blocks: the scalar kernel runs at the memory rate already
     const int zy_chunks = ceil_div(p, ZY_ROWS);
     abszT_y_kernel<LP, MASKED><<<dim3(ceil_div(q, ZY_COLS), zy_chunks), ZY_COLS, 0, st>>>(Z, p, q, w.Y, w.P, S, nwords);
     chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, zy_chunks, (size_t)q * LP, w.Q);
@@ -886,8 +848,8 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
     ZMaps zm;
     zm.use = tc_eligible(Z, q);
     if (zm.use) {
-        rc = make_z_tensor_map(&zm.rows, Z, p, q, TC_KB, 128);
-        if (rc == MDBF_OK) rc = make_z_tensor_map(&zm.cols, Z, p, q, 128, TC_KB);
+        rc = make_z_tensor_map(&zm.rows, Z, p, q, TC_KB, 128, true);
+        if (rc == MDBF_OK) rc = make_z_tensor_map(&zm.cols, Z, p, q, 128, TC_KB, false);
         if (rc) return rc;
     }
     for (int it = 0; it < n_iter; ++it) {
