@@ -491,75 +491,137 @@ __global__ void chunk_sum_kernel(const float *__restrict__ P, int nchunks, size_
 }
 
 // ------------------------------------------------------------------ orth(): Cholesky QR, Gram matrix in fp64
-// partial Gram matrices of chunks of GR_ROWS rows of a tall matrix A (n x LP)
-constexpr int GR_ROWS = 64;
+// One warp, lane k = row k of G in registers: G = L L^T (G: the summed Gram matrix, lower triangle), then lane k = column k
+// of L^-1 by forward substitution; rows of L travel by shuffles.  M[b][a] = (L^-1)[a][b], so that A M has orthonormal
+// columns.  A zero (or numerically vanished) pivot - a padding column, or a block wider than the rank of the matrix -
+// leaves its column as it is instead of dividing by zero.
 template <int LP>
-__global__ void __launch_bounds__(256) gram_kernel(const float *__restrict__ A, int n, double *__restrict__ Gp) {
-    __shared__ float As[GR_ROWS][LP + 1];
-    const int i0 = blockIdx.x * GR_ROWS;
-    const int nrows = min(GR_ROWS, n - i0);
-    for (int e = threadIdx.x; e < GR_ROWS * LP; e += 256) {
-        const int i = e / LP, t = e - i * LP;
-        As[i][t] = i < nrows ? A[(size_t)(i0 + i) * LP + t] : 0.f;
-    }
-    __syncthreads();
-    for (int pr = threadIdx.x; pr < LP * LP; pr += 256) {
-        const int a = pr / LP, b = pr - a * LP;
-        double s = 0.0;
-        if (b <= a)
-            for (int i = 0; i < nrows; ++i) s += (double)As[i][a] * (double)As[i][b];
-        Gp[(size_t)blockIdx.x * LP * LP + pr] = s;
-    }
-}
-// The chunks' partial Gram matrices added up: one warp per entry, lanes stride over the chunks, then a fixed
-// shuffle tree (the order of the additions does not depend on scheduling).
-__global__ void __launch_bounds__(256) gram_sum_kernel(const double *__restrict__ Gp, int nchunks, int nentries, double *__restrict__ G) {
-    const int e = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-    if (e >= nentries) return;
-    double s = 0.0;
-    for (int c = lane; c < nchunks; c += 32) s += Gp[(size_t)c * nentries + e];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (lane == 0) G[e] = s;
-}
-// One warp, lane = row: G = L L^T (G: the summed Gram matrix, lower triangle); M[b][a] = (L^-1)[a][b], so that A M has
-// orthonormal columns.  A zero (or numerically vanished) pivot - a padding column, or a block wider than the rank of
-// the matrix - leaves its column as it is instead of dividing by zero.
-template <int LP>
-__global__ void __launch_bounds__(32) chol_kernel(const double *__restrict__ Gs, float *__restrict__ M) {
-    __shared__ double G[LP][LP + 1], Li[LP][LP + 1];
-    const int k = threadIdx.x;
-    for (int e = k; e < LP * LP; e += 32) {
-        G[e / LP][e % LP] = Gs[e];
-        Li[e / LP][e % LP] = 0.0;
-    }
-    __syncwarp();
+__device__ __forceinline__ void chol_warp(const double (*Gm)[LP + 1], float *__restrict__ M) {
+    const int k = threadIdx.x & 31;
+    double g[LP], invd[LP];
     double scale = 0.0;
-    for (int d = 0; d < LP; ++d) scale = fmax(scale, G[d][d]);
-    // column-by-column Cholesky on the lower triangle
+#pragma unroll
+    for (int j = 0; j < LP; ++j) {
+        g[j] = (k < LP && j <= k) ? Gm[k < LP ? k : 0][j] : 0.0;
+        scale = fmax(scale, Gm[j][j]);
+    }
+#pragma unroll
     for (int c = 0; c < LP; ++c) {
-        if (k == c) {
-            const double d = G[c][c];
-            G[c][c] = d > 1e-24 * scale && d > 0.0 ? sqrt(d) : 0.0;
+        const double dcc = __shfl_sync(0xffffffffu, g[c], c);
+        const double inv = (dcc > 1e-24 * scale && dcc > 0.0) ? rsqrt(dcc) : 0.0;
+        invd[c] = inv;                                           // 1 / L[c][c], the same in every lane
+        g[c] = k == c ? dcc * inv : g[c] * inv;                  // column c of L (zero above the diagonal)
+#pragma unroll
+        for (int jj = c + 1; jj < LP; ++jj) {
+            const double ljc = __shfl_sync(0xffffffffu, g[c], jj);
+            if (k >= jj) g[jj] -= g[c] * ljc;
         }
-        __syncwarp();
-        const double d = G[c][c];
-        if (k > c && k < LP) G[k][c] = d > 0.0 ? G[k][c] / d : 0.0;
-        __syncwarp();
-        if (k > c && k < LP)
-            for (int jj = c + 1; jj <= k; ++jj) G[k][jj] -= G[k][c] * G[jj][c];
-        __syncwarp();
     }
-    // inverse of the lower-triangular factor, one lane per column
+    double x[LP];
+#pragma unroll
+    for (int i = 0; i < LP; ++i) {
+        double sum = i == k ? 1.0 : 0.0;
+#pragma unroll
+        for (int m = 0; m < i; ++m) {
+            const double lim = __shfl_sync(0xffffffffu, g[m], i);     // L[i][m]
+            if (m >= k) sum -= lim * x[m];
+        }
+        x[i] = i >= k ? (invd[i] > 0.0 ? sum * invd[i] : (i == k ? 1.0 : 0.0)) : 0.0;
+    }
     if (k < LP) {
-        for (int i = k; i < LP; ++i) {
-            double sum = i == k ? 1.0 : 0.0;
-            for (int m = k; m < i; ++m) sum -= G[i][m] * Li[m][k];
-            Li[i][k] = G[i][i] > 0.0 ? sum / G[i][i] : (i == k ? 1.0 : 0.0);
+#pragma unroll
+        for (int a = 0; a < LP; ++a) M[k * LP + a] = (float)x[a];
+    }
+}
+// Gram matrix of a tall matrix A (n x LP) in fp64 and what follows it, in one launch.  The CTAs stride over chunks of
+// GR_ROWS rows: where `parts` > 0 a chunk's rows are first formed as the sum of their partial sums P[c] (c < parts, in
+// order) and written to A; every CTA keeps one partial Gram matrix (lower triangle) over its chunks.  The CTA that
+// finishes last adds the CTAs' matrices up in a fixed order and either factors the sum (CHOL: M for right_mul_kernel)
+// or leaves it in Gs for the eigensolver.
+constexpr int GR_ROWS = 128, GR_MAX_CTAS = 128;
+template <int LP, bool CHOL>
+__global__ void __launch_bounds__(256) gram_finish_kernel(float *__restrict__ A, int n, const float *__restrict__ P, int parts,
+                                                          double *__restrict__ Gp, unsigned int *__restrict__ counter,
+                                                          double *__restrict__ Gs, float *__restrict__ M) {
+    constexpr int PER = GR_ROWS * LP / 256 > 0 ? GR_ROWS * LP / 256 : 1;     // elements of a chunk per thread
+    constexpr int ENT = (LP * LP + 255) / 256;                                // Gram entries per thread
+    __shared__ float As[GR_ROWS][LP + 1];
+    __shared__ double Gm[LP][LP + 1];
+    __shared__ bool is_last;
+    double acc[ENT];
+#pragma unroll
+    for (int u = 0; u < ENT; ++u) acc[u] = 0.0;
+    const int nchunks = (n + GR_ROWS - 1) / GR_ROWS;
+    for (int chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+        const int i0 = chunk * GR_ROWS;
+        const size_t base = (size_t)i0 * LP, limit = (size_t)n * LP;
+        float v[PER];
+#pragma unroll
+        for (int u = 0; u < PER; ++u) v[u] = 0.f;
+        if (parts > 0) {
+#pragma unroll 4
+            for (int c = 0; c < parts; ++c)                       // independent loads, additions in the order of c
+#pragma unroll
+                for (int u = 0; u < PER; ++u) {
+                    const size_t at = base + threadIdx.x + 256 * u;
+                    if (threadIdx.x + 256 * u < GR_ROWS * LP && at < limit) v[u] += __ldcs(P + (size_t)c * limit + at);
+                }
+        } else {
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                const size_t at = base + threadIdx.x + 256 * u;
+                if (threadIdx.x + 256 * u < GR_ROWS * LP && at < limit) v[u] = A[at];
+            }
+        }
+        __syncthreads();                                         // the previous chunk's Gram pass has read As
+#pragma unroll
+        for (int u = 0; u < PER; ++u) {
+            const int e = threadIdx.x + 256 * u;
+            if (e < GR_ROWS * LP) {
+                const size_t at = base + e;
+                if (parts > 0 && at < limit) A[at] = v[u];
+                As[e / LP][e % LP] = v[u];                       // rows past the end are zero
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int u = 0; u < ENT; ++u) {
+            const int pr = threadIdx.x + 256 * u;
+            const int a = pr / LP, b = pr - a * LP;
+            if (pr < LP * LP && b <= a) {
+                double s0 = 0.0, s1 = 0.0;
+                for (int i = 0; i < GR_ROWS; i += 2) {
+                    s0 += (double)As[i][a] * (double)As[i][b];
+                    s1 += (double)As[i + 1][a] * (double)As[i + 1][b];
+                }
+                acc[u] += s0 + s1;
+            }
         }
     }
-    __syncwarp();
-    for (int e = k; e < LP * LP; e += 32) M[e] = (float)Li[e % LP][e / LP];      // M[a][b] = Li[b][a]
+#pragma unroll
+    for (int u = 0; u < ENT; ++u)
+        if (threadIdx.x + 256 * u < LP * LP) Gp[(size_t)blockIdx.x * LP * LP + threadIdx.x + 256 * u] = acc[u];
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = atomicAdd(counter, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    for (int pr = threadIdx.x; pr < LP * LP; pr += 256) {
+        double s[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll 4
+        for (int c = 0; c < (int)gridDim.x; c += 4)
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (c + u < (int)gridDim.x) s[u] += __ldcg(Gp + (size_t)(c + u) * LP * LP + pr);
+        const double total = (s[0] + s[1]) + (s[2] + s[3]);
+        if (CHOL) Gm[pr / LP][pr % LP] = total;
+        else Gs[pr] = total;
+    }
+    if (threadIdx.x == 0) *counter = 0u;                         // ready for the next launch on the stream
+    if (!CHOL) return;
+    __syncthreads();
+    if (threadIdx.x < 32) chol_warp<LP>(Gm, M);
 }
 // A <- A M, row by row (M is LP x LP, row-major)
 template <int LP>
@@ -701,6 +763,7 @@ struct Scratch {
     double *Gp, *Gs;
     uint32_t *img;          // operand images of Q for the tensor-core product
     int32_t *status;        // set by a wait that ran out
+    unsigned int *counter;  // CTAs of the Gram kernel that have finished (the word after the status word)
 };
 // how the K blocks of the tensor-core product are split over blockIdx.y: the split that fills whole waves of resident CTAs best,
 // each CTA keeping at least 8 K blocks
@@ -721,7 +784,7 @@ static int tc_split(int p, int q, int LP, int *kb_per_cta) {
 }
 static size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 static size_t carve(Scratch *w, char *base, int p, int q, int LP) {
-    const size_t zy_chunks = ceil_div(p, ZY_ROWS), gchunks = ceil_div(max(p, q), GR_ROWS);
+    const size_t zy_chunks = ceil_div(p, ZY_ROWS), gchunks = GR_MAX_CTAS;
     size_t off = 0;
     auto take = [&](size_t bytes) { char *ptr = base ? base + off : nullptr; off += align256(bytes); return ptr; };
     float *Q = (float *)take((size_t)q * LP * sizeof(float));
@@ -730,13 +793,13 @@ static size_t carve(Scratch *w, char *base, int p, int q, int LP) {
     const size_t tc_parts = (size_t)tc_split(p, q, LP, &kb_per_cta), tc_parts_t = (size_t)tc_split(q, p, LP, &kb_per_cta);
     float *P = (float *)take(std::max(std::max(zy_chunks, tc_parts_t) * q, tc_parts * p) * LP * sizeof(float));
     uint32_t *img = (uint32_t *)take((size_t)ceil_div(std::max(p, q), TC_KB) * 2 * (LP < 16 ? 16 : LP) * 128);
-    int32_t *status = (int32_t *)take(sizeof(int32_t));
+    int32_t *status = (int32_t *)take(2 * sizeof(int32_t));
     double *Gp = (double *)take(gchunks * LP * LP * sizeof(double));
     double *Gs = (double *)take((size_t)LP * LP * sizeof(double));
     float *M = (float *)take((size_t)LP * LP * sizeof(float));
     float *MU = (float *)take((size_t)LP * LP * sizeof(float));
     float *MV = (float *)take((size_t)LP * LP * sizeof(float));
-    if (w) { w->Q = Q; w->Y = Y; w->P = P; w->Gp = Gp; w->Gs = Gs; w->M = M; w->MU = MU; w->MV = MV; w->img = img; w->status = status; }
+    if (w) { w->Q = Q; w->Y = Y; w->P = P; w->Gp = Gp; w->Gs = Gs; w->M = M; w->MU = MU; w->MV = MV; w->img = img; w->status = status; w->counter = (unsigned int *)status + 1; }
     return off;
 }
 static int padded_rank(int l) {
@@ -745,12 +808,10 @@ static int padded_rank(int l) {
     return LP;
 }
 
+// A <- an orthonormal basis of its columns (Cholesky QR); with `parts` > 0, A is first formed as the sum of the partial sums in w.P
 template <int LP>
-static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st) {
-    const int chunks = ceil_div(n, GR_ROWS);
-    gram_kernel<LP><<<chunks, 256, 0, st>>>(A, n, w.Gp);
-    gram_sum_kernel<<<ceil_div(LP * LP, 8), 256, 0, st>>>(w.Gp, chunks, LP * LP, w.Gs);
-    chol_kernel<LP><<<1, 32, 0, st>>>(w.Gs, w.M);
+static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st, int parts = 0) {
+    gram_finish_kernel<LP, true><<<std::min(ceil_div(n, GR_ROWS), GR_MAX_CTAS), 256, 0, st>>>(A, n, w.P, parts, w.Gp, w.counter, w.Gs, w.M);
     right_mul_kernel<LP><<<ceil_div(n, 256), 256, 0, st>>>(A, n, w.M, nullptr, 0);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
@@ -792,11 +853,11 @@ struct ZMaps {
     CUtensorMap rows;       // box of 32 columns x 128 rows, 128B swizzle, for Y = E Q
     CUtensorMap cols;       // box of 128 columns x 32 rows, for W = E^T Y
 };
-// out = E in (TRANS = false: out has p rows, in has q) or E^T in (TRANS = true: out has q rows, in has p), E the envelope
-// of Z (|Z|, or Z with the given mask's signs taken off), on the tensor cores
+// E in (TRANS = false: p output rows, in has q) or E^T in (TRANS = true: q output rows, in has p), E the envelope of Z
+// (|Z|, or Z with the given mask's signs taken off), on the tensor cores; the result is left as *parts_out partial sums in w.P
 template <int LP, bool MASKED, bool TRANS>
-static mdbf_status_t tc_product(const ZMaps &zm, int p, int q, const float *in, float *out, const uint32_t *S, int nwords, Scratch &w,
-                                cudaStream_t st) {
+static mdbf_status_t tc_product(const ZMaps &zm, int p, int q, const float *in, const uint32_t *S, int nwords, Scratch &w,
+                                cudaStream_t st, int *parts_out) {
     using C = TcCfg<LP>;
     static bool attr_set = false;
     if (!attr_set) {
@@ -810,22 +871,26 @@ static mdbf_status_t tc_product(const ZMaps &zm, int p, int q, const float *in, 
     qimg_kernel<LP><<<std::min(ceil_div(nkb * C::N1 * 32, 256), 148 * 8), 256, 0, st>>>(in, k_ext, nkb, w.img);
     envelope_product_tc_kernel<LP, MASKED, TRANS><<<dim3(ceil_div(m_ext, 128), parts), TC_THREADS, C::SMEM, st>>>(
         TRANS ? zm.cols : zm.rows, p, q, w.img, kb_per_cta, w.P, S, nwords, w.status);
-    chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)m_ext * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, parts, (size_t)m_ext * LP, out);
+    *parts_out = parts;                                          // the Gram kernel that follows adds the partial sums up
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
 // Y = E Q
 template <int LP, bool MASKED>
-static mdbf_status_t product(const float *Z, int p, int q, const uint32_t *S, int nwords, const ZMaps &zm, Scratch &w, cudaStream_t st) {
-    if (zm.use) return tc_product<LP, MASKED, false>(zm, p, q, w.Q, w.Y, S, nwords, w, st);
+static mdbf_status_t product(const float *Z, int p, int q, const uint32_t *S, int nwords, const ZMaps &zm, Scratch &w, cudaStream_t st,
+                             int *parts) {
+    if (zm.use) return tc_product<LP, MASKED, false>(zm, p, q, w.Q, S, nwords, w, st, parts);
+    *parts = 0;                                                  // the scalar kernels write the whole result
     absz_q_kernel<LP, MASKED><<<ceil_div(p, AQ_WARPS * AQ_ROWS), AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y, S, nwords);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
 // Q = E^T Y
 template <int LP, bool MASKED>
-static mdbf_status_t product_t(const float *Z, int p, int q, const uint32_t *S, int nwords, const ZMaps &zm, Scratch &w, cudaStream_t st) {
-    if (zm.use && LP >= 8) return tc_product<LP, MASKED, true>(zm, p, q, w.Y, w.Q, S, nwords, w, st);   // narrower blocks: the scalar kernel runs at the memory rate already
+static mdbf_status_t product_t(const float *Z, int p, int q, const uint32_t *S, int nwords, const ZMaps &zm, Scratch &w, cudaStream_t st,
+                               int *parts) {
+    if (zm.use && LP >= 8) return tc_product<LP, MASKED, true>(zm, p, q, w.Y, S, nwords, w, st, parts);
+    *parts = 0;   // narrower blocks: the scalar kernel runs at the memory rate already
     const int zy_chunks = ceil_div(p, ZY_ROWS);
     abszT_y_kernel<LP, MASKED><<<dim3(ceil_div(q, ZY_COLS), zy_chunks), ZY_COLS, 0, st>>>(Z, p, q, w.Y, w.P, S, nwords);
     chunk_sum_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(w.P, zy_chunks, (size_t)q * LP, w.Q);
@@ -838,13 +903,14 @@ template <int LP, bool MASKED>
 static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const float *Q0, uint32_t *S, float *U, float *V, float *sigma,
                          Scratch &w, cudaStream_t st) {
     const int nwords = ceil_div(q, 32);
+    MDBF_CUDA(cudaMemsetAsync(w.status, 0, 2 * sizeof(int32_t), st));           // status word and the Gram kernel's counter
     if (!MASKED) sign_pack_kernel<<<dim3(p, ceil_div(nwords, 8 * SP_WORDS)), 256, 0, st>>>(Z, q, nwords, S);
     pad_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(Q0, (size_t)q, l, LP, w.Q);
     MDBF_CUDA(cudaGetLastError());
     mdbf_status_t rc = orth<LP>(w.Q, q, w, st);                        // twice: the start block may be badly conditioned
     if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st);
     if (rc) return rc;
-    MDBF_CUDA(cudaMemsetAsync(w.status, 0, sizeof(int32_t), st));
+    int parts = 0;
     ZMaps zm;
     zm.use = tc_eligible(Z, q);
     if (zm.use) {
@@ -853,18 +919,16 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
         if (rc) return rc;
     }
     for (int it = 0; it < n_iter; ++it) {
-        rc = product<LP, MASKED>(Z, p, q, S, nwords, zm, w, st);
-        if (rc == MDBF_OK) rc = orth<LP>(w.Y, p, w, st);
-        if (rc == MDBF_OK) rc = product_t<LP, MASKED>(Z, p, q, S, nwords, zm, w, st);
-        if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st);
+        rc = product<LP, MASKED>(Z, p, q, S, nwords, zm, w, st, &parts);
+        if (rc == MDBF_OK) rc = orth<LP>(w.Y, p, w, st, parts);
+        if (rc == MDBF_OK) rc = product_t<LP, MASKED>(Z, p, q, S, nwords, zm, w, st, &parts);
+        if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st, parts);
         if (rc == MDBF_OK && it == n_iter - 1) rc = orth<LP>(w.Q, q, w, st);   // the last block carries the result: orthonormal to fp32
         if (rc) return rc;
     }
-    rc = product<LP, MASKED>(Z, p, q, S, nwords, zm, w, st);
+    rc = product<LP, MASKED>(Z, p, q, S, nwords, zm, w, st, &parts);
     if (rc) return rc;
-    const int ychunks = ceil_div(p, GR_ROWS);
-    gram_kernel<LP><<<ychunks, 256, 0, st>>>(w.Y, p, w.Gp);
-    gram_sum_kernel<<<ceil_div(LP * LP, 8), 256, 0, st>>>(w.Gp, ychunks, LP * LP, w.Gs);
+    gram_finish_kernel<LP, false><<<std::min(ceil_div(p, GR_ROWS), GR_MAX_CTAS), 256, 0, st>>>(w.Y, p, w.P, parts, w.Gp, w.counter, w.Gs, w.M);
     jacobi_kernel<LP><<<1, 32, 0, st>>>(w.Gs, 1, l, sigma, w.MU, w.MV);
     right_mul_kernel<LP><<<ceil_div(p, 256), 256, 0, st>>>(w.Y, p, w.MU, U, l);
     right_mul_kernel<LP><<<ceil_div(q, 256), 256, 0, st>>>(w.Q, q, w.MV, V, l);
