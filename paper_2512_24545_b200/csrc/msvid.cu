@@ -249,10 +249,15 @@ __global__ void __launch_bounds__(256) qimg_kernel(const float *__restrict__ Q, 
         img[(size_t)kb * (N1 * 32) + n * 32 + ((((kappa >> 2) ^ (n & 7)) << 2) | (kappa & 3))] = out;
     }
 }
-template <int LP, bool MASKED, bool TRANS>
+// WRITE_MASK (plain product of |Z| only): the converters also pack the signs of what they read into S_out, the mask of
+// Eq. msvid-def (bit = 1 where the entry is below zero; zeros of either sign count as +1), so that the first pass over Z
+// yields it for free.
+template <int LP, bool MASKED, bool TRANS, bool WRITE_MASK>
 __global__ void __launch_bounds__(TC_THREADS, 2) envelope_product_tc_kernel(const __grid_constant__ CUtensorMap tmap_z, int p, int q,
                                                                   const uint32_t *__restrict__ img, int kb_per_cta, float *__restrict__ P,
-                                                                  const uint32_t *__restrict__ S, int nwords, int32_t *__restrict__ status) {
+                                                                  const uint32_t *__restrict__ S, uint32_t *__restrict__ S_out, int nwords,
+                                                                  int32_t *__restrict__ status) {
+    static_assert(!WRITE_MASK || (!MASKED && !TRANS), "the mask is written by the plain product of |Z|");
     using namespace tm;
     using C = TcCfg<LP>;
     constexpr int LPP = C::LPP, N1 = C::N1, N2 = C::N2, TC_STAGES = C::STAGES;
@@ -323,6 +328,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) envelope_product_tc_kernel(cons
             tc_fence_after();
             const unsigned char *raw = smem_gen + (size_t)rs * TC_TILE;
             const uint32_t a_col = tmem_a0 + lane_base + (uint32_t)(s * 64);
+            uint32_t signs = 0u;
 #pragma unroll
             for (int c8 = 0; c8 < 4; ++c8) {                     // 8 contraction indices at a time
                 float in[8];
@@ -338,6 +344,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) envelope_product_tc_kernel(cons
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     float e;
+                    if (WRITE_MASK) signs |= (in[u] < 0.f ? 1u : 0u) << (8 * c8 + u);
                     if (!MASKED) e = fabsf(in[u]);
                     else if (!TRANS) e = __uint_as_float(__float_as_uint(in[u]) ^ (((word >> (8 * c8 + u)) & 1u) << 31));
                     else e = __uint_as_float(__float_as_uint(in[u]) ^ (((__shfl_sync(0xffffffffu, word, 8 * c8 + u) >> lane) & 1u) << 31));
@@ -346,6 +353,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) envelope_product_tc_kernel(cons
                 tmem_st8(a_col + (uint32_t)(8 * c8), h);
                 tmem_st8(a_col + (uint32_t)(32 + 8 * c8), l);
             }
+            if (WRITE_MASK && row0 + r < p) S_out[(size_t)(row0 + r) * nwords + kb0 + kb] = signs;
             __syncwarp();
             if (lane == 0) mbar_arrive(raw_empty + 8 * rs);
             tmem_st_wait();
@@ -648,103 +656,106 @@ __global__ void __launch_bounds__(256) right_mul_kernel(float *__restrict__ A, i
 }
 
 // ------------------------------------------------------------------ the small eigenproblem
-// One warp, lane k = row / column k: Jacobi on G = Y^T Y (l x l, fp64), eigenvalues sorted in descending order;
+// One CTA: Jacobi on G = Y^T Y (l x l, fp64, given as its lower triangle), eigenvalues sorted in descending order;
 // writes the singular values s_t = sqrt(lambda_t) and the two LP x LP matrices that turn (Y, Q) into the balanced
 // factors: MU[b][t] = W[b][t] s_t^-1/2, MV[b][t] = W[b][t] s_t^1/2 (zero columns beyond l and for vanished values).
+// Round-robin ordering: n - 1 rounds of n / 2 rotations on disjoint index pairs (n = l rounded up to even; a pair with
+// the dummy index is skipped).  Thread i < n / 2 works out the rotation of pair i; then thread (k, i) applies rotation
+// i to row k (columns p, q of G and of W), and after a barrier to column k (rows p, q of G).  The tangent is taken in
+// fp32 (any angle near the optimal one converges; fp64 division and square roots were most of a round), the cosine
+// and sine from it in fp64, so that every rotation is orthogonal to fp64 rounding.
+constexpr int JAC_THREADS = 256;
 template <int LP>
-__global__ void __launch_bounds__(32) jacobi_kernel(const double *__restrict__ Gp, int nchunks, int l, float *__restrict__ sigma,
-                                                    float *__restrict__ MU, float *__restrict__ MV) {
+__global__ void __launch_bounds__(JAC_THREADS) jacobi_kernel(const double *__restrict__ Gs, int l, float *__restrict__ sigma,
+                                                             float *__restrict__ MU, float *__restrict__ MV) {
     __shared__ double G[LP][LP + 1], W[LP][LP + 1], rc[LP], rs[LP];
     __shared__ int order[LP], rp[LP], rq[LP];
-    const int k = threadIdx.x;
-    for (int e = k; e < LP * LP; e += 32) {
+    __shared__ int done;
+    const int tid = threadIdx.x;
+    for (int e = tid; e < LP * LP; e += JAC_THREADS) {
         const int a = e / LP, b = e - a * LP;
-        double s = 0.0;
-        const int lo = b <= a ? a * LP + b : b * LP + a;          // the partial sums hold the lower triangle
-#pragma unroll 8
-        for (int c = 0; c < nchunks; ++c) s += Gp[(size_t)c * LP * LP + lo];
-        G[a][b] = s;
+        G[a][b] = Gs[b <= a ? a * LP + b : b * LP + a];
         W[a][b] = a == b ? 1.0 : 0.0;
     }
-    __syncwarp();
-    // Round-robin ordering: n - 1 rounds of n / 2 rotations on disjoint index pairs (n = l rounded up to even; a pair
-    // with the dummy index is skipped).  Lane i works out the rotation of pair i; then every lane applies all of the
-    // round's rotations to its row (columns p, q of G and of W), then to its column (rows p, q of G).
-    const int n = (l + 1) & ~1;
+    const int n = (l + 1) & ~1, half = n / 2;
     for (int sweep = 0; sweep < 30 && n >= 2; ++sweep) {
-        double off = 0.0, diag = 0.0;
-        if (k < l) {
-            diag = G[k][k] * G[k][k];
-            for (int b = 0; b < k; ++b) off += G[k][b] * G[k][b];
-        }
+        __syncthreads();
+        if (tid < 32) {
+            double off = 0.0, diag = 0.0;
+            for (int k = tid; k < l; k += 32) {
+                diag += G[k][k] * G[k][k];
+                for (int b = 0; b < k; ++b) off += G[k][b] * G[k][b];
+            }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            off += __shfl_xor_sync(0xffffffffu, off, o);
-            diag += __shfl_xor_sync(0xffffffffu, diag, o);
+            for (int o = 16; o > 0; o >>= 1) {
+                off += __shfl_xor_sync(0xffffffffu, off, o);
+                diag += __shfl_xor_sync(0xffffffffu, diag, o);
+            }
+            if (tid == 0) done = off <= 1e-20 * diag;            // off-diagonal mass below 1e-10 of the diagonal's: the eigenvalues are
+                                                                 // then accurate to the square of that
         }
-        if (off <= 1e-20 * diag) break;                          // off-diagonal mass below 1e-10 of the diagonal's: the eigenvalues are then
-                                                                 // accurate to the square of that
+        __syncthreads();
+        if (done) break;
         for (int r = 0; r < n - 1; ++r) {
-            if (k < n / 2) {
-                const int a = k == 0 ? n - 1 : (r + k) % (n - 1), b = k == 0 ? r : (r - k + (n - 1)) % (n - 1);
+            if (tid < half) {
+                const int a = tid == 0 ? n - 1 : (r + tid) % (n - 1), b = tid == 0 ? r : (r - tid + (n - 1)) % (n - 1);
                 const int pi = min(a, b), qi = max(a, b);
                 double c = 1.0, sn = 0.0;
                 if (qi < l) {
                     const double apq = G[pi][qi];
                     if (apq != 0.0) {
-                        const double theta = (G[qi][qi] - G[pi][pi]) / (2.0 * apq);
-                        const double t = (theta >= 0.0 ? 1.0 : -1.0) / (fabs(theta) + sqrt(theta * theta + 1.0));
-                        c = 1.0 / sqrt(t * t + 1.0);
+                        const float theta = (float)((G[qi][qi] - G[pi][pi]) / (2.0 * apq));
+                        const double t = (double)((theta >= 0.f ? 1.f : -1.f) / (fabsf(theta) + sqrtf(theta * theta + 1.f)));
+                        c = rsqrt(t * t + 1.0);
                         sn = t * c;
                     }
                 }
-                rp[k] = pi; rq[k] = qi; rc[k] = c; rs[k] = sn;
+                rp[tid] = pi; rq[tid] = qi; rc[tid] = c; rs[tid] = sn;
             }
-            __syncwarp();
-            if (k < l)
-                for (int i = 0; i < n / 2; ++i) {
-                    const double c = rc[i], sn = rs[i];
-                    if (sn == 0.0) continue;
-                    const int pi = rp[i], qi = rq[i];
-                    const double gkp = G[k][pi], gkq = G[k][qi];
-                    G[k][pi] = c * gkp - sn * gkq;
-                    G[k][qi] = sn * gkp + c * gkq;
-                    const double wkp = W[k][pi], wkq = W[k][qi];
-                    W[k][pi] = c * wkp - sn * wkq;
-                    W[k][qi] = sn * wkp + c * wkq;
-                }
-            __syncwarp();
-            if (k < l)
-                for (int i = 0; i < n / 2; ++i) {
-                    const double c = rc[i], sn = rs[i];
-                    if (sn == 0.0) continue;
-                    const int pi = rp[i], qi = rq[i];
-                    const double gpk = G[pi][k], gqk = G[qi][k];
-                    G[pi][k] = c * gpk - sn * gqk;
-                    G[qi][k] = sn * gpk + c * gqk;
-                }
-            __syncwarp();
+            __syncthreads();
+            for (int idx = tid; idx < l * half; idx += JAC_THREADS) {
+                const int k = idx / half, i = idx - k * half;
+                const double c = rc[i], sn = rs[i];
+                if (sn == 0.0) continue;
+                const int pi = rp[i], qi = rq[i];
+                const double gkp = G[k][pi], gkq = G[k][qi];
+                G[k][pi] = c * gkp - sn * gkq;
+                G[k][qi] = sn * gkp + c * gkq;
+                const double wkp = W[k][pi], wkq = W[k][qi];
+                W[k][pi] = c * wkp - sn * wkq;
+                W[k][qi] = sn * wkp + c * wkq;
+            }
+            __syncthreads();
+            for (int idx = tid; idx < l * half; idx += JAC_THREADS) {
+                const int k = idx / half, i = idx - k * half;
+                const double c = rc[i], sn = rs[i];
+                if (sn == 0.0) continue;
+                const int pi = rp[i], qi = rq[i];
+                const double gpk = G[pi][k], gqk = G[qi][k];
+                G[pi][k] = c * gpk - sn * gqk;
+                G[qi][k] = sn * gpk + c * gqk;
+            }
+            __syncthreads();
         }
     }
-    __syncwarp();
-    if (k == 0) {
+    __syncthreads();
+    if (tid == 0) {
         for (int t = 0; t < l; ++t) order[t] = t;
         for (int t = 0; t < l; ++t)                    // selection sort, descending eigenvalues
             for (int u = t + 1; u < l; ++u)
                 if (G[order[u]][order[u]] > G[order[t]][order[t]]) { const int x = order[t]; order[t] = order[u]; order[u] = x; }
     }
-    __syncwarp();
+    __syncthreads();
     const double top = l > 0 ? fmax(G[order[0]][order[0]], 0.0) : 0.0;
-    for (int t = 0; t < LP; ++t) {
+    for (int e = tid; e < LP * LP; e += JAC_THREADS) {
+        const int k = e / LP, t = e - k * LP;
         double lam = t < l ? G[order[t]][order[t]] : 0.0;
         if (!(lam > 1e-24 * top)) lam = 0.0;
-        const double sv = sqrt(lam), rs = sqrt(sv);
+        const double sv = sqrt(lam), rsv = sqrt(sv);
         if (k == 0 && t < l) sigma[t] = (float)sv;
-        if (k < LP) {
-            const double w = (t < l && k < l) ? W[k][order[t]] : 0.0;
-            MU[k * LP + t] = (float)(rs > 0.0 ? w / rs : 0.0);
-            MV[k * LP + t] = (float)(w * rs);
-        }
+        const double w = (t < l && k < l) ? W[k][order[t]] : 0.0;
+        MU[k * LP + t] = (float)(rsv > 0.0 ? w / rsv : 0.0);
+        MV[k * LP + t] = (float)(w * rsv);
     }
 }
 
@@ -855,13 +866,13 @@ struct ZMaps {
 };
 // E in (TRANS = false: p output rows, in has q) or E^T in (TRANS = true: q output rows, in has p), E the envelope of Z
 // (|Z|, or Z with the given mask's signs taken off), on the tensor cores; the result is left as *parts_out partial sums in w.P
-template <int LP, bool MASKED, bool TRANS>
+template <int LP, bool MASKED, bool TRANS, bool WRITE_MASK = false>
 static mdbf_status_t tc_product(const ZMaps &zm, int p, int q, const float *in, const uint32_t *S, int nwords, Scratch &w,
-                                cudaStream_t st, int *parts_out) {
+                                cudaStream_t st, int *parts_out, uint32_t *S_out = nullptr) {
     using C = TcCfg<LP>;
     static bool attr_set = false;
     if (!attr_set) {
-        MDBF_CUDA(cudaFuncSetAttribute(envelope_product_tc_kernel<LP, MASKED, TRANS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM));
+        MDBF_CUDA(cudaFuncSetAttribute(envelope_product_tc_kernel<LP, MASKED, TRANS, WRITE_MASK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM));
         attr_set = true;
     }
     const int m_ext = TRANS ? q : p, k_ext = TRANS ? p : q;
@@ -869,8 +880,8 @@ static mdbf_status_t tc_product(const ZMaps &zm, int p, int q, const float *in, 
     const int parts = tc_split(m_ext, k_ext, LP, &kb_per_cta);
     const int nkb = ceil_div(k_ext, TC_KB);
     qimg_kernel<LP><<<std::min(ceil_div(nkb * C::N1 * 32, 256), 148 * 8), 256, 0, st>>>(in, k_ext, nkb, w.img);
-    envelope_product_tc_kernel<LP, MASKED, TRANS><<<dim3(ceil_div(m_ext, 128), parts), TC_THREADS, C::SMEM, st>>>(
-        TRANS ? zm.cols : zm.rows, p, q, w.img, kb_per_cta, w.P, S, nwords, w.status);
+    envelope_product_tc_kernel<LP, MASKED, TRANS, WRITE_MASK><<<dim3(ceil_div(m_ext, 128), parts), TC_THREADS, C::SMEM, st>>>(
+        TRANS ? zm.cols : zm.rows, p, q, w.img, kb_per_cta, w.P, S, S_out, nwords, w.status);
     *parts_out = parts;                                          // the Gram kernel that follows adds the partial sums up
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
@@ -878,8 +889,12 @@ static mdbf_status_t tc_product(const ZMaps &zm, int p, int q, const float *in, 
 // Y = E Q
 template <int LP, bool MASKED>
 static mdbf_status_t product(const float *Z, int p, int q, const uint32_t *S, int nwords, const ZMaps &zm, Scratch &w, cudaStream_t st,
-                             int *parts) {
-    if (zm.use) return tc_product<LP, MASKED, false>(zm, p, q, w.Q, S, nwords, w, st, parts);
+                             int *parts, uint32_t *S_out = nullptr) {
+    if (zm.use) {
+        if constexpr (!MASKED)
+            if (S_out) return tc_product<LP, false, false, true>(zm, p, q, w.Q, S, nwords, w, st, parts, S_out);
+        return tc_product<LP, MASKED, false>(zm, p, q, w.Q, S, nwords, w, st, parts);
+    }
     *parts = 0;                                                  // the scalar kernels write the whole result
     absz_q_kernel<LP, MASKED><<<ceil_div(p, AQ_WARPS * AQ_ROWS), AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y, S, nwords);
     MDBF_CUDA(cudaGetLastError());
@@ -904,22 +919,23 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
                          Scratch &w, cudaStream_t st) {
     const int nwords = ceil_div(q, 32);
     MDBF_CUDA(cudaMemsetAsync(w.status, 0, 2 * sizeof(int32_t), st));           // status word and the Gram kernel's counter
-    if (!MASKED) sign_pack_kernel<<<dim3(p, ceil_div(nwords, 8 * SP_WORDS)), 256, 0, st>>>(Z, q, nwords, S);
+    ZMaps zm;
+    zm.use = tc_eligible(Z, q);
+    if (zm.use) {
+        mdbf_status_t rcm = make_z_tensor_map(&zm.rows, Z, p, q, TC_KB, 128, true);
+        if (rcm == MDBF_OK) rcm = make_z_tensor_map(&zm.cols, Z, p, q, 128, TC_KB, false);
+        if (rcm) return rcm;
+    }
+    // the mask of Z itself: packed by the first tensor-core pass over Z, else by a pass of its own
+    if (!MASKED && !zm.use) sign_pack_kernel<<<dim3(p, ceil_div(nwords, 8 * SP_WORDS)), 256, 0, st>>>(Z, q, nwords, S);
     pad_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(Q0, (size_t)q, l, LP, w.Q);
     MDBF_CUDA(cudaGetLastError());
     mdbf_status_t rc = orth<LP>(w.Q, q, w, st);                        // twice: the start block may be badly conditioned
     if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st);
     if (rc) return rc;
     int parts = 0;
-    ZMaps zm;
-    zm.use = tc_eligible(Z, q);
-    if (zm.use) {
-        rc = make_z_tensor_map(&zm.rows, Z, p, q, TC_KB, 128, true);
-        if (rc == MDBF_OK) rc = make_z_tensor_map(&zm.cols, Z, p, q, 128, TC_KB, false);
-        if (rc) return rc;
-    }
     for (int it = 0; it < n_iter; ++it) {
-        rc = product<LP, MASKED>(Z, p, q, S, nwords, zm, w, st, &parts);
+        rc = product<LP, MASKED>(Z, p, q, S, nwords, zm, w, st, &parts, (!MASKED && it == 0) ? S : nullptr);
         if (rc == MDBF_OK) rc = orth<LP>(w.Y, p, w, st, parts);
         if (rc == MDBF_OK) rc = product_t<LP, MASKED>(Z, p, q, S, nwords, zm, w, st, &parts);
         if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st, parts);
@@ -929,7 +945,7 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
     rc = product<LP, MASKED>(Z, p, q, S, nwords, zm, w, st, &parts);
     if (rc) return rc;
     gram_finish_kernel<LP, false><<<std::min(ceil_div(p, GR_ROWS), GR_MAX_CTAS), 256, 0, st>>>(w.Y, p, w.P, parts, w.Gp, w.counter, w.Gs, w.M);
-    jacobi_kernel<LP><<<1, 32, 0, st>>>(w.Gs, 1, l, sigma, w.MU, w.MV);
+    jacobi_kernel<LP><<<1, JAC_THREADS, 0, st>>>(w.Gs, l, sigma, w.MU, w.MV);
     right_mul_kernel<LP><<<ceil_div(p, 256), 256, 0, st>>>(w.Y, p, w.MU, U, l);
     right_mul_kernel<LP><<<ceil_div(q, 256), 256, 0, st>>>(w.Q, q, w.MV, V, l);
     MDBF_CUDA(cudaGetLastError());
