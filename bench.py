@@ -451,8 +451,8 @@ def measure(workload, kernel, steps, warmup, dist, world, local, no_graph=False,
 # ------------------------------------------------------------ quantizer, first step (MSVID)
 def measure_msvid(workload, steps, warmup, dist, world, local, want_e2e=True, min_timed_ms=0.0):
     """msvid_<rows>x<cols>_l<l>[_it<n>]: one step = one mdbf_msvid call on a resident rows x cols fp32 matrix (sign mask +
-    rank-l envelope, n subspace iterations).  Algorithmic bytes: the sign pass and the 2 n + 1 product passes each
-    read Z once (rows * cols * 4 bytes; |Z| is never stored), plus the mask and the factors written."""
+    rank-l envelope, n subspace iterations).  Algorithmic bytes: the 2 n + 1 product passes each read Z once (rows * cols * 4
+    bytes; |Z| is never stored, and the sign mask comes out of the first pass), plus the mask and the factors written."""
     import re
     import torch
     from paper_2512_24545_b200 import inputs, mdbf as M, replicas
@@ -475,7 +475,7 @@ def measure_msvid(workload, steps, warmup, dist, world, local, want_e2e=True, mi
     Sh, Uh, Vh = (torch.zeros_like(t, device="cpu").pin_memory() for t in (Sd, Ud, Vd))
     ws_bytes = M.mdbf_msvid_workspace_bytes(rows, cols, l)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
-    passes = 2 * n_iter + 2
+    passes = 2 * n_iter + 1
     step_bytes = passes * rows * cols * 4 + rows * nwords * 4 + (rows + cols) * l * 4
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda") if rows * cols * 4 < 2 * 126e6 else None
 
@@ -549,7 +549,7 @@ def measure_msvid(workload, steps, warmup, dist, world, local, want_e2e=True, mi
 
 def cpu_baseline_msvid(rows, cols, l, n_iter):
     """The oracle's MSVID (sign mask + full SVD of |Z|, fp64) on a leading block of the workload's matrix, rated in the
-    algorithmic bytes the GPU arm's call counts for the same elements (sign pass + 2 n + 1 product passes)."""
+    algorithmic bytes the GPU arm's call counts for the same elements (2 n + 1 passes)."""
     from oracle import mdbf_oracle as orc
     from paper_2512_24545_b200 import inputs
     Z = inputs.make_factor_matrix(min(rows, 2048), min(cols, 4096), seed=8)
@@ -557,7 +557,7 @@ def cpu_baseline_msvid(rows, cols, l, n_iter):
     orc.msvid(Z, l)
     dt = time.perf_counter() - t0
     cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
-    return {"value": (2 * n_iter + 2) * Z.size * 4 / 1e9 / dt, "unit": "GB/s", "cores": cores, "kind": "oracle",
+    return {"value": (2 * n_iter + 1) * Z.size * 4 / 1e9 / dt, "unit": "GB/s", "cores": cores, "kind": "oracle",
             "sample": f"fp64 sign mask + full SVD of a {Z.shape[0]} x {Z.shape[1]} block of the workload's matrix, one call, {dt:.1f} s"}
 
 
@@ -657,7 +657,7 @@ def run_reference(args):
     cores = len(os.sched_getaffinity(0))
     if args.workload.startswith("msvid"):
         # the oracle's MSVID (sign mask + full SVD, fp64) on a leading block of the workload's matrix per step; the metric
-        # counts the same algorithmic bytes per element of Z as the GPU arm's call (sign pass + 2 n + 1 product passes)
+        # counts the same algorithmic bytes per element of Z as the GPU arm's call (2 n + 1 passes)
         import re
         from oracle import mdbf_oracle as orc
         from paper_2512_24545_b200 import inputs
@@ -674,7 +674,7 @@ def run_reference(args):
         for _ in range(args.steps):
             orc.msvid(Z, l)
         total = time.perf_counter() - t0
-        value = (2 * n_iter + 2) * Z.size * 4 / 1e9 * args.steps / total
+        value = (2 * n_iter + 1) * Z.size * 4 / 1e9 * args.steps / total
         sample = f"fp64 sign mask + full SVD of a {sub_r} x {sub_c} block of the workload's matrix per step"
         print(json.dumps({
             "impl": "reference", "metric": "msvid_algorithmic_GBps", "value": value, "unit": "GB/s",

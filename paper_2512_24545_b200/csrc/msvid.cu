@@ -553,7 +553,7 @@ __global__ void __launch_bounds__(256) gram_finish_kernel(float *__restrict__ A,
                                                           double *__restrict__ Gs, float *__restrict__ M) {
     constexpr int PER = GR_ROWS * LP / 256 > 0 ? GR_ROWS * LP / 256 : 1;     // elements of a chunk per thread
     constexpr int ENT = (LP * LP + 255) / 256;                                // Gram entries per thread
-    __shared__ float As[GR_ROWS][LP + 1];
+    __shared__ double As[GR_ROWS][LP + 1];                       // converted once on the way in, not once per product
     __shared__ double Gm[LP][LP + 1];
     __shared__ bool is_last;
     double acc[ENT];
@@ -588,7 +588,7 @@ __global__ void __launch_bounds__(256) gram_finish_kernel(float *__restrict__ A,
             if (e < GR_ROWS * LP) {
                 const size_t at = base + e;
                 if (parts > 0 && at < limit) A[at] = v[u];
-                As[e / LP][e % LP] = v[u];                       // rows past the end are zero
+                As[e / LP][e % LP] = (double)v[u];               // rows past the end are zero
             }
         }
         __syncthreads();
@@ -599,8 +599,8 @@ __global__ void __launch_bounds__(256) gram_finish_kernel(float *__restrict__ A,
             if (pr < LP * LP && b <= a) {
                 double s0 = 0.0, s1 = 0.0;
                 for (int i = 0; i < GR_ROWS; i += 2) {
-                    s0 += (double)As[i][a] * (double)As[i][b];
-                    s1 += (double)As[i + 1][a] * (double)As[i + 1][b];
+                    s0 += As[i][a] * As[i][b];
+                    s1 += As[i + 1][a] * As[i + 1][b];
                 }
                 acc[u] += s0 + s1;
             }
@@ -704,7 +704,7 @@ __global__ void __launch_bounds__(JAC_THREADS) jacobi_kernel(const double *__res
                 if (qi < l) {
                     const double apq = G[pi][qi];
                     if (apq != 0.0) {
-                        const float theta = (float)((G[qi][qi] - G[pi][pi]) / (2.0 * apq));
+                        const float theta = (float)(G[qi][qi] - G[pi][pi]) / (2.f * (float)apq);
                         const double t = (double)((theta >= 0.f ? 1.f : -1.f) / (fabsf(theta) + sqrtf(theta * theta + 1.f)));
                         c = rsqrt(t * t + 1.0);
                         sn = t * c;
