@@ -274,9 +274,18 @@ __global__ void __launch_bounds__(TC_THREADS, 2) envelope_product_tc_kernel(cons
     const uint32_t raw_full = smem_u32(&bars[2 * TC_STAGES]), raw_empty = smem_u32(&bars[2 * TC_STAGES + TC_RAW]);
     const uint32_t accum_bar = smem_u32(&bars[2 * TC_STAGES + 2 * TC_RAW]);
     const int m_ext = TRANS ? q : p, k_ext = TRANS ? p : q;
-    const int row0 = blockIdx.x * 128;                           // first output row (a row of Z, or a column when TRANS)
+    // Order of the CTAs over Z, so that a pass starts on what the pass before it read last and finds part of it in L2:
+    // W = E^T Y walks the row ranges from the top down (x = column block fastest, y = row range); Y = E Q then walks the
+    // row blocks from the bottom up, all column ranges of a row block together.
+    int bx = blockIdx.x, by = blockIdx.y;
+    if (!TRANS) {
+        const int lin = blockIdx.x + gridDim.x * blockIdx.y;
+        by = lin % gridDim.y;
+        bx = gridDim.x - 1 - lin / gridDim.y;
+    }
+    const int row0 = bx * 128;                                   // first output row (a row of Z, or a column when TRANS)
     const int nkb_total = (k_ext + TC_KB - 1) / TC_KB;
-    const int kb0 = blockIdx.y * kb_per_cta;
+    const int kb0 = by * kb_per_cta;
     const int nkb = max(0, min(kb_per_cta, nkb_total - kb0));
     if (tid == 0) {
         for (int s = 0; s < TC_STAGES; ++s) {
@@ -381,7 +390,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) envelope_product_tc_kernel(cons
                 }
             }
             if (grow < m_ext) {
-                float *out = P + ((size_t)blockIdx.y * m_ext + grow) * LP;
+                float *out = P + ((size_t)by * m_ext + grow) * LP;
 #pragma unroll
                 for (int t = 0; t < LP; ++t) out[t] = alive ? y[t] : __int_as_float(0x7fc00000);
             }
@@ -631,22 +640,35 @@ __global__ void __launch_bounds__(256) gram_finish_kernel(float *__restrict__ A,
     __syncthreads();
     if (threadIdx.x < 32) chol_warp<LP>(Gm, M);
 }
-// A <- A M, row by row (M is LP x LP, row-major)
+// A <- A M, row by row (M is LP x LP, row-major).  With `img`, the rows' operand images for the tensor-core product that
+// reads A next are written on the way out (the layout qimg_kernel documents; rows past the end are zero).
 template <int LP>
 __global__ void __launch_bounds__(256) right_mul_kernel(float *__restrict__ A, int n, const float *__restrict__ M, float *__restrict__ out,
-                                                        int out_cols) {
+                                                        int out_cols, uint32_t *__restrict__ img) {
     __shared__ float Ms[LP][LP];
     for (int e = threadIdx.x; e < LP * LP; e += 256) Ms[e / LP][e % LP] = M[e];
     __syncthreads();
     const int i = blockIdx.x * 256 + threadIdx.x;
-    if (i >= n) return;
     float a[LP], o[LP];
 #pragma unroll
-    for (int t = 0; t < LP; ++t) { a[t] = A[(size_t)i * LP + t]; o[t] = 0.f; }
+    for (int t = 0; t < LP; ++t) { a[t] = i < n ? A[(size_t)i * LP + t] : 0.f; o[t] = 0.f; }
 #pragma unroll
     for (int b = 0; b < LP; ++b)
 #pragma unroll
         for (int t = 0; t < LP; ++t) o[t] = fmaf(a[b], Ms[b][t], o[t]);
+    if (img && i < ((n + TC_KB - 1) / TC_KB) * TC_KB) {
+        constexpr int LPP = TcCfg<LP>::LPP, N1 = TcCfg<LP>::N1;
+        const int kappa = i & 31;
+        uint32_t *dst = img + (size_t)(i >> 5) * (N1 * 32);
+#pragma unroll
+        for (int t = 0; t < LPP; ++t) {
+            const float v = t < LP ? o[t < LP ? t : 0] : 0.f;
+            const uint32_t hi = tf32_round(v);
+            dst[t * 32 + ((((kappa >> 2) ^ (t & 7)) << 2) | (kappa & 3))] = hi;
+            dst[(LPP + t) * 32 + ((((kappa >> 2) ^ ((LPP + t) & 7)) << 2) | (kappa & 3))] = tf32_round(v - __uint_as_float(hi));
+        }
+    }
+    if (i >= n) return;
     if (out) {
         for (int t = 0; t < out_cols; ++t) out[(size_t)i * out_cols + t] = o[t];     // compact result (the first out_cols columns)
     } else {
@@ -819,11 +841,12 @@ static int padded_rank(int l) {
     return LP;
 }
 
-// A <- an orthonormal basis of its columns (Cholesky QR); with `parts` > 0, A is first formed as the sum of the partial sums in w.P
+// A <- an orthonormal basis of its columns (Cholesky QR); with `parts` > 0, A is first formed as the sum of the partial sums
+// in w.P; with `img`, the operand images of the result are written for the tensor-core product that reads it next
 template <int LP>
-static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st, int parts = 0) {
+static mdbf_status_t orth(float *A, int n, Scratch &w, cudaStream_t st, int parts = 0, uint32_t *img = nullptr) {
     gram_finish_kernel<LP, true><<<std::min(ceil_div(n, GR_ROWS), GR_MAX_CTAS), 256, 0, st>>>(A, n, w.P, parts, w.Gp, w.counter, w.Gs, w.M);
-    right_mul_kernel<LP><<<ceil_div(n, 256), 256, 0, st>>>(A, n, w.M, nullptr, 0);
+    right_mul_kernel<LP><<<ceil_div(n, 256), 256, 0, st>>>(A, n, w.M, nullptr, 0, img);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
@@ -864,10 +887,11 @@ struct ZMaps {
     CUtensorMap rows;       // box of 32 columns x 128 rows, 128B swizzle, for Y = E Q
     CUtensorMap cols;       // box of 128 columns x 32 rows, for W = E^T Y
 };
-// E in (TRANS = false: p output rows, in has q) or E^T in (TRANS = true: q output rows, in has p), E the envelope of Z
-// (|Z|, or Z with the given mask's signs taken off), on the tensor cores; the result is left as *parts_out partial sums in w.P
+// E F (TRANS = false: p output rows, F has q) or E^T F (TRANS = true: q output rows, F has p) on the tensor cores, E the
+// envelope of Z (|Z|, or Z with the given mask's signs taken off) and F the factor whose operand images the preceding
+// right_mul_kernel left in w.img; the result is left as *parts_out partial sums in w.P
 template <int LP, bool MASKED, bool TRANS, bool WRITE_MASK = false>
-static mdbf_status_t tc_product(const ZMaps &zm, int p, int q, const float *in, const uint32_t *S, int nwords, Scratch &w,
+static mdbf_status_t tc_product(const ZMaps &zm, int p, int q, const uint32_t *S, int nwords, Scratch &w,
                                 cudaStream_t st, int *parts_out, uint32_t *S_out = nullptr) {
     using C = TcCfg<LP>;
     static bool attr_set = false;
@@ -878,8 +902,6 @@ static mdbf_status_t tc_product(const ZMaps &zm, int p, int q, const float *in, 
     const int m_ext = TRANS ? q : p, k_ext = TRANS ? p : q;
     int kb_per_cta = 0;
     const int parts = tc_split(m_ext, k_ext, LP, &kb_per_cta);
-    const int nkb = ceil_div(k_ext, TC_KB);
-    qimg_kernel<LP><<<std::min(ceil_div(nkb * C::N1 * 32, 256), 148 * 8), 256, 0, st>>>(in, k_ext, nkb, w.img);
     envelope_product_tc_kernel<LP, MASKED, TRANS, WRITE_MASK><<<dim3(ceil_div(m_ext, 128), parts), TC_THREADS, C::SMEM, st>>>(
         TRANS ? zm.cols : zm.rows, p, q, w.img, kb_per_cta, w.P, S, S_out, nwords, w.status);
     *parts_out = parts;                                          // the Gram kernel that follows adds the partial sums up
@@ -892,8 +914,8 @@ static mdbf_status_t product(const float *Z, int p, int q, const uint32_t *S, in
                              int *parts, uint32_t *S_out = nullptr) {
     if (zm.use) {
         if constexpr (!MASKED)
-            if (S_out) return tc_product<LP, false, false, true>(zm, p, q, w.Q, S, nwords, w, st, parts, S_out);
-        return tc_product<LP, MASKED, false>(zm, p, q, w.Q, S, nwords, w, st, parts);
+            if (S_out) return tc_product<LP, false, false, true>(zm, p, q, S, nwords, w, st, parts, S_out);
+        return tc_product<LP, MASKED, false>(zm, p, q, S, nwords, w, st, parts);
     }
     *parts = 0;                                                  // the scalar kernels write the whole result
     absz_q_kernel<LP, MASKED><<<ceil_div(p, AQ_WARPS * AQ_ROWS), AQ_WARPS * 32, 0, st>>>(Z, p, q, w.Q, w.Y, S, nwords);
@@ -904,7 +926,7 @@ static mdbf_status_t product(const float *Z, int p, int q, const uint32_t *S, in
 template <int LP, bool MASKED>
 static mdbf_status_t product_t(const float *Z, int p, int q, const uint32_t *S, int nwords, const ZMaps &zm, Scratch &w, cudaStream_t st,
                                int *parts) {
-    if (zm.use && LP >= 8) return tc_product<LP, MASKED, true>(zm, p, q, w.Y, S, nwords, w, st, parts);
+    if (zm.use && LP >= 8) return tc_product<LP, MASKED, true>(zm, p, q, S, nwords, w, st, parts);
     *parts = 0;   // narrower blocks: the scalar kernel runs at the memory rate already
     const int zy_chunks = ceil_div(p, ZY_ROWS);
     abszT_y_kernel<LP, MASKED><<<dim3(ceil_div(q, ZY_COLS), zy_chunks), ZY_COLS, 0, st>>>(Z, p, q, w.Y, w.P, S, nwords);
@@ -931,23 +953,24 @@ static mdbf_status_t run(const float *Z, int p, int q, int l, int n_iter, const 
     pad_kernel<<<(int)std::min<size_t>(((size_t)q * LP + 255) / 256, 148u * 8), 256, 0, st>>>(Q0, (size_t)q, l, LP, w.Q);
     MDBF_CUDA(cudaGetLastError());
     mdbf_status_t rc = orth<LP>(w.Q, q, w, st);                        // twice: the start block may be badly conditioned
-    if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st);
+    uint32_t *img_q = zm.use ? w.img : nullptr, *img_y = (zm.use && LP >= 8) ? w.img : nullptr;   // which products run on the tensor cores
+    if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st, 0, img_q);
     if (rc) return rc;
     int parts = 0;
     for (int it = 0; it < n_iter; ++it) {
         rc = product<LP, MASKED>(Z, p, q, S, nwords, zm, w, st, &parts, (!MASKED && it == 0) ? S : nullptr);
-        if (rc == MDBF_OK) rc = orth<LP>(w.Y, p, w, st, parts);
+        if (rc == MDBF_OK) rc = orth<LP>(w.Y, p, w, st, parts, img_y);
         if (rc == MDBF_OK) rc = product_t<LP, MASKED>(Z, p, q, S, nwords, zm, w, st, &parts);
-        if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st, parts);
-        if (rc == MDBF_OK && it == n_iter - 1) rc = orth<LP>(w.Q, q, w, st);   // the last block carries the result: orthonormal to fp32
+        if (rc == MDBF_OK) rc = orth<LP>(w.Q, q, w, st, parts, it == n_iter - 1 ? nullptr : img_q);
+        if (rc == MDBF_OK && it == n_iter - 1) rc = orth<LP>(w.Q, q, w, st, 0, img_q);   // the last block carries the result: orthonormal to fp32
         if (rc) return rc;
     }
     rc = product<LP, MASKED>(Z, p, q, S, nwords, zm, w, st, &parts);
     if (rc) return rc;
     gram_finish_kernel<LP, false><<<std::min(ceil_div(p, GR_ROWS), GR_MAX_CTAS), 256, 0, st>>>(w.Y, p, w.P, parts, w.Gp, w.counter, w.Gs, w.M);
     jacobi_kernel<LP><<<1, JAC_THREADS, 0, st>>>(w.Gs, l, sigma, w.MU, w.MV);
-    right_mul_kernel<LP><<<ceil_div(p, 256), 256, 0, st>>>(w.Y, p, w.MU, U, l);
-    right_mul_kernel<LP><<<ceil_div(q, 256), 256, 0, st>>>(w.Q, q, w.MV, V, l);
+    right_mul_kernel<LP><<<ceil_div(p, 256), 256, 0, st>>>(w.Y, p, w.MU, U, l, nullptr);
+    right_mul_kernel<LP><<<ceil_div(q, 256), 256, 0, st>>>(w.Q, q, w.MV, V, l, nullptr);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
