@@ -43,9 +43,9 @@ NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     ("decode_mlp_T16", "mat_small_kernel"): 6340000,               # up stage B (stage A: 6.11 MB, down stage A: 2.47 MB)
     ("prefill_4096_l16_bpw10", "mat_stage_kernel"): 17858048,      # stage B: x read once + signs + images; nothing reaches DRAM on the way out
     ("prefill_4096_l16_bpw10", "gemm_stage_kernel"): 370142976,    # stage B: 269.4 MB read + 100.7 MB written
-    ("msvid_28672x6016_l16", "absz_q_kernel"): 703000000,         # Z once per pass (689.9 MB) + the skinny operand and result, scaled by
-                                                                   # rows x cols from the 8192 x 8192 capture (273.6 MB for 268.4 MB of Z)
-    ("msvid_8192x8192_l16", "absz_q_kernel"): 273649664,
+    ("msvid_28672x6016_l16", "envelope_product_tc_kernel"): 708300000,   # Z once per pass (689.9 MB) + operand images and partial sums,
+                                                                           # scaled by rows x cols from the 8192 x 8192 capture
+    ("msvid_8192x8192_l16", "envelope_product_tc_kernel"): 275523328,      # 269.6 MB read + 5.9 MB written for 268.4 MB of Z
     ("block70b_T2048", "mat_stage_kernel"): 197116928,             # its largest launch, down stage B (185.9 MB read: 117 MB of x, partly twice,
                                                                    # + signs; 11.3 MB written); gate / up stage A: 123.3 MB
 }
@@ -525,7 +525,9 @@ def measure_msvid(workload, steps, warmup, dist, world, local, want_e2e=True, mi
     value = replicas.aggregate_throughput(step_bytes * steps / 1e9, world, ms_max / 1e3)
     per_gpu = step_bytes * steps / 1e9 / (ms_max / 1e3)
     peak = peaks["hbm_gbs"]
-    launches_per_call = 2 + 2 * 4 + n_iter * (1 + 4 + 2 + 4) + 4 + 1 + 3 + 2          # as msvid.cu issues them
+    # as msvid.cu issues them for these shapes: start block 1 + 2 x 2, per iteration 2 products + 2 x 2 (+ 1 where the narrow
+    # transposed product takes the scalar kernel and its partial-sum pass), last block once more 2, final product and factors 5
+    launches_per_call = 1 + 4 + n_iter * (6 + (1 if l <= 4 else 0)) + 2 + 5
     out = {
         "metric": "msvid_algorithmic_GBps", "value": value, "unit": "GB/s", "steps": steps, "warmup": max(3, warmup),
         "ms_per_step": ms_max / steps,
@@ -539,8 +541,8 @@ def measure_msvid(workload, steps, warmup, dist, world, local, want_e2e=True, mi
         "gpu_launches": launches_per_call * steps,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
-                     "peak_source": f"of {peak_kind}", "kernel": "absz_q_kernel / abszT_y_kernel",
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((workload, "absz_q_kernel"))},
+                     "peak_source": f"of {peak_kind}", "kernel": "envelope_product_tc_kernel",
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((workload, "envelope_product_tc_kernel"))},
     }
     del Zd, Qd, Sd, Ud, Vd, ws, flush
     torch.cuda.empty_cache()

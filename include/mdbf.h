@@ -304,10 +304,14 @@ mdbf_status_t mdbf_poll_status(mdbf_handle_t h, int32_t *device_status);
  *             common sign only, and up to rotations inside a group of equal singular values)
  *   sigma     device, l fp32, written: the estimated singular values; each is a lower bound of the exact one
  *   workspace device, at least mdbf_msvid_workspace_bytes(rows, cols, l) bytes on a 256-byte boundary, scratch of the
- *             call (about (rows + cols + cols * ceil(rows / 256)) * l floats); free again when the stream has passed it
- * The truncated SVD is computed by block subspace iteration (hand-written CUDA-core kernels, fp32 with the small
- * Gram matrices in fp64), not to machine precision: see n_iter.  Asynchronous on `stream`; allocates nothing and does
- * not synchronise.  Errors: INVALID_ARG (NULL pointer, workspace too small or misaligned), SHAPE, ARCH, CUDA. */
+ *             call (the two blocks, the partial sums of a product - up to 16 per output row - and operand images:
+ *             ask mdbf_msvid_workspace_bytes); free again when the stream has passed it
+ * The truncated SVD is computed by block subspace iteration, not to machine precision: see n_iter.  The two products
+ * with |Z| run on the tensor cores (TF32 operands in a three-term split that keeps fp32 accuracy, fp32 accumulation)
+ * when cols is a multiple of 4 and Z sits on a 16-byte boundary, else in scalar fp32 kernels; the small Gram matrices
+ * are fp64.  Results do not depend on scheduling (no floating-point atomics).  Asynchronous on `stream`; allocates
+ * nothing and does not synchronise.  Should one of the kernel's bounded waits expire (not expected), the outputs are
+ * NaN.  Errors: INVALID_ARG (NULL pointer, workspace too small or misaligned), SHAPE, ARCH, CUDA. */
 mdbf_status_t mdbf_msvid(const float *Z, int64_t rows, int64_t cols, int32_t l, int32_t n_iter, const float *Q0,
                          uint32_t *S_packed, float *U, float *V, float *sigma, void *workspace, size_t workspace_bytes,
                          void *stream);

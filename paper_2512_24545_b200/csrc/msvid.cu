@@ -181,7 +181,8 @@ __global__ void __launch_bounds__(AQ_WARPS * 32) absz_q_kernel(const float *__re
 //     straight into tensor memory as the A operand: shared memory carries each byte of Z once in and once out,
 //     where operand tiles in shared memory would carry it six times and bound the kernel;
 //   one lane bulk-copies the K block's image of the other factor: rows [0, LPP) = q_hi, [LPP, 2 LPP) = q_lo of the 32
-//     contraction indices, already in the K-major 128B-swizzled operand layout (qimg_kernel builds the images once per pass);
+//     contraction indices, already in the K-major 128B-swizzled operand layout (right_mul_kernel writes the images
+//     when it writes the factor);
 //   two lanes issue the MMAs, four K steps of 8 each: D1 (+)= E_hi [q_hi | q_lo] (N = 2 LPP), D2 (+)= E_lo q_hi (N = LPP).
 // Epilogue: y[t] = D1[t] + D1[LPP + t] + D2[t] into the range's partial sums.
 // TRANS = false: Y = E Q    (output rows = rows of Z, contraction over its columns; TMA box of 32 columns x 128 rows,
@@ -231,23 +232,6 @@ __device__ __forceinline__ uint32_t make_idesc_tf32(int n) {
     d |= (uint32_t)(n >> 3) << 17;      // N
     d |= (uint32_t)(128 >> 4) << 24;    // M
     return d;
-}
-// images of a tall factor F (n x LP) for one pass: K block kb holds rows r of 32 TF32 values, 128 bytes each, 128B swizzle
-template <int LP>
-__global__ void __launch_bounds__(256) qimg_kernel(const float *__restrict__ Q, int q, int nkb, uint32_t *__restrict__ img) {
-    constexpr int LPP = TcCfg<LP>::LPP, N1 = TcCfg<LP>::N1;
-    const size_t total = (size_t)nkb * N1 * 32;
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
-        const int kappa = (int)(e & 31);
-        const int n = (int)((e >> 5) % N1);
-        const int kb = (int)(e / ((size_t)N1 * 32));
-        const int t = n < LPP ? n : n - LPP;
-        const int col = kb * 32 + kappa;
-        const float v = (t < LP && col < q) ? Q[(size_t)col * LP + t] : 0.f;
-        const uint32_t hi = tf32_round(v);
-        const uint32_t out = n < LPP ? hi : tf32_round(v - __uint_as_float(hi));
-        img[(size_t)kb * (N1 * 32) + n * 32 + ((((kappa >> 2) ^ (n & 7)) << 2) | (kappa & 3))] = out;
-    }
 }
 // WRITE_MASK (plain product of |Z| only): the converters also pack the signs of what they read into S_out, the mask of
 // Eq. msvid-def (bit = 1 where the entry is below zero; zeros of either sign count as +1), so that the first pass over Z
@@ -641,7 +625,9 @@ __global__ void __launch_bounds__(256) gram_finish_kernel(float *__restrict__ A,
     if (threadIdx.x < 32) chol_warp<LP>(Gm, M);
 }
 // A <- A M, row by row (M is LP x LP, row-major).  With `img`, the rows' operand images for the tensor-core product that
-// reads A next are written on the way out (the layout qimg_kernel documents; rows past the end are zero).
+// reads A next are written on the way out: per block of 32 rows (= 32 contraction indices kappa) a tile of 2 LPP rows of
+// 32 TF32 values, 128 bytes each, 16-byte chunk c of row r at position c ^ (r & 7) (the 128B swizzle of a K-major
+// operand); row t < LPP holds the TF32 rounding of column t, row LPP + t the rounded residual; rows past the end are zero.
 template <int LP>
 __global__ void __launch_bounds__(256) right_mul_kernel(float *__restrict__ A, int n, const float *__restrict__ M, float *__restrict__ out,
                                                         int out_cols, uint32_t *__restrict__ img) {

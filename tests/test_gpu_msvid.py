@@ -43,8 +43,11 @@ def envelope_error(Z, U, V):
     return np.linalg.norm(np.abs(Z.astype(np.float64)) - U @ V.T)
 
 
-@pytest.mark.parametrize("shape", [(300, 517), (1024, 768), (129, 33), (64, 2000), (2000, 64), (33, 40)])
-@pytest.mark.parametrize("l", [1, 4, 16])
+# shapes whose column count is a multiple of four run the tensor-core products (ragged last row block and K block
+# included), the others the scalar kernels; l = 8 and 32 take the remaining operand widths
+@pytest.mark.parametrize("shape,l", [(s, l) for s in [(300, 517), (1024, 768), (129, 33), (64, 2000), (2000, 64), (33, 40)]
+                                     for l in (1, 4, 16)] + [((333, 516), 8), ((333, 516), 32), ((1000, 260), 8), ((1000, 260), 32),
+                                                             ((515, 1028), 16)])
 def test_sign_mask_exact_and_envelope_near_the_optimum(shape, l):
     rows, cols = shape
     Z = inputs.make_factor_matrix(rows, cols, seed=5)
@@ -71,6 +74,38 @@ def test_sign_mask_exact_and_envelope_near_the_optimum(shape, l):
     # balanced factors: both columns of a pair carry the square root of their singular value
     np.testing.assert_allclose(np.linalg.norm(U, axis=0), np.sqrt(s), rtol=2e-4)
     np.testing.assert_allclose(np.linalg.norm(V, axis=0), np.sqrt(s), rtol=2e-4)
+
+
+def test_tensor_core_and_scalar_products_agree():
+    """The same matrix at a 16-byte aligned address (tensor-core products, three-term TF32 split) and four bytes further on
+    (the scalar fp32 kernels): the same mask, and singular values that agree to fp32 accuracy."""
+    rows, cols, l = 700, 1028, 16
+    Z = inputs.make_factor_matrix(rows, cols, seed=6)
+    Q0 = inputs.make_start_block(cols, l, 12)
+    buf = torch.zeros(rows * cols + 1, dtype=torch.float32, device="cuda")
+    Zt = torch.from_numpy(Z).cuda().reshape(-1)
+    nwords = (cols + 31) // 32
+    nbytes = M.mdbf_msvid_workspace_bytes(rows, cols, l)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    Qd = torch.from_numpy(Q0).cuda()
+    res = []
+    for off in (0, 1):
+        buf.zero_()
+        buf[off:off + rows * cols] = Zt
+        Sd = torch.zeros((rows, nwords), dtype=torch.int32, device="cuda")
+        Ud = torch.zeros((rows, l), dtype=torch.float32, device="cuda")
+        Vd = torch.zeros((cols, l), dtype=torch.float32, device="cuda")
+        sd = torch.zeros((l,), dtype=torch.float32, device="cuda")
+        assert (buf.data_ptr() + 4 * off) % 16 == (0 if off == 0 else 4)
+        M.mdbf_msvid(buf.data_ptr() + 4 * off, rows, cols, l, 6, Qd.data_ptr(), Sd.data_ptr(), Ud.data_ptr(), Vd.data_ptr(),
+                     sd.data_ptr(), ws.data_ptr(), nbytes, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        res.append((Sd.cpu().numpy(), sd.cpu().numpy().astype(np.float64), Ud.cpu().numpy().astype(np.float64),
+                    Vd.cpu().numpy().astype(np.float64)))
+    np.testing.assert_array_equal(res[0][0], res[1][0])
+    np.testing.assert_allclose(res[0][1], res[1][1], rtol=2e-5)
+    e0, e1 = envelope_error(Z, res[0][2], res[0][3]), envelope_error(Z, res[1][2], res[1][3])
+    assert abs(e0 - e1) <= 1e-5 * e1
 
 
 def test_error_decreases_with_envelope_rank_and_with_iterations():
