@@ -29,7 +29,10 @@ demodulation rank and isometry (Eq. me-dbf-envelope-rank, Lemma sign-mask
 isometry), a hand-worked example (tests/golden/), the bit-packing definition
 against numpy.packbits, the exact-projection error against the singular-value
 tail (Theorem 1); the sum of terms against the two-term product of Eq. dbf-residual-comp written
-out per entry and against the sum of single-term forwards.  No function here is "parity unpinned".
+out per entry and against the sum of single-term forwards.  The ADMM factor update (tests/test_oracle_admm.py):
+a scalar instance worked by hand, the stationarity and minimality of its least-squares step, the limit of a large
+penalty, the fixed point at an exactly representable factor, the envelope rank of its result.  No function here is
+"parity unpinned".
 """
 from __future__ import annotations
 
@@ -38,7 +41,7 @@ import numpy as np
 __all__ = [
     "envelope", "modulated_factor", "reconstruct", "reconstruct_rows", "forward",
     "forward_staged", "reconstruct_sum", "forward_sum", "rel_frobenius", "pack_signs", "unpack_signs",
-    "bits_per_weight", "largest_inner_rank", "project_fixed_mask", "msvid",
+    "bits_per_weight", "largest_inner_rank", "project_fixed_mask", "msvid", "admm_factor_update",
 ]
 
 
@@ -258,3 +261,38 @@ def msvid(Z, l):
     Uu, s, Vt = np.linalg.svd(np.abs(Z), full_matrices=False)
     r = np.sqrt(s[:l])
     return S, Uu[:, :l] * r, Vt[:l].T * r
+
+
+# --------------------------------------------------------------------------
+# ADMM refinement of one factor with the other held fixed (Section "ADMM
+# Refinement", Eq. admm-U-tilde, Eq. admm-U-prox, Eq. admm-U-dual).  The update
+# of the other factor is the same function on the transposed problem.
+# --------------------------------------------------------------------------
+def admm_factor_update(W, V, U, Lam, rho, l, n_inner=1):
+    """n_inner ADMM inner iterations on U (N x R, dense values of the factor) for min ||W - U V^T||_F^2 with V (M x R)
+    fixed, auxiliary variable U_tilde and scaled dual variable Lam (N x R):
+
+        U_tilde = (W V + rho (U - Lam)) (V^T V + rho I)^-1        Eq. admm-U-tilde
+        U       = MSVID_l[U_tilde + Lam]                          Eq. admm-U-prox
+        Lam     = Lam + U_tilde - U                               Eq. admm-U-dual
+
+    Returns (U, Lam, U_tildes, masks): the new U and Lam, and per inner iteration the least-squares iterate and the sign
+    mask MSVID chose.
+    """
+    W, V, U, Lam = _f64(W), _f64(V), _f64(U), _f64(Lam)
+    R = V.shape[1]
+    if W.shape != (U.shape[0], V.shape[0]) or U.shape[1] != R or Lam.shape != U.shape:
+        raise ValueError("shapes do not fit W (N x M), V (M x R), U and Lam (N x R)")
+    if not rho > 0:
+        raise ValueError("rho must be positive")
+    G = V.T @ V + rho * np.eye(R)
+    WV = W @ V
+    tildes, masks = [], []
+    for _ in range(n_inner):
+        U_tilde = np.linalg.solve(G, (WV + rho * (U - Lam)).T).T          # G is symmetric
+        S, Ul, Vl = msvid(U_tilde + Lam, l)
+        U = S * (Ul @ Vl.T)
+        Lam = Lam + U_tilde - U
+        tildes.append(U_tilde)
+        masks.append(S)
+    return U, Lam, tildes, masks
