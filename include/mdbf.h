@@ -329,6 +329,40 @@ mdbf_status_t mdbf_project_fixed_mask(const float *Z, const uint32_t *S_packed, 
 /* Size of the workspace mdbf_msvid needs for this shape (host computation, no device needed).  Errors: INVALID_ARG, SHAPE. */
 mdbf_status_t mdbf_msvid_workspace_bytes(int64_t rows, int64_t cols, int32_t l, size_t *bytes);
 
+/* ---------------------------------------------------------------- quantizer, refinement
+ * n_inner ADMM inner iterations on one factor with the other held fixed (Section "ADMM Refinement"), for the
+ * objective ||W - U V^T||_F^2 with the multi-envelope structure imposed by MSVID_l:
+ *     U_tilde = (W V + rho (U - Lam)) (V^T V + rho I)^-1        (Eq. admm-U-tilde)
+ *     U       = MSVID_l[U_tilde + Lam]                          (Eq. admm-U-prox)
+ *     Lam     = Lam + U_tilde - U                               (Eq. admm-U-dual)
+ * With N x M = the shape of op(W): op(W) = W (w_rows x w_cols) for transpose_w = 0 and W^T for transpose_w != 0 -
+ * the update of the other factor is this call on the transposed problem, with the roles of the factors exchanged.
+ *   W          device, w_rows x w_cols fp32 row-major, read only
+ *   V          device, M x R fp32 row-major: the dense values of the fixed factor, read only
+ *   U, Lambda  device, N x R fp32 row-major, read and written: the dense values of the factor being refined and the
+ *              scaled dual variable (zeros to start with)
+ *   rho        penalty, > 0
+ *   l, n_iter, Q0 (R x l)   as for mdbf_msvid, which performs the prox step (the same Q0 starts every inner iteration)
+ *   S_packed (N x ceil(R / 32)), Ul (N x l), Vl (R x l), sigma (l)   device, written: the compact form of the new U,
+ *              U = S (.) (Ul Vl^T), as mdbf_msvid returns it in the last inner iteration
+ *   U_tilde    device, N x R fp32, written with the last inner iteration's least-squares iterate; may be NULL
+ *   workspace  device, mdbf_admm_workspace_bytes(N, R, l) bytes on a 256-byte boundary (three N x R matrices, the R x R
+ *              system and mdbf_msvid's workspace)
+ * The two plain dense products and the Cholesky factorisation and solve of the R x R system are cuBLAS / cuSOLVER
+ * calls in fp32; the MSVID step, the elementwise passes and the reconstruction of the dense factor fused with the
+ * dual update are this library's kernels.  Asynchronous on `stream`.  The first call on a host thread creates the
+ * libraries' handles and allocates the scratch the factorisation asks for (kept for later calls; a larger request
+ * synchronises the stream and reallocates).  A failed factorisation (not expected for rho > 0) turns sigma into NaN.
+ * Errors: INVALID_ARG (NULL pointer, rho <= 0, counts out of range, workspace too small or misaligned), SHAPE, ARCH, CUDA. */
+mdbf_status_t mdbf_admm_factor_update(const float *W, int64_t w_rows, int64_t w_cols, int32_t transpose_w, const float *V, int64_t r,
+                                      float *U, float *Lambda, float rho, int32_t l, int32_t n_inner, int32_t n_iter,
+                                      const float *Q0, uint32_t *S_packed, float *Ul, float *Vl, float *sigma, float *U_tilde,
+                                      void *workspace, size_t workspace_bytes, void *stream);
+
+/* Size of the workspace mdbf_admm_factor_update needs for an N x R factor (host computation, no device needed).
+ * Errors: INVALID_ARG, SHAPE. */
+mdbf_status_t mdbf_admm_workspace_bytes(int64_t n, int64_t r, int32_t l, size_t *bytes);
+
 /* Test hook (no counterpart in the paper): the `nth` device allocation that the calling thread makes
  * inside this library from now on fails with MDBF_ERR_ALLOC without touching the device; nth <= 0
  * cancels a pending request.  A call that fails this way frees what it had allocated, publishes

@@ -1,0 +1,233 @@
+// ADMM refinement of one MDBF factor with the other held fixed (Section "ADMM Refinement"):
+//
+//     U_tilde = (W V + rho (U - Lam)) (V^T V + rho I)^-1        Eq. admm-U-tilde
+//     U       = MSVID_l[U_tilde + Lam]                          Eq. admm-U-prox
+//     Lam     = Lam + U_tilde - U                               Eq. admm-U-dual
+//
+// W is N x M, V is M x R, U and Lam are N x R (dense values of the factor), all fp32 row-major on the device.  The
+// update of the other factor is the same call on the transposed problem (transpose_w).
+//
+// The two plain dense products (W V once per call, V^T V once per call) and the Cholesky factorisation and solve of
+// the R x R system are library routines (cuBLAS, cuSOLVER); everything specific to the method is this library's own:
+// the MSVID step (mdbf_msvid: sign mask + rank-l envelope on the tensor cores), the elementwise passes around it, and
+// the reconstruction of the dense factor from the compact one fused with the dual update.
+//
+// Row-major matrices are handed to the column-major libraries as their transposes: a row-major n x r matrix is a
+// column-major r x n one with leading dimension r, so that  B = W V  becomes  B^T = V^T W^T  and the solve
+// X G = T  becomes  G X^T = T^T  on the same memory.
+#include <cublas_v2.h>
+#include <cusolverDn.h>
+
+#include <algorithm>
+#include <cstdint>
+
+#include "common.cuh"
+
+namespace mdbf {
+namespace admm {
+
+struct Libs {
+    cublasHandle_t blas = nullptr;
+    cusolverDnHandle_t solver = nullptr;
+    float *potrf_ws = nullptr;          // the factorisation's scratch, as large as the largest request so far
+    int potrf_floats = 0;
+    int device = -1;
+};
+static thread_local Libs g_libs;
+
+static mdbf_status_t get_libs(int device, cudaStream_t st, Libs **out) {
+    Libs &L = g_libs;
+    if (L.device != device) {
+        if (L.blas) cublasDestroy(L.blas);
+        if (L.solver) cusolverDnDestroy(L.solver);
+        if (L.potrf_ws) cudaFree(L.potrf_ws);
+        L = Libs();
+        if (cublasCreate(&L.blas) != CUBLAS_STATUS_SUCCESS) { L = Libs(); set_error("cublasCreate failed"); return MDBF_ERR_CUDA; }
+        if (cusolverDnCreate(&L.solver) != CUSOLVER_STATUS_SUCCESS) {
+            cublasDestroy(L.blas);
+            L = Libs();
+            set_error("cusolverDnCreate failed");
+            return MDBF_ERR_CUDA;
+        }
+        cublasSetMathMode(L.blas, CUBLAS_PEDANTIC_MATH);          // plain fp32 products
+        L.device = device;
+    }
+    if (cublasSetStream(L.blas, st) != CUBLAS_STATUS_SUCCESS || cusolverDnSetStream(L.solver, st) != CUSOLVER_STATUS_SUCCESS) {
+        set_error("could not bind the dense-algebra libraries to the stream");
+        return MDBF_ERR_CUDA;
+    }
+    *out = &L;
+    return MDBF_OK;
+}
+
+__global__ void ridge_kernel(float *__restrict__ G, int r, float rho) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < r) G[(size_t)i * r + i] += rho;
+}
+// T = B0 + rho (U - Lam)
+__global__ void rhs_kernel(const float *__restrict__ B0, const float *__restrict__ U, const float *__restrict__ Lam, float rho,
+                           float *__restrict__ T, size_t count) {
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < count; e += (size_t)gridDim.x * blockDim.x)
+        T[e] = B0[e] + rho * (U[e] - Lam[e]);
+}
+// Z = U_tilde + Lam
+__global__ void sum_kernel(const float *__restrict__ Ut, const float *__restrict__ Lam, float *__restrict__ Z, size_t count) {
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < count; e += (size_t)gridDim.x * blockDim.x) Z[e] = Ut[e] + Lam[e];
+}
+// U = S (.) (Ul Vl^T) entry by entry from the compact MSVID result, and Lam += U_tilde - U.
+// CTA = 8 rows x 256 columns; thread = column (its row of Vl in registers), the rows' Ul in shared memory.
+constexpr int RC_ROWS = 8, RC_COLS = 256, RC_MAXL = 32;
+__global__ void __launch_bounds__(RC_COLS) recon_dual_kernel(const uint32_t *__restrict__ S, const float *__restrict__ Ul,
+                                                             const float *__restrict__ Vl, int l, const float *__restrict__ Ut,
+                                                             float *__restrict__ U, float *__restrict__ Lam, int n, int r, int nwords) {
+    __shared__ float us[RC_ROWS][RC_MAXL];
+    const int i0 = blockIdx.y * RC_ROWS;
+    for (int e = threadIdx.x; e < RC_ROWS * RC_MAXL; e += RC_COLS) {
+        const int i = e / RC_MAXL, t = e - i * RC_MAXL;
+        us[i][t] = (i0 + i < n && t < l) ? Ul[(size_t)(i0 + i) * l + t] : 0.f;
+    }
+    __syncthreads();
+    const int j = blockIdx.x * RC_COLS + threadIdx.x;
+    if (j >= r) return;
+    float v[RC_MAXL];
+#pragma unroll
+    for (int t = 0; t < RC_MAXL; ++t) v[t] = t < l ? Vl[(size_t)j * l + t] : 0.f;
+    for (int i = 0; i < RC_ROWS && i0 + i < n; ++i) {
+        float e = 0.f;
+#pragma unroll
+        for (int t = 0; t < RC_MAXL; ++t) e = fmaf(us[i][t], v[t], e);
+        const uint32_t word = S[(size_t)(i0 + i) * nwords + (j >> 5)];
+        const float u = ((word >> (j & 31)) & 1u) ? -e : e;
+        const size_t at = (size_t)(i0 + i) * r + j;
+        U[at] = u;
+        Lam[at] += Ut[at] - u;
+    }
+}
+// a failed factorisation (not expected: the system is positive definite for rho > 0) turns the singular values into NaN
+__global__ void flag_kernel(const int *__restrict__ info, float *__restrict__ sigma, int l) {
+    if (*info != 0 && threadIdx.x < l) sigma[threadIdx.x] = __int_as_float(0x7fc00000);
+}
+
+static size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
+struct Scratch {
+    float *B0, *T, *Z, *G;
+    int *info;
+    char *msvid;
+    size_t msvid_bytes;
+};
+static mdbf_status_t carve(Scratch *w, char *base, int64_t n, int64_t r, int32_t l, size_t *total) {
+    size_t msv = 0;
+    mdbf_status_t rc = mdbf_msvid_workspace_bytes(n, r, l, &msv);
+    if (rc) return rc;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char *p = base ? base + off : nullptr; off += align256(bytes); return p; };
+    float *B0 = (float *)take((size_t)n * r * sizeof(float));
+    float *T = (float *)take((size_t)n * r * sizeof(float));
+    float *Z = (float *)take((size_t)n * r * sizeof(float));
+    float *G = (float *)take((size_t)r * r * sizeof(float));
+    int *info = (int *)take(sizeof(int));
+    char *m = take(msv);
+    if (w) { w->B0 = B0; w->T = T; w->Z = Z; w->G = G; w->info = info; w->msvid = m; w->msvid_bytes = msv; }
+    *total = off;
+    return MDBF_OK;
+}
+static mdbf_status_t check_shape(const char *who, int64_t n, int64_t m, int64_t r, int32_t l) {
+    if (n < 1 || m < 1 || r < 1 || n > (1 << 24) || m > (1 << 24) || r > 32768 || n * r > (1LL << 31) - 1 || n * m > (1LL << 40)) {
+        set_error("%s: sizes N=%lld M=%lld R=%lld outside the supported range", who, (long long)n, (long long)m, (long long)r);
+        return MDBF_ERR_SHAPE;
+    }
+    if (l < 1 || l > kMaxL || l > n || l > r) {
+        set_error("%s: l=%d outside [1, min(%d, N, R)]", who, l, kMaxL);
+        return MDBF_ERR_SHAPE;
+    }
+    return MDBF_OK;
+}
+
+}  // namespace admm
+}  // namespace mdbf
+
+using namespace mdbf;
+
+extern "C" mdbf_status_t mdbf_admm_workspace_bytes(int64_t n, int64_t r, int32_t l, size_t *bytes) {
+    if (!bytes) { set_error("mdbf_admm_workspace_bytes: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
+    mdbf_status_t rc = admm::check_shape("mdbf_admm_workspace_bytes", n, 1, r, l);
+    if (rc) return rc;
+    return admm::carve(nullptr, nullptr, n, r, l, bytes);
+}
+
+extern "C" mdbf_status_t mdbf_admm_factor_update(const float *W, int64_t w_rows, int64_t w_cols, int32_t transpose_w, const float *V,
+                                                 int64_t r, float *U, float *Lambda, float rho, int32_t l, int32_t n_inner,
+                                                 int32_t n_iter, const float *Q0, uint32_t *S_packed, float *Ul, float *Vl,
+                                                 float *sigma, float *U_tilde, void *workspace, size_t workspace_bytes, void *stream) {
+    const char *who = "mdbf_admm_factor_update";
+    if (!W || !V || !U || !Lambda || !Q0 || !S_packed || !Ul || !Vl || !sigma || !workspace) {
+        set_error("%s: NULL pointer", who);
+        return MDBF_ERR_INVALID_ARG;
+    }
+    const int64_t n = transpose_w ? w_cols : w_rows, m = transpose_w ? w_rows : w_cols;
+    mdbf_status_t rc = admm::check_shape(who, n, m, r, l);
+    if (rc) return rc;
+    if (!(rho > 0.f) || n_inner < 1 || n_inner > 1000 || n_iter < 1 || n_iter > 1000) {
+        set_error("%s: rho=%g must be positive, n_inner=%d and n_iter=%d in [1, 1000]", who, (double)rho, n_inner, n_iter);
+        return MDBF_ERR_INVALID_ARG;
+    }
+    admm::Scratch w;
+    size_t need = 0;
+    rc = admm::carve(&w, (char *)workspace, n, r, l, &need);
+    if (rc) return rc;
+    if (workspace_bytes < need || ((uintptr_t)workspace & 255u) != 0) {
+        set_error("%s: the workspace must hold %zu bytes (mdbf_admm_workspace_bytes) on a 256-byte boundary; got %zu at %p", who, need,
+                  workspace_bytes, workspace);
+        return MDBF_ERR_INVALID_ARG;
+    }
+    int device = 0;
+    rc = require_device(&device);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    admm::Libs *L = nullptr;
+    rc = admm::get_libs(device, st, &L);
+    if (rc) return rc;
+    const int ni = (int)n, mi = (int)m, ri = (int)r;
+    const float one = 1.f, zero = 0.f;
+    // B0 = op(W) V:  B0^T (r x n) = V^T (r x m, the memory of V) * op(W)^T (m x n)
+    cublasStatus_t bs = cublasSgemm(L->blas, CUBLAS_OP_N, transpose_w ? CUBLAS_OP_T : CUBLAS_OP_N, ri, ni, mi, &one, V, ri, W,
+                                    transpose_w ? ni : mi, &zero, w.B0, ri);
+    // G = V^T V (lower triangle in column-major terms) + rho I
+    if (bs == CUBLAS_STATUS_SUCCESS) bs = cublasSsyrk(L->blas, CUBLAS_FILL_MODE_LOWER, CUBLAS_OP_N, ri, mi, &one, V, ri, &zero, w.G, ri);
+    if (bs != CUBLAS_STATUS_SUCCESS) { set_error("%s: cuBLAS returned %d", who, (int)bs); return MDBF_ERR_CUDA; }
+    admm::ridge_kernel<<<ceil_div(ri, 256), 256, 0, st>>>(w.G, ri, rho);
+    int lwork = 0;
+    cusolverStatus_t ss = cusolverDnSpotrf_bufferSize(L->solver, CUBLAS_FILL_MODE_LOWER, ri, w.G, ri, &lwork);
+    if (ss != CUSOLVER_STATUS_SUCCESS) { set_error("%s: cusolverDnSpotrf_bufferSize returned %d", who, (int)ss); return MDBF_ERR_CUDA; }
+    if (lwork > L->potrf_floats) {
+        MDBF_CUDA(cudaStreamSynchronize(st));                     // the old scratch may still be in use
+        if (L->potrf_ws) cudaFree(L->potrf_ws);
+        L->potrf_ws = nullptr;
+        L->potrf_floats = 0;
+        if (dev_malloc(&L->potrf_ws, (size_t)lwork * sizeof(float)) != cudaSuccess) {
+            set_error("%s: out of device memory for the factorisation's scratch (%zu bytes)", who, (size_t)lwork * sizeof(float));
+            return MDBF_ERR_CUDA;
+        }
+        L->potrf_floats = lwork;
+    }
+    ss = cusolverDnSpotrf(L->solver, CUBLAS_FILL_MODE_LOWER, ri, w.G, ri, L->potrf_ws, L->potrf_floats, w.info);
+    if (ss != CUSOLVER_STATUS_SUCCESS) { set_error("%s: cusolverDnSpotrf returned %d", who, (int)ss); return MDBF_ERR_CUDA; }
+    const size_t count = (size_t)n * r;
+    const int ew_grid = (int)std::min<size_t>((count + 255) / 256, 148u * 16);
+    const int nwords = (int)((r + 31) / 32);
+    for (int it = 0; it < n_inner; ++it) {
+        admm::rhs_kernel<<<ew_grid, 256, 0, st>>>(w.B0, U, Lambda, rho, w.T, count);
+        // U_tilde G = T  <=>  G U_tilde^T = T^T, in place on the memory of T
+        ss = cusolverDnSpotrs(L->solver, CUBLAS_FILL_MODE_LOWER, ri, ni, w.G, ri, w.T, ri, w.info + 1);
+        if (ss != CUSOLVER_STATUS_SUCCESS) { set_error("%s: cusolverDnSpotrs returned %d", who, (int)ss); return MDBF_ERR_CUDA; }
+        admm::sum_kernel<<<ew_grid, 256, 0, st>>>(w.T, Lambda, w.Z, count);
+        rc = mdbf_msvid(w.Z, n, r, l, n_iter, Q0, S_packed, Ul, Vl, sigma, w.msvid, w.msvid_bytes, stream);
+        if (rc) return rc;
+        admm::recon_dual_kernel<<<dim3(ceil_div(ri, admm::RC_COLS), ceil_div(ni, admm::RC_ROWS)), admm::RC_COLS, 0, st>>>(
+            S_packed, Ul, Vl, l, w.T, U, Lambda, ni, ri, nwords);
+    }
+    if (U_tilde) MDBF_CUDA(cudaMemcpyAsync(U_tilde, w.T, count * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    admm::flag_kernel<<<1, 32, 0, st>>>(w.info, sigma, l);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}

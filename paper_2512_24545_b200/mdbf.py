@@ -29,7 +29,7 @@ EXPORTS = (
     "mdbf_pack_signs", "mdbf_unpack_signs", "mdbf_pack", "mdbf_get_packed", "mdbf_get_envelope",
     "mdbf_get_desc", "mdbf_set_kernel", "mdbf_linear_forward", "mdbf_linear_forward_host", "mdbf_linear_forward_host_async", "mdbf_prepare_host_staging",
     "mdbf_linear_forward_static", "mdbf_linear_forward_sum", "mdbf_linear_forward_siblings", "mdbf_linear_forward_group",
-    "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_msvid", "mdbf_msvid_workspace_bytes", "mdbf_project_fixed_mask", "mdbf_poll_status", "mdbf_selftest_wait_timeout", "mdbf_debug_fail_alloc",
+    "mdbf_get_intermediate", "mdbf_reconstruct", "mdbf_msvid", "mdbf_msvid_workspace_bytes", "mdbf_project_fixed_mask", "mdbf_admm_factor_update", "mdbf_admm_workspace_bytes", "mdbf_poll_status", "mdbf_selftest_wait_timeout", "mdbf_debug_fail_alloc",
     "mdbf_last_launch_count",
     "mdbf_last_kernel",
     "mdbf_destroy", "mdbf_last_error", "mdbf_version",
@@ -82,6 +82,9 @@ def lib() -> ctypes.CDLL:
     L.mdbf_msvid.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     L.mdbf_project_fixed_mask.argtypes = [vp, vp, i64, i64, i32, i32, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     L.mdbf_msvid_workspace_bytes.argtypes = [i64, i64, i32, ctypes.POINTER(ctypes.c_size_t)]
+    L.mdbf_admm_workspace_bytes.argtypes = [i64, i64, i32, ctypes.POINTER(ctypes.c_size_t)]
+    L.mdbf_admm_factor_update.argtypes = [vp, i64, i64, i32, vp, i64, vp, vp, ctypes.c_float, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp,
+                                          ctypes.c_size_t, vp]
     L.mdbf_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
     L.mdbf_selftest_wait_timeout.argtypes = [vp, vp]
     L.mdbf_debug_fail_alloc.argtypes = [i32]
@@ -249,6 +252,22 @@ def mdbf_project_fixed_mask(Z, S_packed, rows: int, cols: int, l: int, n_iter: i
     singular values; device addresses throughout, asynchronous.  See include/mdbf.h."""
     _check(lib().mdbf_project_fixed_mask(_addr(Z), _addr(S_packed), rows, cols, l, n_iter, _addr(Q0), _addr(U), _addr(V), _addr(sigma),
                                          _addr(workspace), workspace_bytes, stream))
+
+
+def mdbf_admm_workspace_bytes(n: int, r: int, l: int) -> int:
+    v = ctypes.c_size_t()
+    _check(lib().mdbf_admm_workspace_bytes(n, r, l, ctypes.byref(v)))
+    return v.value
+
+
+def mdbf_admm_factor_update(W, w_rows: int, w_cols: int, transpose_w: bool, V, r: int, U, Lambda, rho: float, l: int, n_inner: int,
+                            n_iter: int, Q0, S_packed, Ul, Vl, sigma, U_tilde, workspace, workspace_bytes: int, stream: int = 0) -> None:
+    """n_inner ADMM inner iterations on the factor U (N x R dense, updated in place with its dual Lambda) for
+    ||op(W) - U V^T||_F^2 with V fixed, the prox step being MSVID_l; device addresses throughout (U_tilde may be None),
+    asynchronous.  See include/mdbf.h."""
+    _check(lib().mdbf_admm_factor_update(_addr(W), w_rows, w_cols, int(bool(transpose_w)), _addr(V), r, _addr(U), _addr(Lambda),
+                                         float(rho), l, n_inner, n_iter, _addr(Q0), _addr(S_packed), _addr(Ul), _addr(Vl), _addr(sigma),
+                                         _addr(U_tilde) if U_tilde is not None else None, _addr(workspace), workspace_bytes, stream))
 
 
 def mdbf_debug_fail_alloc(nth: int) -> None:
