@@ -563,6 +563,125 @@ def cpu_baseline_msvid(rows, cols, l, n_iter):
             "sample": f"fp64 sign mask + full SVD of a {Z.shape[0]} x {Z.shape[1]} block of the workload's matrix, one call, {dt:.1f} s"}
 
 
+# ------------------------------------------------------------ quantizer, refinement (ADMM factor update)
+FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 148 SMs x 128 FP32 FMA lanes x 2 flops at the maximum SM clock
+
+
+def admm_shape(workload):
+    import re
+    m = re.match(r"admm_(\d+)x(\d+)_r(\d+)_l(\d+)(?:_in(\d+))?$", workload)
+    if not m:
+        raise SystemExit(f"unknown workload {workload}")
+    return int(m.group(1)), int(m.group(2)), int(m.group(3)), int(m.group(4)), int(m.group(5)) if m.group(5) else 1
+
+
+def admm_flops(N, Mc, R, n_inner):
+    """Dense-algebra flops of the least-squares step: W V, V^T V (one triangle), the Cholesky factor, two triangular
+    solves with N right-hand sides per inner iteration.  The MSVID step's flops (a few per cent) are not counted."""
+    return 2.0 * N * Mc * R + 1.0 * Mc * R * R + R ** 3 / 3.0 + n_inner * 2.0 * N * R * R
+
+
+def measure_admm(workload, steps, warmup, dist, world, local, want_e2e=True):
+    """admm_<N>x<M>_r<R>_l<l>[_in<n>]: one step = one mdbf_admm_factor_update call (n inner iterations, 4 subspace
+    iterations in each MSVID step) on resident fp32 matrices W (N x M), V (M x R), U and Lambda (N x R)."""
+    import torch
+    from paper_2512_24545_b200 import inputs, mdbf as M, replicas
+    N, Mc, R, l, n_inner = admm_shape(workload)
+    n_iter = 4
+    stream = torch.cuda.Stream()
+    st = stream.cuda_stream
+    host = [torch.from_numpy(inputs.make_factor_matrix(a, b, seed=60 + i, special_values=False)).pin_memory()
+            for i, (a, b) in enumerate([(N, Mc), (Mc, R), (N, R)])]
+    Wd, Vd, U0 = (h.cuda() for h in host)
+    Ud, Ld = U0.clone(), torch.zeros_like(U0)
+    Qd = torch.from_numpy(inputs.make_start_block(R, l, seed=8)).cuda()
+    nwords = (R + 31) // 32
+    Sd = torch.zeros((N, nwords), dtype=torch.int32, device="cuda")
+    Uld = torch.zeros((N, l), dtype=torch.float32, device="cuda")
+    Vld = torch.zeros((R, l), dtype=torch.float32, device="cuda")
+    sd = torch.zeros((l,), dtype=torch.float32, device="cuda")
+    Uh, Lh, Sh = (torch.zeros_like(t, device="cpu").pin_memory() for t in (Ud, Ld, Sd))
+    ws_bytes = M.mdbf_admm_workspace_bytes(N, R, l)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    rho = float((host[1].double() ** 2).sum()) / R
+    flops = admm_flops(N, Mc, R, n_inner)
+
+    def step():
+        M.mdbf_admm_factor_update(Wd.data_ptr(), N, Mc, False, Vd.data_ptr(), R, Ud.data_ptr(), Ld.data_ptr(), rho, l, n_inner, n_iter,
+                                  Qd.data_ptr(), Sd.data_ptr(), Uld.data_ptr(), Vld.data_ptr(), sd.data_ptr(), None, ws.data_ptr(),
+                                  ws_bytes, st)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(3, warmup)):
+            step()
+        barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for (e0, e1) in ev:
+            e0.record(stream)
+            step()
+            e1.record(stream)
+        barrier()
+        clocks = sampler.stop()
+        ms = sum(e0.elapsed_time(e1) for e0, e1 in ev)
+        e2e_steps, e2e_s = max(1, min(steps, 3)), 0.0
+        if want_e2e:
+            t0 = time.perf_counter()
+            for _ in range(e2e_steps):
+                Wd.copy_(host[0], non_blocking=True); Vd.copy_(host[1], non_blocking=True); Ud.copy_(host[2], non_blocking=True)
+                Ld.zero_()
+                step()
+                Uh.copy_(Ud, non_blocking=True); Lh.copy_(Ld, non_blocking=True); Sh.copy_(Sd, non_blocking=True)
+                stream.synchronize()
+            e2e_s = time.perf_counter() - t0
+    ms_max, e2e_ms_max = replicas.max_over_ranks([ms, e2e_s * 1e3], dist, device="cuda")
+    value = replicas.aggregate_throughput(flops * steps / 1e12, world, ms_max / 1e3)
+    per_gpu = flops * steps / 1e12 / (ms_max / 1e3)
+    msvid_launches = 1 + 4 + n_iter * (6 + (1 if l <= 4 else 0)) + 2 + 5
+    out = {
+        "metric": "admm_update_TFLOPs", "value": value, "unit": "TFLOP/s", "steps": steps, "warmup": max(3, warmup),
+        "ms_per_step": ms_max / steps,
+        "config": {"workload": workload, "description": f"ADMM update of an {N} x {R} factor for a {N} x {Mc} matrix, l={l}, {n_inner} inner "
+                                                        f"iteration(s), {n_iter} subspace iterations per MSVID step; dense-algebra flops of the "
+                                                        "least-squares step (cuBLAS / cuSOLVER fp32) counted",
+                   "layers": 1, "T": 0, "weights_MB": round(N * Mc * 4 / 1e6, 1), "l2_policy": "matrices larger than L2",
+                   "launch": "stream launches", "kernel": "admm", "grouping": "one call per step", "replicas": world},
+        "e2e": ({"value": replicas.aggregate_throughput(flops * e2e_steps / 1e12, world, e2e_ms_max / 1e3), "unit": "TFLOP/s",
+                 "h2d_bytes_per_step": (N * Mc + Mc * R + N * R) * 4, "d2h_bytes_per_step": 2 * N * R * 4 + N * nwords * 4}
+                if want_e2e else None),
+        "gpu_launches": (2 + n_inner * (3 + msvid_launches)) * steps,          # this library's kernels; the libraries' are not counted
+        "clocks": clocks,
+        "roofline": {"bound": "alu", "achieved": per_gpu, "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": per_gpu / FP32_PEAK_TFLOPS,
+                     "peak_source": "derived: 148 SMs x 128 FP32 FMA lanes x 2 x 1.965 GHz", "kernel": "cuBLAS sgemm (W V), library",
+                     "traffic": None},
+    }
+    del Wd, Vd, U0, Ud, Ld, ws
+    torch.cuda.empty_cache()
+    return out, ("admm", N, Mc, R, l, n_inner)
+
+
+def cpu_baseline_admm(N, Mc, R, l, n_inner):
+    """The oracle's update (fp64, exact SVD in the prox step) on a leading block of the workload, rated in the same flops."""
+    from oracle import mdbf_oracle as orc
+    from paper_2512_24545_b200 import inputs
+    n, m, r = min(N, 1024), min(Mc, 1024), min(R, 512)
+    W, V, U = (inputs.make_factor_matrix(a, b, seed=60 + i, special_values=False) for i, (a, b) in enumerate([(n, m), (m, r), (n, r)]))
+    rho = float(np.sum(V.astype(np.float64) ** 2)) / r
+    t0 = time.perf_counter()
+    orc.admm_factor_update(W, V, U, np.zeros_like(U), rho, min(l, r), n_inner)
+    dt = time.perf_counter() - t0
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    return {"value": admm_flops(n, m, r, n_inner) / 1e12 / dt, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+            "sample": f"fp64 update of a {n} x {r} factor for a {n} x {m} block, one call, {dt:.1f} s"}
+
+
 # workloads the default line reports beside the headline one: the largest decode configuration, the MLP shapes at one
 # and at sixteen tokens, the prefill point under the library's own choice and under the expanded order (the metric's
 # own unit), the block prefill, and the quantizer's first step on a factor of the block's largest layer
@@ -578,13 +697,15 @@ def run_mdbf(args):
     torch.cuda.set_device(local)
     if args.workload.startswith("msvid"):
         main, cpu_args = measure_msvid(args.workload, args.steps, args.warmup, dist, world, local)
+    elif args.workload.startswith("admm"):
+        main, cpu_args = measure_admm(args.workload, args.steps, args.warmup, dist, world, local)
     else:
         main, cpu_args = measure(args.workload, args.kernel, args.steps, args.warmup, dist, world, local,
                                  no_graph=args.no_graph, no_siblings=args.no_siblings, copies=args.copies, fuse_block=args.fuse_block)
     out = {
         "metric": main["metric"], "value": main["value"], "unit": main["unit"], "n_gpus": world, "steps": main["steps"],
         "warmup": main["warmup"], "ms_per_step": main["ms_per_step"], "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if args.workload.startswith("msvid") else "bf16", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if args.workload.startswith(("msvid", "admm")) else "bf16", "data": "synthetic",
         "config": main["config"], "e2e": main["e2e"], "gpu_launches": main["gpu_launches"], "clocks": main["clocks"],
         "roofline": main["roofline"],
     }
@@ -604,6 +725,8 @@ def run_mdbf(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         if cpu_args[0] == "msvid":
             out["cpu_baseline"] = cpu_baseline_msvid(*cpu_args[1:])
+        elif cpu_args[0] == "admm":
+            out["cpu_baseline"] = cpu_baseline_admm(*cpu_args[1:])
         else:
             spec0, T, bound, mat0 = cpu_args
             out["cpu_baseline"] = cpu_baseline(spec0, T, bound, budget_s=20.0, mat=mat0)
@@ -686,6 +809,31 @@ def run_reference(args):
             "config": {"workload": args.workload, "description": f"MSVID_l of a {rows} x {cols} fp32 factor, l={l}"},
             "cpu_baseline": {"value": value, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        }))
+        return
+    if args.workload.startswith("admm"):
+        from oracle import mdbf_oracle as orc
+        from paper_2512_24545_b200 import inputs
+        N, Mc, R, l, n_inner = admm_shape(args.workload)
+        n, m, r = min(N, 512), min(Mc, 512), min(R, 256)
+        W, V, U = (inputs.make_factor_matrix(a, b, seed=60 + i, special_values=False) for i, (a, b) in enumerate([(n, m), (m, r), (n, r)]))
+        rho = float(np.sum(V.astype(np.float64) ** 2)) / r
+        for _ in range(args.warmup):
+            orc.admm_factor_update(W, V, U, np.zeros_like(U), rho, min(l, r), n_inner)
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            orc.admm_factor_update(W, V, U, np.zeros_like(U), rho, min(l, r), n_inner)
+        total = time.perf_counter() - t0
+        value = admm_flops(n, m, r, n_inner) / 1e12 * args.steps / total
+        sample = f"fp64 update of a {n} x {r} factor for a {n} x {m} block of the workload per step"
+        print(json.dumps({
+            "impl": "reference", "metric": "admm_update_TFLOPs", "value": value, "unit": "TFLOP/s",
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": total / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "description": f"ADMM update of an {N} x {R} factor for a {N} x {Mc} matrix, l={l}"},
+            "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         }))
         return
     groups, T, bound, desc = workload_specs(args.workload)

@@ -75,8 +75,8 @@ __global__ void sum_kernel(const float *__restrict__ Ut, const float *__restrict
     for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < count; e += (size_t)gridDim.x * blockDim.x) Z[e] = Ut[e] + Lam[e];
 }
 // U = S (.) (Ul Vl^T) entry by entry from the compact MSVID result, and Lam += U_tilde - U.
-// CTA = 8 rows x 256 columns; thread = column (its row of Vl in registers), the rows' Ul in shared memory.
-constexpr int RC_ROWS = 8, RC_COLS = 256, RC_MAXL = 32;
+// CTA = 32 rows x 256 columns; thread = column (its row of Vl in registers), the rows' Ul in shared memory.
+constexpr int RC_ROWS = 32, RC_COLS = 256, RC_MAXL = 32;
 __global__ void __launch_bounds__(RC_COLS) recon_dual_kernel(const uint32_t *__restrict__ S, const float *__restrict__ Ul,
                                                              const float *__restrict__ Vl, int l, const float *__restrict__ Ut,
                                                              float *__restrict__ U, float *__restrict__ Lam, int n, int r, int nwords) {

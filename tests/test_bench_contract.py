@@ -21,7 +21,8 @@ def run_reference(*args):
 
 
 @pytest.mark.parametrize("workload,metric,unit", [("decode_qproj", "decode_algorithmic_GBps", "GB/s"),
-                                                  ("msvid_512x384_l4", "msvid_algorithmic_GBps", "GB/s")])
+                                                  ("msvid_512x384_l4", "msvid_algorithmic_GBps", "GB/s"),
+                                                  ("admm_300x260_r64_l4", "admm_update_TFLOPs", "TFLOP/s")])
 def test_reference_arm_line(workload, metric, unit):
     d = run_reference("--workload", workload)
     assert KEYS <= set(d)
@@ -30,6 +31,15 @@ def test_reference_arm_line(workload, metric, unit):
     assert d["config"]["workload"] == workload
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and d["cpu_baseline"]["value"] == d["value"]
     assert d["e2e"] == {"value": d["value"], "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+
+
+def test_admm_flop_count_by_hand():
+    sys.path.insert(0, ROOT)
+    import bench
+    # N = 4, M = 3, R = 2, one inner iteration: W V 2*4*3*2 = 48, V^T V (a triangle) 3*2*2 = 12, Cholesky 8/3, solves 2*4*2*2 = 32
+    assert abs(bench.admm_flops(4, 3, 2, 1) - (48 + 12 + 8 / 3 + 32)) < 1e-9
+    assert abs(bench.admm_flops(4, 3, 2, 3) - (48 + 12 + 8 / 3 + 96)) < 1e-9
+    assert bench.admm_shape("admm_8192x4096_r1664_l16_in3") == (8192, 4096, 1664, 16, 3)
 
 
 def test_accounting_against_hand_counts():
