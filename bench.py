@@ -601,7 +601,7 @@ def measure_admm(workload, steps, warmup, dist, world, local, want_e2e=True):
     Vld = torch.zeros((R, l), dtype=torch.float32, device="cuda")
     sd = torch.zeros((l,), dtype=torch.float32, device="cuda")
     Uh, Lh, Sh = (torch.zeros_like(t, device="cpu").pin_memory() for t in (Ud, Ld, Sd))
-    ws_bytes = M.mdbf_admm_workspace_bytes(N, R, l)
+    ws_bytes = M.mdbf_admm_workspace_bytes(N, Mc, R, l)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     rho = float((host[1].double() ** 2).sum()) / R
     flops = admm_flops(N, Mc, R, n_inner)

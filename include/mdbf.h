@@ -346,22 +346,25 @@ mdbf_status_t mdbf_msvid_workspace_bytes(int64_t rows, int64_t cols, int32_t l, 
  *   S_packed (N x ceil(R / 32)), Ul (N x l), Vl (R x l), sigma (l)   device, written: the compact form of the new U,
  *              U = S (.) (Ul Vl^T), as mdbf_msvid returns it in the last inner iteration
  *   U_tilde    device, N x R fp32, written with the last inner iteration's least-squares iterate; may be NULL
- *   workspace  device, mdbf_admm_workspace_bytes(N, R, l) bytes on a 256-byte boundary (three N x R matrices, the R x R
- *              system and mdbf_msvid's workspace)
- * The two plain dense products and the Cholesky factorisation and solve of the R x R system are cuBLAS / cuSOLVER
- * calls in fp32; the MSVID step, the elementwise passes and the reconstruction of the dense factor fused with the
- * dual update are this library's kernels.  Asynchronous on `stream`.  The first call on a host thread creates the
- * libraries' handles and allocates the scratch the factorisation asks for (kept for later calls; a larger request
- * synchronises the stream and reallocates).  A failed factorisation (not expected for rho > 0) turns sigma into NaN.
+ *   workspace  device, mdbf_admm_workspace_bytes(N, M, R, l) bytes on a 256-byte boundary (three N x R matrices, the R x R
+ *              system, the operand images of op(W) and V - twice their size - and mdbf_msvid's workspace)
+ * The two dense products (W V, V^T V) run on the tensor cores with fp32 accuracy (TF32 operands in a three-term
+ * split, fp32 accumulation); the Cholesky factorisation and the solves of the R x R system are cuSOLVER calls in
+ * fp32; the MSVID step, the elementwise passes and the reconstruction of the dense factor fused with the dual update
+ * are this library's kernels.  Asynchronous on `stream`.  The first call on a host thread creates the solver's
+ * handles and allocates the scratch the factorisation asks for (kept for later calls; a larger request synchronises
+ * the stream and reallocates).  A failed factorisation (not expected for rho > 0) or an expired wait of a kernel turns
+ * sigma into NaN.
  * Errors: INVALID_ARG (NULL pointer, rho <= 0, counts out of range, workspace too small or misaligned), SHAPE, ARCH, CUDA. */
 mdbf_status_t mdbf_admm_factor_update(const float *W, int64_t w_rows, int64_t w_cols, int32_t transpose_w, const float *V, int64_t r,
                                       float *U, float *Lambda, float rho, int32_t l, int32_t n_inner, int32_t n_iter,
                                       const float *Q0, uint32_t *S_packed, float *Ul, float *Vl, float *sigma, float *U_tilde,
                                       void *workspace, size_t workspace_bytes, void *stream);
 
-/* Size of the workspace mdbf_admm_factor_update needs for an N x R factor (host computation, no device needed).
+/* Size of the workspace mdbf_admm_factor_update needs for an N x R factor of an N x M matrix (host computation, no device
+ * needed).
  * Errors: INVALID_ARG, SHAPE. */
-mdbf_status_t mdbf_admm_workspace_bytes(int64_t n, int64_t r, int32_t l, size_t *bytes);
+mdbf_status_t mdbf_admm_workspace_bytes(int64_t n, int64_t m, int64_t r, int32_t l, size_t *bytes);
 
 /* Test hook (no counterpart in the paper): the `nth` device allocation that the calling thread makes
  * inside this library from now on fails with MDBF_ERR_ALLOC without touching the device; nth <= 0

@@ -17,7 +17,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmdbf.so")
-SOURCES = ["mdbf_api.cu", "pack.cu", "reconstruct.cu", "forward_alu.cu", "forward_prefill.cu", "forward_tmem_t1.cu", "forward_t1.cu", "forward_static.cu", "forward_mat.cu", "msvid.cu", "admm.cu"]
+SOURCES = ["mdbf_api.cu", "pack.cu", "reconstruct.cu", "forward_alu.cu", "forward_prefill.cu", "forward_tmem_t1.cu", "forward_t1.cu", "forward_static.cu", "forward_mat.cu", "msvid.cu", "gemm3x.cu", "admm.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 STAMP = os.path.join(HERE, "libmdbf.variant")          # which variant libmdbf.so holds

@@ -7,14 +7,15 @@
 // W is N x M, V is M x R, U and Lam are N x R (dense values of the factor), all fp32 row-major on the device.  The
 // update of the other factor is the same call on the transposed problem (transpose_w).
 //
-// The two plain dense products (W V once per call, V^T V once per call) and the Cholesky factorisation and solve of
-// the R x R system are library routines (cuBLAS, cuSOLVER); everything specific to the method is this library's own:
-// the MSVID step (mdbf_msvid: sign mask + rank-l envelope on the tensor cores), the elementwise passes around it, and
-// the reconstruction of the dense factor from the compact one fused with the dual update.
+// The two dense products (W V and V^T V, once per call) run on the tensor cores with fp32 accuracy (gemm3x.cu: TF32
+// operands in a three-term split); V's operand images serve both, as the right operand of W V and as both operands of
+// V^T V.  The Cholesky factorisation and the solves of the R x R system are library routines (cuSOLVER).  Everything
+// specific to the method is this library's own: the MSVID step (mdbf_msvid: sign mask + rank-l envelope on the tensor
+// cores), the elementwise passes around it, and the reconstruction of the dense factor from the compact one fused with
+// the dual update.
 //
-// Row-major matrices are handed to the column-major libraries as their transposes: a row-major n x r matrix is a
-// column-major r x n one with leading dimension r, so that  B = W V  becomes  B^T = V^T W^T  and the solve
-// X G = T  becomes  G X^T = T^T  on the same memory.
+// Row-major matrices are handed to the column-major solver as their transposes: a row-major n x r matrix is a
+// column-major r x n one with leading dimension r, so that the solve  X G = T  becomes  G X^T = T^T  on the same memory.
 #include <cublas_v2.h>
 #include <cusolverDn.h>
 
@@ -103,19 +104,21 @@ __global__ void __launch_bounds__(RC_COLS) recon_dual_kernel(const uint32_t *__r
         Lam[at] += Ut[at] - u;
     }
 }
-// a failed factorisation (not expected: the system is positive definite for rho > 0) turns the singular values into NaN
+// a failed factorisation (not expected: the system is positive definite for rho > 0) or an expired wait of the product
+// kernel turns the singular values into NaN
 __global__ void flag_kernel(const int *__restrict__ info, float *__restrict__ sigma, int l) {
-    if (*info != 0 && threadIdx.x < l) sigma[threadIdx.x] = __int_as_float(0x7fc00000);
+    if ((info[0] != 0 || info[2] != 0) && threadIdx.x < l) sigma[threadIdx.x] = __int_as_float(0x7fc00000);
 }
 
 static size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 struct Scratch {
     float *B0, *T, *Z, *G;
-    int *info;
+    uint32_t *Wimg, *Vimg;      // operand images of op(W) (N row tiles, M deep) and of V^T (R row tiles, M deep)
+    int *info;                  // [0], [1]: the solver's; [2]: status word of the product kernel
     char *msvid;
     size_t msvid_bytes;
 };
-static mdbf_status_t carve(Scratch *w, char *base, int64_t n, int64_t r, int32_t l, size_t *total) {
+static mdbf_status_t carve(Scratch *w, char *base, int64_t n, int64_t m, int64_t r, int32_t l, size_t *total) {
     size_t msv = 0;
     mdbf_status_t rc = mdbf_msvid_workspace_bytes(n, r, l, &msv);
     if (rc) return rc;
@@ -125,9 +128,11 @@ static mdbf_status_t carve(Scratch *w, char *base, int64_t n, int64_t r, int32_t
     float *T = (float *)take((size_t)n * r * sizeof(float));
     float *Z = (float *)take((size_t)n * r * sizeof(float));
     float *G = (float *)take((size_t)r * r * sizeof(float));
-    int *info = (int *)take(sizeof(int));
-    char *m = take(msv);
-    if (w) { w->B0 = B0; w->T = T; w->Z = Z; w->G = G; w->info = info; w->msvid = m; w->msvid_bytes = msv; }
+    uint32_t *Wimg = (uint32_t *)take(gemm3x_image_bytes(n, m));
+    uint32_t *Vimg = (uint32_t *)take(gemm3x_image_bytes(r, m));
+    int *info = (int *)take(4 * sizeof(int));
+    char *mw = take(msv);
+    if (w) { w->B0 = B0; w->T = T; w->Z = Z; w->G = G; w->Wimg = Wimg; w->Vimg = Vimg; w->info = info; w->msvid = mw; w->msvid_bytes = msv; }
     *total = off;
     return MDBF_OK;
 }
@@ -148,11 +153,11 @@ static mdbf_status_t check_shape(const char *who, int64_t n, int64_t m, int64_t 
 
 using namespace mdbf;
 
-extern "C" mdbf_status_t mdbf_admm_workspace_bytes(int64_t n, int64_t r, int32_t l, size_t *bytes) {
+extern "C" mdbf_status_t mdbf_admm_workspace_bytes(int64_t n, int64_t m, int64_t r, int32_t l, size_t *bytes) {
     if (!bytes) { set_error("mdbf_admm_workspace_bytes: NULL pointer"); return MDBF_ERR_INVALID_ARG; }
-    mdbf_status_t rc = admm::check_shape("mdbf_admm_workspace_bytes", n, 1, r, l);
+    mdbf_status_t rc = admm::check_shape("mdbf_admm_workspace_bytes", n, m, r, l);
     if (rc) return rc;
-    return admm::carve(nullptr, nullptr, n, r, l, bytes);
+    return admm::carve(nullptr, nullptr, n, m, r, l, bytes);
 }
 
 extern "C" mdbf_status_t mdbf_admm_factor_update(const float *W, int64_t w_rows, int64_t w_cols, int32_t transpose_w, const float *V,
@@ -173,7 +178,7 @@ extern "C" mdbf_status_t mdbf_admm_factor_update(const float *W, int64_t w_rows,
     }
     admm::Scratch w;
     size_t need = 0;
-    rc = admm::carve(&w, (char *)workspace, n, r, l, &need);
+    rc = admm::carve(&w, (char *)workspace, n, m, r, l, &need);
     if (rc) return rc;
     if (workspace_bytes < need || ((uintptr_t)workspace & 255u) != 0) {
         set_error("%s: the workspace must hold %zu bytes (mdbf_admm_workspace_bytes) on a 256-byte boundary; got %zu at %p", who, need,
@@ -188,13 +193,14 @@ extern "C" mdbf_status_t mdbf_admm_factor_update(const float *W, int64_t w_rows,
     rc = admm::get_libs(device, st, &L);
     if (rc) return rc;
     const int ni = (int)n, mi = (int)m, ri = (int)r;
-    const float one = 1.f, zero = 0.f;
-    // B0 = op(W) V:  B0^T (r x n) = V^T (r x m, the memory of V) * op(W)^T (m x n)
-    cublasStatus_t bs = cublasSgemm(L->blas, CUBLAS_OP_N, transpose_w ? CUBLAS_OP_T : CUBLAS_OP_N, ri, ni, mi, &one, V, ri, W,
-                                    transpose_w ? ni : mi, &zero, w.B0, ri);
-    // G = V^T V (lower triangle in column-major terms) + rho I
-    if (bs == CUBLAS_STATUS_SUCCESS) bs = cublasSsyrk(L->blas, CUBLAS_FILL_MODE_LOWER, CUBLAS_OP_N, ri, mi, &one, V, ri, &zero, w.G, ri);
-    if (bs != CUBLAS_STATUS_SUCCESS) { set_error("%s: cuBLAS returned %d", who, (int)bs); return MDBF_ERR_CUDA; }
+    MDBF_CUDA(cudaMemsetAsync(w.info, 0, 4 * sizeof(int), st));
+    // images: op(W)[i][k] = W[i * w_cols + k], or W[k * w_cols + i] when transposed;  V^T[j][k] = V[k * r + j]
+    rc = transpose_w ? gemm3x_split(W, 1, (size_t)w_cols, ni, mi, w.Wimg, st) : gemm3x_split(W, (size_t)w_cols, 1, ni, mi, w.Wimg, st);
+    if (rc == MDBF_OK) rc = gemm3x_split(V, 1, (size_t)r, ri, mi, w.Vimg, st);
+    // B0 = op(W) V  and  G = V^T V (+ rho I below)
+    if (rc == MDBF_OK) rc = gemm3x_run(w.Wimg, w.Vimg, w.B0, ni, ri, mi, w.info + 2, st);
+    if (rc == MDBF_OK) rc = gemm3x_run(w.Vimg, w.Vimg, w.G, ri, ri, mi, w.info + 2, st);
+    if (rc) return rc;
     admm::ridge_kernel<<<ceil_div(ri, 256), 256, 0, st>>>(w.G, ri, rho);
     int lwork = 0;
     cusolverStatus_t ss = cusolverDnSpotrf_bufferSize(L->solver, CUBLAS_FILL_MODE_LOWER, ri, w.G, ri, &lwork);
@@ -227,7 +233,7 @@ extern "C" mdbf_status_t mdbf_admm_factor_update(const float *W, int64_t w_rows,
             S_packed, Ul, Vl, l, w.T, U, Lambda, ni, ri, nwords);
     }
     if (U_tilde) MDBF_CUDA(cudaMemcpyAsync(U_tilde, w.T, count * sizeof(float), cudaMemcpyDeviceToDevice, st));
-    admm::flag_kernel<<<1, 32, 0, st>>>(w.info, sigma, l);
+    admm::flag_kernel<<<1, 32, 0, st>>>(w.info, sigma, l);                      // the factorisation's flag or an expired wait
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }

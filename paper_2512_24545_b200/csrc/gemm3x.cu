@@ -1,0 +1,238 @@
+// Dense fp32 product C = A B on the tensor cores with fp32 accuracy: tcgen05 kind::tf32 and the three-term split
+//     a b  ~  a_hi b_hi + a_hi b_lo + a_lo b_hi          (each part a TF32 number; the dropped a_lo b_lo is below 2^-21 a b)
+// with fp32 accumulation in tensor memory.  It serves the least-squares step of the ADMM refinement (W V and V^T V,
+// Eq. admm-U-tilde), where the FP32 pipe would need five times as long.
+//
+// Two passes.  split_image_kernel turns an operand into "images": per tile of 128 rows (output rows for A, output
+// columns for B) and block of 32 contraction indices one 32 KB piece holding hi (128 rows of 32 TF32 values, 128 bytes
+// each) and lo (the same shape behind it), rows K-major with the 128B swizzle a shared-memory matrix descriptor expects
+// (16-byte chunk c of row r at position c ^ (r & 7)); tails are zero.  Either operand may be given transposed: an
+// element is read at src[i * stride_i + k * stride_k] with one of the strides equal to one.
+// gemm3x_kernel: CTA = one 128 x 128 tile of C; one lane streams the A and B pieces of each K block into a ring by
+// bulk copies, one lane issues  D1 (+)= A_hi [B_hi | B_lo]  (N = 256)  and  D2 (+)= A_lo B_hi  (N = 128), four K steps
+// of 8 each; the four epilogue warps add the three column groups and store.  CTAs that share a row tile of A are
+// neighbours in launch order, so its pieces are found in L2 by all but the first.  Every wait is bounded; on expiry the
+// status word is set and the tile is written as NaN.
+#include <algorithm>
+#include <cstdint>
+
+#include "common.cuh"
+#include "tmem_ptx.cuh"
+
+namespace mdbf {
+namespace g3x {
+
+constexpr int TILE = 128, KB = 32;
+constexpr int HALF = TILE * KB * 4;            // bytes of the hi (or lo) part of a piece
+constexpr int PIECE = 2 * HALF;                // 32 KB
+constexpr int STAGES = 3;
+constexpr int THREADS = 6 * 32;                // 4 epilogue warps, loader, issuer
+constexpr size_t SMEM = 1024 + (size_t)STAGES * 2 * PIECE;
+
+__device__ __forceinline__ void split_tf32(float v, uint32_t &hi, uint32_t &lo) {
+    hi = __float_as_uint(v) & 0xFFFFE000u;                                             // truncation: the residual is exact
+    lo = (__float_as_uint(v - __uint_as_float(hi)) + 0x1000u) & 0xFFFFE000u;           // rounded to nearest TF32
+}
+// grid: (K blocks, tiles); block 256 = 128 rows x 2 halves of the 8 chunks
+template <bool K_CONTIGUOUS>
+__global__ void __launch_bounds__(256) split_image_kernel(const float *__restrict__ src, size_t stride_i, size_t stride_k, int ni, int nk,
+                                                          int nkb, uint32_t *__restrict__ img) {
+    const int kb = blockIdx.x, it = blockIdx.y;
+    unsigned char *piece = reinterpret_cast<unsigned char *>(img) + ((size_t)it * nkb + kb) * PIECE;
+    if (K_CONTIGUOUS) {
+        // a quarter warp = one row's 128 bytes: whole-line reads, 16-byte writes that cover a row
+        const int chunk = threadIdx.x & 7;
+        for (int r = threadIdx.x >> 3; r < TILE; r += 32) {
+            const int i = it * TILE + r, k0 = kb * KB + 4 * chunk;
+            uint32_t h[4], l[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float v = (i < ni && k0 + u < nk) ? src[(size_t)i * stride_i + (size_t)(k0 + u)] : 0.f;
+                split_tf32(v, h[u], l[u]);
+            }
+            const int off = r * 128 + ((chunk ^ (r & 7)) << 4);
+            *reinterpret_cast<uint4 *>(piece + off) = make_uint4(h[0], h[1], h[2], h[3]);
+            *reinterpret_cast<uint4 *>(piece + HALF + off) = make_uint4(l[0], l[1], l[2], l[3]);
+        }
+    } else {
+        // thread = row (consecutive rows are consecutive in memory), two threads per row share its 8 chunks
+        const int r = threadIdx.x & 127, i = it * TILE + r;
+        for (int chunk = threadIdx.x >> 7; chunk < 8; chunk += 2) {
+            const int k0 = kb * KB + 4 * chunk;
+            uint32_t h[4], l[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float v = (i < ni && k0 + u < nk) ? src[(size_t)i + (size_t)(k0 + u) * stride_k] : 0.f;
+                split_tf32(v, h[u], l[u]);
+            }
+            const int off = r * 128 + ((chunk ^ (r & 7)) << 4);
+            *reinterpret_cast<uint4 *>(piece + off) = make_uint4(h[0], h[1], h[2], h[3]);
+            *reinterpret_cast<uint4 *>(piece + HALF + off) = make_uint4(l[0], l[1], l[2], l[3]);
+        }
+    }
+}
+
+__device__ __forceinline__ void umma_ss_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// instruction descriptor: fp32 accumulator, A and B TF32, both K-major, M = 128
+__device__ __forceinline__ uint32_t idesc_tf32(int n) {
+    uint32_t d = 0;
+    d |= 1u << 4;                       // D: fp32
+    d |= 2u << 7;                       // A: tf32
+    d |= 2u << 10;                      // B: tf32
+    d |= (uint32_t)(n >> 3) << 17;      // N
+    d |= (uint32_t)(128 >> 4) << 24;    // M
+    return d;
+}
+
+__global__ void __launch_bounds__(THREADS, 1) gemm3x_kernel(const uint32_t *__restrict__ Aimg, const uint32_t *__restrict__ Bimg,
+                                                            float *__restrict__ C, int n, int r, int nkb, int ntn,
+                                                            int32_t *__restrict__ status) {
+    using namespace tm;
+    extern __shared__ unsigned char g3_smem_raw[];
+    __shared__ __align__(8) uint64_t bars[2 * STAGES + 1];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag_s;
+    volatile int *abort_flag = &abort_flag_s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t smem_base = (smem_u32(g3_smem_raw) + 1023u) & ~1023u;
+    const uint32_t full_bar = smem_u32(&bars[0]), empty_bar = smem_u32(&bars[STAGES]), accum_bar = smem_u32(&bars[2 * STAGES]);
+    const int mt = blockIdx.x / ntn, nt = blockIdx.x - mt * ntn;
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar + 8 * s, 1);                      // the loader's expect_tx
+            mbar_init(empty_bar + 8 * s, 1);                     // the issuer's commit
+        }
+        mbar_init(accum_bar, 1);
+        abort_flag_s = 0;
+        fence_barrier_init();
+    }
+    if (warp == 5) {
+        tmem_alloc(smem_u32(&tmem_base_slot), 512u);             // D1: columns [0, 256), D2: [256, 384); one CTA per SM
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_slot;
+
+    if (warp < 4) {
+        // ===================================== epilogue =====================================
+        bool alive = mbar_wait(accum_bar, 0u, abort_flag, status);
+        alive = __all_sync(0xffffffffu, alive);
+        tc_fence_after();
+        const int row = mt * TILE + warp * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const bool vec = (r & 3) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0;
+#pragma unroll 1
+        for (int c = 0; c < TILE; c += 16) {
+            float y[16];
+            if (alive && nkb > 0) {
+                uint32_t d1[16], d2[16], d3[16];
+                tmem_ld16(tmem + lane_base + (uint32_t)c, d1);
+                tmem_ld16(tmem + lane_base + (uint32_t)(TILE + c), d2);
+                tmem_ld16(tmem + lane_base + (uint32_t)(2 * TILE + c), d3);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 16; ++e) y[e] = (__uint_as_float(d1[e]) + __uint_as_float(d2[e])) + __uint_as_float(d3[e]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) y[e] = alive ? 0.f : __int_as_float(0x7fc00000);
+            }
+            const int col = nt * TILE + c;
+            if (row < n) {
+                float *out = C + (size_t)row * r + col;
+                if (vec && col + 16 <= r) {
+#pragma unroll
+                    for (int e = 0; e < 16; e += 4) *reinterpret_cast<float4 *>(out + e) = make_float4(y[e], y[e + 1], y[e + 2], y[e + 3]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        if (col + e < r) out[e] = y[e];
+                }
+            }
+        }
+    } else if (warp == 4) {
+        // ====================================== loader ======================================
+        if (lane == 0) {
+            const uint32_t *a_src = Aimg + (size_t)mt * nkb * (PIECE / 4), *b_src = Bimg + (size_t)nt * nkb * (PIECE / 4);
+            bool alive = true;
+            for (int kb = 0; kb < nkb && alive; ++kb) {
+                const int s = kb % STAGES;
+                alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(kb / STAGES)) & 1u) ^ 1u, abort_flag, status);
+                if (!alive) break;
+                const uint32_t dst = smem_base + (uint32_t)(s * 2 * PIECE);
+                mbar_arrive_expect_tx(full_bar + 8 * s, (uint32_t)(2 * PIECE));
+                bulk_load(dst, a_src + (size_t)kb * (PIECE / 4), (uint32_t)PIECE, full_bar + 8 * s);
+                bulk_load(dst + (uint32_t)PIECE, b_src + (size_t)kb * (PIECE / 4), (uint32_t)PIECE, full_bar + 8 * s);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ====================================== issuer ======================================
+        if (lane == 0) {
+            const uint32_t idesc1 = idesc_tf32(2 * TILE), idesc2 = idesc_tf32(TILE);
+            bool alive = true;
+            for (int kb = 0; kb < nkb && alive; ++kb) {
+                const int s = kb % STAGES;
+                alive = mbar_wait(full_bar + 8 * s, ((uint32_t)(kb / STAGES)) & 1u, abort_flag, status);
+                if (!alive) break;
+                tc_fence_after();
+                const uint32_t stage = smem_base + (uint32_t)(s * 2 * PIECE);
+                const uint64_t a_hi = make_smem_desc(stage), a_lo = make_smem_desc(stage + (uint32_t)HALF);
+                const uint64_t b_all = make_smem_desc(stage + (uint32_t)PIECE);      // rows 0..127 = B_hi, 128..255 = B_lo
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)                   // 8 TF32 = 32 bytes per K step
+                    umma_ss_tf32(tmem, a_hi + (uint64_t)(2 * ks), b_all + (uint64_t)(2 * ks), idesc1, (kb > 0 || ks > 0) ? 1u : 0u);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_ss_tf32(tmem + (uint32_t)(2 * TILE), a_lo + (uint64_t)(2 * ks), b_all + (uint64_t)(2 * ks), idesc2,
+                                 (kb > 0 || ks > 0) ? 1u : 0u);
+                umma_commit(empty_bar + 8 * s);
+            }
+            if (alive && nkb > 0) umma_commit(accum_bar);
+            else mbar_arrive(accum_bar);
+        }
+        __syncwarp();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) drain_delay();                              // let copies in flight land before the shared memory goes back
+    if (warp == 5) tmem_dealloc(tmem, 512u);
+}
+
+}  // namespace g3x
+
+size_t gemm3x_image_bytes(int64_t rows, int64_t depth) {
+    return (size_t)ceil_div((int)rows, g3x::TILE) * (size_t)ceil_div((int)depth, g3x::KB) * g3x::PIECE;
+}
+
+// images of an operand with `rows` tile rows and `depth` contraction indices; element (i, k) at src[i * stride_i + k * stride_k]
+mdbf_status_t gemm3x_split(const float *src, size_t stride_i, size_t stride_k, int rows, int depth, uint32_t *img, cudaStream_t st) {
+    const dim3 grid(ceil_div(depth, g3x::KB), ceil_div(rows, g3x::TILE));
+    if (stride_k == 1) g3x::split_image_kernel<true><<<grid, 256, 0, st>>>(src, stride_i, stride_k, rows, depth, (int)grid.x, img);
+    else if (stride_i == 1) g3x::split_image_kernel<false><<<grid, 256, 0, st>>>(src, stride_i, stride_k, rows, depth, (int)grid.x, img);
+    else { set_error("gemm3x_split: one of the strides must be 1"); return MDBF_ERR_INVALID_ARG; }
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}
+
+// C (n x r, row-major) = A B from the operands' images (A: n rows, B: r rows, both `depth` deep)
+mdbf_status_t gemm3x_run(const uint32_t *Aimg, const uint32_t *Bimg, float *C, int n, int r, int depth, int32_t *status, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        MDBF_CUDA(cudaFuncSetAttribute(g3x::gemm3x_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g3x::SMEM));
+        attr_set = true;
+    }
+    const int ntm = ceil_div(n, g3x::TILE), ntn = ceil_div(r, g3x::TILE);
+    g3x::gemm3x_kernel<<<ntm * ntn, g3x::THREADS, g3x::SMEM, st>>>(Aimg, Bimg, C, n, r, ceil_div(depth, g3x::KB), ntn, status);
+    MDBF_CUDA(cudaGetLastError());
+    return MDBF_OK;
+}
+
+}  // namespace mdbf

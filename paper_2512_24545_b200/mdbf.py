@@ -82,7 +82,7 @@ def lib() -> ctypes.CDLL:
     L.mdbf_msvid.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     L.mdbf_project_fixed_mask.argtypes = [vp, vp, i64, i64, i32, i32, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     L.mdbf_msvid_workspace_bytes.argtypes = [i64, i64, i32, ctypes.POINTER(ctypes.c_size_t)]
-    L.mdbf_admm_workspace_bytes.argtypes = [i64, i64, i32, ctypes.POINTER(ctypes.c_size_t)]
+    L.mdbf_admm_workspace_bytes.argtypes = [i64, i64, i64, i32, ctypes.POINTER(ctypes.c_size_t)]
     L.mdbf_admm_factor_update.argtypes = [vp, i64, i64, i32, vp, i64, vp, vp, ctypes.c_float, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp,
                                           ctypes.c_size_t, vp]
     L.mdbf_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
@@ -254,9 +254,9 @@ def mdbf_project_fixed_mask(Z, S_packed, rows: int, cols: int, l: int, n_iter: i
                                          _addr(workspace), workspace_bytes, stream))
 
 
-def mdbf_admm_workspace_bytes(n: int, r: int, l: int) -> int:
+def mdbf_admm_workspace_bytes(n: int, m: int, r: int, l: int) -> int:
     v = ctypes.c_size_t()
-    _check(lib().mdbf_admm_workspace_bytes(n, r, l, ctypes.byref(v)))
+    _check(lib().mdbf_admm_workspace_bytes(n, m, r, l, ctypes.byref(v)))
     return v.value
 
 

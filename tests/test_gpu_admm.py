@@ -39,7 +39,7 @@ def run_update(W, V, U, Lam, rho, l, n_inner, n_iter, transpose=False, want_tild
     Vld = torch.zeros((R, l), dtype=torch.float32, device="cuda")
     sd = torch.zeros((l,), dtype=torch.float32, device="cuda")
     Td = torch.zeros((N, R), dtype=torch.float32, device="cuda") if want_tilde else None
-    nbytes = M.mdbf_admm_workspace_bytes(N, R, l)
+    nbytes = M.mdbf_admm_workspace_bytes(N, Wop.shape[1], R, l)
     ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
     M.mdbf_admm_factor_update(Wd.data_ptr(), W.shape[0], W.shape[1], transpose, Vd.data_ptr(), R, Ud.data_ptr(), Ld.data_ptr(), rho, l,
                               n_inner, n_iter, Qd.data_ptr(), Sd.data_ptr(), Uld.data_ptr(), Vld.data_ptr(), sd.data_ptr(),
@@ -135,7 +135,7 @@ def test_argument_errors():
     with pytest.raises(M.MdbfError):
         run_update(W, V, U, Lam, 1.0, 33, 1, 4)
     with pytest.raises(M.MdbfError):
-        M.mdbf_admm_workspace_bytes(0, 32, 4)
+        M.mdbf_admm_workspace_bytes(0, 48, 32, 4)
     d = torch.zeros(16, device="cuda")
     with pytest.raises(M.MdbfError):           # workspace too small
         M.mdbf_admm_factor_update(d.data_ptr(), 64, 48, False, d.data_ptr(), 32, d.data_ptr(), d.data_ptr(), 1.0, 4, 1, 4, d.data_ptr(),
