@@ -9,13 +9,15 @@
 //
 // The two dense products (W V and V^T V, once per call) run on the tensor cores with fp32 accuracy (gemm3x.cu: TF32
 // operands in a three-term split); V's operand images serve both, as the right operand of W V and as both operands of
-// V^T V.  The Cholesky factorisation and the solves of the R x R system are library routines (cuSOLVER).  Everything
+// V^T V.  The Cholesky factorisation of the R x R system (cuSOLVER) and one triangular solve for the factor's inverse
+// (cuBLAS) are library routines; the inverse of the system is formed and then applied, in every inner iteration, by the
+// same tensor-core product.  Everything
 // specific to the method is this library's own: the MSVID step (mdbf_msvid: sign mask + rank-l envelope on the tensor
 // cores), the elementwise passes around it, and the reconstruction of the dense factor from the compact one fused with
 // the dual update.
 //
-// Row-major matrices are handed to the column-major solver as their transposes: a row-major n x r matrix is a
-// column-major r x n one with leading dimension r, so that the solve  X G = T  becomes  G X^T = T^T  on the same memory.
+// The system is symmetric, so the column-major solver works on the row-major memory as it is; what it calls the lower
+// triangle are the rows above the diagonal here.
 #include <cublas_v2.h>
 #include <cusolverDn.h>
 
@@ -61,9 +63,28 @@ static mdbf_status_t get_libs(int device, cudaStream_t st, Libs **out) {
     return MDBF_OK;
 }
 
+// the solver's scratch, as large as the largest request so far
+static mdbf_status_t grow_scratch(Libs *L, int floats, cudaStream_t st, const char *who) {
+    if (floats <= L->potrf_floats) return MDBF_OK;
+    MDBF_CUDA(cudaStreamSynchronize(st));                         // the old scratch may still be in use
+    if (L->potrf_ws) cudaFree(L->potrf_ws);
+    L->potrf_ws = nullptr;
+    L->potrf_floats = 0;
+    if (dev_malloc(&L->potrf_ws, (size_t)floats * sizeof(float)) != cudaSuccess) {
+        set_error("%s: out of device memory for the solver's scratch (%zu bytes)", who, (size_t)floats * sizeof(float));
+        return MDBF_ERR_CUDA;
+    }
+    L->potrf_floats = floats;
+    return MDBF_OK;
+}
+
 __global__ void ridge_kernel(float *__restrict__ G, int r, float rho) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < r) G[(size_t)i * r + i] += rho;
+}
+__global__ void identity_kernel(float *__restrict__ X, int r) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x, a = blockIdx.y;
+    if (b < r) X[(size_t)a * r + b] = a == b ? 1.f : 0.f;
 }
 // T = B0 + rho (U - Lam)
 __global__ void rhs_kernel(const float *__restrict__ B0, const float *__restrict__ U, const float *__restrict__ Lam, float rho,
@@ -141,6 +162,10 @@ static mdbf_status_t check_shape(const char *who, int64_t n, int64_t m, int64_t 
         set_error("%s: sizes N=%lld M=%lld R=%lld outside the supported range", who, (long long)n, (long long)m, (long long)r);
         return MDBF_ERR_SHAPE;
     }
+    if (r > n || r > m) {
+        set_error("%s: the inner dimension R=%lld exceeds min(N, M) = min(%lld, %lld)", who, (long long)r, (long long)n, (long long)m);
+        return MDBF_ERR_SHAPE;
+    }
     if (l < 1 || l > kMaxL || l > n || l > r) {
         set_error("%s: l=%d outside [1, min(%d, N, R)]", who, l, kMaxL);
         return MDBF_ERR_SHAPE;
@@ -205,27 +230,32 @@ extern "C" mdbf_status_t mdbf_admm_factor_update(const float *W, int64_t w_rows,
     int lwork = 0;
     cusolverStatus_t ss = cusolverDnSpotrf_bufferSize(L->solver, CUBLAS_FILL_MODE_LOWER, ri, w.G, ri, &lwork);
     if (ss != CUSOLVER_STATUS_SUCCESS) { set_error("%s: cusolverDnSpotrf_bufferSize returned %d", who, (int)ss); return MDBF_ERR_CUDA; }
-    if (lwork > L->potrf_floats) {
-        MDBF_CUDA(cudaStreamSynchronize(st));                     // the old scratch may still be in use
-        if (L->potrf_ws) cudaFree(L->potrf_ws);
-        L->potrf_ws = nullptr;
-        L->potrf_floats = 0;
-        if (dev_malloc(&L->potrf_ws, (size_t)lwork * sizeof(float)) != cudaSuccess) {
-            set_error("%s: out of device memory for the factorisation's scratch (%zu bytes)", who, (size_t)lwork * sizeof(float));
-            return MDBF_ERR_CUDA;
-        }
-        L->potrf_floats = lwork;
-    }
+    rc = admm::grow_scratch(L, lwork, st, who);
+    if (rc) return rc;
     ss = cusolverDnSpotrf(L->solver, CUBLAS_FILL_MODE_LOWER, ri, w.G, ri, L->potrf_ws, L->potrf_floats, w.info);
     if (ss != CUSOLVER_STATUS_SUCCESS) { set_error("%s: cusolverDnSpotrf returned %d", who, (int)ss); return MDBF_ERR_CUDA; }
+    // (V^T V + rho I)^-1 written out, as Eq. admm-U-tilde has it: every inner iteration's solve is then one product on
+    // the tensor cores instead of two triangular solves with N right-hand sides on the FP32 pipe.  With G = L L^T:
+    // L X = I by one triangular solve (X = L^-1, column-major; read row-major it is Y = L^-T), then G^-1 = Y Y^T, a
+    // product of Y's images with themselves.  Z and the space of W's images are free at this point.
+    admm::identity_kernel<<<dim3(ceil_div(ri, 256), ri), 256, 0, st>>>(w.Z, ri);
+    const float one = 1.f;
+    cublasStatus_t bs = cublasStrsm(L->blas, CUBLAS_SIDE_LEFT, CUBLAS_FILL_MODE_LOWER, CUBLAS_OP_N, CUBLAS_DIAG_NON_UNIT, ri, ri, &one,
+                                    w.G, ri, w.Z, ri);
+    if (bs != CUBLAS_STATUS_SUCCESS) { set_error("%s: cublasStrsm returned %d", who, (int)bs); return MDBF_ERR_CUDA; }
+    rc = gemm3x_split(w.Z, (size_t)r, 1, ri, ri, w.Wimg, st);
+    if (rc == MDBF_OK) rc = gemm3x_run(w.Wimg, w.Wimg, w.G, ri, ri, ri, w.info + 2, st);
+    if (rc == MDBF_OK) rc = gemm3x_split(w.G, (size_t)r, 1, ri, ri, w.Vimg, st);   // symmetric: rows serve as columns; V's images are done with
+    if (rc) return rc;
     const size_t count = (size_t)n * r;
     const int ew_grid = (int)std::min<size_t>((count + 255) / 256, 148u * 16);
     const int nwords = (int)((r + 31) / 32);
     for (int it = 0; it < n_inner; ++it) {
         admm::rhs_kernel<<<ew_grid, 256, 0, st>>>(w.B0, U, Lambda, rho, w.T, count);
-        // U_tilde G = T  <=>  G U_tilde^T = T^T, in place on the memory of T
-        ss = cusolverDnSpotrs(L->solver, CUBLAS_FILL_MODE_LOWER, ri, ni, w.G, ri, w.T, ri, w.info + 1);
-        if (ss != CUSOLVER_STATUS_SUCCESS) { set_error("%s: cusolverDnSpotrs returned %d", who, (int)ss); return MDBF_ERR_CUDA; }
+        // U_tilde = T G^-1, over T's own memory (its images live where W's were)
+        rc = gemm3x_split(w.T, (size_t)r, 1, ni, ri, w.Wimg, st);
+        if (rc == MDBF_OK) rc = gemm3x_run(w.Wimg, w.Vimg, w.T, ni, ri, ri, w.info + 2, st);
+        if (rc) return rc;
         admm::sum_kernel<<<ew_grid, 256, 0, st>>>(w.T, Lambda, w.Z, count);
         rc = mdbf_msvid(w.Z, n, r, l, n_iter, Q0, S_packed, Ul, Vl, sigma, w.msvid, w.msvid_bytes, stream);
         if (rc) return rc;
