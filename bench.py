@@ -691,9 +691,11 @@ def cpu_baseline_admm(N, Mc, R, l, n_inner):
 
 # workloads the default line reports beside the headline one: the largest decode configuration, the MLP shapes at one
 # and at sixteen tokens, the prefill point under the library's own choice and under the expanded order (the metric's
-# own unit), the block prefill, and the quantizer's first step on a factor of the block's largest layer
+# own unit), the block prefill, the quantizer's first step on a factor of the block's largest layer and one refinement
+# update at the shape of the block's q / o projections
 ALSO = [("block70b_T1", "auto"), ("block70b_T1", "fused"), ("decode_mlp_T1", "auto"), ("decode_mlp_T16", "auto"), ("prefill_4096_l16_bpw10", "auto"),
-        ("prefill_4096_l16_bpw10", "prefill"), ("block70b_T2048", "auto"), ("msvid_28672x6016_l16", "auto")]
+        ("prefill_4096_l16_bpw10", "prefill"), ("block70b_T2048", "auto"), ("msvid_28672x6016_l16", "auto"),
+        ("admm_8192x8192_r3712_l16", "auto")]
 
 
 def run_mdbf(args):
@@ -721,6 +723,8 @@ def run_mdbf(args):
         for (wl, kern) in ALSO:
             if wl.startswith("msvid"):
                 m, _ = measure_msvid(wl, max(3, min(args.steps, 10)), args.warmup, None, 1, local, want_e2e=False, min_timed_ms=60.0)
+            elif wl.startswith("admm"):
+                m, _ = measure_admm(wl, max(3, min(args.steps, 10)), args.warmup, None, 1, local, want_e2e=False)
             else:
                 m, _ = measure(wl, "auto" if kern == "fused" else kern, max(3, min(args.steps, 10)), args.warmup, None, 1, local,
                                want_e2e=False, fuse_block=kern == "fused", min_timed_ms=60.0)

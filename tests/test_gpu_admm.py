@@ -128,6 +128,35 @@ def test_refinement_of_an_msvid_initialisation_lowers_the_objective():
     assert np.isfinite(end) and abs(end - end_o) <= 0.03 * end_o
 
 
+def test_failed_allocation_of_the_solver_scratch_is_reported_and_leaves_the_library_usable():
+    """The factorisation's scratch is the one allocation of this call (first call of a host thread).  A fresh thread with the
+    library's allocation-failure hook armed gets an error, not a fault; the same thread's next call succeeds and matches a
+    run in the main thread."""
+    import threading
+    W, V, U, Lam = problem(128, 96, 32, seed=61)
+    rho = float(np.sum(V.astype(np.float64) ** 2)) / 32
+    ref = run_update(W, V, U, Lam, rho, 4, 1, 6)
+    out = {}
+
+    def worker():
+        torch.cuda.set_device(0)
+        M.mdbf_debug_fail_alloc(1)
+        try:
+            run_update(W, V, U, Lam, rho, 4, 1, 6)
+            out["first"] = "no error"
+        except M.MdbfError as e:
+            out["first"] = str(e)
+        finally:
+            M.mdbf_debug_fail_alloc(0)
+        out["second"] = run_update(W, V, U, Lam, rho, 4, 1, 6)
+    t = threading.Thread(target=worker)
+    t.start()
+    t.join()
+    assert "out of device memory" in out["first"], out["first"]
+    np.testing.assert_array_equal(out["second"]["tilde"], ref["tilde"])
+    np.testing.assert_array_equal(out["second"]["S"], ref["S"])
+
+
 def test_argument_errors():
     W, V, U, Lam = problem(64, 48, 32, seed=3)
     with pytest.raises(M.MdbfError):
