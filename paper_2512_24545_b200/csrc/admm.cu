@@ -158,7 +158,7 @@ static mdbf_status_t carve(Scratch *w, char *base, int64_t n, int64_t m, int64_t
     return MDBF_OK;
 }
 static mdbf_status_t check_shape(const char *who, int64_t n, int64_t m, int64_t r, int32_t l) {
-    if (n < 1 || m < 1 || r < 1 || n > (1 << 24) || m > (1 << 24) || r > 32768 || n * r > (1LL << 31) - 1 || n * m > (1LL << 40)) {
+    if (n < 1 || m < 1 || r < 1 || n > (1 << 21) || m > (1 << 21) || r > 32768 || n * r > (1LL << 31) - 1 || n * m > (1LL << 40)) {   // grid limits of the tiled kernels
         set_error("%s: sizes N=%lld M=%lld R=%lld outside the supported range", who, (long long)n, (long long)m, (long long)r);
         return MDBF_ERR_SHAPE;
     }

@@ -224,11 +224,8 @@ mdbf_status_t gemm3x_split(const float *src, size_t stride_i, size_t stride_k, i
 
 // C (n x r, row-major) = A B from the operands' images (A: n rows, B: r rows, both `depth` deep)
 mdbf_status_t gemm3x_run(const uint32_t *Aimg, const uint32_t *Bimg, float *C, int n, int r, int depth, int32_t *status, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        MDBF_CUDA(cudaFuncSetAttribute(g3x::gemm3x_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g3x::SMEM));
-        attr_set = true;
-    }
+    static PerDeviceOnce once;
+    if (once.first()) MDBF_CUDA(cudaFuncSetAttribute(g3x::gemm3x_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g3x::SMEM));
     const int ntm = ceil_div(n, g3x::TILE), ntn = ceil_div(r, g3x::TILE);
     g3x::gemm3x_kernel<<<ntm * ntn, g3x::THREADS, g3x::SMEM, st>>>(Aimg, Bimg, C, n, r, ceil_div(depth, g3x::KB), ntn, status);
     MDBF_CUDA(cudaGetLastError());

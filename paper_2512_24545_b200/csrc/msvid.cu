@@ -880,11 +880,10 @@ template <int LP, bool MASKED, bool TRANS, bool WRITE_MASK = false>
 static mdbf_status_t tc_product(const ZMaps &zm, int p, int q, const uint32_t *S, int nwords, Scratch &w,
                                 cudaStream_t st, int *parts_out, uint32_t *S_out = nullptr) {
     using C = TcCfg<LP>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        MDBF_CUDA(cudaFuncSetAttribute(envelope_product_tc_kernel<LP, MASKED, TRANS, WRITE_MASK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM));
-        attr_set = true;
-    }
+    static PerDeviceOnce once;
+    if (once.first())
+        MDBF_CUDA(cudaFuncSetAttribute(envelope_product_tc_kernel<LP, MASKED, TRANS, WRITE_MASK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)C::SMEM));
     const int m_ext = TRANS ? q : p, k_ext = TRANS ? p : q;
     int kb_per_cta = 0;
     const int parts = tc_split(m_ext, k_ext, LP, &kb_per_cta);
