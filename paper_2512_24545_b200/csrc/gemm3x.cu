@@ -8,11 +8,11 @@
 // each) and lo (the same shape behind it), rows K-major with the 128B swizzle a shared-memory matrix descriptor expects
 // (16-byte chunk c of row r at position c ^ (r & 7)); tails are zero.  Either operand may be given transposed: an
 // element is read at src[i * stride_i + k * stride_k] with one of the strides equal to one.
-// gemm3x_kernel: CTA = one 128 x 128 tile of C; one lane streams the A and B pieces of each K block into a ring by
-// bulk copies, one lane issues  D1 (+)= A_hi [B_hi | B_lo]  (N = 256)  and  D2 (+)= A_lo B_hi  (N = 128), four K steps
-// of 8 each; the four epilogue warps add the three column groups and store.  CTAs that share a row tile of A are
-// neighbours in launch order, so its pieces are found in L2 by all but the first.  Every wait is bounded; on expiry the
-// status word is set and the tile is written as NaN.
+// gemm3x_kernel: one CTA per SM walks over 128 x 256 tiles of C (two column tiles of B side by side: the stream from L2
+// into shared memory, 96 KB per K block, is what bounds the kernel, and a wider tile spends less of it per flop); one
+// lane streams the pieces of each K block into a ring by bulk copies, one lane issues  D (+)= A_hi B_hi, D += A_hi B_lo,
+// D += A_lo B_hi  (N = 256, four K steps of 8 each), the four epilogue warps read the accumulator and store.  Every wait is bounded; on expiry the status word is
+// set and the tiles still to be written come out as NaN.
 #include <algorithm>
 #include <cstdint>
 
@@ -25,9 +25,10 @@ namespace g3x {
 constexpr int TILE = 128, KB = 32;
 constexpr int HALF = TILE * KB * 4;            // bytes of the hi (or lo) part of a piece
 constexpr int PIECE = 2 * HALF;                // 32 KB
-constexpr int STAGES = 3;
+constexpr int STAGES = 2;
+constexpr int STAGE_BYTES = 3 * PIECE;         // A piece, then B_hi of two column tiles, then their B_lo
 constexpr int THREADS = 6 * 32;                // 4 epilogue warps, loader, issuer
-constexpr size_t SMEM = 1024 + (size_t)STAGES * 2 * PIECE;
+constexpr size_t SMEM = 1024 + (size_t)STAGES * STAGE_BYTES;
 
 __device__ __forceinline__ void split_tf32(float v, uint32_t &hi, uint32_t &lo) {
     hi = __float_as_uint(v) & 0xFFFFE000u;                                             // truncation: the residual is exact
@@ -90,30 +91,38 @@ __device__ __forceinline__ uint32_t idesc_tf32(int n) {
     return d;
 }
 
+// Persistent: CTA c takes the tiles c, c + gridDim.x, ... (row tile = t / ntn2, so that CTAs running side by side share
+// their pieces of A in L2).  Two accumulators of 256 tensor-memory columns alternate between tiles: the epilogue of
+// one tile runs under the products of the next.  All three terms of a tile accumulate into the same columns.  ntn is
+// the number of 128-column tiles of B's images, ntn2 = ceil(ntn / 2) the number of tiles here; an odd last tile has no
+// second half: nothing is copied for it, the products read whatever the buffer holds, and nothing of it is stored.
 __global__ void __launch_bounds__(THREADS, 1) gemm3x_kernel(const uint32_t *__restrict__ Aimg, const uint32_t *__restrict__ Bimg,
-                                                            float *__restrict__ C, int n, int r, int nkb, int ntn,
+                                                            float *__restrict__ C, int n, int r, int nkb, int ntn, int ntn2, int ntiles,
                                                             int32_t *__restrict__ status) {
     using namespace tm;
     extern __shared__ unsigned char g3_smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * STAGES + 1];
+    __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
     volatile int *abort_flag = &abort_flag_s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = (smem_u32(g3_smem_raw) + 1023u) & ~1023u;
-    const uint32_t full_bar = smem_u32(&bars[0]), empty_bar = smem_u32(&bars[STAGES]), accum_bar = smem_u32(&bars[2 * STAGES]);
-    const int mt = blockIdx.x / ntn, nt = blockIdx.x - mt * ntn;
+    const uint32_t full_bar = smem_u32(&bars[0]), empty_bar = smem_u32(&bars[STAGES]);
+    const uint32_t acc_full = smem_u32(&bars[2 * STAGES]), acc_empty = smem_u32(&bars[2 * STAGES + 2]);
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar + 8 * s, 1);                      // the loader's expect_tx
             mbar_init(empty_bar + 8 * s, 1);                     // the issuer's commit
         }
-        mbar_init(accum_bar, 1);
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(acc_full + 8 * a, 1);                      // the issuer's commit after a tile's last K block
+            mbar_init(acc_empty + 8 * a, 128);                   // every epilogue thread, once it has read its row
+        }
         abort_flag_s = 0;
         fence_barrier_init();
     }
     if (warp == 5) {
-        tmem_alloc(smem_u32(&tmem_base_slot), 512u);             // D1: columns [0, 256), D2: [256, 384); one CTA per SM
+        tmem_alloc(smem_u32(&tmem_base_slot), 512u);             // two accumulators of 256 columns; one CTA per SM
         tmem_relinquish();
     }
     tc_fence_before();
@@ -123,80 +132,107 @@ __global__ void __launch_bounds__(THREADS, 1) gemm3x_kernel(const uint32_t *__re
 
     if (warp < 4) {
         // ===================================== epilogue =====================================
-        bool alive = mbar_wait(accum_bar, 0u, abort_flag, status);
-        alive = __all_sync(0xffffffffu, alive);
-        tc_fence_after();
-        const int row = mt * TILE + warp * 32 + lane;
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         const bool vec = (r & 3) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0;
+        bool alive = true;
+        int it = 0;
+        for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
+            const int as = it & 1;
+            const int mt = t / ntn2, nt2 = t - mt * ntn2;
+            if (alive) alive = mbar_wait(acc_full + 8 * as, ((uint32_t)(it >> 1)) & 1u, abort_flag, status);
+            alive = __all_sync(0xffffffffu, alive);
+            tc_fence_after();
+            const int row = mt * TILE + warp * 32 + lane;
 #pragma unroll 1
-        for (int c = 0; c < TILE; c += 16) {
-            float y[16];
-            if (alive && nkb > 0) {
-                uint32_t d1[16], d2[16], d3[16];
-                tmem_ld16(tmem + lane_base + (uint32_t)c, d1);
-                tmem_ld16(tmem + lane_base + (uint32_t)(TILE + c), d2);
-                tmem_ld16(tmem + lane_base + (uint32_t)(2 * TILE + c), d3);
-                tmem_ld_wait();
+            for (int c = 0; c < 2 * TILE; c += 16) {
+                if (nt2 * 2 * TILE + c >= r) break;                  // past the last column (the same for the whole warp)
+                float y[16];
+                if (alive && nkb > 0) {
+                    uint32_t d[16];
+                    tmem_ld16(tmem + lane_base + (uint32_t)(as * 2 * TILE + c), d);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int e = 0; e < 16; ++e) y[e] = (__uint_as_float(d1[e]) + __uint_as_float(d2[e])) + __uint_as_float(d3[e]);
-            } else {
-#pragma unroll
-                for (int e = 0; e < 16; ++e) y[e] = alive ? 0.f : __int_as_float(0x7fc00000);
-            }
-            const int col = nt * TILE + c;
-            if (row < n) {
-                float *out = C + (size_t)row * r + col;
-                if (vec && col + 16 <= r) {
-#pragma unroll
-                    for (int e = 0; e < 16; e += 4) *reinterpret_cast<float4 *>(out + e) = make_float4(y[e], y[e + 1], y[e + 2], y[e + 3]);
+                    for (int e = 0; e < 16; ++e) y[e] = __uint_as_float(d[e]);
                 } else {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e)
-                        if (col + e < r) out[e] = y[e];
+                    for (int e = 0; e < 16; ++e) y[e] = alive ? 0.f : __int_as_float(0x7fc00000);
+                }
+                const int col = nt2 * 2 * TILE + c;
+                if (row < n) {
+                    float *out = C + (size_t)row * r + col;
+                    if (vec && col + 16 <= r) {
+#pragma unroll
+                        for (int e = 0; e < 16; e += 4) *reinterpret_cast<float4 *>(out + e) = make_float4(y[e], y[e + 1], y[e + 2], y[e + 3]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e)
+                            if (col + e < r) out[e] = y[e];
+                    }
                 }
             }
+            tc_fence_before();
+            if (alive) mbar_arrive(acc_empty + 8 * as);           // the accumulator may be overwritten
         }
     } else if (warp == 4) {
         // ====================================== loader ======================================
         if (lane == 0) {
-            const uint32_t *a_src = Aimg + (size_t)mt * nkb * (PIECE / 4), *b_src = Bimg + (size_t)nt * nkb * (PIECE / 4);
             bool alive = true;
-            for (int kb = 0; kb < nkb && alive; ++kb) {
-                const int s = kb % STAGES;
-                alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(kb / STAGES)) & 1u) ^ 1u, abort_flag, status);
-                if (!alive) break;
-                const uint32_t dst = smem_base + (uint32_t)(s * 2 * PIECE);
-                mbar_arrive_expect_tx(full_bar + 8 * s, (uint32_t)(2 * PIECE));
-                bulk_load(dst, a_src + (size_t)kb * (PIECE / 4), (uint32_t)PIECE, full_bar + 8 * s);
-                bulk_load(dst + (uint32_t)PIECE, b_src + (size_t)kb * (PIECE / 4), (uint32_t)PIECE, full_bar + 8 * s);
+            int g = 0;                                           // K blocks issued so far, over all of this CTA's tiles
+            for (int t = blockIdx.x; t < ntiles && alive; t += gridDim.x) {
+                const int mt = t / ntn2, nt2 = t - mt * ntn2;
+                const bool two = 2 * nt2 + 1 < ntn;              // the tile has a second column tile
+                const uint32_t *a_src = Aimg + (size_t)mt * nkb * (PIECE / 4);
+                const uint32_t *b0_src = Bimg + (size_t)(2 * nt2) * nkb * (PIECE / 4), *b1_src = b0_src + (size_t)nkb * (PIECE / 4);
+                for (int kb = 0; kb < nkb && alive; ++kb, ++g) {
+                    const int s = g % STAGES;
+                    alive = mbar_wait(empty_bar + 8 * s, (((uint32_t)(g / STAGES)) & 1u) ^ 1u, abort_flag, status);
+                    if (!alive) break;
+                    const uint32_t dst = smem_base + (uint32_t)(s * STAGE_BYTES);
+                    mbar_arrive_expect_tx(full_bar + 8 * s, (uint32_t)(two ? 3 * PIECE : 2 * PIECE));
+                    bulk_load(dst, a_src + (size_t)kb * (PIECE / 4), (uint32_t)PIECE, full_bar + 8 * s);
+                    const uint32_t *b0 = b0_src + (size_t)kb * (PIECE / 4), *b1 = b1_src + (size_t)kb * (PIECE / 4);
+                    bulk_load(dst + (uint32_t)PIECE, b0, (uint32_t)HALF, full_bar + 8 * s);                          // B_hi, first 128 rows
+                    bulk_load(dst + (uint32_t)(2 * PIECE), b0 + HALF / 4, (uint32_t)HALF, full_bar + 8 * s);         // B_lo, first 128 rows
+                    if (two) {
+                        bulk_load(dst + (uint32_t)(PIECE + HALF), b1, (uint32_t)HALF, full_bar + 8 * s);             // B_hi, rows 128..255
+                        bulk_load(dst + (uint32_t)(2 * PIECE + HALF), b1 + HALF / 4, (uint32_t)HALF, full_bar + 8 * s);
+                    }
+                }
             }
         }
         __syncwarp();
     } else {
         // ====================================== issuer ======================================
         if (lane == 0) {
-            const uint32_t idesc1 = idesc_tf32(2 * TILE), idesc2 = idesc_tf32(TILE);
+            const uint32_t idesc = idesc_tf32(2 * TILE);
             bool alive = true;
-            for (int kb = 0; kb < nkb && alive; ++kb) {
-                const int s = kb % STAGES;
-                alive = mbar_wait(full_bar + 8 * s, ((uint32_t)(kb / STAGES)) & 1u, abort_flag, status);
+            int g = 0, it = 0;
+            for (int t = blockIdx.x; t < ntiles && alive; t += gridDim.x, ++it) {
+                const int as = it & 1;
+                alive = mbar_wait(acc_empty + 8 * as, (((uint32_t)(it >> 1)) & 1u) ^ 1u, abort_flag, status);
                 if (!alive) break;
                 tc_fence_after();
-                const uint32_t stage = smem_base + (uint32_t)(s * 2 * PIECE);
-                const uint64_t a_hi = make_smem_desc(stage), a_lo = make_smem_desc(stage + (uint32_t)HALF);
-                const uint64_t b_all = make_smem_desc(stage + (uint32_t)PIECE);      // rows 0..127 = B_hi, 128..255 = B_lo
+                const uint32_t d = tmem + (uint32_t)(as * 2 * TILE);
+                for (int kb = 0; kb < nkb && alive; ++kb, ++g) {
+                    const int s = g % STAGES;
+                    alive = mbar_wait(full_bar + 8 * s, ((uint32_t)(g / STAGES)) & 1u, abort_flag, status);
+                    if (!alive) break;
+                    tc_fence_after();
+                    const uint32_t stage = smem_base + (uint32_t)(s * STAGE_BYTES);
+                    const uint64_t a_hi = make_smem_desc(stage), a_lo = make_smem_desc(stage + (uint32_t)HALF);
+                    const uint64_t b_hi = make_smem_desc(stage + (uint32_t)PIECE), b_lo = make_smem_desc(stage + (uint32_t)(2 * PIECE));
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)                   // 8 TF32 = 32 bytes per K step
-                    umma_ss_tf32(tmem, a_hi + (uint64_t)(2 * ks), b_all + (uint64_t)(2 * ks), idesc1, (kb > 0 || ks > 0) ? 1u : 0u);
+                    for (int ks = 0; ks < 4; ++ks)               // 8 TF32 = 32 bytes per K step
+                        umma_ss_tf32(d, a_hi + (uint64_t)(2 * ks), b_hi + (uint64_t)(2 * ks), idesc, (kb > 0 || ks > 0) ? 1u : 0u);
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_ss_tf32(tmem + (uint32_t)(2 * TILE), a_lo + (uint64_t)(2 * ks), b_all + (uint64_t)(2 * ks), idesc2,
-                                 (kb > 0 || ks > 0) ? 1u : 0u);
-                umma_commit(empty_bar + 8 * s);
+                    for (int ks = 0; ks < 4; ++ks) umma_ss_tf32(d, a_hi + (uint64_t)(2 * ks), b_lo + (uint64_t)(2 * ks), idesc, 1u);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) umma_ss_tf32(d, a_lo + (uint64_t)(2 * ks), b_hi + (uint64_t)(2 * ks), idesc, 1u);
+                    umma_commit(empty_bar + 8 * s);
+                }
+                if (alive && nkb > 0) umma_commit(acc_full + 8 * as);
+                else mbar_arrive(acc_full + 8 * as);
             }
-            if (alive && nkb > 0) umma_commit(accum_bar);
-            else mbar_arrive(accum_bar);
         }
         __syncwarp();
     }
@@ -227,7 +263,18 @@ mdbf_status_t gemm3x_run(const uint32_t *Aimg, const uint32_t *Bimg, float *C, i
     static PerDeviceOnce once;
     if (once.first()) MDBF_CUDA(cudaFuncSetAttribute(g3x::gemm3x_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g3x::SMEM));
     const int ntm = ceil_div(n, g3x::TILE), ntn = ceil_div(r, g3x::TILE);
-    g3x::gemm3x_kernel<<<ntm * ntn, g3x::THREADS, g3x::SMEM, st>>>(Aimg, Bimg, C, n, r, ceil_div(depth, g3x::KB), ntn, status);
+    static int sms_of_device[64] = {};
+    int dev = 0, sms = 0;
+    MDBF_CUDA(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < 64 && sms_of_device[dev]) {
+        sms = sms_of_device[dev];
+    } else {
+        MDBF_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        if (dev >= 0 && dev < 64) sms_of_device[dev] = sms;
+    }
+    const int ntn2 = ceil_div(ntn, 2), ntiles = ntm * ntn2;
+    g3x::gemm3x_kernel<<<std::min(ntiles, sms), g3x::THREADS, g3x::SMEM, st>>>(Aimg, Bimg, C, n, r, ceil_div(depth, g3x::KB), ntn, ntn2,
+                                                                              ntiles, status);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
 }
