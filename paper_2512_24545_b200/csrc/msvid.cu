@@ -610,11 +610,13 @@ __global__ void __launch_bounds__(256) gram_finish_kernel(float *__restrict__ A,
     __threadfence();
     for (int pr = threadIdx.x; pr < LP * LP; pr += 256) {
         double s[4] = {0.0, 0.0, 0.0, 0.0};
-#pragma unroll 4
-        for (int c = 0; c < (int)gridDim.x; c += 4)
+        for (int c = 0; c < (int)gridDim.x; c += 16) {           // sixteen loads in flight, added in the order of c
+            double v[16];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (c + u < (int)gridDim.x) s[u] += __ldcg(Gp + (size_t)(c + u) * LP * LP + pr);
+            for (int u = 0; u < 16; ++u) v[u] = c + u < (int)gridDim.x ? __ldcg(Gp + (size_t)(c + u) * LP * LP + pr) : 0.0;
+#pragma unroll
+            for (int u = 0; u < 16; ++u) s[u & 3] += v[u];
+        }
         const double total = (s[0] + s[1]) + (s[2] + s[3]);
         if (CHOL) Gm[pr / LP][pr % LP] = total;
         else Gs[pr] = total;
