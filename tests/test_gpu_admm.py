@@ -169,3 +169,28 @@ def test_argument_errors():
     with pytest.raises(M.MdbfError):           # workspace too small
         M.mdbf_admm_factor_update(d.data_ptr(), 64, 48, False, d.data_ptr(), 32, d.data_ptr(), d.data_ptr(), 1.0, 4, 1, 4, d.data_ptr(),
                                   d.data_ptr(), d.data_ptr(), d.data_ptr(), d.data_ptr(), None, d.data_ptr(), 64, 0)
+
+
+def test_bench_size_update_on_sampled_rows():
+    """The shape bench.py times (N = M = 8192, R = 3712, l = 16): the least-squares iterate of sampled rows against the
+    definition evaluated in fp64 (Eq. admm-U-tilde row by row: a row of U_tilde depends on its rows of W, U and Lambda and
+    on V only), the mask of those rows, and the identities that tie the outputs together."""
+    N, Mc, R, l = 8192, 8192, 3712, 16
+    W, V, U = (inputs.make_factor_matrix(a, b, seed=60 + i, special_values=False) for i, (a, b) in enumerate([(N, Mc), (Mc, R), (N, R)]))
+    Lam = (0.1 * inputs.make_factor_matrix(N, R, seed=63, special_values=False)).astype(np.float32)
+    V64 = V.astype(np.float64)
+    rho = float(np.sum(V64 ** 2)) / R
+    g = run_update(W, V, U, Lam, rho, l, 1, 4)
+    rows = np.random.default_rng(5).choice(N, size=24, replace=False)
+    G = V64.T @ V64 + rho * np.eye(R)
+    rhs = W[rows].astype(np.float64) @ V64 + rho * (U[rows].astype(np.float64) - Lam[rows].astype(np.float64))
+    tilde_ref = np.linalg.solve(G, rhs.T).T
+    scale = np.max(np.abs(tilde_ref))
+    assert np.max(np.abs(g["tilde"][rows] - tilde_ref)) <= 2e-4 * scale
+    Z = tilde_ref + Lam[rows].astype(np.float64)
+    Sg = orc.unpack_signs(g["S"][rows], R)
+    clear = np.abs(Z) > 5e-4 * scale
+    np.testing.assert_array_equal(Sg[clear], np.where(Z >= 0, 1, -1)[clear])
+    np.testing.assert_allclose(g["U"][rows], Sg * (g["Ul"][rows] @ g["Vl"].T), atol=2e-5 * scale)
+    np.testing.assert_allclose(g["Lam"][rows], Lam[rows].astype(np.float64) + g["tilde"][rows] - g["U"][rows], atol=2e-5 * scale)
+    assert np.all(np.isfinite(g["sigma"])) and np.all(np.diff(g["sigma"]) <= 1e-6 * g["sigma"][0])

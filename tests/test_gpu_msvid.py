@@ -76,6 +76,32 @@ def test_sign_mask_exact_and_envelope_near_the_optimum(shape, l):
     np.testing.assert_allclose(np.linalg.norm(V, axis=0), np.sqrt(s), rtol=2e-4)
 
 
+def test_bench_size_factor_properties():
+    """The factor bench.py times (28672 x 6016, l = 16, four iterations), too large for a full SVD in the test: the mask of
+    sampled rows bit for bit, and what holds for the result at any size - singular values in descending order, balanced
+    column norms, and the residual of every sampled row orthogonal to the right factors (U is the product of |Z| with an
+    orthonormal basis of V's range, so (|z_i| - u_i V^T) V = 0 up to rounding), which pins the last pass over Z."""
+    rows, cols, l = 28672, 6016, 16
+    Z = inputs.make_factor_matrix(rows, cols, seed=8)
+    Sp, U, V, s = run_msvid(Z, l, n_iter=4, seed=8)
+    pick = np.random.default_rng(3).choice(rows, size=64, replace=False)
+    np.testing.assert_array_equal(Sp[pick], orc.pack_signs(np.where(Z[pick] >= 0, 1, -1).astype(np.int8)))
+    assert np.all(np.isfinite(s)) and np.all(np.diff(s) <= 1e-6 * s[0]) and s[-1] > 0
+    np.testing.assert_allclose(np.linalg.norm(U, axis=0), np.sqrt(s), rtol=5e-4)
+    np.testing.assert_allclose(np.linalg.norm(V, axis=0), np.sqrt(s), rtol=5e-4)
+    E = np.abs(Z[pick].astype(np.float64))
+    resid = E - U[pick] @ V.T
+    assert np.max(np.abs(resid @ V)) <= 2e-4 * np.max(np.abs(E @ V))
+    # the leading singular value against a few steps of the power method in fp64 on a block of rows is a lower bound check:
+    # sigma_1 of the whole matrix is at least that of any block of its rows
+    blk = np.abs(Z[:2048].astype(np.float64))
+    v = np.ones(cols) / np.sqrt(cols)
+    for _ in range(6):
+        v = blk.T @ (blk @ v)
+        v /= np.linalg.norm(v)
+    assert s[0] >= np.linalg.norm(blk @ v) * (1 - 1e-6)
+
+
 def test_tensor_core_and_scalar_products_agree():
     """The same matrix at a 16-byte aligned address (tensor-core products, three-term TF32 split) and four bytes further on
     (the scalar fp32 kernels): the same mask, and singular values that agree to fp32 accuracy."""
