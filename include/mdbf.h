@@ -307,7 +307,8 @@ mdbf_status_t mdbf_poll_status(mdbf_handle_t h, int32_t *device_status);
  *             call (the two blocks, the partial sums of a product - up to 16 per output row - and operand images:
  *             ask mdbf_msvid_workspace_bytes); free again when the stream has passed it
  * The truncated SVD is computed by block subspace iteration, not to machine precision: see n_iter.  The two products
- * with |Z| run on the tensor cores (TF32 operands in a three-term split that keeps fp32 accuracy, fp32 accumulation)
+ * with |Z| run on the tensor cores (TF32 operands in a three-term split, fp32 accumulation; within a few 1e-6 of the
+ * scalar fp32 kernels' results)
  * when cols is a multiple of 4 and Z sits on a 16-byte boundary, else in scalar fp32 kernels; the small Gram matrices
  * are fp64.  Results do not depend on scheduling (no floating-point atomics).  Asynchronous on `stream`; allocates
  * nothing and does not synchronise.  Should one of the kernel's bounded waits expire (not expected), the outputs are
@@ -348,8 +349,9 @@ mdbf_status_t mdbf_msvid_workspace_bytes(int64_t rows, int64_t cols, int32_t l, 
  *   U_tilde    device, N x R fp32, written with the last inner iteration's least-squares iterate; may be NULL
  *   workspace  device, mdbf_admm_workspace_bytes(N, M, R, l) bytes on a 256-byte boundary (three N x R matrices, the R x R
  *              system, the operand images of op(W) and V - twice their size - and mdbf_msvid's workspace)
- * The two dense products (W V, V^T V) run on the tensor cores with fp32 accuracy (TF32 operands in a three-term
- * split, fp32 accumulation); the Cholesky factorisation and the solves of the R x R system are cuSOLVER calls in
+ * The dense products (W V, V^T V, the inverse of the system and its application) run on the tensor cores (TF32
+ * operands in a three-term split, fp32 accumulation in chunks of 512 contraction indices; U_tilde comes out within about
+ * 1e-5 of its largest entry of the exact result); the Cholesky factorisation and the solves of the R x R system are cuSOLVER calls in
  * fp32; the MSVID step, the elementwise passes and the reconstruction of the dense factor fused with the dual update
  * are this library's kernels.  Asynchronous on `stream`.  The first call on a host thread creates the solver's
  * handles and allocates the scratch the factorisation asks for (kept for later calls; a larger request synchronises

@@ -1,5 +1,5 @@
 // Dense fp32 product C = A B on the tensor cores with fp32 accuracy: tcgen05 kind::tf32 and the three-term split
-//     a b  ~  a_hi b_hi + a_hi b_lo + a_lo b_hi          (each part a TF32 number; the dropped a_lo b_lo is below 2^-21 a b)
+//     a b  ~  a_hi b_hi + a_hi b_lo + a_lo b_hi          (each part a TF32 number; the dropped a_lo b_lo is below 2^-24 a b)
 // with fp32 accumulation in tensor memory.  It serves the least-squares step of the ADMM refinement (W V and V^T V,
 // Eq. admm-U-tilde), where the FP32 pipe would need five times as long.
 //
@@ -26,13 +26,17 @@ constexpr int TILE = 128, KB = 32;
 constexpr int HALF = TILE * KB * 4;            // bytes of the hi (or lo) part of a piece
 constexpr int PIECE = 2 * HALF;                // 32 KB
 constexpr int STAGES = 2;
+constexpr int KCHUNK = 16;                     // K blocks accumulated in tensor memory before the sum moves to fp32 registers
 constexpr int STAGE_BYTES = 3 * PIECE;         // A piece, then B_hi of two column tiles, then their B_lo
 constexpr int THREADS = 6 * 32;                // 4 epilogue warps, loader, issuer
 constexpr size_t SMEM = 1024 + (size_t)STAGES * STAGE_BYTES;
 
+// hi = v rounded to the nearest TF32 number (half-ulp add on the bits; the top binade is truncated so that nothing rounds
+// up to infinity), lo = the exact residual rounded the same way
 __device__ __forceinline__ void split_tf32(float v, uint32_t &hi, uint32_t &lo) {
-    hi = __float_as_uint(v) & 0xFFFFE000u;                                             // truncation: the residual is exact
-    lo = (__float_as_uint(v - __uint_as_float(hi)) + 0x1000u) & 0xFFFFE000u;           // rounded to nearest TF32
+    const uint32_t b = __float_as_uint(v);
+    hi = ((b & 0x7F000000u) == 0x7F000000u ? b : b + 0x1000u) & 0xFFFFE000u;
+    lo = (__float_as_uint(v - __uint_as_float(hi)) + 0x1000u) & 0xFFFFE000u;
 }
 // grid: (K blocks, tiles); block 256 = 128 rows x 2 halves of the 8 chunks
 template <bool K_CONTIGUOUS>
@@ -93,7 +97,10 @@ __device__ __forceinline__ uint32_t idesc_tf32(int n) {
 
 // Persistent: CTA c takes the tiles c, c + gridDim.x, ... (row tile = t / ntn2, so that CTAs running side by side share
 // their pieces of A in L2).  Two accumulators of 256 tensor-memory columns alternate between tiles: the epilogue of
-// one tile runs under the products of the next.  All three terms of a tile accumulate into the same columns.  ntn is
+// one tile runs under the products of the next.  All three terms of a tile accumulate into the same columns, for KCHUNK
+// K blocks at a time: the tensor core's accumulation is not rounded to nearest, and its one-sided error grows with the
+// number of accumulations (5e-5 of the result over 8192 contraction indices, measured); the chunks' sums are added in
+// fp32 by the epilogue, through C.  ntn is
 // the number of 128-column tiles of B's images, ntn2 = ceil(ntn / 2) the number of tiles here; an odd last tile has no
 // second half: nothing is copied for it, the products read whatever the buffer holds, and nothing of it is stored.
 __global__ void __launch_bounds__(THREADS, 1) gemm3x_kernel(const uint32_t *__restrict__ Aimg, const uint32_t *__restrict__ Bimg,
@@ -136,42 +143,61 @@ __global__ void __launch_bounds__(THREADS, 1) gemm3x_kernel(const uint32_t *__re
         const bool vec = (r & 3) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0;
         bool alive = true;
         int it = 0;
-        for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
-            const int as = it & 1;
+        const int nch = nkb > 0 ? (nkb + KCHUNK - 1) / KCHUNK : 1;
+        for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
             const int mt = t / ntn2, nt2 = t - mt * ntn2;
-            if (alive) alive = mbar_wait(acc_full + 8 * as, ((uint32_t)(it >> 1)) & 1u, abort_flag, status);
-            alive = __all_sync(0xffffffffu, alive);
-            tc_fence_after();
             const int row = mt * TILE + warp * 32 + lane;
+            for (int ch = 0; ch < nch; ++ch, ++it) {             // a chunk's sum is added to what the chunks before it left in C
+                const int as = it & 1;
+                if (alive) alive = mbar_wait(acc_full + 8 * as, ((uint32_t)(it >> 1)) & 1u, abort_flag, status);
+                alive = __all_sync(0xffffffffu, alive);
+                tc_fence_after();
 #pragma unroll 1
-            for (int c = 0; c < 2 * TILE; c += 16) {
-                if (nt2 * 2 * TILE + c >= r) break;                  // past the last column (the same for the whole warp)
-                float y[16];
-                if (alive && nkb > 0) {
-                    uint32_t d[16];
-                    tmem_ld16(tmem + lane_base + (uint32_t)(as * 2 * TILE + c), d);
-                    tmem_ld_wait();
+                for (int c0 = 0; c0 < 2 * TILE; c0 += 64) {      // 64 columns at a time: what C holds is requested first
+                    const int col0 = nt2 * 2 * TILE + c0;
+                    if (col0 >= r) break;                        // past the last column (the same for the whole warp)
+                    float *out0 = C + (size_t)row * r + col0;
+                    const bool fast = vec && col0 + 64 <= r;
+                    float4 prev[16];
+                    if (fast && ch > 0 && row < n) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) y[e] = __uint_as_float(d[e]);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) y[e] = alive ? 0.f : __int_as_float(0x7fc00000);
-                }
-                const int col = nt2 * 2 * TILE + c;
-                if (row < n) {
-                    float *out = C + (size_t)row * r + col;
-                    if (vec && col + 16 <= r) {
-#pragma unroll
-                        for (int e = 0; e < 16; e += 4) *reinterpret_cast<float4 *>(out + e) = make_float4(y[e], y[e + 1], y[e + 2], y[e + 3]);
+                        for (int e = 0; e < 16; ++e) prev[e] = *reinterpret_cast<const float4 *>(out0 + 4 * e);
                     } else {
 #pragma unroll
-                        for (int e = 0; e < 16; ++e)
-                            if (col + e < r) out[e] = y[e];
+                        for (int e = 0; e < 16; ++e) prev[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+#pragma unroll
+                    for (int c = 0; c < 64; c += 16) {
+                        float y[16];
+                        if (alive && nkb > 0) {
+                            uint32_t d[16];
+                            tmem_ld16(tmem + lane_base + (uint32_t)(as * 2 * TILE + c0 + c), d);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) y[e] = __uint_as_float(d[e]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) y[e] = alive ? 0.f : __int_as_float(0x7fc00000);
+                        }
+                        if (row < n) {
+                            float *out = out0 + c;
+                            if (fast) {
+#pragma unroll
+                                for (int e = 0; e < 16; e += 4) {
+                                    const float4 o = prev[(c + e) >> 2];
+                                    *reinterpret_cast<float4 *>(out + e) = make_float4(y[e] + o.x, y[e + 1] + o.y, y[e + 2] + o.z, y[e + 3] + o.w);
+                                }
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 16; ++e)
+                                    if (col0 + c + e < r) out[e] = ch > 0 ? out[e] + y[e] : y[e];
+                            }
+                        }
                     }
                 }
+                tc_fence_before();
+                if (alive) mbar_arrive(acc_empty + 8 * as);       // the accumulator may be overwritten
             }
-            tc_fence_before();
-            if (alive) mbar_arrive(acc_empty + 8 * as);           // the accumulator may be overwritten
         }
     } else if (warp == 4) {
         // ====================================== loader ======================================
@@ -207,31 +233,36 @@ __global__ void __launch_bounds__(THREADS, 1) gemm3x_kernel(const uint32_t *__re
             const uint32_t idesc = idesc_tf32(2 * TILE);
             bool alive = true;
             int g = 0, it = 0;
-            for (int t = blockIdx.x; t < ntiles && alive; t += gridDim.x, ++it) {
-                const int as = it & 1;
-                alive = mbar_wait(acc_empty + 8 * as, (((uint32_t)(it >> 1)) & 1u) ^ 1u, abort_flag, status);
-                if (!alive) break;
-                tc_fence_after();
-                const uint32_t d = tmem + (uint32_t)(as * 2 * TILE);
-                for (int kb = 0; kb < nkb && alive; ++kb, ++g) {
-                    const int s = g % STAGES;
-                    alive = mbar_wait(full_bar + 8 * s, ((uint32_t)(g / STAGES)) & 1u, abort_flag, status);
+            const int nch = nkb > 0 ? (nkb + KCHUNK - 1) / KCHUNK : 1;
+            for (int t = blockIdx.x; t < ntiles && alive; t += gridDim.x) {
+                for (int ch = 0; ch < nch && alive; ++ch, ++it) {
+                    const int as = it & 1;
+                    alive = mbar_wait(acc_empty + 8 * as, (((uint32_t)(it >> 1)) & 1u) ^ 1u, abort_flag, status);
                     if (!alive) break;
                     tc_fence_after();
-                    const uint32_t stage = smem_base + (uint32_t)(s * STAGE_BYTES);
-                    const uint64_t a_hi = make_smem_desc(stage), a_lo = make_smem_desc(stage + (uint32_t)HALF);
-                    const uint64_t b_hi = make_smem_desc(stage + (uint32_t)PIECE), b_lo = make_smem_desc(stage + (uint32_t)(2 * PIECE));
+                    const uint32_t d = tmem + (uint32_t)(as * 2 * TILE);
+                    const int kb_end = min(nkb, (ch + 1) * KCHUNK);
+                    for (int kb = ch * KCHUNK; kb < kb_end && alive; ++kb, ++g) {
+                        const int s = g % STAGES;
+                        alive = mbar_wait(full_bar + 8 * s, ((uint32_t)(g / STAGES)) & 1u, abort_flag, status);
+                        if (!alive) break;
+                        tc_fence_after();
+                        const uint32_t stage = smem_base + (uint32_t)(s * STAGE_BYTES);
+                        const uint64_t a_hi = make_smem_desc(stage), a_lo = make_smem_desc(stage + (uint32_t)HALF);
+                        const uint64_t b_hi = make_smem_desc(stage + (uint32_t)PIECE), b_lo = make_smem_desc(stage + (uint32_t)(2 * PIECE));
+                        const bool fresh = kb == ch * KCHUNK;    // the chunk starts on a cleared accumulator
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)               // 8 TF32 = 32 bytes per K step
-                        umma_ss_tf32(d, a_hi + (uint64_t)(2 * ks), b_hi + (uint64_t)(2 * ks), idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+                        for (int ks = 0; ks < 4; ++ks)           // 8 TF32 = 32 bytes per K step
+                            umma_ss_tf32(d, a_hi + (uint64_t)(2 * ks), b_hi + (uint64_t)(2 * ks), idesc, (!fresh || ks > 0) ? 1u : 0u);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) umma_ss_tf32(d, a_hi + (uint64_t)(2 * ks), b_lo + (uint64_t)(2 * ks), idesc, 1u);
+                        for (int ks = 0; ks < 4; ++ks) umma_ss_tf32(d, a_hi + (uint64_t)(2 * ks), b_lo + (uint64_t)(2 * ks), idesc, 1u);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) umma_ss_tf32(d, a_lo + (uint64_t)(2 * ks), b_hi + (uint64_t)(2 * ks), idesc, 1u);
-                    umma_commit(empty_bar + 8 * s);
+                        for (int ks = 0; ks < 4; ++ks) umma_ss_tf32(d, a_lo + (uint64_t)(2 * ks), b_hi + (uint64_t)(2 * ks), idesc, 1u);
+                        umma_commit(empty_bar + 8 * s);
+                    }
+                    if (alive && nkb > 0) umma_commit(acc_full + 8 * as);
+                    else mbar_arrive(acc_full + 8 * as);
                 }
-                if (alive && nkb > 0) umma_commit(acc_full + 8 * as);
-                else mbar_arrive(acc_full + 8 * as);
             }
         }
         __syncwarp();

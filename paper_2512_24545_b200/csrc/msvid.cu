@@ -172,7 +172,7 @@ __global__ void __launch_bounds__(AQ_WARPS * 32) absz_q_kernel(const float *__re
 // ------------------------------------------------------------------ Y = |Z| Q and W = |Z|^T Y on the tensor cores
 // The two products of the subspace iteration with tcgen05 (kind::tf32, fp32 accumulators in tensor memory) and a
 // three-term split that keeps fp32 accuracy:  e = e_hi + e_lo,  q = q_hi + q_lo  (each part a TF32 number),
-//     e q  ~  e_hi q_hi + e_hi q_lo + e_lo q_hi                      (the dropped e_lo q_lo is below 2^-21 e q).
+//     e q  ~  e_hi q_hi + e_hi q_lo + e_lo q_hi                      (the dropped e_lo q_lo is below 2^-24 e q).
 // CTA = 128 output rows x a range of K blocks of 32 (split over blockIdx.y, partial sums per range).  Per K block:
 //   one lane brings the raw 128 x 32 tile of Z into a ring of buffers by TMA (zero fill outside the matrix), so the
 //     bytes in flight do not depend on how many threads wait for them;
@@ -208,11 +208,13 @@ __device__ __forceinline__ uint32_t tf32_round(float x) {
     asm("cvt.rna.tf32.f32 %0, %1;\n" : "=r"(r) : "f"(x));
     return r;
 }
-// e = hi + lo with hi the TF32 truncation of e (the residual is then exact in fp32) and lo the residual rounded to
-// nearest TF32 by an integer half-ulp add: plain ALU work (the cvt instruction runs on the quarter-rate pipe).
-// |e - hi - lo| <= 2^-22 |e|.
+// e = hi + lo with hi = e rounded to the nearest TF32 number (an integer half-ulp add on the bits, then the low 13 bits
+// cleared; values in the top binade are truncated instead so that nothing rounds up to infinity), the residual e - hi
+// exact in fp32, and lo that residual rounded the same way: plain ALU work (the cvt instruction runs on the quarter-rate
+// pipe).  |e - hi - lo| <= 2^-24 |e|.
 __device__ __forceinline__ void tf32_split(float e, uint32_t &hi, uint32_t &lo) {
-    hi = __float_as_uint(e) & 0xFFFFE000u;
+    const uint32_t b = __float_as_uint(e);
+    hi = ((b & 0x7F000000u) == 0x7F000000u ? b : b + 0x1000u) & 0xFFFFE000u;
     lo = (__float_as_uint(e - __uint_as_float(hi)) + 0x1000u) & 0xFFFFE000u;
 }
 // D[tmem] (+)= A[tmem] * B[smem], TF32 operands
