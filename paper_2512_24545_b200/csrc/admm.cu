@@ -7,7 +7,7 @@
 // W is N x M, V is M x R, U and Lam are N x R (dense values of the factor), all fp32 row-major on the device.  The
 // update of the other factor is the same call on the transposed problem (transpose_w).
 //
-// The two dense products (W V and V^T V, once per call) run on the tensor cores with fp32 accuracy (gemm3x.cu: TF32
+// The two dense products (W V and V^T V, once per call) run on the tensor cores at close to fp32 accuracy (gemm3x.cu: TF32
 // operands in a three-term split); V's operand images serve both, as the right operand of W V and as both operands of
 // V^T V.  The Cholesky factorisation of the R x R system (cuSOLVER) and one triangular solve for the factor's inverse
 // (cuBLAS) are library routines; the inverse of the system is formed and then applied, in every inner iteration, by the

@@ -1,4 +1,4 @@
-// Dense fp32 product C = A B on the tensor cores with fp32 accuracy: tcgen05 kind::tf32 and the three-term split
+// Dense fp32 product C = A B on the tensor cores at close to fp32 accuracy: tcgen05 kind::tf32 and the three-term split
 //     a b  ~  a_hi b_hi + a_hi b_lo + a_lo b_hi          (each part a TF32 number; the dropped a_lo b_lo is below 2^-24 a b)
 // with fp32 accumulation in tensor memory.  It serves the least-squares step of the ADMM refinement (W V and V^T V,
 // Eq. admm-U-tilde), where the FP32 pipe would need five times as long.

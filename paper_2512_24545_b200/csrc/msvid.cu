@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(AQ_WARPS * 32) absz_q_kernel(const float *__re
 
 // ------------------------------------------------------------------ Y = |Z| Q and W = |Z|^T Y on the tensor cores
 // The two products of the subspace iteration with tcgen05 (kind::tf32, fp32 accumulators in tensor memory) and a
-// three-term split that keeps fp32 accuracy:  e = e_hi + e_lo,  q = q_hi + q_lo  (each part a TF32 number),
+// three-term split of the fp32 operands:  e = e_hi + e_lo,  q = q_hi + q_lo  (each part a TF32 number),
 //     e q  ~  e_hi q_hi + e_hi q_lo + e_lo q_hi                      (the dropped e_lo q_lo is below 2^-24 e q).
 // CTA = 128 output rows x a range of K blocks of 32 (split over blockIdx.y, partial sums per range).  Per K block:
 //   one lane brings the raw 128 x 32 tile of Z into a ring of buffers by TMA (zero fill outside the matrix), so the
