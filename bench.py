@@ -46,8 +46,8 @@ NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     ("msvid_28672x6016_l16", "envelope_product_tc_kernel"): 708300000,   # Z once per pass (689.9 MB) + operand images and partial sums,
                                                                            # scaled by rows x cols from the 8192 x 8192 capture
     ("msvid_8192x8192_l16", "envelope_product_tc_kernel"): 275523328,      # 269.6 MB read + 5.9 MB written for 268.4 MB of Z
-    ("admm_8192x8192_r3712_l16", "gemm3x_kernel"): 1174788208,            # its largest launch, W V: 1.049 GB read (images 0.78 GB; V's are re-read
-                                                                           # by every row tile, four fifths of that from L2) + 125.4 MB written
+    ("admm_8192x8192_r3712_l16", "gemm3x_kernel"): 1156590808,            # its largest launch, W V: 1.038 GB read (images 0.78 GB; V's are re-read
+                                                                           # by every row tile, four fifths of that from L2) + 118.6 MB written
     ("block70b_T2048", "mat_stage_kernel"): 197116928,             # its largest launch, down stage B (185.9 MB read: 117 MB of x, partly twice,
                                                                    # + signs; 11.3 MB written); gate / up stage A: 123.3 MB
 }

@@ -350,8 +350,8 @@ mdbf_status_t mdbf_msvid_workspace_bytes(int64_t rows, int64_t cols, int32_t l, 
  *   workspace  device, mdbf_admm_workspace_bytes(N, M, R, l) bytes on a 256-byte boundary (three N x R matrices, the R x R
  *              system, the operand images of op(W) and V - twice their size - and mdbf_msvid's workspace)
  * The dense products (W V, V^T V, the inverse of the system and its application) run on the tensor cores (TF32
- * operands in a three-term split, fp32 accumulation in chunks of 512 contraction indices; U_tilde comes out within about
- * 1e-5 of its largest entry of the exact result); the Cholesky factorisation and the solves of the R x R system are cuSOLVER calls in
+ * operands in a three-term split, fp32 accumulation in chunks of 128 contraction indices; U_tilde comes out within a few
+ * 1e-6 of its largest entry of the exact result); the Cholesky factorisation and the solves of the R x R system are cuSOLVER calls in
  * fp32; the MSVID step, the elementwise passes and the reconstruction of the dense factor fused with the dual update
  * are this library's kernels.  Asynchronous on `stream`.  The first call on a host thread creates the solver's
  * handles and allocates the scratch the factorisation asks for (kept for later calls; a larger request synchronises

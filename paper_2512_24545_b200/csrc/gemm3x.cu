@@ -11,7 +11,7 @@
 // gemm3x_kernel: one CTA per SM walks over 128 x 256 tiles of C (two column tiles of B side by side: the stream from L2
 // into shared memory, 96 KB per K block, is what bounds the kernel, and a wider tile spends less of it per flop); one
 // lane streams the pieces of each K block into a ring by bulk copies, one lane issues  D (+)= A_hi B_hi, D += A_hi B_lo,
-// D += A_lo B_hi  (N = 256, four K steps of 8 each), the four epilogue warps read the accumulator and store.  Every wait is bounded; on expiry the status word is
+// D += A_lo B_hi  (N = 256, four K steps of 8 each), the eight epilogue warps read the accumulators and store.  Every wait is bounded; on expiry the status word is
 // set and the tiles still to be written come out as NaN.
 #include <algorithm>
 #include <cstdint>
@@ -26,9 +26,10 @@ constexpr int TILE = 128, KB = 32;
 constexpr int HALF = TILE * KB * 4;            // bytes of the hi (or lo) part of a piece
 constexpr int PIECE = 2 * HALF;                // 32 KB
 constexpr int STAGES = 2;
-constexpr int KCHUNK = 16;                     // K blocks accumulated in tensor memory before the sum moves to fp32 registers
+constexpr int KCHUNK = 4;                      // K blocks accumulated in tensor memory before the sum moves to fp32 registers
 constexpr int STAGE_BYTES = 3 * PIECE;         // A piece, then B_hi of two column tiles, then their B_lo
-constexpr int THREADS = 6 * 32;                // 4 epilogue warps, loader, issuer
+constexpr int EPI_WARPS = 8;                   // two per quarter of the TMEM lanes, each with half of the tile's columns
+constexpr int THREADS = (EPI_WARPS + 2) * 32;  // epilogue warps, loader, issuer
 constexpr size_t SMEM = 1024 + (size_t)STAGES * STAGE_BYTES;
 
 // hi = v rounded to the nearest TF32 number (half-ulp add on the bits; the top binade is truncated so that nothing rounds
@@ -99,8 +100,8 @@ __device__ __forceinline__ uint32_t idesc_tf32(int n) {
 // their pieces of A in L2).  Two accumulators of 256 tensor-memory columns alternate between tiles: the epilogue of
 // one tile runs under the products of the next.  All three terms of a tile accumulate into the same columns, for KCHUNK
 // K blocks at a time: the tensor core's accumulation is not rounded to nearest, and its one-sided error grows with the
-// number of accumulations (5e-5 of the result over 8192 contraction indices, measured); the chunks' sums are added in
-// fp32 by the epilogue, through C.  ntn is
+// number of accumulations (6e-5 of the result over 8192 contraction indices, measured); the chunks' sums are added in
+// fp32 by the epilogue, in registers.  ntn is
 // the number of 128-column tiles of B's images, ntn2 = ceil(ntn / 2) the number of tiles here; an odd last tile has no
 // second half: nothing is copied for it, the products read whatever the buffer holds, and nothing of it is stored.
 __global__ void __launch_bounds__(THREADS, 1) gemm3x_kernel(const uint32_t *__restrict__ Aimg, const uint32_t *__restrict__ Bimg,
@@ -123,12 +124,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm3x_kernel(const uint32_t *__re
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(acc_full + 8 * a, 1);                      // the issuer's commit after a tile's last K block
-            mbar_init(acc_empty + 8 * a, 128);                   // every epilogue thread, once it has read its row
+            mbar_init(acc_empty + 8 * a, EPI_WARPS * 32);        // every epilogue thread, once it has read its part
         }
         abort_flag_s = 0;
         fence_barrier_init();
     }
-    if (warp == 5) {
+    if (warp == EPI_WARPS + 1) {
         tmem_alloc(smem_u32(&tmem_base_slot), 512u);             // two accumulators of 256 columns; one CTA per SM
         tmem_relinquish();
     }
@@ -137,69 +138,54 @@ __global__ void __launch_bounds__(THREADS, 1) gemm3x_kernel(const uint32_t *__re
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
 
-    if (warp < 4) {
+    if (warp < EPI_WARPS) {
         // ===================================== epilogue =====================================
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        // thread = one row and one half (128 columns) of the tile; the chunks' sums are added in registers, in fp32
+        const int half = warp >> 2;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const bool vec = (r & 3) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0;
         bool alive = true;
         int it = 0;
         const int nch = nkb > 0 ? (nkb + KCHUNK - 1) / KCHUNK : 1;
         for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
             const int mt = t / ntn2, nt2 = t - mt * ntn2;
-            const int row = mt * TILE + warp * 32 + lane;
-            for (int ch = 0; ch < nch; ++ch, ++it) {             // a chunk's sum is added to what the chunks before it left in C
+            const int row = mt * TILE + (warp & 3) * 32 + lane;
+            const int col0 = nt2 * 2 * TILE + half * TILE;
+            float sum[TILE];
+            for (int ch = 0; ch < nch; ++ch, ++it) {
                 const int as = it & 1;
                 if (alive) alive = mbar_wait(acc_full + 8 * as, ((uint32_t)(it >> 1)) & 1u, abort_flag, status);
                 alive = __all_sync(0xffffffffu, alive);
                 tc_fence_after();
-#pragma unroll 1
-                for (int c0 = 0; c0 < 2 * TILE; c0 += 64) {      // 64 columns at a time: what C holds is requested first
-                    const int col0 = nt2 * 2 * TILE + c0;
-                    if (col0 >= r) break;                        // past the last column (the same for the whole warp)
-                    float *out0 = C + (size_t)row * r + col0;
-                    const bool fast = vec && col0 + 64 <= r;
-                    float4 prev[16];
-                    if (fast && ch > 0 && row < n) {
+                if (alive && nkb > 0) {
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) prev[e] = *reinterpret_cast<const float4 *>(out0 + 4 * e);
-                    } else {
+                    for (int j = 0; j < TILE / 16; ++j) {
+                        uint32_t d[16];
+                        tmem_ld16(tmem + lane_base + (uint32_t)(as * 2 * TILE + half * TILE + 16 * j), d);
+                        tmem_ld_wait();
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) prev[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int e = 0; e < 16; ++e) sum[16 * j + e] = ch == 0 ? __uint_as_float(d[e]) : sum[16 * j + e] + __uint_as_float(d[e]);
                     }
+                } else {
 #pragma unroll
-                    for (int c = 0; c < 64; c += 16) {
-                        float y[16];
-                        if (alive && nkb > 0) {
-                            uint32_t d[16];
-                            tmem_ld16(tmem + lane_base + (uint32_t)(as * 2 * TILE + c0 + c), d);
-                            tmem_ld_wait();
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) y[e] = __uint_as_float(d[e]);
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) y[e] = alive ? 0.f : __int_as_float(0x7fc00000);
-                        }
-                        if (row < n) {
-                            float *out = out0 + c;
-                            if (fast) {
-#pragma unroll
-                                for (int e = 0; e < 16; e += 4) {
-                                    const float4 o = prev[(c + e) >> 2];
-                                    *reinterpret_cast<float4 *>(out + e) = make_float4(y[e] + o.x, y[e + 1] + o.y, y[e + 2] + o.z, y[e + 3] + o.w);
-                                }
-                            } else {
-#pragma unroll
-                                for (int e = 0; e < 16; ++e)
-                                    if (col0 + c + e < r) out[e] = ch > 0 ? out[e] + y[e] : y[e];
-                            }
-                        }
-                    }
+                    for (int e = 0; e < TILE; ++e) sum[e] = alive ? 0.f : __int_as_float(0x7fc00000);
                 }
                 tc_fence_before();
                 if (alive) mbar_arrive(acc_empty + 8 * as);       // the accumulator may be overwritten
             }
+            if (row < n && col0 < r) {
+                float *out = C + (size_t)row * r + col0;
+                if (vec && col0 + TILE <= r) {
+#pragma unroll
+                    for (int e = 0; e < TILE; e += 4) *reinterpret_cast<float4 *>(out + e) = make_float4(sum[e], sum[e + 1], sum[e + 2], sum[e + 3]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < TILE; ++e)
+                        if (col0 + e < r) out[e] = sum[e];
+                }
+            }
         }
-    } else if (warp == 4) {
+    } else if (warp == EPI_WARPS) {
         // ====================================== loader ======================================
         if (lane == 0) {
             bool alive = true;
@@ -270,7 +256,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm3x_kernel(const uint32_t *__re
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) drain_delay();                              // let copies in flight land before the shared memory goes back
-    if (warp == 5) tmem_dealloc(tmem, 512u);
+    if (warp == EPI_WARPS + 1) tmem_dealloc(tmem, 512u);
 }
 
 }  // namespace g3x

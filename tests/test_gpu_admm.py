@@ -186,9 +186,9 @@ def test_bench_size_update_on_sampled_rows():
     rhs = W[rows].astype(np.float64) @ V64 + rho * (U[rows].astype(np.float64) - Lam[rows].astype(np.float64))
     tilde_ref = np.linalg.solve(G, rhs.T).T
     scale = np.max(np.abs(tilde_ref))
-    # 8e-6 measured; one accumulator over all 8192 contraction indices would be at 6e-5 (the tensor core's accumulation is not
+    # 3e-6 measured; one accumulator over all 8192 contraction indices would be at 6e-5 (the tensor core's accumulation is not
     # rounded to nearest), which is why the product kernel accumulates in chunks
-    assert np.max(np.abs(g["tilde"][rows] - tilde_ref)) <= 3e-5 * scale
+    assert np.max(np.abs(g["tilde"][rows] - tilde_ref)) <= 1.5e-5 * scale
     Z = tilde_ref + Lam[rows].astype(np.float64)
     Sg = orc.unpack_signs(g["S"][rows], R)
     clear = np.abs(Z) > 5e-4 * scale
