@@ -114,15 +114,28 @@ __global__ void __launch_bounds__(RC_COLS) recon_dual_kernel(const uint32_t *__r
     float v[RC_MAXL];
 #pragma unroll
     for (int t = 0; t < RC_MAXL; ++t) v[t] = t < l ? Vl[(size_t)j * l + t] : 0.f;
-    for (int i = 0; i < RC_ROWS && i0 + i < n; ++i) {
-        float e = 0.f;
+    for (int ib = 0; ib < RC_ROWS && i0 + ib < n; ib += 4) {     // four rows at a time: their loads are in flight together
+        float ut[4], lm[4];
+        uint32_t word[4];
 #pragma unroll
-        for (int t = 0; t < RC_MAXL; ++t) e = fmaf(us[i][t], v[t], e);
-        const uint32_t word = S[(size_t)(i0 + i) * nwords + (j >> 5)];
-        const float u = ((word >> (j & 31)) & 1u) ? -e : e;
-        const size_t at = (size_t)(i0 + i) * r + j;
-        U[at] = u;
-        Lam[at] += Ut[at] - u;
+        for (int u = 0; u < 4; ++u) {
+            const bool in = i0 + ib + u < n;
+            const size_t at = (size_t)(i0 + ib + u) * r + j;
+            ut[u] = in ? Ut[at] : 0.f;
+            lm[u] = in ? Lam[at] : 0.f;
+            word[u] = in ? S[(size_t)(i0 + ib + u) * nwords + (j >> 5)] : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (i0 + ib + u >= n) break;
+            float e = 0.f;
+#pragma unroll
+            for (int t = 0; t < RC_MAXL; ++t) e = fmaf(us[ib + u][t], v[t], e);
+            const float val = ((word[u] >> (j & 31)) & 1u) ? -e : e;
+            const size_t at = (size_t)(i0 + ib + u) * r + j;
+            U[at] = val;
+            Lam[at] = lm[u] + (ut[u] - val);
+        }
     }
 }
 // a failed factorisation (not expected: the system is positive definite for rho > 0) or an expired wait of the product
