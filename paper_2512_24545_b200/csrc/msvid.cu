@@ -12,9 +12,12 @@
 //     Y  <- |Z| Q;   Y^T Y = W diag(s^2) W^T        (l x l symmetric eigenproblem, Jacobi)
 //     U  <- Y W diag(s^-1/2),   V <- Q W diag(s^1/2)      balanced factors:  U V^T = Y Q^T ~ TSVD_l(|Z|)
 //
-// Two passes over Z per iteration, each a tall-skinny product on the CUDA cores (16 FMAs per 4 bytes of Z at
-// l = 16: the kernels are bound by HBM, not by arithmetic, so there is nothing for the tensor cores to win);
-// orth() is a Cholesky QR with the l x l Gram matrix accumulated and factorised in fp64.  What the iteration
+// Two passes over Z per iteration, each a tall-skinny product.  At l = 16 that is 16 FMAs per 4 bytes of Z: on the
+// CUDA cores the FP32 pipe needs as long as HBM does, so the products run on the tensor cores
+// (envelope_product_tc_kernel: TF32 operands in a three-term split, the envelope written straight into tensor
+// memory) and reach three quarters of the memory rate; the scalar kernels absz_q_kernel / abszT_y_kernel serve the
+// shapes a tensor map cannot take.  The first pass also packs the sign mask.  orth() is a Cholesky QR with the
+// l x l Gram matrix accumulated and factorised in fp64, one launch for the Gram matrix, its reduction and its factor.  What the iteration
 // leaves short of the exact TSVD is the mixing among the nearly equal singular values of the bulk: the largest
 // singular value converges in two iterations, the squared error of the envelope stays within a fraction of a
 // per cent of the optimum of Theorem 1 (the GPU tests bound it), and every Ritz value is a lower bound of the
