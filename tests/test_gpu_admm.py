@@ -83,6 +83,26 @@ def test_one_inner_iteration(N, Mc, R, l, transpose):
     assert abs(obj_g - obj_o) <= 0.01 * obj_o
 
 
+@pytest.mark.parametrize("trial", range(12))
+def test_random_ragged_shapes(trial):
+    """Sizes drawn at random, none a multiple of a tile: the products' tails (rows, columns, contraction indices, an odd number
+    of 128-column tiles), both orientations of W."""
+    rng = np.random.default_rng(900 + trial)
+    N, Mc = int(rng.integers(2, 900)), int(rng.integers(2, 900))
+    R = int(min(rng.integers(1, min(N, Mc) + 1), 600))
+    l = int(min(rng.choice([1, 2, 4, 8, 16, 32]), R, N))
+    transpose = bool(trial % 2)
+    Wop, V, U, Lam = problem(N, Mc, R, seed=500 + trial)
+    W = np.ascontiguousarray(Wop.T) if transpose else Wop
+    rho = float(np.sum(V.astype(np.float64) ** 2)) / R
+    g = run_update(W, V, U, Lam, rho, l, 1, 6, transpose)
+    _, _, tildes, _ = orc.admm_factor_update(Wop, V, U, Lam, rho, l, 1)
+    scale = np.max(np.abs(tildes[0]))
+    assert np.max(np.abs(g["tilde"] - tildes[0])) <= 2e-5 * scale
+    np.testing.assert_allclose(g["Lam"], Lam.astype(np.float64) + g["tilde"] - g["U"], atol=2e-5 * scale)
+    assert np.all(np.isfinite(g["U"])) and np.all(np.isfinite(g["sigma"]))
+
+
 def test_several_inner_iterations_follow_the_oracle():
     W, V, U, Lam = problem(400, 320, 96, seed=41)
     rho = float(np.sum(V.astype(np.float64) ** 2)) / 96
