@@ -134,6 +134,50 @@ def test_tensor_core_and_scalar_products_agree():
     assert abs(e0 - e1) <= 1e-5 * e1
 
 
+@pytest.mark.parametrize("trial", range(12))
+def test_random_shapes_both_product_paths(trial):
+    """Randomly drawn sizes with a column count that the tensor-core path accepts, each run twice: at an aligned address
+    (tensor-core products) and four bytes further on (scalar fp32 kernels).  Same mask, singular values and envelope error
+    that agree to the accuracy of the split (a few 1e-6 of the norm); every third case under a given mask."""
+    rng = np.random.default_rng(1200 + trial)
+    rows, cols = int(rng.integers(1, 1200)), 4 * int(rng.integers(1, 400))
+    l = int(min(rng.choice([1, 2, 3, 4, 7, 8, 13, 16, 20, 32]), rows, cols))
+    masked = trial % 3 == 2
+    Z = inputs.make_factor_matrix(rows, cols, seed=1000 + trial)
+    S = inputs.make_signs(rows, cols, seed=trial, stream="S_A") if masked else None
+    Qd = torch.from_numpy(inputs.make_start_block(cols, l, 2000 + trial)).cuda()
+    buf = torch.zeros(rows * cols + 1, dtype=torch.float32, device="cuda")
+    Zt = torch.from_numpy(Z).cuda().reshape(-1)
+    nwords = (cols + 31) // 32
+    nbytes = M.mdbf_msvid_workspace_bytes(rows, cols, l)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    res = []
+    for off in (0, 1):
+        buf.zero_()
+        buf[off:off + rows * cols] = Zt
+        Sd = (torch.from_numpy(orc.pack_signs(S).view(np.int32)).cuda() if masked
+              else torch.zeros((rows, nwords), dtype=torch.int32, device="cuda"))
+        Ud = torch.zeros((rows, l), dtype=torch.float32, device="cuda")
+        Vd = torch.zeros((cols, l), dtype=torch.float32, device="cuda")
+        sd = torch.zeros((l,), dtype=torch.float32, device="cuda")
+        if masked:
+            M.mdbf_project_fixed_mask(buf.data_ptr() + 4 * off, Sd.data_ptr(), rows, cols, l, 5, Qd.data_ptr(), Ud.data_ptr(), Vd.data_ptr(),
+                                      sd.data_ptr(), ws.data_ptr(), nbytes, st)
+        else:
+            M.mdbf_msvid(buf.data_ptr() + 4 * off, rows, cols, l, 5, Qd.data_ptr(), Sd.data_ptr(), Ud.data_ptr(), Vd.data_ptr(), sd.data_ptr(),
+                         ws.data_ptr(), nbytes, st)
+        torch.cuda.synchronize()
+        res.append((Sd.cpu().numpy(), sd.cpu().numpy().astype(np.float64), Ud.cpu().numpy().astype(np.float64),
+                    Vd.cpu().numpy().astype(np.float64)))
+    np.testing.assert_array_equal(res[0][0], res[1][0])
+    assert np.all(np.isfinite(res[0][1]))
+    np.testing.assert_allclose(res[0][1], res[1][1], rtol=5e-4, atol=1e-6 * res[1][1][0])
+    E = Z.astype(np.float64) * S if masked else np.abs(Z.astype(np.float64))
+    e0, e1 = np.linalg.norm(E - res[0][2] @ res[0][3].T), np.linalg.norm(E - res[1][2] @ res[1][3].T)
+    assert abs(e0 - e1) <= 2e-4 * e1 + 1e-5 * np.linalg.norm(E)
+
+
 def test_error_decreases_with_envelope_rank_and_with_iterations():
     Z = inputs.make_factor_matrix(700, 900, seed=6)
     errs_l = [envelope_error(Z, *run_msvid(Z, l, n_iter=6)[1:3]) for l in (1, 2, 4, 8, 16, 32)]
