@@ -353,8 +353,9 @@ mdbf_status_t mdbf_msvid_workspace_bytes(int64_t rows, int64_t cols, int32_t l, 
  * operands in a three-term split, fp32 accumulation in chunks of 128 contraction indices; U_tilde comes out within a few
  * 1e-6 of its largest entry of the exact result); the Cholesky factorisation and the solves of the R x R system are cuSOLVER calls in
  * fp32; the MSVID step, the elementwise passes and the reconstruction of the dense factor fused with the dual update
- * are this library's kernels.  Asynchronous on `stream`.  The first call on a host thread creates the solver's
- * handles and allocates the scratch the factorisation asks for (kept for later calls; a larger request synchronises
+ * are this library's kernels.  Asynchronous on `stream`; part of the work runs on a stream of the library's own that
+ * is forked from `stream` and joined to it by events inside the call.  The first call on a host thread creates the
+ * solver's handles, that stream and its events, and allocates the scratch the factorisation asks for (kept for later calls; a larger request synchronises
  * the stream and reallocates).  A failed factorisation (not expected for rho > 0) or an expired wait of a kernel turns
  * sigma into NaN.
  * Errors: INVALID_ARG (NULL pointer, rho <= 0, counts out of range, workspace too small or misaligned), SHAPE, ARCH, CUDA. */

@@ -35,6 +35,8 @@ struct Libs {
     float *potrf_ws = nullptr;          // the factorisation's scratch, as large as the largest request so far
     int potrf_floats = 0;
     int device = -1;
+    cudaStream_t side = nullptr;        // the R x R system is factored and inverted here while W V runs on the caller's stream
+    cudaEvent_t fork = nullptr, join = nullptr;
 };
 static thread_local Libs g_libs;
 
@@ -44,6 +46,9 @@ static mdbf_status_t get_libs(int device, cudaStream_t st, Libs **out) {
         if (L.blas) cublasDestroy(L.blas);
         if (L.solver) cusolverDnDestroy(L.solver);
         if (L.potrf_ws) cudaFree(L.potrf_ws);
+        if (L.side) cudaStreamDestroy(L.side);
+        if (L.fork) cudaEventDestroy(L.fork);
+        if (L.join) cudaEventDestroy(L.join);
         L = Libs();
         if (cublasCreate(&L.blas) != CUBLAS_STATUS_SUCCESS) { L = Libs(); set_error("cublasCreate failed"); return MDBF_ERR_CUDA; }
         if (cusolverDnCreate(&L.solver) != CUSOLVER_STATUS_SUCCESS) {
@@ -53,12 +58,22 @@ static mdbf_status_t get_libs(int device, cudaStream_t st, Libs **out) {
             return MDBF_ERR_CUDA;
         }
         cublasSetMathMode(L.blas, CUBLAS_PEDANTIC_MATH);          // plain fp32 products
+        if (cudaStreamCreateWithFlags(&L.side, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&L.fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&L.join, cudaEventDisableTiming) != cudaSuccess ||
+            cublasSetStream(L.blas, L.side) != CUBLAS_STATUS_SUCCESS || cusolverDnSetStream(L.solver, L.side) != CUSOLVER_STATUS_SUCCESS) {
+            cublasDestroy(L.blas);
+            cusolverDnDestroy(L.solver);
+            if (L.side) cudaStreamDestroy(L.side);
+            if (L.fork) cudaEventDestroy(L.fork);
+            if (L.join) cudaEventDestroy(L.join);
+            L = Libs();
+            set_error("could not create the side stream of the refinement step");
+            return MDBF_ERR_CUDA;
+        }
         L.device = device;
     }
-    if (cublasSetStream(L.blas, st) != CUBLAS_STATUS_SUCCESS || cusolverDnSetStream(L.solver, st) != CUSOLVER_STATUS_SUCCESS) {
-        set_error("could not bind the dense-algebra libraries to the stream");
-        return MDBF_ERR_CUDA;
-    }
+    (void)st;
     *out = &L;
     return MDBF_OK;
 }
@@ -66,7 +81,7 @@ static mdbf_status_t get_libs(int device, cudaStream_t st, Libs **out) {
 // the solver's scratch, as large as the largest request so far
 static mdbf_status_t grow_scratch(Libs *L, int floats, cudaStream_t st, const char *who) {
     if (floats <= L->potrf_floats) return MDBF_OK;
-    MDBF_CUDA(cudaStreamSynchronize(st));                         // the old scratch may still be in use
+    MDBF_CUDA(cudaStreamSynchronize(st));                         // the stream that uses it: the old scratch may still be in use
     if (L->potrf_ws) cudaFree(L->potrf_ws);
     L->potrf_ws = nullptr;
     L->potrf_floats = 0;
@@ -148,6 +163,7 @@ static size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 struct Scratch {
     float *B0, *T, *Z, *G;
     uint32_t *Wimg, *Vimg;      // operand images of op(W) (N row tiles, M deep) and of V^T (R row tiles, M deep)
+    uint32_t *Yimg;             // images of L^-T (R x R), formed on the side stream while W's are in use
     int *info;                  // [0], [1]: the solver's; [2]: status word of the product kernel
     char *msvid;
     size_t msvid_bytes;
@@ -164,9 +180,10 @@ static mdbf_status_t carve(Scratch *w, char *base, int64_t n, int64_t m, int64_t
     float *G = (float *)take((size_t)r * r * sizeof(float));
     uint32_t *Wimg = (uint32_t *)take(gemm3x_image_bytes(n, m));
     uint32_t *Vimg = (uint32_t *)take(gemm3x_image_bytes(r, m));
+    uint32_t *Yimg = (uint32_t *)take(gemm3x_image_bytes(r, r));
     int *info = (int *)take(4 * sizeof(int));
     char *mw = take(msv);
-    if (w) { w->B0 = B0; w->T = T; w->Z = Z; w->G = G; w->Wimg = Wimg; w->Vimg = Vimg; w->info = info; w->msvid = mw; w->msvid_bytes = msv; }
+    if (w) { w->B0 = B0; w->T = T; w->Z = Z; w->G = G; w->Wimg = Wimg; w->Vimg = Vimg; w->Yimg = Yimg; w->info = info; w->msvid = mw; w->msvid_bytes = msv; }
     *total = off;
     return MDBF_OK;
 }
@@ -233,32 +250,41 @@ extern "C" mdbf_status_t mdbf_admm_factor_update(const float *W, int64_t w_rows,
     const int ni = (int)n, mi = (int)m, ri = (int)r;
     MDBF_CUDA(cudaMemsetAsync(w.info, 0, 4 * sizeof(int), st));
     // images: op(W)[i][k] = W[i * w_cols + k], or W[k * w_cols + i] when transposed;  V^T[j][k] = V[k * r + j]
-    rc = transpose_w ? gemm3x_split(W, 1, (size_t)w_cols, ni, mi, w.Wimg, st) : gemm3x_split(W, (size_t)w_cols, 1, ni, mi, w.Wimg, st);
-    if (rc == MDBF_OK) rc = gemm3x_split(V, 1, (size_t)r, ri, mi, w.Vimg, st);
-    // B0 = op(W) V  and  G = V^T V (+ rho I below)
-    if (rc == MDBF_OK) rc = gemm3x_run(w.Wimg, w.Vimg, w.B0, ni, ri, mi, w.info + 2, st);
-    if (rc == MDBF_OK) rc = gemm3x_run(w.Vimg, w.Vimg, w.G, ri, ri, mi, w.info + 2, st);
+    rc = gemm3x_split(V, 1, (size_t)r, ri, mi, w.Vimg, st);
     if (rc) return rc;
-    admm::ridge_kernel<<<ceil_div(ri, 256), 256, 0, st>>>(w.G, ri, rho);
+    // Fork.  Side stream: G = V^T V + rho I, its Cholesky factor, L X = I by one triangular solve (X = L^-1, column-major;
+    // read row-major it is Y = L^-T), G^-1 = Y Y^T as a product of Y's images with themselves - the inverse written out,
+    // as Eq. admm-U-tilde has it, so that every inner iteration's solve is one product on the tensor cores instead of two
+    // triangular solves with N right-hand sides on the FP32 pipe.  Caller's stream meanwhile: W's images and B0 = op(W) V,
+    // on all SMs but a few that are left to the solver's small kernels.  Z is free until the loop below.
+    cudaStream_t s2 = L->side;
+    MDBF_CUDA(cudaEventRecord(L->fork, st));
+    MDBF_CUDA(cudaStreamWaitEvent(s2, L->fork, 0));
+    rc = gemm3x_run(w.Vimg, w.Vimg, w.G, ri, ri, mi, w.info + 2, s2);
+    if (rc) return rc;
+    admm::ridge_kernel<<<ceil_div(ri, 256), 256, 0, s2>>>(w.G, ri, rho);
     int lwork = 0;
     cusolverStatus_t ss = cusolverDnSpotrf_bufferSize(L->solver, CUBLAS_FILL_MODE_LOWER, ri, w.G, ri, &lwork);
     if (ss != CUSOLVER_STATUS_SUCCESS) { set_error("%s: cusolverDnSpotrf_bufferSize returned %d", who, (int)ss); return MDBF_ERR_CUDA; }
-    rc = admm::grow_scratch(L, lwork, st, who);
+    rc = admm::grow_scratch(L, lwork, s2, who);
     if (rc) return rc;
     ss = cusolverDnSpotrf(L->solver, CUBLAS_FILL_MODE_LOWER, ri, w.G, ri, L->potrf_ws, L->potrf_floats, w.info);
     if (ss != CUSOLVER_STATUS_SUCCESS) { set_error("%s: cusolverDnSpotrf returned %d", who, (int)ss); return MDBF_ERR_CUDA; }
-    // (V^T V + rho I)^-1 written out, as Eq. admm-U-tilde has it: every inner iteration's solve is then one product on
-    // the tensor cores instead of two triangular solves with N right-hand sides on the FP32 pipe.  With G = L L^T:
-    // L X = I by one triangular solve (X = L^-1, column-major; read row-major it is Y = L^-T), then G^-1 = Y Y^T, a
-    // product of Y's images with themselves.  Z and the space of W's images are free at this point.
-    admm::identity_kernel<<<dim3(ceil_div(ri, 256), ri), 256, 0, st>>>(w.Z, ri);
+    admm::identity_kernel<<<dim3(ceil_div(ri, 256), ri), 256, 0, s2>>>(w.Z, ri);
     const float one = 1.f;
     cublasStatus_t bs = cublasStrsm(L->blas, CUBLAS_SIDE_LEFT, CUBLAS_FILL_MODE_LOWER, CUBLAS_OP_N, CUBLAS_DIAG_NON_UNIT, ri, ri, &one,
                                     w.G, ri, w.Z, ri);
     if (bs != CUBLAS_STATUS_SUCCESS) { set_error("%s: cublasStrsm returned %d", who, (int)bs); return MDBF_ERR_CUDA; }
-    rc = gemm3x_split(w.Z, (size_t)r, 1, ri, ri, w.Wimg, st);
-    if (rc == MDBF_OK) rc = gemm3x_run(w.Wimg, w.Wimg, w.G, ri, ri, ri, w.info + 2, st);
-    if (rc == MDBF_OK) rc = gemm3x_split(w.G, (size_t)r, 1, ri, ri, w.Vimg, st);   // symmetric: rows serve as columns; V's images are done with
+    rc = gemm3x_split(w.Z, (size_t)r, 1, ri, ri, w.Yimg, s2);
+    if (rc == MDBF_OK) rc = gemm3x_run(w.Yimg, w.Yimg, w.G, ri, ri, ri, w.info + 2, s2);
+    if (rc) return rc;
+    MDBF_CUDA(cudaEventRecord(L->join, s2));
+    rc = transpose_w ? gemm3x_split(W, 1, (size_t)w_cols, ni, mi, w.Wimg, st) : gemm3x_split(W, (size_t)w_cols, 1, ni, mi, w.Wimg, st);
+    if (rc == MDBF_OK) rc = gemm3x_run(w.Wimg, w.Vimg, w.B0, ni, ri, mi, w.info + 2, st, 24);
+    if (rc) return rc;
+    // Join; the inverse's images go where V's were (symmetric: rows serve as columns)
+    MDBF_CUDA(cudaStreamWaitEvent(st, L->join, 0));
+    rc = gemm3x_split(w.G, (size_t)r, 1, ri, ri, w.Vimg, st);
     if (rc) return rc;
     const size_t count = (size_t)n * r;
     const int ew_grid = (int)std::min<size_t>((count + 255) / 256, 148u * 16);

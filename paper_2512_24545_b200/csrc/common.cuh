@@ -109,7 +109,8 @@ mdbf_status_t require_device(int *dev_out);
 // fp32-accurate dense product on the tensor cores (gemm3x.cu): operand images, then C = A B
 size_t gemm3x_image_bytes(int64_t rows, int64_t depth);
 mdbf_status_t gemm3x_split(const float *src, size_t stride_i, size_t stride_k, int rows, int depth, uint32_t *img, cudaStream_t st);
-mdbf_status_t gemm3x_run(const uint32_t *Aimg, const uint32_t *Bimg, float *C, int n, int r, int depth, int32_t *status, cudaStream_t st);
+mdbf_status_t gemm3x_run(const uint32_t *Aimg, const uint32_t *Bimg, float *C, int n, int r, int depth, int32_t *status, cudaStream_t st,
+                         int spare_sms = 0);
 // Every device allocation of the library goes through here: cudaMalloc, or - after mdbf_debug_fail_alloc(n) on the
 // calling thread - cudaErrorMemoryAllocation for the n-th call from now on without touching the device (the tests
 // inject allocation failures this way, on the host).

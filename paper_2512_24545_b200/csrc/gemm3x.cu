@@ -275,8 +275,10 @@ mdbf_status_t gemm3x_split(const float *src, size_t stride_i, size_t stride_k, i
     return MDBF_OK;
 }
 
-// C (n x r, row-major) = A B from the operands' images (A: n rows, B: r rows, both `depth` deep)
-mdbf_status_t gemm3x_run(const uint32_t *Aimg, const uint32_t *Bimg, float *C, int n, int r, int depth, int32_t *status, cudaStream_t st) {
+// C (n x r, row-major) = A B from the operands' images (A: n rows, B: r rows, both `depth` deep); spare_sms SMs are left
+// to kernels of another stream
+mdbf_status_t gemm3x_run(const uint32_t *Aimg, const uint32_t *Bimg, float *C, int n, int r, int depth, int32_t *status, cudaStream_t st,
+                         int spare_sms) {
     static PerDeviceOnce once;
     if (once.first()) MDBF_CUDA(cudaFuncSetAttribute(g3x::gemm3x_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g3x::SMEM));
     const int ntm = ceil_div(n, g3x::TILE), ntn = ceil_div(r, g3x::TILE);
@@ -290,7 +292,7 @@ mdbf_status_t gemm3x_run(const uint32_t *Aimg, const uint32_t *Bimg, float *C, i
         if (dev >= 0 && dev < 64) sms_of_device[dev] = sms;
     }
     const int ntn2 = ceil_div(ntn, 2), ntiles = ntm * ntn2;
-    g3x::gemm3x_kernel<<<std::min(ntiles, sms), g3x::THREADS, g3x::SMEM, st>>>(Aimg, Bimg, C, n, r, ceil_div(depth, g3x::KB), ntn, ntn2,
+    g3x::gemm3x_kernel<<<std::min(ntiles, std::max(1, sms - spare_sms)), g3x::THREADS, g3x::SMEM, st>>>(Aimg, Bimg, C, n, r, ceil_div(depth, g3x::KB), ntn, ntn2,
                                                                               ntiles, status);
     MDBF_CUDA(cudaGetLastError());
     return MDBF_OK;
